@@ -1,0 +1,115 @@
+/*
+ * path_attn.h -- C ABI of the PaTH attention library for NVIDIA B200 (sm_100a).
+ *
+ * PaTH attention (paper Sec. 2.1-2.2) is causal softmax attention whose logit
+ * between query i and key j <= i is
+ *
+ *     s_ij = scale * k_j^T ( H_{j+1} H_{j+2} ... H_i ) q_i + sum_{t=j+1..i} log f_t ,
+ *     H_t  = I - beta_t w_t w_t^T ,
+ *
+ * where the log f_t term (PaTH-FoX, paper Sec. 2.2 "Extension") is optional.
+ * The library computes it blockwise (paper Sec. 3.1-3.3): a per-chunk compact
+ * (UT transform) representation of the Householder products, boundary-adjusted
+ * queries and keys, chunk products, and a FlashAttention-style sweep with an
+ * online softmax.
+ *
+ * Conventions shared by every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller, 16-byte
+ *     aligned, contiguous row-major.  q, k, v, w, o, d_o, dq, dk, dv, dw are
+ *     [B, H, L, d] in the I/O dtype `dt`; beta, log_f, lse, dbeta, dlog_f are
+ *     [B, H, L] float32.  d is 64 or 128; L >= 1 is arbitrary.
+ *   - Inputs are read-only.  Outputs are fully overwritten.  Nothing is
+ *     allocated: scratch memory is the caller's `workspace` of at least
+ *     path_attn_workspace_bytes(...) bytes (256-byte aligned), which a call may
+ *     overwrite entirely.  Two calls may run concurrently only with distinct
+ *     workspaces.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*;
+ *     NULL is the default stream) and never synchronise it.
+ *   - Return value: PATH_OK or a negative path_status_t.  Argument errors are
+ *     detected on the host before anything is launched.  There is no CPU
+ *     fallback: an unsupported argument is an error.
+ *   - w and beta are used as given (no normalisation, no clipping).  `scale`
+ *     multiplies the bilinear term only; the gate is added after scaling.
+ *   - Device-side waits are bounded.  If one runs out, the kernel records it in
+ *     a status word at the start of the workspace and returns; read it with
+ *     path_attn_device_status after synchronising the stream.
+ */
+#ifndef PATH_ATTN_H_
+#define PATH_ATTN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* I/O dtype of q, k, v, w, o and their gradients.  Arithmetic: bf16 tensor-core
+ * products with float32 accumulation; PATH_FP32 splits each float32 operand of
+ * the logit products into two bf16 terms so that logits keep ~16 mantissa bits. */
+typedef enum { PATH_BF16 = 0, PATH_FP32 = 1 } path_dtype_t;
+
+typedef enum {
+    PATH_OK = 0,
+    PATH_ERR_NULL = -1,      /* a required pointer is NULL, or dlog_f / log_f given without the other */
+    PATH_ERR_SHAPE = -2,     /* d not in {64,128}, or B, H, L < 1, or sizes overflow */
+    PATH_ERR_DTYPE = -3,     /* unknown dtype, or dtype not supported by this entry point */
+    PATH_ERR_ALIGN = -4,     /* a pointer is not 16-byte aligned (workspace: 256-byte) */
+    PATH_ERR_WORKSPACE = -5, /* workspace_bytes too small */
+    PATH_ERR_ARCH = -6,      /* current device is not compute capability 10.x */
+    PATH_ERR_LAUNCH = -7,    /* a CUDA runtime / driver call failed (see path_attn_last_cuda_error) */
+    PATH_ERR_TIMEOUT = -8    /* reported by path_attn_device_status: a bounded device wait ran out */
+} path_status_t;
+
+/* Bytes of scratch memory path_attn_fwd (for_backward = 0) or path_attn_bwd
+ * (for_backward = 1) needs for this problem.  Returns 0 for invalid arguments. */
+size_t path_attn_workspace_bytes(int B, int H, int L, int d, path_dtype_t dt, int has_gate,
+                                 int for_backward);
+
+/*
+ * Forward (paper Sec. 3.3): o_i = sum_{j<=i} softmax_j(s_ij) v_j and
+ * lse_i = log sum_{j<=i} exp(s_ij) (natural log, scale and gate included).
+ *   q,k,v,w : [B,H,L,d] in dt          beta  : [B,H,L] float32
+ *   log_f   : [B,H,L] float32 per-step log f_t, or NULL for plain PaTH
+ *   o       : [B,H,L,d] in dt (out)    lse   : [B,H,L] float32 (out)
+ * Bitwise reproducible from run to run.
+ */
+int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, const float* beta,
+                  const float* log_f, void* o, float* lse, int B, int H, int L, int d, float scale,
+                  path_dtype_t dt, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward of the same function (the paper gives no backward; this is the chain
+ * rule through the Sec. 3.1-3.3 formulation): given d_o it returns the gradients
+ * of sum(o * d_o).
+ *   o, lse  : the forward's outputs for the same inputs
+ *   d_o     : [B,H,L,d] in dt
+ *   dq,dk,dv,dw : [B,H,L,d] in dt (out)   dbeta : [B,H,L] float32 (out)
+ *   dlog_f  : [B,H,L] float32 (out); must be NULL exactly when log_f is NULL
+ * dt must be PATH_BF16.  Uses float32 atomics: results are reproducible to
+ * rounding, not bitwise.
+ */
+int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, const float* beta,
+                  const float* log_f, const void* o, const float* lse, const void* d_o, void* dq,
+                  void* dk, void* dv, void* dw, float* dbeta, float* dlog_f, int B, int H, int L,
+                  int d, float scale, path_dtype_t dt, void* workspace, size_t workspace_bytes,
+                  void* cuda_stream);
+
+/* Reads the device status word the last call on this workspace left behind.
+ * Synchronises `cuda_stream`.  Returns PATH_OK, PATH_ERR_TIMEOUT, or
+ * PATH_ERR_LAUNCH if the copy itself failed.  If `detail` is not NULL it
+ * receives the raw status word (0 = clean; otherwise a code naming the wait). */
+int path_attn_device_status(const void* workspace, void* cuda_stream, unsigned int* detail);
+
+/* Static description of a status code. */
+const char* path_attn_strerror(int status);
+
+/* cudaError_t (as int) of the CUDA call behind the calling thread's most recent PATH_ERR_LAUNCH. */
+int path_attn_last_cuda_error(void);
+
+/* Number of kernel launches the calling thread's most recent fwd / bwd call issued. */
+int path_attn_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PATH_ATTN_H_ */

@@ -1,0 +1,148 @@
+"""Python binding of the C-ABI library: argument marshalling only.
+
+Every step of the path runs in the CUDA kernels behind ``include/path_attn.h``;
+torch is used here for device memory and the current stream.  There is no CPU
+fallback: if the shared library has not been built or the tensors are not on a
+CUDA device, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libpath_attn.so"
+_lib = None
+
+PATH_BF16, PATH_FP32 = 0, 1
+PATH_OK = 0
+EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_attn_device_status",
+           "path_attn_strerror", "path_attn_last_cuda_error", "path_attn_last_launch_count"]
+
+
+class PathAttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        lib = load()
+        msg = lib.path_attn_strerror(status).decode()
+        extra = f" (cudaError {lib.path_attn_last_cuda_error()})" if status == -7 else ""
+        super().__init__(f"{where}: {msg}{extra} [status {status}]")
+        self.status = status
+
+
+def load():
+    """Loads ``libpath_attn.so`` (built by ``paper_2505_16381_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise FileNotFoundError(
+                f"{_LIB_PATH} not found: build it with `python -m paper_2505_16381_b200.build` (there is no fallback)")
+        lib = ctypes.CDLL(str(_LIB_PATH))
+        P, I, F, Z = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        lib.path_attn_workspace_bytes.restype = Z
+        lib.path_attn_workspace_bytes.argtypes = [I, I, I, I, I, I, I]
+        lib.path_attn_fwd.restype = I
+        lib.path_attn_fwd.argtypes = [P, P, P, P, P, P, P, P, I, I, I, I, F, I, P, Z, P]
+        lib.path_attn_bwd.restype = I
+        lib.path_attn_bwd.argtypes = [P] * 15 + [I, I, I, I, F, I, P, Z, P]
+        lib.path_attn_device_status.restype = I
+        lib.path_attn_device_status.argtypes = [P, P, ctypes.POINTER(ctypes.c_uint)]
+        lib.path_attn_strerror.restype = ctypes.c_char_p
+        lib.path_attn_strerror.argtypes = [I]
+        lib.path_attn_last_cuda_error.restype = I
+        lib.path_attn_last_launch_count.restype = I
+        _lib = lib
+    return _lib
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return PATH_BF16
+    if t.dtype == torch.float32:
+        return PATH_FP32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _check(q, *others):
+    if not q.is_cuda:
+        raise RuntimeError("path_attn: tensors must live on a CUDA device (there is no CPU path)")
+    for t in others:
+        if t is not None and (t.device != q.device or not t.is_contiguous()):
+            raise RuntimeError("path_attn: all tensors must be contiguous and on the same device")
+    if q.dim() != 4 or not q.is_contiguous():
+        raise RuntimeError("path_attn: q must be a contiguous [B, H, L, d] tensor")
+
+
+def workspace_bytes(B, H, L, d, dtype=PATH_BF16, has_gate=False, for_backward=False) -> int:
+    return int(load().path_attn_workspace_bytes(B, H, L, d, dtype, int(has_gate), int(for_backward)))
+
+
+def alloc_workspace(q, has_gate=False, for_backward=False) -> torch.Tensor:
+    B, H, L, d = q.shape
+    n = workspace_bytes(B, H, L, d, _dt(q), has_gate, for_backward)
+    if n == 0:
+        raise PathAttnError(-2, "path_attn_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=q.device)
+
+
+def path_attn_fwd(q, k, v, w, beta, log_f=None, scale=1.0, workspace=None, out=None):
+    """Forward.  Returns ``(o, lse)``; asynchronous on the current stream."""
+    _check(q, k, v, w, beta, log_f)
+    lib = load()
+    B, H, L, d = q.shape
+    if workspace is None:
+        workspace = alloc_workspace(q, log_f is not None, False)
+    o = torch.empty_like(q) if out is None else out[0]
+    lse = torch.empty(B, H, L, dtype=torch.float32, device=q.device) if out is None else out[1]
+    st = torch.cuda.current_stream(q.device).cuda_stream
+    with torch.cuda.device(q.device):
+        rc = lib.path_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(beta), _ptr(log_f), _ptr(o), _ptr(lse),
+                               B, H, L, d, float(scale), _dt(q), _ptr(workspace), workspace.numel(),
+                               ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_fwd")
+    return o, lse
+
+
+def path_attn_bwd(q, k, v, w, beta, o, lse, d_o, log_f=None, scale=1.0, workspace=None, out=None):
+    """Backward.  Returns a dict dq, dk, dv, dw, dbeta (and dlog_f when gated)."""
+    _check(q, k, v, w, beta, log_f, o, lse, d_o)
+    lib = load()
+    B, H, L, d = q.shape
+    if workspace is None:
+        workspace = alloc_workspace(q, log_f is not None, True)
+    if out is None:
+        out = {n: torch.empty_like(q) for n in ("dq", "dk", "dv", "dw")}
+        out["dbeta"] = torch.empty_like(beta)
+        if log_f is not None:
+            out["dlog_f"] = torch.empty_like(log_f)
+    st = torch.cuda.current_stream(q.device).cuda_stream
+    with torch.cuda.device(q.device):
+        rc = lib.path_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(beta), _ptr(log_f), _ptr(o), _ptr(lse),
+                               _ptr(d_o), _ptr(out["dq"]), _ptr(out["dk"]), _ptr(out["dv"]), _ptr(out["dw"]),
+                               _ptr(out["dbeta"]), _ptr(out.get("dlog_f")), B, H, L, d, float(scale), _dt(q),
+                               _ptr(workspace), workspace.numel(), ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_bwd")
+    return out
+
+
+def device_status(workspace) -> int:
+    """Synchronises the current stream and returns the device status word of the last call on ``workspace``
+    (0 = clean).  Raises on a timed-out device wait."""
+    lib = load()
+    detail = ctypes.c_uint(0)
+    st = torch.cuda.current_stream(workspace.device).cuda_stream
+    with torch.cuda.device(workspace.device):
+        rc = lib.path_attn_device_status(_ptr(workspace), ctypes.c_void_p(st), ctypes.byref(detail))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, f"path_attn_device_status (word 0x{detail.value:x})")
+    return int(detail.value)
+
+
+def last_launch_count() -> int:
+    return int(load().path_attn_last_launch_count())

@@ -1,0 +1,61 @@
+// Shared declarations of the PaTH attention library's translation units.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace path {
+
+constexpr int CHUNK = 128;  // chunk size B of the blockwise algorithm == query tile == key tile
+
+// Codes written to the device status word when a bounded wait runs out.
+enum : uint32_t {
+    ST_OK = 0,
+    ST_FWD_PRODUCER = 0x101, ST_FWD_MMA = 0x102, ST_FWD_SOFTMAX = 0x103,
+    ST_DKV_PRODUCER = 0x201, ST_DKV_MMA = 0x202, ST_DKV_COMPUTE = 0x203,
+    ST_DQ_PRODUCER = 0x301, ST_DQ_MMA = 0x302, ST_DQ_COMPUTE = 0x303,
+};
+
+__host__ __device__ inline int msb32(unsigned x) {
+#ifdef __CUDA_ARCH__
+    return 31 - __clz((int)x);
+#else
+    int r = -1;
+    while (x) { ++r; x >>= 1; }
+    return r;
+#endif
+}
+// Storage slot of the level-l version of query chunk I / key chunk J.  Slot 0 holds the
+// boundary-adjusted tile itself, which is the version at the chunk's first usable level
+// (lowest set bit of I, lowest clear bit of J); higher levels live in slot == level.
+__host__ __device__ inline int lowest_set(unsigned x) {
+#ifdef __CUDA_ARCH__
+    return __ffs((int)x) - 1;
+#else
+    int r = 0;
+    if (!x) return -1;
+    while (!(x & 1u)) { ++r; x >>= 1; }
+    return r;
+#endif
+}
+__host__ __device__ inline int qslot(int level, int I) { return level == lowest_set((unsigned)I) ? 0 : level; }
+__host__ __device__ inline int kslot(int level, int J) { return level == lowest_set(~(unsigned)J) ? 0 : level; }
+
+struct FwdTensorMaps {
+    CUtensorMap q_raw, k_raw, v, qv, kv, xqn, yt;  // qv/kv also serve as the low parts' maps in split mode
+};
+
+struct FwdParams {
+    void* o;            // [S, L, HD] bf16 or f32
+    float* lse;         // [S, L]
+    const float* G;     // [S, Lp] inclusive prefix of the log gate, or nullptr
+    uint32_t* status;   // device status word
+    int S, L, Lp, N;
+    float scale;
+    int out_fp32;
+};
+
+cudaError_t launch_fa_fwd(const FwdTensorMaps& tm, const FwdParams& p, int hd, cudaStream_t st);
+
+}  // namespace path

@@ -1,0 +1,335 @@
+// C-ABI entry points of the PaTH attention library: argument validation, workspace planning, tensor-map
+// encoding and the launch sequence.  All arithmetic runs in the kernels of linear.cu / fa_fwd.cu / fa_bwd.cu.
+#include "../../include/path_attn.h"
+
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+#include "linear.cuh"
+
+namespace path {
+
+static thread_local int g_last_cuda_error = 0;
+static thread_local int g_launches = 0;
+
+#define CK(expr)                                                  \
+    do {                                                          \
+        cudaError_t e__ = (expr);                                 \
+        if (e__ != cudaSuccess) {                                 \
+            g_last_cuda_error = (int)e__;                         \
+            return PATH_ERR_LAUNCH;                               \
+        }                                                         \
+    } while (0)
+#define LAUNCH(expr) do { CK(expr); ++g_launches; } while (0)
+
+// ------------------------------------------------------------------------------------------- tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][cols] (row pitch = cols), box = [128 rows][64 cols], 128-byte swizzle.
+static bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// ------------------------------------------------------------------------------------------- workspace plan
+struct Plan {
+    int S, L, Lp, N, d, nlev, nslot, gate, bwd, ragged;
+    LevelTable lv;
+    size_t total;
+    // offsets (bytes)
+    size_t status, qp, kp, vp, wp, betap, G, Gm, Ai, Tt, U, Dy, Xq, Xk, Y, Xqn, Yt, Qv32, Kv32, Qv16, Kv16;
+};
+
+static size_t bump(size_t& cur, size_t bytes) {
+    size_t o = cur;
+    cur += (bytes + 255) & ~(size_t)255;
+    return o;
+}
+
+static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Plan& p) {
+    if (B < 1 || H < 1 || L < 1 || (d != 64 && d != 128)) return false;
+    if (dt != PATH_BF16 && dt != PATH_FP32) return false;
+    const long long S = (long long)B * H;
+    const long long Lp = ((long long)L + CHUNK - 1) / CHUNK * CHUNK;
+    if (S > (1 << 20) || Lp > (1 << 22) || S * Lp > (1LL << 31) / 16) return false;
+    memset(&p, 0, sizeof(p));
+    p.S = (int)S; p.L = L; p.Lp = (int)Lp; p.N = (int)(Lp / CHUNK); p.d = d; p.gate = gate; p.bwd = bwd;
+    p.nlev = p.N > 1 ? msb32((unsigned)(p.N - 1)) + 1 : 0;
+    p.nslot = p.nlev > 0 ? p.nlev : 1;
+    p.ragged = (L != p.Lp);
+    size_t cur = 0;
+    const size_t SLd = (size_t)S * Lp * d, SL = (size_t)S * Lp, SNBB = (size_t)S * p.N * CHUNK * CHUNK;
+    p.status = bump(cur, 256);
+    if (p.ragged) {
+        p.qp = bump(cur, SLd * 2); p.kp = bump(cur, SLd * 2); p.vp = bump(cur, SLd * 2); p.wp = bump(cur, SLd * 2);
+    }
+    p.betap = bump(cur, SL * 4);
+    if (gate) p.G = bump(cur, SL * 4);
+    p.Gm = bump(cur, SNBB * 4);
+    p.Ai = bump(cur, bwd ? SNBB * 4 : 0);
+    p.Tt = bump(cur, SNBB * 4);
+    p.U = bump(cur, SLd * 4);
+    size_t dy_elems = 0;
+    for (int l = 0; l < 20; ++l) {
+        p.lv.dy_off[l] = (long)dy_elems;
+        p.lv.dy_cnt[l] = p.N >> l;
+        if (l == 0 || l <= p.nlev - 2) dy_elems += (size_t)S * (p.N >> l) * d * d;
+    }
+    p.Dy = bump(cur, dy_elems * 4);
+    p.Xq = bump(cur, SNBB * 4);
+    p.Xk = bump(cur, SNBB * 4);
+    p.Y = bump(cur, SNBB * 4);
+    p.Xqn = bump(cur, SL * CHUNK * 2);
+    p.Yt = bump(cur, SL * CHUNK * 2);
+    p.Qv32 = bump(cur, SLd * 4 * p.nslot);
+    p.Kv32 = bump(cur, SLd * 4 * p.nslot);
+    p.Qv16 = bump(cur, SLd * 2 * p.nslot);
+    p.Kv16 = bump(cur, SLd * 2 * p.nslot);
+    p.total = cur;
+    return true;
+}
+
+template <class T>
+static T* at(void* ws, size_t off) { return reinterpret_cast<T*>((char*)ws + off); }
+
+static AffineBatch chunk_batch(const Plan& p, long a, long b, long c, long c2, long dd) {
+    // one batch entry per chunk, buffers padded: single stride per pointer
+    AffineBatch ab{};
+    ab.nb1 = 1 << 30;  // z0 = 0, z1 = z
+    ab.a1 = a; ab.b1 = b; ab.c1 = c; ab.c21 = c2; ab.d1 = dd;
+    return ab;
+}
+
+// Chunk preparation + dyadic run products + version chains (paper Sec. 3.1, 3.3).  Shared by forward and backward.
+static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const void* w, cudaStream_t st) {
+    const int d = p.d, nch = p.S * p.N;
+    const long Bd = (long)CHUNK * d, BB = (long)CHUNK * CHUNK, dd = (long)d * d;
+    float* Gm = at<float>(ws, p.Gm); float* Tt = at<float>(ws, p.Tt); float* U = at<float>(ws, p.U);
+    float* Ai = p.bwd ? at<float>(ws, p.Ai) : nullptr;
+    float* Dy = at<float>(ws, p.Dy); float* Xq = at<float>(ws, p.Xq); float* Xk = at<float>(ws, p.Xk);
+    float* Y = at<float>(ws, p.Y);
+    __nv_bfloat16* Xqn = at<__nv_bfloat16>(ws, p.Xqn); __nv_bfloat16* Yt = at<__nv_bfloat16>(ws, p.Yt);
+    float* Qv32 = at<float>(ws, p.Qv32); float* Kv32 = at<float>(ws, p.Kv32);
+    __nv_bfloat16* Qv16 = at<__nv_bfloat16>(ws, p.Qv16); __nv_bfloat16* Kv16 = at<__nv_bfloat16>(ws, p.Kv16);
+    const float* betap = at<float>(ws, p.betap);
+
+    // Gm = W W^T
+    {
+        GemmProblem g = gemm_problem(Operand{w, d, 1, 0}, Operand{w, d, 1, 0}, CHUNK, CHUNK, d);
+        g.C = Gm; g.c_f32 = 1; g.ldc = CHUNK;
+        LAUNCH(launch_gemm(g, chunk_batch(p, Bd, Bd, BB, 0, 0), nch, st));
+    }
+    LAUNCH(launch_tri_inverse(Gm, betap, Ai, Tt, nch, st));
+    // U = T~ W
+    {
+        GemmProblem g = gemm_problem(Operand{Tt, CHUNK, 1, 1}, Operand{w, 1, d, 0}, CHUNK, d, CHUNK);
+        g.C = U; g.c_f32 = 1; g.ldc = d;
+        LAUNCH(launch_gemm(g, chunk_batch(p, BB, Bd, Bd, 0, 0), nch, st));
+    }
+    // P = I - W^T U  -> Dy level 0
+    {
+        GemmProblem g = gemm_problem(Operand{w, 1, d, 0}, Operand{U, 1, d, 1}, d, d, CHUNK);
+        g.C = Dy; g.c_f32 = 1; g.ldc = d; g.alpha = -1.f; g.identity = 1;
+        LAUNCH(launch_gemm(g, chunk_batch(p, Bd, Bd, dd, 0, 0), nch, st));
+    }
+    // Xq = lower(Q W^T); Xqn = -Xq (bf16, A operand of the diagonal correction)
+    {
+        GemmProblem g = gemm_problem(Operand{q, d, 1, 0}, Operand{w, d, 1, 0}, CHUNK, CHUNK, d);
+        g.C = Xq; g.c_f32 = 1; g.ldc = CHUNK; g.mask = MASK_LOWER;
+        g.C2 = Xqn; g.ldc2 = CHUNK; g.alpha2 = -1.f;
+        LAUNCH(launch_gemm(g, chunk_batch(p, Bd, Bd, BB, BB, 0), nch, st));
+    }
+    // Qleft = Q - Xq U  -> version slot 0
+    {
+        GemmProblem g = gemm_problem(Operand{Xq, CHUNK, 1, 1}, Operand{U, 1, d, 1}, CHUNK, d, CHUNK);
+        g.C = Qv32; g.c_f32 = 1; g.ldc = d; g.alpha = -1.f;
+        g.D = q; g.d_f32 = 0; g.ldd = d;
+        g.C2 = Qv16; g.ldc2 = d;
+        LAUNCH(launch_gemm(g, chunk_batch(p, BB, Bd, Bd, Bd, Bd), nch, st));
+    }
+    // Xk = strictLower(W K^T)
+    {
+        GemmProblem g = gemm_problem(Operand{w, d, 1, 0}, Operand{k, d, 1, 0}, CHUNK, CHUNK, d);
+        g.C = Xk; g.c_f32 = 1; g.ldc = CHUNK; g.mask = MASK_STRICT;
+        LAUNCH(launch_gemm(g, chunk_batch(p, Bd, Bd, BB, 0, 0), nch, st));
+    }
+    // Y = T~ Xk; Yt = Y^T (bf16, B operand of the diagonal correction)
+    {
+        GemmProblem g = gemm_problem(Operand{Tt, CHUNK, 1, 1}, Operand{Xk, 1, CHUNK, 1}, CHUNK, CHUNK, CHUNK);
+        g.C = Y; g.c_f32 = 1; g.ldc = CHUNK;
+        g.C2 = Yt; g.ldc2 = CHUNK; g.c2_trans = 1;
+        LAUNCH(launch_gemm(g, chunk_batch(p, BB, BB, BB, BB, 0), nch, st));
+    }
+    // Kright = K - Y^T W  -> version slot 0
+    {
+        GemmProblem g = gemm_problem(Operand{Y, 1, CHUNK, 1}, Operand{w, 1, d, 0}, CHUNK, d, CHUNK);
+        g.C = Kv32; g.c_f32 = 1; g.ldc = d; g.alpha = -1.f;
+        g.D = k; g.d_f32 = 0; g.ldd = d;
+        g.C2 = Kv16; g.ldc2 = d;
+        LAUNCH(launch_gemm(g, chunk_batch(p, BB, Bd, Bd, Bd, Bd), nch, st));
+    }
+    // dyadic run products Dy[l+1][b] = Dy[l][2b+1] Dy[l][2b]
+    for (int l = 0; l + 1 <= p.nlev - 2; ++l) {
+        const int cnt = p.N >> l, cnt2 = p.N >> (l + 1);
+        const float* src = Dy + p.lv.dy_off[l];
+        GemmProblem g = gemm_problem(Operand{src + dd, d, 1, 1}, Operand{src, 1, d, 1}, d, d, d);
+        g.C = Dy + p.lv.dy_off[l + 1]; g.c_f32 = 1; g.ldc = d;
+        AffineBatch ab{};
+        ab.nb1 = cnt2;
+        ab.a0 = (long)cnt * dd; ab.a1 = 2 * dd; ab.b0 = ab.a0; ab.b1 = ab.a1;
+        ab.c0 = (long)cnt2 * dd; ab.c1 = dd;
+        LAUNCH(launch_gemm(g, ab, p.S * cnt2, st));
+    }
+    // version chains
+    for (int l2 = 1; l2 < p.nlev; ++l2) {
+        for (int is_key = 0; is_key < 2; ++is_key) {
+            VersionBatch v{};
+            v.is_key = is_key; v.mode = 0; v.l2 = l2; v.S = p.S; v.N = p.N; v.Lp = p.Lp; v.d = d; v.lv = p.lv;
+            v.xv = is_key ? Kv32 : Qv32; v.out32 = is_key ? Kv32 : Qv32; v.out16 = is_key ? Kv16 : Qv16;
+            v.dy = Dy;
+            LAUNCH(launch_gemm_version(v, st));
+        }
+    }
+    return PATH_OK;
+}
+
+static int check_arch() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PATH_ERR_LAUNCH;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return PATH_ERR_LAUNCH;
+    return major == 10 ? PATH_OK : PATH_ERR_ARCH;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+// Pads q, k, v, w (ragged L) and beta into the workspace; returns the pointers the kernels should read.
+static int stage_inputs(const Plan& p, void* ws, const void*& q, const void*& k, const void*& v, const void*& w,
+                        const float* beta, const float* log_f, cudaStream_t st) {
+    if (p.ragged) {
+        LAUNCH(launch_pad_rows(q, at<void>(ws, p.qp), p.S, p.L, p.Lp, p.d, 0, st)); q = at<void>(ws, p.qp);
+        LAUNCH(launch_pad_rows(k, at<void>(ws, p.kp), p.S, p.L, p.Lp, p.d, 0, st)); k = at<void>(ws, p.kp);
+        LAUNCH(launch_pad_rows(v, at<void>(ws, p.vp), p.S, p.L, p.Lp, p.d, 0, st)); v = at<void>(ws, p.vp);
+        LAUNCH(launch_pad_rows(w, at<void>(ws, p.wp), p.S, p.L, p.Lp, p.d, 0, st)); w = at<void>(ws, p.wp);
+    }
+    LAUNCH(launch_pad_vec(beta, at<float>(ws, p.betap), p.S, p.L, p.Lp, st));
+    if (log_f) LAUNCH(launch_gate_prefix(log_f, at<float>(ws, p.G), p.S, p.L, p.Lp, st));
+    return PATH_OK;
+}
+
+}  // namespace path
+
+using namespace path;
+
+extern "C" {
+
+size_t path_attn_workspace_bytes(int B, int H, int L, int d, path_dtype_t dt, int has_gate, int for_backward) {
+    Plan p;
+    if (!make_plan(B, H, L, d, (int)dt, has_gate ? 1 : 0, for_backward ? 1 : 0, p)) return 0;
+    return p.total;
+}
+
+int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, const float* beta, const float* log_f,
+                  void* o, float* lse, int B, int H, int L, int d, float scale, path_dtype_t dt, void* workspace,
+                  size_t workspace_bytes, void* cuda_stream) {
+    g_launches = 0;
+    if (!q || !k || !v || !w || !beta || !o || !lse || !workspace) return PATH_ERR_NULL;
+    Plan p;
+    if (dt != PATH_BF16 && dt != PATH_FP32) return PATH_ERR_DTYPE;
+    if (!make_plan(B, H, L, d, (int)dt, log_f ? 1 : 0, 0, p)) return PATH_ERR_SHAPE;
+    if (dt != PATH_BF16) return PATH_ERR_DTYPE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(w) || !aligned16(beta) || !aligned16(o) ||
+        !aligned16(lse) || (log_f && !aligned16(log_f)) || ((uintptr_t)workspace & 255))
+        return PATH_ERR_ALIGN;
+    if (workspace_bytes < p.total) return PATH_ERR_WORKSPACE;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CK(cudaMemsetAsync(workspace, 0, 256, st));
+
+    rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, st);
+    if (rc != PATH_OK) return rc;
+    rc = run_prep(p, workspace, q, k, w, st);
+    if (rc != PATH_OK) return rc;
+
+    FwdTensorMaps tm;
+    const uint64_t rows = (uint64_t)p.S * p.Lp;
+    bool ok = make_map(&tm.q_raw, q, rows, d) && make_map(&tm.k_raw, k, rows, d) && make_map(&tm.v, v, rows, d) &&
+              make_map(&tm.qv, at<void>(workspace, p.Qv16), rows * p.nslot, d) &&
+              make_map(&tm.kv, at<void>(workspace, p.Kv16), rows * p.nslot, d) &&
+              make_map(&tm.xqn, at<void>(workspace, p.Xqn), rows, CHUNK) &&
+              make_map(&tm.yt, at<void>(workspace, p.Yt), rows, CHUNK);
+    if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+    FwdParams fp{};
+    fp.o = o; fp.lse = lse; fp.G = log_f ? at<float>(workspace, p.G) : nullptr;
+    fp.status = at<uint32_t>(workspace, p.status);
+    fp.S = p.S; fp.L = L; fp.Lp = p.Lp; fp.N = p.N; fp.scale = scale; fp.out_fp32 = 0;
+    LAUNCH(launch_fa_fwd(tm, fp, d, st));
+    return PATH_OK;
+}
+
+int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, const float* beta, const float* log_f,
+                  const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
+                  float* dbeta, float* dlog_f, int B, int H, int L, int d, float scale, path_dtype_t dt,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    g_launches = 0;
+    (void)q; (void)k; (void)v; (void)w; (void)beta; (void)log_f; (void)o; (void)lse; (void)d_o; (void)dq; (void)dk;
+    (void)dv; (void)dw; (void)dbeta; (void)dlog_f; (void)B; (void)H; (void)L; (void)d; (void)scale; (void)dt;
+    (void)workspace; (void)workspace_bytes; (void)cuda_stream;
+    return PATH_ERR_DTYPE;
+}
+
+int path_attn_device_status(const void* workspace, void* cuda_stream, unsigned int* detail) {
+    if (!workspace) return PATH_ERR_NULL;
+    unsigned int word = 0;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        g_last_cuda_error = (int)cudaGetLastError();
+        return PATH_ERR_LAUNCH;
+    }
+    if (detail) *detail = word;
+    return word == 0 ? PATH_OK : PATH_ERR_TIMEOUT;
+}
+
+const char* path_attn_strerror(int status) {
+    switch (status) {
+        case PATH_OK: return "ok";
+        case PATH_ERR_NULL: return "a required pointer is NULL (or log_f / dlog_f not given together)";
+        case PATH_ERR_SHAPE: return "unsupported shape (d must be 64 or 128; B, H, L >= 1)";
+        case PATH_ERR_DTYPE: return "unsupported dtype for this entry point";
+        case PATH_ERR_ALIGN: return "pointer not 16-byte aligned (workspace: 256-byte)";
+        case PATH_ERR_WORKSPACE: return "workspace too small";
+        case PATH_ERR_ARCH: return "device is not compute capability 10.x";
+        case PATH_ERR_LAUNCH: return "a CUDA call failed";
+        case PATH_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown status";
+    }
+}
+
+int path_attn_last_cuda_error(void) { return g_last_cuda_error; }
+int path_attn_last_launch_count(void) { return g_launches; }
+
+}  // extern "C"
