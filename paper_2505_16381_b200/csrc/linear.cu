@@ -320,7 +320,105 @@ __global__ void __launch_bounds__(1024) gate_prefix_kernel(const float* __restri
     }
 }
 
+// dbeta term 1 and the column scaling of dT (per chunk, 128 threads = columns):
+//   t1[c] = sum_r Ainv[r][c] dT[r][c];   dT[r][c] *= beta[c]   (in place: dT becomes dT D)
+__global__ void __launch_bounds__(128) beta_cols_kernel(const float* __restrict__ Ainv, float* __restrict__ dT,
+                                                        const float* __restrict__ beta, float* __restrict__ t1) {
+    const size_t base = (size_t)blockIdx.x * CHUNK * CHUNK;
+    const int c = threadIdx.x;
+    const float b = beta[(size_t)blockIdx.x * CHUNK + c];
+    float acc = 0.f;
+    for (int r = 0; r < CHUNK; ++r) {
+        const float t = dT[base + r * CHUNK + c];
+        acc += Ainv[base + r * CHUNK + c] * t;
+        dT[base + r * CHUNK + c] = t * b;
+    }
+    t1[(size_t)blockIdx.x * CHUNK + c] = acc;
+}
+
+// dbeta term 2 and the row scaling of dA (per chunk, one warp per row):
+//   dbeta[r] = t1[r] + sum_c dA[r][c] Gm[r][c];   dA[r][c] *= beta[r]   (in place: dA becomes dGm)
+__global__ void __launch_bounds__(256) beta_rows_kernel(float* __restrict__ dA, const float* __restrict__ Gm,
+                                                        const float* __restrict__ beta, const float* __restrict__ t1,
+                                                        float* __restrict__ dbeta, int N, int L) {
+    const size_t base = (size_t)blockIdx.x * CHUNK * CHUNK;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int s = blockIdx.x / N, ch = blockIdx.x % N;
+    for (int r = warp; r < CHUNK; r += 8) {
+        const float b = beta[(size_t)blockIdx.x * CHUNK + r];
+        float acc = 0.f;
+        for (int c = lane; c < CHUNK; c += 32) {
+            const float a = dA[base + r * CHUNK + c];
+            acc += a * Gm[base + r * CHUNK + c];
+            dA[base + r * CHUNK + c] = a * b;
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        const int pos = ch * CHUNK + r;
+        if (lane == 0 && pos < L) dbeta[(size_t)s * L + pos] = acc + t1[(size_t)blockIdx.x * CHUNK + r];
+    }
+}
+
+// rs[chunk*128 + i] = sum_k dsd[chunk][i][k]; one warp per row.
+__global__ void __launch_bounds__(256) dsd_rowsum_kernel(const float* __restrict__ dsd, float* __restrict__ rs) {
+    const size_t base = (size_t)blockIdx.x * CHUNK * CHUNK;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int r = warp; r < CHUNK; r += 8) {
+        float acc = 0.f;
+        for (int c = lane; c < CHUNK; c += 32) acc += dsd[base + r * CHUNK + c];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (lane == 0) rs[(size_t)blockIdx.x * CHUNK + r] = acc;
+    }
+}
+
+// dlog_f[t] = sum_{m >= t} (dGa + dGb + dGc)[m]: reverse inclusive scan per slice (inputs [S][Lp], output [S][L]).
+__global__ void __launch_bounds__(1024) gate_suffix_kernel(const float* __restrict__ dGa, const float* __restrict__ dGb,
+                                                           const float* __restrict__ dGc, float* __restrict__ out, int L,
+                                                           int Lp) {
+    __shared__ float part[1024];
+    const int tid = threadIdx.x;
+    const int seg = (L + 1023) / 1024;
+    const int hi = L - tid * seg, lo = max(hi - seg, 0);  // this thread owns positions [lo, hi), scanning downwards
+    const size_t so = (size_t)blockIdx.x * Lp;
+    float* os = out + (size_t)blockIdx.x * L;
+    float acc = 0.f;
+    for (int i = hi - 1; i >= lo; --i) acc += (dGa[so + i] + dGb[so + i]) + dGc[so + i];
+    part[tid] = acc;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+        float v = (tid >= off) ? part[tid - off] : 0.f;
+        __syncthreads();
+        part[tid] += v;
+        __syncthreads();
+    }
+    acc = (tid > 0) ? part[tid - 1] : 0.f;
+    for (int i = hi - 1; i >= lo; --i) {
+        acc += (dGa[so + i] + dGb[so + i]) + dGc[so + i];
+        os[i] = acc;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_beta_cols(const float* Ainv, float* dT, const float* beta, float* t1, int nchunks, cudaStream_t st) {
+    beta_cols_kernel<<<nchunks, 128, 0, st>>>(Ainv, dT, beta, t1);
+    return cudaGetLastError();
+}
+cudaError_t launch_beta_rows(float* dA, const float* Gm, const float* beta, const float* t1, float* dbeta, int S, int N,
+                             int L, cudaStream_t st) {
+    beta_rows_kernel<<<S * N, 256, 0, st>>>(dA, Gm, beta, t1, dbeta, N, L);
+    return cudaGetLastError();
+}
+cudaError_t launch_gate_suffix(const float* dGa, const float* dGb, const float* dGc, float* out, int S, int L, int Lp,
+                               cudaStream_t st) {
+    gate_suffix_kernel<<<S, 1024, 0, st>>>(dGa, dGb, dGc, out, L, Lp);
+    return cudaGetLastError();
+}
+cudaError_t launch_dsd_rowsum(const float* dsd, float* rs, int nchunks, cudaStream_t st) {
+    dsd_rowsum_kernel<<<nchunks, 256, 0, st>>>(dsd, rs);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_gemm(const GemmProblem& g, const AffineBatch& b, int nbatch, cudaStream_t st) {
     if (nbatch <= 0) return cudaSuccess;

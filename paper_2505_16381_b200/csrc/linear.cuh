@@ -77,4 +77,14 @@ cudaError_t launch_pad_vec(const float* src, float* dst, int S, int L, int Lp, c
 // G[S][Lp] <- inclusive prefix sum of g[S][L] (tail repeats the last value).
 cudaError_t launch_gate_prefix(const float* g, float* G, int S, int L, int Lp, cudaStream_t st);
 
+// Pieces of the UT-transform chain rule that are not matrix products (see path_attn.cu, chunk chain rule).
+cudaError_t launch_beta_cols(const float* Ainv, float* dT, const float* beta, float* t1, int nchunks, cudaStream_t st);
+cudaError_t launch_beta_rows(float* dA, const float* Gm, const float* beta, const float* t1, float* dbeta, int S, int N,
+                             int L, cudaStream_t st);
+// out[S][L] <- reverse inclusive prefix sum of (dGa + dGb + dGc)[S][Lp] over positions < L.
+cudaError_t launch_gate_suffix(const float* dGa, const float* dGb, const float* dGc, float* out, int S, int L, int Lp,
+                               cudaStream_t st);
+// rs[chunk][i] = sum_k dsd[chunk][i][k]
+cudaError_t launch_dsd_rowsum(const float* dsd, float* rs, int nchunks, cudaStream_t st);
+
 }  // namespace path

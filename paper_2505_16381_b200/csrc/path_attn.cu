@@ -60,6 +60,9 @@ struct Plan {
     size_t total;
     // offsets (bytes)
     size_t status, qp, kp, vp, wp, betap, G, Gm, Ai, Tt, U, Dy, Xq, Xk, Y, Xqn, Yt, Qv32, Kv32, Qv16, Kv16;
+    // backward only
+    size_t dop, delta, lse2, dQv, dKv, dSd, dG, dGrow, dGdiag, dDy, dXq, dY, dT, dXk, tmpBB, dA, dU, tq, tk, tw, t1;
+    size_t dy_bytes;
 };
 
 static size_t bump(size_t& cur, size_t bytes) {
@@ -107,6 +110,19 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
     p.Kv32 = bump(cur, SLd * 4 * p.nslot);
     p.Qv16 = bump(cur, SLd * 2 * p.nslot);
     p.Kv16 = bump(cur, SLd * 2 * p.nslot);
+    p.dy_bytes = dy_elems * 4;
+    if (bwd) {
+        if (p.ragged) p.dop = bump(cur, SLd * 2);
+        p.delta = bump(cur, SL * 4); p.lse2 = bump(cur, SL * 4);
+        p.dQv = bump(cur, SLd * 4 * p.nslot); p.dKv = bump(cur, SLd * 4 * p.nslot);
+        p.dSd = bump(cur, SNBB * 4); p.dG = bump(cur, SL * 4);
+        p.dGrow = bump(cur, gate ? SL * 4 : 0); p.dGdiag = bump(cur, gate ? SL * 4 : 0);
+        p.dDy = bump(cur, dy_elems * 4);
+        p.dXq = bump(cur, SNBB * 4); p.dY = bump(cur, SNBB * 4); p.dT = bump(cur, SNBB * 4);
+        p.dXk = bump(cur, SNBB * 4); p.tmpBB = bump(cur, SNBB * 4); p.dA = bump(cur, SNBB * 4);
+        p.dU = bump(cur, SLd * 4); p.tq = bump(cur, SLd * 4); p.tk = bump(cur, SLd * 4); p.tw = bump(cur, SLd * 4);
+        p.t1 = bump(cur, SL * 4);
+    }
     p.total = cur;
     return true;
 }
@@ -241,6 +257,172 @@ static int stage_inputs(const Plan& p, void* ws, const void*& q, const void*& k,
 
 }  // namespace path
 
+namespace path {
+
+// Per-chunk chain rule through the UT transform and the boundary-adjusted tiles (no counterpart in the paper):
+// from dQleft, dKright, dSd (diagonal logits), dP (chunk product) back to dq, dk, dw, dbeta.
+static int run_chunk_chain(const Plan& p, void* ws, const void* q, const void* k, const void* w, void* dq, void* dk,
+                           void* dw, float* dbeta, float scale, cudaStream_t st) {
+    const int d = p.d, nch = p.S * p.N;
+    const long Bd = (long)CHUNK * d, BB = (long)CHUNK * CHUNK, dd = (long)d * d;
+    float* Gm = at<float>(ws, p.Gm); float* Tt = at<float>(ws, p.Tt); float* U = at<float>(ws, p.U);
+    float* Ai = at<float>(ws, p.Ai); float* Xq = at<float>(ws, p.Xq); float* Xk = at<float>(ws, p.Xk);
+    float* Y = at<float>(ws, p.Y);
+    float* dQl = at<float>(ws, p.dQv); float* dKr = at<float>(ws, p.dKv);  // slot 0 of the version gradients
+    float* dSd = at<float>(ws, p.dSd); float* dP = at<float>(ws, p.dDy);  // level 0 of the run-product gradients
+    float* dXq = at<float>(ws, p.dXq); float* dY = at<float>(ws, p.dY); float* dT = at<float>(ws, p.dT);
+    float* dXk = at<float>(ws, p.dXk); float* tmp = at<float>(ws, p.tmpBB); float* dA = at<float>(ws, p.dA);
+    float* dU = at<float>(ws, p.dU); float* tq = at<float>(ws, p.tq); float* tk = at<float>(ws, p.tk);
+    float* tw = at<float>(ws, p.tw); float* t1 = at<float>(ws, p.t1);
+    const float* betap = at<float>(ws, p.betap);
+
+    // operand shorthands: R = row-major as stored, T = transposed view
+    auto R = [](const void* ptr, long ld, int f32) { return Operand{ptr, ld, 1, f32}; };   // A(m,k) = X[m][k]
+    auto Tr = [](const void* ptr, long ld, int f32) { return Operand{ptr, 1, ld, f32}; };  // A(m,k) = X[k][m]
+    // for the B operand B(k,n): Tr(X) means B(k,n) = X[k][n] (s_mn = 1, s_k = ld); R(X) means B(k,n) = X[n][k]
+    auto run = [&](Operand A, long sa, Operand B, long sb, int M, int N, int K, float* C, long sc, float alpha, int mask,
+                   int acc, const float* D = nullptr, long sd = 0, void* C2 = nullptr) -> int {
+        GemmProblem g = gemm_problem(A, B, M, N, K);
+        g.C = C; g.c_f32 = 1; g.ldc = N; g.alpha = alpha; g.mask = mask; g.accumulate = acc;
+        if (D) { g.D = D; g.d_f32 = 1; g.ldd = N; }
+        AffineBatch ab{};
+        if (C2) {
+            g.C2 = C2; g.ldc2 = N;
+            ab.nb1 = p.N; ab.rows_total = p.L;
+            ab.a0 = sa * p.N; ab.a1 = sa; ab.b0 = sb * p.N; ab.b1 = sb; ab.c0 = sc * p.N; ab.c1 = sc;
+            ab.d0 = sd * p.N; ab.d1 = sd; ab.c20 = (long)p.L * d; ab.c21 = Bd;
+        } else {
+            ab = chunk_batch(p, sa, sb, sc, 0, sd);
+        }
+        LAUNCH(launch_gemm(g, ab, nch, st));
+        return PATH_OK;
+    };
+#define RUN(...) do { int rc__ = run(__VA_ARGS__); if (rc__ != PATH_OK) return rc__; } while (0)
+    const int B = CHUNK;
+    // dSd below is the unscaled lower(dS) of the diagonal chunk; `scale` enters through the alphas.
+    // dXq = lower(-dQl U^T - scale dSd Y^T)
+    RUN(R(dQl, d, 1), Bd, R(U, d, 1), Bd, B, B, d, dXq, BB, -1.f, MASK_LOWER, ACC_NONE);
+    RUN(R(dSd, B, 1), BB, R(Y, B, 1), BB, B, B, B, dXq, BB, -scale, MASK_LOWER, ACC_ADD);
+    // dU = -Xq^T dQl - W dP
+    RUN(Tr(Xq, B, 1), BB, Tr(dQl, d, 1), Bd, B, d, B, dU, Bd, -1.f, MASK_NONE, ACC_NONE);
+    RUN(R(w, d, 0), Bd, Tr(dP, d, 1), dd, B, d, d, dU, Bd, -1.f, MASK_NONE, ACC_ADD);
+    // dY = -W dKr^T - Xq^T dSd
+    RUN(R(w, d, 0), Bd, R(dKr, d, 1), Bd, B, B, d, dY, BB, -1.f, MASK_NONE, ACC_NONE);
+    RUN(Tr(Xq, B, 1), BB, Tr(dSd, B, 1), BB, B, B, B, dY, BB, -scale, MASK_NONE, ACC_ADD);
+    // dT = lower(dY Xk^T + dU W^T)
+    RUN(R(dY, B, 1), BB, R(Xk, B, 1), BB, B, B, B, dT, BB, 1.f, MASK_LOWER, ACC_NONE);
+    RUN(R(dU, d, 1), Bd, R(w, d, 0), Bd, B, B, d, dT, BB, 1.f, MASK_LOWER, ACC_ADD);
+    // dXk = strictLower(T~^T dY)
+    RUN(Tr(Tt, B, 1), BB, Tr(dY, B, 1), BB, B, B, B, dXk, BB, 1.f, MASK_STRICT, ACC_NONE);
+    // dbeta (first term) and dT <- dT D;  dA = strictLower(-Ainv^T (dT D) Ainv^T)
+    LAUNCH(launch_beta_cols(Ai, dT, betap, t1, nch, st));
+    RUN(Tr(Ai, B, 1), BB, Tr(dT, B, 1), BB, B, B, B, tmp, BB, 1.f, MASK_NONE, ACC_NONE);
+    RUN(R(tmp, B, 1), BB, R(Ai, B, 1), BB, B, B, B, dA, BB, -1.f, MASK_STRICT, ACC_NONE);
+    // dbeta (second term, final) and dA <- D dA = dGm
+    LAUNCH(launch_beta_rows(dA, Gm, betap, t1, dbeta, p.S, p.N, p.L, st));
+    // dq = dQl + dSd K + dXq W
+    RUN(R(dSd, B, 1), BB, Tr(k, d, 0), Bd, B, d, B, tq, Bd, scale, MASK_NONE, ACC_NONE, dQl, Bd);
+    RUN(R(dXq, B, 1), BB, Tr(w, d, 0), Bd, B, d, B, tq, Bd, 1.f, MASK_NONE, ACC_ADD, nullptr, 0, dq);
+    // dk = dKr + dSd^T Q + dXk^T W
+    RUN(Tr(dSd, B, 1), BB, Tr(q, d, 0), Bd, B, d, B, tk, Bd, scale, MASK_NONE, ACC_NONE, dKr, Bd);
+    RUN(Tr(dXk, B, 1), BB, Tr(w, d, 0), Bd, B, d, B, tk, Bd, 1.f, MASK_NONE, ACC_ADD, nullptr, 0, dk);
+    // dw = -Y dKr - U dP^T + T~^T dU + dXq^T Q + dXk K + dGm W + dGm^T W
+    RUN(R(Y, B, 1), BB, Tr(dKr, d, 1), Bd, B, d, B, tw, Bd, -1.f, MASK_NONE, ACC_NONE);
+    RUN(R(U, d, 1), Bd, R(dP, d, 1), dd, B, d, d, tw, Bd, -1.f, MASK_NONE, ACC_ADD);
+    RUN(Tr(Tt, B, 1), BB, Tr(dU, d, 1), Bd, B, d, B, tw, Bd, 1.f, MASK_NONE, ACC_ADD);
+    RUN(Tr(dXq, B, 1), BB, Tr(q, d, 0), Bd, B, d, B, tw, Bd, 1.f, MASK_NONE, ACC_ADD);
+    RUN(R(dXk, B, 1), BB, Tr(k, d, 0), Bd, B, d, B, tw, Bd, 1.f, MASK_NONE, ACC_ADD);
+    RUN(R(dA, B, 1), BB, Tr(w, d, 0), Bd, B, d, B, tw, Bd, 1.f, MASK_NONE, ACC_ADD);
+    RUN(Tr(dA, B, 1), BB, Tr(w, d, 0), Bd, B, d, B, tw, Bd, 1.f, MASK_NONE, ACC_ADD, nullptr, 0, dw);
+#undef RUN
+    return PATH_OK;
+}
+
+static int run_backward(const Plan& p, void* ws, const void* q, const void* k, const void* v, const void* w,
+                        const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
+                        float* dbeta, float* dlog_f, float scale, cudaStream_t st) {
+    const int d = p.d;
+    const long dd = (long)d * d;
+    const size_t SLd = (size_t)p.S * p.Lp * d;
+    float* Dy = at<float>(ws, p.Dy); float* dDy = at<float>(ws, p.dDy);
+    float* dQv = at<float>(ws, p.dQv); float* dKv = at<float>(ws, p.dKv);
+
+    LAUNCH(launch_rowstats(o, d_o, lse, at<float>(ws, p.delta), at<float>(ws, p.lse2), p.S, p.L, p.Lp, d, st));
+    const void* dop = d_o;
+    if (p.ragged) {
+        LAUNCH(launch_pad_rows(d_o, at<void>(ws, p.dop), p.S, p.L, p.Lp, d, 0, st));
+        dop = at<void>(ws, p.dop);
+    }
+    CK(cudaMemsetAsync(dQv, 0, SLd * 4 * p.nslot, st));
+    CK(cudaMemsetAsync(dKv, 0, SLd * 4 * p.nslot, st));
+    CK(cudaMemsetAsync(dDy, 0, p.dy_bytes, st));
+    if (p.gate) CK(cudaMemsetAsync(at<float>(ws, p.dGrow), 0, (size_t)p.S * p.Lp * 4, st));
+
+    BwdTensorMaps tm;
+    const uint64_t rows = (uint64_t)p.S * p.Lp;
+    bool ok = make_map(&tm.q_raw, q, rows, d) && make_map(&tm.k_raw, k, rows, d) && make_map(&tm.v, v, rows, d) &&
+              make_map(&tm.qv, at<void>(ws, p.Qv16), rows * p.nslot, d) &&
+              make_map(&tm.kv, at<void>(ws, p.Kv16), rows * p.nslot, d) &&
+              make_map(&tm.xqn, at<void>(ws, p.Xqn), rows, CHUNK) && make_map(&tm.yt, at<void>(ws, p.Yt), rows, CHUNK) &&
+              make_map(&tm.d_o, dop, rows, d);
+    if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+    BwdParams bp{};
+    bp.dqv = dQv; bp.dkv = dKv; bp.dv = dv; bp.dsd = at<float>(ws, p.dSd); bp.dG = at<float>(ws, p.dG); bp.dGrow = at<float>(ws, p.dGrow);
+    bp.lse2 = at<float>(ws, p.lse2); bp.delta = at<float>(ws, p.delta);
+    bp.G = p.gate ? at<float>(ws, p.G) : nullptr;
+    bp.status = at<uint32_t>(ws, p.status);
+    bp.S = p.S; bp.L = p.L; bp.Lp = p.Lp; bp.N = p.N; bp.scale = scale;
+    CK(launch_fa_bwd(tm, bp, d, st));
+    g_launches += 2;
+
+    // version chains, top level first: gradients of the run products, then of the lower versions
+    for (int l2 = p.nlev - 1; l2 >= 1; --l2)
+        for (int is_key = 0; is_key < 2; ++is_key)
+            for (int mode = 2; mode >= 1; --mode) {
+                VersionBatch vb{};
+                vb.is_key = is_key; vb.mode = mode; vb.l2 = l2; vb.S = p.S; vb.N = p.N; vb.Lp = p.Lp; vb.d = d;
+                vb.lv = p.lv;
+                vb.xv = is_key ? at<float>(ws, p.Kv32) : at<float>(ws, p.Qv32);
+                vb.dxv = is_key ? dKv : dQv;
+                vb.dy = Dy; vb.ddy = dDy;
+                LAUNCH(launch_gemm_version(vb, st));
+            }
+    // run products, top-down: Dy[l][b] = Dy[l-1][2b+1] Dy[l-1][2b]
+    for (int l = p.nlev - 2; l >= 1; --l) {
+        const int cnt = p.N >> l, cntl = p.N >> (l - 1);
+        const float* lo = Dy + p.lv.dy_off[l - 1];
+        float* dlo = dDy + p.lv.dy_off[l - 1];
+        const float* dup = dDy + p.lv.dy_off[l];
+        AffineBatch ab{};
+        ab.nb1 = cnt;
+        ab.a0 = (long)cnt * dd; ab.a1 = dd;
+        ab.b0 = (long)cntl * dd; ab.b1 = 2 * dd;
+        ab.c0 = (long)cntl * dd; ab.c1 = 2 * dd;
+        {   // d(left factor, index 2b+1) += dUp * (right factor)^T
+            GemmProblem g = gemm_problem(Operand{dup, d, 1, 1}, Operand{lo, d, 1, 1}, d, d, d);
+            g.C = dlo + dd; g.c_f32 = 1; g.ldc = d; g.accumulate = ACC_ADD;
+            LAUNCH(launch_gemm(g, ab, p.S * cnt, st));
+        }
+        {   // d(right factor, index 2b) += (left factor)^T * dUp
+            AffineBatch ab2 = ab;
+            ab2.a0 = ab.b0; ab2.a1 = ab.b1; ab2.b0 = ab.a0; ab2.b1 = ab.a1;
+            GemmProblem g = gemm_problem(Operand{lo + dd, 1, d, 1}, Operand{dup, 1, d, 1}, d, d, d);
+            g.C = dlo; g.c_f32 = 1; g.ldc = d; g.accumulate = ACC_ADD;
+            LAUNCH(launch_gemm(g, ab2, p.S * cnt, st));
+        }
+    }
+    int rc = run_chunk_chain(p, ws, q, k, w, dq, dk, dw, dbeta, scale, st);
+    if (rc != PATH_OK) return rc;
+    if (dlog_f) {
+        LAUNCH(launch_dsd_rowsum(at<float>(ws, p.dSd), at<float>(ws, p.dGdiag), p.S * p.N, st));
+        LAUNCH(launch_gate_suffix(at<float>(ws, p.dG), at<float>(ws, p.dGrow), at<float>(ws, p.dGdiag), dlog_f, p.S, p.L,
+                                  p.Lp, st));
+    }
+    return PATH_OK;
+}
+
+}  // namespace path
+
 using namespace path;
 
 extern "C" {
@@ -295,10 +477,27 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
                   float* dbeta, float* dlog_f, int B, int H, int L, int d, float scale, path_dtype_t dt,
                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
     g_launches = 0;
-    (void)q; (void)k; (void)v; (void)w; (void)beta; (void)log_f; (void)o; (void)lse; (void)d_o; (void)dq; (void)dk;
-    (void)dv; (void)dw; (void)dbeta; (void)dlog_f; (void)B; (void)H; (void)L; (void)d; (void)scale; (void)dt;
-    (void)workspace; (void)workspace_bytes; (void)cuda_stream;
-    return PATH_ERR_DTYPE;
+    if (!q || !k || !v || !w || !beta || !o || !lse || !d_o || !dq || !dk || !dv || !dw || !dbeta || !workspace)
+        return PATH_ERR_NULL;
+    if ((log_f == nullptr) != (dlog_f == nullptr)) return PATH_ERR_NULL;
+    if (dt != PATH_BF16 && dt != PATH_FP32) return PATH_ERR_DTYPE;
+    Plan p;
+    if (!make_plan(B, H, L, d, (int)dt, log_f ? 1 : 0, 1, p)) return PATH_ERR_SHAPE;
+    if (dt != PATH_BF16) return PATH_ERR_DTYPE;
+    const void* ptrs[] = {q, k, v, w, beta, log_f, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f};
+    for (const void* x : ptrs)
+        if (x && !aligned16(x)) return PATH_ERR_ALIGN;
+    if ((uintptr_t)workspace & 255) return PATH_ERR_ALIGN;
+    if (workspace_bytes < p.total) return PATH_ERR_WORKSPACE;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CK(cudaMemsetAsync(workspace, 0, 256, st));
+    rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, st);
+    if (rc != PATH_OK) return rc;
+    rc = run_prep(p, workspace, q, k, w, st);
+    if (rc != PATH_OK) return rc;
+    return run_backward(p, workspace, q, k, v, w, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, scale, st);
 }
 
 int path_attn_device_status(const void* workspace, void* cuda_stream, unsigned int* detail) {
