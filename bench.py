@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the PaTH attention hot path (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload C3]
+
+One step = one pass of the whole hot path over one batch of seeded synthetic input:
+path_attn_fwd followed by path_attn_bwd on the headline workload (B=4, H=16, L=4096,
+d=128, bf16).  Rank 0 prints ONE JSON line.  With N > 1 (launched by torchrun) every
+rank runs its own batch of the same shape (the (batch, head) slices are independent:
+no data-path collective), times are reduced with max over ranks, and `value` is the
+aggregate of all ranks ("weak" scaling).
+
+FLOP models (both reported; neither counts masked-out work):
+  M1  attention-equivalent: forward 2*B*H*L*(L+1)*d, backward 2.5x forward.  `value` uses M1.
+  M2  M1 + the Householder work the method executes at chunk size 128 (chunk preparation,
+      run products, version chains, diagonal corrections and their chain rules), each
+      contraction counted once (no split-precision or recomputation multipliers).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2505_16381_b200 import synth  # noqa: E402
+
+CHUNK = 128
+METRIC = "PaTH attn fwd+bwd TFLOP/s (attention-equivalent FLOPs) at L=4096, d=128"
+UNIT = "TFLOP/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the kernel named by `roofline.kernel`,
+# from the ncu capture summarised under profiles/ (None until one exists for that kernel).
+NCU_TRAFFIC_BYTES = {}
+
+
+# ----------------------------------------------------------------------------------------- FLOP models
+def flops_m1(B, H, L, d):
+    fwd = 2.0 * B * H * L * (L + 1) * d
+    return fwd, 2.5 * fwd
+
+
+def _version_steps(N):
+    """(query-side, key-side) number of (chunk, level) version-chain products of one slice."""
+    nlev = (N - 1).bit_length() if N > 1 else 0
+    nq = nk = 0
+    for l2 in range(1, nlev):
+        for c in range(N):
+            low = c & ((1 << l2) - 1)
+            if (c >> l2) & 1 and low:
+                nq += 1
+            lowz = ~c & ((1 << l2) - 1)
+            if not (c >> l2) & 1 and lowz and (((c >> l2) + 1) << l2) <= N - 1:
+                nk += 1
+    return nq, nk, nlev
+
+
+def flops_m2(B, H, L, d):
+    S = B * H
+    N = -(-L // CHUNK)
+    Bc = CHUNK
+    f1, b1 = flops_m1(B, H, L, d)
+    prep = S * N * (12 * Bc * Bc * d + 2 * Bc * d * d + 2.67 * Bc ** 3)
+    nq, nk, nlev = _version_steps(N)
+    dy = sum(S * (N >> l) * 2 * d ** 3 for l in range(1, max(nlev - 1, 0)))
+    ver = S * (nq + nk) * 2 * Bc * d * d
+    diag = S * N * 2 * Bc ** 3
+    fwd = f1 + prep + dy + ver + diag
+    chain = S * N * (14 * 2 * Bc * Bc * d + 6 * 2 * Bc ** 3 + 2 * 2 * Bc * d * d)
+    bwd = b1 + (prep + dy + ver) + 2 * diag + 2 * ver + 2 * dy + chain
+    return fwd, bwd
+
+
+# ----------------------------------------------------------------------------------------- helpers
+def shard_info():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def max_over_ranks(x: float, world: int, device=None) -> float:
+    """Maximum of a per-rank scalar over all ranks (identity for one rank)."""
+    if world == 1:
+        return float(x)
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"burst": p["bf16_tflops"], "sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "hbm": p["hbm_gbs"], "source": "measured"}
+    return {"burst": 1590.0, "sustained": 1400.0, "hbm": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) >= 6:
+                self.samples.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm = sorted(int(s[0]) for s in self.samples if s[0].isdigit())
+        mx = [int(s[1]) for s in self.samples if s[1].isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        ids = [x for x in vis.split(",") if x.strip() != ""]
+        if local < len(ids) and ids[local].strip().isdigit():
+            return int(ids[local])
+    return local
+
+
+# ----------------------------------------------------------------------------------------- reference arm
+def oracle_sample(cfg, inp, n_slices=1):
+    """Forward + backward of the float64 oracle on the first `n_slices` (batch, head) slices.  Returns seconds."""
+    from oracle import path_oracle as po
+    f = synth.to_f64
+    sl = lambda t: None if t is None else f(t.reshape(-1, *t.shape[2:])[:n_slices])
+    q, k, v, w, beta, d_o, g = (sl(inp[n]) for n in ("q", "k", "v", "w", "beta", "d_o", "log_f"))
+    t0 = time.perf_counter()
+    po.forward(q, k, v, w, beta, g, scale=inp["scale"])
+    po.backward(q, k, v, w, beta, d_o, g, scale=inp["scale"])
+    return time.perf_counter() - t0, po.num_threads()
+
+
+def run_reference(args, cfg):
+    rank, world, _ = shard_info()
+    if rank != 0:
+        return
+    inp = synth.make_config(args.workload)
+    f1, b1 = flops_m1(1, 1, cfg["L"], cfg["d"])  # one slice per step
+    for _ in range(args.warmup):
+        oracle_sample(cfg, inp)
+    secs = []
+    cores = 1
+    for _ in range(args.steps):
+        s, cores = oracle_sample(cfg, inp)
+        secs.append(s)
+    ms = 1e3 * sum(secs) / len(secs)
+    val = (f1 + b1) / (ms * 1e-3) / 1e12
+    sample = f"1 of {cfg['B'] * cfg['H']} (batch, head) slices of {args.workload} per step, forward + backward, float64"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: B={cfg['B']} H={cfg['H']} L={cfg['L']} d={cfg['d']} fwd+bwd",
+                   "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------- our arm
+def run_ours(args, cfg):
+    from paper_2505_16381_b200 import binding
+    rank, world, local = shard_info()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the hot path has no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    binding.load()
+
+    B, H, L, d = cfg["B"], cfg["H"], cfg["L"], cfg["d"]
+    inp = synth.make_inputs(B, H, L, d, dtype=cfg["dtype"], qk_scaled=cfg["qk_scaled"], gate=cfg["gate"],
+                            seed=synth.BASE_SEED + cfg["index"] + 1000 * rank)
+    names = ["q", "k", "v", "w", "beta", "d_o"] + (["log_f"] if cfg["gate"] else [])
+    host = {n: inp[n].pin_memory() for n in names}
+    devt = {n: host[n].to(dev, non_blocking=True) for n in names}
+    devt.setdefault("log_f", None)
+    scale = inp["scale"]
+    ws = binding.alloc_workspace(devt["q"], cfg["gate"], True)
+    o = torch.empty_like(devt["q"])
+    lse = torch.empty(B, H, L, dtype=torch.float32, device=dev)
+    gout = {n: torch.empty_like(devt["q"]) for n in ("dq", "dk", "dv", "dw")}
+    gout["dbeta"] = torch.empty_like(devt["beta"])
+    if cfg["gate"]:
+        gout["dlog_f"] = torch.empty_like(devt["beta"])
+    launches = [0]
+
+    def step(t):
+        binding.path_attn_fwd(t["q"], t["k"], t["v"], t["w"], t["beta"], t["log_f"], scale=scale, workspace=ws,
+                              out=(o, lse))
+        n = binding.last_launch_count()
+        binding.path_attn_bwd(t["q"], t["k"], t["v"], t["w"], t["beta"], o, lse, t["d_o"], t["log_f"], scale=scale,
+                              workspace=ws, out=gout)
+        launches[0] = n + binding.last_launch_count()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing, with per-stage events
+    for _ in range(args.warmup):
+        step(devt)
+    binding.device_status(ws)
+    binding.profile_enable(True)
+    stage_ms = {}
+    sampler = ClockSampler(physical_gpu_index(local))
+    barrier()
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step(devt)
+        for k_, v_ in binding.profile_read().items():  # waits for this step's events
+            stage_ms[k_] = stage_ms.get(k_, 0.0) + v_
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1) / args.steps
+    clocks = sampler.stop() if rank == 0 else None
+    binding.profile_enable(False)
+    binding.device_status(ws)
+    ms = max_over_ranks(ms, world, dev)
+    stage_ms = {k_: v_ / args.steps for k_, v_ in stage_ms.items()}
+
+    # ---- end to end: host buffers in, host buffers out, every step
+    hout = {n: torch.empty(t.shape, dtype=t.dtype).pin_memory() for n, t in gout.items()}
+    h2d = sum(host[n].numel() * host[n].element_size() for n in names)
+    d2h = sum(t.numel() * t.element_size() for t in hout.values())
+
+    def e2e_step():
+        t = {n: host[n].to(dev, non_blocking=True) for n in names}
+        t.setdefault("log_f", None)
+        step(t)
+        for n in hout:
+            hout[n].copy_(gout[n], non_blocking=True)
+
+    for _ in range(min(args.warmup, 3)):
+        e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, dev)
+
+    # ---- report
+    f1, b1 = flops_m1(B, H, L, d)
+    f2, b2 = flops_m2(B, H, L, d)
+    peaks = load_peaks()
+    tf = lambda fl, t_ms: fl / (t_ms * 1e-3) / 1e12
+    value = world * tf(f1 + b1, ms)
+    stage_flops = {"fa_fwd": f1 + B * H * (L // CHUNK) * 2 * CHUNK ** 3, "fa_bwd_dkv": 2.0 * f1, "fa_bwd_dq": 1.5 * f1}
+    top = max(stage_ms, key=stage_ms.get) if stage_ms else None
+    roof = None
+    if top is not None:
+        fl = stage_flops.get(top)
+        if fl is None:  # a multi-kernel linear stage: report its M2 share
+            fl = {"chunk_prep": f2 - f1, "bwd_chunk_prep": f2 - f1, "bwd_chains": b2 - b1 - (f2 - f1)}.get(top, 0.0)
+        ach = tf(fl, stage_ms[top])
+        roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["sustained"], "unit": "TFLOP/s",
+                "frac": ach / peaks["sustained"], "traffic": NCU_TRAFFIC_BYTES.get(top),
+                "peak_source": f"{peaks['source']} cuBLAS bf16, sustained", "ms_per_launch": stage_ms[top],
+                "flops_per_launch": fl}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"{args.workload}: B={B} H={H} L={L} d={d} bf16 fwd+bwd per GPU", "global_batch": B * world,
+                   "seq_len": L, "parallelism": f"{world} independent replicas (no collective)",
+                   "l2_policy": "inputs + workspace exceed L2 (no flush needed)", "chunk": CHUNK},
+        "clocks": clocks,
+        "e2e": {"value": world * tf(f1 + b1, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches[0] * args.steps,
+        "roofline": roof,
+        "detail": {
+            "tflops_m2": world * tf(f2 + b2, ms),
+            "frac_of_burst_peak_m1": tf(f1 + b1, ms) / peaks["burst"], "frac_of_burst_peak_m2": tf(f2 + b2, ms) / peaks["burst"],
+            "frac_of_nominal_m1": tf(f1 + b1, ms) / 2250.0,
+            "stage_ms": stage_ms,
+            "stage_tflops": {k_: tf(stage_flops[k_], v_) for k_, v_ in stage_ms.items() if k_ in stage_flops},
+            "launches_per_step": launches[0], "peaks": peaks,
+        },
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        secs1, cores = oracle_sample(cfg, inp)                       # sizes the sample: aim at ~15 s of CPU work
+        n = int(min(B * H, max(1, round(15.0 / max(secs1, 1e-3)))))
+        secs, cores = oracle_sample(cfg, inp, n)
+        s1, sb1 = flops_m1(1, 1, L, d)
+        line["cpu_baseline"] = {"value": n * (s1 + sb1) / secs / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{n} of {B * H} (batch, head) slices of {args.workload}, forward + backward, "
+                                          f"float64, {secs:.1f} s"}
+    else:
+        line["cpu_baseline"] = None
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="C3", choices=[n for n, c in synth.CONFIGS.items() if c["backward"]])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling captures)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = dict(synth.CONFIGS[args.workload])
+    if args.batch > 0:
+        cfg["B"] = args.batch
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

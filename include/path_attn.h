@@ -103,6 +103,23 @@ int path_attn_device_status(const void* workspace, void* cuda_stream, unsigned i
 /* Static description of a status code. */
 const char* path_attn_strerror(int status);
 
+/*
+ * Optional stage timing for benchmarks (no counterpart in the paper).  After
+ * path_attn_profile_enable(1), every fwd / bwd call of the calling thread records
+ * CUDA events on its stream around its stages: "chunk_prep" (UT transform,
+ * boundary-adjusted tiles, run products, versions; Sec. 3.1/3.3), "fa_fwd" (the
+ * fused sweep, one kernel); and for bwd "bwd_chunk_prep" (the same preparation,
+ * recomputed), "rowstats", "fa_bwd_dkv", "fa_bwd_dq" (one kernel each) and
+ * "bwd_chains".  path_attn_profile_read waits for those events and writes the
+ * milliseconds per stage of the most recent fwd and the most recent bwd call
+ * into ms[0..n) (-1 for a stage that did not run); it returns the number of entries written or a
+ * negative status.  The events are created on first use and live until the
+ * thread exits; nothing else is allocated.
+ */
+int path_attn_profile_enable(int on);
+int path_attn_profile_read(float* ms, int n);
+const char* path_attn_profile_stage_name(int i);
+
 /* cudaError_t (as int) of the CUDA call behind the calling thread's most recent PATH_ERR_LAUNCH. */
 int path_attn_last_cuda_error(void);
 

@@ -18,7 +18,8 @@ _lib = None
 PATH_BF16, PATH_FP32 = 0, 1
 PATH_OK = 0
 EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_attn_device_status",
-           "path_attn_strerror", "path_attn_last_cuda_error", "path_attn_last_launch_count"]
+           "path_attn_strerror", "path_attn_last_cuda_error", "path_attn_last_launch_count",
+           "path_attn_profile_enable", "path_attn_profile_read", "path_attn_profile_stage_name"]
 
 
 class PathAttnError(RuntimeError):
@@ -51,6 +52,12 @@ def load():
         lib.path_attn_strerror.argtypes = [I]
         lib.path_attn_last_cuda_error.restype = I
         lib.path_attn_last_launch_count.restype = I
+        lib.path_attn_profile_enable.restype = I
+        lib.path_attn_profile_enable.argtypes = [I]
+        lib.path_attn_profile_read.restype = I
+        lib.path_attn_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), I]
+        lib.path_attn_profile_stage_name.restype = ctypes.c_char_p
+        lib.path_attn_profile_stage_name.argtypes = [I]
         _lib = lib
     return _lib
 
@@ -146,3 +153,18 @@ def device_status(workspace) -> int:
 
 def last_launch_count() -> int:
     return int(load().path_attn_last_launch_count())
+
+
+def profile_enable(on: bool = True) -> None:
+    """Turns the library's per-stage CUDA-event timing on or off for the calling thread."""
+    load().path_attn_profile_enable(int(on))
+
+
+def profile_read() -> dict:
+    """Milliseconds per stage of the most recent fwd / bwd call (stages that did not run are omitted)."""
+    lib = load()
+    buf = (ctypes.c_float * 16)()
+    n = lib.path_attn_profile_read(buf, 16)
+    if n < 0:
+        raise PathAttnError(n, "path_attn_profile_read")
+    return {lib.path_attn_profile_stage_name(i).decode(): float(buf[i]) for i in range(n) if buf[i] >= 0}

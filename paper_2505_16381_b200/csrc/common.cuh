@@ -75,7 +75,7 @@ struct BwdParams {
     float scale;
 };
 
-cudaError_t launch_fa_bwd(const BwdTensorMaps& tm, const BwdParams& p, int hd, cudaStream_t st);
+cudaError_t launch_fa_bwd(const BwdTensorMaps& tm, const BwdParams& p, int hd, int which, cudaStream_t st);
 cudaError_t launch_rowstats(const void* o, const void* d_o, const float* lse, float* delta, float* lse2, int S, int L,
                             int Lp, int hd, cudaStream_t st);
 cudaError_t launch_fa_fwd(const FwdTensorMaps& tm, const FwdParams& p, int hd, cudaStream_t st);

@@ -478,23 +478,25 @@ constexpr int kDkvSmem = 6 * kSlotBytes + 256 + 2 * 3 * kTile * 4 + 1024;
 constexpr int kDqSmem = 7 * kSlotBytes + 256 + 2 * kTile * 4 + 1024;
 
 template <int HD, bool GATE>
-cudaError_t launch_both(const BwdTensorMaps& tm, const BwdParams& p, cudaStream_t st) {
-    cudaError_t e = set_smem(dkv_kernel<HD, GATE>, kDkvSmem);
-    if (e != cudaSuccess) return e;
-    e = set_smem(dq_kernel<HD, GATE>, kDqSmem);
-    if (e != cudaSuccess) return e;
-    dkv_kernel<HD, GATE><<<dim3(p.N, p.S), 192, kDkvSmem, st>>>(tm, p);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    dq_kernel<HD, GATE><<<dim3(p.N, p.S), 192, kDqSmem, st>>>(tm, p);
+cudaError_t launch_one(const BwdTensorMaps& tm, const BwdParams& p, int which, cudaStream_t st) {
+    if (which == 0) {
+        cudaError_t e = set_smem(dkv_kernel<HD, GATE>, kDkvSmem);
+        if (e != cudaSuccess) return e;
+        dkv_kernel<HD, GATE><<<dim3(p.N, p.S), 192, kDkvSmem, st>>>(tm, p);
+    } else {
+        cudaError_t e = set_smem(dq_kernel<HD, GATE>, kDqSmem);
+        if (e != cudaSuccess) return e;
+        dq_kernel<HD, GATE><<<dim3(p.N, p.S), 192, kDqSmem, st>>>(tm, p);
+    }
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_fa_bwd(const BwdTensorMaps& tm, const BwdParams& p, int hd, cudaStream_t st) {
-    if (hd == 64) return p.G ? launch_both<64, true>(tm, p, st) : launch_both<64, false>(tm, p, st);
-    return p.G ? launch_both<128, true>(tm, p, st) : launch_both<128, false>(tm, p, st);
+// which = 0: dK/dV sweep, which = 1: dQ sweep.
+cudaError_t launch_fa_bwd(const BwdTensorMaps& tm, const BwdParams& p, int hd, int which, cudaStream_t st) {
+    if (hd == 64) return p.G ? launch_one<64, true>(tm, p, which, st) : launch_one<64, false>(tm, p, which, st);
+    return p.G ? launch_one<128, true>(tm, p, which, st) : launch_one<128, false>(tm, p, which, st);
 }
 
 cudaError_t launch_rowstats(const void* o, const void* d_o, const float* lse, float* delta, float* lse2, int S, int L,

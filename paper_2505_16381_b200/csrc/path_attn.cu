@@ -23,6 +23,31 @@ static thread_local int g_launches = 0;
     } while (0)
 #define LAUNCH(expr) do { CK(expr); ++g_launches; } while (0)
 
+// ------------------------------------------------------------------------------------------- stage timing
+// Optional per-thread instrumentation: CUDA events around groups of launches of the most recent call.
+enum Stage { STG_PREP = 0, STG_FA_FWD, STG_PREP_BWD, STG_ROWSTATS, STG_FA_DKV, STG_FA_DQ, STG_CHAINS, STG_COUNT };
+static const char* const kStageNames[STG_COUNT] = {"chunk_prep", "fa_fwd", "bwd_chunk_prep", "rowstats", "fa_bwd_dkv",
+                                                   "fa_bwd_dq", "bwd_chains"};
+struct Profiler {
+    bool on = false, created = false;
+    cudaEvent_t ev[2 * STG_COUNT];
+    bool used[STG_COUNT];
+};
+static thread_local Profiler g_prof;
+
+static void prof_reset(int first = 0, int last = STG_COUNT) {
+    for (int i = first; i < last; ++i) g_prof.used[i] = false;
+}
+static void prof_mark(int stage, int end, cudaStream_t st) {
+    if (!g_prof.on) return;
+    if (!g_prof.created) {
+        for (int i = 0; i < 2 * STG_COUNT; ++i) cudaEventCreate(&g_prof.ev[i]);
+        g_prof.created = true;
+    }
+    cudaEventRecord(g_prof.ev[2 * stage + end], st);
+    if (end) g_prof.used[stage] = true;
+}
+
 // ------------------------------------------------------------------------------------------- tensor maps
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -347,6 +372,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     float* Dy = at<float>(ws, p.Dy); float* dDy = at<float>(ws, p.dDy);
     float* dQv = at<float>(ws, p.dQv); float* dKv = at<float>(ws, p.dKv);
 
+    prof_mark(STG_ROWSTATS, 0, st);
     LAUNCH(launch_rowstats(o, d_o, lse, at<float>(ws, p.delta), at<float>(ws, p.lse2), p.S, p.L, p.Lp, d, st));
     const void* dop = d_o;
     if (p.ragged) {
@@ -372,8 +398,14 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     bp.G = p.gate ? at<float>(ws, p.G) : nullptr;
     bp.status = at<uint32_t>(ws, p.status);
     bp.S = p.S; bp.L = p.L; bp.Lp = p.Lp; bp.N = p.N; bp.scale = scale;
-    CK(launch_fa_bwd(tm, bp, d, st));
-    g_launches += 2;
+    prof_mark(STG_ROWSTATS, 1, st);
+    prof_mark(STG_FA_DKV, 0, st);
+    LAUNCH(launch_fa_bwd(tm, bp, d, 0, st));
+    prof_mark(STG_FA_DKV, 1, st);
+    prof_mark(STG_FA_DQ, 0, st);
+    LAUNCH(launch_fa_bwd(tm, bp, d, 1, st));
+    prof_mark(STG_FA_DQ, 1, st);
+    prof_mark(STG_CHAINS, 0, st);
 
     // version chains, top level first: gradients of the run products, then of the lower versions
     for (int l2 = p.nlev - 1; l2 >= 1; --l2)
@@ -418,6 +450,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
         LAUNCH(launch_gate_suffix(at<float>(ws, p.dG), at<float>(ws, p.dGrow), at<float>(ws, p.dGdiag), dlog_f, p.S, p.L,
                                   p.Lp, st));
     }
+    prof_mark(STG_CHAINS, 1, st);
     return PATH_OK;
 }
 
@@ -451,10 +484,13 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     cudaStream_t st = (cudaStream_t)cuda_stream;
     CK(cudaMemsetAsync(workspace, 0, 256, st));
 
+    prof_reset(STG_PREP, STG_PREP_BWD);
+    prof_mark(STG_PREP, 0, st);
     rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, st);
     if (rc != PATH_OK) return rc;
     rc = run_prep(p, workspace, q, k, w, st);
     if (rc != PATH_OK) return rc;
+    prof_mark(STG_PREP, 1, st);
 
     FwdTensorMaps tm;
     const uint64_t rows = (uint64_t)p.S * p.Lp;
@@ -468,7 +504,9 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     fp.o = o; fp.lse = lse; fp.G = log_f ? at<float>(workspace, p.G) : nullptr;
     fp.status = at<uint32_t>(workspace, p.status);
     fp.S = p.S; fp.L = L; fp.Lp = p.Lp; fp.N = p.N; fp.scale = scale; fp.out_fp32 = 0;
+    prof_mark(STG_FA_FWD, 0, st);
     LAUNCH(launch_fa_fwd(tm, fp, d, st));
+    prof_mark(STG_FA_FWD, 1, st);
     return PATH_OK;
 }
 
@@ -493,10 +531,13 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
     if (rc != PATH_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     CK(cudaMemsetAsync(workspace, 0, 256, st));
+    prof_reset(STG_PREP_BWD, STG_COUNT);
+    prof_mark(STG_PREP_BWD, 0, st);
     rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, st);
     if (rc != PATH_OK) return rc;
     rc = run_prep(p, workspace, q, k, w, st);
     if (rc != PATH_OK) return rc;
+    prof_mark(STG_PREP_BWD, 1, st);
     return run_backward(p, workspace, q, k, v, w, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, scale, st);
 }
 
@@ -527,6 +568,29 @@ const char* path_attn_strerror(int status) {
         default: return "unknown status";
     }
 }
+
+int path_attn_profile_enable(int on) {
+    g_prof.on = on != 0;
+    if (!on) prof_reset();
+    return PATH_OK;
+}
+
+int path_attn_profile_read(float* ms, int n) {
+    if (!ms) return PATH_ERR_NULL;
+    int written = 0;
+    for (int i = 0; i < STG_COUNT && i < n; ++i, ++written) {
+        ms[i] = -1.f;
+        if (!g_prof.on || !g_prof.created || !g_prof.used[i]) continue;
+        if (cudaEventSynchronize(g_prof.ev[2 * i + 1]) != cudaSuccess ||
+            cudaEventElapsedTime(&ms[i], g_prof.ev[2 * i], g_prof.ev[2 * i + 1]) != cudaSuccess) {
+            g_last_cuda_error = (int)cudaGetLastError();
+            return PATH_ERR_LAUNCH;
+        }
+    }
+    return written;
+}
+
+const char* path_attn_profile_stage_name(int i) { return (i >= 0 && i < STG_COUNT) ? kStageNames[i] : ""; }
 
 int path_attn_last_cuda_error(void) { return g_last_cuda_error; }
 int path_attn_last_launch_count(void) { return g_launches; }

@@ -1,0 +1,181 @@
+"""Parity of the CUDA path (through the C ABI) with the float64 oracle on identical seeded inputs.
+
+Tolerances (bf16 I/O, float32 accumulation): relative Frobenius error <= 1e-2 and max-abs error
+<= 2e-2 on O and every gradient.  The absolute bound is scaled by max(1, max|reference|): an output
+stored in bf16 cannot be closer than half an ulp (2^-9 relative) to the reference, so for gradients whose
+magnitude exceeds ~5 the unscaled bound would be below the storage format's resolution.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_16381_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+REL_FRO, MAX_ABS = 1e-2, 2e-2
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2505_16381_b200 import binding as b
+    b.load()
+    assert torch.cuda.is_available()
+    return b
+
+
+def to_dev(inp):
+    return {k: (v.cuda() if torch.is_tensor(v) else v) for k, v in inp.items()}
+
+
+def gpu_forward(b, dev, scale):
+    ws = b.alloc_workspace(dev["q"], dev["log_f"] is not None, False)
+    o, lse = b.path_attn_fwd(dev["q"], dev["k"], dev["v"], dev["w"], dev["beta"], dev["log_f"], scale=scale, workspace=ws)
+    assert b.device_status(ws) == 0
+    return o, lse
+
+
+def gpu_backward(b, dev, o, lse, scale):
+    ws = b.alloc_workspace(dev["q"], dev["log_f"] is not None, True)
+    g = b.path_attn_bwd(dev["q"], dev["k"], dev["v"], dev["w"], dev["beta"], o, lse, dev["d_o"], dev["log_f"],
+                        scale=scale, workspace=ws)
+    assert b.device_status(ws) == 0
+    return g
+
+
+def check(name, got, ref, rel=REL_FRO, mx=MAX_ABS):
+    got = got.detach().float().cpu().double().numpy() if torch.is_tensor(got) else got
+    err = np.abs(got - ref).max()
+    nrm = np.linalg.norm(ref)
+    relerr = np.linalg.norm(got - ref) / nrm if nrm > 0 else np.linalg.norm(got)
+    assert np.isfinite(got).all(), name
+    assert relerr <= rel, (name, "rel-fro", relerr)
+    assert err <= mx * max(1.0, np.abs(ref).max()), (name, "max-abs", err)
+
+
+def slices(inp, idx):
+    """Float64 views of the chosen flattened (batch, head) slices."""
+    f = synth.to_f64
+    pick = lambda t: None if t is None else f(t.reshape(-1, *t.shape[2:])[idx])
+    return {n: pick(inp[n]) for n in ("q", "k", "v", "w", "beta", "d_o", "log_f")}
+
+
+def compare_all(b, oracle, inp, scale=1.0, idx=None, backward=True):
+    dev = to_dev(inp)
+    S = inp["q"].shape[0] * inp["q"].shape[1]
+    idx = list(range(S)) if idx is None else idx
+    o, lse = gpu_forward(b, dev, scale)
+    x = slices(inp, idx)
+    o_ref, lse_ref = oracle.forward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["log_f"], scale=scale)
+    flat = lambda t: t.reshape(-1, *t.shape[2:])[idx]
+    check("o", flat(o), o_ref)
+    assert np.abs(flat(lse).cpu().double().numpy() - lse_ref).max() <= 2e-3 * max(1.0, np.abs(lse_ref).max())
+    if not backward:
+        return o, lse, None
+    g = gpu_backward(b, dev, o, lse, scale)
+    ref = oracle.backward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["d_o"], x["log_f"], scale=scale)
+    for name, r in ref.items():
+        check(name, flat(g[name]), r)
+    return o, lse, g
+
+
+# ---------------------------------------------------------------- small shapes: several tiles, ragged tails
+
+@pytest.mark.parametrize("B,H,L,d,gate,sharp", [
+    (1, 2, 300, 64, False, False),
+    (1, 1, 1000, 128, True, False),
+    (2, 2, 512, 64, True, True),
+    (1, 2, 1024, 128, False, True),
+    (1, 3, 1408, 128, False, False),     # 11 chunks: version chains with a non-power-of-two count
+    (1, 2, 1, 64, False, False),
+    (1, 2, 127, 64, True, False),
+    (1, 2, 128, 128, False, False),
+    (1, 2, 129, 128, True, False),
+])
+def test_small_shapes_match_oracle(binding, oracle, B, H, L, d, gate, sharp):
+    inp = synth.make_inputs(B, H, L, d, "bf16", gate=gate, seed=11 + L + d, sharp=sharp)
+    compare_all(binding, oracle, inp)
+
+
+def test_explicit_scale(binding, oracle):
+    inp = synth.make_inputs(1, 2, 640, 64, "bf16", qk_scaled=False, gate=True, seed=5)
+    compare_all(binding, oracle, inp, scale=1.0 / 8.0)
+
+
+@pytest.mark.parametrize("mode", ["beta0", "beta2", "beta1", "w0"])
+def test_degenerate_householders(binding, oracle, mode):
+    """beta = 0 (plain causal attention), beta = 2 (exact reflections), beta = 1 (projections), some w = 0."""
+    inp = synth.make_inputs(1, 2, 512, 64, "bf16", seed=23, sharp=True)
+    if mode == "beta0":
+        inp["beta"].zero_()
+    elif mode == "beta2":
+        inp["beta"].fill_(2.0)
+    elif mode == "beta1":
+        inp["beta"].fill_(1.0)
+    else:
+        inp["w"][:, :, ::3] = 0
+    compare_all(binding, oracle, inp)
+
+
+def test_forward_is_bitwise_reproducible_and_workspace_is_reusable(binding):
+    inp = to_dev(synth.make_inputs(2, 2, 1024, 128, "bf16", gate=True, seed=3))
+    ws = binding.alloc_workspace(inp["q"], True, True)   # backward-sized: shared by both directions
+    run = lambda: binding.path_attn_fwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"], inp["log_f"], workspace=ws)
+    o1, l1 = run()
+    g1 = binding.path_attn_bwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"], o1, l1, inp["d_o"], inp["log_f"],
+                               workspace=ws)
+    o2, l2 = run()
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+    g2 = binding.path_attn_bwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"], o1, l1, inp["d_o"], inp["log_f"],
+                               workspace=ws)
+    for n in g1:  # float atomics in the run-product gradients: equal to rounding, not bitwise
+        assert torch.allclose(g1[n].float(), g2[n].float(), rtol=2e-2, atol=1e-3), n
+    assert torch.equal(g1["dv"], g2["dv"])
+    assert binding.device_status(ws) == 0
+
+
+# ---------------------------------------------------------------- the named workloads at full size
+
+def test_c2_full_size_sampled_slices(binding, oracle):
+    inp = synth.make_config("C2")
+    compare_all(binding, oracle, inp, idx=[0, 37, 127])
+
+
+def test_c3_headline_full_size_sampled_slices_and_invariants(binding, oracle):
+    inp = synth.make_config("C3")
+    o, lse, g = compare_all(binding, oracle, inp, idx=[0, 63])
+    # exact invariants that hold at any size (all slices)
+    w, beta = inp["w"].double(), inp["beta"].double()
+    dw, dbeta = g["dw"].cpu().double(), g["dbeta"].cpu().double()
+    lhs, rhs = (w * dw).sum(-1), 2 * beta * dbeta
+    assert (lhs - rhs).norm() <= 2e-2 * rhs.norm()
+    qdq = (inp["q"].double() * g["dq"].cpu().double()).sum((-1, -2))
+    kdk = (inp["k"].double() * g["dk"].cpu().double()).sum((-1, -2))
+    assert (qdq - kdk).abs().max() <= 2e-2 * kdk.abs().max()
+    assert dw[:, :, 0].abs().max() <= 1e-3 and dbeta[:, :, 0].abs().max() <= 1e-3
+    assert torch.isfinite(g["dq"]).all() and torch.isfinite(o).all()
+
+
+def test_c4_path_fox_full_size_one_slice(binding, oracle):
+    inp = synth.make_config("C4")
+    compare_all(binding, oracle, inp, idx=[17])
+
+
+def test_c5_long_prefill_forward_sampled_rows(binding, oracle):
+    inp = synth.make_config("C5")
+    dev = to_dev({k: v for k, v in inp.items() if k != "d_o"})
+    dev["log_f"] = None
+    o, lse = gpu_forward(binding, dev, 1.0)
+    L = inp["q"].shape[2]
+    rng = np.random.default_rng(5)
+    rows = sorted(set([0, 127, 128, L - 1] + rng.integers(0, L, 60).tolist()))
+    idx = [0, 9, 20, 31]
+    f = synth.to_f64
+    pick = lambda t: f(t.reshape(-1, *t.shape[2:])[idx])
+    o_ref, lse_ref = oracle.forward(pick(inp["q"]), pick(inp["k"]), pick(inp["v"]), pick(inp["w"]), pick(inp["beta"]),
+                                    None, scale=1.0, rows=rows)
+    og = o.reshape(-1, L, o.shape[-1])[idx][:, rows]
+    check("o", og, o_ref)
+    lg = lse.reshape(-1, L)[idx][:, rows].cpu().double().numpy()
+    assert np.abs(lg - lse_ref).max() <= 2e-3 * max(1.0, np.abs(lse_ref).max())
+    assert torch.isfinite(o).all()
