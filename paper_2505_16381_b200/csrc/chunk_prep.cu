@@ -1,0 +1,357 @@
+// Per-chunk compact representation of the Householder product (paper Sec. 3.1 UT transform) and the
+// boundary-adjusted queries / keys and chunk product built from it (Sec. 3.3), fused into one kernel.
+//
+// One CTA owns one 128-token chunk.  With W, Q, K the chunk's rows and D = diag(beta):
+//   Gm = W W^T,  Xq = lower(Q W^T),  Xk = strictLower(W K^T)                      (MMA group 1)
+//   T~ = (I + strictLower(D Gm))^-1 D                                             (float32, blocked substitution)
+//   U = T~ W,  Y = T~ Xk                                                          (MMA group 2)
+//   Qleft = Q - Xq U,  Kright = K - Y^T W,  P = I - W^T U                          (MMA group 3)
+// and the bf16 operands of the diagonal-chunk correction of the attention sweep, Xqn = -Xq and Yt = Y^T.
+//
+// Every product is a 128 x 128 x {64,128} tcgen05 MMA whose operands sit in shared memory as row-major
+// 128-byte-swizzled tiles; whether a tile enters as X, X^T, on the left or on the right is only a matter of
+// the descriptor's major-ness, so nothing is ever transposed in memory.  Accumulators live in tensor memory and
+// are read back one row per thread.  T~ is kept as a bf16 pair (hi + lo) because everything downstream
+// depends on it; the other intermediates are rounded to bf16 once, like the tiles the attention sweep consumes.
+#include "common.cuh"
+#include "tc5.cuh"
+
+namespace path {
+using namespace tc5;
+
+namespace {
+
+constexpr int kT = 128;
+constexpr uint32_t kTileB = 32768, kPanelB = 16384;
+constexpr int kLd = kT + 1;  // row stride of the float32 triangular buffer
+
+struct PrepSmem {
+    static constexpr uint32_t offW = 0;
+    static constexpr uint32_t offQK = offW + kTileB;            // Q, K  ->  T hi, T lo  ->  U, Y
+    static constexpr uint32_t offBig = offQK + 2 * kTileB;      // float32 triangular buffer  ->  Xq, Xk tiles
+    static constexpr uint32_t bigBytes = ((kT * kLd * 4 + 1023) / 1024) * 1024;
+    static constexpr uint32_t offDiag = offBig + bigBytes;      // [8][16][17] float
+    static constexpr uint32_t offZ = offDiag + 8 * 16 * 17 * 4; // [16][128] float
+    static constexpr uint32_t offBeta = offZ + 16 * kT * 4;     // [128] float
+    static constexpr uint32_t offBar = offBeta + kT * 4;
+    static constexpr uint32_t total = offBar + 64;
+    static constexpr uint32_t alloc = total + 1024;
+};
+
+// K-major view: contraction over the tile's columns.  MN-major view: contraction over the tile's rows.
+__device__ __forceinline__ uint64_t desc_k(uint32_t tile, int kk) {
+    return umma_desc(tile + (kk >> 2) * kPanelB + (kk & 3) * 32, 16, 1024);
+}
+__device__ __forceinline__ uint64_t desc_mn(uint32_t tile, int kk) { return umma_desc(tile + kk * 2048, kPanelB, 1024); }
+
+enum { OP_K = 0, OP_MN = 1 };
+// D (+)= op(A) op(B) over `ksteps` steps of 16.
+__device__ __forceinline__ void mma(uint32_t d_tmem, uint32_t a_tile, int a_op, uint32_t b_tile, int b_op, int ksteps,
+                                    int n, bool acc) {
+    const uint32_t idesc = umma_idesc(128, n, a_op, b_op);
+    for (int kk = 0; kk < ksteps; ++kk)
+        umma_ss(d_tmem, a_op == OP_K ? desc_k(a_tile, kk) : desc_mn(a_tile, kk),
+                b_op == OP_K ? desc_k(b_tile, kk) : desc_mn(b_tile, kk), idesc, (acc || kk > 0) ? 1u : 0u);
+}
+
+// Stores 32 consecutive columns (c0 .. c0+31) of `row` of a row-major swizzled bf16 tile.
+__device__ __forceinline__ void tile_store32(uint8_t* tile, int row, int c0, const float (&v)[32]) {
+    uint8_t* panel = tile + (c0 >> 6) * kPanelB;
+    const int ch0 = (c0 & 63) >> 3;
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch)
+        *reinterpret_cast<uint4*>(panel + sw128_off((uint32_t)row, (uint32_t)(ch0 + ch))) =
+            make_uint4(pack_bf16(v[8 * ch], v[8 * ch + 1]), pack_bf16(v[8 * ch + 2], v[8 * ch + 3]),
+                       pack_bf16(v[8 * ch + 4], v[8 * ch + 5]), pack_bf16(v[8 * ch + 6], v[8 * ch + 7]));
+}
+__device__ __forceinline__ void gstore_f32x32(float* dst, const float (&v)[32]) {
+#pragma unroll
+    for (int x = 0; x < 8; ++x)
+        reinterpret_cast<float4*>(dst)[x] = make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
+}
+__device__ __forceinline__ void gstore_bf16x32(__nv_bfloat16* dst, const float (&v)[32]) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+        reinterpret_cast<uint4*>(dst)[x] =
+            make_uint4(pack_bf16(v[8 * x], v[8 * x + 1]), pack_bf16(v[8 * x + 2], v[8 * x + 3]),
+                       pack_bf16(v[8 * x + 4], v[8 * x + 5]), pack_bf16(v[8 * x + 6], v[8 * x + 7]));
+}
+__device__ __forceinline__ void gload_bf16x32(const __nv_bfloat16* src, float (&v)[32]) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const uint4 u = reinterpret_cast<const uint4*>(src)[x];
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[y]));
+            v[8 * x + 2 * y] = f.x;
+            v[8 * x + 2 * y + 1] = f.y;
+        }
+    }
+}
+
+template <int HD, bool SAVE>
+__global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constant__ PrepTensorMaps tm, const PrepParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* sW = smem + PrepSmem::offW;
+    uint8_t* sQK = smem + PrepSmem::offQK;
+    uint8_t* sBig = smem + PrepSmem::offBig;
+    float* Xb = (float*)sBig;
+    float* diagX = (float*)(smem + PrepSmem::offDiag);
+    float* Z = (float*)(smem + PrepSmem::offZ);
+    float* bt = (float*)(smem + PrepSmem::offBeta);
+    uint64_t* bars = (uint64_t*)(smem + PrepSmem::offBar);  // [0] loads, [1] MMA groups
+    uint32_t* tmem_slot = (uint32_t*)(bars + 2);
+    volatile uint32_t* abort_flag = (volatile uint32_t*)(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int chunk = blockIdx.x;                 // flattened (slice, chunk): rows chunk*128 .. +127 of the padded arrays
+    const int row = (warp & 3) * 32 + lane;       // accumulator row (TMEM lane) of this thread
+    const int half = warp >> 2;                   // which half of the accumulator's columns
+    const size_t grow = (size_t)chunk * kT + row; // global row
+
+    if (tid == 0) {
+        mbar_init(&bars[0], 1);
+        mbar_init(&bars[1], 1);
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    if (warp == 0) tmem_alloc(tmem_slot, 512);
+    if (tid < kT) bt[tid] = p.beta[(size_t)chunk * kT + tid];
+    if (HD == 64) {  // second panel of W must read as zeros when W^T is used with M = 128
+        for (int i = tid; i < (int)(kPanelB / 16); i += 256) reinterpret_cast<uint4*>(sW + kPanelB)[i] = make_uint4(0, 0, 0, 0);
+        fence_proxy_async_smem();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t aW = smem_u32(sW), aQ = smem_u32(sQK), aK = smem_u32(sQK + kTileB), aBig = smem_u32(sBig);
+    constexpr int KS = HD / 16;  // k-steps over the head dimension
+    bool ok = true;
+    uint32_t r[32];
+    float v[32];
+
+    if (tid == 0) {
+        mbar_expect_tx(&bars[0], 3 * kT * HD * 2);
+        for (int h = 0; h < HD / 64; ++h) {
+            tma_load_2d(sW + h * kPanelB, &tm.w, &bars[0], h * 64, chunk * kT);
+            tma_load_2d(sQK + h * kPanelB, &tm.q, &bars[0], h * 64, chunk * kT);
+            tma_load_2d(sQK + kTileB + h * kPanelB, &tm.k, &bars[0], h * 64, chunk * kT);
+        }
+        if (!mbar_wait(&bars[0], 0, abort_flag, ST_PREP)) ok = false;
+        tc_fence_after_sync();
+        if (ok) {   // group 1: Gm -> col 0, Xq -> col 128, Xk -> col 256
+            mma(tmem + 0, aW, OP_K, aW, OP_K, KS, 128, false);
+            mma(tmem + 128, aQ, OP_K, aW, OP_K, KS, 128, false);
+            mma(tmem + 256, aW, OP_K, aK, OP_K, KS, 128, false);
+            umma_commit(&bars[1]);
+        }
+    }
+    if (!mbar_wait(&bars[1], 0, abort_flag, ST_PREP)) ok = false;
+    ok = __syncthreads_and(ok);
+    tc_fence_after_sync();
+    if (!ok) goto done;
+
+    // ---- E1: Gm -> strictLower(D Gm) in the float32 buffer
+    for (int c = 0; c < 2; ++c) {
+        const int c0 = half * 64 + c * 32;
+        tmem_ld32(tl + 0 + c0, r);
+        tmem_ld_wait();
+        const float b = bt[row];
+#pragma unroll
+        for (int x = 0; x < 32; ++x) {
+            v[x] = __uint_as_float(r[x]);
+            Xb[row * kLd + c0 + x] = (c0 + x < row) ? b * v[x] : 0.f;
+        }
+        if (SAVE) gstore_f32x32(p.Gm + grow * kT + c0, v);
+    }
+    __syncthreads();
+
+    // ---- (I + Nl)^-1 in place, 16-row panels
+    if (lane < 16) {   // diagonal blocks: warp w inverts block w, lane j owns column j
+        const int o = warp * 16, j = lane;
+        float* dx = diagX + warp * 16 * 17;
+        for (int rr = 0; rr < 16; ++rr) {
+            float acc = (rr == j) ? 1.f : 0.f;
+            for (int c = j; c < rr; ++c) acc -= Xb[(o + rr) * kLd + o + c] * dx[c * 17 + j];
+            dx[rr * 17 + j] = (rr >= j) ? acc : 0.f;
+        }
+    }
+    __syncthreads();
+    for (int bi = 0; bi < kT / 16; ++bi) {
+        const int R = bi * 16;
+        const float* dx = diagX + bi * 16 * 17;
+        if (bi > 0) {
+            for (int idx = tid; idx < 4 * R; idx += 256) {
+                const int rg = idx / R, c = idx - rg * R;
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+                const float* n0 = Xb + (R + rg) * kLd;
+                for (int k = (c & ~15); k < R; ++k) {
+                    const float x = Xb[k * kLd + c];
+                    a0 += n0[k] * x;
+                    a1 += n0[4 * kLd + k] * x;
+                    a2 += n0[8 * kLd + k] * x;
+                    a3 += n0[12 * kLd + k] * x;
+                }
+                Z[rg * kT + c] = a0; Z[(rg + 4) * kT + c] = a1; Z[(rg + 8) * kT + c] = a2; Z[(rg + 12) * kT + c] = a3;
+            }
+            __syncthreads();
+            for (int idx = tid; idx < 16 * R; idx += 256) {
+                const int rr = idx / R, c = idx - rr * R;
+                float acc = 0.f;
+                for (int k = 0; k <= rr; ++k) acc -= dx[rr * 17 + k] * Z[k * kT + c];
+                Xb[(R + rr) * kLd + c] = acc;
+            }
+        }
+        { const int rr = tid >> 4, k = tid & 15; Xb[(R + rr) * kLd + R + k] = dx[rr * 17 + k]; }
+        __syncthreads();
+    }
+
+    // ---- T~ = X D as a bf16 pair into the Q / K tiles' space (group 1 has finished with them)
+    for (int c = 0; c < 2; ++c) {
+        const int c0 = half * 64 + c * 32;
+        float hi[32], lo[32];
+#pragma unroll
+        for (int x = 0; x < 32; ++x) {
+            const float xv = Xb[row * kLd + c0 + x];
+            const float t = xv * bt[c0 + x];
+            v[x] = xv;
+            hi[x] = __bfloat162float(__float2bfloat16_rn(t));
+            lo[x] = t - hi[x];
+        }
+        if (SAVE) gstore_f32x32(p.Ai + grow * kT + c0, v);
+        tile_store32(sQK, row, c0, hi);
+        tile_store32(sQK + kTileB, row, c0, lo);
+        if (SAVE) {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) v[x] = hi[x] + lo[x];
+            gstore_f32x32(p.Tt + grow * kT + c0, v);
+        }
+    }
+    __syncthreads();  // everyone has read the float32 buffer; it now becomes the Xq / Xk tiles
+
+    // ---- E1b: Xq = lower(.), Xk = strictLower(.) -> bf16 tiles; Xqn = -Xq -> global
+    for (int c = 0; c < 2; ++c) {
+        const int c0 = half * 64 + c * 32;
+        tmem_ld32(tl + 128 + c0, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int x = 0; x < 32; ++x) v[x] = (c0 + x <= row) ? __uint_as_float(r[x]) : 0.f;
+        tile_store32(sBig, row, c0, v);
+        if (SAVE) gstore_f32x32(p.Xq + grow * kT + c0, v);
+#pragma unroll
+        for (int x = 0; x < 32; ++x) v[x] = -v[x];
+        gstore_bf16x32(p.Xqn + grow * kT + c0, v);
+        tmem_ld32(tl + 256 + c0, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int x = 0; x < 32; ++x) v[x] = (c0 + x < row) ? __uint_as_float(r[x]) : 0.f;
+        tile_store32(sBig + kTileB, row, c0, v);
+        if (SAVE) gstore_f32x32(p.Xk + grow * kT + c0, v);
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {   // group 2: U = T~ W -> col 0, Y = T~ Xk -> col 128
+        tc_fence_after_sync();
+        mma(tmem + 0, aQ, OP_K, aW, OP_MN, 8, HD, false);
+        mma(tmem + 0, aK, OP_K, aW, OP_MN, 8, HD, true);
+        mma(tmem + 128, aQ, OP_K, aBig + kTileB, OP_MN, 8, 128, false);
+        mma(tmem + 128, aK, OP_K, aBig + kTileB, OP_MN, 8, 128, true);
+        umma_commit(&bars[1]);
+    }
+    if (!mbar_wait(&bars[1], 1, abort_flag, ST_PREP)) ok = false;
+    ok = __syncthreads_and(ok);
+    tc_fence_after_sync();
+    if (!ok) goto done;
+
+    // ---- E2: U, Y -> bf16 tiles over T~ (dead now); Yt = Y^T -> global
+    for (int c = 0; c < HD / 64; ++c) {
+        const int c0 = half * (HD / 2) + c * 32;
+        tmem_ld32(tl + 0 + c0, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
+        tile_store32(sQK, row, c0, v);
+        if (SAVE) gstore_f32x32(p.U + grow * HD + c0, v);
+    }
+    for (int c = 0; c < 2; ++c) {
+        const int c0 = half * 64 + c * 32;
+        tmem_ld32(tl + 128 + c0, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
+        tile_store32(sQK + kTileB, row, c0, v);
+        if (SAVE) gstore_f32x32(p.Y + grow * kT + c0, v);
+        __nv_bfloat16* yt = p.Yt + ((size_t)chunk * kT + c0) * kT + row;
+#pragma unroll
+        for (int x = 0; x < 32; ++x) yt[(size_t)x * kT] = __float2bfloat16_rn(v[x]);
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {   // group 3: Xq U -> col 256, Y^T W -> col 384, W^T U -> col 0
+        tc_fence_after_sync();
+        mma(tmem + 256, aBig, OP_K, aQ, OP_MN, 8, HD, false);
+        mma(tmem + 384, aK, OP_MN, aW, OP_MN, 8, HD, false);
+        mma(tmem + 0, aW, OP_MN, aQ, OP_MN, 8, HD, false);
+        umma_commit(&bars[1]);
+    }
+    if (!mbar_wait(&bars[1], 0, abort_flag, ST_PREP)) ok = false;
+    ok = __syncthreads_and(ok);
+    tc_fence_after_sync();
+    if (!ok) goto done;
+
+    // ---- E3: Qleft = Q - Xq U, Kright = K - Y^T W, P = I - W^T U
+    for (int c = 0; c < HD / 64; ++c) {
+        const int c0 = half * (HD / 2) + c * 32;
+        float in[32];
+        tmem_ld32(tl + 256 + c0, r);
+        tmem_ld_wait();
+        gload_bf16x32(p.q + grow * HD + c0, in);
+#pragma unroll
+        for (int x = 0; x < 32; ++x) v[x] = in[x] - __uint_as_float(r[x]);
+        gstore_bf16x32(p.ql + grow * HD + c0, v);
+        tmem_ld32(tl + 384 + c0, r);
+        tmem_ld_wait();
+        gload_bf16x32(p.k + grow * HD + c0, in);
+#pragma unroll
+        for (int x = 0; x < 32; ++x) v[x] = in[x] - __uint_as_float(r[x]);
+        gstore_bf16x32(p.kr + grow * HD + c0, v);
+        tmem_ld32(tl + 0 + c0, r);
+        tmem_ld_wait();
+        if (row < HD) {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) v[x] = ((c0 + x == row) ? 1.f : 0.f) - __uint_as_float(r[x]);
+            gstore_f32x32(p.P + ((size_t)chunk * HD + row) * HD + c0, v);
+        }
+    }
+
+done:
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && *abort_flag != 0) atomicCAS(p.status, 0u, *abort_flag);
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_chunk_prep(const PrepTensorMaps& tm, const PrepParams& p, int hd, int save, int nchunks,
+                              cudaStream_t st) {
+    auto go = [&](auto kern) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PrepSmem::alloc);
+        if (e != cudaSuccess) return e;
+        kern<<<nchunks, 256, PrepSmem::alloc, st>>>(tm, p);
+        return cudaGetLastError();
+    };
+    if (hd == 64) return save ? go(chunk_prep_kernel<64, true>) : go(chunk_prep_kernel<64, false>);
+    return save ? go(chunk_prep_kernel<128, true>) : go(chunk_prep_kernel<128, false>);
+}
+
+}  // namespace path

@@ -15,6 +15,7 @@ enum : uint32_t {
     ST_FWD_PRODUCER = 0x101, ST_FWD_MMA = 0x102, ST_FWD_SOFTMAX = 0x103,
     ST_DKV_PRODUCER = 0x201, ST_DKV_MMA = 0x202, ST_DKV_COMPUTE = 0x203,
     ST_DQ_PRODUCER = 0x301, ST_DQ_MMA = 0x302, ST_DQ_COMPUTE = 0x303,
+    ST_PREP = 0x401,
 };
 
 __host__ __device__ inline int msb32(unsigned x) {
@@ -55,6 +56,27 @@ struct FwdParams {
     float scale;
     int out_fp32;
 };
+
+struct PrepTensorMaps {
+    CUtensorMap w, q, k;   // [S*Lp][d] bf16, box 128 rows x 64 columns, 128-byte swizzle
+};
+
+struct PrepParams {
+    const float* beta;            // [S*Lp] (zero in the ragged tail)
+    const __nv_bfloat16* q;       // [S*Lp][d]
+    const __nv_bfloat16* k;
+    __nv_bfloat16* ql;            // [S*Lp][d]   boundary-adjusted queries (version slot 0)
+    __nv_bfloat16* kr;            // [S*Lp][d]   boundary-adjusted keys (version slot 0)
+    __nv_bfloat16* Xqn;           // [S*Lp][128] -lower(Q W^T)
+    __nv_bfloat16* Yt;            // [S*Lp][128] (T~ strictLower(W K^T))^T
+    float* P;                     // [S*N][d][d] chunk products
+    float *Gm, *Ai, *Tt, *Xq, *Xk, *Y;   // [S*N][128][128], written only by the backward's instance
+    float* U;                     // [S*Lp][d], likewise
+    uint32_t* status;
+};
+
+cudaError_t launch_chunk_prep(const PrepTensorMaps& tm, const PrepParams& p, int hd, int save, int nchunks,
+                              cudaStream_t st);
 
 struct BwdTensorMaps {
     CUtensorMap q_raw, k_raw, v, qv, kv, xqn, yt, d_o;

@@ -110,25 +110,23 @@ __device__ __forceinline__ bool resolve(GemmProblem& g, const VersionBatch& v, i
     g.D = nullptr; g.C2 = nullptr; g.c_f32 = 1; g.c2_trans = 0;
     r.D = nullptr; r.C2 = nullptr; r.c2_rows = 1 << 30;
     if (v.mode == 0 || v.mode == 1) {
-        const float* a = (v.mode == 0) ? v.xv + row_src * d : v.dxv + row_dst * d;
-        r.A = Operand{a, d, 1, 1};
+        r.A = (v.mode == 0) ? Operand{v.xv + row_src * d, d, 1, 0} : Operand{v.dxv + row_dst * d, d, 1, 1};
         r.B = dy_transposed ? Operand{v.dy + dy_idx, d, 1, 1} : Operand{v.dy + dy_idx, 1, d, 1};
         r.M = CHUNK; r.N = (int)d; r.K = (int)d;
         g.ldc = d;
         if (v.mode == 0) {
-            r.C = v.out32 + row_dst * d;
-            r.C2 = v.out16 + row_dst * d;
-            g.C2 = r.C2; g.ldc2 = d;
+            r.C = v.out16 + row_dst * d;
+            g.c_f32 = 0;
             g.accumulate = ACC_NONE;
         } else {
             r.C = v.dxv + row_src * d;
             g.accumulate = ACC_ADD;
         }
     } else {
-        const float* x = v.xv + row_src * d;
+        const __nv_bfloat16* x = v.xv + row_src * d;
         const float* gup = v.dxv + row_dst * d;
-        if (!v.is_key) { r.A = Operand{x, 1, d, 1}; r.B = Operand{gup, 1, d, 1}; }
-        else           { r.A = Operand{gup, 1, d, 1}; r.B = Operand{x, 1, d, 1}; }
+        if (!v.is_key) { r.A = Operand{x, 1, d, 0}; r.B = Operand{gup, 1, d, 1}; }
+        else           { r.A = Operand{gup, 1, d, 1}; r.B = Operand{x, 1, d, 0}; }
         r.M = (int)d; r.N = (int)d; r.K = CHUNK;
         r.C = v.ddy + dy_idx;
         g.ldc = d;

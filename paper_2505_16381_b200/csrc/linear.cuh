@@ -56,12 +56,11 @@ struct LevelTable {
 struct VersionBatch {
     int is_key, mode, l2, S, N, Lp, d;
     LevelTable lv;
-    const float* xv;   // [slots][S][Lp][d] float versions
-    float* dxv;        // gradients, same layout (modes 1, 2)
-    const float* dy;   // dyadic run products
-    float* ddy;        // their gradients (mode 2)
-    float* out32;      // mode 0: float versions (same buffer as xv)
-    __nv_bfloat16* out16;  // mode 0: bf16 versions for the attention kernel
+    const __nv_bfloat16* xv;  // [slots][S][Lp][d] bf16 versions (what the attention kernels consume)
+    float* dxv;               // float gradients, same layout (modes 1, 2)
+    const float* dy;          // dyadic run products
+    float* ddy;               // their gradients (mode 2)
+    __nv_bfloat16* out16;     // mode 0: destination (same buffer as xv)
 };
 
 cudaError_t launch_gemm(const GemmProblem& g, const AffineBatch& b, int nbatch, cudaStream_t st);

@@ -84,7 +84,7 @@ struct Plan {
     LevelTable lv;
     size_t total;
     // offsets (bytes)
-    size_t status, qp, kp, vp, wp, betap, G, Gm, Ai, Tt, U, Dy, Xq, Xk, Y, Xqn, Yt, Qv32, Kv32, Qv16, Kv16;
+    size_t status, qp, kp, vp, wp, betap, G, Gm, Ai, Tt, U, Dy, Xq, Xk, Y, Xqn, Yt, Qv16, Kv16;
     // backward only
     size_t dop, delta, lse2, dQv, dKv, dSd, dG, dGrow, dGdiag, dDy, dXq, dY, dT, dXk, tmpBB, dA, dU, tq, tk, tw, t1;
     size_t dy_bytes;
@@ -115,10 +115,11 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
     }
     p.betap = bump(cur, SL * 4);
     if (gate) p.G = bump(cur, SL * 4);
-    p.Gm = bump(cur, SNBB * 4);
-    p.Ai = bump(cur, bwd ? SNBB * 4 : 0);
-    p.Tt = bump(cur, SNBB * 4);
-    p.U = bump(cur, SLd * 4);
+    const size_t keep = bwd ? 1 : 0;   // float intermediates of the chunk preparation, kept for the chain rule
+    p.Gm = bump(cur, keep * SNBB * 4);
+    p.Ai = bump(cur, keep * SNBB * 4);
+    p.Tt = bump(cur, keep * SNBB * 4);
+    p.U = bump(cur, keep * SLd * 4);
     size_t dy_elems = 0;
     for (int l = 0; l < 20; ++l) {
         p.lv.dy_off[l] = (long)dy_elems;
@@ -126,13 +127,11 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
         if (l == 0 || l <= p.nlev - 2) dy_elems += (size_t)S * (p.N >> l) * d * d;
     }
     p.Dy = bump(cur, dy_elems * 4);
-    p.Xq = bump(cur, SNBB * 4);
-    p.Xk = bump(cur, SNBB * 4);
-    p.Y = bump(cur, SNBB * 4);
+    p.Xq = bump(cur, keep * SNBB * 4);
+    p.Xk = bump(cur, keep * SNBB * 4);
+    p.Y = bump(cur, keep * SNBB * 4);
     p.Xqn = bump(cur, SL * CHUNK * 2);
     p.Yt = bump(cur, SL * CHUNK * 2);
-    p.Qv32 = bump(cur, SLd * 4 * p.nslot);
-    p.Kv32 = bump(cur, SLd * 4 * p.nslot);
     p.Qv16 = bump(cur, SLd * 2 * p.nslot);
     p.Kv16 = bump(cur, SLd * 2 * p.nslot);
     p.dy_bytes = dy_elems * 4;
@@ -166,70 +165,31 @@ static AffineBatch chunk_batch(const Plan& p, long a, long b, long c, long c2, l
 // Chunk preparation + dyadic run products + version chains (paper Sec. 3.1, 3.3).  Shared by forward and backward.
 static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const void* w, cudaStream_t st) {
     const int d = p.d, nch = p.S * p.N;
-    const long Bd = (long)CHUNK * d, BB = (long)CHUNK * CHUNK, dd = (long)d * d;
-    float* Gm = at<float>(ws, p.Gm); float* Tt = at<float>(ws, p.Tt); float* U = at<float>(ws, p.U);
-    float* Ai = p.bwd ? at<float>(ws, p.Ai) : nullptr;
-    float* Dy = at<float>(ws, p.Dy); float* Xq = at<float>(ws, p.Xq); float* Xk = at<float>(ws, p.Xk);
-    float* Y = at<float>(ws, p.Y);
-    __nv_bfloat16* Xqn = at<__nv_bfloat16>(ws, p.Xqn); __nv_bfloat16* Yt = at<__nv_bfloat16>(ws, p.Yt);
-    float* Qv32 = at<float>(ws, p.Qv32); float* Kv32 = at<float>(ws, p.Kv32);
+    const long dd = (long)d * d;
+    float* Dy = at<float>(ws, p.Dy);
     __nv_bfloat16* Qv16 = at<__nv_bfloat16>(ws, p.Qv16); __nv_bfloat16* Kv16 = at<__nv_bfloat16>(ws, p.Kv16);
-    const float* betap = at<float>(ws, p.betap);
 
-    // Gm = W W^T
+    // fused per-chunk kernel: UT transform, boundary-adjusted tiles (version slot 0), chunk products (Dy level 0)
     {
-        GemmProblem g = gemm_problem(Operand{w, d, 1, 0}, Operand{w, d, 1, 0}, CHUNK, CHUNK, d);
-        g.C = Gm; g.c_f32 = 1; g.ldc = CHUNK;
-        LAUNCH(launch_gemm(g, chunk_batch(p, Bd, Bd, BB, 0, 0), nch, st));
-    }
-    LAUNCH(launch_tri_inverse(Gm, betap, Ai, Tt, nch, st));
-    // U = T~ W
-    {
-        GemmProblem g = gemm_problem(Operand{Tt, CHUNK, 1, 1}, Operand{w, 1, d, 0}, CHUNK, d, CHUNK);
-        g.C = U; g.c_f32 = 1; g.ldc = d;
-        LAUNCH(launch_gemm(g, chunk_batch(p, BB, Bd, Bd, 0, 0), nch, st));
-    }
-    // P = I - W^T U  -> Dy level 0
-    {
-        GemmProblem g = gemm_problem(Operand{w, 1, d, 0}, Operand{U, 1, d, 1}, d, d, CHUNK);
-        g.C = Dy; g.c_f32 = 1; g.ldc = d; g.alpha = -1.f; g.identity = 1;
-        LAUNCH(launch_gemm(g, chunk_batch(p, Bd, Bd, dd, 0, 0), nch, st));
-    }
-    // Xq = lower(Q W^T); Xqn = -Xq (bf16, A operand of the diagonal correction)
-    {
-        GemmProblem g = gemm_problem(Operand{q, d, 1, 0}, Operand{w, d, 1, 0}, CHUNK, CHUNK, d);
-        g.C = Xq; g.c_f32 = 1; g.ldc = CHUNK; g.mask = MASK_LOWER;
-        g.C2 = Xqn; g.ldc2 = CHUNK; g.alpha2 = -1.f;
-        LAUNCH(launch_gemm(g, chunk_batch(p, Bd, Bd, BB, BB, 0), nch, st));
-    }
-    // Qleft = Q - Xq U  -> version slot 0
-    {
-        GemmProblem g = gemm_problem(Operand{Xq, CHUNK, 1, 1}, Operand{U, 1, d, 1}, CHUNK, d, CHUNK);
-        g.C = Qv32; g.c_f32 = 1; g.ldc = d; g.alpha = -1.f;
-        g.D = q; g.d_f32 = 0; g.ldd = d;
-        g.C2 = Qv16; g.ldc2 = d;
-        LAUNCH(launch_gemm(g, chunk_batch(p, BB, Bd, Bd, Bd, Bd), nch, st));
-    }
-    // Xk = strictLower(W K^T)
-    {
-        GemmProblem g = gemm_problem(Operand{w, d, 1, 0}, Operand{k, d, 1, 0}, CHUNK, CHUNK, d);
-        g.C = Xk; g.c_f32 = 1; g.ldc = CHUNK; g.mask = MASK_STRICT;
-        LAUNCH(launch_gemm(g, chunk_batch(p, Bd, Bd, BB, 0, 0), nch, st));
-    }
-    // Y = T~ Xk; Yt = Y^T (bf16, B operand of the diagonal correction)
-    {
-        GemmProblem g = gemm_problem(Operand{Tt, CHUNK, 1, 1}, Operand{Xk, 1, CHUNK, 1}, CHUNK, CHUNK, CHUNK);
-        g.C = Y; g.c_f32 = 1; g.ldc = CHUNK;
-        g.C2 = Yt; g.ldc2 = CHUNK; g.c2_trans = 1;
-        LAUNCH(launch_gemm(g, chunk_batch(p, BB, BB, BB, BB, 0), nch, st));
-    }
-    // Kright = K - Y^T W  -> version slot 0
-    {
-        GemmProblem g = gemm_problem(Operand{Y, 1, CHUNK, 1}, Operand{w, 1, d, 0}, CHUNK, d, CHUNK);
-        g.C = Kv32; g.c_f32 = 1; g.ldc = d; g.alpha = -1.f;
-        g.D = k; g.d_f32 = 0; g.ldd = d;
-        g.C2 = Kv16; g.ldc2 = d;
-        LAUNCH(launch_gemm(g, chunk_batch(p, BB, Bd, Bd, Bd, Bd), nch, st));
+        PrepTensorMaps tm;
+        const uint64_t rows = (uint64_t)p.S * p.Lp;
+        if (!(make_map(&tm.w, w, rows, d) && make_map(&tm.q, q, rows, d) && make_map(&tm.k, k, rows, d))) {
+            g_last_cuda_error = (int)cudaErrorUnknown;
+            return PATH_ERR_LAUNCH;
+        }
+        PrepParams pp{};
+        pp.beta = at<float>(ws, p.betap);
+        pp.q = (const __nv_bfloat16*)q; pp.k = (const __nv_bfloat16*)k;
+        pp.ql = Qv16; pp.kr = Kv16;
+        pp.Xqn = at<__nv_bfloat16>(ws, p.Xqn); pp.Yt = at<__nv_bfloat16>(ws, p.Yt);
+        pp.P = Dy;
+        if (p.bwd) {
+            pp.Gm = at<float>(ws, p.Gm); pp.Ai = at<float>(ws, p.Ai); pp.Tt = at<float>(ws, p.Tt);
+            pp.Xq = at<float>(ws, p.Xq); pp.Xk = at<float>(ws, p.Xk); pp.Y = at<float>(ws, p.Y);
+            pp.U = at<float>(ws, p.U);
+        }
+        pp.status = at<uint32_t>(ws, p.status);
+        LAUNCH(launch_chunk_prep(tm, pp, d, p.bwd, nch, st));
     }
     // dyadic run products Dy[l+1][b] = Dy[l][2b+1] Dy[l][2b]
     for (int l = 0; l + 1 <= p.nlev - 2; ++l) {
@@ -248,7 +208,7 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
         for (int is_key = 0; is_key < 2; ++is_key) {
             VersionBatch v{};
             v.is_key = is_key; v.mode = 0; v.l2 = l2; v.S = p.S; v.N = p.N; v.Lp = p.Lp; v.d = d; v.lv = p.lv;
-            v.xv = is_key ? Kv32 : Qv32; v.out32 = is_key ? Kv32 : Qv32; v.out16 = is_key ? Kv16 : Qv16;
+            v.xv = is_key ? Kv16 : Qv16; v.out16 = is_key ? Kv16 : Qv16;
             v.dy = Dy;
             LAUNCH(launch_gemm_version(v, st));
         }
@@ -414,7 +374,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
                 VersionBatch vb{};
                 vb.is_key = is_key; vb.mode = mode; vb.l2 = l2; vb.S = p.S; vb.N = p.N; vb.Lp = p.Lp; vb.d = d;
                 vb.lv = p.lv;
-                vb.xv = is_key ? at<float>(ws, p.Kv32) : at<float>(ws, p.Qv32);
+                vb.xv = is_key ? at<__nv_bfloat16>(ws, p.Kv16) : at<__nv_bfloat16>(ws, p.Qv16);
                 vb.dxv = is_key ? dKv : dQv;
                 vb.dy = Dy; vb.ddy = dDy;
                 LAUNCH(launch_gemm_version(vb, st));
