@@ -1,0 +1,320 @@
+// Per-chunk chain rule of the backward pass (the paper gives no backward): from the gradients of the
+// boundary-adjusted tiles (dQl, dKr), of the diagonal-chunk logits (dSd) and of the chunk product (dP) back through
+// the UT transform to dq, dk, dw, dbeta.  With Xq = lower(Q W^T), Xk = strictLower(W K^T), Y = T~ Xk, U = T~ W,
+// T~ = Ainv D, Ainv = (I + strictLower(D W W^T))^-1 and s = scale:
+//   dXq = lower(-dQl U^T - s dSd Y^T)            dY  = -W dKr^T - s Xq^T dSd           dU = -Xq^T dQl - W dP
+//   dT  = lower(dY Xk^T + dU W^T)                dXk = strictLower(T~^T dY)
+//   M   = Ainv^T dT,   dbeta_c  = M_cc,          dA  = strictLower(-(M D) Ainv^T)
+//   dbeta_r += sum_c dA_rc (W W^T)_rc,           dGm = D dA
+//   dq = dQl + s dSd K + dXq W                   dk = dKr + s dSd^T Q + dXk^T W
+//   dw = -Y dKr - U dP^T + T~^T dU + dXq^T Q + dXk K + (dGm + dGm^T) W
+// One CTA per chunk runs these ~25 products as tcgen05 MMAs on swizzled shared-memory tiles, in lockstep:
+// thread 0 loads tiles (TMA) and issues MMAs, all 256 threads convert float gradients into tiles and turn
+// accumulators (tensor memory, one row per thread) into the next operand tiles.  T~ and Ainv enter as bf16
+// hi + lo pairs, everything else is rounded to bf16 once; dw accumulates in tensor memory across all phases.
+#include "tileops.cuh"
+
+namespace path {
+using namespace tile;
+
+namespace {
+
+constexpr int kSlots = 7;
+constexpr uint32_t kBarOff = kSlots * kTileB;
+constexpr uint32_t kChainSmem = kBarOff + 64 + kT * 4 + kT * 4 + 1024;
+
+template <int HD>
+__global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_constant__ ChainTensorMaps tm,
+                                                             const ChainParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = (uint64_t*)(smem + kBarOff);  // [0] loads, [1] MMA groups
+    uint32_t* tmem_slot = (uint32_t*)(bars + 2);
+    volatile uint32_t* abort_flag = (volatile uint32_t*)(tmem_slot + 1);
+    float* bt = (float*)(smem + kBarOff + 64);
+    float* t1 = bt + kT;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int chunk = blockIdx.x;
+    const int row = (warp & 3) * 32 + lane, half = warp >> 2;
+    const size_t grow = (size_t)chunk * kT + row;
+    const int s_idx = chunk / p.N, pos = (chunk % p.N) * kT + row;   // slice and position of this thread's row
+    const bool row_valid = pos < p.L;
+    const size_t urow = (size_t)s_idx * p.L + pos;                   // row in the caller's [S][L][.] tensors
+
+    if (tid == 0) {
+        mbar_init(&bars[0], 1);
+        mbar_init(&bars[1], 1);
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    if (warp == 0) tmem_alloc(tmem_slot, 512);
+    if (tid < kT) bt[tid] = p.beta[(size_t)chunk * kT + tid];
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    auto slot = [&](int i) { return smem + i * kTileB; };
+    auto sa = [&](int i) { return smem_u32(smem + i * kTileB); };
+    constexpr int KD = HD / 16, K8 = 8;
+    constexpr uint32_t cDW = 0, cA = 128, cB = 256, cG = 384;   // tensor-memory columns: dw, two work accumulators, W W^T
+    bool ok = true;
+    uint32_t ph_load = 0, ph_mma = 0;
+    float v[32];
+
+    // thread 0: start TMA loads of bf16 tiles; everyone: wait for them
+    auto loads_wait = [&]() {
+        if (!mbar_wait(&bars[0], ph_load, abort_flag, ST_CHAIN)) ok = false;
+        ph_load ^= 1;
+    };
+    // everyone: tiles written by threads become visible to the MMA unit, accumulator reads are ordered
+    auto publish = [&]() {
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        __syncthreads();
+    };
+    auto mma_wait = [&]() {
+        __syncwarp();
+        if (!mbar_wait(&bars[1], ph_mma, abort_flag, ST_CHAIN)) ok = false;
+        ph_mma ^= 1;
+        ok = __syncthreads_and(ok);
+        tc_fence_after_sync();
+    };
+    // float rows of a [128][ncols] global matrix -> bf16 tile (optionally scaled)
+    auto conv = [&](const float* src, int ncols, int nrows, uint8_t* dst, float mul) {
+        const int per = ncols / 2;
+        for (int c = 0; c < per / 32; ++c) {
+            const int c0 = half * per + c * 32;
+            if (row < nrows) {
+                gload_f32x32(src + (size_t)row * ncols + c0, v);
+#pragma unroll
+                for (int x = 0; x < 32; ++x) v[x] *= mul;
+            } else {
+#pragma unroll
+                for (int x = 0; x < 32; ++x) v[x] = 0.f;
+            }
+            tile_store32(dst, row, c0, v);
+        }
+    };
+    // accumulator [128][ncols] -> f(row values) -> bf16 tile
+    enum { M_NONE = 0, M_LOWER = 1, M_STRICT = 2 };
+    auto acc_to_tile = [&](uint32_t col, int ncols, uint8_t* dst, float mul, int mask) {
+        const int per = ncols / 2;
+        for (int c = 0; c < per / 32; ++c) {
+            const int c0 = half * per + c * 32;
+            tmem_row32(tl + col + c0, v);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+                const bool keep = mask == M_NONE || (mask == M_LOWER ? (c0 + x <= row) : (c0 + x < row));
+                v[x] = keep ? v[x] * mul : 0.f;
+            }
+            tile_store32(dst, row, c0, v);
+        }
+    };
+
+    const float* g_dql = p.dql + (size_t)chunk * kT * HD;
+    const float* g_dkr = p.dkr + (size_t)chunk * kT * HD;
+    const float* g_dsd = p.dsd + (size_t)chunk * kT * kT;
+    const float* g_dp = p.dp + (size_t)chunk * HD * HD;
+    const int r0 = chunk * kT;
+
+    // slots: 0 U->W   1 dQl->dT->tmp->dGm   2 Y->Xq->Xk->T->Ah   3 dSd   4 dXq   5 dKr->dY->dXk   6 dP->dU->Al..K/Q
+    // ---- phase 0a: dXq = lower(-(dQl U^T + s dSd Y^T))
+    if (tid == 0) {
+        mbar_expect_tx(&bars[0], kT * HD * 2 + kTileB);
+        tma_tile(slot(0), &tm.u, &bars[0], HD, r0);
+        tma_tile(slot(2), &tm.y, &bars[0], kT, r0);
+    }
+    conv(g_dql, HD, kT, slot(1), 1.f);
+    conv(g_dsd, kT, kT, slot(3), p.scale);
+    conv(g_dkr, HD, kT, slot(5), 1.f);
+    conv(g_dp, HD, HD, slot(6), 1.f);
+    loads_wait();
+    publish();
+    if (tid == 0) {
+        tc_fence_after_sync();
+        mma(tmem + cA, sa(1), OP_K, sa(0), OP_K, KD, 128, false);
+        mma(tmem + cA, sa(3), OP_K, sa(2), OP_K, K8, 128, true);
+        // phase 0b: dw = -Y dKr - U dP^T
+        mma(tmem + cDW, sa(2), OP_K, sa(5), OP_MN, K8, HD, false, true);
+        mma(tmem + cDW, sa(0), OP_K, sa(6), OP_K, KD, HD, true, true);
+        umma_commit(&bars[1]);
+    }
+    mma_wait();
+    if (!ok) goto done;
+    acc_to_tile(cA, kT, slot(4), -1.f, M_LOWER);                    // dXq
+    // ---- phase 1: dY = -(W dKr^T + Xq^T s dSd),  dU = -(Xq^T dQl + W dP),  Gm = W W^T
+    if (tid == 0) {
+        mbar_expect_tx(&bars[0], kT * HD * 2 + kTileB);
+        tma_tile(slot(0), &tm.w, &bars[0], HD, r0);
+        tma_tile(slot(2), &tm.xq, &bars[0], kT, r0);
+    }
+    loads_wait();
+    publish();
+    if (tid == 0) {
+        tc_fence_after_sync();
+        mma(tmem + cA, sa(0), OP_K, sa(5), OP_K, KD, 128, false);
+        mma(tmem + cA, sa(2), OP_MN, sa(3), OP_MN, K8, 128, true);
+        mma(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, HD, false);
+        mma(tmem + cB, sa(0), OP_K, sa(6), OP_MN, KD, HD, true);
+        mma(tmem + cG, sa(0), OP_K, sa(0), OP_K, KD, 128, false);
+        umma_commit(&bars[1]);
+    }
+    mma_wait();
+    if (!ok) goto done;
+    acc_to_tile(cA, kT, slot(5), -1.f, M_NONE);                     // dY (over dKr)
+    acc_to_tile(cB, HD, slot(6), -1.f, M_NONE);                     // dU (over dP)
+    // ---- phase 2: dT = lower(dY Xk^T + dU W^T)
+    if (tid == 0) {
+        mbar_expect_tx(&bars[0], kTileB);
+        tma_tile(slot(2), &tm.xk, &bars[0], kT, r0);
+    }
+    loads_wait();
+    publish();
+    if (tid == 0) {
+        tc_fence_after_sync();
+        mma(tmem + cA, sa(5), OP_K, sa(2), OP_K, K8, 128, false);
+        mma(tmem + cA, sa(6), OP_K, sa(0), OP_K, KD, 128, true);
+        umma_commit(&bars[1]);
+    }
+    mma_wait();
+    if (!ok) goto done;
+    acc_to_tile(cA, kT, slot(1), 1.f, M_LOWER);                     // dT (over dQl)
+    // ---- phase 3: dXk = strictLower(T~^T dY),  dw += T~^T dU   (hi, then lo through the same slot)
+    for (int part = 0; part < 2; ++part) {
+        if (tid == 0) {
+            mbar_expect_tx(&bars[0], kTileB);
+            tma_tile(slot(2), part == 0 ? &tm.th : &tm.tl, &bars[0], kT, r0);
+        }
+        loads_wait();
+        publish();
+        if (tid == 0) {
+            tc_fence_after_sync();
+            mma(tmem + cA, sa(2), OP_MN, sa(5), OP_MN, K8, 128, part > 0);
+            mma(tmem + cDW, sa(2), OP_MN, sa(6), OP_MN, K8, HD, true);
+            umma_commit(&bars[1]);
+        }
+        mma_wait();
+        if (!ok) goto done;
+    }
+    // ---- phase 4: M = Ainv^T dT;  dbeta_c = M_cc;  tmp = M D;  dA = strictLower(-tmp Ainv^T)
+    if (tid == 0) {
+        mbar_expect_tx(&bars[0], 2 * kTileB);
+        tma_tile(slot(2), &tm.ah, &bars[0], kT, r0);
+        tma_tile(slot(6), &tm.al, &bars[0], kT, r0);
+    }
+    acc_to_tile(cA, kT, slot(5), 1.f, M_STRICT);                    // dXk (over dY)
+    loads_wait();
+    publish();
+    if (tid == 0) {
+        tc_fence_after_sync();
+        mma(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, 128, false);
+        mma(tmem + cB, sa(6), OP_MN, sa(1), OP_MN, K8, 128, true);
+        umma_commit(&bars[1]);
+    }
+    mma_wait();
+    if (!ok) goto done;
+    for (int c = 0; c < 2; ++c) {                                   // tmp = M D (over dT), diagonal -> t1
+        const int c0 = half * 64 + c * 32;
+        tmem_row32(tl + cB + c0, v);
+#pragma unroll
+        for (int x = 0; x < 32; ++x) {
+            if (c0 + x == row) t1[row] = v[x];
+            v[x] *= bt[c0 + x];
+        }
+        tile_store32(slot(1), row, c0, v);
+    }
+    publish();
+    if (tid == 0) {
+        tc_fence_after_sync();
+        mma(tmem + cA, sa(1), OP_K, sa(2), OP_K, K8, 128, false);
+        mma(tmem + cA, sa(1), OP_K, sa(6), OP_K, K8, 128, true);
+        umma_commit(&bars[1]);
+    }
+    mma_wait();
+    if (!ok) goto done;
+    {   // dA = strictLower(-acc);  dbeta_r = t1_r + sum_c dA_rc Gm_rc;  dGm = D dA -> tile (over tmp)
+        float part = 0.f;
+        const float b = bt[row];
+        for (int c = 0; c < 2; ++c) {
+            const int c0 = half * 64 + c * 32;
+            float gm[32];
+            tmem_row32(tl + cA + c0, v);
+            tmem_row32(tl + cG + c0, gm);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+                const float da = (c0 + x < row) ? -v[x] : 0.f;
+                part += da * gm[x];
+                v[x] = b * da;
+            }
+            tile_store32(slot(1), row, c0, v);
+        }
+        // the two threads of a row add their halves through shared memory
+        __syncthreads();
+        if (half == 1) t1[row] += part;
+        __syncthreads();
+        if (half == 0 && row_valid) p.dbeta[urow] = t1[row] + part;
+    }
+    // ---- phase 5: dq, dk and the rest of dw
+    if (tid == 0) {
+        mbar_expect_tx(&bars[0], 2 * kT * HD * 2);
+        tma_tile(slot(2), &tm.k, &bars[0], HD, r0);
+        tma_tile(slot(6), &tm.q, &bars[0], HD, r0);
+    }
+    loads_wait();
+    publish();
+    if (tid == 0) {
+        tc_fence_after_sync();
+        mma(tmem + cA, sa(3), OP_K, sa(2), OP_MN, K8, HD, false);    // s dSd K
+        mma(tmem + cA, sa(4), OP_K, sa(0), OP_MN, K8, HD, true);     // dXq W
+        mma(tmem + cB, sa(3), OP_MN, sa(6), OP_MN, K8, HD, false);   // s dSd^T Q
+        mma(tmem + cB, sa(5), OP_MN, sa(0), OP_MN, K8, HD, true);    // dXk^T W
+        mma(tmem + cDW, sa(4), OP_MN, sa(6), OP_MN, K8, HD, true);   // dXq^T Q
+        mma(tmem + cDW, sa(5), OP_K, sa(2), OP_MN, K8, HD, true);    // dXk K
+        mma(tmem + cDW, sa(1), OP_K, sa(0), OP_MN, K8, HD, true);    // dGm W
+        mma(tmem + cDW, sa(1), OP_MN, sa(0), OP_MN, K8, HD, true);   // dGm^T W
+        umma_commit(&bars[1]);
+    }
+    mma_wait();
+    if (!ok) goto done;
+    for (int c = 0; c < HD / 64; ++c) {
+        const int c0 = half * (HD / 2) + c * 32;
+        float in[32];
+        tmem_row32(tl + cA + c0, v);
+        gload_f32x32(g_dql + (size_t)row * HD + c0, in);
+#pragma unroll
+        for (int x = 0; x < 32; ++x) v[x] += in[x];
+        if (row_valid) gstore_bf16x32(p.dq + urow * HD + c0, v);
+        tmem_row32(tl + cB + c0, v);
+        gload_f32x32(g_dkr + (size_t)row * HD + c0, in);
+#pragma unroll
+        for (int x = 0; x < 32; ++x) v[x] += in[x];
+        if (row_valid) gstore_bf16x32(p.dk + urow * HD + c0, v);
+        tmem_row32(tl + cDW + c0, v);
+        if (row_valid) gstore_bf16x32(p.dw + urow * HD + c0, v);
+    }
+
+done:
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && *abort_flag != 0) atomicCAS(p.status, 0u, *abort_flag);
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_chunk_chain(const ChainTensorMaps& tm, const ChainParams& p, int hd, int nchunks, cudaStream_t st) {
+    auto go = [&](auto kern) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kChainSmem);
+        if (e != cudaSuccess) return e;
+        kern<<<nchunks, 256, kChainSmem, st>>>(tm, p);
+        return cudaGetLastError();
+    };
+    return hd == 64 ? go(chunk_chain_kernel<64>) : go(chunk_chain_kernel<128>);
+}
+
+}  // namespace path

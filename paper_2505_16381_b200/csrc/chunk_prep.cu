@@ -13,16 +13,14 @@
 // the descriptor's major-ness, so nothing is ever transposed in memory.  Accumulators live in tensor memory and
 // are read back one row per thread.  T~ is kept as a bf16 pair (hi + lo) because everything downstream
 // depends on it; the other intermediates are rounded to bf16 once, like the tiles the attention sweep consumes.
-#include "common.cuh"
-#include "tc5.cuh"
+#include "tileops.cuh"
 
 namespace path {
 using namespace tc5;
 
 namespace {
 
-constexpr int kT = 128;
-constexpr uint32_t kTileB = 32768, kPanelB = 16384;
+using namespace tile;
 constexpr int kLd = kT + 1;  // row stride of the float32 triangular buffer
 
 struct PrepSmem {
@@ -37,58 +35,6 @@ struct PrepSmem {
     static constexpr uint32_t total = offBar + 64;
     static constexpr uint32_t alloc = total + 1024;
 };
-
-// K-major view: contraction over the tile's columns.  MN-major view: contraction over the tile's rows.
-__device__ __forceinline__ uint64_t desc_k(uint32_t tile, int kk) {
-    return umma_desc(tile + (kk >> 2) * kPanelB + (kk & 3) * 32, 16, 1024);
-}
-__device__ __forceinline__ uint64_t desc_mn(uint32_t tile, int kk) { return umma_desc(tile + kk * 2048, kPanelB, 1024); }
-
-enum { OP_K = 0, OP_MN = 1 };
-// D (+)= op(A) op(B) over `ksteps` steps of 16.
-__device__ __forceinline__ void mma(uint32_t d_tmem, uint32_t a_tile, int a_op, uint32_t b_tile, int b_op, int ksteps,
-                                    int n, bool acc) {
-    const uint32_t idesc = umma_idesc(128, n, a_op, b_op);
-    for (int kk = 0; kk < ksteps; ++kk)
-        umma_ss(d_tmem, a_op == OP_K ? desc_k(a_tile, kk) : desc_mn(a_tile, kk),
-                b_op == OP_K ? desc_k(b_tile, kk) : desc_mn(b_tile, kk), idesc, (acc || kk > 0) ? 1u : 0u);
-}
-
-// Stores 32 consecutive columns (c0 .. c0+31) of `row` of a row-major swizzled bf16 tile.
-__device__ __forceinline__ void tile_store32(uint8_t* tile, int row, int c0, const float (&v)[32]) {
-    uint8_t* panel = tile + (c0 >> 6) * kPanelB;
-    const int ch0 = (c0 & 63) >> 3;
-#pragma unroll
-    for (int ch = 0; ch < 4; ++ch)
-        *reinterpret_cast<uint4*>(panel + sw128_off((uint32_t)row, (uint32_t)(ch0 + ch))) =
-            make_uint4(pack_bf16(v[8 * ch], v[8 * ch + 1]), pack_bf16(v[8 * ch + 2], v[8 * ch + 3]),
-                       pack_bf16(v[8 * ch + 4], v[8 * ch + 5]), pack_bf16(v[8 * ch + 6], v[8 * ch + 7]));
-}
-__device__ __forceinline__ void gstore_f32x32(float* dst, const float (&v)[32]) {
-#pragma unroll
-    for (int x = 0; x < 8; ++x)
-        reinterpret_cast<float4*>(dst)[x] = make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
-}
-__device__ __forceinline__ void gstore_bf16x32(__nv_bfloat16* dst, const float (&v)[32]) {
-#pragma unroll
-    for (int x = 0; x < 4; ++x)
-        reinterpret_cast<uint4*>(dst)[x] =
-            make_uint4(pack_bf16(v[8 * x], v[8 * x + 1]), pack_bf16(v[8 * x + 2], v[8 * x + 3]),
-                       pack_bf16(v[8 * x + 4], v[8 * x + 5]), pack_bf16(v[8 * x + 6], v[8 * x + 7]));
-}
-__device__ __forceinline__ void gload_bf16x32(const __nv_bfloat16* src, float (&v)[32]) {
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-        const uint4 u = reinterpret_cast<const uint4*>(src)[x];
-        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-        for (int y = 0; y < 4; ++y) {
-            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[y]));
-            v[8 * x + 2 * y] = f.x;
-            v[8 * x + 2 * y + 1] = f.y;
-        }
-    }
-}
 
 template <int HD, bool SAVE>
 __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constant__ PrepTensorMaps tm, const PrepParams p) {
@@ -150,6 +96,7 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
             umma_commit(&bars[1]);
         }
     }
+    __syncwarp();  // lanes 1-31 of the issuing warp block here instead of spinning against lane 0
     if (!mbar_wait(&bars[1], 0, abort_flag, ST_PREP)) ok = false;
     ok = __syncthreads_and(ok);
     tc_fence_after_sync();
@@ -166,7 +113,6 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
             v[x] = __uint_as_float(r[x]);
             Xb[row * kLd + c0 + x] = (c0 + x < row) ? b * v[x] : 0.f;
         }
-        if (SAVE) gstore_f32x32(p.Gm + grow * kT + c0, v);
     }
     __syncthreads();
 
@@ -222,13 +168,18 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
             hi[x] = __bfloat162float(__float2bfloat16_rn(t));
             lo[x] = t - hi[x];
         }
-        if (SAVE) gstore_f32x32(p.Ai + grow * kT + c0, v);
         tile_store32(sQK, row, c0, hi);
         tile_store32(sQK + kTileB, row, c0, lo);
         if (SAVE) {
+            gstore_bf16x32(p.sTh + grow * kT + c0, hi);
+            gstore_bf16x32(p.sTl + grow * kT + c0, lo);
 #pragma unroll
-            for (int x = 0; x < 32; ++x) v[x] = hi[x] + lo[x];
-            gstore_f32x32(p.Tt + grow * kT + c0, v);
+            for (int x = 0; x < 32; ++x) {
+                hi[x] = __bfloat162float(__float2bfloat16_rn(v[x]));
+                lo[x] = v[x] - hi[x];
+            }
+            gstore_bf16x32(p.sAh + grow * kT + c0, hi);
+            gstore_bf16x32(p.sAl + grow * kT + c0, lo);
         }
     }
     __syncthreads();  // everyone has read the float32 buffer; it now becomes the Xq / Xk tiles
@@ -241,7 +192,7 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] = (c0 + x <= row) ? __uint_as_float(r[x]) : 0.f;
         tile_store32(sBig, row, c0, v);
-        if (SAVE) gstore_f32x32(p.Xq + grow * kT + c0, v);
+        if (SAVE) gstore_bf16x32(p.sXq + grow * kT + c0, v);
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] = -v[x];
         gstore_bf16x32(p.Xqn + grow * kT + c0, v);
@@ -250,7 +201,7 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] = (c0 + x < row) ? __uint_as_float(r[x]) : 0.f;
         tile_store32(sBig + kTileB, row, c0, v);
-        if (SAVE) gstore_f32x32(p.Xk + grow * kT + c0, v);
+        if (SAVE) gstore_bf16x32(p.sXk + grow * kT + c0, v);
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
@@ -263,6 +214,7 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
         mma(tmem + 128, aK, OP_K, aBig + kTileB, OP_MN, 8, 128, true);
         umma_commit(&bars[1]);
     }
+    __syncwarp();
     if (!mbar_wait(&bars[1], 1, abort_flag, ST_PREP)) ok = false;
     ok = __syncthreads_and(ok);
     tc_fence_after_sync();
@@ -276,7 +228,7 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
         tile_store32(sQK, row, c0, v);
-        if (SAVE) gstore_f32x32(p.U + grow * HD + c0, v);
+        if (SAVE) gstore_bf16x32(p.sU + grow * HD + c0, v);
     }
     for (int c = 0; c < 2; ++c) {
         const int c0 = half * 64 + c * 32;
@@ -285,7 +237,7 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
         tile_store32(sQK + kTileB, row, c0, v);
-        if (SAVE) gstore_f32x32(p.Y + grow * kT + c0, v);
+        if (SAVE) gstore_bf16x32(p.sY + grow * kT + c0, v);
         __nv_bfloat16* yt = p.Yt + ((size_t)chunk * kT + c0) * kT + row;
 #pragma unroll
         for (int x = 0; x < 32; ++x) yt[(size_t)x * kT] = __float2bfloat16_rn(v[x]);
@@ -300,6 +252,7 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
         mma(tmem + 0, aW, OP_MN, aQ, OP_MN, 8, HD, false);
         umma_commit(&bars[1]);
     }
+    __syncwarp();
     if (!mbar_wait(&bars[1], 0, abort_flag, ST_PREP)) ok = false;
     ok = __syncthreads_and(ok);
     tc_fence_after_sync();

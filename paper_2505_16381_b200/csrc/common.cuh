@@ -15,7 +15,7 @@ enum : uint32_t {
     ST_FWD_PRODUCER = 0x101, ST_FWD_MMA = 0x102, ST_FWD_SOFTMAX = 0x103,
     ST_DKV_PRODUCER = 0x201, ST_DKV_MMA = 0x202, ST_DKV_COMPUTE = 0x203,
     ST_DQ_PRODUCER = 0x301, ST_DQ_MMA = 0x302, ST_DQ_COMPUTE = 0x303,
-    ST_PREP = 0x401,
+    ST_PREP = 0x401, ST_CHAIN = 0x501,
 };
 
 __host__ __device__ inline int msb32(unsigned x) {
@@ -70,13 +70,34 @@ struct PrepParams {
     __nv_bfloat16* Xqn;           // [S*Lp][128] -lower(Q W^T)
     __nv_bfloat16* Yt;            // [S*Lp][128] (T~ strictLower(W K^T))^T
     float* P;                     // [S*N][d][d] chunk products
-    float *Gm, *Ai, *Tt, *Xq, *Xk, *Y;   // [S*N][128][128], written only by the backward's instance
-    float* U;                     // [S*Lp][d], likewise
+    // bf16 copies for the chain rule, written only by the backward's instance ([S*Lp][128]; sU is [S*Lp][d]):
+    // T~ and (I + N)^-1 as hi + lo pairs, Xq, Xk, Y, U rounded once
+    __nv_bfloat16 *sTh, *sTl, *sAh, *sAl, *sXq, *sXk, *sY, *sU;
     uint32_t* status;
 };
 
 cudaError_t launch_chunk_prep(const PrepTensorMaps& tm, const PrepParams& p, int hd, int save, int nchunks,
                               cudaStream_t st);
+
+struct ChainTensorMaps {
+    CUtensorMap w, q, k, u;                       // [S*Lp][d]
+    CUtensorMap y, xq, xk, th, tl, ah, al;        // [S*Lp][128]
+};
+
+struct ChainParams {
+    const float* dql;     // [S*Lp][d]  gradient of the boundary-adjusted queries (version slot 0)
+    const float* dkr;     // [S*Lp][d]  gradient of the boundary-adjusted keys
+    const float* dsd;     // [S*N][128][128] lower(dS) of the diagonal chunks (unscaled)
+    const float* dp;      // [S*N][d][d] gradient of the chunk products
+    const float* beta;    // [S*Lp]
+    __nv_bfloat16 *dq, *dk, *dw;   // [S][L][d] outputs
+    float* dbeta;         // [S][L]
+    uint32_t* status;
+    int N, L;
+    float scale;
+};
+
+cudaError_t launch_chunk_chain(const ChainTensorMaps& tm, const ChainParams& p, int hd, int nchunks, cudaStream_t st);
 
 struct BwdTensorMaps {
     CUtensorMap q_raw, k_raw, v, qv, kv, xqn, yt, d_o;

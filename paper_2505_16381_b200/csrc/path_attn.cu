@@ -84,9 +84,10 @@ struct Plan {
     LevelTable lv;
     size_t total;
     // offsets (bytes)
-    size_t status, qp, kp, vp, wp, betap, G, Gm, Ai, Tt, U, Dy, Xq, Xk, Y, Xqn, Yt, Qv16, Kv16;
+    size_t status, qp, kp, vp, wp, betap, G, Dy, Xqn, Yt, Qv16, Kv16;
     // backward only
-    size_t dop, delta, lse2, dQv, dKv, dSd, dG, dGrow, dGdiag, dDy, dXq, dY, dT, dXk, tmpBB, dA, dU, tq, tk, tw, t1;
+    size_t dop, delta, lse2, dQv, dKv, dSd, dG, dGrow, dGdiag, dDy;
+    size_t sTh, sTl, sAh, sAl, sXq, sXk, sY, sU;   // bf16 tiles kept by the chunk preparation for the chain rule
     size_t dy_bytes;
 };
 
@@ -115,11 +116,11 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
     }
     p.betap = bump(cur, SL * 4);
     if (gate) p.G = bump(cur, SL * 4);
-    const size_t keep = bwd ? 1 : 0;   // float intermediates of the chunk preparation, kept for the chain rule
-    p.Gm = bump(cur, keep * SNBB * 4);
-    p.Ai = bump(cur, keep * SNBB * 4);
-    p.Tt = bump(cur, keep * SNBB * 4);
-    p.U = bump(cur, keep * SLd * 4);
+    const size_t keep = bwd ? 1 : 0;   // bf16 intermediates of the chunk preparation, kept for the chain rule
+    p.sTh = bump(cur, keep * SNBB * 2); p.sTl = bump(cur, keep * SNBB * 2);
+    p.sAh = bump(cur, keep * SNBB * 2); p.sAl = bump(cur, keep * SNBB * 2);
+    p.sXq = bump(cur, keep * SNBB * 2); p.sXk = bump(cur, keep * SNBB * 2); p.sY = bump(cur, keep * SNBB * 2);
+    p.sU = bump(cur, keep * SLd * 2);
     size_t dy_elems = 0;
     for (int l = 0; l < 20; ++l) {
         p.lv.dy_off[l] = (long)dy_elems;
@@ -127,9 +128,6 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
         if (l == 0 || l <= p.nlev - 2) dy_elems += (size_t)S * (p.N >> l) * d * d;
     }
     p.Dy = bump(cur, dy_elems * 4);
-    p.Xq = bump(cur, keep * SNBB * 4);
-    p.Xk = bump(cur, keep * SNBB * 4);
-    p.Y = bump(cur, keep * SNBB * 4);
     p.Xqn = bump(cur, SL * CHUNK * 2);
     p.Yt = bump(cur, SL * CHUNK * 2);
     p.Qv16 = bump(cur, SLd * 2 * p.nslot);
@@ -142,10 +140,6 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
         p.dSd = bump(cur, SNBB * 4); p.dG = bump(cur, SL * 4);
         p.dGrow = bump(cur, gate ? SL * 4 : 0); p.dGdiag = bump(cur, gate ? SL * 4 : 0);
         p.dDy = bump(cur, dy_elems * 4);
-        p.dXq = bump(cur, SNBB * 4); p.dY = bump(cur, SNBB * 4); p.dT = bump(cur, SNBB * 4);
-        p.dXk = bump(cur, SNBB * 4); p.tmpBB = bump(cur, SNBB * 4); p.dA = bump(cur, SNBB * 4);
-        p.dU = bump(cur, SLd * 4); p.tq = bump(cur, SLd * 4); p.tk = bump(cur, SLd * 4); p.tw = bump(cur, SLd * 4);
-        p.t1 = bump(cur, SL * 4);
     }
     p.total = cur;
     return true;
@@ -184,9 +178,9 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
         pp.Xqn = at<__nv_bfloat16>(ws, p.Xqn); pp.Yt = at<__nv_bfloat16>(ws, p.Yt);
         pp.P = Dy;
         if (p.bwd) {
-            pp.Gm = at<float>(ws, p.Gm); pp.Ai = at<float>(ws, p.Ai); pp.Tt = at<float>(ws, p.Tt);
-            pp.Xq = at<float>(ws, p.Xq); pp.Xk = at<float>(ws, p.Xk); pp.Y = at<float>(ws, p.Y);
-            pp.U = at<float>(ws, p.U);
+            typedef __nv_bfloat16 bf;
+            pp.sTh = at<bf>(ws, p.sTh); pp.sTl = at<bf>(ws, p.sTl); pp.sAh = at<bf>(ws, p.sAh); pp.sAl = at<bf>(ws, p.sAl);
+            pp.sXq = at<bf>(ws, p.sXq); pp.sXk = at<bf>(ws, p.sXk); pp.sY = at<bf>(ws, p.sY); pp.sU = at<bf>(ws, p.sU);
         }
         pp.status = at<uint32_t>(ws, p.status);
         LAUNCH(launch_chunk_prep(tm, pp, d, p.bwd, nch, st));
@@ -244,82 +238,26 @@ static int stage_inputs(const Plan& p, void* ws, const void*& q, const void*& k,
 
 namespace path {
 
-// Per-chunk chain rule through the UT transform and the boundary-adjusted tiles (no counterpart in the paper):
-// from dQleft, dKright, dSd (diagonal logits), dP (chunk product) back to dq, dk, dw, dbeta.
+// Per-chunk chain rule through the UT transform and the boundary-adjusted tiles: one fused kernel.
 static int run_chunk_chain(const Plan& p, void* ws, const void* q, const void* k, const void* w, void* dq, void* dk,
                            void* dw, float* dbeta, float scale, cudaStream_t st) {
-    const int d = p.d, nch = p.S * p.N;
-    const long Bd = (long)CHUNK * d, BB = (long)CHUNK * CHUNK, dd = (long)d * d;
-    float* Gm = at<float>(ws, p.Gm); float* Tt = at<float>(ws, p.Tt); float* U = at<float>(ws, p.U);
-    float* Ai = at<float>(ws, p.Ai); float* Xq = at<float>(ws, p.Xq); float* Xk = at<float>(ws, p.Xk);
-    float* Y = at<float>(ws, p.Y);
-    float* dQl = at<float>(ws, p.dQv); float* dKr = at<float>(ws, p.dKv);  // slot 0 of the version gradients
-    float* dSd = at<float>(ws, p.dSd); float* dP = at<float>(ws, p.dDy);  // level 0 of the run-product gradients
-    float* dXq = at<float>(ws, p.dXq); float* dY = at<float>(ws, p.dY); float* dT = at<float>(ws, p.dT);
-    float* dXk = at<float>(ws, p.dXk); float* tmp = at<float>(ws, p.tmpBB); float* dA = at<float>(ws, p.dA);
-    float* dU = at<float>(ws, p.dU); float* tq = at<float>(ws, p.tq); float* tk = at<float>(ws, p.tk);
-    float* tw = at<float>(ws, p.tw); float* t1 = at<float>(ws, p.t1);
-    const float* betap = at<float>(ws, p.betap);
-
-    // operand shorthands: R = row-major as stored, T = transposed view
-    auto R = [](const void* ptr, long ld, int f32) { return Operand{ptr, ld, 1, f32}; };   // A(m,k) = X[m][k]
-    auto Tr = [](const void* ptr, long ld, int f32) { return Operand{ptr, 1, ld, f32}; };  // A(m,k) = X[k][m]
-    // for the B operand B(k,n): Tr(X) means B(k,n) = X[k][n] (s_mn = 1, s_k = ld); R(X) means B(k,n) = X[n][k]
-    auto run = [&](Operand A, long sa, Operand B, long sb, int M, int N, int K, float* C, long sc, float alpha, int mask,
-                   int acc, const float* D = nullptr, long sd = 0, void* C2 = nullptr) -> int {
-        GemmProblem g = gemm_problem(A, B, M, N, K);
-        g.C = C; g.c_f32 = 1; g.ldc = N; g.alpha = alpha; g.mask = mask; g.accumulate = acc;
-        if (D) { g.D = D; g.d_f32 = 1; g.ldd = N; }
-        AffineBatch ab{};
-        if (C2) {
-            g.C2 = C2; g.ldc2 = N;
-            ab.nb1 = p.N; ab.rows_total = p.L;
-            ab.a0 = sa * p.N; ab.a1 = sa; ab.b0 = sb * p.N; ab.b1 = sb; ab.c0 = sc * p.N; ab.c1 = sc;
-            ab.d0 = sd * p.N; ab.d1 = sd; ab.c20 = (long)p.L * d; ab.c21 = Bd;
-        } else {
-            ab = chunk_batch(p, sa, sb, sc, 0, sd);
-        }
-        LAUNCH(launch_gemm(g, ab, nch, st));
-        return PATH_OK;
-    };
-#define RUN(...) do { int rc__ = run(__VA_ARGS__); if (rc__ != PATH_OK) return rc__; } while (0)
-    const int B = CHUNK;
-    // dSd below is the unscaled lower(dS) of the diagonal chunk; `scale` enters through the alphas.
-    // dXq = lower(-dQl U^T - scale dSd Y^T)
-    RUN(R(dQl, d, 1), Bd, R(U, d, 1), Bd, B, B, d, dXq, BB, -1.f, MASK_LOWER, ACC_NONE);
-    RUN(R(dSd, B, 1), BB, R(Y, B, 1), BB, B, B, B, dXq, BB, -scale, MASK_LOWER, ACC_ADD);
-    // dU = -Xq^T dQl - W dP
-    RUN(Tr(Xq, B, 1), BB, Tr(dQl, d, 1), Bd, B, d, B, dU, Bd, -1.f, MASK_NONE, ACC_NONE);
-    RUN(R(w, d, 0), Bd, Tr(dP, d, 1), dd, B, d, d, dU, Bd, -1.f, MASK_NONE, ACC_ADD);
-    // dY = -W dKr^T - Xq^T dSd
-    RUN(R(w, d, 0), Bd, R(dKr, d, 1), Bd, B, B, d, dY, BB, -1.f, MASK_NONE, ACC_NONE);
-    RUN(Tr(Xq, B, 1), BB, Tr(dSd, B, 1), BB, B, B, B, dY, BB, -scale, MASK_NONE, ACC_ADD);
-    // dT = lower(dY Xk^T + dU W^T)
-    RUN(R(dY, B, 1), BB, R(Xk, B, 1), BB, B, B, B, dT, BB, 1.f, MASK_LOWER, ACC_NONE);
-    RUN(R(dU, d, 1), Bd, R(w, d, 0), Bd, B, B, d, dT, BB, 1.f, MASK_LOWER, ACC_ADD);
-    // dXk = strictLower(T~^T dY)
-    RUN(Tr(Tt, B, 1), BB, Tr(dY, B, 1), BB, B, B, B, dXk, BB, 1.f, MASK_STRICT, ACC_NONE);
-    // dbeta (first term) and dT <- dT D;  dA = strictLower(-Ainv^T (dT D) Ainv^T)
-    LAUNCH(launch_beta_cols(Ai, dT, betap, t1, nch, st));
-    RUN(Tr(Ai, B, 1), BB, Tr(dT, B, 1), BB, B, B, B, tmp, BB, 1.f, MASK_NONE, ACC_NONE);
-    RUN(R(tmp, B, 1), BB, R(Ai, B, 1), BB, B, B, B, dA, BB, -1.f, MASK_STRICT, ACC_NONE);
-    // dbeta (second term, final) and dA <- D dA = dGm
-    LAUNCH(launch_beta_rows(dA, Gm, betap, t1, dbeta, p.S, p.N, p.L, st));
-    // dq = dQl + dSd K + dXq W
-    RUN(R(dSd, B, 1), BB, Tr(k, d, 0), Bd, B, d, B, tq, Bd, scale, MASK_NONE, ACC_NONE, dQl, Bd);
-    RUN(R(dXq, B, 1), BB, Tr(w, d, 0), Bd, B, d, B, tq, Bd, 1.f, MASK_NONE, ACC_ADD, nullptr, 0, dq);
-    // dk = dKr + dSd^T Q + dXk^T W
-    RUN(Tr(dSd, B, 1), BB, Tr(q, d, 0), Bd, B, d, B, tk, Bd, scale, MASK_NONE, ACC_NONE, dKr, Bd);
-    RUN(Tr(dXk, B, 1), BB, Tr(w, d, 0), Bd, B, d, B, tk, Bd, 1.f, MASK_NONE, ACC_ADD, nullptr, 0, dk);
-    // dw = -Y dKr - U dP^T + T~^T dU + dXq^T Q + dXk K + dGm W + dGm^T W
-    RUN(R(Y, B, 1), BB, Tr(dKr, d, 1), Bd, B, d, B, tw, Bd, -1.f, MASK_NONE, ACC_NONE);
-    RUN(R(U, d, 1), Bd, R(dP, d, 1), dd, B, d, d, tw, Bd, -1.f, MASK_NONE, ACC_ADD);
-    RUN(Tr(Tt, B, 1), BB, Tr(dU, d, 1), Bd, B, d, B, tw, Bd, 1.f, MASK_NONE, ACC_ADD);
-    RUN(Tr(dXq, B, 1), BB, Tr(q, d, 0), Bd, B, d, B, tw, Bd, 1.f, MASK_NONE, ACC_ADD);
-    RUN(R(dXk, B, 1), BB, Tr(k, d, 0), Bd, B, d, B, tw, Bd, 1.f, MASK_NONE, ACC_ADD);
-    RUN(R(dA, B, 1), BB, Tr(w, d, 0), Bd, B, d, B, tw, Bd, 1.f, MASK_NONE, ACC_ADD);
-    RUN(Tr(dA, B, 1), BB, Tr(w, d, 0), Bd, B, d, B, tw, Bd, 1.f, MASK_NONE, ACC_ADD, nullptr, 0, dw);
-#undef RUN
+    const int d = p.d;
+    const uint64_t rows = (uint64_t)p.S * p.Lp;
+    ChainTensorMaps tm;
+    bool ok = make_map(&tm.w, w, rows, d) && make_map(&tm.q, q, rows, d) && make_map(&tm.k, k, rows, d) &&
+              make_map(&tm.u, at<void>(ws, p.sU), rows, d) && make_map(&tm.y, at<void>(ws, p.sY), rows, CHUNK) &&
+              make_map(&tm.xq, at<void>(ws, p.sXq), rows, CHUNK) && make_map(&tm.xk, at<void>(ws, p.sXk), rows, CHUNK) &&
+              make_map(&tm.th, at<void>(ws, p.sTh), rows, CHUNK) && make_map(&tm.tl, at<void>(ws, p.sTl), rows, CHUNK) &&
+              make_map(&tm.ah, at<void>(ws, p.sAh), rows, CHUNK) && make_map(&tm.al, at<void>(ws, p.sAl), rows, CHUNK);
+    if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+    ChainParams cp{};
+    cp.dql = at<float>(ws, p.dQv); cp.dkr = at<float>(ws, p.dKv);   // slot 0 of the version gradients
+    cp.dsd = at<float>(ws, p.dSd); cp.dp = at<float>(ws, p.dDy);    // level 0 of the run-product gradients
+    cp.beta = at<float>(ws, p.betap);
+    cp.dq = (__nv_bfloat16*)dq; cp.dk = (__nv_bfloat16*)dk; cp.dw = (__nv_bfloat16*)dw; cp.dbeta = dbeta;
+    cp.status = at<uint32_t>(ws, p.status);
+    cp.N = p.N; cp.L = p.L; cp.scale = scale;
+    LAUNCH(launch_chunk_chain(tm, cp, d, p.S * p.N, st));
     return PATH_OK;
 }
 

@@ -1,0 +1,87 @@
+// Building blocks of the "lockstep" chunk kernels: every matrix of the chunk-level algebra is a 128-row
+// bf16 tile in shared memory (row-major, 64-column panels, 128-byte swizzle), every product a tcgen05 MMA into
+// tensor memory issued by thread 0, every result read back one row per thread (256 threads: two per row, each
+// taking half of the columns).
+#pragma once
+#include "common.cuh"
+#include "tc5.cuh"
+
+namespace path {
+namespace tile {
+using namespace tc5;
+
+constexpr int kT = 128;
+constexpr uint32_t kTileB = 32768, kPanelB = 16384;
+
+// K view: contraction over the tile's columns.  MN view: contraction over the tile's rows.
+enum { OP_K = 0, OP_MN = 1 };
+__device__ __forceinline__ uint64_t desc_k(uint32_t t, int kk) {
+    return umma_desc(t + (kk >> 2) * kPanelB + (kk & 3) * 32, 16, 1024);
+}
+__device__ __forceinline__ uint64_t desc_mn(uint32_t t, int kk) { return umma_desc(t + kk * 2048, kPanelB, 1024); }
+
+// D[128 x n] (+)= (+-) op(A) op(B), `ksteps` steps of 16 along the contraction.
+__device__ __forceinline__ void mma(uint32_t d_tmem, uint32_t a_tile, int a_op, uint32_t b_tile, int b_op, int ksteps,
+                                    int n, bool acc, bool negate = false) {
+    const uint32_t idesc = umma_idesc(128, n, a_op, b_op) | (negate ? (1u << 13) : 0u);
+    for (int kk = 0; kk < ksteps; ++kk)
+        umma_ss(d_tmem, a_op == OP_K ? desc_k(a_tile, kk) : desc_mn(a_tile, kk),
+                b_op == OP_K ? desc_k(b_tile, kk) : desc_mn(b_tile, kk), idesc, (acc || kk > 0) ? 1u : 0u);
+}
+
+// Stores columns c0 .. c0+31 of `row` of a swizzled bf16 tile.
+__device__ __forceinline__ void tile_store32(uint8_t* t, int row, int c0, const float (&v)[32]) {
+    uint8_t* panel = t + (c0 >> 6) * kPanelB;
+    const int ch0 = (c0 & 63) >> 3;
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch)
+        *reinterpret_cast<uint4*>(panel + sw128_off((uint32_t)row, (uint32_t)(ch0 + ch))) =
+            make_uint4(pack_bf16(v[8 * ch], v[8 * ch + 1]), pack_bf16(v[8 * ch + 2], v[8 * ch + 3]),
+                       pack_bf16(v[8 * ch + 4], v[8 * ch + 5]), pack_bf16(v[8 * ch + 6], v[8 * ch + 7]));
+}
+__device__ __forceinline__ void gstore_f32x32(float* dst, const float (&v)[32]) {
+#pragma unroll
+    for (int x = 0; x < 8; ++x)
+        reinterpret_cast<float4*>(dst)[x] = make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
+}
+__device__ __forceinline__ void gload_f32x32(const float* src, float (&v)[32]) {
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+        const float4 f = reinterpret_cast<const float4*>(src)[x];
+        v[4 * x] = f.x; v[4 * x + 1] = f.y; v[4 * x + 2] = f.z; v[4 * x + 3] = f.w;
+    }
+}
+__device__ __forceinline__ void gstore_bf16x32(__nv_bfloat16* dst, const float (&v)[32]) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+        reinterpret_cast<uint4*>(dst)[x] =
+            make_uint4(pack_bf16(v[8 * x], v[8 * x + 1]), pack_bf16(v[8 * x + 2], v[8 * x + 3]),
+                       pack_bf16(v[8 * x + 4], v[8 * x + 5]), pack_bf16(v[8 * x + 6], v[8 * x + 7]));
+}
+__device__ __forceinline__ void gload_bf16x32(const __nv_bfloat16* src, float (&v)[32]) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const uint4 u = reinterpret_cast<const uint4*>(src)[x];
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[y]));
+            v[8 * x + 2 * y] = f.x;
+            v[8 * x + 2 * y + 1] = f.y;
+        }
+    }
+}
+__device__ __forceinline__ void tmem_row32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    tmem_ld32(taddr, r);
+    tmem_ld_wait();
+#pragma unroll
+    for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
+}
+// TMA load of a [128 x ncols] bf16 tile (ncols = 64 or 128) whose first row is `row0` of the mapped matrix.
+__device__ __forceinline__ void tma_tile(uint8_t* dst, const CUtensorMap* m, uint64_t* bar, int ncols, int row0) {
+    for (int h = 0; h < ncols / 64; ++h) tma_load_2d(dst + h * kPanelB, m, bar, h * 64, row0);
+}
+
+}  // namespace tile
+}  // namespace path
