@@ -37,7 +37,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int chunk = blockIdx.x;
     const int row = (warp & 3) * 32 + lane, half = warp >> 2;
-    const size_t grow = (size_t)chunk * kT + row;
     const int s_idx = chunk / p.N, pos = (chunk % p.N) * kT + row;   // slice and position of this thread's row
     const bool row_valid = pos < p.L;
     const size_t urow = (size_t)s_idx * p.L + pos;                   // row in the caller's [S][L][.] tensors

@@ -15,7 +15,7 @@ enum : uint32_t {
     ST_FWD_PRODUCER = 0x101, ST_FWD_MMA = 0x102, ST_FWD_SOFTMAX = 0x103,
     ST_DKV_PRODUCER = 0x201, ST_DKV_MMA = 0x202, ST_DKV_COMPUTE = 0x203,
     ST_DQ_PRODUCER = 0x301, ST_DQ_MMA = 0x302, ST_DQ_COMPUTE = 0x303,
-    ST_PREP = 0x401, ST_CHAIN = 0x501,
+    ST_PREP = 0x401, ST_CHAIN = 0x501, ST_LEVELS = 0x601,
 };
 
 __host__ __device__ inline int msb32(unsigned x) {
@@ -57,6 +57,30 @@ struct FwdParams {
     int out_fp32;
 };
 
+// Placement of the dyadic run products: level l holds dy_cnt[l] = N >> l matrices per slice, starting
+// dy_off[l] elements into the buffer (same layout for the bf16 hi / lo planes and the float gradients).
+struct LevelTable {
+    long dy_off[20];
+    int dy_cnt[20];
+};
+
+struct LevelTensorMaps {
+    CUtensorMap dyh, dyl;   // [matrices * d][d] bf16 hi / lo planes of the run products
+    CUtensorMap qv, kv;     // [slots * S * Lp][d] bf16 versions
+};
+
+struct LevelParams {
+    LevelTable lv;
+    int l;                  // dyadic kernels: level being produced (fwd: l -> l + 1) / consumed (bwd); version kernels: l2
+    int S, N, Lp;
+    __nv_bfloat16 *dyh, *dyl, *qv, *kv;
+    float *dqv, *dkv, *ddy;
+    uint32_t* status;
+};
+
+enum { LEVEL_DYADIC_FWD = 0, LEVEL_VERSION_FWD, LEVEL_VERSION_BWD, LEVEL_DYADIC_BWD };
+cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const LevelParams& p, int hd, cudaStream_t st);
+
 struct PrepTensorMaps {
     CUtensorMap w, q, k;   // [S*Lp][d] bf16, box 128 rows x 64 columns, 128-byte swizzle
 };
@@ -69,7 +93,7 @@ struct PrepParams {
     __nv_bfloat16* kr;            // [S*Lp][d]   boundary-adjusted keys (version slot 0)
     __nv_bfloat16* Xqn;           // [S*Lp][128] -lower(Q W^T)
     __nv_bfloat16* Yt;            // [S*Lp][128] (T~ strictLower(W K^T))^T
-    float* P;                     // [S*N][d][d] chunk products
+    __nv_bfloat16 *Ph, *Pl;       // [S*N][d][d] chunk products as a bf16 hi + lo pair (level 0 of the run products)
     // bf16 copies for the chain rule, written only by the backward's instance ([S*Lp][128]; sU is [S*Lp][d]):
     // T~ and (I + N)^-1 as hi + lo pairs, Xq, Xk, Y, U rounded once
     __nv_bfloat16 *sTh, *sTl, *sAh, *sAl, *sXq, *sXk, *sY, *sU;

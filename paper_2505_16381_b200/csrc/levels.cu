@@ -1,0 +1,342 @@
+// Dyadic run products and version chains (forward and backward), as tcgen05 tile kernels.
+//
+// The attention sweep never updates a query while it walks the keys (the paper's Sec. 3.3 loop does, once per
+// key chunk).  Instead query chunk I and key chunk J < I meet at the dyadic boundary e = (I >> l) << l,
+// l = msb(I xor J), which is the same logit by associativity (the key-advance identity of Sec. 3.4):
+//     Qv[l][I] = Qleft_I  P_{I-1} ... P_e          Kv[l][J] = Kright_J P_{J+1}^T ... P_{e-1}^T
+// Both follow from products of aligned runs of chunk matrices, Dy[l][b] = P_{(b+1) 2^l - 1} ... P_{b 2^l}:
+//     Dy[l+1][b] = Dy[l][2b+1] Dy[l][2b]                                                (dyadic_fwd)
+//     Qv[l2][I]  = Qv[l1][I] Dy[l1][(I >> l2 << l2) >> l1]      l1 < l2 consecutive set bits of I     (version_fwd)
+//     Kv[l2][J]  = Kv[l1][J] Dy[l1][(J >> l1) + 1]^T            l1 < l2 consecutive clear bits of J
+// and the backward kernels apply the chain rule to exactly these products.  Run products are stored as bf16
+// hi + lo pairs (they are multiplied up to log2(N) times); versions are bf16, the values the sweep consumes.
+#include "tileops.cuh"
+
+namespace path {
+using namespace tile;
+
+namespace {
+
+struct Ctx {
+    uint8_t* smem;
+    uint64_t* bars;
+    volatile uint32_t* abort_flag;
+    uint32_t tmem, tl;
+    int tid, warp, lane, row, half;
+    uint32_t ph_load, ph_mma;
+    bool ok;
+};
+
+template <int NCOLS>
+__device__ __forceinline__ void setup(Ctx& c, uint8_t* smem_raw, uint32_t bar_off) {
+    c.smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    c.bars = (uint64_t*)(c.smem + bar_off);
+    uint32_t* tmem_slot = (uint32_t*)(c.bars + 2);
+    c.abort_flag = (volatile uint32_t*)(tmem_slot + 1);
+    c.tid = threadIdx.x; c.warp = c.tid >> 5; c.lane = c.tid & 31;
+    c.row = (c.warp & 3) * 32 + c.lane; c.half = c.warp >> 2;
+    c.ph_load = c.ph_mma = 0; c.ok = true;
+    if (c.tid == 0) {
+        mbar_init(&c.bars[0], 1);
+        mbar_init(&c.bars[1], 1);
+        *c.abort_flag = 0;
+        mbar_fence_init();
+    }
+    if (c.warp == 0) tmem_alloc(tmem_slot, NCOLS);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    c.tmem = *tmem_slot;
+    c.tl = c.tmem + ((uint32_t)((c.warp & 3) * 32) << 16);
+}
+template <int NCOLS>
+__device__ __forceinline__ void teardown(Ctx& c, uint32_t* status) {
+    tc_fence_before_sync();
+    __syncthreads();
+    if (c.tid == 0 && *c.abort_flag != 0) atomicCAS(status, 0u, *c.abort_flag);
+    if (c.warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(c.tmem, NCOLS);
+    }
+}
+__device__ __forceinline__ void loads_wait(Ctx& c) {
+    if (!mbar_wait(&c.bars[0], c.ph_load, c.abort_flag, ST_LEVELS)) c.ok = false;
+    c.ph_load ^= 1;
+}
+__device__ __forceinline__ void publish() {
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+}
+__device__ __forceinline__ void mma_wait(Ctx& c) {
+    __syncwarp();
+    if (!mbar_wait(&c.bars[1], c.ph_mma, c.abort_flag, ST_LEVELS)) c.ok = false;
+    c.ph_mma ^= 1;
+    c.ok = __syncthreads_and(c.ok);
+    tc_fence_after_sync();
+}
+// float rows [nrows][ncols] of a global matrix -> bf16 tile (rows >= nrows are zero-filled)
+__device__ __forceinline__ void conv(const Ctx& c, const float* src, int ncols, int nrows, uint8_t* dst) {
+    const int per = ncols / 2;
+    float v[32];
+    for (int i = 0; i < per / 32; ++i) {
+        const int c0 = c.half * per + i * 32;
+        if (c.row < nrows) gload_f32x32(src + (size_t)c.row * ncols + c0, v);
+        else {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) v[x] = 0.f;
+        }
+        tile_store32(dst, c.row, c0, v);
+    }
+}
+// accumulator rows -> global float matrix [nrows][ncols]: dst += acc (plain or atomic)
+template <bool ATOMIC>
+__device__ __forceinline__ void acc_add_global(const Ctx& c, uint32_t col, int ncols, int nrows, float* dst) {
+    const int per = ncols / 2;
+    float v[32];
+    for (int i = 0; i < per / 32; ++i) {
+        const int c0 = c.half * per + i * 32;
+        tmem_row32(c.tl + col + c0, v);
+        if (c.row >= nrows) continue;
+        float* d = dst + (size_t)c.row * ncols + c0;
+        if (ATOMIC) {
+#pragma unroll
+            for (int x = 0; x < 32; ++x) atomicAdd(d + x, v[x]);
+        } else {
+            float o[32];
+            gload_f32x32(d, o);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) o[x] += v[x];
+            gstore_f32x32(d, o);
+        }
+    }
+}
+
+// Resolves the version-chain step of chunk c at level l2.  Returns false if there is none.
+__device__ __forceinline__ bool version_step(int is_key, int c, int l2, int N, int& l1, int& b, int& src_slot) {
+    if (!is_key) {
+        const unsigned low = (unsigned)c & ((1u << l2) - 1u);
+        if (!((c >> l2) & 1) || low == 0) return false;
+        l1 = msb32(low);
+        b = ((c >> l2) << l2) >> l1;
+        src_slot = qslot(l1, c);
+    } else {
+        const unsigned lowz = ~(unsigned)c & ((1u << l2) - 1u);
+        if (((c >> l2) & 1) || lowz == 0) return false;
+        if ((((c >> l2) + 1) << l2) > N - 1) return false;
+        l1 = msb32(lowz);
+        b = (c >> l1) + 1;
+        src_slot = kslot(l1, c);
+    }
+    return true;
+}
+
+constexpr uint32_t kBar3 = 3 * kTileB, kBar4 = 4 * kTileB, kBar5 = 5 * kTileB;
+constexpr uint32_t smem_bytes(uint32_t slots) { return slots * kTileB + 64 + 1024; }
+
+// ---------------------------------------------------------------------------------------------- dyadic forward
+// grid.x = S * cnt2.  Dy[l+1][b] = Dy[l][2b+1] Dy[l][2b] with hi/lo operands (three products).
+template <int HD>
+__global__ void __launch_bounds__(256, 1) dyadic_fwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    Ctx c;
+    setup<128>(c, smem_raw, kBar4);
+    const int cnt2 = p.lv.dy_cnt[p.l + 1], cnt = p.lv.dy_cnt[p.l];
+    const int s = blockIdx.x / cnt2, b = blockIdx.x % cnt2;
+    const long mat_lo = p.lv.dy_off[p.l] / (HD * HD) + (long)s * cnt + 2 * b;        // right factor; left is +1
+    const long mat_out = p.lv.dy_off[p.l + 1] / (HD * HD) + (long)s * cnt2 + b;
+    uint8_t* sm = c.smem;
+    if (c.tid == 0) {
+        mbar_expect_tx(&c.bars[0], 4 * kT * HD * 2);
+        tma_tile(sm + 0 * kTileB, &tm.dyh, &c.bars[0], HD, (int)((mat_lo + 1) * HD));
+        tma_tile(sm + 1 * kTileB, &tm.dyl, &c.bars[0], HD, (int)((mat_lo + 1) * HD));
+        tma_tile(sm + 2 * kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat_lo * HD));
+        tma_tile(sm + 3 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat_lo * HD));
+    }
+    loads_wait(c);
+    if (c.tid == 0 && c.ok) {
+        tc_fence_after_sync();
+        const uint32_t a = smem_u32(sm);
+        mma(c.tmem, a, OP_K, a + 2 * kTileB, OP_MN, HD / 16, HD, false);
+        mma(c.tmem, a, OP_K, a + 3 * kTileB, OP_MN, HD / 16, HD, true);
+        mma(c.tmem, a + kTileB, OP_K, a + 2 * kTileB, OP_MN, HD / 16, HD, true);
+        umma_commit(&c.bars[1]);
+    }
+    mma_wait(c);
+    if (c.ok) {
+        float v[32], hi[32];
+        for (int i = 0; i < HD / 64; ++i) {
+            const int c0 = c.half * (HD / 2) + i * 32;
+            tmem_row32(c.tl + c0, v);
+            if (c.row < HD) {
+#pragma unroll
+                for (int x = 0; x < 32; ++x) {
+                    hi[x] = __bfloat162float(__float2bfloat16_rn(v[x]));
+                    v[x] -= hi[x];
+                }
+                const size_t o = ((size_t)mat_out * HD + c.row) * HD + c0;
+                gstore_bf16x32(p.dyh + o, hi);
+                gstore_bf16x32(p.dyl + o, v);
+            }
+        }
+    }
+    teardown<128>(c, p.status);
+}
+
+// ---------------------------------------------------------------------------------------------- version forward
+// grid = (S * N, 2): y = 0 queries, y = 1 keys.  Xv[l2][chunk] = Xv[l1][chunk] * Dy (queries) or Dy^T (keys).
+template <int HD>
+__global__ void __launch_bounds__(256, 2) version_fwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
+    const int is_key = blockIdx.y, s = blockIdx.x / p.N, ch = blockIdx.x % p.N;
+    int l1, b, src;
+    if (!version_step(is_key, ch, p.l, p.N, l1, b, src)) return;
+    extern __shared__ uint8_t smem_raw[];
+    Ctx c;
+    setup<128>(c, smem_raw, kBar3);
+    const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
+    const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
+    const long row_dst = ((long)p.l * p.S + s) * p.Lp + (long)ch * kT;
+    uint8_t* sm = c.smem;
+    if (c.tid == 0) {
+        mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2);
+        tma_tile(sm, is_key ? &tm.kv : &tm.qv, &c.bars[0], HD, (int)row_src);
+        tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
+        tma_tile(sm + 2 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
+    }
+    loads_wait(c);
+    if (c.tid == 0 && c.ok) {
+        tc_fence_after_sync();
+        const uint32_t a = smem_u32(sm);
+        const int bop = is_key ? OP_K : OP_MN;
+        mma(c.tmem, a, OP_K, a + kTileB, bop, HD / 16, HD, false);
+        mma(c.tmem, a, OP_K, a + 2 * kTileB, bop, HD / 16, HD, true);
+        umma_commit(&c.bars[1]);
+    }
+    mma_wait(c);
+    if (c.ok) {
+        float v[32];
+        __nv_bfloat16* out = (is_key ? p.kv : p.qv) + (size_t)row_dst * HD;
+        for (int i = 0; i < HD / 64; ++i) {
+            const int c0 = c.half * (HD / 2) + i * 32;
+            tmem_row32(c.tl + c0, v);
+            gstore_bf16x32(out + (size_t)c.row * HD + c0, v);
+        }
+    }
+    teardown<128>(c, p.status);
+}
+
+// ---------------------------------------------------------------------------------------------- version backward
+// With g = dXv[l2][chunk]:   dXv[l1][chunk] += g Dy^T (queries) or g Dy (keys);
+//                            dDy[l1][b]     += Xv[l1]^T g (queries) or g^T Xv[l1] (keys), atomically.
+template <int HD>
+__global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
+    const int is_key = blockIdx.y, s = blockIdx.x / p.N, ch = blockIdx.x % p.N;
+    int l1, b, src;
+    if (!version_step(is_key, ch, p.l, p.N, l1, b, src)) return;
+    extern __shared__ uint8_t smem_raw[];
+    Ctx c;
+    setup<256>(c, smem_raw, kBar4);
+    const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
+    const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
+    const long row_dst = ((long)p.l * p.S + s) * p.Lp + (long)ch * kT;
+    float* dxv = is_key ? p.dkv : p.dqv;
+    uint8_t* sm = c.smem;   // slots: 0 g, 1 Dy hi, 2 Dy lo, 3 Xv
+    if (c.tid == 0) {
+        mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2);
+        tma_tile(sm + 1 * kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
+        tma_tile(sm + 2 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
+        tma_tile(sm + 3 * kTileB, is_key ? &tm.kv : &tm.qv, &c.bars[0], HD, (int)row_src);
+    }
+    conv(c, dxv + (size_t)row_dst * HD, HD, kT, sm);
+    loads_wait(c);
+    publish();
+    if (c.tid == 0 && c.ok) {
+        tc_fence_after_sync();
+        const uint32_t a = smem_u32(sm);
+        const int bop = is_key ? OP_MN : OP_K;
+        mma(c.tmem, a, OP_K, a + kTileB, bop, HD / 16, HD, false);
+        mma(c.tmem, a, OP_K, a + 2 * kTileB, bop, HD / 16, HD, true);
+        if (!is_key) mma(c.tmem + 128, a + 3 * kTileB, OP_MN, a, OP_MN, 8, HD, false);
+        else         mma(c.tmem + 128, a, OP_MN, a + 3 * kTileB, OP_MN, 8, HD, false);
+        umma_commit(&c.bars[1]);
+    }
+    mma_wait(c);
+    if (c.ok) {
+        acc_add_global<false>(c, 0, HD, kT, dxv + (size_t)row_src * HD);
+        acc_add_global<true>(c, 128, HD, HD, p.ddy + (size_t)mat * HD * HD);
+    }
+    teardown<256>(c, p.status);
+}
+
+// ---------------------------------------------------------------------------------------------- dyadic backward
+// grid.x = S * cnt(l).  With dC = dDy[l][b], A = Dy[l-1][2b+1], B = Dy[l-1][2b]:  dA += dC B^T,  dB += A^T dC.
+template <int HD>
+__global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    Ctx c;
+    setup<256>(c, smem_raw, kBar5);
+    const int cnt = p.lv.dy_cnt[p.l], cntl = p.lv.dy_cnt[p.l - 1];
+    const int s = blockIdx.x / cnt, b = blockIdx.x % cnt;
+    const long mat_up = p.lv.dy_off[p.l] / (HD * HD) + (long)s * cnt + b;
+    const long mat_lo = p.lv.dy_off[p.l - 1] / (HD * HD) + (long)s * cntl + 2 * b;   // B; A is +1
+    uint8_t* sm = c.smem;   // slots: 0 dC, 1 A hi, 2 A lo, 3 B hi, 4 B lo
+    if (c.tid == 0) {
+        mbar_expect_tx(&c.bars[0], 4 * kT * HD * 2);
+        tma_tile(sm + 1 * kTileB, &tm.dyh, &c.bars[0], HD, (int)((mat_lo + 1) * HD));
+        tma_tile(sm + 2 * kTileB, &tm.dyl, &c.bars[0], HD, (int)((mat_lo + 1) * HD));
+        tma_tile(sm + 3 * kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat_lo * HD));
+        tma_tile(sm + 4 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat_lo * HD));
+    }
+    conv(c, p.ddy + (size_t)mat_up * HD * HD, HD, HD, sm);
+    loads_wait(c);
+    publish();
+    if (c.tid == 0 && c.ok) {
+        tc_fence_after_sync();
+        const uint32_t a = smem_u32(sm);
+        mma(c.tmem, a, OP_K, a + 3 * kTileB, OP_K, HD / 16, HD, false);            // dC B^T
+        mma(c.tmem, a, OP_K, a + 4 * kTileB, OP_K, HD / 16, HD, true);
+        mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a, OP_MN, HD / 16, HD, false);    // A^T dC
+        mma(c.tmem + 128, a + 2 * kTileB, OP_MN, a, OP_MN, HD / 16, HD, true);
+        umma_commit(&c.bars[1]);
+    }
+    mma_wait(c);
+    if (c.ok) {
+        acc_add_global<false>(c, 0, HD, HD, p.ddy + (size_t)(mat_lo + 1) * HD * HD);
+        acc_add_global<false>(c, 128, HD, HD, p.ddy + (size_t)mat_lo * HD * HD);
+    }
+    teardown<256>(c, p.status);
+}
+
+template <class K>
+cudaError_t launch(K kern, dim3 grid, uint32_t slots, const LevelTensorMaps& tm, const LevelParams& p, cudaStream_t st) {
+    const uint32_t bytes = smem_bytes(slots);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, 256, bytes, st>>>(tm, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const LevelParams& p, int hd, cudaStream_t st) {
+    switch (which) {
+        case LEVEL_DYADIC_FWD: {
+            dim3 g(p.S * p.lv.dy_cnt[p.l + 1]);
+            return hd == 64 ? launch(dyadic_fwd_kernel<64>, g, 4, tm, p, st) : launch(dyadic_fwd_kernel<128>, g, 4, tm, p, st);
+        }
+        case LEVEL_VERSION_FWD: {
+            dim3 g(p.S * p.N, 2);
+            return hd == 64 ? launch(version_fwd_kernel<64>, g, 3, tm, p, st) : launch(version_fwd_kernel<128>, g, 3, tm, p, st);
+        }
+        case LEVEL_VERSION_BWD: {
+            dim3 g(p.S * p.N, 2);
+            return hd == 64 ? launch(version_bwd_kernel<64>, g, 4, tm, p, st) : launch(version_bwd_kernel<128>, g, 4, tm, p, st);
+        }
+        default: {
+            dim3 g(p.S * p.lv.dy_cnt[p.l]);
+            return hd == 64 ? launch(dyadic_bwd_kernel<64>, g, 5, tm, p, st) : launch(dyadic_bwd_kernel<128>, g, 5, tm, p, st);
+        }
+    }
+}
+
+}  // namespace path

@@ -84,11 +84,11 @@ struct Plan {
     LevelTable lv;
     size_t total;
     // offsets (bytes)
-    size_t status, qp, kp, vp, wp, betap, G, Dy, Xqn, Yt, Qv16, Kv16;
+    size_t status, qp, kp, vp, wp, betap, G, Dyh, Dyl, Xqn, Yt, Qv16, Kv16;
     // backward only
     size_t dop, delta, lse2, dQv, dKv, dSd, dG, dGrow, dGdiag, dDy;
     size_t sTh, sTl, sAh, sAl, sXq, sXk, sY, sU;   // bf16 tiles kept by the chunk preparation for the chain rule
-    size_t dy_bytes;
+    size_t dy_bytes, dy_mats;
 };
 
 static size_t bump(size_t& cur, size_t bytes) {
@@ -127,7 +127,9 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
         p.lv.dy_cnt[l] = p.N >> l;
         if (l == 0 || l <= p.nlev - 2) dy_elems += (size_t)S * (p.N >> l) * d * d;
     }
-    p.Dy = bump(cur, dy_elems * 4);
+    p.Dyh = bump(cur, dy_elems * 2);
+    p.Dyl = bump(cur, dy_elems * 2);
+    p.dy_mats = dy_elems / ((size_t)d * d);
     p.Xqn = bump(cur, SL * CHUNK * 2);
     p.Yt = bump(cur, SL * CHUNK * 2);
     p.Qv16 = bump(cur, SLd * 2 * p.nslot);
@@ -148,22 +150,27 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
 template <class T>
 static T* at(void* ws, size_t off) { return reinterpret_cast<T*>((char*)ws + off); }
 
-static AffineBatch chunk_batch(const Plan& p, long a, long b, long c, long c2, long dd) {
-    // one batch entry per chunk, buffers padded: single stride per pointer
-    AffineBatch ab{};
-    ab.nb1 = 1 << 30;  // z0 = 0, z1 = z
-    ab.a1 = a; ab.b1 = b; ab.c1 = c; ab.c21 = c2; ab.d1 = dd;
-    return ab;
+static bool make_level_maps(const Plan& p, void* ws, LevelTensorMaps& tm) {
+    const uint64_t rows = (uint64_t)p.S * p.Lp * p.nslot;
+    return make_map(&tm.dyh, at<void>(ws, p.Dyh), (uint64_t)p.dy_mats * p.d, p.d) &&
+           make_map(&tm.dyl, at<void>(ws, p.Dyl), (uint64_t)p.dy_mats * p.d, p.d) &&
+           make_map(&tm.qv, at<void>(ws, p.Qv16), rows, p.d) && make_map(&tm.kv, at<void>(ws, p.Kv16), rows, p.d);
+}
+
+static LevelParams level_params(const Plan& p, void* ws) {
+    LevelParams lp{};
+    lp.lv = p.lv; lp.S = p.S; lp.N = p.N; lp.Lp = p.Lp;
+    lp.dyh = at<__nv_bfloat16>(ws, p.Dyh); lp.dyl = at<__nv_bfloat16>(ws, p.Dyl);
+    lp.qv = at<__nv_bfloat16>(ws, p.Qv16); lp.kv = at<__nv_bfloat16>(ws, p.Kv16);
+    if (p.bwd) { lp.dqv = at<float>(ws, p.dQv); lp.dkv = at<float>(ws, p.dKv); lp.ddy = at<float>(ws, p.dDy); }
+    lp.status = at<uint32_t>(ws, p.status);
+    return lp;
 }
 
 // Chunk preparation + dyadic run products + version chains (paper Sec. 3.1, 3.3).  Shared by forward and backward.
 static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const void* w, cudaStream_t st) {
     const int d = p.d, nch = p.S * p.N;
-    const long dd = (long)d * d;
-    float* Dy = at<float>(ws, p.Dy);
-    __nv_bfloat16* Qv16 = at<__nv_bfloat16>(ws, p.Qv16); __nv_bfloat16* Kv16 = at<__nv_bfloat16>(ws, p.Kv16);
-
-    // fused per-chunk kernel: UT transform, boundary-adjusted tiles (version slot 0), chunk products (Dy level 0)
+    // fused per-chunk kernel: UT transform, boundary-adjusted tiles (version slot 0), chunk products (level 0)
     {
         PrepTensorMaps tm;
         const uint64_t rows = (uint64_t)p.S * p.Lp;
@@ -171,41 +178,31 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
             g_last_cuda_error = (int)cudaErrorUnknown;
             return PATH_ERR_LAUNCH;
         }
+        typedef __nv_bfloat16 bf;
         PrepParams pp{};
         pp.beta = at<float>(ws, p.betap);
-        pp.q = (const __nv_bfloat16*)q; pp.k = (const __nv_bfloat16*)k;
-        pp.ql = Qv16; pp.kr = Kv16;
-        pp.Xqn = at<__nv_bfloat16>(ws, p.Xqn); pp.Yt = at<__nv_bfloat16>(ws, p.Yt);
-        pp.P = Dy;
+        pp.q = (const bf*)q; pp.k = (const bf*)k;
+        pp.ql = at<bf>(ws, p.Qv16); pp.kr = at<bf>(ws, p.Kv16);
+        pp.Xqn = at<bf>(ws, p.Xqn); pp.Yt = at<bf>(ws, p.Yt);
+        pp.Ph = at<bf>(ws, p.Dyh); pp.Pl = at<bf>(ws, p.Dyl);
         if (p.bwd) {
-            typedef __nv_bfloat16 bf;
             pp.sTh = at<bf>(ws, p.sTh); pp.sTl = at<bf>(ws, p.sTl); pp.sAh = at<bf>(ws, p.sAh); pp.sAl = at<bf>(ws, p.sAl);
             pp.sXq = at<bf>(ws, p.sXq); pp.sXk = at<bf>(ws, p.sXk); pp.sY = at<bf>(ws, p.sY); pp.sU = at<bf>(ws, p.sU);
         }
         pp.status = at<uint32_t>(ws, p.status);
         LAUNCH(launch_chunk_prep(tm, pp, d, p.bwd, nch, st));
     }
-    // dyadic run products Dy[l+1][b] = Dy[l][2b+1] Dy[l][2b]
-    for (int l = 0; l + 1 <= p.nlev - 2; ++l) {
-        const int cnt = p.N >> l, cnt2 = p.N >> (l + 1);
-        const float* src = Dy + p.lv.dy_off[l];
-        GemmProblem g = gemm_problem(Operand{src + dd, d, 1, 1}, Operand{src, 1, d, 1}, d, d, d);
-        g.C = Dy + p.lv.dy_off[l + 1]; g.c_f32 = 1; g.ldc = d;
-        AffineBatch ab{};
-        ab.nb1 = cnt2;
-        ab.a0 = (long)cnt * dd; ab.a1 = 2 * dd; ab.b0 = ab.a0; ab.b1 = ab.a1;
-        ab.c0 = (long)cnt2 * dd; ab.c1 = dd;
-        LAUNCH(launch_gemm(g, ab, p.S * cnt2, st));
+    if (p.nlev < 2) return PATH_OK;
+    LevelTensorMaps tm;
+    if (!make_level_maps(p, ws, tm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+    LevelParams lp = level_params(p, ws);
+    for (int l = 0; l + 1 <= p.nlev - 2; ++l) {   // run products of 2, 4, ... chunks
+        lp.l = l;
+        LAUNCH(launch_level_kernel(LEVEL_DYADIC_FWD, tm, lp, d, st));
     }
-    // version chains
-    for (int l2 = 1; l2 < p.nlev; ++l2) {
-        for (int is_key = 0; is_key < 2; ++is_key) {
-            VersionBatch v{};
-            v.is_key = is_key; v.mode = 0; v.l2 = l2; v.S = p.S; v.N = p.N; v.Lp = p.Lp; v.d = d; v.lv = p.lv;
-            v.xv = is_key ? Kv16 : Qv16; v.out16 = is_key ? Kv16 : Qv16;
-            v.dy = Dy;
-            LAUNCH(launch_gemm_version(v, st));
-        }
+    for (int l2 = 1; l2 < p.nlev; ++l2) {         // query and key versions, level by level
+        lp.l = l2;
+        LAUNCH(launch_level_kernel(LEVEL_VERSION_FWD, tm, lp, d, st));
     }
     return PATH_OK;
 }
@@ -265,9 +262,8 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
                         const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
                         float* dbeta, float* dlog_f, float scale, cudaStream_t st) {
     const int d = p.d;
-    const long dd = (long)d * d;
     const size_t SLd = (size_t)p.S * p.Lp * d;
-    float* Dy = at<float>(ws, p.Dy); float* dDy = at<float>(ws, p.dDy);
+    float* dDy = at<float>(ws, p.dDy);
     float* dQv = at<float>(ws, p.dQv); float* dKv = at<float>(ws, p.dKv);
 
     prof_mark(STG_ROWSTATS, 0, st);
@@ -305,40 +301,18 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     prof_mark(STG_FA_DQ, 1, st);
     prof_mark(STG_CHAINS, 0, st);
 
-    // version chains, top level first: gradients of the run products, then of the lower versions
-    for (int l2 = p.nlev - 1; l2 >= 1; --l2)
-        for (int is_key = 0; is_key < 2; ++is_key)
-            for (int mode = 2; mode >= 1; --mode) {
-                VersionBatch vb{};
-                vb.is_key = is_key; vb.mode = mode; vb.l2 = l2; vb.S = p.S; vb.N = p.N; vb.Lp = p.Lp; vb.d = d;
-                vb.lv = p.lv;
-                vb.xv = is_key ? at<__nv_bfloat16>(ws, p.Kv16) : at<__nv_bfloat16>(ws, p.Qv16);
-                vb.dxv = is_key ? dKv : dQv;
-                vb.dy = Dy; vb.ddy = dDy;
-                LAUNCH(launch_gemm_version(vb, st));
-            }
-    // run products, top-down: Dy[l][b] = Dy[l-1][2b+1] Dy[l-1][2b]
-    for (int l = p.nlev - 2; l >= 1; --l) {
-        const int cnt = p.N >> l, cntl = p.N >> (l - 1);
-        const float* lo = Dy + p.lv.dy_off[l - 1];
-        float* dlo = dDy + p.lv.dy_off[l - 1];
-        const float* dup = dDy + p.lv.dy_off[l];
-        AffineBatch ab{};
-        ab.nb1 = cnt;
-        ab.a0 = (long)cnt * dd; ab.a1 = dd;
-        ab.b0 = (long)cntl * dd; ab.b1 = 2 * dd;
-        ab.c0 = (long)cntl * dd; ab.c1 = 2 * dd;
-        {   // d(left factor, index 2b+1) += dUp * (right factor)^T
-            GemmProblem g = gemm_problem(Operand{dup, d, 1, 1}, Operand{lo, d, 1, 1}, d, d, d);
-            g.C = dlo + dd; g.c_f32 = 1; g.ldc = d; g.accumulate = ACC_ADD;
-            LAUNCH(launch_gemm(g, ab, p.S * cnt, st));
+    // version chains, top level first, then the run products top-down
+    if (p.nlev >= 2) {
+        LevelTensorMaps ltm;
+        if (!make_level_maps(p, ws, ltm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+        LevelParams lp = level_params(p, ws);
+        for (int l2 = p.nlev - 1; l2 >= 1; --l2) {
+            lp.l = l2;
+            LAUNCH(launch_level_kernel(LEVEL_VERSION_BWD, ltm, lp, d, st));
         }
-        {   // d(right factor, index 2b) += (left factor)^T * dUp
-            AffineBatch ab2 = ab;
-            ab2.a0 = ab.b0; ab2.a1 = ab.b1; ab2.b0 = ab.a0; ab2.b1 = ab.a1;
-            GemmProblem g = gemm_problem(Operand{lo + dd, 1, d, 1}, Operand{dup, 1, d, 1}, d, d, d);
-            g.C = dlo; g.c_f32 = 1; g.ldc = d; g.accumulate = ACC_ADD;
-            LAUNCH(launch_gemm(g, ab2, p.S * cnt, st));
+        for (int l = p.nlev - 2; l >= 1; --l) {
+            lp.l = l;
+            LAUNCH(launch_level_kernel(LEVEL_DYADIC_BWD, ltm, lp, d, st));
         }
     }
     int rc = run_chunk_chain(p, ws, q, k, w, dq, dk, dw, dbeta, scale, st);
