@@ -11,7 +11,8 @@
 // One CTA per chunk runs these ~25 products as tcgen05 MMAs on swizzled shared-memory tiles, in lockstep:
 // thread 0 loads tiles (TMA) and issues MMAs, all 256 threads convert float gradients into tiles and turn
 // accumulators (tensor memory, one row per thread) into the next operand tiles.  T~ and Ainv enter as bf16
-// hi + lo pairs, everything else is rounded to bf16 once; dw accumulates in tensor memory across all phases.
+// hi + lo pairs, and so do the in-kernel intermediates dT, M D and dGm (the lo tile follows the hi tile through
+// the same slot); everything else is rounded to bf16 once.  dw accumulates in tensor memory across all phases.
 #include "tileops.cuh"
 
 namespace path {
@@ -112,6 +113,24 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         }
     };
 
+    // accumulator [128][128] -> f(value, column) -> hi or lo part of its bf16 pair -> tile
+    auto split_to_tile = [&](uint32_t col, uint8_t* dst, bool want_lo, auto&& f) {
+        for (int c = 0; c < 2; ++c) {
+            const int c0 = half * 64 + c * 32;
+            tmem_row32(tl + col + c0, v);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+                const float t = f(v[x], c0 + x);
+                const float h = __bfloat162float(__float2bfloat16_rn(t));
+                v[x] = want_lo ? t - h : h;
+            }
+            tile_store32(dst, row, c0, v);
+        }
+    };
+    auto f_dT = [&](float x, int col) { return col <= row ? x : 0.f; };
+    auto f_tmp = [&](float x, int col) { return x * bt[col]; };
+    auto f_dGm = [&](float x, int col) { return col < row ? -bt[row] * x : 0.f; };
+
     const float* g_dql = p.dql + (size_t)chunk * kT * HD;
     const float* g_dkr = p.dkr + (size_t)chunk * kT * HD;
     const float* g_dsd = p.dsd + (size_t)chunk * kT * kT;
@@ -179,8 +198,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     mma_wait();
     if (!ok) goto done;
-    acc_to_tile(cA, kT, slot(1), 1.f, M_LOWER);                     // dT (over dQl)
-    // ---- phase 3: dXk = strictLower(T~^T dY),  dw += T~^T dU   (hi, then lo through the same slot)
+    // dT stays in tensor memory (cA); its bf16 hi part goes to slot 1 now, the lo part follows in phase 4
+    split_to_tile(cA, slot(1), false, f_dT);
+    // ---- phase 3: dXk = strictLower(T~^T dY) -> cB,  dw += T~^T dU   (hi, then lo through the same slot)
     for (int part = 0; part < 2; ++part) {
         if (tid == 0) {
             mbar_expect_tx(&bars[0], kTileB);
@@ -190,20 +210,20 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         publish();
         if (tid == 0) {
             tc_fence_after_sync();
-            mma(tmem + cA, sa(2), OP_MN, sa(5), OP_MN, K8, 128, part > 0);
+            mma(tmem + cB, sa(2), OP_MN, sa(5), OP_MN, K8, 128, part > 0);
             mma(tmem + cDW, sa(2), OP_MN, sa(6), OP_MN, K8, HD, true);
             umma_commit(&bars[1]);
         }
         mma_wait();
         if (!ok) goto done;
     }
-    // ---- phase 4: M = Ainv^T dT;  dbeta_c = M_cc;  tmp = M D;  dA = strictLower(-tmp Ainv^T)
+    // ---- phase 4: M = Ainv^T dT -> cB;  dbeta_c = M_cc;  tmp = M D;  dA = strictLower(-tmp Ainv^T) -> cA
     if (tid == 0) {
         mbar_expect_tx(&bars[0], 2 * kTileB);
         tma_tile(slot(2), &tm.ah, &bars[0], kT, r0);
         tma_tile(slot(6), &tm.al, &bars[0], kT, r0);
     }
-    acc_to_tile(cA, kT, slot(5), 1.f, M_STRICT);                    // dXk (over dY)
+    acc_to_tile(cB, kT, slot(5), 1.f, M_STRICT);                    // dXk (over dY)
     loads_wait();
     publish();
     if (tid == 0) {
@@ -214,16 +234,25 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     mma_wait();
     if (!ok) goto done;
-    for (int c = 0; c < 2; ++c) {                                   // tmp = M D (over dT), diagonal -> t1
-        const int c0 = half * 64 + c * 32;
-        tmem_row32(tl + cB + c0, v);
-#pragma unroll
-        for (int x = 0; x < 32; ++x) {
-            if (c0 + x == row) t1[row] = v[x];
-            v[x] *= bt[c0 + x];
-        }
-        tile_store32(slot(1), row, c0, v);
+    split_to_tile(cA, slot(1), true, f_dT);                         // dT lo
+    publish();
+    if (tid == 0) {
+        tc_fence_after_sync();
+        mma(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, 128, true);
+        umma_commit(&bars[1]);
     }
+    mma_wait();
+    if (!ok) goto done;
+    {   // diagonal of M -> t1
+        const int c0 = (row >> 5) << 5;
+        if ((c0 >> 6) == half) {
+            tmem_row32(tl + cB + c0, v);
+#pragma unroll
+            for (int x = 0; x < 32; ++x)
+                if (c0 + x == row) t1[row] = v[x];
+        }
+    }
+    split_to_tile(cB, slot(1), false, f_tmp);                       // tmp = M D, hi
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
@@ -233,21 +262,25 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     mma_wait();
     if (!ok) goto done;
-    {   // dA = strictLower(-acc);  dbeta_r = t1_r + sum_c dA_rc Gm_rc;  dGm = D dA -> tile (over tmp)
+    split_to_tile(cB, slot(1), true, f_tmp);                        // tmp lo
+    publish();
+    if (tid == 0) {
+        tc_fence_after_sync();
+        mma(tmem + cA, sa(1), OP_K, sa(2), OP_K, K8, 128, true);
+        umma_commit(&bars[1]);
+    }
+    mma_wait();
+    if (!ok) goto done;
+    {   // dA = strictLower(-cA);  dbeta_r = t1_r + sum_c dA_rc Gm_rc
         float part = 0.f;
-        const float b = bt[row];
         for (int c = 0; c < 2; ++c) {
             const int c0 = half * 64 + c * 32;
             float gm[32];
             tmem_row32(tl + cA + c0, v);
             tmem_row32(tl + cG + c0, gm);
 #pragma unroll
-            for (int x = 0; x < 32; ++x) {
-                const float da = (c0 + x < row) ? -v[x] : 0.f;
-                part += da * gm[x];
-                v[x] = b * da;
-            }
-            tile_store32(slot(1), row, c0, v);
+            for (int x = 0; x < 32; ++x)
+                if (c0 + x < row) part -= v[x] * gm[x];
         }
         // the two threads of a row add their halves through shared memory
         __syncthreads();
@@ -255,7 +288,8 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         __syncthreads();
         if (half == 0 && row_valid) p.dbeta[urow] = t1[row] + part;
     }
-    // ---- phase 5: dq, dk and the rest of dw
+    split_to_tile(cA, slot(1), false, f_dGm);                       // dGm = D dA, hi
+    // ---- phase 5: dq -> cB, dk -> cG and the rest of dw
     if (tid == 0) {
         mbar_expect_tx(&bars[0], 2 * kT * HD * 2);
         tma_tile(slot(2), &tm.k, &bars[0], HD, r0);
@@ -265,10 +299,10 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma(tmem + cA, sa(3), OP_K, sa(2), OP_MN, K8, HD, false);    // s dSd K
-        mma(tmem + cA, sa(4), OP_K, sa(0), OP_MN, K8, HD, true);     // dXq W
-        mma(tmem + cB, sa(3), OP_MN, sa(6), OP_MN, K8, HD, false);   // s dSd^T Q
-        mma(tmem + cB, sa(5), OP_MN, sa(0), OP_MN, K8, HD, true);    // dXk^T W
+        mma(tmem + cB, sa(3), OP_K, sa(2), OP_MN, K8, HD, false);    // s dSd K
+        mma(tmem + cB, sa(4), OP_K, sa(0), OP_MN, K8, HD, true);     // dXq W
+        mma(tmem + cG, sa(3), OP_MN, sa(6), OP_MN, K8, HD, false);   // s dSd^T Q
+        mma(tmem + cG, sa(5), OP_MN, sa(0), OP_MN, K8, HD, true);    // dXk^T W
         mma(tmem + cDW, sa(4), OP_MN, sa(6), OP_MN, K8, HD, true);   // dXq^T Q
         mma(tmem + cDW, sa(5), OP_K, sa(2), OP_MN, K8, HD, true);    // dXk K
         mma(tmem + cDW, sa(1), OP_K, sa(0), OP_MN, K8, HD, true);    // dGm W
@@ -277,15 +311,25 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     mma_wait();
     if (!ok) goto done;
+    split_to_tile(cA, slot(1), true, f_dGm);                        // dGm lo
+    publish();
+    if (tid == 0) {
+        tc_fence_after_sync();
+        mma(tmem + cDW, sa(1), OP_K, sa(0), OP_MN, K8, HD, true);
+        mma(tmem + cDW, sa(1), OP_MN, sa(0), OP_MN, K8, HD, true);
+        umma_commit(&bars[1]);
+    }
+    mma_wait();
+    if (!ok) goto done;
     for (int c = 0; c < HD / 64; ++c) {
         const int c0 = half * (HD / 2) + c * 32;
         float in[32];
-        tmem_row32(tl + cA + c0, v);
+        tmem_row32(tl + cB + c0, v);
         gload_f32x32(g_dql + (size_t)row * HD + c0, in);
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] += in[x];
         if (row_valid) gstore_bf16x32(p.dq + urow * HD + c0, v);
-        tmem_row32(tl + cB + c0, v);
+        tmem_row32(tl + cG + c0, v);
         gload_f32x32(g_dkr + (size_t)row * HD + c0, in);
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] += in[x];

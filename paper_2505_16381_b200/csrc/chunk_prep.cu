@@ -23,17 +23,19 @@ namespace {
 using namespace tile;
 constexpr int kLd = kT + 1;  // row stride of the float32 triangular buffer
 
+// Seven 32 KB tile slots.  0: W.  1, 2: Q, K -> T~ hi, lo -> U hi, lo.  3..6: float32 triangular buffer and its
+// scratch -> Xq hi, lo, Xk hi, lo -> (5, 6) Y hi, lo.
 struct PrepSmem {
     static constexpr uint32_t offW = 0;
-    static constexpr uint32_t offQK = offW + kTileB;            // Q, K  ->  T hi, T lo  ->  U, Y
-    static constexpr uint32_t offBig = offQK + 2 * kTileB;      // float32 triangular buffer  ->  Xq, Xk tiles
-    static constexpr uint32_t bigBytes = ((kT * kLd * 4 + 1023) / 1024) * 1024;
-    static constexpr uint32_t offDiag = offBig + bigBytes;      // [8][16][17] float
-    static constexpr uint32_t offZ = offDiag + 8 * 16 * 17 * 4; // [16][128] float
-    static constexpr uint32_t offBeta = offZ + 16 * kT * 4;     // [128] float
-    static constexpr uint32_t offBar = offBeta + kT * 4;
+    static constexpr uint32_t offQK = kTileB;
+    static constexpr uint32_t offBig = 3 * kTileB;
+    static constexpr uint32_t offDiag = offBig + ((kT * kLd * 4 + 1023) / 1024) * 1024;   // [8][16][17] float
+    static constexpr uint32_t offZ = offDiag + 8 * 16 * 17 * 4;                            // [16][128] float
+    static constexpr uint32_t offBeta = offZ + 16 * kT * 4;                                // [128] float
+    static constexpr uint32_t offBar = 7 * kTileB;
     static constexpr uint32_t total = offBar + 64;
     static constexpr uint32_t alloc = total + 1024;
+    static_assert(offBeta + kT * 4 <= offBar, "scratch must fit in the tile slots it aliases");
 };
 
 template <int HD, bool SAVE>
@@ -184,14 +186,20 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
     }
     __syncthreads();  // everyone has read the float32 buffer; it now becomes the Xq / Xk tiles
 
-    // ---- E1b: Xq = lower(.), Xk = strictLower(.) -> bf16 tiles; Xqn = -Xq -> global
+    // ---- E1b: Xq = lower(.), Xk = strictLower(.) -> bf16 hi / lo tiles (slots 3..6); Xqn = -Xq -> global
     for (int c = 0; c < 2; ++c) {
         const int c0 = half * 64 + c * 32;
+        float lo[32];
         tmem_ld32(tl + 128 + c0, r);
         tmem_ld_wait();
 #pragma unroll
-        for (int x = 0; x < 32; ++x) v[x] = (c0 + x <= row) ? __uint_as_float(r[x]) : 0.f;
+        for (int x = 0; x < 32; ++x) {
+            const float t = (c0 + x <= row) ? __uint_as_float(r[x]) : 0.f;
+            v[x] = __bfloat162float(__float2bfloat16_rn(t));
+            lo[x] = t - v[x];
+        }
         tile_store32(sBig, row, c0, v);
+        tile_store32(sBig + kTileB, row, c0, lo);
         if (SAVE) gstore_bf16x32(p.sXq + grow * kT + c0, v);
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] = -v[x];
@@ -199,19 +207,25 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
         tmem_ld32(tl + 256 + c0, r);
         tmem_ld_wait();
 #pragma unroll
-        for (int x = 0; x < 32; ++x) v[x] = (c0 + x < row) ? __uint_as_float(r[x]) : 0.f;
-        tile_store32(sBig + kTileB, row, c0, v);
+        for (int x = 0; x < 32; ++x) {
+            const float t = (c0 + x < row) ? __uint_as_float(r[x]) : 0.f;
+            v[x] = __bfloat162float(__float2bfloat16_rn(t));
+            lo[x] = t - v[x];
+        }
+        tile_store32(sBig + 2 * kTileB, row, c0, v);
+        tile_store32(sBig + 3 * kTileB, row, c0, lo);
         if (SAVE) gstore_bf16x32(p.sXk + grow * kT + c0, v);
     }
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0) {   // group 2: U = T~ W -> col 0, Y = T~ Xk -> col 128
+    if (tid == 0) {   // group 2: U = T~ W -> col 0, Y = T~ Xk -> col 128 (lo x lo terms dropped)
         tc_fence_after_sync();
         mma(tmem + 0, aQ, OP_K, aW, OP_MN, 8, HD, false);
         mma(tmem + 0, aK, OP_K, aW, OP_MN, 8, HD, true);
-        mma(tmem + 128, aQ, OP_K, aBig + kTileB, OP_MN, 8, 128, false);
-        mma(tmem + 128, aK, OP_K, aBig + kTileB, OP_MN, 8, 128, true);
+        mma(tmem + 128, aQ, OP_K, aBig + 2 * kTileB, OP_MN, 8, 128, false);
+        mma(tmem + 128, aK, OP_K, aBig + 2 * kTileB, OP_MN, 8, 128, true);
+        mma(tmem + 128, aQ, OP_K, aBig + 3 * kTileB, OP_MN, 8, 128, true);
         umma_commit(&bars[1]);
     }
     __syncwarp();
@@ -220,23 +234,35 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
     tc_fence_after_sync();
     if (!ok) goto done;
 
-    // ---- E2: U, Y -> bf16 tiles over T~ (dead now); Yt = Y^T -> global
+    // ---- E2: U -> hi / lo tiles over T~ (slots 1, 2); Y -> hi / lo tiles over Xk (slots 5, 6); Yt = Y^T -> global
     for (int c = 0; c < HD / 64; ++c) {
         const int c0 = half * (HD / 2) + c * 32;
+        float lo[32];
         tmem_ld32(tl + 0 + c0, r);
         tmem_ld_wait();
 #pragma unroll
-        for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
+        for (int x = 0; x < 32; ++x) {
+            const float t = __uint_as_float(r[x]);
+            v[x] = __bfloat162float(__float2bfloat16_rn(t));
+            lo[x] = t - v[x];
+        }
         tile_store32(sQK, row, c0, v);
+        tile_store32(sQK + kTileB, row, c0, lo);
         if (SAVE) gstore_bf16x32(p.sU + grow * HD + c0, v);
     }
     for (int c = 0; c < 2; ++c) {
         const int c0 = half * 64 + c * 32;
+        float lo[32];
         tmem_ld32(tl + 128 + c0, r);
         tmem_ld_wait();
 #pragma unroll
-        for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
-        tile_store32(sQK + kTileB, row, c0, v);
+        for (int x = 0; x < 32; ++x) {
+            const float t = __uint_as_float(r[x]);
+            v[x] = __bfloat162float(__float2bfloat16_rn(t));
+            lo[x] = t - v[x];
+        }
+        tile_store32(sBig + 2 * kTileB, row, c0, v);
+        tile_store32(sBig + 3 * kTileB, row, c0, lo);
         if (SAVE) gstore_bf16x32(p.sY + grow * kT + c0, v);
         __nv_bfloat16* yt = p.Yt + ((size_t)chunk * kT + c0) * kT + row;
 #pragma unroll
@@ -248,8 +274,12 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
     if (tid == 0) {   // group 3: Xq U -> col 256, Y^T W -> col 384, W^T U -> col 0
         tc_fence_after_sync();
         mma(tmem + 256, aBig, OP_K, aQ, OP_MN, 8, HD, false);
-        mma(tmem + 384, aK, OP_MN, aW, OP_MN, 8, HD, false);
+        mma(tmem + 256, aBig + kTileB, OP_K, aQ, OP_MN, 8, HD, true);
+        mma(tmem + 256, aBig, OP_K, aK, OP_MN, 8, HD, true);
+        mma(tmem + 384, aBig + 2 * kTileB, OP_MN, aW, OP_MN, 8, HD, false);
+        mma(tmem + 384, aBig + 3 * kTileB, OP_MN, aW, OP_MN, 8, HD, true);
         mma(tmem + 0, aW, OP_MN, aQ, OP_MN, 8, HD, false);
+        mma(tmem + 0, aW, OP_MN, aK, OP_MN, 8, HD, true);
         umma_commit(&bars[1]);
     }
     __syncwarp();
