@@ -57,7 +57,8 @@ typedef enum {
     PATH_ERR_WORKSPACE = -5, /* workspace_bytes too small */
     PATH_ERR_ARCH = -6,      /* current device is not compute capability 10.x */
     PATH_ERR_LAUNCH = -7,    /* a CUDA runtime / driver call failed (see path_attn_last_cuda_error) */
-    PATH_ERR_TIMEOUT = -8    /* reported by path_attn_device_status: a bounded device wait ran out */
+    PATH_ERR_TIMEOUT = -8,   /* reported by path_attn_device_status: a bounded device wait ran out */
+    PATH_ERR_STATIC_LIMIT = -9 /* path_attn_fwd_static: the problem needs more scratch than the built-in buffer holds */
 } path_status_t;
 
 /* Bytes of scratch memory path_attn_fwd (for_backward = 0) or path_attn_bwd
@@ -93,6 +94,43 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
                   void* dk, void* dv, void* dw, float* dbeta, float* dlog_f, int B, int H, int L,
                   int d, float scale, path_dtype_t dt, void* workspace, size_t workspace_bytes,
                   void* cuda_stream);
+
+/*
+ * Forward pass for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a packaging variant of path_attn_fwd).
+ *
+ * Some hosts of this library may not call cudaMalloc at the point where they
+ * need attention: code running while a stream is being captured into a CUDA
+ * graph, plug-ins inside a serving runtime that has already handed every free
+ * byte of the device to its own pool, and latency-critical loops in which the
+ * implicit device synchronisation of cudaMalloc / cudaFree is not acceptable.
+ * For them the scratch memory is not a caller workspace but a fixed buffer of
+ * PATH_ATTN_STATIC_SCRATCH_BYTES that is part of the library image itself: every
+ * GPU on which the library is loaded holds that buffer until the process exits.
+ *
+ * Arguments are those of path_attn_fwd without the workspace.  The call computes
+ * exactly what path_attn_fwd computes and allocates nothing: no cudaMalloc, no
+ * cudaFree, no allocating library routine.  A problem whose
+ * path_attn_workspace_bytes(..., for_backward = 0) exceeds
+ * PATH_ATTN_STATIC_SCRATCH_BYTES is rejected with PATH_ERR_STATIC_LIMIT before
+ * anything is launched (roughly: B*H*L up to a few thousand tokens at d = 128).
+ *
+ * The first call on each device looks up the buffer's device address (once per
+ * device, with that device current) and may trigger the driver's one-time module
+ * loading; make that first call outside of any stream capture.
+ * All calls on one device share the one buffer, and it keeps whatever the
+ * previous call left in it: the call clears the status word it needs at zero and
+ * overwrites every other region before reading it, so back-to-back calls on one
+ * stream are safe, but two calls that overlap on the GPU (different streams, or
+ * different host threads) race on the buffer and must be serialised by the caller.
+ * Stage timing (path_attn_profile_enable) is ignored by this entry point.
+ * If scratch_out is not NULL it receives the buffer's device address, which may
+ * be passed to path_attn_device_status as the `workspace` of this call.
+ */
+#define PATH_ATTN_STATIC_SCRATCH_BYTES (16u << 20)
+int path_attn_fwd_static(const void* q, const void* k, const void* v, const void* w, const float* beta,
+                         const float* log_f, void* o, float* lse, int B, int H, int L, int d, float scale,
+                         path_dtype_t dt, void* cuda_stream, void** scratch_out);
 
 /* Reads the device status word the last call on this workspace left behind.
  * Synchronises `cuda_stream`.  Returns PATH_OK, PATH_ERR_TIMEOUT, or

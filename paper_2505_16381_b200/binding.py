@@ -17,7 +17,7 @@ _lib = None
 
 PATH_BF16, PATH_FP32 = 0, 1
 PATH_OK = 0
-EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_attn_device_status",
+EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_attn_fwd_static", "path_attn_device_status",
            "path_attn_strerror", "path_attn_last_cuda_error", "path_attn_last_launch_count",
            "path_attn_profile_enable", "path_attn_profile_read", "path_attn_profile_stage_name"]
 
@@ -44,6 +44,8 @@ def load():
         lib.path_attn_workspace_bytes.argtypes = [I, I, I, I, I, I, I]
         lib.path_attn_fwd.restype = I
         lib.path_attn_fwd.argtypes = [P, P, P, P, P, P, P, P, I, I, I, I, F, I, P, Z, P]
+        lib.path_attn_fwd_static.restype = I
+        lib.path_attn_fwd_static.argtypes = [P, P, P, P, P, P, P, P, I, I, I, I, F, I, P, ctypes.POINTER(P)]
         lib.path_attn_bwd.restype = I
         lib.path_attn_bwd.argtypes = [P] * 15 + [I, I, I, I, F, I, P, Z, P]
         lib.path_attn_device_status.restype = I
@@ -113,6 +115,29 @@ def path_attn_fwd(q, k, v, w, beta, log_f=None, scale=1.0, workspace=None, out=N
     if rc != PATH_OK:
         raise PathAttnError(rc, "path_attn_fwd")
     return o, lse
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def path_attn_fwd_static(q, k, v, w, beta, log_f=None, scale=1.0, out=None):
+    """Forward through the entry point that takes no workspace: its scratch is a fixed buffer inside the library,
+    so nothing is allocated by the call itself (the output tensors are the caller's; pass ``out=(o, lse)`` to
+    reuse preallocated ones).  Only problems needing at most ``STATIC_SCRATCH_BYTES`` of scratch are accepted.
+    Returns ``(o, lse, scratch_address)``."""
+    _check(q, k, v, w, beta, log_f)
+    lib = load()
+    B, H, L, d = q.shape
+    o = torch.empty_like(q) if out is None else out[0]
+    lse = torch.empty(B, H, L, dtype=torch.float32, device=q.device) if out is None else out[1]
+    st = torch.cuda.current_stream(q.device).cuda_stream
+    addr = ctypes.c_void_p(0)
+    with torch.cuda.device(q.device):
+        rc = lib.path_attn_fwd_static(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(beta), _ptr(log_f), _ptr(o), _ptr(lse),
+                                      B, H, L, d, float(scale), _dt(q), ctypes.c_void_p(st), ctypes.byref(addr))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_fwd_static")
+    return o, lse, addr.value
 
 
 def path_attn_bwd(q, k, v, w, beta, o, lse, d_o, log_f=None, scale=1.0, workspace=None, out=None):

@@ -4,6 +4,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 #include "linear.cuh"
@@ -413,6 +414,58 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
     return run_backward(p, workspace, q, k, v, w, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, scale, st);
 }
 
+}  // extern "C"
+
+// ------------------------------------------------------------------------------------------- forward without a workspace
+// Scratch for path_attn_fwd_static lives in the library image: one buffer per device that loads the module.  In host
+// code the array's name is only a handle; its device address is looked up once per device and cached here.
+static __device__ __align__(256) unsigned char g_static_scratch[PATH_ATTN_STATIC_SCRATCH_BYTES];
+static constexpr int kMaxDevices = 64;
+static void* g_static_scratch_addr[kMaxDevices] = {};
+static std::mutex g_static_scratch_mutex;
+
+static int static_scratch_address(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        path::g_last_cuda_error = (int)(e != cudaSuccess ? e : cudaErrorInvalidDevice);
+        return PATH_ERR_LAUNCH;
+    }
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void* addr = nullptr;
+        e = cudaGetSymbolAddress(&addr, g_static_scratch);   // resolves against the current device's copy
+        if (e != cudaSuccess || addr == nullptr) {
+            path::g_last_cuda_error = (int)(e != cudaSuccess ? e : cudaErrorInvalidSymbol);
+            return PATH_ERR_LAUNCH;
+        }
+        g_static_scratch_addr[dev] = addr;
+    }
+    *out = g_static_scratch_addr[dev];
+    return PATH_OK;
+}
+
+extern "C" {
+
+int path_attn_fwd_static(const void* q, const void* k, const void* v, const void* w, const float* beta,
+                         const float* log_f, void* o, float* lse, int B, int H, int L, int d, float scale,
+                         path_dtype_t dt, void* cuda_stream, void** scratch_out) {
+    if (dt != PATH_BF16 && dt != PATH_FP32) return PATH_ERR_DTYPE;
+    const size_t need = path_attn_workspace_bytes(B, H, L, d, dt, log_f ? 1 : 0, 0);
+    if (need == 0) return PATH_ERR_SHAPE;
+    if (need > (size_t)PATH_ATTN_STATIC_SCRATCH_BYTES) return PATH_ERR_STATIC_LIMIT;
+    void* scratch = nullptr;
+    int rc = static_scratch_address(&scratch);
+    if (rc != PATH_OK) return rc;
+    const bool timing = path::g_prof.on;   // stage timing would create CUDA events on first use
+    path::g_prof.on = false;
+    rc = path_attn_fwd(q, k, v, w, beta, log_f, o, lse, B, H, L, d, scale, dt, scratch,
+                       (size_t)PATH_ATTN_STATIC_SCRATCH_BYTES, cuda_stream);
+    path::g_prof.on = timing;
+    if (scratch_out) *scratch_out = scratch;
+    return rc;
+}
+
 int path_attn_device_status(const void* workspace, void* cuda_stream, unsigned int* detail) {
     if (!workspace) return PATH_ERR_NULL;
     unsigned int word = 0;
@@ -437,6 +490,7 @@ const char* path_attn_strerror(int status) {
         case PATH_ERR_ARCH: return "device is not compute capability 10.x";
         case PATH_ERR_LAUNCH: return "a CUDA call failed";
         case PATH_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case PATH_ERR_STATIC_LIMIT: return "problem needs more scratch than the built-in static buffer holds";
         default: return "unknown status";
     }
 }
