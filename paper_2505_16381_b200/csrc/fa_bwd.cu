@@ -245,6 +245,10 @@ __global__ void __launch_bounds__(192, 1) dkv_kernel(const __grid_constant__ Bwd
         tc_fence_after_sync();
         if (ok) {
             if (T > 1) flush_dk(level(T - 1));
+            else {  // last chunk: no later query chunk, the boundary-adjusted keys get a zero gradient from the sweep
+                float4* dst = reinterpret_cast<float4*>(p.dkv + ((size_t)ver_row(0, J) + row) * HD);
+                for (int x = 0; x < HD / 4; ++x) dst[x] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
             for (int c = 0; c < HD / 32; ++c) {
                 tmem_ld32(tlane + colDV + c * 32, rs);
                 tmem_ld_wait();
@@ -277,7 +281,11 @@ enum { Q_QFULL = 0, Q_QEMPTY, Q_DOFULL, Q_KFULL, Q_KEMPTY = Q_KFULL + 2, Q_VFULL
 template <int HD, bool GATE>
 __global__ void __launch_bounds__(192, 1) dq_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
     const int I = (int)gridDim.x - 1 - (int)blockIdx.x, s = blockIdx.y;
-    if (I == 0) return;  // chunk 0 has no earlier keys; its row block of the gradient buffer was zeroed
+    if (I == 0) {  // chunk 0 has no earlier keys: its boundary-adjusted queries get a zero gradient from the sweep
+        float4* dst = reinterpret_cast<float4*>(p.dqv + (size_t)s * p.Lp * HD);
+        for (int i = threadIdx.x; i < kTile * HD / 4; i += blockDim.x) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;

@@ -263,7 +263,24 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
     mma_wait(c);
     if (c.ok) {
         acc_add_global<false>(c, 0, HD, kT, dxv + (size_t)row_src * HD);
-        acc_add_global<true>(c, 128, HD, HD, p.ddy + (size_t)mat * HD * HD);
+        // run-product gradient: stage the [d][d] accumulator in shared memory (the tiles are dead) so that the
+        // atomic adds of a warp fall on consecutive addresses
+        constexpr int LDS = HD + 4;
+        float* stage = (float*)sm;
+        float v[32];
+        for (int i = 0; i < HD / 64; ++i) {
+            const int c0 = c.half * (HD / 2) + i * 32;
+            tmem_row32(c.tl + 128 + c0, v);
+            if (c.row < HD) {
+#pragma unroll
+                for (int x = 0; x < 8; ++x)
+                    *reinterpret_cast<float4*>(stage + c.row * LDS + c0 + 4 * x) =
+                        make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
+            }
+        }
+        __syncthreads();
+        float* dst = p.ddy + (size_t)mat * HD * HD;
+        for (int idx = c.tid; idx < HD * HD; idx += 256) atomicAdd(dst + idx, stage[(idx / HD) * LDS + (idx % HD)]);
     }
     teardown<256>(c, p.status);
 }

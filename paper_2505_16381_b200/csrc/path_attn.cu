@@ -263,7 +263,6 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
                         const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
                         float* dbeta, float* dlog_f, float scale, cudaStream_t st) {
     const int d = p.d;
-    const size_t SLd = (size_t)p.S * p.Lp * d;
     float* dDy = at<float>(ws, p.dDy);
     float* dQv = at<float>(ws, p.dQv); float* dKv = at<float>(ws, p.dKv);
 
@@ -274,8 +273,6 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
         LAUNCH(launch_pad_rows(d_o, at<void>(ws, p.dop), p.S, p.L, p.Lp, d, 0, st));
         dop = at<void>(ws, p.dop);
     }
-    CK(cudaMemsetAsync(dQv, 0, SLd * 4 * p.nslot, st));
-    CK(cudaMemsetAsync(dKv, 0, SLd * 4 * p.nslot, st));
     CK(cudaMemsetAsync(dDy, 0, p.dy_bytes, st));
     if (p.gate) CK(cudaMemsetAsync(at<float>(ws, p.dGrow), 0, (size_t)p.S * p.Lp * 4, st));
 
