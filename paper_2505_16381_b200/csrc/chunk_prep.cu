@@ -21,7 +21,7 @@ using namespace tc5;
 namespace {
 
 using namespace tile;
-constexpr int kLd = kT + 1;  // row stride of the float32 triangular buffer
+constexpr int kLd = kT + 4;  // row stride of the float32 triangular buffer (rows stay 16-byte aligned)
 
 // Seven 32 KB tile slots.  0: W.  1, 2: Q, K -> T~ hi, lo -> U hi, lo.  3..6: float32 triangular buffer and its
 // scratch -> Xq hi, lo, Xk hi, lo -> (5, 6) Y hi, lo.
@@ -81,6 +81,7 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
     bool ok = true;
     uint32_t r[32];
     float v[32];
+    uint4 pre_q[HD / 64][4], pre_k[HD / 64][4];
 
     if (tid == 0) {
         mbar_expect_tx(&bars[0], 3 * kT * HD * 2);
@@ -111,21 +112,25 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
         tmem_ld_wait();
         const float b = bt[row];
 #pragma unroll
-        for (int x = 0; x < 32; ++x) {
-            v[x] = __uint_as_float(r[x]);
-            Xb[row * kLd + c0 + x] = (c0 + x < row) ? b * v[x] : 0.f;
-        }
+        for (int x = 0; x < 32; ++x) v[x] = (c0 + x < row) ? b * __uint_as_float(r[x]) : 0.f;
+#pragma unroll
+        for (int x = 0; x < 8; ++x)
+            *reinterpret_cast<float4*>(Xb + row * kLd + c0 + 4 * x) = make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
     }
     __syncthreads();
 
     // ---- (I + Nl)^-1 in place, 16-row panels
-    if (lane < 16) {   // diagonal blocks: warp w inverts block w, lane j owns column j
+    if (lane < 16) {   // diagonal blocks: warp w inverts block w by forward substitution, lane j keeps column j in registers
         const int o = warp * 16, j = lane;
         float* dx = diagX + warp * 16 * 17;
+        float x[16];
+#pragma unroll
         for (int rr = 0; rr < 16; ++rr) {
             float acc = (rr == j) ? 1.f : 0.f;
-            for (int c = j; c < rr; ++c) acc -= Xb[(o + rr) * kLd + o + c] * dx[c * 17 + j];
-            dx[rr * 17 + j] = (rr >= j) ? acc : 0.f;
+#pragma unroll
+            for (int c = 0; c < rr; ++c) acc -= Xb[(o + rr) * kLd + o + c] * x[c];
+            x[rr] = (rr >= j) ? acc : 0.f;
+            dx[rr * 17 + j] = x[rr];
         }
     }
     __syncthreads();
@@ -133,25 +138,49 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
         const int R = bi * 16;
         const float* dx = diagX + bi * 16 * 17;
         if (bi > 0) {
+            // Z = Nl[panel, <R] X[<R, <R]: each thread 4 rows x 1 column, 4 contraction steps per iteration
             for (int idx = tid; idx < 4 * R; idx += 256) {
                 const int rg = idx / R, c = idx - rg * R;
                 float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
                 const float* n0 = Xb + (R + rg) * kLd;
-                for (int k = (c & ~15); k < R; ++k) {
-                    const float x = Xb[k * kLd + c];
-                    a0 += n0[k] * x;
-                    a1 += n0[4 * kLd + k] * x;
-                    a2 += n0[8 * kLd + k] * x;
-                    a3 += n0[12 * kLd + k] * x;
+                for (int k = (c & ~15); k < R; k += 4) {
+                    const float x0 = Xb[k * kLd + c], x1 = Xb[(k + 1) * kLd + c], x2 = Xb[(k + 2) * kLd + c],
+                                x3 = Xb[(k + 3) * kLd + c];
+                    const float4 na = *reinterpret_cast<const float4*>(n0 + k);
+                    const float4 nb = *reinterpret_cast<const float4*>(n0 + 4 * kLd + k);
+                    const float4 nc = *reinterpret_cast<const float4*>(n0 + 8 * kLd + k);
+                    const float4 nd = *reinterpret_cast<const float4*>(n0 + 12 * kLd + k);
+                    a0 += na.x * x0 + na.y * x1 + na.z * x2 + na.w * x3;
+                    a1 += nb.x * x0 + nb.y * x1 + nb.z * x2 + nb.w * x3;
+                    a2 += nc.x * x0 + nc.y * x1 + nc.z * x2 + nc.w * x3;
+                    a3 += nd.x * x0 + nd.y * x1 + nd.z * x2 + nd.w * x3;
                 }
                 Z[rg * kT + c] = a0; Z[(rg + 4) * kT + c] = a1; Z[(rg + 8) * kT + c] = a2; Z[(rg + 12) * kT + c] = a3;
             }
             __syncthreads();
-            for (int idx = tid; idx < 16 * R; idx += 256) {
-                const int rr = idx / R, c = idx - rr * R;
-                float acc = 0.f;
-                for (int k = 0; k <= rr; ++k) acc -= dx[rr * 17 + k] * Z[k * kT + c];
-                Xb[(R + rr) * kLd + c] = acc;
+            // X[panel, <R] = -X[panel, panel] Z: two threads per column (rows 0..10 and 11..15: equal work)
+            for (int idx = tid; idx < 2 * R; idx += 256) {
+                const int h = idx / R, c = idx - h * R;
+                float z[16];
+#pragma unroll
+                for (int k = 0; k < 16; ++k) z[k] = Z[k * kT + c];
+                if (h == 0) {
+#pragma unroll
+                    for (int rr = 0; rr <= 10; ++rr) {
+                        float acc = 0.f;
+#pragma unroll
+                        for (int k = 0; k <= rr; ++k) acc -= dx[rr * 17 + k] * z[k];
+                        Xb[(R + rr) * kLd + c] = acc;
+                    }
+                } else {
+#pragma unroll
+                    for (int rr = 11; rr < 16; ++rr) {
+                        float acc = 0.f;
+#pragma unroll
+                        for (int k = 0; k <= rr; ++k) acc -= dx[rr * 17 + k] * z[k];
+                        Xb[(R + rr) * kLd + c] = acc;
+                    }
+                }
             }
         }
         { const int rr = tid >> 4, k = tid & 15; Xb[(R + rr) * kLd + R + k] = dx[rr * 17 + k]; }
@@ -163,8 +192,13 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
         const int c0 = half * 64 + c * 32;
         float hi[32], lo[32];
 #pragma unroll
+        for (int x = 0; x < 8; ++x) {
+            const float4 f = *reinterpret_cast<const float4*>(Xb + row * kLd + c0 + 4 * x);
+            v[4 * x] = f.x; v[4 * x + 1] = f.y; v[4 * x + 2] = f.z; v[4 * x + 3] = f.w;
+        }
+#pragma unroll
         for (int x = 0; x < 32; ++x) {
-            const float xv = Xb[row * kLd + c0 + x];
+            const float xv = v[x];
             const float t = xv * bt[c0 + x];
             v[x] = xv;
             hi[x] = __bfloat162float(__float2bfloat16_rn(t));
@@ -283,6 +317,16 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
         umma_commit(&bars[1]);
     }
     __syncwarp();
+    // the q / k rows of the final subtraction are fetched while the MMAs run
+#pragma unroll
+    for (int c = 0; c < HD / 64; ++c) {
+        const int c0 = half * (HD / 2) + c * 32;
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            pre_q[c][x] = reinterpret_cast<const uint4*>(p.q + grow * HD + c0)[x];
+            pre_k[c][x] = reinterpret_cast<const uint4*>(p.k + grow * HD + c0)[x];
+        }
+    }
     if (!mbar_wait(&bars[1], 0, abort_flag, ST_PREP)) ok = false;
     ok = __syncthreads_and(ok);
     tc_fence_after_sync();
@@ -294,13 +338,13 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
         float in[32];
         tmem_ld32(tl + 256 + c0, r);
         tmem_ld_wait();
-        gload_bf16x32(p.q + grow * HD + c0, in);
+        unpack_bf16x32(pre_q[c], in);
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] = in[x] - __uint_as_float(r[x]);
         gstore_bf16x32(p.ql + grow * HD + c0, v);
         tmem_ld32(tl + 384 + c0, r);
         tmem_ld_wait();
-        gload_bf16x32(p.k + grow * HD + c0, in);
+        unpack_bf16x32(pre_k[c], in);
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] = in[x] - __uint_as_float(r[x]);
         gstore_bf16x32(p.kr + grow * HD + c0, v);

@@ -71,6 +71,18 @@ __device__ __forceinline__ void gload_bf16x32(const __nv_bfloat16* src, float (&
         }
     }
 }
+__device__ __forceinline__ void unpack_bf16x32(const uint4 (&u4)[4], float (&v)[32]) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const uint32_t w[4] = {u4[x].x, u4[x].y, u4[x].z, u4[x].w};
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[y]));
+            v[8 * x + 2 * y] = f.x;
+            v[8 * x + 2 * y + 1] = f.y;
+        }
+    }
+}
 __device__ __forceinline__ void tmem_row32(uint32_t taddr, float (&v)[32]) {
     uint32_t r[32];
     tmem_ld32(taddr, r);
