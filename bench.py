@@ -39,7 +39,12 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the kernel named by `roofline.kernel`,
 # from the ncu capture summarised under profiles/ (None until one exists for that kernel).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/dkv_kernel_C3_batch2.md: 600.4 MB per launch at batch 2; slices are independent, so batch 4 moves twice that
+    "fa_bwd_dkv": 2 * (370.438144e6 + 229.984e6),
+    # profiles/fa_fwd_kernel_C3_batch2.md: 363.0 MB per launch at batch 2
+    "fa_fwd": 2 * (335.659776e6 + 27.35104e6),
+}
 
 
 # ----------------------------------------------------------------------------------------- FLOP models
@@ -291,18 +296,30 @@ def run_ours(args, cfg):
     peaks = load_peaks()
     tf = lambda fl, t_ms: fl / (t_ms * 1e-3) / 1e12
     value = world * tf(f1 + b1, ms)
-    stage_flops = {"fa_fwd": f1 + B * H * (L // CHUNK) * 2 * CHUNK ** 3, "fa_bwd_dkv": 2.0 * f1, "fa_bwd_dq": 1.5 * f1}
-    top = max(stage_ms, key=stage_ms.get) if stage_ms else None
+    # work models of the single-kernel stages: FLOPs for the attention sweeps (tensor-bound),
+    # algorithmic bytes for the per-chunk kernels (HBM-bound)
+    nch = B * H * (-(-L // CHUNK))
+    diag = nch * 2 * CHUNK ** 3
+    stage_flops = {"fa_fwd": f1 + diag, "fa_bwd_dkv": 2.0 * f1 + diag, "fa_bwd_dq": 1.5 * f1}
+    t_d, t_b = CHUNK * d * 2, CHUNK * CHUNK * 2                 # bytes of a [128 x d] / [128 x 128] bf16 tile
+    prep_bytes = nch * (3 * t_d + 2 * t_d + 2 * t_b + 2 * d * d * 2)
+    stage_bytes = {"chunk_prep": prep_bytes, "bwd_chunk_prep": prep_bytes + nch * (7 * t_b + t_d),
+                   "bwd_chunk_chain": nch * (4 * t_d + 7 * t_b + 2 * 2 * t_d + 2 * t_b + d * d * 4 + 3 * t_d)}
+    single = [k_ for k_ in stage_ms if k_ in stage_flops or k_ in stage_bytes]
+    top = max(single, key=stage_ms.get) if single else None
     roof = None
-    if top is not None:
-        fl = stage_flops.get(top)
-        if fl is None:  # a multi-kernel linear stage: report its M2 share
-            fl = {"chunk_prep": f2 - f1, "bwd_chunk_prep": f2 - f1, "bwd_chains": b2 - b1 - (f2 - f1)}.get(top, 0.0)
-        ach = tf(fl, stage_ms[top])
+    if top in stage_flops:
+        ach = tf(stage_flops[top], stage_ms[top])
         roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["sustained"], "unit": "TFLOP/s",
                 "frac": ach / peaks["sustained"], "traffic": NCU_TRAFFIC_BYTES.get(top),
                 "peak_source": f"{peaks['source']} cuBLAS bf16, sustained", "ms_per_launch": stage_ms[top],
-                "flops_per_launch": fl}
+                "flops_per_launch": stage_flops[top]}
+    elif top is not None:
+        ach = stage_bytes[top] / (stage_ms[top] * 1e-3) / 1e9
+        roof = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peaks["hbm"], "unit": "GB/s",
+                "frac": ach / peaks["hbm"], "traffic": NCU_TRAFFIC_BYTES.get(top),
+                "peak_source": f"{peaks['source']} copy bandwidth", "ms_per_launch": stage_ms[top],
+                "bytes_per_launch": stage_bytes[top]}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
@@ -321,6 +338,7 @@ def run_ours(args, cfg):
             "frac_of_nominal_m1": tf(f1 + b1, ms) / 2250.0,
             "stage_ms": stage_ms,
             "stage_tflops": {k_: tf(stage_flops[k_], v_) for k_, v_ in stage_ms.items() if k_ in stage_flops},
+            "stage_gbs": {k_: stage_bytes[k_] / (v_ * 1e-3) / 1e9 for k_, v_ in stage_ms.items() if k_ in stage_bytes},
             "launches_per_step": launches[0], "peaks": peaks,
         },
     }

@@ -144,11 +144,12 @@ const char* path_attn_strerror(int status);
 /*
  * Optional stage timing for benchmarks (no counterpart in the paper).  After
  * path_attn_profile_enable(1), every fwd / bwd call of the calling thread records
- * CUDA events on its stream around its stages: "chunk_prep" (UT transform,
- * boundary-adjusted tiles, run products, versions; Sec. 3.1/3.3), "fa_fwd" (the
- * fused sweep, one kernel); and for bwd "bwd_chunk_prep" (the same preparation,
- * recomputed), "rowstats", "fa_bwd_dkv", "fa_bwd_dq" (one kernel each) and
- * "bwd_chains".  path_attn_profile_read waits for those events and writes the
+ * CUDA events on its stream around its stages: "chunk_prep" (UT transform and
+ * boundary-adjusted tiles, Sec. 3.1/3.3, one kernel), "levels_fwd" (run products
+ * and versions, several launches), "fa_fwd" (the fused sweep, one kernel); and
+ * for bwd "bwd_chunk_prep" and "bwd_levels_fwd" (the same preparation,
+ * recomputed), "rowstats", "fa_bwd_dkv", "fa_bwd_dq", "bwd_chunk_chain" (one
+ * kernel each), "bwd_levels" (several launches) and "bwd_gate".  path_attn_profile_read waits for those events and writes the
  * milliseconds per stage of the most recent fwd and the most recent bwd call
  * into ms[0..n) (-1 for a stage that did not run); it returns the number of entries written or a
  * negative status.  The events are created on first use and live until the

@@ -26,9 +26,11 @@ static thread_local int g_launches = 0;
 
 // ------------------------------------------------------------------------------------------- stage timing
 // Optional per-thread instrumentation: CUDA events around groups of launches of the most recent call.
-enum Stage { STG_PREP = 0, STG_FA_FWD, STG_PREP_BWD, STG_ROWSTATS, STG_FA_DKV, STG_FA_DQ, STG_CHAINS, STG_COUNT };
-static const char* const kStageNames[STG_COUNT] = {"chunk_prep", "fa_fwd", "bwd_chunk_prep", "rowstats", "fa_bwd_dkv",
-                                                   "fa_bwd_dq", "bwd_chains"};
+enum Stage { STG_PREP = 0, STG_LEVELS, STG_FA_FWD, STG_PREP_BWD, STG_LEVELS_BWDPREP, STG_ROWSTATS, STG_FA_DKV, STG_FA_DQ,
+             STG_LEVELS_BWD, STG_CHAIN, STG_GATE, STG_COUNT };
+static const char* const kStageNames[STG_COUNT] = {"chunk_prep", "levels_fwd", "fa_fwd", "bwd_chunk_prep", "bwd_levels_fwd",
+                                                   "rowstats", "fa_bwd_dkv", "fa_bwd_dq", "bwd_levels", "bwd_chunk_chain",
+                                                   "bwd_gate"};
 struct Profiler {
     bool on = false, created = false;
     cudaEvent_t ev[2 * STG_COUNT];
@@ -171,6 +173,7 @@ static LevelParams level_params(const Plan& p, void* ws) {
 // Chunk preparation + dyadic run products + version chains (paper Sec. 3.1, 3.3).  Shared by forward and backward.
 static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const void* w, cudaStream_t st) {
     const int d = p.d, nch = p.S * p.N;
+    const int stg_prep = p.bwd ? STG_PREP_BWD : STG_PREP, stg_lev = p.bwd ? STG_LEVELS_BWDPREP : STG_LEVELS;
     // fused per-chunk kernel: UT transform, boundary-adjusted tiles (version slot 0), chunk products (level 0)
     {
         PrepTensorMaps tm;
@@ -191,12 +194,15 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
             pp.sXq = at<bf>(ws, p.sXq); pp.sXk = at<bf>(ws, p.sXk); pp.sY = at<bf>(ws, p.sY); pp.sU = at<bf>(ws, p.sU);
         }
         pp.status = at<uint32_t>(ws, p.status);
+        prof_mark(stg_prep, 0, st);
         LAUNCH(launch_chunk_prep(tm, pp, d, p.bwd, nch, st));
+        prof_mark(stg_prep, 1, st);
     }
     if (p.nlev < 2) return PATH_OK;
     LevelTensorMaps tm;
     if (!make_level_maps(p, ws, tm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
     LevelParams lp = level_params(p, ws);
+    prof_mark(stg_lev, 0, st);
     for (int l = 0; l + 1 <= p.nlev - 2; ++l) {   // run products of 2, 4, ... chunks
         lp.l = l;
         LAUNCH(launch_level_kernel(LEVEL_DYADIC_FWD, tm, lp, d, st));
@@ -205,6 +211,7 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
         lp.l = l2;
         LAUNCH(launch_level_kernel(LEVEL_VERSION_FWD, tm, lp, d, st));
     }
+    prof_mark(stg_lev, 1, st);
     return PATH_OK;
 }
 
@@ -297,7 +304,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     prof_mark(STG_FA_DQ, 0, st);
     LAUNCH(launch_fa_bwd(tm, bp, d, 1, st));
     prof_mark(STG_FA_DQ, 1, st);
-    prof_mark(STG_CHAINS, 0, st);
+    prof_mark(STG_LEVELS_BWD, 0, st);
 
     // version chains, top level first, then the run products top-down
     if (p.nlev >= 2) {
@@ -313,14 +320,18 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
             LAUNCH(launch_level_kernel(LEVEL_DYADIC_BWD, ltm, lp, d, st));
         }
     }
+    prof_mark(STG_LEVELS_BWD, 1, st);
+    prof_mark(STG_CHAIN, 0, st);
     int rc = run_chunk_chain(p, ws, q, k, w, dq, dk, dw, dbeta, scale, st);
     if (rc != PATH_OK) return rc;
+    prof_mark(STG_CHAIN, 1, st);
+    prof_mark(STG_GATE, 0, st);
     if (dlog_f) {
         LAUNCH(launch_dsd_rowsum(at<float>(ws, p.dSd), at<float>(ws, p.dGdiag), p.S * p.N, st));
         LAUNCH(launch_gate_suffix(at<float>(ws, p.dG), at<float>(ws, p.dGrow), at<float>(ws, p.dGdiag), dlog_f, p.S, p.L,
                                   p.Lp, st));
     }
-    prof_mark(STG_CHAINS, 1, st);
+    prof_mark(STG_GATE, 1, st);
     return PATH_OK;
 }
 
@@ -355,12 +366,10 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     CK(cudaMemsetAsync(workspace, 0, 256, st));
 
     prof_reset(STG_PREP, STG_PREP_BWD);
-    prof_mark(STG_PREP, 0, st);
     rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, st);
     if (rc != PATH_OK) return rc;
     rc = run_prep(p, workspace, q, k, w, st);
     if (rc != PATH_OK) return rc;
-    prof_mark(STG_PREP, 1, st);
 
     FwdTensorMaps tm;
     const uint64_t rows = (uint64_t)p.S * p.Lp;
@@ -402,12 +411,10 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
     cudaStream_t st = (cudaStream_t)cuda_stream;
     CK(cudaMemsetAsync(workspace, 0, 256, st));
     prof_reset(STG_PREP_BWD, STG_COUNT);
-    prof_mark(STG_PREP_BWD, 0, st);
     rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, st);
     if (rc != PATH_OK) return rc;
     rc = run_prep(p, workspace, q, k, w, st);
     if (rc != PATH_OK) return rc;
-    prof_mark(STG_PREP_BWD, 1, st);
     return run_backward(p, workspace, q, k, v, w, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, scale, st);
 }
 
