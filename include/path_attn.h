@@ -88,6 +88,13 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
  *   dlog_f  : [B,H,L] float32 (out); must be NULL exactly when log_f is NULL
  * dt must be PATH_BF16.  Uses float32 atomics: results are reproducible to
  * rounding, not bitwise.
+ *
+ * Reuse of the forward's work: if path_attn_fwd ran on this same workspace with
+ * these same input pointers and shape, and the workspace was at least
+ * path_attn_workspace_bytes(..., for_backward = 1) bytes, the chunk preparation
+ * it left there (Sec. 3.1 / 3.3 quantities) is reused instead of recomputed.
+ * Any other call on the workspace in between, or different pointers, makes the
+ * backward recompute it.  (As always, o and lse must belong to the inputs.)
  */
 int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, const float* beta,
                   const float* log_f, const void* o, const float* lse, const void* d_o, void* dq,

@@ -51,6 +51,37 @@ static void prof_mark(int stage, int end, cudaStream_t st) {
     if (end) g_prof.used[stage] = true;
 }
 
+// ------------------------------------------------------------------------------------------- forward state reuse
+// A forward that ran on a backward-sized workspace leaves the chunk preparation (with the tiles the chain rule needs)
+// in it.  The table remembers, per workspace pointer, which problem that state belongs to, so that the backward of
+// the same problem can skip recomputing it.  Host-side only; entries are overwritten by any later call on the workspace.
+struct StateTag {
+    const void *ws, *q, *k, *v, *w, *beta, *log_f;
+    int B, H, L, d;
+};
+static std::mutex g_tag_mutex;
+static StateTag g_tags[64];
+static int g_tag_next = 0;
+
+static bool tag_equal(const StateTag& a, const StateTag& b) {
+    return a.ws == b.ws && a.q == b.q && a.k == b.k && a.v == b.v && a.w == b.w && a.beta == b.beta &&
+           a.log_f == b.log_f && a.B == b.B && a.H == b.H && a.L == b.L && a.d == b.d;
+}
+static void tag_store(const StateTag& t, bool valid) {   // valid = false: forget whatever was known about t.ws
+    std::lock_guard<std::mutex> lock(g_tag_mutex);
+    for (auto& e : g_tags)
+        if (e.ws == t.ws) { if (valid) e = t; else e = StateTag{}; return; }
+    if (!valid) return;
+    g_tags[g_tag_next] = t;
+    g_tag_next = (g_tag_next + 1) % 64;
+}
+static bool tag_matches(const StateTag& t) {
+    std::lock_guard<std::mutex> lock(g_tag_mutex);
+    for (const auto& e : g_tags)
+        if (e.ws == t.ws) return tag_equal(e, t);
+    return false;
+}
+
 // ------------------------------------------------------------------------------------------- tensor maps
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -171,9 +202,10 @@ static LevelParams level_params(const Plan& p, void* ws) {
 }
 
 // Chunk preparation + dyadic run products + version chains (paper Sec. 3.1, 3.3).  Shared by forward and backward.
-static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const void* w, cudaStream_t st) {
+static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const void* w, bool in_backward,
+                    cudaStream_t st) {
     const int d = p.d, nch = p.S * p.N;
-    const int stg_prep = p.bwd ? STG_PREP_BWD : STG_PREP, stg_lev = p.bwd ? STG_LEVELS_BWDPREP : STG_LEVELS;
+    const int stg_prep = in_backward ? STG_PREP_BWD : STG_PREP, stg_lev = in_backward ? STG_LEVELS_BWDPREP : STG_LEVELS;
     // fused per-chunk kernel: UT transform, boundary-adjusted tiles (version slot 0), chunk products (level 0)
     {
         PrepTensorMaps tm;
@@ -226,16 +258,22 @@ static int check_arch() {
 static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
 // Pads q, k, v, w (ragged L) and beta into the workspace; returns the pointers the kernels should read.
+// With run = false only the pointers are redirected (the padded copies are already in the workspace).
 static int stage_inputs(const Plan& p, void* ws, const void*& q, const void*& k, const void*& v, const void*& w,
-                        const float* beta, const float* log_f, cudaStream_t st) {
+                        const float* beta, const float* log_f, bool run, cudaStream_t st) {
     if (p.ragged) {
-        LAUNCH(launch_pad_rows(q, at<void>(ws, p.qp), p.S, p.L, p.Lp, p.d, 0, st)); q = at<void>(ws, p.qp);
-        LAUNCH(launch_pad_rows(k, at<void>(ws, p.kp), p.S, p.L, p.Lp, p.d, 0, st)); k = at<void>(ws, p.kp);
-        LAUNCH(launch_pad_rows(v, at<void>(ws, p.vp), p.S, p.L, p.Lp, p.d, 0, st)); v = at<void>(ws, p.vp);
-        LAUNCH(launch_pad_rows(w, at<void>(ws, p.wp), p.S, p.L, p.Lp, p.d, 0, st)); w = at<void>(ws, p.wp);
+        if (run) {
+            LAUNCH(launch_pad_rows(q, at<void>(ws, p.qp), p.S, p.L, p.Lp, p.d, 0, st));
+            LAUNCH(launch_pad_rows(k, at<void>(ws, p.kp), p.S, p.L, p.Lp, p.d, 0, st));
+            LAUNCH(launch_pad_rows(v, at<void>(ws, p.vp), p.S, p.L, p.Lp, p.d, 0, st));
+            LAUNCH(launch_pad_rows(w, at<void>(ws, p.wp), p.S, p.L, p.Lp, p.d, 0, st));
+        }
+        q = at<void>(ws, p.qp); k = at<void>(ws, p.kp); v = at<void>(ws, p.vp); w = at<void>(ws, p.wp);
     }
-    LAUNCH(launch_pad_vec(beta, at<float>(ws, p.betap), p.S, p.L, p.Lp, st));
-    if (log_f) LAUNCH(launch_gate_prefix(log_f, at<float>(ws, p.G), p.S, p.L, p.Lp, st));
+    if (run) {
+        LAUNCH(launch_pad_vec(beta, at<float>(ws, p.betap), p.S, p.L, p.Lp, st));
+        if (log_f) LAUNCH(launch_gate_prefix(log_f, at<float>(ws, p.G), p.S, p.L, p.Lp, st));
+    }
     return PATH_OK;
 }
 
@@ -356,6 +394,14 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     if (dt != PATH_BF16 && dt != PATH_FP32) return PATH_ERR_DTYPE;
     if (!make_plan(B, H, L, d, (int)dt, log_f ? 1 : 0, 0, p)) return PATH_ERR_SHAPE;
     if (dt != PATH_BF16) return PATH_ERR_DTYPE;
+    // A workspace large enough for the backward gets the backward's layout: the chunk preparation then also keeps
+    // the tiles the chain rule needs, and path_attn_bwd on the same workspace and inputs does not redo it.
+    const StateTag tag{workspace, q, k, v, w, beta, log_f, B, H, L, d};
+    bool keep_state = false;
+    {
+        Plan pb;
+        if (make_plan(B, H, L, d, (int)dt, log_f ? 1 : 0, 1, pb) && workspace_bytes >= pb.total) { p = pb; keep_state = true; }
+    }
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(w) || !aligned16(beta) || !aligned16(o) ||
         !aligned16(lse) || (log_f && !aligned16(log_f)) || ((uintptr_t)workspace & 255))
         return PATH_ERR_ALIGN;
@@ -366,9 +412,10 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     CK(cudaMemsetAsync(workspace, 0, 256, st));
 
     prof_reset(STG_PREP, STG_PREP_BWD);
-    rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, st);
+    tag_store(tag, false);
+    rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, true, st);
     if (rc != PATH_OK) return rc;
-    rc = run_prep(p, workspace, q, k, w, st);
+    rc = run_prep(p, workspace, q, k, w, false, st);
     if (rc != PATH_OK) return rc;
 
     FwdTensorMaps tm;
@@ -386,6 +433,7 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     prof_mark(STG_FA_FWD, 0, st);
     LAUNCH(launch_fa_fwd(tm, fp, d, st));
     prof_mark(STG_FA_FWD, 1, st);
+    if (keep_state) tag_store(tag, true);
     return PATH_OK;
 }
 
@@ -411,10 +459,16 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
     cudaStream_t st = (cudaStream_t)cuda_stream;
     CK(cudaMemsetAsync(workspace, 0, 256, st));
     prof_reset(STG_PREP_BWD, STG_COUNT);
-    rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, st);
+    const StateTag tag{workspace, q, k, v, w, beta, log_f, B, H, L, d};
+    const bool reuse = tag_matches(tag);   // the forward of this very problem left its preparation in this workspace
+    if (!reuse) tag_store(tag, false);
+    rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, !reuse, st);
     if (rc != PATH_OK) return rc;
-    rc = run_prep(p, workspace, q, k, w, st);
-    if (rc != PATH_OK) return rc;
+    if (!reuse) {
+        rc = run_prep(p, workspace, q, k, w, true, st);
+        if (rc != PATH_OK) return rc;
+        tag_store(tag, true);
+    }
     return run_backward(p, workspace, q, k, v, w, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, scale, st);
 }
 

@@ -134,6 +134,30 @@ def test_forward_is_bitwise_reproducible_and_workspace_is_reusable(binding):
     assert binding.device_status(ws) == 0
 
 
+def test_backward_reuses_forward_state_only_for_the_same_problem(binding):
+    a = to_dev(synth.make_inputs(1, 2, 700, 128, "bf16", gate=True, seed=31))
+    b_ = to_dev(synth.make_inputs(1, 2, 700, 128, "bf16", gate=True, seed=32))
+    args = lambda t: (t["q"], t["k"], t["v"], t["w"], t["beta"])
+    ws = binding.alloc_workspace(a["q"], True, True)
+    fresh = lambda t, o, lse: binding.path_attn_bwd(*args(t), o, lse, t["d_o"], t["log_f"],
+                                                    workspace=binding.alloc_workspace(t["q"], True, True))
+    o_a, lse_a = binding.path_attn_fwd(*args(a), a["log_f"], workspace=ws)          # leaves its preparation in ws
+    g_reuse = binding.path_attn_bwd(*args(a), o_a, lse_a, a["d_o"], a["log_f"], workspace=ws)
+    n_reuse = binding.last_launch_count()
+    g_fresh = fresh(a, o_a, lse_a)
+    assert n_reuse < binding.last_launch_count()                                   # the preparation was skipped
+    for n in g_fresh:
+        assert torch.allclose(g_reuse[n].float(), g_fresh[n].float(), rtol=2e-2, atol=1e-3), n
+    # same workspace, other problem: nothing stale may be reused
+    o_b, lse_b = binding.path_attn_fwd(*args(b_), b_["log_f"])
+    binding.path_attn_fwd(*args(a), a["log_f"], workspace=ws)
+    g_b = binding.path_attn_bwd(*args(b_), o_b, lse_b, b_["d_o"], b_["log_f"], workspace=ws)
+    g_b_fresh = fresh(b_, o_b, lse_b)
+    for n in g_b_fresh:
+        assert torch.allclose(g_b[n].float(), g_b_fresh[n].float(), rtol=2e-2, atol=1e-3), n
+    assert binding.device_status(ws) == 0
+
+
 # ---------------------------------------------------------------- the named workloads at full size
 
 def test_c2_full_size_sampled_slices(binding, oracle):
