@@ -13,7 +13,11 @@
 //               (TMEM lanes = keys): S^T = K Q^T, dP^T = V dO^T, dV += P^T dO, dK += dS^T Q.
 //   dq_kernel : one CTA per query chunk I, sweeps J = I-1..0: S = Q K^T, dP = dO V^T, dQ += dS K.
 // The accumulator of a version is flushed to global memory when the sweep crosses into the next level.
-// Warp roles as in the forward: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 elementwise math.
+// P^T / dS^T (dkv) and dS (dq) never touch shared memory: they overwrite the first half of the columns their thread
+// read, as packed bf16, and enter the second products as tensor-memory A operands.  The shared memory this frees
+// double-buffers the per-step tiles.
+// Warps: 0 = TMA producer, 1 = tcgen05 MMA issuer, 2-9 = elementwise math (two warps per TMEM lane quadrant, each
+// taking 64 of the 128 columns of a row).
 #include "common.cuh"
 #include "tc5.cuh"
 
@@ -32,6 +36,15 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 
 // D[tmem] (+)= A B^T with both operands K-major [rows][kdim] tiles (two 64-column panels per 128 of kdim).
 __device__ __forceinline__ void mma_kk(uint32_t d_tmem, uint32_t a0, uint32_t b0, int kdim, uint32_t idesc, bool acc) {
@@ -40,53 +53,42 @@ __device__ __forceinline__ void mma_kk(uint32_t d_tmem, uint32_t a0, uint32_t b0
         umma_ss(d_tmem, umma_desc(a0 + off, 16, 1024), umma_desc(b0 + off, 16, 1024), idesc, (acc || kk > 0) ? 1u : 0u);
     }
 }
-// D[tmem] (+)= A B with A K-major [128][128] and B MN-major [128 (k)][HD] (64-column panels 16 KB apart).
-__device__ __forceinline__ void mma_kn(uint32_t d_tmem, uint32_t a0, uint32_t b0, uint32_t idesc, bool acc) {
-    for (int kk = 0; kk < kTile / 16; ++kk) {
-        const uint32_t aoff = (kk >> 2) * kPanelBytes + (kk & 3) * 32;
-        umma_ss(d_tmem, umma_desc(a0 + aoff, 16, 1024), umma_desc(b0 + kk * 2048, kPanelBytes, 1024), idesc,
+// D[tmem] (+)= A B with A in tensor memory (packed bf16: the 64 contraction indices [64h, 64h+64) of a row sit in the
+// 32 columns starting at a_col + 64h) and B MN-major [128 (k)][HD] in shared memory.
+__device__ __forceinline__ void mma_tn(uint32_t d_tmem, uint32_t a_col, uint32_t b0, uint32_t idesc, bool acc) {
+    for (int kk = 0; kk < kTile / 16; ++kk)
+        umma_ts(d_tmem, a_col + (kk >> 2) * 64 + (kk & 3) * 8, umma_desc(b0 + kk * 2048, kPanelBytes, 1024), idesc,
                 (acc || kk > 0) ? 1u : 0u);
-    }
 }
 
 __device__ __forceinline__ void tma_tile(uint8_t* dst, const CUtensorMap* m, uint64_t* bar, int kdim, int row0) {
     for (int h = 0; h < kdim / 64; ++h) tma_load_2d(dst + h * kPanelBytes, m, bar, h * 64, row0);
 }
 
-// Writes 32 consecutive bf16 values of `row` (columns c*32 .. c*32+31 of a [128][128] K-major tile).
-__device__ __forceinline__ void store_row_chunk(uint8_t* tile, int row, int c, const uint32_t (&pk)[16]) {
-    uint8_t* panel = tile + (c >> 1) * kPanelBytes;
-#pragma unroll
-    for (int ch = 0; ch < 4; ++ch)
-        *reinterpret_cast<uint4*>(panel + sw128_off((uint32_t)row, (uint32_t)((c & 1) * 4 + ch))) =
-            make_uint4(pk[ch * 4], pk[ch * 4 + 1], pk[ch * 4 + 2], pk[ch * 4 + 3]);
-}
-
 // ------------------------------------------------------------------------------------------------ dK, dV
-enum { K_KFULL = 0, K_KEMPTY, K_QFULL, K_QEMPTY, K_DOFULL, K_DOEMPTY, K_VFULL, K_XFULL, K_SFULL, K_PFULL,
-       K_MMA2, K_COUNT };
+enum { K_KFULL = 0, K_KEMPTY, K_VFULL, K_QFULL, K_QEMPTY = K_QFULL + 2, K_DOFULL = K_QEMPTY + 2,
+       K_DOEMPTY = K_DOFULL + 2, K_SFULL = K_DOEMPTY + 2, K_PFULL, K_FINAL, K_COUNT };
 
 template <int HD, bool GATE>
-__global__ void __launch_bounds__(192, 1) dkv_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
+__global__ void __launch_bounds__(320, 1) dkv_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sK = smem;
     uint8_t* sV = sK + kSlotBytes;
-    uint8_t* sQ = sV + kSlotBytes;
-    uint8_t* sDO = sQ + kSlotBytes;
-    uint8_t* sPt = sDO + kSlotBytes;
-    uint8_t* sDSt = sPt + kSlotBytes;
-    uint64_t* bars = (uint64_t*)(sDSt + kSlotBytes);
+    uint8_t* sQ = sV + kSlotBytes;          // 2 slots: rawQ, Xqn, then Q of step t >= 1 in slot (t + 1) & 1
+    uint8_t* sDO = sQ + 2 * kSlotBytes;     // 2 slots: dO(0), Yt, then dO of step t >= 1 in slot (t + 1) & 1
+    uint64_t* bars = (uint64_t*)(sDO + 2 * kSlotBytes);
     uint32_t* tmem_slot = (uint32_t*)(bars + K_COUNT);
     volatile uint32_t* abort_flag = (volatile uint32_t*)(tmem_slot + 1);
     float* rowstat = (float*)(smem + 6 * kSlotBytes + 256);  // [2][3][128]: lse2, delta, G of the query chunk
+    float* dsum_x = rowstat + 2 * 3 * kTile;                 // [128] exchange of the gate row sums
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int J = blockIdx.x, s = blockIdx.y;
     const int T = p.N - J;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < K_COUNT; ++i) mbar_init(&bars[i], i == K_PFULL ? 128u : 1u);
+        for (int i = 0; i < K_COUNT; ++i) mbar_init(&bars[i], i == K_PFULL ? 256u : 1u);
         *abort_flag = 0;
         mbar_fence_init();
     }
@@ -104,8 +106,15 @@ __global__ void __launch_bounds__(192, 1) dkv_kernel(const __grid_constant__ Bwd
         if (lane == 0) {
             bool ok = true;
             int nk = 0;
-            auto wait_empty = [&](int bar, int n) {
-                if (ok && !mbar_wait(&bars[bar], (n & 1) ^ 1, abort_flag, ST_DKV_PRODUCER)) ok = false;
+            auto wait_empty = [&](int bar, int use) {
+                if (ok && !mbar_wait(&bars[bar], (use & 1) ^ 1, abort_flag, ST_DKV_PRODUCER)) ok = false;
+            };
+            auto ring_load = [&](uint8_t* base, int bfull, int bempty, int item, const CUtensorMap* m, int kdim, int row0) {
+                const int slot = item & 1;
+                wait_empty(bempty + slot, item >> 1);
+                if (!ok) return;
+                mbar_expect_tx(&bars[bfull + slot], (uint32_t)(kTile * kdim * 2));
+                tma_tile(base + slot * kSlotBytes, m, &bars[bfull + slot], kdim, row0);
             };
             for (int t = 0; t < T && ok; ++t) {
                 const int I = J + t, l = level(t);
@@ -120,19 +129,14 @@ __global__ void __launch_bounds__(192, 1) dkv_kernel(const __grid_constant__ Bwd
                 if (t == 0) {
                     mbar_expect_tx(&bars[K_VFULL], kTile * HD * 2);
                     tma_tile(sV, &tm.v, &bars[K_VFULL], HD, rowJ);
-                    mbar_expect_tx(&bars[K_XFULL], 2 * kSlotBytes);
-                    tma_tile(sPt, &tm.yt, &bars[K_XFULL], kTile, rowJ);
-                    tma_tile(sDSt, &tm.xqn, &bars[K_XFULL], kTile, rowJ);
+                    ring_load(sQ, K_QFULL, K_QEMPTY, 0, &tm.q_raw, HD, rowJ);
+                    ring_load(sDO, K_DOFULL, K_DOEMPTY, 0, &tm.d_o, HD, rowJ);
+                    ring_load(sQ, K_QFULL, K_QEMPTY, 1, &tm.xqn, kTile, rowJ);
+                    ring_load(sDO, K_DOFULL, K_DOEMPTY, 1, &tm.yt, kTile, rowJ);
+                } else {
+                    ring_load(sQ, K_QFULL, K_QEMPTY, t + 1, &tm.qv, HD, ver_row(qslot(l, I), I));
+                    ring_load(sDO, K_DOFULL, K_DOEMPTY, t + 1, &tm.d_o, HD, s * p.Lp + I * kTile);
                 }
-                wait_empty(K_QEMPTY, t);
-                if (!ok) break;
-                mbar_expect_tx(&bars[K_QFULL], kTile * HD * 2);
-                if (t == 0) tma_tile(sQ, &tm.q_raw, &bars[K_QFULL], HD, rowJ);
-                else tma_tile(sQ, &tm.qv, &bars[K_QFULL], HD, ver_row(qslot(l, I), I));
-                wait_empty(K_DOEMPTY, t);
-                if (!ok) break;
-                mbar_expect_tx(&bars[K_DOFULL], kTile * HD * 2);
-                tma_tile(sDO, &tm.d_o, &bars[K_DOFULL], HD, s * p.Lp + I * kTile);
             }
         }
     } else if (warp == 1) {
@@ -146,40 +150,51 @@ __global__ void __launch_bounds__(192, 1) dkv_kernel(const __grid_constant__ Bwd
             };
             for (int t = 0; t < T && ok; ++t) {
                 const int l = level(t);
+                const int item = (t == 0) ? 0 : t + 1, slot = item & 1;
+                const uint32_t aQ = smem_u32(sQ + slot * kSlotBytes), aDO = smem_u32(sDO + slot * kSlotBytes);
                 if (t == 0 || l != level(t - 1)) { wait(K_KFULL, nk); ++nk; }
-                wait(K_QFULL, t);
-                if (t == 0) { wait(K_XFULL, 0); wait(K_VFULL, 0); }
-                wait(K_DOFULL, t);
+                wait(K_QFULL + slot, item >> 1);
+                wait(K_DOFULL + slot, item >> 1);
+                if (t == 0) { wait(K_VFULL, 0); wait(K_QFULL + 1, 0); wait(K_DOFULL + 1, 0); }
                 tc_fence_after_sync();
                 if (!ok) break;
-                mma_kk(tmem + colS, smem_u32(sK), smem_u32(sQ), HD, idescT, false);
-                if (t == 0) mma_kk(tmem + colS, smem_u32(sPt), smem_u32(sDSt), kTile, idescT, true);
-                mma_kk(tmem + colDP, smem_u32(sV), smem_u32(sDO), HD, idescT, false);
+                mma_kk(tmem + colS, smem_u32(sK), aQ, HD, idescT, false);
+                if (t == 0) mma_kk(tmem + colS, smem_u32(sDO + kSlotBytes), smem_u32(sQ + kSlotBytes), kTile, idescT, true);
+                mma_kk(tmem + colDP, smem_u32(sV), aDO, HD, idescT, false);
                 umma_commit(&bars[K_SFULL]);
+                if (t == 0) {   // raw q and the two correction operands are only needed by the products above
+                    umma_commit(&bars[K_QEMPTY + 0]);
+                    umma_commit(&bars[K_QEMPTY + 1]);
+                    umma_commit(&bars[K_DOEMPTY + 1]);
+                }
                 if (t + 1 < T && level(t + 1) != l) umma_commit(&bars[K_KEMPTY]);
                 wait(K_PFULL, t);
                 tc_fence_after_sync();
                 if (!ok) break;
-                mma_kn(tmem + colDV, smem_u32(sPt), smem_u32(sDO), idescD, t > 0);
-                if (t > 0) mma_kn(tmem + colDK, smem_u32(sDSt), smem_u32(sQ), idescD, !(t == 1 || l != level(t - 1)));
-                umma_commit(&bars[K_MMA2]);
-                umma_commit(&bars[K_QEMPTY]);
-                umma_commit(&bars[K_DOEMPTY]);
+                mma_tn(tmem + colDV, tmem + colS, aDO, idescD, t > 0);
+                if (t > 0) {
+                    mma_tn(tmem + colDK, tmem + colDP, aQ, idescD, !(t == 1 || l != level(t - 1)));
+                    umma_commit(&bars[K_QEMPTY + slot]);
+                }
+                umma_commit(&bars[K_DOEMPTY + slot]);
+                if (t == T - 1) umma_commit(&bars[K_FINAL]);
             }
         }
     } else {
-        const int q4 = warp & 3, row = q4 * 32 + lane, tid = threadIdx.x - 64;
+        const int q4 = warp & 3, h = (warp - 2) >> 2, row = q4 * 32 + lane;
+        const int tid = threadIdx.x - 64;       // 0..255
         const uint32_t tlane = tmem + ((uint32_t)(q4 * 32) << 16);
-        const int kj = J * kTile + row;  // key position of this thread
+        const int kj = J * kTile + row;          // key position of this thread's row
         const float sl2 = p.scale * kLog2e;
         float gj2 = 0.f, dsum = 0.f;
         if (GATE) gj2 = p.G[(size_t)s * p.Lp + kj] * kLog2e;
         bool ok = true;
         uint32_t rs[32], rp[32];
+        constexpr int CW = HD / 2;               // accumulator columns per thread when flushing
         auto flush_dk = [&](int lvl) {
-            float* dst = p.dkv + ((size_t)ver_row(kslot(lvl, J), J) + row) * HD;
-            for (int c = 0; c < HD / 32; ++c) {
-                tmem_ld32(tlane + colDK + c * 32, rs);
+            float* dst = p.dkv + ((size_t)ver_row(kslot(lvl, J), J) + row) * HD + h * CW;
+            for (int c = 0; c < CW / 32; ++c) {
+                tmem_ld32(tlane + colDK + h * CW + c * 32, rs);
                 tmem_ld_wait();
 #pragma unroll
                 for (int x = 0; x < 8; ++x)
@@ -191,28 +206,30 @@ __global__ void __launch_bounds__(192, 1) dkv_kernel(const __grid_constant__ Bwd
         for (int t = 0; t < T; ++t) {
             const int I = J + t, b = t & 1;
             float* st_ = rowstat + b * 3 * kTile;
-            {
+            if (tid < kTile) {
                 const size_t gi = (size_t)s * p.Lp + I * kTile + tid;
                 st_[tid] = p.lse2[gi];
                 st_[kTile + tid] = p.delta[gi];
                 if (GATE) st_[2 * kTile + tid] = p.G[gi] * kLog2e;
-                asm volatile("bar.sync 1, 128;" ::: "memory");
             }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             if (ok && !mbar_wait(&bars[K_SFULL], t & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
-            if (t > 0 && ok && !mbar_wait(&bars[K_MMA2], (t - 1) & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after_sync();
             if (ok) {
+                // S^T / dP^T ready means every earlier product has retired: dK of the finished level can be flushed
                 if (t >= 2 && level(t) != level(t - 1)) flush_dk(level(t - 1));
-                for (int c = 0; c < 4; ++c) {
-                    tmem_ld32(tlane + colS + c * 32, rs);
-                    tmem_ld32(tlane + colDP + c * 32, rp);
+                uint32_t pkP[32], pkS[32];
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int c0 = h * 64 + c * 32;      // query columns of this pass
+                    tmem_ld32(tlane + colS + c0, rs);
+                    tmem_ld32(tlane + colDP + c0, rp);
                     tmem_ld_wait();
-                    uint32_t pkP[16], pkS[16];
                     float dsv[32];
 #pragma unroll
                     for (int x = 0; x < 32; ++x) {
-                        const int col = c * 32 + x;  // query within chunk I
+                        const int col = c0 + x;
                         float v = __uint_as_float(rs[x]) * sl2 - st_[col];
                         if (GATE) v += st_[2 * kTile + col] - gj2;
                         float pr = ex2(v);
@@ -224,36 +241,41 @@ __global__ void __launch_bounds__(192, 1) dkv_kernel(const __grid_constant__ Bwd
                     }
 #pragma unroll
                     for (int x = 0; x < 32; x += 2) {
-                        pkP[x >> 1] = pack_bf16(__uint_as_float(rs[x]), __uint_as_float(rs[x + 1]));
-                        pkS[x >> 1] = pack_bf16(dsv[x], dsv[x + 1]);
+                        pkP[c * 16 + (x >> 1)] = pack_bf16(__uint_as_float(rs[x]), __uint_as_float(rs[x + 1]));
+                        pkS[c * 16 + (x >> 1)] = pack_bf16(dsv[x], dsv[x + 1]);
                     }
-                    store_row_chunk(sPt, row, c, pkP);
-                    store_row_chunk(sDSt, row, c, pkS);
                     if (t == 0) {
                         float* dsd = p.dsd + ((size_t)(s * p.N + J) * kTile) * kTile;
 #pragma unroll
-                        for (int x = 0; x < 32; ++x) dsd[(size_t)(c * 32 + x) * kTile + row] = dsv[x];
+                        for (int x = 0; x < 32; ++x) dsd[(size_t)(c0 + x) * kTile + row] = dsv[x];
                     }
                 }
+                tmem_st32(tlane + colS + h * 64, pkP);
+                tmem_st32(tlane + colDP + h * 64, pkS);
+                tmem_st_wait();
             }
             tc_fence_before_sync();
-            fence_proxy_async_smem();
             mbar_arrive(&bars[K_PFULL]);
         }
-        if (ok && !mbar_wait(&bars[K_MMA2], (T - 1) & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
+        if (ok && !mbar_wait(&bars[K_FINAL], 0, abort_flag, ST_DKV_COMPUTE)) ok = false;
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after_sync();
+        if (GATE) {   // the two threads of a key row add their halves of the column sum
+            if (h == 1) dsum_x[row] = dsum;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (h == 0 && ok) p.dG[(size_t)s * p.Lp + kj] = -(dsum + dsum_x[row]);
+        }
         if (ok) {
             if (T > 1) flush_dk(level(T - 1));
             else {  // last chunk: no later query chunk, the boundary-adjusted keys get a zero gradient from the sweep
-                float4* dst = reinterpret_cast<float4*>(p.dkv + ((size_t)ver_row(0, J) + row) * HD);
-                for (int x = 0; x < HD / 4; ++x) dst[x] = make_float4(0.f, 0.f, 0.f, 0.f);
+                float4* dst = reinterpret_cast<float4*>(p.dkv + ((size_t)ver_row(0, J) + row) * HD + h * CW);
+                for (int x = 0; x < CW / 4; ++x) dst[x] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            for (int c = 0; c < HD / 32; ++c) {
-                tmem_ld32(tlane + colDV + c * 32, rs);
+            for (int c = 0; c < CW / 32; ++c) {
+                tmem_ld32(tlane + colDV + h * CW + c * 32, rs);
                 tmem_ld_wait();
                 if (kj < p.L) {
-                    uint4* dst = reinterpret_cast<uint4*>((__nv_bfloat16*)p.dv + ((size_t)s * p.L + kj) * HD + c * 32);
+                    uint4* dst = reinterpret_cast<uint4*>((__nv_bfloat16*)p.dv + ((size_t)s * p.L + kj) * HD + h * CW + c * 32);
 #pragma unroll
                     for (int x = 0; x < 4; ++x)
                         dst[x] = make_uint4(pack_bf16(__uint_as_float(rs[8 * x]), __uint_as_float(rs[8 * x + 1])),
@@ -262,7 +284,6 @@ __global__ void __launch_bounds__(192, 1) dkv_kernel(const __grid_constant__ Bwd
                                             pack_bf16(__uint_as_float(rs[8 * x + 6]), __uint_as_float(rs[8 * x + 7])));
                 }
             }
-            if (GATE) p.dG[(size_t)s * p.Lp + kj] = -dsum;
         }
     }
     tc_fence_before_sync();
@@ -276,10 +297,10 @@ __global__ void __launch_bounds__(192, 1) dkv_kernel(const __grid_constant__ Bwd
 
 // ------------------------------------------------------------------------------------------------ dQ
 enum { Q_QFULL = 0, Q_QEMPTY, Q_DOFULL, Q_KFULL, Q_KEMPTY = Q_KFULL + 2, Q_VFULL = Q_KEMPTY + 2,
-       Q_VEMPTY = Q_VFULL + 2, Q_SFULL = Q_VEMPTY + 2, Q_SEMPTY, Q_DSFULL, Q_DQDONE, Q_COUNT };
+       Q_VEMPTY = Q_VFULL + 2, Q_SFULL = Q_VEMPTY + 2, Q_DSFULL, Q_FINAL, Q_COUNT };
 
 template <int HD, bool GATE>
-__global__ void __launch_bounds__(192, 1) dq_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
+__global__ void __launch_bounds__(320, 1) dq_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
     const int I = (int)gridDim.x - 1 - (int)blockIdx.x, s = blockIdx.y;
     if (I == 0) {  // chunk 0 has no earlier keys: its boundary-adjusted queries get a zero gradient from the sweep
         float4* dst = reinterpret_cast<float4*>(p.dqv + (size_t)s * p.Lp * HD);
@@ -292,17 +313,17 @@ __global__ void __launch_bounds__(192, 1) dq_kernel(const __grid_constant__ BwdT
     uint8_t* sDO = sQ + kSlotBytes;
     uint8_t* sK = sDO + kSlotBytes;        // 2 slots
     uint8_t* sV = sK + 2 * kSlotBytes;     // 2 slots
-    uint8_t* sDS = sV + 2 * kSlotBytes;
-    uint64_t* bars = (uint64_t*)(sDS + kSlotBytes);
+    uint64_t* bars = (uint64_t*)(sV + 2 * kSlotBytes);
     uint32_t* tmem_slot = (uint32_t*)(bars + Q_COUNT);
     volatile uint32_t* abort_flag = (volatile uint32_t*)(tmem_slot + 1);
-    float* gk = (float*)(smem + 7 * kSlotBytes + 256);  // [2][128] gate prefix of the key chunk
+    float* gk = (float*)(smem + 6 * kSlotBytes + 256);  // [2][128] gate prefix of the key chunk
+    float* dsum_x = gk + 2 * kTile;                     // [128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int T = I;  // steps t = 0..I-1, J = I-1-t
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < Q_COUNT; ++i) mbar_init(&bars[i], (i == Q_SEMPTY || i == Q_DSFULL) ? 128u : 1u);
+        for (int i = 0; i < Q_COUNT; ++i) mbar_init(&bars[i], i == Q_DSFULL ? 256u : 1u);
         *abort_flag = 0;
         mbar_fence_init();
     }
@@ -358,9 +379,10 @@ __global__ void __launch_bounds__(192, 1) dq_kernel(const __grid_constant__ BwdT
                 if (t == 0 || l != level(t - 1)) { wait(Q_QFULL, nq); ++nq; }
                 wait(Q_KFULL + slot, t >> 1);
                 wait(Q_VFULL + slot, t >> 1);
-                if (t > 0) wait(Q_SEMPTY, t - 1);  // S / dP of the previous step have been read
                 tc_fence_after_sync();
                 if (!ok) break;
+                // these overwrite S and dS of the previous step: in-order execution puts them after its dQ product,
+                // and that product was only issued once every thread had finished reading (Q_DSFULL)
                 mma_kk(tmem + colS, smem_u32(sQ), smem_u32(sK + slot * kSlotBytes), HD, idescS, false);
                 mma_kk(tmem + colDP, smem_u32(sDO), smem_u32(sV + slot * kSlotBytes), HD, idescS, false);
                 umma_commit(&bars[Q_SFULL]);
@@ -369,14 +391,14 @@ __global__ void __launch_bounds__(192, 1) dq_kernel(const __grid_constant__ BwdT
                 wait(Q_DSFULL, t);
                 tc_fence_after_sync();
                 if (!ok) break;
-                mma_kn(tmem + colDQ, smem_u32(sDS), smem_u32(sK + slot * kSlotBytes), idescD,
-                       !(t == 0 || l != level(t - 1)));
-                umma_commit(&bars[Q_DQDONE]);
+                mma_tn(tmem + colDQ, tmem + colDP, smem_u32(sK + slot * kSlotBytes), idescD, !(t == 0 || l != level(t - 1)));
                 umma_commit(&bars[Q_KEMPTY + slot]);
+                if (t == T - 1) umma_commit(&bars[Q_FINAL]);
             }
         }
     } else {
-        const int q4 = warp & 3, row = q4 * 32 + lane, tid = threadIdx.x - 64;
+        const int q4 = warp & 3, h = (warp - 2) >> 2, row = q4 * 32 + lane;
+        const int tid = threadIdx.x - 64;
         const uint32_t tlane = tmem + ((uint32_t)(q4 * 32) << 16);
         const size_t qi = (size_t)s * p.Lp + I * kTile + row;
         const float sl2 = p.scale * kLog2e;
@@ -385,10 +407,11 @@ __global__ void __launch_bounds__(192, 1) dq_kernel(const __grid_constant__ BwdT
         if (GATE) gi2 = p.G[qi] * kLog2e;
         bool ok = true;
         uint32_t rs[32], rp[32];
+        constexpr int CW = HD / 2;
         auto flush_dq = [&](int lvl) {
-            float* dst = p.dqv + ((size_t)ver_row(qslot(lvl, I), I) + row) * HD;
-            for (int c = 0; c < HD / 32; ++c) {
-                tmem_ld32(tlane + colDQ + c * 32, rs);
+            float* dst = p.dqv + ((size_t)ver_row(qslot(lvl, I), I) + row) * HD + h * CW;
+            for (int c = 0; c < CW / 32; ++c) {
+                tmem_ld32(tlane + colDQ + h * CW + c * 32, rs);
                 tmem_ld_wait();
 #pragma unroll
                 for (int x = 0; x < 8; ++x)
@@ -400,47 +423,49 @@ __global__ void __launch_bounds__(192, 1) dq_kernel(const __grid_constant__ BwdT
         for (int t = 0; t < T; ++t) {
             const int J = I - 1 - t, b = t & 1;
             if (GATE) {
-                gk[b * kTile + tid] = p.G[(size_t)s * p.Lp + J * kTile + tid] * kLog2e;
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (tid < kTile) gk[b * kTile + tid] = p.G[(size_t)s * p.Lp + J * kTile + tid] * kLog2e;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
             }
             if (ok && !mbar_wait(&bars[Q_SFULL], t & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
-            if (t > 0 && ok && !mbar_wait(&bars[Q_DQDONE], (t - 1) & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after_sync();
             if (ok) {
                 if (t >= 1 && level(t) != level(t - 1)) flush_dq(level(t - 1));
-                for (int c = 0; c < 4; ++c) {
-                    tmem_ld32(tlane + colS + c * 32, rs);
-                    tmem_ld32(tlane + colDP + c * 32, rp);
+                uint32_t pk[32];
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int c0 = h * 64 + c * 32;   // key columns of this pass
+                    tmem_ld32(tlane + colS + c0, rs);
+                    tmem_ld32(tlane + colDP + c0, rp);
                     tmem_ld_wait();
-                    uint32_t pk[16];
 #pragma unroll
                     for (int x = 0; x < 32; x += 2) {
                         float v0 = __uint_as_float(rs[x]) * sl2 - lse2, v1 = __uint_as_float(rs[x + 1]) * sl2 - lse2;
                         if (GATE) {
-                            v0 += gi2 - gk[b * kTile + c * 32 + x];
-                            v1 += gi2 - gk[b * kTile + c * 32 + x + 1];
+                            v0 += gi2 - gk[b * kTile + c0 + x];
+                            v1 += gi2 - gk[b * kTile + c0 + x + 1];
                         }
                         const float d0 = ex2(v0) * (__uint_as_float(rp[x]) - delta);
                         const float d1 = ex2(v1) * (__uint_as_float(rp[x + 1]) - delta);
                         if (GATE) dsum += d0 + d1;
-                        pk[x >> 1] = pack_bf16(d0, d1);
+                        pk[c * 16 + (x >> 1)] = pack_bf16(d0, d1);
                     }
-                    store_row_chunk(sDS, row, c, pk);
                 }
+                tmem_st32(tlane + colDP + h * 64, pk);
+                tmem_st_wait();
             }
             tc_fence_before_sync();
-            mbar_arrive(&bars[Q_SEMPTY]);
-            fence_proxy_async_smem();
             mbar_arrive(&bars[Q_DSFULL]);
         }
-        if (ok && !mbar_wait(&bars[Q_DQDONE], (T - 1) & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
+        if (ok && !mbar_wait(&bars[Q_FINAL], 0, abort_flag, ST_DQ_COMPUTE)) ok = false;
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after_sync();
-        if (ok) {
-            flush_dq(level(T - 1));
-            if (GATE) p.dGrow[qi] = dsum;
+        if (GATE) {
+            if (h == 1) dsum_x[row] = dsum;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (h == 0 && ok) p.dGrow[qi] = dsum + dsum_x[row];
         }
+        if (ok) flush_dq(level(T - 1));
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -482,19 +507,19 @@ cudaError_t set_smem(K kern, int bytes) {
     return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
-constexpr int kDkvSmem = 6 * kSlotBytes + 256 + 2 * 3 * kTile * 4 + 1024;
-constexpr int kDqSmem = 7 * kSlotBytes + 256 + 2 * kTile * 4 + 1024;
+constexpr int kDkvSmem = 6 * kSlotBytes + 256 + (2 * 3 + 1) * kTile * 4 + 1024;
+constexpr int kDqSmem = 6 * kSlotBytes + 256 + 3 * kTile * 4 + 1024;
 
 template <int HD, bool GATE>
 cudaError_t launch_one(const BwdTensorMaps& tm, const BwdParams& p, int which, cudaStream_t st) {
     if (which == 0) {
         cudaError_t e = set_smem(dkv_kernel<HD, GATE>, kDkvSmem);
         if (e != cudaSuccess) return e;
-        dkv_kernel<HD, GATE><<<dim3(p.N, p.S), 192, kDkvSmem, st>>>(tm, p);
+        dkv_kernel<HD, GATE><<<dim3(p.N, p.S), 320, kDkvSmem, st>>>(tm, p);
     } else {
         cudaError_t e = set_smem(dq_kernel<HD, GATE>, kDqSmem);
         if (e != cudaSuccess) return e;
-        dq_kernel<HD, GATE><<<dim3(p.N, p.S), 192, kDqSmem, st>>>(tm, p);
+        dq_kernel<HD, GATE><<<dim3(p.N, p.S), 320, kDqSmem, st>>>(tm, p);
     }
     return cudaGetLastError();
 }
