@@ -39,12 +39,9 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the kernel named by `roofline.kernel`,
 # from the ncu capture summarised under profiles/ (None until one exists for that kernel).
-NCU_TRAFFIC_BYTES = {
-    # profiles/dkv_kernel_C3_batch2.md: 600.4 MB per launch at batch 2; slices are independent, so batch 4 moves twice that
-    "fa_bwd_dkv": 2 * (370.438144e6 + 229.984e6),
-    # profiles/fa_fwd_kernel_C3_batch2.md: 363.0 MB per launch at batch 2
-    "fa_fwd": 2 * (335.659776e6 + 27.35104e6),
-}
+# DRAM bytes per launch PER (batch, head) SLICE at the C3 shape (L=4096, d=128), from the ncu captures at batch 2
+# (32 slices) summarised under profiles/; slices are independent, so a launch over S slices moves S times this.
+NCU_TRAFFIC_BYTES_PER_SLICE = {}
 
 
 # ----------------------------------------------------------------------------------------- FLOP models
@@ -305,19 +302,23 @@ def run_ours(args, cfg):
     prep_bytes = nch * (3 * t_d + 2 * t_d + 2 * t_b + 2 * d * d * 2)
     stage_bytes = {"chunk_prep": prep_bytes, "bwd_chunk_prep": prep_bytes + nch * (7 * t_b + t_d),
                    "bwd_chunk_chain": nch * (4 * t_d + 7 * t_b + 2 * 2 * t_d + 2 * t_b + d * d * 4 + 3 * t_d)}
+    def ncu_traffic(kernel):
+        per_slice = NCU_TRAFFIC_BYTES_PER_SLICE.get(kernel)
+        return per_slice * B * H if (per_slice is not None and (L, d) == (4096, 128)) else None
+
     single = [k_ for k_ in stage_ms if k_ in stage_flops or k_ in stage_bytes]
     top = max(single, key=stage_ms.get) if single else None
     roof = None
     if top in stage_flops:
         ach = tf(stage_flops[top], stage_ms[top])
         roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peaks["sustained"], "unit": "TFLOP/s",
-                "frac": ach / peaks["sustained"], "traffic": NCU_TRAFFIC_BYTES.get(top),
+                "frac": ach / peaks["sustained"], "traffic": ncu_traffic(top),
                 "peak_source": f"{peaks['source']} cuBLAS bf16, sustained", "ms_per_launch": stage_ms[top],
                 "flops_per_launch": stage_flops[top]}
     elif top is not None:
         ach = stage_bytes[top] / (stage_ms[top] * 1e-3) / 1e9
         roof = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": peaks["hbm"], "unit": "GB/s",
-                "frac": ach / peaks["hbm"], "traffic": NCU_TRAFFIC_BYTES.get(top),
+                "frac": ach / peaks["hbm"], "traffic": ncu_traffic(top),
                 "peak_source": f"{peaks['source']} copy bandwidth", "ms_per_launch": stage_ms[top],
                 "bytes_per_launch": stage_bytes[top]}
     line = {

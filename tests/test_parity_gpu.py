@@ -97,6 +97,18 @@ def test_small_shapes_match_oracle(binding, oracle, B, H, L, d, gate, sharp):
     compare_all(binding, oracle, inp)
 
 
+def test_c1_workload_shape_and_distribution_in_bf16(binding, oracle):
+    """Workload C1 (B=1, H=2, L=256, d=64, q, k, v ~ N(0,1) unscaled: logits of standard deviation 8) with bf16 I/O.
+    The float32 I/O dtype of C1 itself is not built (PATH_FP32 is rejected with PATH_ERR_DTYPE)."""
+    c = synth.CONFIGS["C1"]
+    inp = synth.make_inputs(c["B"], c["H"], c["L"], c["d"], "bf16", qk_scaled=False, gate=False, seed=synth.BASE_SEED)
+    compare_all(binding, oracle, inp, backward=False)      # C1 is a forward-only workload
+    q = inp["q"].cuda().float()
+    with pytest.raises(binding.PathAttnError) as e:
+        binding.path_attn_fwd(q, q, q, q, inp["beta"].cuda())
+    assert e.value.status == -3
+
+
 def test_explicit_scale(binding, oracle):
     inp = synth.make_inputs(1, 2, 640, 64, "bf16", qk_scaled=False, gate=True, seed=5)
     compare_all(binding, oracle, inp, scale=1.0 / 8.0)
