@@ -134,8 +134,8 @@ struct BwdParams {
     float* dsd;          // [S*N][128 q][128 k] lower(dS) of the diagonal chunks (not yet multiplied by scale)
     float* dG;           // [S][Lp] minus the column sums of dS (gated problems only)
     float* dGrow;        // [S][Lp] row sums of dS over the off-diagonal chunks (gated problems only)
-    const float* lse2;   // [S][Lp] lse * log2(e)
-    const float* delta;  // [S][Lp] dO . O
+    const float* lse2;   // [S][Lp] (gate prefix - lse) * log2(e)
+    const float* delta;  // [S][Lp] -(dO . O)
     const float* G;      // [S][Lp] gate prefix or nullptr
     uint32_t* status;
     int S, L, Lp, N;
@@ -143,8 +143,8 @@ struct BwdParams {
 };
 
 cudaError_t launch_fa_bwd(const BwdTensorMaps& tm, const BwdParams& p, int hd, int which, cudaStream_t st);
-cudaError_t launch_rowstats(const void* o, const void* d_o, const float* lse, float* delta, float* lse2, int S, int L,
-                            int Lp, int hd, cudaStream_t st);
+cudaError_t launch_rowstats(const void* o, const void* d_o, const float* lse, const float* G, float* delta, float* lse2,
+                            int S, int L, int Lp, int hd, cudaStream_t st);
 cudaError_t launch_fa_fwd(const FwdTensorMaps& tm, const FwdParams& p, int hd, cudaStream_t st);
 
 }  // namespace path

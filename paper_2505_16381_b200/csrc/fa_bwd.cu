@@ -14,10 +14,15 @@
 //   dq_kernel : one CTA per query chunk I, sweeps J = I-1..0: S = Q K^T, dP = dO V^T, dQ += dS K.
 // The accumulator of a version is flushed to global memory when the sweep crosses into the next level.
 // P^T / dS^T (dkv) and dS (dq) never touch shared memory: they overwrite the first half of the columns their thread
-// read, as packed bf16, and enter the second products as tensor-memory A operands.  The shared memory this frees
-// double-buffers the per-step tiles.
-// Warps: 0 = TMA producer, 1 = tcgen05 MMA issuer, 2-9 = elementwise math (two warps per TMEM lane quadrant, each
-// taking 64 of the 128 columns of a row).
+// read, as packed bf16, and enter the second products as tensor-memory A operands.
+//
+// The elementwise work of a step is split in two so that it overlaps the tensor pipe: part A turns S into P (the
+// exponentials) as soon as S is there, while the dP product still runs; part B forms dS once dP has arrived.  The
+// products are issued in the order  dV(t), S(t+1), dK(t), dP(t+1)  (dkv) and  dQ(t), dP(t+1), S(t+2)  (dq, which has
+// room for two S tiles), so the pipe always has the next step's logits in flight.
+// Warps: 0 = TMA producer, 1 = tcgen05 MMA issuer, 2-3 idle (their registers go to the others), 4-11 = elementwise
+// math (two warps per TMEM lane quadrant, each taking 64 of the 128 columns of a row).
+#include <type_traits>
 #include "common.cuh"
 #include "tc5.cuh"
 
@@ -30,11 +35,42 @@ constexpr int kTile = 128;
 constexpr uint32_t kSlotBytes = 32768;
 constexpr uint32_t kPanelBytes = 16384;
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr uint32_t kSmemAlloc = 232448;   // everything an SM offers one CTA
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+// Two-wide float arithmetic on register pairs.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// Plain (untiled) bulk copy global -> shared, completion counted in bytes on `bar`; 16-byte aligned, size % 16 == 0.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
 }
 __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                         uint32_t accumulate) {
@@ -66,32 +102,40 @@ __device__ __forceinline__ void tma_tile(uint8_t* dst, const CUtensorMap* m, uin
 }
 
 // ------------------------------------------------------------------------------------------------ dK, dV
-enum { K_KFULL = 0, K_KEMPTY, K_VFULL, K_QFULL, K_QEMPTY = K_QFULL + 2, K_DOFULL = K_QEMPTY + 2,
-       K_DOEMPTY = K_DOFULL + 2, K_SFULL = K_DOEMPTY + 2, K_PFULL, K_FINAL, K_COUNT };
+enum { K_KFULL = 0, K_KEMPTY, K_VFULL, K_QFULL, K_QEMPTY = K_QFULL + 3, K_DOFULL = K_QEMPTY + 3,
+       K_DOEMPTY = K_DOFULL + 2, K_SFULL = K_DOEMPTY + 2, K_DPFULL, K_PFULL, K_DSFULL, K_FINAL,
+       K_STFULL, K_STEMPTY = K_STFULL + 2, K_COUNT = K_STEMPTY + 2 };
+constexpr uint32_t kDkvStat = 7 * kSlotBytes + 256;           // [2][2][128] floats: -lse2 (plus gate), -delta
+constexpr uint32_t kDkvTotal = kDkvStat + 2 * 2 * kTile * 4;
 
 template <int HD, bool GATE>
-__global__ void __launch_bounds__(320, 1) dkv_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
-    extern __shared__ uint8_t smem_raw[];
+__global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    if ((uint32_t)(smem - smem_raw) + kDkvTotal > kSmemAlloc) {   // uniform over the CTA
+        if (threadIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)ST_DKV_PRODUCER);
+        return;
+    }
     uint8_t* sK = smem;
     uint8_t* sV = sK + kSlotBytes;
-    uint8_t* sQ = sV + kSlotBytes;          // 2 slots: rawQ, Xqn, then Q of step t >= 1 in slot (t + 1) & 1
-    uint8_t* sDO = sQ + 2 * kSlotBytes;     // 2 slots: dO(0), Yt, then dO of step t >= 1 in slot (t + 1) & 1
-    uint64_t* bars = (uint64_t*)(sDO + 2 * kSlotBytes);
+    uint8_t* sQ = sV + kSlotBytes;          // 3 slots: rawQ, Xqn, then Q of step t >= 1 as item t + 1
+    uint8_t* sDO = sQ + 3 * kSlotBytes;     // 2 slots: dO(0), Yt, then dO of step t >= 1 as item t + 1
+    uint64_t* bars = (uint64_t*)(smem + 7 * kSlotBytes);
     uint32_t* tmem_slot = (uint32_t*)(bars + K_COUNT);
     volatile uint32_t* abort_flag = (volatile uint32_t*)(tmem_slot + 1);
-    float* rowstat = (float*)(smem + 6 * kSlotBytes + 256);  // [2][3][128]: lse2, delta, G of the query chunk
-    float* dsum_x = rowstat + 2 * 3 * kTile;                 // [128] exchange of the gate row sums
+    float* rowstat = (float*)(smem + kDkvStat);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int J = blockIdx.x, s = blockIdx.y;
     const int T = p.N - J;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < K_COUNT; ++i) mbar_init(&bars[i], i == K_PFULL ? 256u : 1u);
+        for (int i = 0; i < K_COUNT; ++i)
+            mbar_init(&bars[i], (i == K_PFULL || i == K_DSFULL || i == K_STEMPTY || i == K_STEMPTY + 1) ? 256u : 1u);
         *abort_flag = 0;
         mbar_fence_init();
     }
+    if (warp == 2 && lane < 8) tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(&tm) + lane);
     if (warp == 1) tmem_alloc(tmem_slot, 512);
     tc_fence_before_sync();
     __syncthreads();
@@ -102,19 +146,27 @@ __global__ void __launch_bounds__(320, 1) dkv_kernel(const __grid_constant__ Bwd
     auto ver_row = [&](int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
     auto level = [&](int t) { return t == 0 ? -1 : msb32((unsigned)((J + t) ^ J)); };
 
-    if (warp == 0) {
-        if (lane == 0) {
+    if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+        if (warp == 0 && lane == 0) {
             bool ok = true;
             int nk = 0;
             auto wait_empty = [&](int bar, int use) {
                 if (ok && !mbar_wait(&bars[bar], (use & 1) ^ 1, abort_flag, ST_DKV_PRODUCER)) ok = false;
             };
-            auto ring_load = [&](uint8_t* base, int bfull, int bempty, int item, const CUtensorMap* m, int kdim, int row0) {
-                const int slot = item & 1;
-                wait_empty(bempty + slot, item >> 1);
+            auto load_q = [&](int item, const CUtensorMap* m, int kdim, int row0) {
+                const int slot = item % 3;
+                wait_empty(K_QEMPTY + slot, item / 3);
                 if (!ok) return;
-                mbar_expect_tx(&bars[bfull + slot], (uint32_t)(kTile * kdim * 2));
-                tma_tile(base + slot * kSlotBytes, m, &bars[bfull + slot], kdim, row0);
+                mbar_expect_tx(&bars[K_QFULL + slot], (uint32_t)(kTile * kdim * 2));
+                tma_tile(sQ + slot * kSlotBytes, m, &bars[K_QFULL + slot], kdim, row0);
+            };
+            auto load_do = [&](int item, const CUtensorMap* m, int kdim, int row0) {
+                const int slot = item & 1;
+                wait_empty(K_DOEMPTY + slot, item >> 1);
+                if (!ok) return;
+                mbar_expect_tx(&bars[K_DOFULL + slot], (uint32_t)(kTile * kdim * 2));
+                tma_tile(sDO + slot * kSlotBytes, m, &bars[K_DOFULL + slot], kdim, row0);
             };
             for (int t = 0; t < T && ok; ++t) {
                 const int I = J + t, l = level(t);
@@ -127,20 +179,25 @@ __global__ void __launch_bounds__(320, 1) dkv_kernel(const __grid_constant__ Bwd
                     ++nk;
                 }
                 if (t == 0) {
+                    load_q(0, &tm.q_raw, HD, rowJ);
+                    load_q(1, &tm.xqn, kTile, rowJ);
+                    load_do(1, &tm.yt, kTile, rowJ);
                     mbar_expect_tx(&bars[K_VFULL], kTile * HD * 2);
                     tma_tile(sV, &tm.v, &bars[K_VFULL], HD, rowJ);
-                    ring_load(sQ, K_QFULL, K_QEMPTY, 0, &tm.q_raw, HD, rowJ);
-                    ring_load(sDO, K_DOFULL, K_DOEMPTY, 0, &tm.d_o, HD, rowJ);
-                    ring_load(sQ, K_QFULL, K_QEMPTY, 1, &tm.xqn, kTile, rowJ);
-                    ring_load(sDO, K_DOFULL, K_DOEMPTY, 1, &tm.yt, kTile, rowJ);
+                    load_do(0, &tm.d_o, HD, rowJ);
                 } else {
-                    ring_load(sQ, K_QFULL, K_QEMPTY, t + 1, &tm.qv, HD, ver_row(qslot(l, I), I));
-                    ring_load(sDO, K_DOFULL, K_DOEMPTY, t + 1, &tm.d_o, HD, s * p.Lp + I * kTile);
+                    load_q(t + 1, &tm.qv, HD, ver_row(qslot(l, I), I));
+                    load_do(t + 1, &tm.d_o, HD, s * p.Lp + I * kTile);
                 }
+                // per-query statistics of the step
+                wait_empty(K_STEMPTY + (t & 1), t >> 1);
+                if (!ok) break;
+                mbar_expect_tx(&bars[K_STFULL + (t & 1)], 2 * kTile * 4);
+                const size_t gi = (size_t)s * p.Lp + I * kTile;
+                bulk_load(rowstat + (t & 1) * 2 * kTile, p.lse2 + gi, kTile * 4, &bars[K_STFULL + (t & 1)]);
+                bulk_load(rowstat + (t & 1) * 2 * kTile + kTile, p.delta + gi, kTile * 4, &bars[K_STFULL + (t & 1)]);
             }
-        }
-    } else if (warp == 1) {
-        if (lane == 0) {
+        } else if (warp == 1 && lane == 0) {
             constexpr uint32_t idescT = umma_idesc(128, 128, 0, 0);
             constexpr uint32_t idescD = umma_idesc(128, HD, 0, 1);
             bool ok = true;
@@ -148,122 +205,198 @@ __global__ void __launch_bounds__(320, 1) dkv_kernel(const __grid_constant__ Bwd
             auto wait = [&](int bar, int parity) {
                 if (ok && !mbar_wait(&bars[bar], parity & 1, abort_flag, ST_DKV_MMA)) ok = false;
             };
+            auto q_addr = [&](int item) { return smem_u32(sQ + (item % 3) * kSlotBytes); };
+            auto do_addr = [&](int item) { return smem_u32(sDO + (item & 1) * kSlotBytes); };
+            // step 0: S^T of the diagonal chunk (two contractions) and its dP^T
+            wait(K_KFULL, nk); ++nk;
+            wait(K_QFULL + 0, 0);
+            wait(K_QFULL + 1, 0);
+            wait(K_DOFULL + 1, 0);
+            tc_fence_after_sync();
+            if (ok) {
+                mma_kk(tmem + colS, smem_u32(sK), q_addr(0), HD, idescT, false);
+                mma_kk(tmem + colS, do_addr(1), q_addr(1), kTile, idescT, true);
+                umma_commit(&bars[K_SFULL]);
+                umma_commit(&bars[K_QEMPTY + 0]);   // raw q and the two correction operands are only needed here
+                umma_commit(&bars[K_QEMPTY + 1]);
+                umma_commit(&bars[K_DOEMPTY + 1]);
+                if (T > 1) umma_commit(&bars[K_KEMPTY]);
+            }
+            wait(K_VFULL, 0);
+            wait(K_DOFULL + 0, 0);
+            tc_fence_after_sync();
+            if (ok) {
+                mma_kk(tmem + colDP, smem_u32(sV), do_addr(0), HD, idescT, false);
+                umma_commit(&bars[K_DPFULL]);
+            }
             for (int t = 0; t < T && ok; ++t) {
                 const int l = level(t);
-                const int item = (t == 0) ? 0 : t + 1, slot = item & 1;
-                const uint32_t aQ = smem_u32(sQ + slot * kSlotBytes), aDO = smem_u32(sDO + slot * kSlotBytes);
-                if (t == 0 || l != level(t - 1)) { wait(K_KFULL, nk); ++nk; }
-                wait(K_QFULL + slot, item >> 1);
-                wait(K_DOFULL + slot, item >> 1);
-                if (t == 0) { wait(K_VFULL, 0); wait(K_QFULL + 1, 0); wait(K_DOFULL + 1, 0); }
-                tc_fence_after_sync();
-                if (!ok) break;
-                mma_kk(tmem + colS, smem_u32(sK), aQ, HD, idescT, false);
-                if (t == 0) mma_kk(tmem + colS, smem_u32(sDO + kSlotBytes), smem_u32(sQ + kSlotBytes), kTile, idescT, true);
-                mma_kk(tmem + colDP, smem_u32(sV), aDO, HD, idescT, false);
-                umma_commit(&bars[K_SFULL]);
-                if (t == 0) {   // raw q and the two correction operands are only needed by the products above
-                    umma_commit(&bars[K_QEMPTY + 0]);
-                    umma_commit(&bars[K_QEMPTY + 1]);
-                    umma_commit(&bars[K_DOEMPTY + 1]);
-                }
-                if (t + 1 < T && level(t + 1) != l) umma_commit(&bars[K_KEMPTY]);
+                const int item = (t == 0) ? 0 : t + 1;
+                // dV += P^T dO
                 wait(K_PFULL, t);
                 tc_fence_after_sync();
                 if (!ok) break;
-                mma_tn(tmem + colDV, tmem + colS, aDO, idescD, t > 0);
-                if (t > 0) {
-                    mma_tn(tmem + colDK, tmem + colDP, aQ, idescD, !(t == 1 || l != level(t - 1)));
-                    umma_commit(&bars[K_QEMPTY + slot]);
+                mma_tn(tmem + colDV, tmem + colS, do_addr(item), idescD, t > 0);
+                umma_commit(&bars[K_DOEMPTY + (item & 1)]);
+                // S^T of the next step overwrites P^T: in-order execution puts it after the product above
+                if (t + 1 < T) {
+                    const int l1 = level(t + 1);
+                    if (l1 != l) { wait(K_KFULL, nk); ++nk; }
+                    wait(K_QFULL + (t + 2) % 3, (t + 2) / 3);
+                    tc_fence_after_sync();
+                    if (!ok) break;
+                    mma_kk(tmem + colS, smem_u32(sK), q_addr(t + 2), HD, idescT, false);
+                    umma_commit(&bars[K_SFULL]);
+                    if (t + 2 < T && level(t + 2) != l1) umma_commit(&bars[K_KEMPTY]);
                 }
-                umma_commit(&bars[K_DOEMPTY + slot]);
-                if (t == T - 1) umma_commit(&bars[K_FINAL]);
+                // dK += dS^T Q
+                wait(K_DSFULL, t);
+                tc_fence_after_sync();
+                if (!ok) break;
+                if (t > 0) {
+                    mma_tn(tmem + colDK, tmem + colDP, q_addr(item), idescD, !(t == 1 || l != level(t - 1)));
+                    umma_commit(&bars[K_QEMPTY + item % 3]);
+                }
+                if (t + 1 < T) {
+                    wait(K_DOFULL + ((t + 2) & 1), (t + 2) >> 1);
+                    tc_fence_after_sync();
+                    if (!ok) break;
+                    mma_kk(tmem + colDP, smem_u32(sV), do_addr(t + 2), HD, idescT, false);
+                    umma_commit(&bars[K_DPFULL]);
+                } else {
+                    umma_commit(&bars[K_FINAL]);
+                }
             }
         }
     } else {
-        const int q4 = warp & 3, h = (warp - 2) >> 2, row = q4 * 32 + lane;
-        const int tid = threadIdx.x - 64;       // 0..255
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        const int q4 = warp & 3, h = (warp - 4) >> 2, row = q4 * 32 + lane;
         const uint32_t tlane = tmem + ((uint32_t)(q4 * 32) << 16);
         const int kj = J * kTile + row;          // key position of this thread's row
         const float sl2 = p.scale * kLog2e;
         float gj2 = 0.f, dsum = 0.f;
         if (GATE) gj2 = p.G[(size_t)s * p.Lp + kj] * kLog2e;
         bool ok = true;
-        uint32_t rs[32], rp[32];
         constexpr int CW = HD / 2;               // accumulator columns per thread when flushing
         auto flush_dk = [&](int lvl) {
-            float* dst = p.dkv + ((size_t)ver_row(kslot(lvl, J), J) + row) * HD + h * CW;
+            float* dst = p.dkv + ((size_t)ver_row(kslot(lvl, J), J) + q4 * 32) * HD + h * CW;   // the warp's 32 rows
+#pragma unroll 1
             for (int c = 0; c < CW / 32; ++c) {
-                tmem_ld32(tlane + colDK + h * CW + c * 32, rs);
+                uint32_t r[32];
+                tmem_ld32(tlane + colDK + h * CW + c * 32, r);
                 tmem_ld_wait();
 #pragma unroll
-                for (int x = 0; x < 8; ++x)
-                    reinterpret_cast<float4*>(dst + c * 32)[x] =
-                        make_float4(__uint_as_float(rs[4 * x]) * p.scale, __uint_as_float(rs[4 * x + 1]) * p.scale,
-                                    __uint_as_float(rs[4 * x + 2]) * p.scale, __uint_as_float(rs[4 * x + 3]) * p.scale);
+                for (int x = 0; x < 32; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * p.scale);
+                warp_store_rows128(dst + c * 32, (size_t)HD * 4, r);
             }
         };
-        for (int t = 0; t < T; ++t) {
-            const int I = J + t, b = t & 1;
-            float* st_ = rowstat + b * 3 * kTile;
-            if (tid < kTile) {
-                const size_t gi = (size_t)s * p.Lp + I * kTile + tid;
-                st_[tid] = p.lse2[gi];
-                st_[kTile + tid] = p.delta[gi];
-                if (GATE) st_[2 * kTile + tid] = p.G[gi] * kLog2e;
-            }
-            asm volatile("bar.sync 1, 256;" ::: "memory");
+        const uint64_t sl2x2 = pack2(sl2, sl2), ngj2 = pack2(-gj2, -gj2);
+        auto step = [&](auto first_tag, const int t) {
+            constexpr bool FIRST = decltype(first_tag)::value;   // the diagonal chunk: causal mask, dSd written out
+            const float* st_ = rowstat + (t & 1) * 2 * kTile;   // [0,128): -lse2 (+gate), [128,256): -delta of the queries
+            const int c0 = h * 64;               // query columns of this thread
+            uint32_t pr[2][32];                  // S^T, then P^T (float bits)
+            // ---- part A: P^T = exp2(S^T * scale - lse)
+            if (ok && !mbar_wait(&bars[K_STFULL + (t & 1)], (t >> 1) & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
             if (ok && !mbar_wait(&bars[K_SFULL], t & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after_sync();
             if (ok) {
-                // S^T / dP^T ready means every earlier product has retired: dK of the finished level can be flushed
-                if (t >= 2 && level(t) != level(t - 1)) flush_dk(level(t - 1));
-                uint32_t pkP[32], pkS[32];
+                tmem_ld32(tlane + colS + c0, pr[0]);
+                tmem_ld32(tlane + colS + c0 + 32, pr[1]);
+                tmem_ld_wait();
+                uint32_t pk[32];
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    const int c0 = h * 64 + c * 32;      // query columns of this pass
-                    tmem_ld32(tlane + colS + c0, rs);
-                    tmem_ld32(tlane + colDP + c0, rp);
-                    tmem_ld_wait();
-                    float dsv[32];
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
-                    for (int x = 0; x < 32; ++x) {
-                        const int col = c0 + x;
-                        float v = __uint_as_float(rs[x]) * sl2 - st_[col];
-                        if (GATE) v += st_[2 * kTile + col] - gj2;
-                        float pr = ex2(v);
-                        if (t == 0 && col < row) pr = 0.f;
-                        const float ds = pr * (__uint_as_float(rp[x]) - st_[kTile + col]);
-                        dsum += ds;
-                        dsv[x] = ds;
-                        rs[x] = __float_as_uint(pr);
+                    for (int x = 0; x < 32; x += 4) {
+                        const float4 ls = *reinterpret_cast<const float4*>(st_ + c0 + c * 32 + x);
+                        uint64_t v01 = fma2(pack2(__uint_as_float(pr[c][x]), __uint_as_float(pr[c][x + 1])), sl2x2, pack2(ls.x, ls.y));
+                        uint64_t v23 = fma2(pack2(__uint_as_float(pr[c][x + 2]), __uint_as_float(pr[c][x + 3])), sl2x2, pack2(ls.z, ls.w));
+                        if (GATE) { v01 = add2(v01, ngj2); v23 = add2(v23, ngj2); }
+                        float e[4];
+                        unpack2(v01, e[0], e[1]);
+                        unpack2(v23, e[2], e[3]);
+#pragma unroll
+                        for (int y = 0; y < 4; ++y) {
+                            e[y] = ex2(e[y]);
+                            if (FIRST && c0 + c * 32 + x + y < row) e[y] = 0.f;
+                            pr[c][x + y] = __float_as_uint(e[y]);
+                        }
+                        pk[c * 16 + (x >> 1)] = pack_bf16(e[0], e[1]);
+                        pk[c * 16 + (x >> 1) + 1] = pack_bf16(e[2], e[3]);
                     }
-#pragma unroll
-                    for (int x = 0; x < 32; x += 2) {
-                        pkP[c * 16 + (x >> 1)] = pack_bf16(__uint_as_float(rs[x]), __uint_as_float(rs[x + 1]));
-                        pkS[c * 16 + (x >> 1)] = pack_bf16(dsv[x], dsv[x + 1]);
-                    }
-                    if (t == 0) {
-                        float* dsd = p.dsd + ((size_t)(s * p.N + J) * kTile) * kTile;
-#pragma unroll
-                        for (int x = 0; x < 32; ++x) dsd[(size_t)(c0 + x) * kTile + row] = dsv[x];
-                    }
-                }
-                tmem_st32(tlane + colS + h * 64, pkP);
-                tmem_st32(tlane + colDP + h * 64, pkS);
+                tmem_st32(tlane + colS + c0, pk);
                 tmem_st_wait();
             }
             tc_fence_before_sync();
             mbar_arrive(&bars[K_PFULL]);
-        }
+            // ---- part B: dS^T = P^T o (dP^T - delta)
+            if (ok && !mbar_wait(&bars[K_DPFULL], t & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            tc_fence_after_sync();
+            // dP^T ready means every product issued before it has retired: dK of a finished level is complete.  It is
+            // taken into registers now and written out after dS^T has been delivered, off the tensor pipe's path.
+            if (!FIRST && ok && t >= 2 && level(t) != level(t - 1)) flush_dk(level(t - 1));
+            const bool fl = false;
+            uint32_t fr[CW / 32][32];
+            if (ok) {
+                const float* dl_ = st_ + kTile;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t dp[32], pk[16];
+                    tmem_ld32(tlane + colDP + c0 + c * 32, dp);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int x = 0; x < 32; x += 4) {
+                        const float4 dl = *reinterpret_cast<const float4*>(dl_ + c0 + c * 32 + x);
+                        const uint64_t d01 = mul2(pack2(__uint_as_float(pr[c][x]), __uint_as_float(pr[c][x + 1])),
+                                                  add2(pack2(__uint_as_float(dp[x]), __uint_as_float(dp[x + 1])), pack2(dl.x, dl.y)));
+                        const uint64_t d23 = mul2(pack2(__uint_as_float(pr[c][x + 2]), __uint_as_float(pr[c][x + 3])),
+                                                  add2(pack2(__uint_as_float(dp[x + 2]), __uint_as_float(dp[x + 3])), pack2(dl.z, dl.w)));
+                        float d[4];
+                        unpack2(d01, d[0], d[1]);
+                        unpack2(d23, d[2], d[3]);
+                        if (GATE) dsum += (d[0] + d[1]) + (d[2] + d[3]);
+                        pk[x >> 1] = pack_bf16(d[0], d[1]);
+                        pk[(x >> 1) + 1] = pack_bf16(d[2], d[3]);
+                        if (FIRST) {
+#pragma unroll
+                            for (int y = 0; y < 4; ++y) dp[x + y] = __float_as_uint(d[y]);
+                        }
+                    }
+                    tmem_st16(tlane + colDP + c0 + c * 16, pk);
+                    if (FIRST) {
+                        float* dsd = p.dsd + ((size_t)(s * p.N + J) * kTile) * kTile;
+#pragma unroll
+                        for (int x = 0; x < 32; ++x) dsd[(size_t)(c0 + c * 32 + x) * kTile + row] = __uint_as_float(dp[x]);
+                    }
+                }
+                tmem_st_wait();
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&bars[K_DSFULL]);
+            mbar_arrive(&bars[K_STEMPTY + (t & 1)]);
+            if (fl) {
+                float* dst = p.dkv + ((size_t)ver_row(kslot(level(t - 1), J), J) + q4 * 32) * HD + h * CW;
+#pragma unroll
+                for (int c = 0; c < CW / 32; ++c) {
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) fr[c][x] = __float_as_uint(__uint_as_float(fr[c][x]) * p.scale);
+                    warp_store_rows128(dst + c * 32, (size_t)HD * 4, fr[c]);
+                }
+            }
+        };
+        step(std::true_type{}, 0);
+#pragma unroll 1
+        for (int t = 1; t < T; ++t) step(std::false_type{}, t);
         if (ok && !mbar_wait(&bars[K_FINAL], 0, abort_flag, ST_DKV_COMPUTE)) ok = false;
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after_sync();
         if (GATE) {   // the two threads of a key row add their halves of the column sum
-            if (h == 1) dsum_x[row] = dsum;
+            if (h == 1) rowstat[row] = dsum;
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (h == 0 && ok) p.dG[(size_t)s * p.Lp + kj] = -(dsum + dsum_x[row]);
+            if (h == 0 && ok) p.dG[(size_t)s * p.Lp + kj] = -(dsum + rowstat[row]);
         }
         if (ok) {
             if (T > 1) flush_dk(level(T - 1));
@@ -271,17 +404,33 @@ __global__ void __launch_bounds__(320, 1) dkv_kernel(const __grid_constant__ Bwd
                 float4* dst = reinterpret_cast<float4*>(p.dkv + ((size_t)ver_row(0, J) + row) * HD + h * CW);
                 for (int x = 0; x < CW / 4; ++x) dst[x] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
+            if (CW == 64) {   // 64 bf16 = one 128-byte line per row: coalesced exchange
+                uint32_t r0[32], r1[32], w[32];
+                tmem_ld32(tlane + colDV + h * CW, r0);
+                tmem_ld32(tlane + colDV + h * CW + 32, r1);
+                tmem_ld_wait();
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    w[x] = pack_bf16(__uint_as_float(r0[2 * x]), __uint_as_float(r0[2 * x + 1]));
+                    w[16 + x] = pack_bf16(__uint_as_float(r1[2 * x]), __uint_as_float(r1[2 * x + 1]));
+                }
+                const int row0 = J * kTile + q4 * 32;
+                warp_store_rows128((__nv_bfloat16*)p.dv + ((size_t)s * p.L + row0) * HD + h * CW, (size_t)HD * 2, w,
+                                   p.L - row0);
+            } else
+#pragma unroll 1
             for (int c = 0; c < CW / 32; ++c) {
-                tmem_ld32(tlane + colDV + h * CW + c * 32, rs);
+                uint32_t r[32];
+                tmem_ld32(tlane + colDV + h * CW + c * 32, r);
                 tmem_ld_wait();
                 if (kj < p.L) {
                     uint4* dst = reinterpret_cast<uint4*>((__nv_bfloat16*)p.dv + ((size_t)s * p.L + kj) * HD + h * CW + c * 32);
 #pragma unroll
                     for (int x = 0; x < 4; ++x)
-                        dst[x] = make_uint4(pack_bf16(__uint_as_float(rs[8 * x]), __uint_as_float(rs[8 * x + 1])),
-                                            pack_bf16(__uint_as_float(rs[8 * x + 2]), __uint_as_float(rs[8 * x + 3])),
-                                            pack_bf16(__uint_as_float(rs[8 * x + 4]), __uint_as_float(rs[8 * x + 5])),
-                                            pack_bf16(__uint_as_float(rs[8 * x + 6]), __uint_as_float(rs[8 * x + 7])));
+                        dst[x] = make_uint4(pack_bf16(__uint_as_float(r[8 * x]), __uint_as_float(r[8 * x + 1])),
+                                            pack_bf16(__uint_as_float(r[8 * x + 2]), __uint_as_float(r[8 * x + 3])),
+                                            pack_bf16(__uint_as_float(r[8 * x + 4]), __uint_as_float(r[8 * x + 5])),
+                                            pack_bf16(__uint_as_float(r[8 * x + 6]), __uint_as_float(r[8 * x + 7])));
                 }
             }
         }
@@ -296,76 +445,90 @@ __global__ void __launch_bounds__(320, 1) dkv_kernel(const __grid_constant__ Bwd
 }
 
 // ------------------------------------------------------------------------------------------------ dQ
-enum { Q_QFULL = 0, Q_QEMPTY, Q_DOFULL, Q_KFULL, Q_KEMPTY = Q_KFULL + 2, Q_VFULL = Q_KEMPTY + 2,
-       Q_VEMPTY = Q_VFULL + 2, Q_SFULL = Q_VEMPTY + 2, Q_DSFULL, Q_FINAL, Q_COUNT };
+enum { Q_QFULL = 0, Q_QEMPTY, Q_DOFULL, Q_KFULL, Q_KEMPTY = Q_KFULL + 3, Q_VFULL = Q_KEMPTY + 3,
+       Q_VEMPTY = Q_VFULL + 2, Q_SFULL = Q_VEMPTY + 2, Q_DPFULL = Q_SFULL + 2, Q_DSFULL, Q_FINAL,
+       Q_GKFULL, Q_GKEMPTY = Q_GKFULL + 2, Q_COUNT = Q_GKEMPTY + 2 };
+constexpr uint32_t kDqGk = 7 * kSlotBytes + 256;              // [2][128] gate prefix of the key chunk, [128] exchange
+constexpr uint32_t kDqTotal = kDqGk + 3 * kTile * 4;
 
 template <int HD, bool GATE>
-__global__ void __launch_bounds__(320, 1) dq_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
+__global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
     const int I = (int)gridDim.x - 1 - (int)blockIdx.x, s = blockIdx.y;
     if (I == 0) {  // chunk 0 has no earlier keys: its boundary-adjusted queries get a zero gradient from the sweep
         float4* dst = reinterpret_cast<float4*>(p.dqv + (size_t)s * p.Lp * HD);
         for (int i = threadIdx.x; i < kTile * HD / 4; i += blockDim.x) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         return;
     }
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    if ((uint32_t)(smem - smem_raw) + kDqTotal > kSmemAlloc) {   // uniform over the CTA
+        if (threadIdx.x == 0) atomicCAS(p.status, 0u, (uint32_t)ST_DQ_PRODUCER);
+        return;
+    }
     uint8_t* sQ = smem;
     uint8_t* sDO = sQ + kSlotBytes;
-    uint8_t* sK = sDO + kSlotBytes;        // 2 slots
-    uint8_t* sV = sK + 2 * kSlotBytes;     // 2 slots
-    uint64_t* bars = (uint64_t*)(sV + 2 * kSlotBytes);
+    uint8_t* sK = sDO + kSlotBytes;        // 3 slots
+    uint8_t* sV = sK + 3 * kSlotBytes;     // 2 slots
+    uint64_t* bars = (uint64_t*)(smem + 7 * kSlotBytes);
     uint32_t* tmem_slot = (uint32_t*)(bars + Q_COUNT);
     volatile uint32_t* abort_flag = (volatile uint32_t*)(tmem_slot + 1);
-    float* gk = (float*)(smem + 6 * kSlotBytes + 256);  // [2][128] gate prefix of the key chunk
-    float* dsum_x = gk + 2 * kTile;                     // [128]
+    float* gk = (float*)(smem + kDqGk);
+    float* dsum_x = gk + 2 * kTile;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int T = I;  // steps t = 0..I-1, J = I-1-t
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < Q_COUNT; ++i) mbar_init(&bars[i], i == Q_DSFULL ? 256u : 1u);
+        for (int i = 0; i < Q_COUNT; ++i)
+            mbar_init(&bars[i], (i == Q_DSFULL || i == Q_GKEMPTY || i == Q_GKEMPTY + 1) ? 256u : 1u);
         *abort_flag = 0;
         mbar_fence_init();
     }
+    if (warp == 2 && lane < 8) tma_prefetch_desc(reinterpret_cast<const CUtensorMap*>(&tm) + lane);
     if (warp == 1) tmem_alloc(tmem_slot, 512);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
-    constexpr uint32_t colS = 0, colDP = 128, colDQ = 256;
+    constexpr uint32_t colS = 0, colDP = 256, colDQ = 384;   // two S tiles at 0 and 128
     auto ver_row = [&](int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
     auto level = [&](int t) { return msb32((unsigned)(I ^ (I - 1 - t))); };
 
-    if (warp == 0) {
-        if (lane == 0) {
+    if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+        if (warp == 0 && lane == 0) {
             bool ok = true;
             int nq = 0;
-            auto wait_empty = [&](int bar, int parity) {
-                if (ok && !mbar_wait(&bars[bar], parity & 1, abort_flag, ST_DQ_PRODUCER)) ok = false;
+            auto wait_empty = [&](int bar, int use) {
+                if (ok && !mbar_wait(&bars[bar], (use & 1) ^ 1, abort_flag, ST_DQ_PRODUCER)) ok = false;
             };
             mbar_expect_tx(&bars[Q_DOFULL], kTile * HD * 2);
             tma_tile(sDO, &tm.d_o, &bars[Q_DOFULL], HD, s * p.Lp + I * kTile);
             for (int t = 0; t < T && ok; ++t) {
-                const int J = I - 1 - t, l = level(t), slot = t & 1;
+                const int J = I - 1 - t, l = level(t);
                 if (t == 0 || l != level(t - 1)) {
-                    wait_empty(Q_QEMPTY, (nq & 1) ^ 1);
+                    wait_empty(Q_QEMPTY, nq);
                     if (!ok) break;
                     mbar_expect_tx(&bars[Q_QFULL], kTile * HD * 2);
                     tma_tile(sQ, &tm.qv, &bars[Q_QFULL], HD, ver_row(qslot(l, I), I));
                     ++nq;
                 }
-                wait_empty(Q_KEMPTY + slot, ((t >> 1) & 1) ^ 1);
+                wait_empty(Q_KEMPTY + t % 3, t / 3);
                 if (!ok) break;
-                mbar_expect_tx(&bars[Q_KFULL + slot], kTile * HD * 2);
-                tma_tile(sK + slot * kSlotBytes, &tm.kv, &bars[Q_KFULL + slot], HD, ver_row(kslot(l, J), J));
-                wait_empty(Q_VEMPTY + slot, ((t >> 1) & 1) ^ 1);
+                mbar_expect_tx(&bars[Q_KFULL + t % 3], kTile * HD * 2);
+                tma_tile(sK + (t % 3) * kSlotBytes, &tm.kv, &bars[Q_KFULL + t % 3], HD, ver_row(kslot(l, J), J));
+                wait_empty(Q_VEMPTY + (t & 1), t >> 1);
                 if (!ok) break;
-                mbar_expect_tx(&bars[Q_VFULL + slot], kTile * HD * 2);
-                tma_tile(sV + slot * kSlotBytes, &tm.v, &bars[Q_VFULL + slot], HD, s * p.Lp + J * kTile);
+                mbar_expect_tx(&bars[Q_VFULL + (t & 1)], kTile * HD * 2);
+                tma_tile(sV + (t & 1) * kSlotBytes, &tm.v, &bars[Q_VFULL + (t & 1)], HD, s * p.Lp + J * kTile);
+                if (GATE) {   // gate prefix of the key chunk
+                    wait_empty(Q_GKEMPTY + (t & 1), t >> 1);
+                    if (!ok) break;
+                    mbar_expect_tx(&bars[Q_GKFULL + (t & 1)], kTile * 4);
+                    bulk_load(gk + (t & 1) * kTile, p.G + (size_t)s * p.Lp + J * kTile, kTile * 4, &bars[Q_GKFULL + (t & 1)]);
+                }
             }
-        }
-    } else if (warp == 1) {
-        if (lane == 0) {
+        } else if (warp == 1 && lane == 0) {
             constexpr uint32_t idescS = umma_idesc(128, 128, 0, 0);
             constexpr uint32_t idescD = umma_idesc(128, HD, 0, 1);
             bool ok = true;
@@ -373,89 +536,140 @@ __global__ void __launch_bounds__(320, 1) dq_kernel(const __grid_constant__ BwdT
             auto wait = [&](int bar, int parity) {
                 if (ok && !mbar_wait(&bars[bar], parity & 1, abort_flag, ST_DQ_MMA)) ok = false;
             };
-            wait(Q_DOFULL, 0);
-            for (int t = 0; t < T && ok; ++t) {
-                const int l = level(t), slot = t & 1;
-                if (t == 0 || l != level(t - 1)) { wait(Q_QFULL, nq); ++nq; }
-                wait(Q_KFULL + slot, t >> 1);
-                wait(Q_VFULL + slot, t >> 1);
+            auto issue_s = [&](int t) {      // S(t) into tile t & 1
+                if (t == 0 || level(t) != level(t - 1)) { wait(Q_QFULL, nq); ++nq; }
+                wait(Q_KFULL + t % 3, t / 3);
                 tc_fence_after_sync();
-                if (!ok) break;
-                // these overwrite S and dS of the previous step: in-order execution puts them after its dQ product,
-                // and that product was only issued once every thread had finished reading (Q_DSFULL)
-                mma_kk(tmem + colS, smem_u32(sQ), smem_u32(sK + slot * kSlotBytes), HD, idescS, false);
-                mma_kk(tmem + colDP, smem_u32(sDO), smem_u32(sV + slot * kSlotBytes), HD, idescS, false);
-                umma_commit(&bars[Q_SFULL]);
-                umma_commit(&bars[Q_VEMPTY + slot]);
-                if (t + 1 < T && level(t + 1) != l) umma_commit(&bars[Q_QEMPTY]);
+                if (!ok) return;
+                mma_kk(tmem + colS + (t & 1) * 128, smem_u32(sQ), smem_u32(sK + (t % 3) * kSlotBytes), HD, idescS, false);
+                umma_commit(&bars[Q_SFULL + (t & 1)]);
+                if (t + 1 < T && level(t + 1) != level(t)) umma_commit(&bars[Q_QEMPTY]);
+            };
+            auto issue_dp = [&](int t) {
+                wait(Q_VFULL + (t & 1), t >> 1);
+                tc_fence_after_sync();
+                if (!ok) return;
+                mma_kk(tmem + colDP, smem_u32(sDO), smem_u32(sV + (t & 1) * kSlotBytes), HD, idescS, false);
+                umma_commit(&bars[Q_DPFULL]);
+                umma_commit(&bars[Q_VEMPTY + (t & 1)]);
+            };
+            wait(Q_DOFULL, 0);
+            issue_s(0);
+            issue_dp(0);
+            if (T > 1) issue_s(1);
+            for (int t = 0; t < T && ok; ++t) {
+                // dQ += dS K.  dP of the next step overwrites dS, S(t+2) the tile whose P every thread has taken into
+                // registers before it delivered dS: in-order execution keeps both behind what they replace.
                 wait(Q_DSFULL, t);
                 tc_fence_after_sync();
                 if (!ok) break;
-                mma_tn(tmem + colDQ, tmem + colDP, smem_u32(sK + slot * kSlotBytes), idescD, !(t == 0 || l != level(t - 1)));
-                umma_commit(&bars[Q_KEMPTY + slot]);
+                mma_tn(tmem + colDQ, tmem + colDP, smem_u32(sK + (t % 3) * kSlotBytes), idescD,
+                       !(t == 0 || level(t) != level(t - 1)));
+                umma_commit(&bars[Q_KEMPTY + t % 3]);
+                if (t + 1 < T) issue_dp(t + 1);
+                if (t + 2 < T) issue_s(t + 2);
                 if (t == T - 1) umma_commit(&bars[Q_FINAL]);
             }
         }
     } else {
-        const int q4 = warp & 3, h = (warp - 2) >> 2, row = q4 * 32 + lane;
-        const int tid = threadIdx.x - 64;
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        const int q4 = warp & 3, h = (warp - 4) >> 2, row = q4 * 32 + lane;
         const uint32_t tlane = tmem + ((uint32_t)(q4 * 32) << 16);
         const size_t qi = (size_t)s * p.Lp + I * kTile + row;
         const float sl2 = p.scale * kLog2e;
-        const float lse2 = p.lse2[qi], delta = p.delta[qi];
-        float gi2 = 0.f, dsum = 0.f;
-        if (GATE) gi2 = p.G[qi] * kLog2e;
+        const float ndelta = p.delta[qi];            // minus delta
+        const float nl = p.lse2[qi];                 // minus lse2, plus the gate prefix of the row when gated
+        float dsum = 0.f;
         bool ok = true;
-        uint32_t rs[32], rp[32];
         constexpr int CW = HD / 2;
         auto flush_dq = [&](int lvl) {
-            float* dst = p.dqv + ((size_t)ver_row(qslot(lvl, I), I) + row) * HD + h * CW;
+            float* dst = p.dqv + ((size_t)ver_row(qslot(lvl, I), I) + q4 * 32) * HD + h * CW;   // the warp's 32 rows
+#pragma unroll 1
             for (int c = 0; c < CW / 32; ++c) {
-                tmem_ld32(tlane + colDQ + h * CW + c * 32, rs);
+                uint32_t r[32];
+                tmem_ld32(tlane + colDQ + h * CW + c * 32, r);
                 tmem_ld_wait();
 #pragma unroll
-                for (int x = 0; x < 8; ++x)
-                    reinterpret_cast<float4*>(dst + c * 32)[x] =
-                        make_float4(__uint_as_float(rs[4 * x]) * p.scale, __uint_as_float(rs[4 * x + 1]) * p.scale,
-                                    __uint_as_float(rs[4 * x + 2]) * p.scale, __uint_as_float(rs[4 * x + 3]) * p.scale);
+                for (int x = 0; x < 32; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * p.scale);
+                warp_store_rows128(dst + c * 32, (size_t)HD * 4, r);
             }
         };
+        const uint64_t sl2x2 = pack2(sl2, sl2), nl2 = pack2(nl, nl), nd2 = pack2(ndelta, ndelta);
+        const uint64_t nlog2 = pack2(-kLog2e, -kLog2e);
         for (int t = 0; t < T; ++t) {
-            const int J = I - 1 - t, b = t & 1;
-            if (GATE) {
-                if (tid < kTile) gk[b * kTile + tid] = p.G[(size_t)s * p.Lp + J * kTile + tid] * kLog2e;
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-            }
-            if (ok && !mbar_wait(&bars[Q_SFULL], t & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
+            const int c0 = h * 64;               // key columns of this thread
+            uint32_t pr[2][32];                  // S, then P (float bits)
+            // ---- part A: P = exp2(S * scale - lse)
+            if (GATE && ok && !mbar_wait(&bars[Q_GKFULL + (t & 1)], (t >> 1) & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
+            if (ok && !mbar_wait(&bars[Q_SFULL + (t & 1)], (t >> 1) & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after_sync();
             if (ok) {
-                if (t >= 1 && level(t) != level(t - 1)) flush_dq(level(t - 1));
-                uint32_t pk[32];
+                tmem_ld32(tlane + colS + (t & 1) * 128 + c0, pr[0]);
+                tmem_ld32(tlane + colS + (t & 1) * 128 + c0 + 32, pr[1]);
+                tmem_ld_wait();
+                const float* g_ = gk + (t & 1) * kTile + c0;
+#pragma unroll
+                for (int c = 0; c < 2; ++c)
+#pragma unroll
+                    for (int x = 0; x < 32; x += 4) {
+                        uint64_t v01 = fma2(pack2(__uint_as_float(pr[c][x]), __uint_as_float(pr[c][x + 1])), sl2x2, nl2);
+                        uint64_t v23 = fma2(pack2(__uint_as_float(pr[c][x + 2]), __uint_as_float(pr[c][x + 3])), sl2x2, nl2);
+                        if (GATE) {
+                            const float4 g4 = *reinterpret_cast<const float4*>(g_ + c * 32 + x);
+                            v01 = fma2(pack2(g4.x, g4.y), nlog2, v01);
+                            v23 = fma2(pack2(g4.z, g4.w), nlog2, v23);
+                        }
+                        float e[4];
+                        unpack2(v01, e[0], e[1]);
+                        unpack2(v23, e[2], e[3]);
+#pragma unroll
+                        for (int y = 0; y < 4; ++y) pr[c][x + y] = __float_as_uint(ex2(e[y]));
+                    }
+            }
+            // ---- part B: dS = P o (dP - delta)
+            if (ok && !mbar_wait(&bars[Q_DPFULL], t & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            tc_fence_after_sync();
+            // dP ready means every product issued before it has retired: dQ of a finished level is complete.  It is
+            // taken into registers now and written out after dS has been delivered, off the tensor pipe's path.
+            const bool fl = ok && t >= 1 && level(t) != level(t - 1);
+            uint32_t fr[CW / 32][32];
+            if (fl) {
+#pragma unroll
+                for (int c = 0; c < CW / 32; ++c) tmem_ld32(tlane + colDQ + h * CW + c * 32, fr[c]);
+            }
+            if (ok) {
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
-                    const int c0 = h * 64 + c * 32;   // key columns of this pass
-                    tmem_ld32(tlane + colS + c0, rs);
-                    tmem_ld32(tlane + colDP + c0, rp);
+                    uint32_t dp[32], pk[16];
+                    tmem_ld32(tlane + colDP + c0 + c * 32, dp);
                     tmem_ld_wait();
 #pragma unroll
                     for (int x = 0; x < 32; x += 2) {
-                        float v0 = __uint_as_float(rs[x]) * sl2 - lse2, v1 = __uint_as_float(rs[x + 1]) * sl2 - lse2;
-                        if (GATE) {
-                            v0 += gi2 - gk[b * kTile + c0 + x];
-                            v1 += gi2 - gk[b * kTile + c0 + x + 1];
-                        }
-                        const float d0 = ex2(v0) * (__uint_as_float(rp[x]) - delta);
-                        const float d1 = ex2(v1) * (__uint_as_float(rp[x + 1]) - delta);
+                        const uint64_t d01 = mul2(pack2(__uint_as_float(pr[c][x]), __uint_as_float(pr[c][x + 1])),
+                                                  add2(pack2(__uint_as_float(dp[x]), __uint_as_float(dp[x + 1])), nd2));
+                        float d0, d1;
+                        unpack2(d01, d0, d1);
                         if (GATE) dsum += d0 + d1;
-                        pk[c * 16 + (x >> 1)] = pack_bf16(d0, d1);
+                        pk[x >> 1] = pack_bf16(d0, d1);
                     }
+                    tmem_st16(tlane + colDP + c0 + c * 16, pk);
                 }
-                tmem_st32(tlane + colDP + h * 64, pk);
                 tmem_st_wait();
             }
             tc_fence_before_sync();
             mbar_arrive(&bars[Q_DSFULL]);
+            if (GATE) mbar_arrive(&bars[Q_GKEMPTY + (t & 1)]);
+            if (fl) {
+                float* dst = p.dqv + ((size_t)ver_row(qslot(level(t - 1), I), I) + q4 * 32) * HD + h * CW;
+#pragma unroll
+                for (int c = 0; c < CW / 32; ++c) {
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) fr[c][x] = __float_as_uint(__uint_as_float(fr[c][x]) * p.scale);
+                    warp_store_rows128(dst + c * 32, (size_t)HD * 4, fr[c]);
+                }
+            }
         }
         if (ok && !mbar_wait(&bars[Q_FINAL], 0, abort_flag, ST_DQ_COMPUTE)) ok = false;
         ok = __all_sync(0xffffffffu, ok);
@@ -476,11 +690,13 @@ __global__ void __launch_bounds__(320, 1) dq_kernel(const __grid_constant__ BwdT
     }
 }
 
-// delta_i = dO_i . O_i and lse2_i = lse_i * log2(e), padded to Lp (tail rows: 0).  One warp per row.
+// Per-row constants of the backward sweeps, stored negated so that they enter as addends:
+//   delta[i] = -(dO_i . O_i),   lse2[i] = (G_i - lse_i) * log2(e)   (G: gate prefix, absent = 0),
+// padded to Lp (tail rows: 0).  One warp per row.
 template <int HD>
 __global__ void rowstats_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
-                                const float* __restrict__ lse, float* __restrict__ delta, float* __restrict__ lse2,
-                                int L, int Lp) {
+                                const float* __restrict__ lse, const float* __restrict__ G, float* __restrict__ delta,
+                                float* __restrict__ lse2, int L, int Lp) {
     const int s = blockIdx.y;
     const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
@@ -497,8 +713,10 @@ __global__ void rowstats_kernel(const __nv_bfloat16* __restrict__ o, const __nv_
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     if (lane == 0) {
-        delta[(size_t)s * Lp + i] = acc;
-        lse2[(size_t)s * Lp + i] = (i < L) ? lse[(size_t)s * L + i] * kLog2e : 0.f;
+        delta[(size_t)s * Lp + i] = -acc;
+        float v = 0.f;
+        if (i < L) v = ((G ? G[(size_t)s * Lp + i] : 0.f) - lse[(size_t)s * L + i]) * kLog2e;
+        lse2[(size_t)s * Lp + i] = v;
     }
 }
 
@@ -507,19 +725,19 @@ cudaError_t set_smem(K kern, int bytes) {
     return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
-constexpr int kDkvSmem = 6 * kSlotBytes + 256 + (2 * 3 + 1) * kTile * 4 + 1024;
-constexpr int kDqSmem = 6 * kSlotBytes + 256 + 3 * kTile * 4 + 1024;
+constexpr int kDkvSmem = kSmemAlloc;
+constexpr int kDqSmem = kSmemAlloc;
 
 template <int HD, bool GATE>
 cudaError_t launch_one(const BwdTensorMaps& tm, const BwdParams& p, int which, cudaStream_t st) {
     if (which == 0) {
         cudaError_t e = set_smem(dkv_kernel<HD, GATE>, kDkvSmem);
         if (e != cudaSuccess) return e;
-        dkv_kernel<HD, GATE><<<dim3(p.N, p.S), 320, kDkvSmem, st>>>(tm, p);
+        dkv_kernel<HD, GATE><<<dim3(p.N, p.S), 384, kDkvSmem, st>>>(tm, p);
     } else {
         cudaError_t e = set_smem(dq_kernel<HD, GATE>, kDqSmem);
         if (e != cudaSuccess) return e;
-        dq_kernel<HD, GATE><<<dim3(p.N, p.S), 320, kDqSmem, st>>>(tm, p);
+        dq_kernel<HD, GATE><<<dim3(p.N, p.S), 384, kDqSmem, st>>>(tm, p);
     }
     return cudaGetLastError();
 }
@@ -532,13 +750,13 @@ cudaError_t launch_fa_bwd(const BwdTensorMaps& tm, const BwdParams& p, int hd, i
     return p.G ? launch_one<128, true>(tm, p, which, st) : launch_one<128, false>(tm, p, which, st);
 }
 
-cudaError_t launch_rowstats(const void* o, const void* d_o, const float* lse, float* delta, float* lse2, int S, int L,
-                            int Lp, int hd, cudaStream_t st) {
+cudaError_t launch_rowstats(const void* o, const void* d_o, const float* lse, const float* G, float* delta, float* lse2,
+                            int S, int L, int Lp, int hd, cudaStream_t st) {
     dim3 grid((Lp + 7) / 8, S);
     if (hd == 64)
-        rowstats_kernel<64><<<grid, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, delta, lse2, L, Lp);
+        rowstats_kernel<64><<<grid, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, G, delta, lse2, L, Lp);
     else
-        rowstats_kernel<128><<<grid, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, delta, lse2, L, Lp);
+        rowstats_kernel<128><<<grid, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, G, delta, lse2, L, Lp);
     return cudaGetLastError();
 }
 

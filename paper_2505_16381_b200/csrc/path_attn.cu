@@ -312,7 +312,8 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     float* dQv = at<float>(ws, p.dQv); float* dKv = at<float>(ws, p.dKv);
 
     prof_mark(STG_ROWSTATS, 0, st);
-    LAUNCH(launch_rowstats(o, d_o, lse, at<float>(ws, p.delta), at<float>(ws, p.lse2), p.S, p.L, p.Lp, d, st));
+    LAUNCH(launch_rowstats(o, d_o, lse, p.gate ? at<float>(ws, p.G) : nullptr, at<float>(ws, p.delta), at<float>(ws, p.lse2),
+                           p.S, p.L, p.Lp, d, st));
     const void* dop = d_o;
     if (p.ragged) {
         LAUNCH(launch_pad_rows(d_o, at<void>(ws, p.dop), p.S, p.L, p.Lp, d, 0, st));

@@ -43,11 +43,11 @@ constexpr long long kWaitTicks = 2000000000LL;
 
 // Waits for the phase with the given parity.  Returns false (and raises *abort_flag with
 // `code`) if the limit ran out or another thread of the CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t code) {
-    if (mbar_try_wait(bar, parity)) return true;
+__device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code) {
     long long t0 = clock64();
+#pragma unroll 1
     for (;;) {
+#pragma unroll 1      // rolled on purpose: there are dozens of wait sites and the kernels must fit the instruction cache
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag != 0) return false;
@@ -56,6 +56,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
             return false;
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, code);
 }
 
 // ---------------------------------------------------------------- TMA
@@ -185,6 +190,62 @@ __device__ __forceinline__ uint32_t sw128_off(uint32_t row, uint32_t chunk) {
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ---------------------------------------------------------------- coalesced row exchange with global memory
+// A warp owns 32 rows (lane L <-> row L) of 128 bytes each; `w` holds the lane's row as 32 words.  Written or read
+// naively, one instruction touches 32 different lines.  Here the four lanes of a group (L = 4g + j) first swap 32-byte
+// pieces, so that every instruction covers 8 rows with one full 128-byte line each: in round r lane L handles piece j
+// of row 4g + (j ^ r).
+__device__ __forceinline__ void rot4_pieces(uint32_t (&w)[32], int j) {   // piece i <- piece i ^ j (an involution)
+    const bool b0 = j & 1, b1 = j & 2;
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+        const uint32_t p0 = w[x], p1 = w[8 + x], p2 = w[16 + x], p3 = w[24 + x];
+        const uint32_t a0 = b0 ? p1 : p0, a1 = b0 ? p0 : p1, a2 = b0 ? p3 : p2, a3 = b0 ? p2 : p3;
+        w[x] = b1 ? a2 : a0;
+        w[8 + x] = b1 ? a3 : a1;
+        w[16 + x] = b1 ? a0 : a2;
+        w[24 + x] = b1 ? a1 : a3;
+    }
+}
+// `base`: address of row 0's 128-byte segment (warp-uniform, 32-byte aligned), `stride`: bytes between rows
+// (multiple of 32).  Rows >= nrows are not written.  Destroys w.
+__device__ __forceinline__ void warp_store_rows128(void* base, size_t stride, uint32_t (&w)[32], int nrows = 32) {
+    const int lane = threadIdx.x & 31, j = lane & 3, g4 = lane & ~3;
+    rot4_pieces(w, j);
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        uint32_t v[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) v[x] = r == 0 ? w[x] : __shfl_xor_sync(0xffffffffu, w[8 * r + x], r);
+        const int row = g4 + (j ^ r);
+        if (row < nrows) {
+            uint8_t* dst = (uint8_t*)base + (size_t)row * stride + 32 * j;
+            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(v[0]), "r"(v[1]),
+                         "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                         : "memory");
+        }
+    }
+}
+// Counterpart of the store: rows >= nrows read as zero.
+__device__ __forceinline__ void warp_load_rows128(const void* base, size_t stride, uint32_t (&w)[32], int nrows = 32) {
+    const int lane = threadIdx.x & 31, j = lane & 3, g4 = lane & ~3;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        uint32_t v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+        const int row = g4 + (j ^ r);
+        if (row < nrows) {
+            const uint8_t* src = (const uint8_t*)base + (size_t)row * stride + 32 * j;
+            asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                         : "l"(src)
+                         : "memory");
+        }
+#pragma unroll
+        for (int x = 0; x < 8; ++x) w[8 * r + x] = r == 0 ? v[x] : __shfl_xor_sync(0xffffffffu, v[x], r);
+    }
+    rot4_pieces(w, j);
 }
 
 }  // namespace tc5
