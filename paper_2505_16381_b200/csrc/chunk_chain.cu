@@ -20,6 +20,13 @@ using namespace tile;
 
 namespace {
 
+// The kernel below is ~30 products of straight-line code that runs once per CTA; with every product inlined it
+// no longer fits the instruction cache, so the products go through one real function.
+__device__ __noinline__ void mma_call(uint32_t d_tmem, uint32_t a_tile, int a_op, uint32_t b_tile, int b_op, int ksteps, int n,
+                                      bool acc, bool negate = false) {
+    tile::mma(d_tmem, a_tile, a_op, b_tile, b_op, ksteps, n, acc, negate);
+}
+
 constexpr int kSlots = 7;
 constexpr uint32_t kBarOff = kSlots * kTileB;
 constexpr uint32_t kChainSmem = kBarOff + 64 + kT * 4 + kT * 4 + 1024;
@@ -86,14 +93,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         const int per = ncols / 2;
         for (int c = 0; c < per / 32; ++c) {
             const int c0 = half * per + c * 32;
-            if (row < nrows) {
-                gload_f32x32(src + (size_t)row * ncols + c0, v);
+            gload_f32x32(src + (size_t)row * ncols + c0, v, row < nrows);
 #pragma unroll
-                for (int x = 0; x < 32; ++x) v[x] *= mul;
-            } else {
-#pragma unroll
-                for (int x = 0; x < 32; ++x) v[x] = 0.f;
-            }
+            for (int x = 0; x < 32; ++x) v[x] *= mul;
             tile_store32(dst, row, c0, v);
         }
     };
@@ -152,11 +154,11 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma(tmem + cA, sa(1), OP_K, sa(0), OP_K, KD, 128, false);
-        mma(tmem + cA, sa(3), OP_K, sa(2), OP_K, K8, 128, true);
+        mma_call(tmem + cA, sa(1), OP_K, sa(0), OP_K, KD, 128, false);
+        mma_call(tmem + cA, sa(3), OP_K, sa(2), OP_K, K8, 128, true);
         // phase 0b: dw = -Y dKr - U dP^T
-        mma(tmem + cDW, sa(2), OP_K, sa(5), OP_MN, K8, HD, false, true);
-        mma(tmem + cDW, sa(0), OP_K, sa(6), OP_K, KD, HD, true, true);
+        mma_call(tmem + cDW, sa(2), OP_K, sa(5), OP_MN, K8, HD, false, true);
+        mma_call(tmem + cDW, sa(0), OP_K, sa(6), OP_K, KD, HD, true, true);
         umma_commit(&bars[1]);
     }
     mma_wait();
@@ -172,11 +174,11 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma(tmem + cA, sa(0), OP_K, sa(5), OP_K, KD, 128, false);
-        mma(tmem + cA, sa(2), OP_MN, sa(3), OP_MN, K8, 128, true);
-        mma(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, HD, false);
-        mma(tmem + cB, sa(0), OP_K, sa(6), OP_MN, KD, HD, true);
-        mma(tmem + cG, sa(0), OP_K, sa(0), OP_K, KD, 128, false);
+        mma_call(tmem + cA, sa(0), OP_K, sa(5), OP_K, KD, 128, false);
+        mma_call(tmem + cA, sa(2), OP_MN, sa(3), OP_MN, K8, 128, true);
+        mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, HD, false);
+        mma_call(tmem + cB, sa(0), OP_K, sa(6), OP_MN, KD, HD, true);
+        mma_call(tmem + cG, sa(0), OP_K, sa(0), OP_K, KD, 128, false);
         umma_commit(&bars[1]);
     }
     mma_wait();
@@ -192,8 +194,8 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma(tmem + cA, sa(5), OP_K, sa(2), OP_K, K8, 128, false);
-        mma(tmem + cA, sa(6), OP_K, sa(0), OP_K, KD, 128, true);
+        mma_call(tmem + cA, sa(5), OP_K, sa(2), OP_K, K8, 128, false);
+        mma_call(tmem + cA, sa(6), OP_K, sa(0), OP_K, KD, 128, true);
         umma_commit(&bars[1]);
     }
     mma_wait();
@@ -210,8 +212,8 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         publish();
         if (tid == 0) {
             tc_fence_after_sync();
-            mma(tmem + cB, sa(2), OP_MN, sa(5), OP_MN, K8, 128, part > 0);
-            mma(tmem + cDW, sa(2), OP_MN, sa(6), OP_MN, K8, HD, true);
+            mma_call(tmem + cB, sa(2), OP_MN, sa(5), OP_MN, K8, 128, part > 0);
+            mma_call(tmem + cDW, sa(2), OP_MN, sa(6), OP_MN, K8, HD, true);
             umma_commit(&bars[1]);
         }
         mma_wait();
@@ -228,8 +230,8 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, 128, false);
-        mma(tmem + cB, sa(6), OP_MN, sa(1), OP_MN, K8, 128, true);
+        mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, 128, false);
+        mma_call(tmem + cB, sa(6), OP_MN, sa(1), OP_MN, K8, 128, true);
         umma_commit(&bars[1]);
     }
     mma_wait();
@@ -238,7 +240,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, 128, true);
+        mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, 128, true);
         umma_commit(&bars[1]);
     }
     mma_wait();
@@ -256,8 +258,8 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma(tmem + cA, sa(1), OP_K, sa(2), OP_K, K8, 128, false);
-        mma(tmem + cA, sa(1), OP_K, sa(6), OP_K, K8, 128, true);
+        mma_call(tmem + cA, sa(1), OP_K, sa(2), OP_K, K8, 128, false);
+        mma_call(tmem + cA, sa(1), OP_K, sa(6), OP_K, K8, 128, true);
         umma_commit(&bars[1]);
     }
     mma_wait();
@@ -266,7 +268,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma(tmem + cA, sa(1), OP_K, sa(2), OP_K, K8, 128, true);
+        mma_call(tmem + cA, sa(1), OP_K, sa(2), OP_K, K8, 128, true);
         umma_commit(&bars[1]);
     }
     mma_wait();
@@ -299,14 +301,14 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma(tmem + cB, sa(3), OP_K, sa(2), OP_MN, K8, HD, false);    // s dSd K
-        mma(tmem + cB, sa(4), OP_K, sa(0), OP_MN, K8, HD, true);     // dXq W
-        mma(tmem + cG, sa(3), OP_MN, sa(6), OP_MN, K8, HD, false);   // s dSd^T Q
-        mma(tmem + cG, sa(5), OP_MN, sa(0), OP_MN, K8, HD, true);    // dXk^T W
-        mma(tmem + cDW, sa(4), OP_MN, sa(6), OP_MN, K8, HD, true);   // dXq^T Q
-        mma(tmem + cDW, sa(5), OP_K, sa(2), OP_MN, K8, HD, true);    // dXk K
-        mma(tmem + cDW, sa(1), OP_K, sa(0), OP_MN, K8, HD, true);    // dGm W
-        mma(tmem + cDW, sa(1), OP_MN, sa(0), OP_MN, K8, HD, true);   // dGm^T W
+        mma_call(tmem + cB, sa(3), OP_K, sa(2), OP_MN, K8, HD, false);    // s dSd K
+        mma_call(tmem + cB, sa(4), OP_K, sa(0), OP_MN, K8, HD, true);     // dXq W
+        mma_call(tmem + cG, sa(3), OP_MN, sa(6), OP_MN, K8, HD, false);   // s dSd^T Q
+        mma_call(tmem + cG, sa(5), OP_MN, sa(0), OP_MN, K8, HD, true);    // dXk^T W
+        mma_call(tmem + cDW, sa(4), OP_MN, sa(6), OP_MN, K8, HD, true);   // dXq^T Q
+        mma_call(tmem + cDW, sa(5), OP_K, sa(2), OP_MN, K8, HD, true);    // dXk K
+        mma_call(tmem + cDW, sa(1), OP_K, sa(0), OP_MN, K8, HD, true);    // dGm W
+        mma_call(tmem + cDW, sa(1), OP_MN, sa(0), OP_MN, K8, HD, true);   // dGm^T W
         umma_commit(&bars[1]);
     }
     mma_wait();
@@ -315,8 +317,8 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma(tmem + cDW, sa(1), OP_K, sa(0), OP_MN, K8, HD, true);
-        mma(tmem + cDW, sa(1), OP_MN, sa(0), OP_MN, K8, HD, true);
+        mma_call(tmem + cDW, sa(1), OP_K, sa(0), OP_MN, K8, HD, true);
+        mma_call(tmem + cDW, sa(1), OP_MN, sa(0), OP_MN, K8, HD, true);
         umma_commit(&bars[1]);
     }
     mma_wait();
@@ -328,14 +330,14 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         gload_f32x32(g_dql + (size_t)row * HD + c0, in);
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] += in[x];
-        if (row_valid) gstore_bf16x32(p.dq + urow * HD + c0, v);
+        gstore_bf16x32(p.dq + urow * HD + c0, v, row_valid);
         tmem_row32(tl + cG + c0, v);
         gload_f32x32(g_dkr + (size_t)row * HD + c0, in);
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] += in[x];
-        if (row_valid) gstore_bf16x32(p.dk + urow * HD + c0, v);
+        gstore_bf16x32(p.dk + urow * HD + c0, v, row_valid);
         tmem_row32(tl + cDW + c0, v);
-        if (row_valid) gstore_bf16x32(p.dw + urow * HD + c0, v);
+        gstore_bf16x32(p.dw + urow * HD + c0, v, row_valid);
     }
 
 done:

@@ -350,16 +350,14 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
         gstore_bf16x32(p.kr + grow * HD + c0, v);
         tmem_ld32(tl + 0 + c0, r);
         tmem_ld_wait();
-        if (row < HD) {
 #pragma unroll
-            for (int x = 0; x < 32; ++x) {
-                v[x] = ((c0 + x == row) ? 1.f : 0.f) - __uint_as_float(r[x]);
-                in[x] = __bfloat162float(__float2bfloat16_rn(v[x]));
-                v[x] -= in[x];
-            }
-            gstore_bf16x32(p.Ph + ((size_t)chunk * HD + row) * HD + c0, in);
-            gstore_bf16x32(p.Pl + ((size_t)chunk * HD + row) * HD + c0, v);
+        for (int x = 0; x < 32; ++x) {
+            v[x] = ((c0 + x == row) ? 1.f : 0.f) - __uint_as_float(r[x]);
+            in[x] = __bfloat162float(__float2bfloat16_rn(v[x]));
+            v[x] -= in[x];
         }
+        gstore_bf16x32(p.Ph + ((size_t)chunk * HD + row) * HD + c0, in, row < HD);
+        gstore_bf16x32(p.Pl + ((size_t)chunk * HD + row) * HD + c0, v, row < HD);
     }
 
 done:

@@ -81,11 +81,7 @@ __device__ __forceinline__ void conv(const Ctx& c, const float* src, int ncols, 
     float v[32];
     for (int i = 0; i < per / 32; ++i) {
         const int c0 = c.half * per + i * 32;
-        if (c.row < nrows) gload_f32x32(src + (size_t)c.row * ncols + c0, v);
-        else {
-#pragma unroll
-            for (int x = 0; x < 32; ++x) v[x] = 0.f;
-        }
+        gload_f32x32(src + (size_t)c.row * ncols + c0, v, c.row < nrows);
         tile_store32(dst, c.row, c0, v);
     }
 }
@@ -97,17 +93,19 @@ __device__ __forceinline__ void acc_add_global(const Ctx& c, uint32_t col, int n
     for (int i = 0; i < per / 32; ++i) {
         const int c0 = c.half * per + i * 32;
         tmem_row32(c.tl + col + c0, v);
-        if (c.row >= nrows) continue;
+        const bool live = c.row < nrows;
         float* d = dst + (size_t)c.row * ncols + c0;
         if (ATOMIC) {
+            if (live) {
 #pragma unroll
-            for (int x = 0; x < 32; ++x) atomicAdd(d + x, v[x]);
+                for (int x = 0; x < 32; ++x) atomicAdd(d + x, v[x]);
+            }
         } else {
             float o[32];
-            gload_f32x32(d, o);
+            gload_f32x32(d, o, live);
 #pragma unroll
             for (int x = 0; x < 32; ++x) o[x] += v[x];
-            gstore_f32x32(d, o);
+            gstore_f32x32(d, o, live);
         }
     }
 }
@@ -168,16 +166,14 @@ __global__ void __launch_bounds__(256, 1) dyadic_fwd_kernel(const __grid_constan
         for (int i = 0; i < HD / 64; ++i) {
             const int c0 = c.half * (HD / 2) + i * 32;
             tmem_row32(c.tl + c0, v);
-            if (c.row < HD) {
 #pragma unroll
-                for (int x = 0; x < 32; ++x) {
-                    hi[x] = __bfloat162float(__float2bfloat16_rn(v[x]));
-                    v[x] -= hi[x];
-                }
-                const size_t o = ((size_t)mat_out * HD + c.row) * HD + c0;
-                gstore_bf16x32(p.dyh + o, hi);
-                gstore_bf16x32(p.dyl + o, v);
+            for (int x = 0; x < 32; ++x) {
+                hi[x] = __bfloat162float(__float2bfloat16_rn(v[x]));
+                v[x] -= hi[x];
             }
+            const size_t o = ((size_t)mat_out * HD + c.row) * HD + c0;
+            gstore_bf16x32(p.dyh + o, hi, c.row < HD);
+            gstore_bf16x32(p.dyl + o, v, c.row < HD);
         }
     }
     teardown<128>(c, p.status);

@@ -39,24 +39,72 @@ __device__ __forceinline__ void tile_store32(uint8_t* t, int row, int c0, const 
             make_uint4(pack_bf16(v[8 * ch], v[8 * ch + 1]), pack_bf16(v[8 * ch + 2], v[8 * ch + 3]),
                        pack_bf16(v[8 * ch + 4], v[8 * ch + 5]), pack_bf16(v[8 * ch + 6], v[8 * ch + 7]));
 }
-__device__ __forceinline__ void gstore_f32x32(float* dst, const float (&v)[32]) {
-#pragma unroll
-    for (int x = 0; x < 8; ++x)
-        reinterpret_cast<float4*>(dst)[x] = make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
+// Row transfers between registers and global memory.  Lane L of a warp owns one row segment (32 consecutive values
+// starting at its own pointer).  All 32 lanes must call together: the lanes of a group first swap 32-byte pieces so
+// that one instruction covers whole rows (full 128- or 64-byte runs) instead of 32 scattered 16-byte pieces.
+// `valid` = false: the lane's row is not written / reads as zero.
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&v)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]),
+                 "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
 }
-__device__ __forceinline__ void gload_f32x32(const float* src, float (&v)[32]) {
+__device__ __forceinline__ void ld_global_v8(const void* p, uint32_t (&v)[8]) {
+    asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "l"(p)
+                 : "memory");
+}
+__device__ __forceinline__ void gstore_f32x32(float* dst, const float (&v)[32], bool valid = true) {
+    const int j = threadIdx.x & 3;
+    uint32_t w[32];
 #pragma unroll
-    for (int x = 0; x < 8; ++x) {
-        const float4 f = reinterpret_cast<const float4*>(src)[x];
-        v[4 * x] = f.x; v[4 * x + 1] = f.y; v[4 * x + 2] = f.z; v[4 * x + 3] = f.w;
+    for (int x = 0; x < 32; ++x) w[x] = __float_as_uint(v[x]);
+    rot4_pieces(w, j);
+    const unsigned long long mine = (unsigned long long)dst;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {   // piece j of the row of lane (L ^ r)
+        uint32_t d[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) d[x] = r == 0 ? w[x] : __shfl_xor_sync(0xffffffffu, w[8 * r + x], r);
+        const unsigned long long ptr = r == 0 ? mine : __shfl_xor_sync(0xffffffffu, mine, r);
+        const bool ok = r == 0 ? valid : (bool)__shfl_xor_sync(0xffffffffu, (int)valid, r);
+        if (ok) st_global_v8((uint8_t*)ptr + 32 * j, d);
     }
 }
-__device__ __forceinline__ void gstore_bf16x32(__nv_bfloat16* dst, const float (&v)[32]) {
+__device__ __forceinline__ void gload_f32x32(const float* src, float (&v)[32], bool valid = true) {
+    const int j = threadIdx.x & 3;
+    uint32_t w[32];
+    const unsigned long long mine = (unsigned long long)src;
 #pragma unroll
-    for (int x = 0; x < 4; ++x)
-        reinterpret_cast<uint4*>(dst)[x] =
-            make_uint4(pack_bf16(v[8 * x], v[8 * x + 1]), pack_bf16(v[8 * x + 2], v[8 * x + 3]),
-                       pack_bf16(v[8 * x + 4], v[8 * x + 5]), pack_bf16(v[8 * x + 6], v[8 * x + 7]));
+    for (int r = 0; r < 4; ++r) {
+        uint32_t d[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+        const unsigned long long ptr = r == 0 ? mine : __shfl_xor_sync(0xffffffffu, mine, r);
+        const bool ok = r == 0 ? valid : (bool)__shfl_xor_sync(0xffffffffu, (int)valid, r);
+        if (ok) ld_global_v8((const uint8_t*)ptr + 32 * j, d);
+#pragma unroll
+        for (int x = 0; x < 8; ++x) w[8 * r + x] = r == 0 ? d[x] : __shfl_xor_sync(0xffffffffu, d[x], r);
+    }
+    rot4_pieces(w, j);
+#pragma unroll
+    for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(w[x]);
+}
+// 32 bf16 = 64 bytes per row: pairs of lanes.
+__device__ __forceinline__ void gstore_bf16x32(__nv_bfloat16* dst, const float (&v)[32], bool valid = true) {
+    const bool odd = threadIdx.x & 1;
+    uint32_t w[16];
+#pragma unroll
+    for (int x = 0; x < 16; ++x) w[x] = pack_bf16(v[2 * x], v[2 * x + 1]);
+    uint32_t first[8], second[8];   // halves [32 * odd, +32) of the even lane's row and of the odd lane's row
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+        const uint32_t recv = __shfl_xor_sync(0xffffffffu, odd ? w[x] : w[8 + x], 1);
+        first[x] = odd ? recv : w[x];
+        second[x] = odd ? w[8 + x] : recv;
+    }
+    const unsigned long long mine = (unsigned long long)dst, other = __shfl_xor_sync(0xffffffffu, mine, 1);
+    const bool ovalid = (bool)__shfl_xor_sync(0xffffffffu, (int)valid, 1);
+    if (odd ? ovalid : valid) st_global_v8((uint8_t*)(odd ? other : mine) + 32 * (int)odd, first);
+    if (odd ? valid : ovalid) st_global_v8((uint8_t*)(odd ? mine : other) + 32 * (int)odd, second);
 }
 __device__ __forceinline__ void gload_bf16x32(const __nv_bfloat16* src, float (&v)[32]) {
 #pragma unroll
