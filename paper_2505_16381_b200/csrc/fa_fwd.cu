@@ -22,6 +22,7 @@
 //
 // Warps: 0 = TMA producer, 1 = tcgen05 MMA issuer, 2-3 idle (they give their registers to the softmax
 // warps), 4-7 = softmax of stream 0, 8-11 = softmax of stream 1.
+#include <type_traits>
 #include "common.cuh"
 #include "tc5.cuh"
 
@@ -40,11 +41,6 @@ __device__ __forceinline__ float ex2(float x) {
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-__device__ __forceinline__ float min3(float a, float b, float c) {
-    float d;
-    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
 // Two-wide float arithmetic on register pairs.
@@ -191,7 +187,8 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
             }
         } else if (warp == 1 && lane == 0) {
             // ------------------------------------------------------------ MMA issuer
-            constexpr uint32_t idescS = umma_idesc(128, 128, 0, 0);
+            // a negative scale is applied as a sign flip of the logits here (negate-A bit), its magnitude in the softmax
+            const uint32_t idescS = umma_idesc(128, 128, 0, 0) | (p.scale < 0.f ? (1u << 13) : 0u);
             constexpr uint32_t idescO = umma_idesc(128, HD, 0, 1);
             bool ok = true;
             auto wait = [&](int bar, int parity) {
@@ -302,7 +299,7 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
         const uint32_t tlane = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t colS = x * 128, colO = 256 + x * 128;
         const float kLog2e = 1.4426950408889634f;
-        const float sl2 = p.scale * kLog2e;
+        const float sl2 = fabsf(p.scale) * kLog2e;
         const uint64_t sl2x2 = pack2(sl2, sl2);
         bool ok = true;
         int sc = 0;                             // S tiles consumed so far by this stream (all work items)
@@ -325,7 +322,9 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
             // the stat words are shared with the previous item's merge: every thread must have read them
             if (item > 0 && ok && !mbar_wait(&bars[B_OFREE], (item - 1) & 1, abort_flag, ST_FWD_SOFTMAX)) ok = false;
 
-            for (int t = 0; t < TX; ++t) {
+            auto softmax_step = [&](auto diag_tag, const int t) {
+                constexpr bool DIAG = decltype(diag_tag)::value;   // the diagonal chunk (step 0): causal mask
+                constexpr bool PRE = DIAG || GATE;                 // logits are scaled (and gated, masked) in place first
                 const int n = 2 * t + x, J = I - n;
                 if (GATE) {
                     wg_sync();   // everyone is done with the previous chunk's values
@@ -341,50 +340,34 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
 #pragma unroll
                     for (int c = 0; c < 4; ++c) tmem_ld32(tlane + colS + c * 32, r[c]);
                     tmem_ld_wait();
-                    // row maximum of the scaled logits (log2 units)
-                    float mx;
-                    if (GATE) {
+                    if (PRE) {
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
 #pragma unroll
                             for (int e = 0; e < 32; e += 2) {
-                                const float g0 = gi2 - statx[c * 32 + e].x, g1 = gi2 - statx[c * 32 + e + 1].x;
+                                float g0 = 0.f, g1 = 0.f;
+                                if (GATE) { g0 = gi2 - statx[c * 32 + e].x; g1 = gi2 - statx[c * 32 + e + 1].x; }
                                 const uint64_t v = fma2(pack2(__uint_as_float(r[c][e]), __uint_as_float(r[c][e + 1])), sl2x2,
                                                         pack2(g0, g1));
                                 float a, b;
                                 unpack2(v, a, b);
+                                if (DIAG) {
+                                    if (c * 32 + e > row) a = -INFINITY;
+                                    if (c * 32 + e + 1 > row) b = -INFINITY;
+                                }
                                 r[c][e] = __float_as_uint(a);
                                 r[c][e + 1] = __float_as_uint(b);
                             }
                     }
-                    if (n == 0) {   // causal mask inside the diagonal chunk
+                    // row maximum of the scaled logits (log2 units)
+                    float a4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                        for (int c = 0; c < 4; ++c)
+                    for (int c = 0; c < 4; ++c)
 #pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                if (c * 32 + e > row) r[c][e] = 0xff800000u;
-                    }
-                    if (GATE || sl2 >= 0.f) {
-                        float a[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                        for (int c = 0; c < 4; ++c)
-#pragma unroll
-                            for (int e = 0; e < 32; e += 2)
-                                a[(e >> 1) & 3] = max3(a[(e >> 1) & 3], __uint_as_float(r[c][e]), __uint_as_float(r[c][e + 1]));
-                        mx = fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3]));
-                        if (!GATE) mx *= sl2;
-                    } else {        // negative scale: the largest scaled logit is the smallest raw one
-                        float a[4] = {INFINITY, INFINITY, INFINITY, INFINITY};
-#pragma unroll
-                        for (int c = 0; c < 4; ++c)
-#pragma unroll
-                            for (int e = 0; e < 32; e += 2) {
-                                const float u0 = __uint_as_float(r[c][e]), u1 = __uint_as_float(r[c][e + 1]);
-                                a[(e >> 1) & 3] = min3(a[(e >> 1) & 3], u0 == -INFINITY ? INFINITY : u0,
-                                                       u1 == -INFINITY ? INFINITY : u1);
-                            }
-                        mx = fminf(fminf(a[0], a[1]), fminf(a[2], a[3])) * sl2;
-                    }
+                        for (int e = 0; e < 32; e += 2)
+                            a4[(e >> 1) & 3] = max3(a4[(e >> 1) & 3], __uint_as_float(r[c][e]), __uint_as_float(r[c][e + 1]));
+                    float mx = fmaxf(fmaxf(a4[0], a4[1]), fmaxf(a4[2], a4[3]));
+                    if (!PRE) mx *= sl2;
                     // lazy rescaling: tolerate a stale maximum up to 2^8.  O of this stream is stable here: its S
                     // tile only becomes ready after the stream's previous P V has retired
                     float m_new = m;
@@ -406,9 +389,9 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
                         }
                     }
                     m = m_new;
-                    // probabilities -> packed bf16 over the first 64 columns of the S tile (64 keys per store)
+                    // probabilities -> packed bf16 over the first 64 columns of the S tile
                     const uint64_t nm2 = pack2(-m, -m);
-                    const uint64_t mul2 = GATE ? pack2(1.f, 1.f) : sl2x2;
+                    const uint64_t mul2 = PRE ? pack2(1.f, 1.f) : sl2x2;
                     uint64_t lacc = pack2(0.f, 0.f);
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -418,10 +401,6 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
                             const uint64_t v = fma2(pack2(__uint_as_float(r[c][e]), __uint_as_float(r[c][e + 1])), mul2, nm2);
                             float a, b;
                             unpack2(v, a, b);
-                            if (n == 0 && !GATE && sl2 < 0.f) {   // masked entries are -inf before scaling
-                                if (c * 32 + e > row) a = -INFINITY;
-                                if (c * 32 + e + 1 > row) b = -INFINITY;
-                            }
                             a = ex2(a);
                             b = ex2(b);
                             lacc = add2(lacc, pack2(a, b));
@@ -436,6 +415,15 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
                 }
                 tc_fence_before_sync();
                 mbar_arrive(&bars[B_PFULL + x]);
+            };
+            {
+                int t = 0;
+                if (x == 0 && TX > 0) {
+                    softmax_step(std::true_type{}, 0);
+                    t = 1;
+                }
+#pragma unroll 1
+                for (; t < TX; ++t) softmax_step(std::false_type{}, t);
             }
             // ---- merge the two streams and write O, LSE: warpgroup x handles columns [x*HD/2, (x+1)*HD/2)
             if (GATE) wg_sync();

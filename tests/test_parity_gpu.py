@@ -109,9 +109,11 @@ def test_c1_workload_shape_and_distribution_in_bf16(binding, oracle):
     assert e.value.status == -3
 
 
-def test_explicit_scale(binding, oracle):
+@pytest.mark.parametrize("scale", [1.0 / 8.0, -1.0 / 8.0, 0.0])
+def test_explicit_scale(binding, oracle, scale):
+    """Positive, negative (the sign is applied inside the logit products) and zero scale (uniform causal attention)."""
     inp = synth.make_inputs(1, 2, 640, 64, "bf16", qk_scaled=False, gate=True, seed=5)
-    compare_all(binding, oracle, inp, scale=1.0 / 8.0)
+    compare_all(binding, oracle, inp, scale=scale)
 
 
 @pytest.mark.parametrize("mode", ["beta0", "beta2", "beta1", "w0"])
