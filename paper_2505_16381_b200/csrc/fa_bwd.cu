@@ -102,11 +102,15 @@ __device__ __forceinline__ void tma_tile(uint8_t* dst, const CUtensorMap* m, uin
 }
 
 // ------------------------------------------------------------------------------------------------ dK, dV
-enum { K_KFULL = 0, K_KEMPTY, K_VFULL, K_QFULL, K_QEMPTY = K_QFULL + 3, K_DOFULL = K_QEMPTY + 3,
-       K_DOEMPTY = K_DOFULL + 2, K_SFULL = K_DOEMPTY + 2, K_DPFULL, K_PFULL, K_DSFULL, K_FINAL,
+// Persistent: the work items (one key chunk of one slice each) are listed slice after slice as pairs (longest,
+// shortest), (second longest, second shortest), ...; CTA c takes the pairs c, c + gridDim.x, ...  Every ring and phase
+// counter runs on across items, so the loads and the first products of the next item overlap the write-out of the
+// current one.
+enum { K_KFULL = 0, K_KEMPTY, K_VFULL, K_VEMPTY, K_QFULL, K_QEMPTY = K_QFULL + 3, K_DOFULL = K_QEMPTY + 3,
+       K_DOEMPTY = K_DOFULL + 2, K_SFULL = K_DOEMPTY + 2, K_DPFULL, K_PFULL, K_DSFULL, K_ACCFULL, K_ACCFREE,
        K_STFULL, K_STEMPTY = K_STFULL + 2, K_COUNT = K_STEMPTY + 2 };
 constexpr uint32_t kDkvStat = 7 * kSlotBytes + 256;           // [2][2][128] floats: -lse2 (plus gate), -delta
-constexpr uint32_t kDkvTotal = kDkvStat + 2 * 2 * kTile * 4;
+constexpr uint32_t kDkvTotal = kDkvStat + 2 * 2 * kTile * 4 + kTile * 4;   // + [128] exchange of the gate column sums
 
 template <int HD, bool GATE>
 __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
@@ -118,20 +122,21 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
     }
     uint8_t* sK = smem;
     uint8_t* sV = sK + kSlotBytes;
-    uint8_t* sQ = sV + kSlotBytes;          // 3 slots: rawQ, Xqn, then Q of step t >= 1 as item t + 1
-    uint8_t* sDO = sQ + 3 * kSlotBytes;     // 2 slots: dO(0), Yt, then dO of step t >= 1 as item t + 1
+    uint8_t* sQ = sV + kSlotBytes;          // ring of 3; per item: rawQ, Xqn, then Q of step t >= 1 (entry t + 1)
+    uint8_t* sDO = sQ + 3 * kSlotBytes;     // ring of 2; per item: Yt, then dO of step t (entry t + 1)
     uint64_t* bars = (uint64_t*)(smem + 7 * kSlotBytes);
     uint32_t* tmem_slot = (uint32_t*)(bars + K_COUNT);
     volatile uint32_t* abort_flag = (volatile uint32_t*)(tmem_slot + 1);
     float* rowstat = (float*)(smem + kDkvStat);
+    float* dsum_x = rowstat + 2 * 2 * kTile;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int J = blockIdx.x, s = blockIdx.y;
-    const int T = p.N - J;
+    const int items = p.N * p.S;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < K_COUNT; ++i)
-            mbar_init(&bars[i], (i == K_PFULL || i == K_DSFULL || i == K_STEMPTY || i == K_STEMPTY + 1) ? 256u : 1u);
+            mbar_init(&bars[i], (i == K_PFULL || i == K_DSFULL || i == K_ACCFREE || i == K_STEMPTY || i == K_STEMPTY + 1)
+                                    ? 256u : 1u);
         *abort_flag = 0;
         mbar_fence_init();
     }
@@ -142,7 +147,16 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
     constexpr uint32_t colS = 0, colDP = 128, colDV = 256, colDK = 384;
-    const int rowJ = s * p.Lp + J * kTile;
+    // k-th work item of this CTA
+    auto item_of = [&](int k, int& J, int& s) {
+        const int w = 2 * ((int)blockIdx.x + (k >> 1) * (int)gridDim.x) + (k & 1);
+        if (w >= items) return false;
+        s = w / p.N;
+        const int j = w % p.N;
+        J = (j & 1) ? p.N - 1 - (j >> 1) : (j >> 1);
+        return true;
+    };
+    int J = 0, s = 0;   // current item of this thread's role
     auto ver_row = [&](int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
     auto level = [&](int t) { return t == 0 ? -1 : msb32((unsigned)((J + t) ^ J)); };
 
@@ -150,133 +164,155 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
         asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
         if (warp == 0 && lane == 0) {
             bool ok = true;
-            int nk = 0;
+            int nk = 0, nv = 0, qn = 0, dn = 0, sn = 0;   // fills so far: K, V, Q ring, dO ring, statistics ring
             auto wait_empty = [&](int bar, int use) {
                 if (ok && !mbar_wait(&bars[bar], (use & 1) ^ 1, abort_flag, ST_DKV_PRODUCER)) ok = false;
             };
-            auto load_q = [&](int item, const CUtensorMap* m, int kdim, int row0) {
-                const int slot = item % 3;
-                wait_empty(K_QEMPTY + slot, item / 3);
+            auto load_q = [&](const CUtensorMap* m, int kdim, int row0) {
+                const int slot = qn % 3;
+                wait_empty(K_QEMPTY + slot, qn / 3);
                 if (!ok) return;
                 mbar_expect_tx(&bars[K_QFULL + slot], (uint32_t)(kTile * kdim * 2));
                 tma_tile(sQ + slot * kSlotBytes, m, &bars[K_QFULL + slot], kdim, row0);
+                ++qn;
             };
-            auto load_do = [&](int item, const CUtensorMap* m, int kdim, int row0) {
-                const int slot = item & 1;
-                wait_empty(K_DOEMPTY + slot, item >> 1);
+            auto load_do = [&](const CUtensorMap* m, int kdim, int row0) {
+                const int slot = dn & 1;
+                wait_empty(K_DOEMPTY + slot, dn >> 1);
                 if (!ok) return;
                 mbar_expect_tx(&bars[K_DOFULL + slot], (uint32_t)(kTile * kdim * 2));
                 tma_tile(sDO + slot * kSlotBytes, m, &bars[K_DOFULL + slot], kdim, row0);
+                ++dn;
             };
-            for (int t = 0; t < T && ok; ++t) {
-                const int I = J + t, l = level(t);
-                if (t == 0 || l != level(t - 1)) {
-                    wait_empty(K_KEMPTY, nk);
+#pragma unroll 1
+            for (int it = 0; ok && item_of(it, J, s); ++it) {
+                const int T = p.N - J, rowJ = s * p.Lp + J * kTile;
+#pragma unroll 1
+                for (int t = 0; t < T && ok; ++t) {
+                    const int I = J + t, l = level(t);
+                    if (t == 0 || l != level(t - 1)) {
+                        wait_empty(K_KEMPTY, nk);
+                        if (!ok) break;
+                        mbar_expect_tx(&bars[K_KFULL], kTile * HD * 2);
+                        if (t == 0) tma_tile(sK, &tm.k_raw, &bars[K_KFULL], HD, rowJ);
+                        else tma_tile(sK, &tm.kv, &bars[K_KFULL], HD, ver_row(kslot(l, J), J));
+                        ++nk;
+                    }
+                    if (t == 0) {
+                        load_q(&tm.q_raw, HD, rowJ);
+                        load_q(&tm.xqn, kTile, rowJ);
+                        load_do(&tm.yt, kTile, rowJ);
+                        wait_empty(K_VEMPTY, nv);
+                        if (!ok) break;
+                        mbar_expect_tx(&bars[K_VFULL], kTile * HD * 2);
+                        tma_tile(sV, &tm.v, &bars[K_VFULL], HD, rowJ);
+                        ++nv;
+                        load_do(&tm.d_o, HD, rowJ);
+                    } else {
+                        load_q(&tm.qv, HD, ver_row(qslot(l, I), I));
+                        load_do(&tm.d_o, HD, s * p.Lp + I * kTile);
+                    }
+                    // per-query statistics of the step
+                    wait_empty(K_STEMPTY + (sn & 1), sn >> 1);
                     if (!ok) break;
-                    mbar_expect_tx(&bars[K_KFULL], kTile * HD * 2);
-                    if (t == 0) tma_tile(sK, &tm.k_raw, &bars[K_KFULL], HD, rowJ);
-                    else tma_tile(sK, &tm.kv, &bars[K_KFULL], HD, ver_row(kslot(l, J), J));
-                    ++nk;
+                    mbar_expect_tx(&bars[K_STFULL + (sn & 1)], 2 * kTile * 4);
+                    const size_t gi = (size_t)s * p.Lp + I * kTile;
+                    bulk_load(rowstat + (sn & 1) * 2 * kTile, p.lse2 + gi, kTile * 4, &bars[K_STFULL + (sn & 1)]);
+                    bulk_load(rowstat + (sn & 1) * 2 * kTile + kTile, p.delta + gi, kTile * 4, &bars[K_STFULL + (sn & 1)]);
+                    ++sn;
                 }
-                if (t == 0) {
-                    load_q(0, &tm.q_raw, HD, rowJ);
-                    load_q(1, &tm.xqn, kTile, rowJ);
-                    load_do(1, &tm.yt, kTile, rowJ);
-                    mbar_expect_tx(&bars[K_VFULL], kTile * HD * 2);
-                    tma_tile(sV, &tm.v, &bars[K_VFULL], HD, rowJ);
-                    load_do(0, &tm.d_o, HD, rowJ);
-                } else {
-                    load_q(t + 1, &tm.qv, HD, ver_row(qslot(l, I), I));
-                    load_do(t + 1, &tm.d_o, HD, s * p.Lp + I * kTile);
-                }
-                // per-query statistics of the step
-                wait_empty(K_STEMPTY + (t & 1), t >> 1);
-                if (!ok) break;
-                mbar_expect_tx(&bars[K_STFULL + (t & 1)], 2 * kTile * 4);
-                const size_t gi = (size_t)s * p.Lp + I * kTile;
-                bulk_load(rowstat + (t & 1) * 2 * kTile, p.lse2 + gi, kTile * 4, &bars[K_STFULL + (t & 1)]);
-                bulk_load(rowstat + (t & 1) * 2 * kTile + kTile, p.delta + gi, kTile * 4, &bars[K_STFULL + (t & 1)]);
             }
         } else if (warp == 1 && lane == 0) {
             constexpr uint32_t idescT = umma_idesc(128, 128, 0, 0);
             constexpr uint32_t idescD = umma_idesc(128, HD, 0, 1);
             bool ok = true;
-            int nk = 0;
+            int nk = 0, nv = 0, qb = 0, db = 0, g = 0;   // K / V fills consumed; ring entries and steps before this item
             auto wait = [&](int bar, int parity) {
                 if (ok && !mbar_wait(&bars[bar], parity & 1, abort_flag, ST_DKV_MMA)) ok = false;
             };
-            auto q_addr = [&](int item) { return smem_u32(sQ + (item % 3) * kSlotBytes); };
-            auto do_addr = [&](int item) { return smem_u32(sDO + (item & 1) * kSlotBytes); };
-            // step 0: S^T of the diagonal chunk (two contractions) and its dP^T
-            wait(K_KFULL, nk); ++nk;
-            wait(K_QFULL + 0, 0);
-            wait(K_QFULL + 1, 0);
-            wait(K_DOFULL + 1, 0);
-            tc_fence_after_sync();
-            if (ok) {
-                mma_kk(tmem + colS, smem_u32(sK), q_addr(0), HD, idescT, false);
-                mma_kk(tmem + colS, do_addr(1), q_addr(1), kTile, idescT, true);
+            auto q_wait = [&](int e) { wait(K_QFULL + e % 3, e / 3); };
+            auto do_wait = [&](int e) { wait(K_DOFULL + (e & 1), e >> 1); };
+            auto q_addr = [&](int e) { return smem_u32(sQ + (e % 3) * kSlotBytes); };
+            auto do_addr = [&](int e) { return smem_u32(sDO + (e & 1) * kSlotBytes); };
+#pragma unroll 1
+            for (int it = 0; ok && item_of(it, J, s); ++it) {
+                const int T = p.N - J;
+                // step 0: S^T of the diagonal chunk (two contractions) and its dP^T
+                wait(K_KFULL, nk); ++nk;
+                q_wait(qb);
+                q_wait(qb + 1);
+                do_wait(db);
+                tc_fence_after_sync();
+                if (!ok) break;
+                mma_kk(tmem + colS, smem_u32(sK), q_addr(qb), HD, idescT, false);
+                mma_kk(tmem + colS, do_addr(db), q_addr(qb + 1), kTile, idescT, true);
                 umma_commit(&bars[K_SFULL]);
-                umma_commit(&bars[K_QEMPTY + 0]);   // raw q and the two correction operands are only needed here
-                umma_commit(&bars[K_QEMPTY + 1]);
-                umma_commit(&bars[K_DOEMPTY + 1]);
-                if (T > 1) umma_commit(&bars[K_KEMPTY]);
-            }
-            wait(K_VFULL, 0);
-            wait(K_DOFULL + 0, 0);
-            tc_fence_after_sync();
-            if (ok) {
-                mma_kk(tmem + colDP, smem_u32(sV), do_addr(0), HD, idescT, false);
+                umma_commit(&bars[K_QEMPTY + qb % 3]);         // raw q and the two correction operands are only needed here
+                umma_commit(&bars[K_QEMPTY + (qb + 1) % 3]);
+                umma_commit(&bars[K_DOEMPTY + (db & 1)]);
+                umma_commit(&bars[K_KEMPTY]);                  // raw k as well: step 1 uses a key version
+                wait(K_VFULL, nv); ++nv;
+                do_wait(db + 1);
+                tc_fence_after_sync();
+                if (!ok) break;
+                mma_kk(tmem + colDP, smem_u32(sV), do_addr(db + 1), HD, idescT, false);
                 umma_commit(&bars[K_DPFULL]);
-            }
-            for (int t = 0; t < T && ok; ++t) {
-                const int l = level(t);
-                const int item = (t == 0) ? 0 : t + 1;
-                // dV += P^T dO
-                wait(K_PFULL, t);
-                tc_fence_after_sync();
-                if (!ok) break;
-                mma_tn(tmem + colDV, tmem + colS, do_addr(item), idescD, t > 0);
-                umma_commit(&bars[K_DOEMPTY + (item & 1)]);
-                // S^T of the next step overwrites P^T: in-order execution puts it after the product above
-                if (t + 1 < T) {
-                    const int l1 = level(t + 1);
-                    if (l1 != l) { wait(K_KFULL, nk); ++nk; }
-                    wait(K_QFULL + (t + 2) % 3, (t + 2) / 3);
+                if (T == 1) umma_commit(&bars[K_VEMPTY]);
+#pragma unroll 1
+                for (int t = 0; t < T && ok; ++t) {
+                    const int l = level(t);
+                    const int qe = qb + (t == 0 ? 0 : t + 1), de = db + 1 + t;
+                    // dV += P^T dO; the first product of an item overwrites the accumulators the previous item's
+                    // write-out must have read
+                    wait(K_PFULL, g + t);
+                    if (t == 0 && it > 0) wait(K_ACCFREE, it - 1);
                     tc_fence_after_sync();
                     if (!ok) break;
-                    mma_kk(tmem + colS, smem_u32(sK), q_addr(t + 2), HD, idescT, false);
-                    umma_commit(&bars[K_SFULL]);
-                    if (t + 2 < T && level(t + 2) != l1) umma_commit(&bars[K_KEMPTY]);
-                }
-                // dK += dS^T Q
-                wait(K_DSFULL, t);
-                tc_fence_after_sync();
-                if (!ok) break;
-                if (t > 0) {
-                    mma_tn(tmem + colDK, tmem + colDP, q_addr(item), idescD, !(t == 1 || l != level(t - 1)));
-                    umma_commit(&bars[K_QEMPTY + item % 3]);
-                }
-                if (t + 1 < T) {
-                    wait(K_DOFULL + ((t + 2) & 1), (t + 2) >> 1);
+                    mma_tn(tmem + colDV, tmem + colS, do_addr(de), idescD, t > 0);
+                    umma_commit(&bars[K_DOEMPTY + (de & 1)]);
+                    // S^T of the next step overwrites P^T: in-order execution puts it after the product above
+                    if (t + 1 < T) {
+                        const int l1 = level(t + 1);
+                        if (l1 != l) { wait(K_KFULL, nk); ++nk; }
+                        q_wait(qb + t + 2);
+                        tc_fence_after_sync();
+                        if (!ok) break;
+                        mma_kk(tmem + colS, smem_u32(sK), q_addr(qb + t + 2), HD, idescT, false);
+                        umma_commit(&bars[K_SFULL]);
+                        if (t + 2 >= T || level(t + 2) != l1) umma_commit(&bars[K_KEMPTY]);
+                    }
+                    // dK += dS^T Q
+                    wait(K_DSFULL, g + t);
                     tc_fence_after_sync();
                     if (!ok) break;
-                    mma_kk(tmem + colDP, smem_u32(sV), do_addr(t + 2), HD, idescT, false);
-                    umma_commit(&bars[K_DPFULL]);
-                } else {
-                    umma_commit(&bars[K_FINAL]);
+                    if (t > 0) {
+                        mma_tn(tmem + colDK, tmem + colDP, q_addr(qe), idescD, !(t == 1 || l != level(t - 1)));
+                        umma_commit(&bars[K_QEMPTY + qe % 3]);
+                    }
+                    if (t + 1 < T) {
+                        do_wait(de + 1);
+                        tc_fence_after_sync();
+                        if (!ok) break;
+                        mma_kk(tmem + colDP, smem_u32(sV), do_addr(de + 1), HD, idescT, false);
+                        umma_commit(&bars[K_DPFULL]);
+                        if (t + 2 == T) umma_commit(&bars[K_VEMPTY]);   // that was the item's last use of V
+                    } else {
+                        umma_commit(&bars[K_ACCFULL]);
+                    }
                 }
+                g += T; qb += T + 1; db += T + 1;
             }
         }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
         const int q4 = warp & 3, h = (warp - 4) >> 2, row = q4 * 32 + lane;
         const uint32_t tlane = tmem + ((uint32_t)(q4 * 32) << 16);
-        const int kj = J * kTile + row;          // key position of this thread's row
         const float sl2 = p.scale * kLog2e;
-        float gj2 = 0.f, dsum = 0.f;
-        if (GATE) gj2 = p.G[(size_t)s * p.Lp + kj] * kLog2e;
+        const uint64_t sl2x2 = pack2(sl2, sl2);
+        uint64_t ngj2 = 0;
+        float dsum = 0.f;
         bool ok = true;
+        int g = 0;                               // steps before the current item
         constexpr int CW = HD / 2;               // accumulator columns per thread when flushing
         auto flush_dk = [&](int lvl) {
             float* dst = p.dkv + ((size_t)ver_row(kslot(lvl, J), J) + q4 * 32) * HD + h * CW;   // the warp's 32 rows
@@ -290,15 +326,15 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
                 warp_store_rows128(dst + c * 32, (size_t)HD * 4, r);
             }
         };
-        const uint64_t sl2x2 = pack2(sl2, sl2), ngj2 = pack2(-gj2, -gj2);
         auto step = [&](auto first_tag, const int t) {
             constexpr bool FIRST = decltype(first_tag)::value;   // the diagonal chunk: causal mask, dSd written out
-            const float* st_ = rowstat + (t & 1) * 2 * kTile;   // [0,128): -lse2 (+gate), [128,256): -delta of the queries
+            const int gs = g + t;                                // running step number: ring slot and phase
+            const float* st_ = rowstat + (gs & 1) * 2 * kTile;   // [0,128): -lse2 (+gate), [128,256): -delta of the queries
             const int c0 = h * 64;               // query columns of this thread
             uint32_t pr[2][32];                  // S^T, then P^T (float bits)
             // ---- part A: P^T = exp2(S^T * scale - lse)
-            if (ok && !mbar_wait(&bars[K_STFULL + (t & 1)], (t >> 1) & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
-            if (ok && !mbar_wait(&bars[K_SFULL], t & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
+            if (ok && !mbar_wait(&bars[K_STFULL + (gs & 1)], (gs >> 1) & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
+            if (ok && !mbar_wait(&bars[K_SFULL], gs & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after_sync();
             if (ok) {
@@ -332,14 +368,11 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
             tc_fence_before_sync();
             mbar_arrive(&bars[K_PFULL]);
             // ---- part B: dS^T = P^T o (dP^T - delta)
-            if (ok && !mbar_wait(&bars[K_DPFULL], t & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
+            if (ok && !mbar_wait(&bars[K_DPFULL], gs & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after_sync();
-            // dP^T ready means every product issued before it has retired: dK of a finished level is complete.  It is
-            // taken into registers now and written out after dS^T has been delivered, off the tensor pipe's path.
+            // dP^T ready means every product issued before it has retired: dK of a finished level can be flushed
             if (!FIRST && ok && t >= 2 && level(t) != level(t - 1)) flush_dk(level(t - 1));
-            const bool fl = false;
-            uint32_t fr[CW / 32][32];
             if (ok) {
                 const float* dl_ = st_ + kTile;
 #pragma unroll
@@ -376,29 +409,34 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
             }
             tc_fence_before_sync();
             mbar_arrive(&bars[K_DSFULL]);
-            mbar_arrive(&bars[K_STEMPTY + (t & 1)]);
-            if (fl) {
-                float* dst = p.dkv + ((size_t)ver_row(kslot(level(t - 1), J), J) + q4 * 32) * HD + h * CW;
-#pragma unroll
-                for (int c = 0; c < CW / 32; ++c) {
-#pragma unroll
-                    for (int x = 0; x < 32; ++x) fr[c][x] = __float_as_uint(__uint_as_float(fr[c][x]) * p.scale);
-                    warp_store_rows128(dst + c * 32, (size_t)HD * 4, fr[c]);
-                }
-            }
+            mbar_arrive(&bars[K_STEMPTY + (gs & 1)]);
         };
-        step(std::true_type{}, 0);
 #pragma unroll 1
-        for (int t = 1; t < T; ++t) step(std::false_type{}, t);
-        if (ok && !mbar_wait(&bars[K_FINAL], 0, abort_flag, ST_DKV_COMPUTE)) ok = false;
-        ok = __all_sync(0xffffffffu, ok);
-        tc_fence_after_sync();
-        if (GATE) {   // the two threads of a key row add their halves of the column sum
-            if (h == 1) rowstat[row] = dsum;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (h == 0 && ok) p.dG[(size_t)s * p.Lp + kj] = -(dsum + rowstat[row]);
-        }
-        if (ok) {
+        for (int it = 0; item_of(it, J, s); ++it) {
+            const int T = p.N - J;
+            const int kj = J * kTile + row;          // key position of this thread's row
+            if (GATE) {
+                const float gj2 = p.G[(size_t)s * p.Lp + kj] * kLog2e;
+                ngj2 = pack2(-gj2, -gj2);
+                dsum = 0.f;
+            }
+            step(std::true_type{}, 0);
+#pragma unroll 1
+            for (int t = 1; t < T; ++t) step(std::false_type{}, t);
+            g += T;
+            if (ok && !mbar_wait(&bars[K_ACCFULL], it & 1, abort_flag, ST_DKV_COMPUTE)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);
+            tc_fence_after_sync();
+            if (GATE) {   // the two threads of a key row add their halves of the column sum
+                if (h == 1) dsum_x[row] = dsum;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (h == 0 && ok) p.dG[(size_t)s * p.Lp + kj] = -(dsum + dsum_x[row]);
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+            }
+            if (!ok) {
+                mbar_arrive(&bars[K_ACCFREE]);
+                break;
+            }
             if (T > 1) flush_dk(level(T - 1));
             else {  // last chunk: no later query chunk, the boundary-adjusted keys get a zero gradient from the sweep
                 float4* dst = reinterpret_cast<float4*>(p.dkv + ((size_t)ver_row(0, J) + row) * HD + h * CW);
@@ -409,6 +447,8 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
                 tmem_ld32(tlane + colDV + h * CW, r0);
                 tmem_ld32(tlane + colDV + h * CW + 32, r1);
                 tmem_ld_wait();
+                tc_fence_before_sync();
+                mbar_arrive(&bars[K_ACCFREE]);   // both accumulators have been read
 #pragma unroll
                 for (int x = 0; x < 16; ++x) {
                     w[x] = pack_bf16(__uint_as_float(r0[2 * x]), __uint_as_float(r0[2 * x + 1]));
@@ -417,14 +457,14 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
                 const int row0 = J * kTile + q4 * 32;
                 warp_store_rows128((__nv_bfloat16*)p.dv + ((size_t)s * p.L + row0) * HD + h * CW, (size_t)HD * 2, w,
                                    p.L - row0);
-            } else
-#pragma unroll 1
-            for (int c = 0; c < CW / 32; ++c) {
+            } else {
                 uint32_t r[32];
-                tmem_ld32(tlane + colDV + h * CW + c * 32, r);
+                tmem_ld32(tlane + colDV + h * CW, r);
                 tmem_ld_wait();
+                tc_fence_before_sync();
+                mbar_arrive(&bars[K_ACCFREE]);
                 if (kj < p.L) {
-                    uint4* dst = reinterpret_cast<uint4*>((__nv_bfloat16*)p.dv + ((size_t)s * p.L + kj) * HD + h * CW + c * 32);
+                    uint4* dst = reinterpret_cast<uint4*>((__nv_bfloat16*)p.dv + ((size_t)s * p.L + kj) * HD + h * CW);
 #pragma unroll
                     for (int x = 0; x < 4; ++x)
                         dst[x] = make_uint4(pack_bf16(__uint_as_float(r[8 * x]), __uint_as_float(r[8 * x + 1])),
@@ -733,7 +773,13 @@ cudaError_t launch_one(const BwdTensorMaps& tm, const BwdParams& p, int which, c
     if (which == 0) {
         cudaError_t e = set_smem(dkv_kernel<HD, GATE>, kDkvSmem);
         if (e != cudaSuccess) return e;
-        dkv_kernel<HD, GATE><<<dim3(p.N, p.S), 384, kDkvSmem, st>>>(tm, p);
+        int dev = 0, sms = 0;
+        e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        const int pairs = (p.N * p.S + 1) / 2;
+        dkv_kernel<HD, GATE><<<dim3(pairs < sms ? pairs : sms), 384, kDkvSmem, st>>>(tm, p);
     } else {
         cudaError_t e = set_smem(dq_kernel<HD, GATE>, kDqSmem);
         if (e != cudaSuccess) return e;
