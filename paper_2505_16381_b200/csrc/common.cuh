@@ -71,7 +71,7 @@ struct LevelTensorMaps {
 
 struct LevelParams {
     LevelTable lv;
-    int l;                  // dyadic kernels: level being produced (fwd: l -> l + 1) / consumed (bwd); version kernels: l2
+    int l;                  // dyadic kernels: level being produced (fwd: l -> l + 1) / consumed (bwd); version kernels: number of levels
     int S, N, Lp;
     __nv_bfloat16 *dyh, *dyl, *qv, *kv;
     float *dqv, *dkv, *ddy;

@@ -180,104 +180,160 @@ __global__ void __launch_bounds__(256, 1) dyadic_fwd_kernel(const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------- version forward
-// grid = (S * N, 2): y = 0 queries, y = 1 keys.  Xv[l2][chunk] = Xv[l1][chunk] * Dy (queries) or Dy^T (keys).
+// grid = (S * N, 2): y = 0 queries, y = 1 keys; p.l = number of levels.  One CTA walks the whole chain of its chunk,
+// bottom level first:  Xv[l2] = Xv[l1] * Dy (queries) or Dy^T (keys).  The version just produced stays in shared
+// memory as the next step's left operand (the same bf16 values that go to global memory).
 template <int HD>
 __global__ void __launch_bounds__(256, 2) version_fwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
     const int is_key = blockIdx.y, s = blockIdx.x / p.N, ch = blockIdx.x % p.N;
-    int l1, b, src;
-    if (!version_step(is_key, ch, p.l, p.N, l1, b, src)) return;
+    int l1, b, src, l2 = 1;
+    for (; l2 < p.l; ++l2)
+        if (version_step(is_key, ch, l2, p.N, l1, b, src)) break;
+    if (l2 >= p.l) return;
     extern __shared__ uint8_t smem_raw[];
     Ctx c;
     setup<128>(c, smem_raw, kBar3);
-    const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
-    const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
-    const long row_dst = ((long)p.l * p.S + s) * p.Lp + (long)ch * kT;
-    uint8_t* sm = c.smem;
-    if (c.tid == 0) {
-        mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2);
-        tma_tile(sm, is_key ? &tm.kv : &tm.qv, &c.bars[0], HD, (int)row_src);
-        tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
-        tma_tile(sm + 2 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
-    }
-    loads_wait(c);
-    if (c.tid == 0 && c.ok) {
-        tc_fence_after_sync();
-        const uint32_t a = smem_u32(sm);
-        const int bop = is_key ? OP_K : OP_MN;
-        mma(c.tmem, a, OP_K, a + kTileB, bop, HD / 16, HD, false);
-        mma(c.tmem, a, OP_K, a + 2 * kTileB, bop, HD / 16, HD, true);
-        umma_commit(&c.bars[1]);
-    }
-    mma_wait(c);
-    if (c.ok) {
-        float v[32];
-        __nv_bfloat16* out = (is_key ? p.kv : p.qv) + (size_t)row_dst * HD;
-        for (int i = 0; i < HD / 64; ++i) {
-            const int c0 = c.half * (HD / 2) + i * 32;
-            tmem_row32(c.tl + c0, v);
-            gstore_bf16x32(out + (size_t)c.row * HD + c0, v);
+    uint8_t* sm = c.smem;   // slots: 0 current version, 1 Dy hi, 2 Dy lo
+    bool first = true;
+#pragma unroll 1
+    for (; l2 < p.l && c.ok; ++l2) {
+        if (!version_step(is_key, ch, l2, p.N, l1, b, src)) continue;
+        const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
+        const long row_dst = ((long)l2 * p.S + s) * p.Lp + (long)ch * kT;
+        if (c.tid == 0) {
+            mbar_expect_tx(&c.bars[0], (first ? 3 : 2) * kT * HD * 2);
+            if (first) {
+                const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
+                tma_tile(sm, is_key ? &tm.kv : &tm.qv, &c.bars[0], HD, (int)row_src);
+            }
+            tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
+            tma_tile(sm + 2 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
         }
+        loads_wait(c);
+        if (!first) publish();   // the left operand was written by this CTA's threads
+        if (c.tid == 0 && c.ok) {
+            tc_fence_after_sync();
+            const uint32_t a = smem_u32(sm);
+            const int bop = is_key ? OP_K : OP_MN;
+            mma(c.tmem, a, OP_K, a + kTileB, bop, HD / 16, HD, false);
+            mma(c.tmem, a, OP_K, a + 2 * kTileB, bop, HD / 16, HD, true);
+            umma_commit(&c.bars[1]);
+        }
+        mma_wait(c);
+        if (c.ok) {
+            float v[32];
+            __nv_bfloat16* out = (is_key ? p.kv : p.qv) + (size_t)row_dst * HD;
+            for (int i = 0; i < HD / 64; ++i) {
+                const int c0 = c.half * (HD / 2) + i * 32;
+                tmem_row32(c.tl + c0, v);
+                gstore_bf16x32(out + (size_t)c.row * HD + c0, v);
+                tile_store32(sm, c.row, c0, v);
+            }
+        }
+        first = false;
     }
     teardown<128>(c, p.status);
 }
 
 // ---------------------------------------------------------------------------------------------- version backward
-// With g = dXv[l2][chunk]:   dXv[l1][chunk] += g Dy^T (queries) or g Dy (keys);
-//                            dDy[l1][b]     += Xv[l1]^T g (queries) or g^T Xv[l1] (keys), atomically.
+// grid = (S * N, 2), p.l = number of levels.  One CTA walks the chain of its chunk top level first.  With
+// g = dXv[l2][chunk] (what the sweeps wrote there plus what arrived from the level above, which stays in tensor memory):
+//     dXv[l1][chunk] += g Dy^T (queries) or g Dy (keys);
+//     dDy[l1][b]     += Xv[l1]^T g (queries) or g^T Xv[l1] (keys), atomically.
+// Only the bottom of the chain is added back to global memory.  The next step's operands are fetched while the
+// current one runs.
 template <int HD>
 __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
     const int is_key = blockIdx.y, s = blockIdx.x / p.N, ch = blockIdx.x % p.N;
     int l1, b, src;
-    if (!version_step(is_key, ch, p.l, p.N, l1, b, src)) return;
+    auto next_step = [&](int from) {   // highest level <= from with a version step, 0 if none
+        for (int l = from; l >= 1; --l)
+            if (version_step(is_key, ch, l, p.N, l1, b, src)) return l;
+        return 0;
+    };
+    int l2 = next_step(p.l - 1);
+    if (l2 == 0) return;
     extern __shared__ uint8_t smem_raw[];
     Ctx c;
-    setup<256>(c, smem_raw, kBar4);
-    const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
-    const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
-    const long row_dst = ((long)p.l * p.S + s) * p.Lp + (long)ch * kT;
+    setup<256>(c, smem_raw, 7 * kTileB);
     float* dxv = is_key ? p.dkv : p.dqv;
-    uint8_t* sm = c.smem;   // slots: 0 g, 1 Dy hi, 2 Dy lo, 3 Xv
-    if (c.tid == 0) {
+    uint8_t* sm = c.smem;   // slot 0: g; two buffers of three slots: Dy hi, Dy lo, Xv[l1]
+    auto issue_loads = [&](int buf) {   // operands of the step described by (l1, b, src)
+        const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
+        const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
+        uint8_t* base = sm + (1 + 3 * buf) * kTileB;
         mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2);
-        tma_tile(sm + 1 * kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
-        tma_tile(sm + 2 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
-        tma_tile(sm + 3 * kTileB, is_key ? &tm.kv : &tm.qv, &c.bars[0], HD, (int)row_src);
-    }
-    conv(c, dxv + (size_t)row_dst * HD, HD, kT, sm);
-    loads_wait(c);
-    publish();
-    if (c.tid == 0 && c.ok) {
-        tc_fence_after_sync();
-        const uint32_t a = smem_u32(sm);
-        const int bop = is_key ? OP_MN : OP_K;
-        mma(c.tmem, a, OP_K, a + kTileB, bop, HD / 16, HD, false);
-        mma(c.tmem, a, OP_K, a + 2 * kTileB, bop, HD / 16, HD, true);
-        if (!is_key) mma(c.tmem + 128, a + 3 * kTileB, OP_MN, a, OP_MN, 8, HD, false);
-        else         mma(c.tmem + 128, a, OP_MN, a + 3 * kTileB, OP_MN, 8, HD, false);
-        umma_commit(&c.bars[1]);
-    }
-    mma_wait(c);
-    if (c.ok) {
-        acc_add_global<false>(c, 0, HD, kT, dxv + (size_t)row_src * HD);
-        // run-product gradient: stage the [d][d] accumulator in shared memory (the tiles are dead) so that the
-        // atomic adds of a warp fall on consecutive addresses
-        constexpr int LDS = HD + 4;
-        float* stage = (float*)sm;
-        float v[32];
-        for (int i = 0; i < HD / 64; ++i) {
-            const int c0 = c.half * (HD / 2) + i * 32;
-            tmem_row32(c.tl + 128 + c0, v);
-            if (c.row < HD) {
+        tma_tile(base, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
+        tma_tile(base + kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
+        tma_tile(base + 2 * kTileB, is_key ? &tm.kv : &tm.qv, &c.bars[0], HD, (int)row_src);
+    };
+    if (c.tid == 0) issue_loads(0);
+    int buf = 0;
+    bool have_acc = false;
+    long row_low = 0;   // rows of the level the accumulated contribution belongs to
+#pragma unroll 1
+    while (l2 >= 1 && c.ok) {
+        version_step(is_key, ch, l2, p.N, l1, b, src);
+        const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
+        const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
+        const long row_dst = ((long)l2 * p.S + s) * p.Lp + (long)ch * kT;
+        // g = gradient stored at this level (+ the contribution from above) -> bf16 tile
+        {
+            float v[32], a[32];
+            for (int i = 0; i < HD / 64; ++i) {
+                const int c0 = c.half * (HD / 2) + i * 32;
+                gload_f32x32(dxv + ((size_t)row_dst + c.row) * HD + c0, v);
+                if (have_acc) {
+                    tmem_row32(c.tl + c0, a);
 #pragma unroll
-                for (int x = 0; x < 8; ++x)
-                    *reinterpret_cast<float4*>(stage + c.row * LDS + c0 + 4 * x) =
-                        make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
+                    for (int x = 0; x < 32; ++x) v[x] += a[x];
+                }
+                tile_store32(sm, c.row, c0, v);
             }
         }
-        __syncthreads();
-        float* dst = p.ddy + (size_t)mat * HD * HD;
-        for (int idx = c.tid; idx < HD * HD; idx += 256) atomicAdd(dst + idx, stage[(idx / HD) * LDS + (idx % HD)]);
+        // the step after this one (its description replaces l1, b, src only after this step's were copied above)
+        const int l2n = next_step(l2 - 1);
+        loads_wait(c);
+        publish();
+        if (c.tid == 0 && c.ok) {
+            if (l2n >= 1) issue_loads(buf ^ 1);
+            tc_fence_after_sync();
+            const uint32_t g = smem_u32(sm), o = smem_u32(sm + (1 + 3 * buf) * kTileB);
+            const int bop = is_key ? OP_MN : OP_K;
+            mma(c.tmem, g, OP_K, o, bop, HD / 16, HD, false);
+            mma(c.tmem, g, OP_K, o + kTileB, bop, HD / 16, HD, true);
+            if (!is_key) mma(c.tmem + 128, o + 2 * kTileB, OP_MN, g, OP_MN, 8, HD, false);
+            else         mma(c.tmem + 128, g, OP_MN, o + 2 * kTileB, OP_MN, 8, HD, false);
+            umma_commit(&c.bars[1]);
+        }
+        mma_wait(c);
+        if (c.ok) {
+            // run-product gradient: stage the [d][d] accumulator in this step's (now dead) operand slots so that the
+            // atomic adds of a warp fall on consecutive addresses
+            constexpr int LDS = HD + 4;
+            float* stage = (float*)(sm + (1 + 3 * buf) * kTileB);
+            float v[32];
+            for (int i = 0; i < HD / 64; ++i) {
+                const int c0 = c.half * (HD / 2) + i * 32;
+                tmem_row32(c.tl + 128 + c0, v);
+                if (c.row < HD) {
+#pragma unroll
+                    for (int x = 0; x < 8; ++x)
+                        *reinterpret_cast<float4*>(stage + c.row * LDS + c0 + 4 * x) =
+                            make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
+                }
+            }
+            __syncthreads();
+            float* dst = p.ddy + (size_t)mat * HD * HD;
+            for (int idx = c.tid; idx < HD * HD; idx += 256) atomicAdd(dst + idx, stage[(idx / HD) * LDS + (idx % HD)]);
+            __syncthreads();   // the staging area is the buffer the prefetch after next will fill
+        }
+        have_acc = true;
+        row_low = row_src;
+        l2 = l2n;
+        buf ^= 1;
     }
+    if (c.ok && have_acc) acc_add_global<false>(c, 0, HD, kT, dxv + (size_t)row_low * HD);
     teardown<256>(c, p.status);
 }
 
@@ -343,7 +399,7 @@ cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const Leve
         }
         case LEVEL_VERSION_BWD: {
             dim3 g(p.S * p.N, 2);
-            return hd == 64 ? launch(version_bwd_kernel<64>, g, 4, tm, p, st) : launch(version_bwd_kernel<128>, g, 4, tm, p, st);
+            return hd == 64 ? launch(version_bwd_kernel<64>, g, 7, tm, p, st) : launch(version_bwd_kernel<128>, g, 7, tm, p, st);
         }
         default: {
             dim3 g(p.S * p.lv.dy_cnt[p.l]);

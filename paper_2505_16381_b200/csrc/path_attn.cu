@@ -239,10 +239,8 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
         lp.l = l;
         LAUNCH(launch_level_kernel(LEVEL_DYADIC_FWD, tm, lp, d, st));
     }
-    for (int l2 = 1; l2 < p.nlev; ++l2) {         // query and key versions, level by level
-        lp.l = l2;
-        LAUNCH(launch_level_kernel(LEVEL_VERSION_FWD, tm, lp, d, st));
-    }
+    lp.l = p.nlev;                                // query and key versions: one CTA per chunk walks its chain
+    LAUNCH(launch_level_kernel(LEVEL_VERSION_FWD, tm, lp, d, st));
     prof_mark(stg_lev, 1, st);
     return PATH_OK;
 }
@@ -350,10 +348,8 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
         LevelTensorMaps ltm;
         if (!make_level_maps(p, ws, ltm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
         LevelParams lp = level_params(p, ws);
-        for (int l2 = p.nlev - 1; l2 >= 1; --l2) {
-            lp.l = l2;
-            LAUNCH(launch_level_kernel(LEVEL_VERSION_BWD, ltm, lp, d, st));
-        }
+        lp.l = p.nlev;
+        LAUNCH(launch_level_kernel(LEVEL_VERSION_BWD, ltm, lp, d, st));
         for (int l = p.nlev - 2; l >= 1; --l) {
             lp.l = l;
             LAUNCH(launch_level_kernel(LEVEL_DYADIC_BWD, ltm, lp, d, st));
