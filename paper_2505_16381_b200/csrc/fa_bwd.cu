@@ -485,20 +485,15 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
 }
 
 // ------------------------------------------------------------------------------------------------ dQ
-enum { Q_QFULL = 0, Q_QEMPTY, Q_DOFULL, Q_KFULL, Q_KEMPTY = Q_KFULL + 3, Q_VFULL = Q_KEMPTY + 3,
-       Q_VEMPTY = Q_VFULL + 2, Q_SFULL = Q_VEMPTY + 2, Q_DPFULL = Q_SFULL + 2, Q_DSFULL, Q_FINAL,
+// Persistent like the dK/dV sweep: items are the query chunks of a slice, paired (longest, shortest).
+enum { Q_QFULL = 0, Q_QEMPTY, Q_DOFULL, Q_DOEMPTY, Q_KFULL, Q_KEMPTY = Q_KFULL + 3, Q_VFULL = Q_KEMPTY + 3,
+       Q_VEMPTY = Q_VFULL + 2, Q_SFULL = Q_VEMPTY + 2, Q_DPFULL = Q_SFULL + 2, Q_DSFULL, Q_ACCFULL, Q_ACCFREE,
        Q_GKFULL, Q_GKEMPTY = Q_GKFULL + 2, Q_COUNT = Q_GKEMPTY + 2 };
 constexpr uint32_t kDqGk = 7 * kSlotBytes + 256;              // [2][128] gate prefix of the key chunk, [128] exchange
 constexpr uint32_t kDqTotal = kDqGk + 3 * kTile * 4;
 
 template <int HD, bool GATE>
 __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdTensorMaps tm, const BwdParams p) {
-    const int I = (int)gridDim.x - 1 - (int)blockIdx.x, s = blockIdx.y;
-    if (I == 0) {  // chunk 0 has no earlier keys: its boundary-adjusted queries get a zero gradient from the sweep
-        float4* dst = reinterpret_cast<float4*>(p.dqv + (size_t)s * p.Lp * HD);
-        for (int i = threadIdx.x; i < kTile * HD / 4; i += blockDim.x) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        return;
-    }
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     if ((uint32_t)(smem - smem_raw) + kDqTotal > kSmemAlloc) {   // uniform over the CTA
@@ -507,8 +502,8 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
     }
     uint8_t* sQ = smem;
     uint8_t* sDO = sQ + kSlotBytes;
-    uint8_t* sK = sDO + kSlotBytes;        // 3 slots
-    uint8_t* sV = sK + 3 * kSlotBytes;     // 2 slots
+    uint8_t* sK = sDO + kSlotBytes;        // ring of 3
+    uint8_t* sV = sK + 3 * kSlotBytes;     // ring of 2
     uint64_t* bars = (uint64_t*)(smem + 7 * kSlotBytes);
     uint32_t* tmem_slot = (uint32_t*)(bars + Q_COUNT);
     volatile uint32_t* abort_flag = (volatile uint32_t*)(tmem_slot + 1);
@@ -516,11 +511,11 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
     float* dsum_x = gk + 2 * kTile;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int T = I;  // steps t = 0..I-1, J = I-1-t
+    const int items = p.N * p.S;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < Q_COUNT; ++i)
-            mbar_init(&bars[i], (i == Q_DSFULL || i == Q_GKEMPTY || i == Q_GKEMPTY + 1) ? 256u : 1u);
+            mbar_init(&bars[i], (i == Q_DSFULL || i == Q_ACCFREE || i == Q_GKEMPTY || i == Q_GKEMPTY + 1) ? 256u : 1u);
         *abort_flag = 0;
         mbar_fence_init();
     }
@@ -531,6 +526,16 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
     tc_fence_after_sync();
     const uint32_t tmem = *tmem_slot;
     constexpr uint32_t colS = 0, colDP = 256, colDQ = 384;   // two S tiles at 0 and 128
+    // k-th work item of this CTA; query chunk I has I steps (t = 0..I-1, key chunk J = I-1-t)
+    auto item_of = [&](int k, int& I, int& s) {
+        const int w = 2 * ((int)blockIdx.x + (k >> 1) * (int)gridDim.x) + (k & 1);
+        if (w >= items) return false;
+        s = w / p.N;
+        const int j = w % p.N;
+        I = (j & 1) ? (j >> 1) : p.N - 1 - (j >> 1);
+        return true;
+    };
+    int I = 0, s = 0;
     auto ver_row = [&](int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
     auto level = [&](int t) { return msb32((unsigned)(I ^ (I - 1 - t))); };
 
@@ -538,89 +543,113 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
         asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
         if (warp == 0 && lane == 0) {
             bool ok = true;
-            int nq = 0;
+            int nq = 0, nd = 0, kn = 0, vn = 0;   // fills so far: Q, dO, K ring, V ring (= gate ring)
             auto wait_empty = [&](int bar, int use) {
                 if (ok && !mbar_wait(&bars[bar], (use & 1) ^ 1, abort_flag, ST_DQ_PRODUCER)) ok = false;
             };
-            mbar_expect_tx(&bars[Q_DOFULL], kTile * HD * 2);
-            tma_tile(sDO, &tm.d_o, &bars[Q_DOFULL], HD, s * p.Lp + I * kTile);
-            for (int t = 0; t < T && ok; ++t) {
-                const int J = I - 1 - t, l = level(t);
-                if (t == 0 || l != level(t - 1)) {
-                    wait_empty(Q_QEMPTY, nq);
-                    if (!ok) break;
-                    mbar_expect_tx(&bars[Q_QFULL], kTile * HD * 2);
-                    tma_tile(sQ, &tm.qv, &bars[Q_QFULL], HD, ver_row(qslot(l, I), I));
-                    ++nq;
-                }
-                wait_empty(Q_KEMPTY + t % 3, t / 3);
+#pragma unroll 1
+            for (int it = 0; ok && item_of(it, I, s); ++it) {
+                const int T = I;
+                if (T == 0) continue;
+                wait_empty(Q_DOEMPTY, nd);
                 if (!ok) break;
-                mbar_expect_tx(&bars[Q_KFULL + t % 3], kTile * HD * 2);
-                tma_tile(sK + (t % 3) * kSlotBytes, &tm.kv, &bars[Q_KFULL + t % 3], HD, ver_row(kslot(l, J), J));
-                wait_empty(Q_VEMPTY + (t & 1), t >> 1);
-                if (!ok) break;
-                mbar_expect_tx(&bars[Q_VFULL + (t & 1)], kTile * HD * 2);
-                tma_tile(sV + (t & 1) * kSlotBytes, &tm.v, &bars[Q_VFULL + (t & 1)], HD, s * p.Lp + J * kTile);
-                if (GATE) {   // gate prefix of the key chunk
-                    wait_empty(Q_GKEMPTY + (t & 1), t >> 1);
+                mbar_expect_tx(&bars[Q_DOFULL], kTile * HD * 2);
+                tma_tile(sDO, &tm.d_o, &bars[Q_DOFULL], HD, s * p.Lp + I * kTile);
+                ++nd;
+#pragma unroll 1
+                for (int t = 0; t < T && ok; ++t) {
+                    const int J = I - 1 - t, l = level(t);
+                    if (t == 0 || l != level(t - 1)) {
+                        wait_empty(Q_QEMPTY, nq);
+                        if (!ok) break;
+                        mbar_expect_tx(&bars[Q_QFULL], kTile * HD * 2);
+                        tma_tile(sQ, &tm.qv, &bars[Q_QFULL], HD, ver_row(qslot(l, I), I));
+                        ++nq;
+                    }
+                    wait_empty(Q_KEMPTY + kn % 3, kn / 3);
                     if (!ok) break;
-                    mbar_expect_tx(&bars[Q_GKFULL + (t & 1)], kTile * 4);
-                    bulk_load(gk + (t & 1) * kTile, p.G + (size_t)s * p.Lp + J * kTile, kTile * 4, &bars[Q_GKFULL + (t & 1)]);
+                    mbar_expect_tx(&bars[Q_KFULL + kn % 3], kTile * HD * 2);
+                    tma_tile(sK + (kn % 3) * kSlotBytes, &tm.kv, &bars[Q_KFULL + kn % 3], HD, ver_row(kslot(l, J), J));
+                    ++kn;
+                    wait_empty(Q_VEMPTY + (vn & 1), vn >> 1);
+                    if (!ok) break;
+                    mbar_expect_tx(&bars[Q_VFULL + (vn & 1)], kTile * HD * 2);
+                    tma_tile(sV + (vn & 1) * kSlotBytes, &tm.v, &bars[Q_VFULL + (vn & 1)], HD, s * p.Lp + J * kTile);
+                    if (GATE) {   // gate prefix of the key chunk
+                        wait_empty(Q_GKEMPTY + (vn & 1), vn >> 1);
+                        if (!ok) break;
+                        mbar_expect_tx(&bars[Q_GKFULL + (vn & 1)], kTile * 4);
+                        bulk_load(gk + (vn & 1) * kTile, p.G + (size_t)s * p.Lp + J * kTile, kTile * 4,
+                                  &bars[Q_GKFULL + (vn & 1)]);
+                    }
+                    ++vn;
                 }
             }
         } else if (warp == 1 && lane == 0) {
             constexpr uint32_t idescS = umma_idesc(128, 128, 0, 0);
             constexpr uint32_t idescD = umma_idesc(128, HD, 0, 1);
             bool ok = true;
-            int nq = 0;
+            int nq = 0, nd = 0, g = 0, na = 0;   // Q / dO fills consumed, steps before this item, items with steps so far
+            int T = 0;
             auto wait = [&](int bar, int parity) {
                 if (ok && !mbar_wait(&bars[bar], parity & 1, abort_flag, ST_DQ_MMA)) ok = false;
             };
-            auto issue_s = [&](int t) {      // S(t) into tile t & 1
+            auto issue_s = [&](int t) {      // S(t) into the tile of running step g + t
+                const int gs = g + t;
                 if (t == 0 || level(t) != level(t - 1)) { wait(Q_QFULL, nq); ++nq; }
-                wait(Q_KFULL + t % 3, t / 3);
+                wait(Q_KFULL + gs % 3, gs / 3);
                 tc_fence_after_sync();
                 if (!ok) return;
-                mma_kk(tmem + colS + (t & 1) * 128, smem_u32(sQ), smem_u32(sK + (t % 3) * kSlotBytes), HD, idescS, false);
-                umma_commit(&bars[Q_SFULL + (t & 1)]);
-                if (t + 1 < T && level(t + 1) != level(t)) umma_commit(&bars[Q_QEMPTY]);
+                mma_kk(tmem + colS + (gs & 1) * 128, smem_u32(sQ), smem_u32(sK + (gs % 3) * kSlotBytes), HD, idescS, false);
+                umma_commit(&bars[Q_SFULL + (gs & 1)]);
+                if (t + 1 >= T || level(t + 1) != level(t)) umma_commit(&bars[Q_QEMPTY]);
             };
             auto issue_dp = [&](int t) {
-                wait(Q_VFULL + (t & 1), t >> 1);
+                const int gs = g + t;
+                wait(Q_VFULL + (gs & 1), gs >> 1);
                 tc_fence_after_sync();
                 if (!ok) return;
-                mma_kk(tmem + colDP, smem_u32(sDO), smem_u32(sV + (t & 1) * kSlotBytes), HD, idescS, false);
+                mma_kk(tmem + colDP, smem_u32(sDO), smem_u32(sV + (gs & 1) * kSlotBytes), HD, idescS, false);
                 umma_commit(&bars[Q_DPFULL]);
-                umma_commit(&bars[Q_VEMPTY + (t & 1)]);
+                umma_commit(&bars[Q_VEMPTY + (gs & 1)]);
+                if (t + 1 >= T) umma_commit(&bars[Q_DOEMPTY]);   // the item's last use of dO
             };
-            wait(Q_DOFULL, 0);
-            issue_s(0);
-            issue_dp(0);
-            if (T > 1) issue_s(1);
-            for (int t = 0; t < T && ok; ++t) {
-                // dQ += dS K.  dP of the next step overwrites dS, S(t+2) the tile whose P every thread has taken into
-                // registers before it delivered dS: in-order execution keeps both behind what they replace.
-                wait(Q_DSFULL, t);
-                tc_fence_after_sync();
-                if (!ok) break;
-                mma_tn(tmem + colDQ, tmem + colDP, smem_u32(sK + (t % 3) * kSlotBytes), idescD,
-                       !(t == 0 || level(t) != level(t - 1)));
-                umma_commit(&bars[Q_KEMPTY + t % 3]);
-                if (t + 1 < T) issue_dp(t + 1);
-                if (t + 2 < T) issue_s(t + 2);
-                if (t == T - 1) umma_commit(&bars[Q_FINAL]);
+#pragma unroll 1
+            for (int it = 0; ok && item_of(it, I, s); ++it) {
+                T = I;
+                if (T == 0) continue;
+                wait(Q_DOFULL, nd); ++nd;
+                issue_s(0);
+                issue_dp(0);
+                if (T > 1) issue_s(1);
+#pragma unroll 1
+                for (int t = 0; t < T && ok; ++t) {
+                    const int gs = g + t;
+                    // dQ += dS K.  dP of the next step overwrites dS, S(t+2) the tile whose P every thread has taken
+                    // into registers before it delivered dS: in-order execution keeps both behind what they replace.
+                    wait(Q_DSFULL, gs);
+                    if (t == 0 && na > 0) wait(Q_ACCFREE, na - 1);   // the previous item's dQ has been read
+                    tc_fence_after_sync();
+                    if (!ok) break;
+                    mma_tn(tmem + colDQ, tmem + colDP, smem_u32(sK + (gs % 3) * kSlotBytes), idescD,
+                           !(t == 0 || level(t) != level(t - 1)));
+                    umma_commit(&bars[Q_KEMPTY + gs % 3]);
+                    if (t + 1 < T) issue_dp(t + 1);
+                    if (t + 2 < T) issue_s(t + 2);
+                    if (t == T - 1) umma_commit(&bars[Q_ACCFULL]);
+                }
+                g += T;
+                ++na;
             }
         }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
         const int q4 = warp & 3, h = (warp - 4) >> 2, row = q4 * 32 + lane;
         const uint32_t tlane = tmem + ((uint32_t)(q4 * 32) << 16);
-        const size_t qi = (size_t)s * p.Lp + I * kTile + row;
         const float sl2 = p.scale * kLog2e;
-        const float ndelta = p.delta[qi];            // minus delta
-        const float nl = p.lse2[qi];                 // minus lse2, plus the gate prefix of the row when gated
-        float dsum = 0.f;
+        const uint64_t sl2x2 = pack2(sl2, sl2), nlog2 = pack2(-kLog2e, -kLog2e);
         bool ok = true;
+        int g = 0, na = 0;
         constexpr int CW = HD / 2;
         auto flush_dq = [&](int lvl) {
             float* dst = p.dqv + ((size_t)ver_row(qslot(lvl, I), I) + q4 * 32) * HD + h * CW;   // the warp's 32 rows
@@ -634,92 +663,97 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
                 warp_store_rows128(dst + c * 32, (size_t)HD * 4, r);
             }
         };
-        const uint64_t sl2x2 = pack2(sl2, sl2), nl2 = pack2(nl, nl), nd2 = pack2(ndelta, ndelta);
-        const uint64_t nlog2 = pack2(-kLog2e, -kLog2e);
-        for (int t = 0; t < T; ++t) {
-            const int c0 = h * 64;               // key columns of this thread
-            uint32_t pr[2][32];                  // S, then P (float bits)
-            // ---- part A: P = exp2(S * scale - lse)
-            if (GATE && ok && !mbar_wait(&bars[Q_GKFULL + (t & 1)], (t >> 1) & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
-            if (ok && !mbar_wait(&bars[Q_SFULL + (t & 1)], (t >> 1) & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
-            ok = __all_sync(0xffffffffu, ok);
-            tc_fence_after_sync();
-            if (ok) {
-                tmem_ld32(tlane + colS + (t & 1) * 128 + c0, pr[0]);
-                tmem_ld32(tlane + colS + (t & 1) * 128 + c0 + 32, pr[1]);
-                tmem_ld_wait();
-                const float* g_ = gk + (t & 1) * kTile + c0;
-#pragma unroll
-                for (int c = 0; c < 2; ++c)
-#pragma unroll
-                    for (int x = 0; x < 32; x += 4) {
-                        uint64_t v01 = fma2(pack2(__uint_as_float(pr[c][x]), __uint_as_float(pr[c][x + 1])), sl2x2, nl2);
-                        uint64_t v23 = fma2(pack2(__uint_as_float(pr[c][x + 2]), __uint_as_float(pr[c][x + 3])), sl2x2, nl2);
-                        if (GATE) {
-                            const float4 g4 = *reinterpret_cast<const float4*>(g_ + c * 32 + x);
-                            v01 = fma2(pack2(g4.x, g4.y), nlog2, v01);
-                            v23 = fma2(pack2(g4.z, g4.w), nlog2, v23);
-                        }
-                        float e[4];
-                        unpack2(v01, e[0], e[1]);
-                        unpack2(v23, e[2], e[3]);
-#pragma unroll
-                        for (int y = 0; y < 4; ++y) pr[c][x + y] = __float_as_uint(ex2(e[y]));
-                    }
+#pragma unroll 1
+        for (int it = 0; item_of(it, I, s); ++it) {
+            const int T = I;
+            if (T == 0) {  // chunk 0 has no earlier keys: its boundary-adjusted queries get a zero gradient from the sweep
+                float4* dst = reinterpret_cast<float4*>(p.dqv + (size_t)s * p.Lp * HD);
+                for (int i = threadIdx.x - 128; i < kTile * HD / 4; i += 256) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                continue;
             }
-            // ---- part B: dS = P o (dP - delta)
-            if (ok && !mbar_wait(&bars[Q_DPFULL], t & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
-            ok = __all_sync(0xffffffffu, ok);
-            tc_fence_after_sync();
-            // dP ready means every product issued before it has retired: dQ of a finished level is complete.  It is
-            // taken into registers now and written out after dS has been delivered, off the tensor pipe's path.
-            const bool fl = ok && t >= 1 && level(t) != level(t - 1);
-            uint32_t fr[CW / 32][32];
-            if (fl) {
-#pragma unroll
-                for (int c = 0; c < CW / 32; ++c) tmem_ld32(tlane + colDQ + h * CW + c * 32, fr[c]);
-            }
-            if (ok) {
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t dp[32], pk[16];
-                    tmem_ld32(tlane + colDP + c0 + c * 32, dp);
+            const size_t qi = (size_t)s * p.Lp + I * kTile + row;
+            const float ndelta = p.delta[qi];            // minus delta
+            const float nl = p.lse2[qi];                 // minus lse2, plus the gate prefix of the row when gated
+            const uint64_t nl2 = pack2(nl, nl), nd2 = pack2(ndelta, ndelta);
+            float dsum = 0.f;
+#pragma unroll 1
+            for (int t = 0; t < T; ++t) {
+                const int gs = g + t;
+                const int c0 = h * 64;               // key columns of this thread
+                uint32_t pr[2][32];                  // S, then P (float bits)
+                // ---- part A: P = exp2(S * scale - lse)
+                if (GATE && ok && !mbar_wait(&bars[Q_GKFULL + (gs & 1)], (gs >> 1) & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
+                if (ok && !mbar_wait(&bars[Q_SFULL + (gs & 1)], (gs >> 1) & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
+                ok = __all_sync(0xffffffffu, ok);
+                tc_fence_after_sync();
+                if (ok) {
+                    tmem_ld32(tlane + colS + (gs & 1) * 128 + c0, pr[0]);
+                    tmem_ld32(tlane + colS + (gs & 1) * 128 + c0 + 32, pr[1]);
                     tmem_ld_wait();
+                    const float* g_ = gk + (gs & 1) * kTile + c0;
 #pragma unroll
-                    for (int x = 0; x < 32; x += 2) {
-                        const uint64_t d01 = mul2(pack2(__uint_as_float(pr[c][x]), __uint_as_float(pr[c][x + 1])),
-                                                  add2(pack2(__uint_as_float(dp[x]), __uint_as_float(dp[x + 1])), nd2));
-                        float d0, d1;
-                        unpack2(d01, d0, d1);
-                        if (GATE) dsum += d0 + d1;
-                        pk[x >> 1] = pack_bf16(d0, d1);
+                    for (int c = 0; c < 2; ++c)
+#pragma unroll
+                        for (int x = 0; x < 32; x += 4) {
+                            uint64_t v01 = fma2(pack2(__uint_as_float(pr[c][x]), __uint_as_float(pr[c][x + 1])), sl2x2, nl2);
+                            uint64_t v23 = fma2(pack2(__uint_as_float(pr[c][x + 2]), __uint_as_float(pr[c][x + 3])), sl2x2, nl2);
+                            if (GATE) {
+                                const float4 g4 = *reinterpret_cast<const float4*>(g_ + c * 32 + x);
+                                v01 = fma2(pack2(g4.x, g4.y), nlog2, v01);
+                                v23 = fma2(pack2(g4.z, g4.w), nlog2, v23);
+                            }
+                            float e[4];
+                            unpack2(v01, e[0], e[1]);
+                            unpack2(v23, e[2], e[3]);
+#pragma unroll
+                            for (int y = 0; y < 4; ++y) pr[c][x + y] = __float_as_uint(ex2(e[y]));
+                        }
+                }
+                // ---- part B: dS = P o (dP - delta)
+                if (ok && !mbar_wait(&bars[Q_DPFULL], gs & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
+                ok = __all_sync(0xffffffffu, ok);
+                tc_fence_after_sync();
+                // dP ready means every product issued before it has retired: dQ of a finished level can be flushed
+                if (ok && t >= 1 && level(t) != level(t - 1)) flush_dq(level(t - 1));
+                if (ok) {
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t dp[32], pk[16];
+                        tmem_ld32(tlane + colDP + c0 + c * 32, dp);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int x = 0; x < 32; x += 2) {
+                            const uint64_t d01 = mul2(pack2(__uint_as_float(pr[c][x]), __uint_as_float(pr[c][x + 1])),
+                                                      add2(pack2(__uint_as_float(dp[x]), __uint_as_float(dp[x + 1])), nd2));
+                            float d0, d1;
+                            unpack2(d01, d0, d1);
+                            if (GATE) dsum += d0 + d1;
+                            pk[x >> 1] = pack_bf16(d0, d1);
+                        }
+                        tmem_st16(tlane + colDP + c0 + c * 16, pk);
                     }
-                    tmem_st16(tlane + colDP + c0 + c * 16, pk);
+                    tmem_st_wait();
                 }
-                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(&bars[Q_DSFULL]);
+                if (GATE) mbar_arrive(&bars[Q_GKEMPTY + (gs & 1)]);
             }
+            g += T;
+            if (ok && !mbar_wait(&bars[Q_ACCFULL], na & 1, abort_flag, ST_DQ_COMPUTE)) ok = false;
+            ++na;
+            ok = __all_sync(0xffffffffu, ok);
+            tc_fence_after_sync();
+            if (GATE) {
+                if (h == 1) dsum_x[row] = dsum;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (h == 0 && ok) p.dGrow[qi] = dsum + dsum_x[row];
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+            }
+            if (ok) flush_dq(level(T - 1));
             tc_fence_before_sync();
-            mbar_arrive(&bars[Q_DSFULL]);
-            if (GATE) mbar_arrive(&bars[Q_GKEMPTY + (t & 1)]);
-            if (fl) {
-                float* dst = p.dqv + ((size_t)ver_row(qslot(level(t - 1), I), I) + q4 * 32) * HD + h * CW;
-#pragma unroll
-                for (int c = 0; c < CW / 32; ++c) {
-#pragma unroll
-                    for (int x = 0; x < 32; ++x) fr[c][x] = __float_as_uint(__uint_as_float(fr[c][x]) * p.scale);
-                    warp_store_rows128(dst + c * 32, (size_t)HD * 4, fr[c]);
-                }
-            }
+            mbar_arrive(&bars[Q_ACCFREE]);
+            if (!ok) break;
         }
-        if (ok && !mbar_wait(&bars[Q_FINAL], 0, abort_flag, ST_DQ_COMPUTE)) ok = false;
-        ok = __all_sync(0xffffffffu, ok);
-        tc_fence_after_sync();
-        if (GATE) {
-            if (h == 1) dsum_x[row] = dsum;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (h == 0 && ok) p.dGrow[qi] = dsum + dsum_x[row];
-        }
-        if (ok) flush_dq(level(T - 1));
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -783,7 +817,13 @@ cudaError_t launch_one(const BwdTensorMaps& tm, const BwdParams& p, int which, c
     } else {
         cudaError_t e = set_smem(dq_kernel<HD, GATE>, kDqSmem);
         if (e != cudaSuccess) return e;
-        dq_kernel<HD, GATE><<<dim3(p.N, p.S), 384, kDqSmem, st>>>(tm, p);
+        int dev = 0, sms = 0;
+        e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        const int pairs = (p.N * p.S + 1) / 2;
+        dq_kernel<HD, GATE><<<dim3(pairs < sms ? pairs : sms), 384, kDqSmem, st>>>(tm, p);
     }
     return cudaGetLastError();
 }
