@@ -75,15 +75,25 @@ __device__ __forceinline__ void gload_f32x32(const float* src, float (&v)[32], b
     const int j = threadIdx.x & 3;
     uint32_t w[32];
     const unsigned long long mine = (unsigned long long)src;
+    // all four loads are issued before any of their data is touched, so that they are in flight together
+    unsigned long long ptr[4];
+    bool ok[4];
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-        uint32_t d[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-        const unsigned long long ptr = r == 0 ? mine : __shfl_xor_sync(0xffffffffu, mine, r);
-        const bool ok = r == 0 ? valid : (bool)__shfl_xor_sync(0xffffffffu, (int)valid, r);
-        if (ok) ld_global_v8((const uint8_t*)ptr + 32 * j, d);
-#pragma unroll
-        for (int x = 0; x < 8; ++x) w[8 * r + x] = r == 0 ? d[x] : __shfl_xor_sync(0xffffffffu, d[x], r);
+        ptr[r] = r == 0 ? mine : __shfl_xor_sync(0xffffffffu, mine, r);
+        ok[r] = r == 0 ? valid : (bool)__shfl_xor_sync(0xffffffffu, (int)valid, r);
     }
+    uint32_t d[4][8];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+#pragma unroll
+        for (int x = 0; x < 8; ++x) d[r][x] = 0u;
+        if (ok[r]) ld_global_v8((const uint8_t*)ptr[r] + 32 * j, d[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int x = 0; x < 8; ++x) w[8 * r + x] = r == 0 ? d[r][x] : __shfl_xor_sync(0xffffffffu, d[r][x], r);
     rot4_pieces(w, j);
 #pragma unroll
     for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(w[x]);
