@@ -39,9 +39,15 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the kernel named by `roofline.kernel`,
 # from the ncu capture summarised under profiles/ (None until one exists for that kernel).
-# DRAM bytes per launch PER (batch, head) SLICE at the C3 shape (L=4096, d=128), from the ncu captures at batch 2
-# (32 slices) summarised under profiles/; slices are independent, so a launch over S slices moves S times this.
-NCU_TRAFFIC_BYTES_PER_SLICE = {}
+# DRAM bytes per launch PER (batch, head) SLICE at the C3 shape (L=4096, d=128), from the ncu captures at batch 1
+# (16 slices) summarised under profiles/; slices are independent, so a launch over S slices moves S times this.
+NCU_TRAFFIC_BYTES_PER_SLICE = {
+    "chunk_prep": (52.00e6 + 181.54e6) / 16,        # backward instance (the step's forward runs on the shared workspace)
+    "fa_fwd": (168.36e6 + 8.04e6) / 16,
+    "fa_bwd_dkv": (187.07e6 + 100.26e6) / 16,
+    "fa_bwd_dq": (117.71e6 + 47.99e6) / 16,
+    "bwd_chunk_chain": (339.18e6 + 37.59e6) / 16,
+}
 
 
 # ----------------------------------------------------------------------------------------- FLOP models
@@ -300,7 +306,9 @@ def run_ours(args, cfg):
     stage_flops = {"fa_fwd": f1 + diag, "fa_bwd_dkv": 2.0 * f1 + diag, "fa_bwd_dq": 1.5 * f1}
     t_d, t_b = CHUNK * d * 2, CHUNK * CHUNK * 2                 # bytes of a [128 x d] / [128 x 128] bf16 tile
     prep_bytes = nch * (3 * t_d + 2 * t_d + 2 * t_b + 2 * d * d * 2)
-    stage_bytes = {"chunk_prep": prep_bytes, "bwd_chunk_prep": prep_bytes + nch * (7 * t_b + t_d),
+    # the step's forward runs on the backward-sized workspace, so its chunk preparation is the instance that also
+    # stores the bf16 tiles of the chain rule (and the backward then skips its own)
+    stage_bytes = {"chunk_prep": prep_bytes + nch * (7 * t_b + t_d), "bwd_chunk_prep": prep_bytes + nch * (7 * t_b + t_d),
                    "bwd_chunk_chain": nch * (4 * t_d + 7 * t_b + 2 * 2 * t_d + 2 * t_b + d * d * 4 + 3 * t_d)}
     def ncu_traffic(kernel):
         per_slice = NCU_TRAFFIC_BYTES_PER_SLICE.get(kernel)
