@@ -271,18 +271,28 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
     int buf = 0;
     bool have_acc = false;
     long row_low = 0;   // rows of the level the accumulated contribution belongs to
+    // The gradient stored in global memory at the level a step consumes is requested one step ahead (the first one
+    // here), so that its latency hides behind the previous step's products and atomics.
+    constexpr int NI = HD / 64;
+    uint32_t pend[NI][4][8];
+    {
+        const long row_top = ((long)l2 * p.S + s) * p.Lp + (long)ch * kT;
+#pragma unroll
+        for (int i = 0; i < NI; ++i)
+            gload_f32x32_issue(dxv + ((size_t)row_top + c.row) * HD + c.half * (HD / 2) + i * 32, pend[i]);
+    }
 #pragma unroll 1
     while (l2 >= 1 && c.ok) {
         version_step(is_key, ch, l2, p.N, l1, b, src);
         const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
         const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
-        const long row_dst = ((long)l2 * p.S + s) * p.Lp + (long)ch * kT;
         // g = gradient stored at this level (+ the contribution from above) -> bf16 tile
         {
             float v[32], a[32];
-            for (int i = 0; i < HD / 64; ++i) {
+#pragma unroll
+            for (int i = 0; i < NI; ++i) {
                 const int c0 = c.half * (HD / 2) + i * 32;
-                gload_f32x32(dxv + ((size_t)row_dst + c.row) * HD + c0, v);
+                gload_f32x32_finish(pend[i], v);
                 if (have_acc) {
                     tmem_row32(c.tl + c0, a);
 #pragma unroll
@@ -290,6 +300,10 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
                 }
                 tile_store32(sm, c.row, c0, v);
             }
+            // what is stored at the level this step contributes to: the next step's input, or the chain's final sum
+#pragma unroll
+            for (int i = 0; i < NI; ++i)
+                gload_f32x32_issue(dxv + ((size_t)row_src + c.row) * HD + c.half * (HD / 2) + i * 32, pend[i]);
         }
         // the step after this one (its description replaces l1, b, src only after this step's were copied above)
         const int l2n = next_step(l2 - 1);
@@ -325,7 +339,12 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
             }
             __syncthreads();
             float* dst = p.ddy + (size_t)mat * HD * HD;
-            for (int idx = c.tid; idx < HD * HD; idx += 256) atomicAdd(dst + idx, stage[(idx / HD) * LDS + (idx % HD)]);
+            for (int idx = c.tid * 4; idx < HD * HD; idx += 1024) {   // four consecutive elements per reduction
+                const float4 t = *reinterpret_cast<const float4*>(stage + (idx / HD) * LDS + (idx % HD));
+                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + idx), "f"(t.x), "f"(t.y), "f"(t.z),
+                             "f"(t.w)
+                             : "memory");
+            }
             __syncthreads();   // the staging area is the buffer the prefetch after next will fill
         }
         have_acc = true;
@@ -333,7 +352,18 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
         l2 = l2n;
         buf ^= 1;
     }
-    if (c.ok && have_acc) acc_add_global<false>(c, 0, HD, kT, dxv + (size_t)row_low * HD);
+    if (c.ok && have_acc) {   // bottom of the chain: stored value + carried contribution
+        float v[32], a[32];
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+            const int c0 = c.half * (HD / 2) + i * 32;
+            gload_f32x32_finish(pend[i], v);
+            tmem_row32(c.tl + c0, a);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) v[x] += a[x];
+            gstore_f32x32(dxv + ((size_t)row_low + c.row) * HD + c0, v);
+        }
+    }
     teardown<256>(c, p.status);
 }
 
@@ -357,6 +387,15 @@ __global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constan
         tma_tile(sm + 4 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat_lo * HD));
     }
     conv(c, p.ddy + (size_t)mat_up * HD * HD, HD, HD, sm);
+    // the current values of the two gradients this CTA adds to are requested now and used after the products
+    constexpr int NI = HD / 64;
+    uint32_t pend_a[NI][4][8], pend_b[NI][4][8];
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        const size_t o = (size_t)c.row * HD + c.half * (HD / 2) + i * 32;
+        gload_f32x32_issue(p.ddy + (size_t)(mat_lo + 1) * HD * HD + o, pend_a[i], c.row < HD);
+        gload_f32x32_issue(p.ddy + (size_t)mat_lo * HD * HD + o, pend_b[i], c.row < HD);
+    }
     loads_wait(c);
     publish();
     if (c.tid == 0 && c.ok) {
@@ -370,8 +409,22 @@ __global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constan
     }
     mma_wait(c);
     if (c.ok) {
-        acc_add_global<false>(c, 0, HD, HD, p.ddy + (size_t)(mat_lo + 1) * HD * HD);
-        acc_add_global<false>(c, 128, HD, HD, p.ddy + (size_t)mat_lo * HD * HD);
+        float v[32], o[32];
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+            const int c0 = c.half * (HD / 2) + i * 32;
+            const size_t off = (size_t)c.row * HD + c0;
+            tmem_row32(c.tl + c0, v);
+            gload_f32x32_finish(pend_a[i], o);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) o[x] += v[x];
+            gstore_f32x32(p.ddy + (size_t)(mat_lo + 1) * HD * HD + off, o, c.row < HD);
+            tmem_row32(c.tl + 128 + c0, v);
+            gload_f32x32_finish(pend_b[i], o);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) o[x] += v[x];
+            gstore_f32x32(p.ddy + (size_t)mat_lo * HD * HD + off, o, c.row < HD);
+        }
     }
     teardown<256>(c, p.status);
 }

@@ -71,11 +71,10 @@ __device__ __forceinline__ void gstore_f32x32(float* dst, const float (&v)[32], 
         if (ok) st_global_v8((uint8_t*)ptr + 32 * j, d);
     }
 }
-__device__ __forceinline__ void gload_f32x32(const float* src, float (&v)[32], bool valid = true) {
+// The load in two halves, so that a caller can put other work between the request and the first use of the data.
+__device__ __forceinline__ void gload_f32x32_issue(const float* src, uint32_t (&d)[4][8], bool valid = true) {
     const int j = threadIdx.x & 3;
-    uint32_t w[32];
     const unsigned long long mine = (unsigned long long)src;
-    // all four loads are issued before any of their data is touched, so that they are in flight together
     unsigned long long ptr[4];
     bool ok[4];
 #pragma unroll
@@ -83,13 +82,16 @@ __device__ __forceinline__ void gload_f32x32(const float* src, float (&v)[32], b
         ptr[r] = r == 0 ? mine : __shfl_xor_sync(0xffffffffu, mine, r);
         ok[r] = r == 0 ? valid : (bool)__shfl_xor_sync(0xffffffffu, (int)valid, r);
     }
-    uint32_t d[4][8];
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
+    for (int r = 0; r < 4; ++r) {   // all four loads are in flight together
 #pragma unroll
         for (int x = 0; x < 8; ++x) d[r][x] = 0u;
         if (ok[r]) ld_global_v8((const uint8_t*)ptr[r] + 32 * j, d[r]);
     }
+}
+__device__ __forceinline__ void gload_f32x32_finish(const uint32_t (&d)[4][8], float (&v)[32]) {
+    const int j = threadIdx.x & 3;
+    uint32_t w[32];
 #pragma unroll
     for (int r = 0; r < 4; ++r)
 #pragma unroll
@@ -97,6 +99,11 @@ __device__ __forceinline__ void gload_f32x32(const float* src, float (&v)[32], b
     rot4_pieces(w, j);
 #pragma unroll
     for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(w[x]);
+}
+__device__ __forceinline__ void gload_f32x32(const float* src, float (&v)[32], bool valid = true) {
+    uint32_t d[4][8];
+    gload_f32x32_issue(src, d, valid);
+    gload_f32x32_finish(d, v);
 }
 // 32 bf16 = 64 bytes per row: pairs of lanes.
 __device__ __forceinline__ void gstore_bf16x32(__nv_bfloat16* dst, const float (&v)[32], bool valid = true) {
