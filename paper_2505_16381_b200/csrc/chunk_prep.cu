@@ -13,6 +13,7 @@
 // the descriptor's major-ness, so nothing is ever transposed in memory.  Accumulators live in tensor memory and
 // are read back one row per thread.  T~ is kept as a bf16 pair (hi + lo) because everything downstream
 // depends on it; the other intermediates are rounded to bf16 once, like the tiles the attention sweep consumes.
+#include <type_traits>
 #include "tileops.cuh"
 
 namespace path {
@@ -134,57 +135,66 @@ __global__ void __launch_bounds__(256, 1) chunk_prep_kernel(const __grid_constan
         }
     }
     __syncthreads();
-    for (int bi = 0; bi < kT / 16; ++bi) {
-        const int R = bi * 16;
-        const float* dx = diagX + bi * 16 * 17;
-        if (bi > 0) {
-            // Z = Nl[panel, <R] X[<R, <R]: each thread 4 rows x 1 column, 4 contraction steps per iteration
-            for (int idx = tid; idx < 4 * R; idx += 256) {
-                const int rg = idx / R, c = idx - rg * R;
-                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-                const float* n0 = Xb + (R + rg) * kLd;
-                for (int k = (c & ~15); k < R; k += 4) {
-                    const float x0 = Xb[k * kLd + c], x1 = Xb[(k + 1) * kLd + c], x2 = Xb[(k + 2) * kLd + c],
-                                x3 = Xb[(k + 3) * kLd + c];
-                    const float4 na = *reinterpret_cast<const float4*>(n0 + k);
-                    const float4 nb = *reinterpret_cast<const float4*>(n0 + 4 * kLd + k);
-                    const float4 nc = *reinterpret_cast<const float4*>(n0 + 8 * kLd + k);
-                    const float4 nd = *reinterpret_cast<const float4*>(n0 + 12 * kLd + k);
-                    a0 += na.x * x0 + na.y * x1 + na.z * x2 + na.w * x3;
-                    a1 += nb.x * x0 + nb.y * x1 + nb.z * x2 + nb.w * x3;
-                    a2 += nc.x * x0 + nc.y * x1 + nc.z * x2 + nc.w * x3;
-                    a3 += nd.x * x0 + nd.y * x1 + nd.z * x2 + nd.w * x3;
+    for (int bi = 0; bi < kT / 16; ++bi) {   // inverted diagonal blocks into place (their upper triangles are zero)
+        const int rr = tid >> 4, k = tid & 15;
+        Xb[(bi * 16 + rr) * kLd + bi * 16 + k] = diagX[bi * 16 * 17 + rr * 17 + k];
+    }
+    __syncthreads();
+    // Three merge levels on blocks of NB = 16, 32, 64 rows:  [[A,0],[C,B]]^-1 = [[A^-1,0],[-B^-1 C A^-1, B^-1]].
+    // Every level has 64 x NB entries of C blocks in total; each thread owns an (NB/16) x 4 tile of them.
+    // T = C A^-1 goes through the scratch area (the diagonal-block buffer is dead by now), M = -B^-1 T replaces C.
+    {
+        float* T = diagX;   // [64][64]
+        auto merge = [&](auto nb_tag) {
+            constexpr int NB = decltype(nb_tag)::value, RT = NB / 16;
+            const int pr = tid / (4 * NB), u = tid % (4 * NB);
+            const int i0 = (u / (NB / 4)) * RT, j0 = (u % (NB / 4)) * 4, base = pr * 2 * NB;
+            const float* Cp = Xb + (base + NB + i0) * kLd + base;          // rows i0.. of C
+            float acc[RT][4];
+#pragma unroll
+            for (int r_ = 0; r_ < RT; ++r_)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) acc[r_][x] = 0.f;
+            // T[i][j] = sum_{k >= j} C[i][k] A^-1[k][j]   (A^-1 is lower triangular: rows k < j0 contribute nothing)
+#pragma unroll 4
+            for (int k = j0; k < NB; ++k) {
+                const float4 a4 = *reinterpret_cast<const float4*>(Xb + (base + k) * kLd + base + j0);
+#pragma unroll
+                for (int r_ = 0; r_ < RT; ++r_) {
+                    const float ck = Cp[r_ * kLd + k];
+                    acc[r_][0] += ck * a4.x; acc[r_][1] += ck * a4.y; acc[r_][2] += ck * a4.z; acc[r_][3] += ck * a4.w;
                 }
-                Z[rg * kT + c] = a0; Z[(rg + 4) * kT + c] = a1; Z[(rg + 8) * kT + c] = a2; Z[(rg + 12) * kT + c] = a3;
             }
+#pragma unroll
+            for (int r_ = 0; r_ < RT; ++r_)
+                *reinterpret_cast<float4*>(T + (pr * NB + i0 + r_) * 64 + j0) =
+                    make_float4(acc[r_][0], acc[r_][1], acc[r_][2], acc[r_][3]);
             __syncthreads();
-            // X[panel, <R] = -X[panel, panel] Z: two threads per column (rows 0..10 and 11..15: equal work)
-            for (int idx = tid; idx < 2 * R; idx += 256) {
-                const int h = idx / R, c = idx - h * R;
-                float z[16];
+            // M[i][j] = -sum_{k <= i} B^-1[i][k] T[k][j]
 #pragma unroll
-                for (int k = 0; k < 16; ++k) z[k] = Z[k * kT + c];
-                if (h == 0) {
+            for (int r_ = 0; r_ < RT; ++r_)
 #pragma unroll
-                    for (int rr = 0; rr <= 10; ++rr) {
-                        float acc = 0.f;
+                for (int x = 0; x < 4; ++x) acc[r_][x] = 0.f;
+            const float* Bp = Xb + (base + NB + i0) * kLd + base + NB;     // rows i0.. of B^-1
+            const float* Tp = T + (pr * NB) * 64 + j0;
+#pragma unroll 4
+            for (int k = 0; k < i0 + RT; ++k) {                            // B^-1[i][k] = 0 for k > i
+                const float4 t4 = *reinterpret_cast<const float4*>(Tp + k * 64);
 #pragma unroll
-                        for (int k = 0; k <= rr; ++k) acc -= dx[rr * 17 + k] * z[k];
-                        Xb[(R + rr) * kLd + c] = acc;
-                    }
-                } else {
-#pragma unroll
-                    for (int rr = 11; rr < 16; ++rr) {
-                        float acc = 0.f;
-#pragma unroll
-                        for (int k = 0; k <= rr; ++k) acc -= dx[rr * 17 + k] * z[k];
-                        Xb[(R + rr) * kLd + c] = acc;
-                    }
+                for (int r_ = 0; r_ < RT; ++r_) {
+                    const float bk = Bp[r_ * kLd + k];
+                    acc[r_][0] -= bk * t4.x; acc[r_][1] -= bk * t4.y; acc[r_][2] -= bk * t4.z; acc[r_][3] -= bk * t4.w;
                 }
             }
-        }
-        { const int rr = tid >> 4, k = tid & 15; Xb[(R + rr) * kLd + R + k] = dx[rr * 17 + k]; }
-        __syncthreads();
+#pragma unroll
+            for (int r_ = 0; r_ < RT; ++r_)
+                *reinterpret_cast<float4*>(Xb + (base + NB + i0 + r_) * kLd + base + j0) =
+                    make_float4(acc[r_][0], acc[r_][1], acc[r_][2], acc[r_][3]);
+            __syncthreads();
+        };
+        merge(std::integral_constant<int, 16>{});
+        merge(std::integral_constant<int, 32>{});
+        merge(std::integral_constant<int, 64>{});
     }
 
     // ---- T~ = X D as a bf16 pair into the Q / K tiles' space (group 1 has finished with them)
