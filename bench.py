@@ -276,19 +276,52 @@ def run_ours(args, cfg):
     h2d = sum(host[n].numel() * host[n].element_size() for n in names)
     d2h = sum(t.numel() * t.element_size() for t in hout.values())
 
-    def e2e_step():
-        t = {n: host[n].to(dev, non_blocking=True) for n in names}
+    # Three streams (copy-in, compute, copy-out) and two sets of device buffers: every step still copies its inputs
+    # from pinned host memory and its results back inside the timed region, but the copies of neighbouring steps
+    # overlap the kernels, as an input pipeline would.
+    cur = torch.cuda.current_stream(dev)
+    s_in, s_cmp, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    din = [{n: torch.empty_like(devt[n]) for n in names} for _ in range(2)]
+    for t in din:
         t.setdefault("log_f", None)
-        step(t)
-        for n in hout:
-            hout[n].copy_(gout[n], non_blocking=True)
+    gouts = [gout, {n: torch.empty_like(v_) for n, v_ in gout.items()}]
+    ev = lambda: torch.cuda.Event()
+    in_ready, in_free, out_ready, out_free = ([ev(), ev()] for _ in range(4))
 
-    for _ in range(min(args.warmup, 3)):
-        e2e_step()
+    def e2e_run(nsteps):
+        for st in (s_in, s_cmp, s_out):
+            st.wait_stream(cur)
+        for i in range(nsteps):
+            b = i & 1
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(in_free[b])
+                for n in names:
+                    din[b][n].copy_(host[n], non_blocking=True)
+                in_ready[b].record(s_in)
+            with torch.cuda.stream(s_cmp):
+                s_cmp.wait_event(in_ready[b])
+                if i >= 2:
+                    s_cmp.wait_event(out_free[b])
+                t = din[b]
+                binding.path_attn_fwd(t["q"], t["k"], t["v"], t["w"], t["beta"], t["log_f"], scale=scale, workspace=ws,
+                                      out=(o, lse))
+                binding.path_attn_bwd(t["q"], t["k"], t["v"], t["w"], t["beta"], o, lse, t["d_o"], t["log_f"],
+                                      scale=scale, workspace=ws, out=gouts[b])
+                in_free[b].record(s_cmp)
+                out_ready[b].record(s_cmp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(out_ready[b])
+                for n in hout:
+                    hout[n].copy_(gouts[b][n], non_blocking=True)
+                out_free[b].record(s_out)
+        for st in (s_in, s_cmp, s_out):
+            cur.wait_stream(st)
+
+    e2e_run(min(args.warmup, 3))
     barrier()
     e0.record()
-    for _ in range(args.steps):
-        e2e_step()
+    e2e_run(args.steps)
     e1.record()
     barrier()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, dev)
