@@ -771,22 +771,25 @@ template <int HD>
 __global__ void rowstats_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                                 const float* __restrict__ lse, const float* __restrict__ G, float* __restrict__ delta,
                                 float* __restrict__ lse2, int L, int Lp) {
+    constexpr int TPR = HD / 8;                 // threads per row: 16 bytes (8 values) of o and of dO each
     const int s = blockIdx.y;
-    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (i >= Lp) return;
+    const int i = blockIdx.x * (256 / TPR) + threadIdx.x / TPR;
+    const int sub = threadIdx.x % TPR;
     float acc = 0.f;
     if (i < L) {
-        const size_t base = ((size_t)s * L + i) * HD;
-        for (int x = lane * 2; x < HD; x += 64) {
-            const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(o + base + x));
-            const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(d_o + base + x));
-            acc += a.x * b.x + a.y * b.y;
+        const size_t base = ((size_t)s * L + i) * HD + sub * 8;
+        const uint4 a = *reinterpret_cast<const uint4*>(o + base), b = *reinterpret_cast<const uint4*>(d_o + base);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[x]));
+            const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[x]));
+            acc += fa.x * fb.x + fa.y * fb.y;
         }
     }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-    if (lane == 0) {
+    for (int off = TPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (sub == 0 && i < Lp) {
         delta[(size_t)s * Lp + i] = -acc;
         float v = 0.f;
         if (i < L) v = ((G ? G[(size_t)s * Lp + i] : 0.f) - lse[(size_t)s * L + i]) * kLog2e;
@@ -838,7 +841,8 @@ cudaError_t launch_fa_bwd(const BwdTensorMaps& tm, const BwdParams& p, int hd, i
 
 cudaError_t launch_rowstats(const void* o, const void* d_o, const float* lse, const float* G, float* delta, float* lse2,
                             int S, int L, int Lp, int hd, cudaStream_t st) {
-    dim3 grid((Lp + 7) / 8, S);
+    const int rows_per_cta = 256 / (hd / 8);
+    dim3 grid((Lp + rows_per_cta - 1) / rows_per_cta, S);
     if (hd == 64)
         rowstats_kernel<64><<<grid, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, G, delta, lse2, L, Lp);
     else
