@@ -135,19 +135,18 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
 
     const float* g_dql = p.dql + (size_t)chunk * kT * HD;
     const float* g_dkr = p.dkr + (size_t)chunk * kT * HD;
-    const float* g_dsd = p.dsd + (size_t)chunk * kT * kT;
     const float* g_dp = p.dp + (size_t)chunk * HD * HD;
     const int r0 = chunk * kT;
 
     // slots: 0 U->W   1 dQl->dT->tmp->dGm   2 Y->Xq->Xk->T->Ah   3 dSd   4 dXq   5 dKr->dY->dXk   6 dP->dU->Al..K/Q
     // ---- phase 0a: dXq = lower(-(dQl U^T + s dSd Y^T))
     if (tid == 0) {
-        mbar_expect_tx(&bars[0], kT * HD * 2 + kTileB);
+        mbar_expect_tx(&bars[0], kT * HD * 2 + 2 * kTileB);
         tma_tile(slot(0), &tm.u, &bars[0], HD, r0);
         tma_tile(slot(2), &tm.y, &bars[0], kT, r0);
+        tma_tile(slot(3), &tm.dsdt, &bars[0], kT, r0);   // (s dSd)^T: every use below takes the transposed view
     }
     conv(g_dql, HD, kT, slot(1), 1.f);
-    conv(g_dsd, kT, kT, slot(3), p.scale);
     conv(g_dkr, HD, kT, slot(5), 1.f);
     conv(g_dp, HD, HD, slot(6), 1.f);
     loads_wait();
@@ -155,7 +154,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(1), OP_K, sa(0), OP_K, KD, 128, false);
-        mma_call(tmem + cA, sa(3), OP_K, sa(2), OP_K, K8, 128, true);
+        mma_call(tmem + cA, sa(3), OP_MN, sa(2), OP_K, K8, 128, true);
         // phase 0b: dw = -Y dKr - U dP^T
         mma_call(tmem + cDW, sa(2), OP_K, sa(5), OP_MN, K8, HD, false, true);
         mma_call(tmem + cDW, sa(0), OP_K, sa(6), OP_K, KD, HD, true, true);
@@ -175,7 +174,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(0), OP_K, sa(5), OP_K, KD, 128, false);
-        mma_call(tmem + cA, sa(2), OP_MN, sa(3), OP_MN, K8, 128, true);
+        mma_call(tmem + cA, sa(2), OP_MN, sa(3), OP_K, K8, 128, true);
         mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, HD, false);
         mma_call(tmem + cB, sa(0), OP_K, sa(6), OP_MN, KD, HD, true);
         mma_call(tmem + cG, sa(0), OP_K, sa(0), OP_K, KD, 128, false);
@@ -301,9 +300,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
-        mma_call(tmem + cB, sa(3), OP_K, sa(2), OP_MN, K8, HD, false);    // s dSd K
+        mma_call(tmem + cB, sa(3), OP_MN, sa(2), OP_MN, K8, HD, false);   // s dSd K
         mma_call(tmem + cB, sa(4), OP_K, sa(0), OP_MN, K8, HD, true);     // dXq W
-        mma_call(tmem + cG, sa(3), OP_MN, sa(6), OP_MN, K8, HD, false);   // s dSd^T Q
+        mma_call(tmem + cG, sa(3), OP_K, sa(6), OP_MN, K8, HD, false);    // s dSd^T Q
         mma_call(tmem + cG, sa(5), OP_MN, sa(0), OP_MN, K8, HD, true);    // dXk^T W
         mma_call(tmem + cDW, sa(4), OP_MN, sa(6), OP_MN, K8, HD, true);   // dXq^T Q
         mma_call(tmem + cDW, sa(5), OP_K, sa(2), OP_MN, K8, HD, true);    // dXk K

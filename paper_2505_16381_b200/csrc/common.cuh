@@ -106,12 +106,12 @@ cudaError_t launch_chunk_prep(const PrepTensorMaps& tm, const PrepParams& p, int
 struct ChainTensorMaps {
     CUtensorMap w, q, k, u;                       // [S*Lp][d]
     CUtensorMap y, xq, xk, th, tl, ah, al;        // [S*Lp][128]
+    CUtensorMap dsdt;                             // [S*N*128][128] bf16: (scale * lower(dS))^T of the diagonal chunks
 };
 
 struct ChainParams {
     const float* dql;     // [S*Lp][d]  gradient of the boundary-adjusted queries (version slot 0)
     const float* dkr;     // [S*Lp][d]  gradient of the boundary-adjusted keys
-    const float* dsd;     // [S*N][128][128] lower(dS) of the diagonal chunks (unscaled)
     const float* dp;      // [S*N][d][d] gradient of the chunk products
     const float* beta;    // [S*Lp]
     __nv_bfloat16 *dq, *dk, *dw;   // [S][L][d] outputs
@@ -131,7 +131,8 @@ struct BwdParams {
     float* dqv;          // [slots][S][Lp][d] gradients of the query versions (slot convention as the versions)
     float* dkv;          // same for the key versions
     void* dv;            // [S, L, d] bf16, final
-    float* dsd;          // [S*N][128 q][128 k] lower(dS) of the diagonal chunks (not yet multiplied by scale)
+    float* dsd;          // [S*N][128 q][128 k] lower(dS) of the diagonal chunks, unscaled; written for gated problems only
+    __nv_bfloat16* dsdt; // [S*N][128 k][128 q] (scale * lower(dS))^T in bf16: the chain rule's operand
     float* dG;           // [S][Lp] minus the column sums of dS (gated problems only)
     float* dGrow;        // [S][Lp] row sums of dS over the off-diagonal chunks (gated problems only)
     const float* lse2;   // [S][Lp] (gate prefix - lse) * log2(e)

@@ -373,6 +373,7 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
             tc_fence_after_sync();
             // dP^T ready means every product issued before it has retired: dK of a finished level can be flushed
             if (!FIRST && ok && t >= 2 && level(t) != level(t - 1)) flush_dk(level(t - 1));
+            uint32_t dsw[FIRST ? 32 : 1];   // this thread's 64 entries of the transposed diagonal tile
             if (ok) {
                 const float* dl_ = st_ + kTile;
 #pragma unroll
@@ -393,13 +394,17 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
                         if (GATE) dsum += (d[0] + d[1]) + (d[2] + d[3]);
                         pk[x >> 1] = pack_bf16(d[0], d[1]);
                         pk[(x >> 1) + 1] = pack_bf16(d[2], d[3]);
-                        if (FIRST) {
+                        if (FIRST) {   // (scale * dS)^T of the diagonal chunk for the chain rule; unscaled float copy if gated
+                            dsw[c * 16 + (x >> 1)] = pack_bf16(d[0] * p.scale, d[1] * p.scale);
+                            dsw[c * 16 + (x >> 1) + 1] = pack_bf16(d[2] * p.scale, d[3] * p.scale);
+                            if (GATE) {
 #pragma unroll
-                            for (int y = 0; y < 4; ++y) dp[x + y] = __float_as_uint(d[y]);
+                                for (int y = 0; y < 4; ++y) dp[x + y] = __float_as_uint(d[y]);
+                            }
                         }
                     }
                     tmem_st16(tlane + colDP + c0 + c * 16, pk);
-                    if (FIRST) {
+                    if (FIRST && GATE) {
                         float* dsd = p.dsd + ((size_t)(s * p.N + J) * kTile) * kTile;
 #pragma unroll
                         for (int x = 0; x < 32; ++x) dsd[(size_t)(c0 + c * 32 + x) * kTile + row] = __uint_as_float(dp[x]);
@@ -410,6 +415,11 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
             tc_fence_before_sync();
             mbar_arrive(&bars[K_DSFULL]);
             mbar_arrive(&bars[K_STEMPTY + (gs & 1)]);
+            if constexpr (FIRST) {   // rows = keys (this warp's 32 lanes), 64 query columns = 128 bytes per row
+                if (ok)
+                    warp_store_rows128(p.dsdt + ((size_t)(s * p.N + J) * kTile + q4 * 32) * kTile + h * 64, (size_t)kTile * 2,
+                                       dsw);
+            }
         };
 #pragma unroll 1
         for (int it = 0; item_of(it, J, s); ++it) {

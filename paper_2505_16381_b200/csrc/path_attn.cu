@@ -120,7 +120,7 @@ struct Plan {
     // offsets (bytes)
     size_t status, qp, kp, vp, wp, betap, G, Dyh, Dyl, Xqn, Yt, Qv16, Kv16;
     // backward only
-    size_t dop, delta, lse2, dQv, dKv, dSd, dG, dGrow, dGdiag, dDy;
+    size_t dop, delta, lse2, dQv, dKv, dSd, dSdT, dG, dGrow, dGdiag, dDy;
     size_t sTh, sTl, sAh, sAl, sXq, sXk, sY, sU;   // bf16 tiles kept by the chunk preparation for the chain rule
     size_t dy_bytes, dy_mats;
 };
@@ -173,7 +173,7 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
         if (p.ragged) p.dop = bump(cur, SLd * 2);
         p.delta = bump(cur, SL * 4); p.lse2 = bump(cur, SL * 4);
         p.dQv = bump(cur, SLd * 4 * p.nslot); p.dKv = bump(cur, SLd * 4 * p.nslot);
-        p.dSd = bump(cur, SNBB * 4); p.dG = bump(cur, SL * 4);
+        p.dSd = bump(cur, gate ? SNBB * 4 : 0); p.dSdT = bump(cur, SNBB * 2); p.dG = bump(cur, SL * 4);
         p.dGrow = bump(cur, gate ? SL * 4 : 0); p.dGdiag = bump(cur, gate ? SL * 4 : 0);
         p.dDy = bump(cur, dy_elems * 4);
     }
@@ -289,11 +289,12 @@ static int run_chunk_chain(const Plan& p, void* ws, const void* q, const void* k
               make_map(&tm.u, at<void>(ws, p.sU), rows, d) && make_map(&tm.y, at<void>(ws, p.sY), rows, CHUNK) &&
               make_map(&tm.xq, at<void>(ws, p.sXq), rows, CHUNK) && make_map(&tm.xk, at<void>(ws, p.sXk), rows, CHUNK) &&
               make_map(&tm.th, at<void>(ws, p.sTh), rows, CHUNK) && make_map(&tm.tl, at<void>(ws, p.sTl), rows, CHUNK) &&
-              make_map(&tm.ah, at<void>(ws, p.sAh), rows, CHUNK) && make_map(&tm.al, at<void>(ws, p.sAl), rows, CHUNK);
+              make_map(&tm.ah, at<void>(ws, p.sAh), rows, CHUNK) && make_map(&tm.al, at<void>(ws, p.sAl), rows, CHUNK) &&
+              make_map(&tm.dsdt, at<void>(ws, p.dSdT), (uint64_t)p.S * p.N * CHUNK, CHUNK);
     if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
     ChainParams cp{};
     cp.dql = at<float>(ws, p.dQv); cp.dkr = at<float>(ws, p.dKv);   // slot 0 of the version gradients
-    cp.dsd = at<float>(ws, p.dSd); cp.dp = at<float>(ws, p.dDy);    // level 0 of the run-product gradients
+    cp.dp = at<float>(ws, p.dDy);                                   // level 0 of the run-product gradients
     cp.beta = at<float>(ws, p.betap);
     cp.dq = (__nv_bfloat16*)dq; cp.dk = (__nv_bfloat16*)dk; cp.dw = (__nv_bfloat16*)dw; cp.dbeta = dbeta;
     cp.status = at<uint32_t>(ws, p.status);
@@ -329,7 +330,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
               make_map(&tm.d_o, dop, rows, d);
     if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
     BwdParams bp{};
-    bp.dqv = dQv; bp.dkv = dKv; bp.dv = dv; bp.dsd = at<float>(ws, p.dSd); bp.dG = at<float>(ws, p.dG); bp.dGrow = at<float>(ws, p.dGrow);
+    bp.dqv = dQv; bp.dkv = dKv; bp.dv = dv; bp.dsd = p.gate ? at<float>(ws, p.dSd) : nullptr; bp.dsdt = at<__nv_bfloat16>(ws, p.dSdT); bp.dG = at<float>(ws, p.dG); bp.dGrow = at<float>(ws, p.dGrow);
     bp.lse2 = at<float>(ws, p.lse2); bp.delta = at<float>(ws, p.delta);
     bp.G = p.gate ? at<float>(ws, p.G) : nullptr;
     bp.status = at<uint32_t>(ws, p.status);
