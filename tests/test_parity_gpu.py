@@ -97,6 +97,18 @@ def test_small_shapes_match_oracle(binding, oracle, B, H, L, d, gate, sharp):
     compare_all(binding, oracle, inp)
 
 
+@pytest.mark.parametrize("B,H,L,d,gate", [
+    (3, 1, 2176, 64, True),      # 17 chunks x 3 slices: odd item counts, pairs that straddle slices
+    (1, 1, 4224, 128, False),    # 33 chunks: six dyadic levels, one slice on a grid of 17 persistent CTAs
+    (5, 1, 256, 64, False),      # 2 chunks x 5 slices
+    (1, 7, 384, 128, True),      # 3 chunks x 7 slices
+])
+def test_persistent_scheduling_shapes(binding, oracle, B, H, L, d, gate):
+    """Shapes whose work-item lists do not divide evenly over the persistent CTAs of the sweeps."""
+    inp = synth.make_inputs(B, H, L, d, "bf16", gate=gate, seed=700 + L)
+    compare_all(binding, oracle, inp)
+
+
 def test_c1_workload_shape_and_distribution_in_bf16(binding, oracle):
     """Workload C1 (B=1, H=2, L=256, d=64, q, k, v ~ N(0,1) unscaled: logits of standard deviation 8) with bf16 I/O.
     The float32 I/O dtype of C1 itself is not built (PATH_FP32 is rejected with PATH_ERR_DTYPE)."""
