@@ -42,11 +42,11 @@ UNIT = "TFLOP/s"
 # DRAM bytes per launch PER (batch, head) SLICE at the C3 shape (L=4096, d=128), from the ncu captures at batch 1
 # (16 slices) summarised under profiles/; slices are independent, so a launch over S slices moves S times this.
 NCU_TRAFFIC_BYTES_PER_SLICE = {
-    "chunk_prep": (52.00e6 + 181.54e6) / 16,        # backward instance (the step's forward runs on the shared workspace)
-    "fa_fwd": (168.36e6 + 8.04e6) / 16,
-    "fa_bwd_dkv": (187.07e6 + 100.26e6) / 16,
-    "fa_bwd_dq": (117.71e6 + 47.99e6) / 16,
-    "bwd_chunk_chain": (339.18e6 + 37.59e6) / 16,
+    "chunk_prep": (52.02e6 + 181.98e6) / 16,        # backward instance (the step's forward runs on the shared workspace)
+    "fa_fwd": (168.41e6 + 8.34e6) / 16,
+    "fa_bwd_dkv": (187.31e6 + 92.84e6) / 16,
+    "fa_bwd_dq": (117.70e6 + 47.64e6) / 16,
+    "bwd_chunk_chain": (315.35e6 + 34.60e6) / 16,
 }
 
 
