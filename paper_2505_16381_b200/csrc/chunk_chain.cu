@@ -162,13 +162,15 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     mma_wait();
     if (!ok) goto done;
-    acc_to_tile(cA, kT, slot(4), -1.f, M_LOWER);                    // dXq
     // ---- phase 1: dY = -(W dKr^T + Xq^T s dSd),  dU = -(Xq^T dQl + W dP),  Gm = W W^T
+    // (every group's tiles are requested as soon as the products that read the slots have retired, before the
+    // read-out of the accumulators, so that the TMA latency hides behind it)
     if (tid == 0) {
         mbar_expect_tx(&bars[0], kT * HD * 2 + kTileB);
         tma_tile(slot(0), &tm.w, &bars[0], HD, r0);
         tma_tile(slot(2), &tm.xq, &bars[0], kT, r0);
     }
+    acc_to_tile(cA, kT, slot(4), -1.f, M_LOWER);                    // dXq
     loads_wait();
     publish();
     if (tid == 0) {
@@ -182,13 +184,13 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     mma_wait();
     if (!ok) goto done;
-    acc_to_tile(cA, kT, slot(5), -1.f, M_NONE);                     // dY (over dKr)
-    acc_to_tile(cB, HD, slot(6), -1.f, M_NONE);                     // dU (over dP)
     // ---- phase 2: dT = lower(dY Xk^T + dU W^T)
     if (tid == 0) {
         mbar_expect_tx(&bars[0], kTileB);
         tma_tile(slot(2), &tm.xk, &bars[0], kT, r0);
     }
+    acc_to_tile(cA, kT, slot(5), -1.f, M_NONE);                     // dY (over dKr)
+    acc_to_tile(cB, HD, slot(6), -1.f, M_NONE);                     // dU (over dP)
     loads_wait();
     publish();
     if (tid == 0) {
@@ -199,13 +201,17 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     mma_wait();
     if (!ok) goto done;
+    // ---- phase 3: dXk = strictLower(T~^T dY) -> cB,  dw += T~^T dU   (hi, then lo through the same slot)
+    if (tid == 0) {
+        mbar_expect_tx(&bars[0], kTileB);
+        tma_tile(slot(2), &tm.th, &bars[0], kT, r0);
+    }
     // dT stays in tensor memory (cA); its bf16 hi part goes to slot 1 now, the lo part follows in phase 4
     split_to_tile(cA, slot(1), false, f_dT);
-    // ---- phase 3: dXk = strictLower(T~^T dY) -> cB,  dw += T~^T dU   (hi, then lo through the same slot)
     for (int part = 0; part < 2; ++part) {
-        if (tid == 0) {
+        if (tid == 0 && part == 1) {
             mbar_expect_tx(&bars[0], kTileB);
-            tma_tile(slot(2), part == 0 ? &tm.th : &tm.tl, &bars[0], kT, r0);
+            tma_tile(slot(2), &tm.tl, &bars[0], kT, r0);
         }
         loads_wait();
         publish();
@@ -272,6 +278,11 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     mma_wait();
     if (!ok) goto done;
+    if (tid == 0) {   // phase 5's K and Q replace Ainv hi / lo, whose last products have just retired
+        mbar_expect_tx(&bars[0], 2 * kT * HD * 2);
+        tma_tile(slot(2), &tm.k, &bars[0], HD, r0);
+        tma_tile(slot(6), &tm.q, &bars[0], HD, r0);
+    }
     {   // dA = strictLower(-cA);  dbeta_r = t1_r + sum_c dA_rc Gm_rc
         float part = 0.f;
         for (int c = 0; c < 2; ++c) {
@@ -291,11 +302,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     split_to_tile(cA, slot(1), false, f_dGm);                       // dGm = D dA, hi
     // ---- phase 5: dq -> cB, dk -> cG and the rest of dw
-    if (tid == 0) {
-        mbar_expect_tx(&bars[0], 2 * kT * HD * 2);
-        tma_tile(slot(2), &tm.k, &bars[0], HD, r0);
-        tma_tile(slot(6), &tm.q, &bars[0], HD, r0);
-    }
     loads_wait();
     publish();
     if (tid == 0) {
