@@ -105,12 +105,9 @@ __device__ __forceinline__ void gload_f32x32(const float* src, float (&v)[32], b
     gload_f32x32_issue(src, d, valid);
     gload_f32x32_finish(d, v);
 }
-// 32 bf16 = 64 bytes per row: pairs of lanes.
-__device__ __forceinline__ void gstore_bf16x32(__nv_bfloat16* dst, const float (&v)[32], bool valid = true) {
+// 32 bf16 = 64 bytes per row: pairs of lanes.  `w`: the row segment as 16 packed words.
+__device__ __forceinline__ void gstore_bf16_w16(__nv_bfloat16* dst, const uint32_t (&w)[16], bool valid = true) {
     const bool odd = threadIdx.x & 1;
-    uint32_t w[16];
-#pragma unroll
-    for (int x = 0; x < 16; ++x) w[x] = pack_bf16(v[2 * x], v[2 * x + 1]);
     uint32_t first[8], second[8];   // halves [32 * odd, +32) of the even lane's row and of the odd lane's row
 #pragma unroll
     for (int x = 0; x < 8; ++x) {
@@ -122,6 +119,33 @@ __device__ __forceinline__ void gstore_bf16x32(__nv_bfloat16* dst, const float (
     const bool ovalid = (bool)__shfl_xor_sync(0xffffffffu, (int)valid, 1);
     if (odd ? ovalid : valid) st_global_v8((uint8_t*)(odd ? other : mine) + 32 * (int)odd, first);
     if (odd ? valid : ovalid) st_global_v8((uint8_t*)(odd ? mine : other) + 32 * (int)odd, second);
+}
+__device__ __forceinline__ void pack32(const float (&v)[32], uint32_t (&w)[16]) {
+#pragma unroll
+    for (int x = 0; x < 16; ++x) w[x] = pack_bf16(v[2 * x], v[2 * x + 1]);
+}
+__device__ __forceinline__ void gstore_bf16x32(__nv_bfloat16* dst, const float (&v)[32], bool valid = true) {
+    uint32_t w[16];
+    pack32(v, w);
+    gstore_bf16_w16(dst, w, valid);
+}
+// t = hi + lo with hi = bf16(t) and lo = bf16(t - hi), both packed two per word.
+__device__ __forceinline__ void split32(const float (&t)[32], uint32_t (&hi)[16], uint32_t (&lo)[16]) {
+#pragma unroll
+    for (int x = 0; x < 16; ++x) {
+        const uint32_t h = pack_bf16(t[2 * x], t[2 * x + 1]);
+        hi[x] = h;
+        lo[x] = pack_bf16(t[2 * x] - __uint_as_float(h << 16), t[2 * x + 1] - __uint_as_float(h & 0xffff0000u));
+    }
+}
+// Packed counterpart of tile_store32.
+__device__ __forceinline__ void tile_store_w16(uint8_t* t, int row, int c0, const uint32_t (&w)[16]) {
+    uint8_t* panel = t + (c0 >> 6) * kPanelB;
+    const int ch0 = (c0 & 63) >> 3;
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch)
+        *reinterpret_cast<uint4*>(panel + sw128_off((uint32_t)row, (uint32_t)(ch0 + ch))) =
+            make_uint4(w[4 * ch], w[4 * ch + 1], w[4 * ch + 2], w[4 * ch + 3]);
 }
 __device__ __forceinline__ void gload_bf16x32(const __nv_bfloat16* src, float (&v)[32]) {
 #pragma unroll
