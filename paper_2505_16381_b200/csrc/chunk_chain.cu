@@ -8,9 +8,10 @@
 //   dbeta_r += sum_c dA_rc (W W^T)_rc,           dGm = D dA
 //   dq = dQl + s dSd K + dXq W                   dk = dKr + s dSd^T Q + dXk^T W
 //   dw = -Y dKr - U dP^T + T~^T dU + dXq^T Q + dXk K + (dGm + dGm^T) W
-// One CTA per chunk runs these ~25 products as tcgen05 MMAs on swizzled shared-memory tiles, in lockstep:
-// thread 0 loads tiles (TMA) and issues MMAs, all 256 threads convert float gradients into tiles and turn
-// accumulators (tensor memory, one row per thread) into the next operand tiles.  T~ and Ainv enter as bf16
+// A persistent CTA (one per SM) walks over chunks and runs these ~25 products per chunk as tcgen05 MMAs on swizzled
+// shared-memory tiles, in lockstep: thread 0 loads tiles (TMA) and issues MMAs, all 256 threads turn accumulators
+// (tensor memory, one row per thread) into the next operand tiles.  dQl and dKr arrive as bf16 tiles; the next
+// chunk's first tiles are requested before the current chunk's results are written out.  T~ and Ainv enter as bf16
 // hi + lo pairs, and so do the in-kernel intermediates dT, M D and dGm (the lo tile follows the hi tile through
 // the same slot); everything else is rounded to bf16 once.  dw accumulates in tensor memory across all phases.
 #include "tileops.cuh"
@@ -33,7 +34,7 @@ constexpr uint32_t kChainSmem = kBarOff + 64 + kT * 4 + kT * 4 + 1024;
 
 template <int HD>
 __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_constant__ ChainTensorMaps tm,
-                                                             const ChainParams p) {
+                                                             const ChainParams p, const int nchunks) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = (uint64_t*)(smem + kBarOff);  // [0] loads, [1] MMA groups
@@ -43,11 +44,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     float* t1 = bt + kT;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int chunk = blockIdx.x;
     const int row = (warp & 3) * 32 + lane, half = warp >> 2;
-    const int s_idx = chunk / p.N, pos = (chunk % p.N) * kT + row;   // slice and position of this thread's row
-    const bool row_valid = pos < p.L;
-    const size_t urow = (size_t)s_idx * p.L + pos;                   // row in the caller's [S][L][.] tensors
 
     if (tid == 0) {
         mbar_init(&bars[0], 1);
@@ -56,7 +53,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(tmem_slot, 512);
-    if (tid < kT) bt[tid] = p.beta[(size_t)chunk * kT + tid];
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -88,14 +84,12 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         ok = __syncthreads_and(ok);
         tc_fence_after_sync();
     };
-    // float rows of a [128][ncols] global matrix -> bf16 tile (optionally scaled)
-    auto conv = [&](const float* src, int ncols, int nrows, uint8_t* dst, float mul) {
+    // float rows of a [nrows][ncols] global matrix -> bf16 tile (rows >= nrows read as zero)
+    auto conv = [&](const float* src, int ncols, int nrows, uint8_t* dst) {
         const int per = ncols / 2;
         for (int c = 0; c < per / 32; ++c) {
             const int c0 = half * per + c * 32;
             gload_f32x32(src + (size_t)row * ncols + c0, v, row < nrows);
-#pragma unroll
-            for (int x = 0; x < 32; ++x) v[x] *= mul;
             tile_store32(dst, row, c0, v);
         }
     };
@@ -133,22 +127,30 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     auto f_tmp = [&](float x, int col) { return x * bt[col]; };
     auto f_dGm = [&](float x, int col) { return col < row ? -bt[row] * x : 0.f; };
 
-    const float* g_dql = p.dql + (size_t)chunk * kT * HD;
-    const float* g_dkr = p.dkr + (size_t)chunk * kT * HD;
+    // slots: 0 U->W   1 dQl->dT->tmp->dGm   2 Y->Xq->Xk->T->Ah   3 dSd   4 dXq   5 dKr->dY->dXk   6 dP->dU->Al..K/Q
+    // first tiles of a chunk: U, Y, (s dSd)^T (every use below takes the transposed view), dQl, dKr
+    auto first_loads = [&](int ch) {
+        mbar_expect_tx(&bars[0], 3 * kT * HD * 2 + 2 * kTileB);
+        tma_tile(slot(0), &tm.u, &bars[0], HD, ch * kT);
+        tma_tile(slot(2), &tm.y, &bars[0], kT, ch * kT);
+        tma_tile(slot(3), &tm.dsdt, &bars[0], kT, ch * kT);
+        tma_tile(slot(1), &tm.dql, &bars[0], HD, ch * kT);
+        tma_tile(slot(5), &tm.dkr, &bars[0], HD, ch * kT);
+    };
+    if (tid == 0 && (int)blockIdx.x < nchunks) first_loads(blockIdx.x);
+
+#pragma unroll 1
+    for (int chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+    const int s_idx = chunk / p.N, pos = (chunk % p.N) * kT + row;   // slice and position of this thread's row
+    const bool row_valid = pos < p.L;
+    const size_t urow = (size_t)s_idx * p.L + pos;                   // row in the caller's [S][L][.] tensors
+    const __nv_bfloat16* g_dql = p.dql + ((size_t)chunk * kT + row) * HD;
+    const __nv_bfloat16* g_dkr = p.dkr + ((size_t)chunk * kT + row) * HD;
     const float* g_dp = p.dp + (size_t)chunk * HD * HD;
     const int r0 = chunk * kT;
-
-    // slots: 0 U->W   1 dQl->dT->tmp->dGm   2 Y->Xq->Xk->T->Ah   3 dSd   4 dXq   5 dKr->dY->dXk   6 dP->dU->Al..K/Q
+    if (tid < kT) bt[tid] = p.beta[(size_t)chunk * kT + tid];   // first read after several barriers (phase 4)
     // ---- phase 0a: dXq = lower(-(dQl U^T + s dSd Y^T))
-    if (tid == 0) {
-        mbar_expect_tx(&bars[0], kT * HD * 2 + 2 * kTileB);
-        tma_tile(slot(0), &tm.u, &bars[0], HD, r0);
-        tma_tile(slot(2), &tm.y, &bars[0], kT, r0);
-        tma_tile(slot(3), &tm.dsdt, &bars[0], kT, r0);   // (s dSd)^T: every use below takes the transposed view
-    }
-    conv(g_dql, HD, kT, slot(1), 1.f);
-    conv(g_dkr, HD, kT, slot(5), 1.f);
-    conv(g_dp, HD, HD, slot(6), 1.f);
+    conv(g_dp, HD, HD, slot(6));
     loads_wait();
     publish();
     if (tid == 0) {
@@ -161,7 +163,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    if (!ok) goto done;
+    if (!ok) break;
     // ---- phase 1: dY = -(W dKr^T + Xq^T s dSd),  dU = -(Xq^T dQl + W dP),  Gm = W W^T
     // (every group's tiles are requested as soon as the products that read the slots have retired, before the
     // read-out of the accumulators, so that the TMA latency hides behind it)
@@ -183,7 +185,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    if (!ok) goto done;
+    if (!ok) break;
     // ---- phase 2: dT = lower(dY Xk^T + dU W^T)
     if (tid == 0) {
         mbar_expect_tx(&bars[0], kTileB);
@@ -200,7 +202,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    if (!ok) goto done;
+    if (!ok) break;
     // ---- phase 3: dXk = strictLower(T~^T dY) -> cB,  dw += T~^T dU   (hi, then lo through the same slot)
     if (tid == 0) {
         mbar_expect_tx(&bars[0], kTileB);
@@ -222,8 +224,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
             umma_commit(&bars[1]);
         }
         mma_wait();
-        if (!ok) goto done;
+        if (!ok) break;
     }
+    if (!ok) break;
     // ---- phase 4: M = Ainv^T dT -> cB;  dbeta_c = M_cc;  tmp = M D;  dA = strictLower(-tmp Ainv^T) -> cA
     if (tid == 0) {
         mbar_expect_tx(&bars[0], 2 * kTileB);
@@ -240,7 +243,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    if (!ok) goto done;
+    if (!ok) break;
     split_to_tile(cA, slot(1), true, f_dT);                         // dT lo
     publish();
     if (tid == 0) {
@@ -249,7 +252,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    if (!ok) goto done;
+    if (!ok) break;
     {   // diagonal of M -> t1
         const int c0 = (row >> 5) << 5;
         if ((c0 >> 6) == half) {
@@ -268,7 +271,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    if (!ok) goto done;
+    if (!ok) break;
     split_to_tile(cB, slot(1), true, f_tmp);                        // tmp lo
     publish();
     if (tid == 0) {
@@ -277,7 +280,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    if (!ok) goto done;
+    if (!ok) break;
     if (tid == 0) {   // phase 5's K and Q replace Ainv hi / lo, whose last products have just retired
         mbar_expect_tx(&bars[0], 2 * kT * HD * 2);
         tma_tile(slot(2), &tm.k, &bars[0], HD, r0);
@@ -317,7 +320,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    if (!ok) goto done;
+    if (!ok) break;
     split_to_tile(cA, slot(1), true, f_dGm);                        // dGm lo
     publish();
     if (tid == 0) {
@@ -326,26 +329,44 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         mma_call(tmem + cDW, sa(1), OP_MN, sa(0), OP_MN, K8, HD, true);
         umma_commit(&bars[1]);
     }
+    // the dQl / dKr rows of the final sums are fetched while the last products run
+    uint4 pre_q[HD / 64][4], pre_k[HD / 64][4];
+#pragma unroll
+    for (int c = 0; c < HD / 64; ++c) {
+        const int c0 = half * (HD / 2) + c * 32;
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            pre_q[c][x] = reinterpret_cast<const uint4*>(g_dql + c0)[x];
+            pre_k[c][x] = reinterpret_cast<const uint4*>(g_dkr + c0)[x];
+        }
+    }
     mma_wait();
-    if (!ok) goto done;
+    if (!ok) break;
+    // every product of this chunk has retired: all tile slots are free for the next chunk's first tiles
+    if (tid == 0 && chunk + (int)gridDim.x < nchunks) first_loads(chunk + gridDim.x);
+#pragma unroll
     for (int c = 0; c < HD / 64; ++c) {
         const int c0 = half * (HD / 2) + c * 32;
         float in[32];
         tmem_row32(tl + cB + c0, v);
-        gload_f32x32(g_dql + (size_t)row * HD + c0, in);
+        unpack_bf16x32(pre_q[c], in);
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] += in[x];
         gstore_bf16x32(p.dq + urow * HD + c0, v, row_valid);
         tmem_row32(tl + cG + c0, v);
-        gload_f32x32(g_dkr + (size_t)row * HD + c0, in);
+        unpack_bf16x32(pre_k[c], in);
 #pragma unroll
         for (int x = 0; x < 32; ++x) v[x] += in[x];
         gstore_bf16x32(p.dk + urow * HD + c0, v, row_valid);
         tmem_row32(tl + cDW + c0, v);
         gstore_bf16x32(p.dw + urow * HD + c0, v, row_valid);
     }
+    // the next chunk's first products overwrite the accumulators read above
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    }   // chunk loop
 
-done:
     tc_fence_before_sync();
     __syncthreads();
     if (tid == 0 && *abort_flag != 0) atomicCAS(p.status, 0u, *abort_flag);
@@ -358,10 +379,16 @@ done:
 }  // namespace
 
 cudaError_t launch_chunk_chain(const ChainTensorMaps& tm, const ChainParams& p, int hd, int nchunks, cudaStream_t st) {
+    int dev = 0, sms = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 != cudaSuccess) return e0;
+    e0 = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e0 != cudaSuccess) return e0;
+    const int grid = nchunks < sms ? nchunks : sms;
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kChainSmem);
         if (e != cudaSuccess) return e;
-        kern<<<nchunks, 256, kChainSmem, st>>>(tm, p);
+        kern<<<grid, 256, kChainSmem, st>>>(tm, p, nchunks);
         return cudaGetLastError();
     };
     return hd == 64 ? go(chunk_chain_kernel<64>) : go(chunk_chain_kernel<128>);

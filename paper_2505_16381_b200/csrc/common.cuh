@@ -75,6 +75,7 @@ struct LevelParams {
     int S, N, Lp;
     __nv_bfloat16 *dyh, *dyl, *qv, *kv;
     float *dqv, *dkv, *ddy;
+    __nv_bfloat16 *dq16, *dk16;   // [S*Lp][d] final gradients of the slot-0 versions, rounded once (the chain rule's operands)
     uint32_t* status;
 };
 
@@ -107,11 +108,12 @@ struct ChainTensorMaps {
     CUtensorMap w, q, k, u;                       // [S*Lp][d]
     CUtensorMap y, xq, xk, th, tl, ah, al;        // [S*Lp][128]
     CUtensorMap dsdt;                             // [S*N*128][128] bf16: (scale * lower(dS))^T of the diagonal chunks
+    CUtensorMap dql, dkr;                         // [S*Lp][d] bf16 gradients of the boundary-adjusted queries / keys
 };
 
 struct ChainParams {
-    const float* dql;     // [S*Lp][d]  gradient of the boundary-adjusted queries (version slot 0)
-    const float* dkr;     // [S*Lp][d]  gradient of the boundary-adjusted keys
+    const __nv_bfloat16* dql;   // [S*Lp][d]  gradient of the boundary-adjusted queries (version slot 0), bf16
+    const __nv_bfloat16* dkr;   // [S*Lp][d]  gradient of the boundary-adjusted keys, bf16
     const float* dp;      // [S*N][d][d] gradient of the chunk products
     const float* beta;    // [S*Lp]
     __nv_bfloat16 *dq, *dk, *dw;   // [S][L][d] outputs

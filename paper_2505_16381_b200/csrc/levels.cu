@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(256, 2) version_fwd_kernel(const __grid_consta
 // g = dXv[l2][chunk] (what the sweeps wrote there plus what arrived from the level above, which stays in tensor memory):
 //     dXv[l1][chunk] += g Dy^T (queries) or g Dy (keys);
 //     dDy[l1][b]     += Xv[l1]^T g (queries) or g^T Xv[l1] (keys), atomically.
-// Only the bottom of the chain is added back to global memory.  The next step's operands are fetched while the
+// Only the bottom of the chain (always slot 0) leaves the CTA: as the bf16 tile the chunk chain rule loads.  The next step's operands are fetched while the
 // current one runs.
 template <int HD>
 __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
@@ -252,11 +252,29 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
         return 0;
     };
     int l2 = next_step(p.l - 1);
-    if (l2 == 0) return;
+    float* dxv = is_key ? p.dkv : p.dqv;
+    __nv_bfloat16* dx16 = (is_key ? p.dk16 : p.dq16) + ((size_t)s * p.Lp + (size_t)ch * kT) * HD;   // this chunk's rows
+    if (l2 == 0) {   // no chain: what the sweeps left in slot 0 is final
+        const float* src = dxv + ((size_t)s * p.Lp + (size_t)ch * kT) * HD;
+        constexpr int NIT = kT * HD / (256 * 8);   // every load of the thread is in flight before the first store
+        float4 a[NIT], b4[NIT];
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int i = (it * 256 + threadIdx.x) * 8;
+            a[it] = *reinterpret_cast<const float4*>(src + i);
+            b4[it] = *reinterpret_cast<const float4*>(src + i + 4);
+        }
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int i = (it * 256 + threadIdx.x) * 8;
+            *reinterpret_cast<uint4*>(dx16 + i) = make_uint4(pack_bf16(a[it].x, a[it].y), pack_bf16(a[it].z, a[it].w),
+                                                             pack_bf16(b4[it].x, b4[it].y), pack_bf16(b4[it].z, b4[it].w));
+        }
+        return;
+    }
     extern __shared__ uint8_t smem_raw[];
     Ctx c;
     setup<256>(c, smem_raw, 7 * kTileB);
-    float* dxv = is_key ? p.dkv : p.dqv;
     uint8_t* sm = c.smem;   // slot 0: g; two buffers of three slots: Dy hi, Dy lo, Xv[l1]
     auto issue_loads = [&](int buf) {   // operands of the step described by (l1, b, src)
         const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
@@ -270,7 +288,6 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
     if (c.tid == 0) issue_loads(0);
     int buf = 0;
     bool have_acc = false;
-    long row_low = 0;   // rows of the level the accumulated contribution belongs to
     // The gradient stored in global memory at the level a step consumes is requested one step ahead (the first one
     // here), so that its latency hides behind the previous step's products and atomics.
     constexpr int NI = HD / 64;
@@ -348,7 +365,6 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
             __syncthreads();   // the staging area is the buffer the prefetch after next will fill
         }
         have_acc = true;
-        row_low = row_src;
         l2 = l2n;
         buf ^= 1;
     }
@@ -361,7 +377,7 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
             tmem_row32(c.tl + c0, a);
 #pragma unroll
             for (int x = 0; x < 32; ++x) v[x] += a[x];
-            gstore_f32x32(dxv + ((size_t)row_low + c.row) * HD + c0, v);
+            gstore_bf16x32(dx16 + (size_t)c.row * HD + c0, v);   // the chain's bottom is always slot 0
         }
     }
     teardown<256>(c, p.status);

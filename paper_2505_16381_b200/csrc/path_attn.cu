@@ -120,7 +120,7 @@ struct Plan {
     // offsets (bytes)
     size_t status, qp, kp, vp, wp, betap, G, Dyh, Dyl, Xqn, Yt, Qv16, Kv16;
     // backward only
-    size_t dop, delta, lse2, dQv, dKv, dSd, dSdT, dG, dGrow, dGdiag, dDy;
+    size_t dop, delta, lse2, dQv, dKv, dQl16, dKr16, dSd, dSdT, dG, dGrow, dGdiag, dDy;
     size_t sTh, sTl, sAh, sAl, sXq, sXk, sY, sU;   // bf16 tiles kept by the chunk preparation for the chain rule
     size_t dy_bytes, dy_mats;
 };
@@ -173,6 +173,7 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
         if (p.ragged) p.dop = bump(cur, SLd * 2);
         p.delta = bump(cur, SL * 4); p.lse2 = bump(cur, SL * 4);
         p.dQv = bump(cur, SLd * 4 * p.nslot); p.dKv = bump(cur, SLd * 4 * p.nslot);
+        p.dQl16 = bump(cur, SLd * 2); p.dKr16 = bump(cur, SLd * 2);
         p.dSd = bump(cur, gate ? SNBB * 4 : 0); p.dSdT = bump(cur, SNBB * 2); p.dG = bump(cur, SL * 4);
         p.dGrow = bump(cur, gate ? SL * 4 : 0); p.dGdiag = bump(cur, gate ? SL * 4 : 0);
         p.dDy = bump(cur, dy_elems * 4);
@@ -196,7 +197,10 @@ static LevelParams level_params(const Plan& p, void* ws) {
     lp.lv = p.lv; lp.S = p.S; lp.N = p.N; lp.Lp = p.Lp;
     lp.dyh = at<__nv_bfloat16>(ws, p.Dyh); lp.dyl = at<__nv_bfloat16>(ws, p.Dyl);
     lp.qv = at<__nv_bfloat16>(ws, p.Qv16); lp.kv = at<__nv_bfloat16>(ws, p.Kv16);
-    if (p.bwd) { lp.dqv = at<float>(ws, p.dQv); lp.dkv = at<float>(ws, p.dKv); lp.ddy = at<float>(ws, p.dDy); }
+    if (p.bwd) {
+        lp.dqv = at<float>(ws, p.dQv); lp.dkv = at<float>(ws, p.dKv); lp.ddy = at<float>(ws, p.dDy);
+        lp.dq16 = at<__nv_bfloat16>(ws, p.dQl16); lp.dk16 = at<__nv_bfloat16>(ws, p.dKr16);
+    }
     lp.status = at<uint32_t>(ws, p.status);
     return lp;
 }
@@ -290,10 +294,11 @@ static int run_chunk_chain(const Plan& p, void* ws, const void* q, const void* k
               make_map(&tm.xq, at<void>(ws, p.sXq), rows, CHUNK) && make_map(&tm.xk, at<void>(ws, p.sXk), rows, CHUNK) &&
               make_map(&tm.th, at<void>(ws, p.sTh), rows, CHUNK) && make_map(&tm.tl, at<void>(ws, p.sTl), rows, CHUNK) &&
               make_map(&tm.ah, at<void>(ws, p.sAh), rows, CHUNK) && make_map(&tm.al, at<void>(ws, p.sAl), rows, CHUNK) &&
-              make_map(&tm.dsdt, at<void>(ws, p.dSdT), (uint64_t)p.S * p.N * CHUNK, CHUNK);
+              make_map(&tm.dsdt, at<void>(ws, p.dSdT), (uint64_t)p.S * p.N * CHUNK, CHUNK) &&
+              make_map(&tm.dql, at<void>(ws, p.dQl16), rows, d) && make_map(&tm.dkr, at<void>(ws, p.dKr16), rows, d);
     if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
     ChainParams cp{};
-    cp.dql = at<float>(ws, p.dQv); cp.dkr = at<float>(ws, p.dKv);   // slot 0 of the version gradients
+    cp.dql = at<__nv_bfloat16>(ws, p.dQl16); cp.dkr = at<__nv_bfloat16>(ws, p.dKr16);   // slot 0 of the version gradients, final
     cp.dp = at<float>(ws, p.dDy);                                   // level 0 of the run-product gradients
     cp.beta = at<float>(ws, p.betap);
     cp.dq = (__nv_bfloat16*)dq; cp.dk = (__nv_bfloat16*)dk; cp.dw = (__nv_bfloat16*)dw; cp.dbeta = dbeta;
@@ -344,8 +349,9 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     prof_mark(STG_FA_DQ, 1, st);
     prof_mark(STG_LEVELS_BWD, 0, st);
 
-    // version chains, top level first, then the run products top-down
-    if (p.nlev >= 2) {
+    // version chains, top level first (this also rounds the final slot-0 gradients to bf16 for the chain rule, for
+    // every chunk, with or without a chain), then the run products top-down
+    {
         LevelTensorMaps ltm;
         if (!make_level_maps(p, ws, ltm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
         LevelParams lp = level_params(p, ws);
