@@ -140,6 +140,8 @@ struct BwdParams {
     const float* lse2;   // [S][Lp] (gate prefix - lse) * log2(e)
     const float* delta;  // [S][Lp] -(dO . O)
     const float* G;      // [S][Lp] gate prefix or nullptr
+    void* zero_ptr;      // dK/dV sweep: buffer it clears on the side (32-byte aligned, zero_bytes % 32 == 0), or zero_bytes = 0
+    size_t zero_bytes;
     uint32_t* status;
     int S, L, Lp, N;
     float scale;

@@ -302,6 +302,16 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
                 }
                 g += T; qb += T + 1; db += T + 1;
             }
+        } else if (warp >= 2) {
+            // The two spare warps clear this CTA's share of the run-product gradient buffer, which later kernels
+            // accumulate into: the sweep leaves most of the memory bandwidth unused.
+            const size_t n32 = p.zero_bytes / 32, per = (n32 + gridDim.x - 1) / gridDim.x;
+            const size_t lo = (size_t)blockIdx.x * per, hi = lo + per < n32 ? lo + per : n32;
+            for (size_t i = lo + (threadIdx.x - 64); i < hi; i += 64) {   // paced, so that the sweep's own stores are not delayed
+                asm volatile("st.global.v8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"l"((uint8_t*)p.zero_ptr + i * 32), "r"(0u)
+                             : "memory");
+                __nanosleep(300);
+            }
         }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");

@@ -323,7 +323,6 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
         LAUNCH(launch_pad_rows(d_o, at<void>(ws, p.dop), p.S, p.L, p.Lp, d, 0, st));
         dop = at<void>(ws, p.dop);
     }
-    CK(cudaMemsetAsync(dDy, 0, p.dy_bytes, st));
     if (p.gate) CK(cudaMemsetAsync(at<float>(ws, p.dGrow), 0, (size_t)p.S * p.Lp * 4, st));
 
     BwdTensorMaps tm;
@@ -339,6 +338,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     bp.lse2 = at<float>(ws, p.lse2); bp.delta = at<float>(ws, p.delta);
     bp.G = p.gate ? at<float>(ws, p.G) : nullptr;
     bp.status = at<uint32_t>(ws, p.status);
+    bp.zero_ptr = dDy; bp.zero_bytes = p.dy_bytes;   // cleared by the dK/dV sweep, first accumulated into by the version chains
     bp.S = p.S; bp.L = p.L; bp.Lp = p.Lp; bp.N = p.N; bp.scale = scale;
     prof_mark(STG_ROWSTATS, 1, st);
     prof_mark(STG_FA_DKV, 0, st);
