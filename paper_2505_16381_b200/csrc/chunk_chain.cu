@@ -127,12 +127,12 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     auto f_tmp = [&](float x, int col) { return x * bt[col]; };
     auto f_dGm = [&](float x, int col) { return col < row ? -bt[row] * x : 0.f; };
 
-    // slots: 0 U->W   1 dQl->dT->tmp->dGm   2 Y->Xq->Xk->T->Ah   3 dSd   4 dXq   5 dKr->dY->dXk   6 dP->dU->Al..K/Q
+    // slots: 0 U->W   1 dQl->dT->tmp->dGm   2 Y^T->-Xq->Xk->T->Ah   3 dSd   4 dXq   5 dKr->dY->dXk   6 dP->dU->Al..K/Q
     // first tiles of a chunk: U, Y, (s dSd)^T (every use below takes the transposed view), dQl, dKr
     auto first_loads = [&](int ch) {
         mbar_expect_tx(&bars[0], 3 * kT * HD * 2 + 2 * kTileB);
         tma_tile(slot(0), &tm.u, &bars[0], HD, ch * kT);
-        tma_tile(slot(2), &tm.y, &bars[0], kT, ch * kT);
+        tma_tile(slot(2), &tm.yt, &bars[0], kT, ch * kT);
         tma_tile(slot(3), &tm.dsdt, &bars[0], kT, ch * kT);
         tma_tile(slot(1), &tm.dql, &bars[0], HD, ch * kT);
         tma_tile(slot(5), &tm.dkr, &bars[0], HD, ch * kT);
@@ -156,9 +156,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(1), OP_K, sa(0), OP_K, KD, 128, false);
-        mma_call(tmem + cA, sa(3), OP_MN, sa(2), OP_K, K8, 128, true);
+        mma_call(tmem + cA, sa(3), OP_MN, sa(2), OP_MN, K8, 128, true);          // slot 2 holds Y^T
         // phase 0b: dw = -Y dKr - U dP^T
-        mma_call(tmem + cDW, sa(2), OP_K, sa(5), OP_MN, K8, HD, false, true);
+        mma_call(tmem + cDW, sa(2), OP_MN, sa(5), OP_MN, K8, HD, false, true);
         mma_call(tmem + cDW, sa(0), OP_K, sa(6), OP_K, KD, HD, true, true);
         umma_commit(&bars[1]);
     }
@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     if (tid == 0) {
         mbar_expect_tx(&bars[0], kT * HD * 2 + kTileB);
         tma_tile(slot(0), &tm.w, &bars[0], HD, r0);
-        tma_tile(slot(2), &tm.xq, &bars[0], kT, r0);
+        tma_tile(slot(2), &tm.xqn, &bars[0], kT, r0);
     }
     acc_to_tile(cA, kT, slot(4), -1.f, M_LOWER);                    // dXq
     loads_wait();
@@ -178,8 +178,8 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(0), OP_K, sa(5), OP_K, KD, 128, false);
-        mma_call(tmem + cA, sa(2), OP_MN, sa(3), OP_K, K8, 128, true);
-        mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, HD, false);
+        mma_call(tmem + cA, sa(2), OP_MN, sa(3), OP_K, K8, 128, true, true);     // slot 2 holds -Xq: negated back
+        mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, HD, false, true);
         mma_call(tmem + cB, sa(0), OP_K, sa(6), OP_MN, KD, HD, true);
         mma_call(tmem + cG, sa(0), OP_K, sa(0), OP_K, KD, 128, false);
         umma_commit(&bars[1]);

@@ -114,6 +114,9 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                     tma_load_2d(sQK + kTileB + h * kPanelB, &tm.k, &bars[B_LOAD], h * 64, chunk * kT);
                 }
             };
+            auto store = [&](const CUtensorMap* m, const uint8_t* tile_, int ncols, int chunk_) {
+                for (int h = 0; h < ncols / 64; ++h) tma_store_2d(m, tile_ + h * kPanelB, h * 64, chunk_ * kT);
+            };
             int chunk = blockIdx.x;
             bool ok = chunk < nchunks;
             if (ok) {
@@ -143,12 +146,21 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 mma(tmem + 0, aQ, OP_K, aW, OP_MN, 8, HD, false);
                 mma(tmem + 0, aK, OP_K, aW, OP_MN, 8, HD, true);
                 umma_commit(&bars[B_U]);
+                if (SAVE) {   // the tiles kept for the chain rule leave through TMA stores, straight from the operand slots
+                    store(&tm.th, sQK, kT, chunk);
+                    store(&tm.tl, sQK + kTileB, kT, chunk);
+                }
                 // Y = T~ Xk
                 if (!wait(R_XK, par)) break;
                 tc_fence_after_sync();
                 mma(tmem + 384, aQ, OP_K, aBig + 2 * kTileB, OP_MN, 8, 128, false);
                 mma(tmem + 384, aK, OP_K, aBig + 2 * kTileB, OP_MN, 8, 128, true);
                 mma(tmem + 384, aQ, OP_K, aBig + 3 * kTileB, OP_MN, 8, 128, true);
+                if (SAVE) {   // B_Y lets the workers overwrite T~ (with U) and Xk (with Y): the stores must have read them
+                    store(&tm.xk, sBig + 2 * kTileB, kT, chunk);
+                    tma_store_commit();
+                    tma_store_wait_read();
+                }
                 umma_commit(&bars[B_Y]);
                 // Xq U and W^T U
                 if (!wait(R_U, par)) break;
@@ -159,6 +171,10 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 mma(tmem + 128, aW, OP_MN, aQ, OP_MN, 8, HD, false);
                 mma(tmem + 128, aW, OP_MN, aK, OP_MN, 8, HD, true);
                 umma_commit(&bars[B_G3A]);
+                if (SAVE) {
+                    store(&tm.u, sQK, HD, chunk);
+                    tma_store_commit();
+                }
                 // Y^T W
                 if (!wait(R_Y, par)) break;
                 tc_fence_after_sync();
@@ -169,6 +185,7 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 const int next = chunk + (int)gridDim.x;
                 if (next < nchunks) {
                     if (!wait(B_G3B, par)) break;
+                    if (SAVE) tma_store_wait_read();   // the U tile: the loads overwrite it
                     load(next);
                     if (!wait(B_LOAD, par ^ 1)) break;
                     tc_fence_after_sync();
@@ -176,6 +193,7 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                     umma_commit(&bars[B_GM]);
                 }
             }
+            if (SAVE) tma_store_wait_all();
         }
         __syncwarp();
     } else {
@@ -306,8 +324,6 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 tile_store_w16(sQK, row, c0, hi);
                 tile_store_w16(sQK + kTileB, row, c0, lo);
                 if (SAVE) {
-                    gstore_bf16_w16(p.sTh + grow * kT + c0, hi);
-                    gstore_bf16_w16(p.sTl + grow * kT + c0, lo);
                     split32(v, hi, lo);
                     gstore_bf16_w16(p.sAh + grow * kT + c0, hi);
                     gstore_bf16_w16(p.sAl + grow * kT + c0, lo);
@@ -327,7 +343,6 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 split32(v, hi, lo);
                 tile_store_w16(sBig + 2 * kTileB, row, c0, hi);
                 tile_store_w16(sBig + 3 * kTileB, row, c0, lo);
-                if (SAVE) gstore_bf16_w16(p.sXk + grow * kT + c0, hi);
             }
             fence_proxy_async_smem();
             tc_fence_before_sync();
@@ -341,7 +356,6 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 split32(v, hi, lo);
                 tile_store_w16(sBig, row, c0, hi);
                 tile_store_w16(sBig + kTileB, row, c0, lo);
-                if (SAVE) gstore_bf16_w16(p.sXq + grow * kT + c0, hi);
 #pragma unroll
                 for (int x = 0; x < 16; ++x) hi[x] ^= 0x80008000u;   // -Xq
                 gstore_bf16_w16(p.Xqn + grow * kT + c0, hi);
@@ -359,7 +373,6 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
 #pragma unroll
                 for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
                 split32(v, uh[c], ul[c]);
-                if (SAVE) gstore_bf16_w16(p.sU + grow * HD + c0, uh[c]);
             }
             if (!(ok = wwait(B_Y, par))) break;
 #pragma unroll
@@ -380,7 +393,6 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 split32(v, hi, lo);
                 tile_store_w16(sBig + 2 * kTileB, row, c0, hi);
                 tile_store_w16(sBig + 3 * kTileB, row, c0, lo);
-                if (SAVE) gstore_bf16_w16(p.sY + grow * kT + c0, hi);
                 unsigned short* yt = reinterpret_cast<unsigned short*>(p.Yt) + ((size_t)chunk * kT + c0) * kT + row;
 #pragma unroll
                 for (int x = 0; x < 16; ++x) {

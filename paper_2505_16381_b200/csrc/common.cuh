@@ -84,6 +84,8 @@ cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const Leve
 
 struct PrepTensorMaps {
     CUtensorMap w, q, k;   // [S*Lp][d] bf16, box 128 rows x 64 columns, 128-byte swizzle
+    // stores of the tiles kept for the chain rule (backward's instance only): [S*Lp][128]; u is [S*Lp][d]
+    CUtensorMap th, tl, xk, u;
 };
 
 struct PrepParams {
@@ -95,9 +97,9 @@ struct PrepParams {
     __nv_bfloat16* Xqn;           // [S*Lp][128] -lower(Q W^T)
     __nv_bfloat16* Yt;            // [S*Lp][128] (T~ strictLower(W K^T))^T
     __nv_bfloat16 *Ph, *Pl;       // [S*N][d][d] chunk products as a bf16 hi + lo pair (level 0 of the run products)
-    // bf16 copies for the chain rule, written only by the backward's instance ([S*Lp][128]; sU is [S*Lp][d]):
-    // T~ and (I + N)^-1 as hi + lo pairs, Xq, Xk, Y, U rounded once
-    __nv_bfloat16 *sTh, *sTl, *sAh, *sAl, *sXq, *sXk, *sY, *sU;
+    // (I + N)^-1 as a bf16 hi + lo pair for the chain rule, written only by the backward's instance ([S*Lp][128]);
+    // that instance also keeps T~ (hi + lo) and Xk, U rounded once, through the tensor maps
+    __nv_bfloat16 *sAh, *sAl;
     uint32_t* status;
 };
 
@@ -106,7 +108,7 @@ cudaError_t launch_chunk_prep(const PrepTensorMaps& tm, const PrepParams& p, int
 
 struct ChainTensorMaps {
     CUtensorMap w, q, k, u;                       // [S*Lp][d]
-    CUtensorMap y, xq, xk, th, tl, ah, al;        // [S*Lp][128]
+    CUtensorMap yt, xqn, xk, th, tl, ah, al;      // [S*Lp][128]; yt = Y^T and xqn = -Xq are the attention sweep's operands
     CUtensorMap dsdt;                             // [S*N*128][128] bf16: (scale * lower(dS))^T of the diagonal chunks
     CUtensorMap dql, dkr;                         // [S*Lp][d] bf16 gradients of the boundary-adjusted queries / keys
 };

@@ -121,7 +121,7 @@ struct Plan {
     size_t status, qp, kp, vp, wp, betap, G, Dyh, Dyl, Xqn, Yt, Qv16, Kv16;
     // backward only
     size_t dop, delta, lse2, dQv, dKv, dQl16, dKr16, dSd, dSdT, dG, dGrow, dGdiag, dDy;
-    size_t sTh, sTl, sAh, sAl, sXq, sXk, sY, sU;   // bf16 tiles kept by the chunk preparation for the chain rule
+    size_t sTh, sTl, sAh, sAl, sXk, sU;   // bf16 tiles kept by the chunk preparation for the chain rule
     size_t dy_bytes, dy_mats;
 };
 
@@ -153,7 +153,7 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
     const size_t keep = bwd ? 1 : 0;   // bf16 intermediates of the chunk preparation, kept for the chain rule
     p.sTh = bump(cur, keep * SNBB * 2); p.sTl = bump(cur, keep * SNBB * 2);
     p.sAh = bump(cur, keep * SNBB * 2); p.sAl = bump(cur, keep * SNBB * 2);
-    p.sXq = bump(cur, keep * SNBB * 2); p.sXk = bump(cur, keep * SNBB * 2); p.sY = bump(cur, keep * SNBB * 2);
+    p.sXk = bump(cur, keep * SNBB * 2);
     p.sU = bump(cur, keep * SLd * 2);
     size_t dy_elems = 0;
     for (int l = 0; l < 20; ++l) {
@@ -212,7 +212,7 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
     const int stg_prep = in_backward ? STG_PREP_BWD : STG_PREP, stg_lev = in_backward ? STG_LEVELS_BWDPREP : STG_LEVELS;
     // fused per-chunk kernel: UT transform, boundary-adjusted tiles (version slot 0), chunk products (level 0)
     {
-        PrepTensorMaps tm;
+        PrepTensorMaps tm{};
         const uint64_t rows = (uint64_t)p.S * p.Lp;
         if (!(make_map(&tm.w, w, rows, d) && make_map(&tm.q, q, rows, d) && make_map(&tm.k, k, rows, d))) {
             g_last_cuda_error = (int)cudaErrorUnknown;
@@ -226,8 +226,12 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
         pp.Xqn = at<bf>(ws, p.Xqn); pp.Yt = at<bf>(ws, p.Yt);
         pp.Ph = at<bf>(ws, p.Dyh); pp.Pl = at<bf>(ws, p.Dyl);
         if (p.bwd) {
-            pp.sTh = at<bf>(ws, p.sTh); pp.sTl = at<bf>(ws, p.sTl); pp.sAh = at<bf>(ws, p.sAh); pp.sAl = at<bf>(ws, p.sAl);
-            pp.sXq = at<bf>(ws, p.sXq); pp.sXk = at<bf>(ws, p.sXk); pp.sY = at<bf>(ws, p.sY); pp.sU = at<bf>(ws, p.sU);
+            pp.sAh = at<bf>(ws, p.sAh); pp.sAl = at<bf>(ws, p.sAl);
+            if (!(make_map(&tm.th, at<void>(ws, p.sTh), rows, CHUNK) && make_map(&tm.tl, at<void>(ws, p.sTl), rows, CHUNK) &&
+                  make_map(&tm.xk, at<void>(ws, p.sXk), rows, CHUNK) && make_map(&tm.u, at<void>(ws, p.sU), rows, d))) {
+                g_last_cuda_error = (int)cudaErrorUnknown;
+                return PATH_ERR_LAUNCH;
+            }
         }
         pp.status = at<uint32_t>(ws, p.status);
         prof_mark(stg_prep, 0, st);
@@ -290,8 +294,8 @@ static int run_chunk_chain(const Plan& p, void* ws, const void* q, const void* k
     const uint64_t rows = (uint64_t)p.S * p.Lp;
     ChainTensorMaps tm;
     bool ok = make_map(&tm.w, w, rows, d) && make_map(&tm.q, q, rows, d) && make_map(&tm.k, k, rows, d) &&
-              make_map(&tm.u, at<void>(ws, p.sU), rows, d) && make_map(&tm.y, at<void>(ws, p.sY), rows, CHUNK) &&
-              make_map(&tm.xq, at<void>(ws, p.sXq), rows, CHUNK) && make_map(&tm.xk, at<void>(ws, p.sXk), rows, CHUNK) &&
+              make_map(&tm.u, at<void>(ws, p.sU), rows, d) && make_map(&tm.yt, at<void>(ws, p.Yt), rows, CHUNK) &&
+              make_map(&tm.xqn, at<void>(ws, p.Xqn), rows, CHUNK) && make_map(&tm.xk, at<void>(ws, p.sXk), rows, CHUNK) &&
               make_map(&tm.th, at<void>(ws, p.sTh), rows, CHUNK) && make_map(&tm.tl, at<void>(ws, p.sTl), rows, CHUNK) &&
               make_map(&tm.ah, at<void>(ws, p.sAh), rows, CHUNK) && make_map(&tm.al, at<void>(ws, p.sAl), rows, CHUNK) &&
               make_map(&tm.dsdt, at<void>(ws, p.dSdT), (uint64_t)p.S * p.N * CHUNK, CHUNK) &&
