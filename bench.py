@@ -42,11 +42,11 @@ UNIT = "TFLOP/s"
 # DRAM bytes per launch PER (batch, head) SLICE at the C3 shape (L=4096, d=128), from the ncu captures at batch 1
 # (16 slices) summarised under profiles/; slices are independent, so a launch over S slices moves S times this.
 NCU_TRAFFIC_BYTES_PER_SLICE = {
-    "chunk_prep": (52.02e6 + 181.98e6) / 16,        # backward instance (the step's forward runs on the shared workspace)
-    "fa_fwd": (168.41e6 + 8.34e6) / 16,
-    "fa_bwd_dkv": (187.31e6 + 92.84e6) / 16,
-    "fa_bwd_dq": (117.70e6 + 47.64e6) / 16,
-    "bwd_chunk_chain": (315.35e6 + 34.60e6) / 16,
+    "chunk_prep": (54.82e6 + 146.67e6) / 16,        # backward instance (the step's forward runs on the shared workspace)
+    "fa_fwd": (168.90e6 + 8.16e6) / 16,
+    "fa_bwd_dkv": (187.93e6 + 156.76e6) / 16,       # includes clearing the run-product gradient buffer on the side
+    "fa_bwd_dq": (117.81e6 + 49.14e6) / 16,
+    "bwd_chunk_chain": (278.71e6 + 32.33e6) / 16,
 }
 
 
@@ -341,8 +341,10 @@ def run_ours(args, cfg):
     prep_bytes = nch * (3 * t_d + 2 * t_d + 2 * t_b + 2 * d * d * 2)
     # the step's forward runs on the backward-sized workspace, so its chunk preparation is the instance that also
     # stores the bf16 tiles of the chain rule (and the backward then skips its own)
-    stage_bytes = {"chunk_prep": prep_bytes + nch * (7 * t_b + t_d), "bwd_chunk_prep": prep_bytes + nch * (7 * t_b + t_d),
-                   "bwd_chunk_chain": nch * (4 * t_d + 7 * t_b + 2 * 2 * t_d + 2 * t_b + d * d * 4 + 3 * t_d)}
+    # (kept tiles: T~ and (I+N)^-1 as hi + lo, Xk [128 x 128] and U [128 x d]; the chain rule reads w, q, k, U, the seven
+    # [128 x 128] tiles, (s dSd)^T, bf16 dQl / dKr, the float32 dP and writes dq, dk, dw)
+    stage_bytes = {"chunk_prep": prep_bytes + nch * (5 * t_b + t_d), "bwd_chunk_prep": prep_bytes + nch * (5 * t_b + t_d),
+                   "bwd_chunk_chain": nch * (4 * t_d + 7 * t_b + t_b + 2 * t_d + d * d * 4 + 3 * t_d)}
     def ncu_traffic(kernel):
         per_slice = NCU_TRAFFIC_BYTES_PER_SLICE.get(kernel)
         return per_slice * B * H if (per_slice is not None and (L, d) == (4096, 128)) else None
