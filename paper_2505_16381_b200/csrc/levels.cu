@@ -325,6 +325,7 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
         // the step after this one (its description replaces l1, b, src only after this step's were copied above)
         const int l2n = next_step(l2 - 1);
         loads_wait(c);
+        tma_store_wait_read();   // the previous step's reductions have read their staging area: the prefetch below refills it
         publish();
         if (c.tid == 0 && c.ok) {
             if (l2n >= 1) issue_loads(buf ^ 1);
@@ -339,8 +340,7 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
         }
         mma_wait(c);
         if (c.ok) {
-            // run-product gradient: stage the [d][d] accumulator in this step's (now dead) operand slots so that the
-            // atomic adds of a warp fall on consecutive addresses
+            // run-product gradient: stage the [d][d] accumulator in this step's (now dead) operand slots
             constexpr int LDS = HD + 4;
             float* stage = (float*)(sm + (1 + 3 * buf) * kTileB);
             float v[32];
@@ -354,15 +354,13 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
                             make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
                 }
             }
+            fence_proxy_async_smem();
             __syncthreads();
-            float* dst = p.ddy + (size_t)mat * HD * HD;
-            for (int idx = c.tid * 4; idx < HD * HD; idx += 1024) {   // four consecutive elements per reduction
-                const float4 t = *reinterpret_cast<const float4*>(stage + (idx / HD) * LDS + (idx % HD));
-                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + idx), "f"(t.x), "f"(t.y), "f"(t.z),
-                             "f"(t.w)
-                             : "memory");
+            // one bulk reduction per row: the adds happen at the memory side while this CTA goes on with its next step
+            if (c.tid < HD) {
+                bulk_reduce_add_f32(p.ddy + (size_t)mat * HD * HD + (size_t)c.tid * HD, stage + c.tid * LDS, HD * 4);
+                tma_store_commit();
             }
-            __syncthreads();   // the staging area is the buffer the prefetch after next will fill
         }
         have_acc = true;
         l2 = l2n;
@@ -380,6 +378,7 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
             gstore_bf16x32(dx16 + (size_t)c.row * HD + c0, v);   // the chain's bottom is always slot 0
         }
     }
+    tma_store_wait_all();
     teardown<256>(c, p.status);
 }
 
@@ -403,15 +402,7 @@ __global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constan
         tma_tile(sm + 4 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat_lo * HD));
     }
     conv(c, p.ddy + (size_t)mat_up * HD * HD, HD, HD, sm);
-    // the current values of the two gradients this CTA adds to are requested now and used after the products
     constexpr int NI = HD / 64;
-    uint32_t pend_a[NI][4][8], pend_b[NI][4][8];
-#pragma unroll
-    for (int i = 0; i < NI; ++i) {
-        const size_t o = (size_t)c.row * HD + c.half * (HD / 2) + i * 32;
-        gload_f32x32_issue(p.ddy + (size_t)(mat_lo + 1) * HD * HD + o, pend_a[i], c.row < HD);
-        gload_f32x32_issue(p.ddy + (size_t)mat_lo * HD * HD + o, pend_b[i], c.row < HD);
-    }
     loads_wait(c);
     publish();
     if (c.tid == 0 && c.ok) {
@@ -425,21 +416,32 @@ __global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constan
     }
     mma_wait(c);
     if (c.ok) {
-        float v[32], o[32];
+        // both [d][d] accumulators are staged in the (now dead) operand slots and added to the gradients of the two
+        // factors by bulk reductions, one per row: the adds happen at the memory side
+        constexpr int LDS = HD + 4;
+        float* stage = (float*)sm;
+        float v[32];
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
             const int c0 = c.half * (HD / 2) + i * 32;
-            const size_t off = (size_t)c.row * HD + c0;
-            tmem_row32(c.tl + c0, v);
-            gload_f32x32_finish(pend_a[i], o);
 #pragma unroll
-            for (int x = 0; x < 32; ++x) o[x] += v[x];
-            gstore_f32x32(p.ddy + (size_t)(mat_lo + 1) * HD * HD + off, o, c.row < HD);
-            tmem_row32(c.tl + 128 + c0, v);
-            gload_f32x32_finish(pend_b[i], o);
+            for (int m = 0; m < 2; ++m) {
+                tmem_row32(c.tl + m * 128 + c0, v);
+                if (c.row < HD) {
 #pragma unroll
-            for (int x = 0; x < 32; ++x) o[x] += v[x];
-            gstore_f32x32(p.ddy + (size_t)mat_lo * HD * HD + off, o, c.row < HD);
+                    for (int x = 0; x < 8; ++x)
+                        *reinterpret_cast<float4*>(stage + (m * HD + c.row) * LDS + c0 + 4 * x) =
+                            make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
+                }
+            }
+        }
+        fence_proxy_async_smem();
+        __syncthreads();
+        if (c.tid < 2 * HD) {   // rows 0 .. d-1: dA (factor 2b+1), rows d .. 2d-1: dB (factor 2b)
+            const int m = c.tid / HD, r = c.tid % HD;
+            bulk_reduce_add_f32(p.ddy + (size_t)(mat_lo + 1 - m) * HD * HD + (size_t)r * HD, stage + c.tid * LDS, HD * 4);
+            tma_store_commit();
+            tma_store_wait_read();
         }
     }
     teardown<256>(c, p.status);
