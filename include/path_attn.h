@@ -43,9 +43,11 @@
 extern "C" {
 #endif
 
-/* I/O dtype of q, k, v, w, o and their gradients.  Arithmetic: bf16 tensor-core
- * products with float32 accumulation; PATH_FP32 splits each float32 operand of
- * the logit products into two bf16 terms so that logits keep ~16 mantissa bits. */
+/* I/O dtype of q, k, v, w, o and their gradients.
+ * PATH_BF16: bf16 tensor-core products with float32 accumulation (the training path, forward and backward).
+ * PATH_FP32: forward only; the definition of Sec. 2.2 evaluated in float32 on the CUDA cores (one warp per query
+ * position carrying u <- H_j u over the keys), O(L^2 d) work: an accuracy path for float32 tensors, not a fast one.
+ * path_attn_bwd and for_backward = 1 do not accept it. */
 typedef enum { PATH_BF16 = 0, PATH_FP32 = 1 } path_dtype_t;
 
 typedef enum {
@@ -62,7 +64,8 @@ typedef enum {
 } path_status_t;
 
 /* Bytes of scratch memory path_attn_fwd (for_backward = 0) or path_attn_bwd
- * (for_backward = 1) needs for this problem.  Returns 0 for invalid arguments. */
+ * (for_backward = 1) needs for this problem.  Returns 0 for invalid arguments
+ * (PATH_FP32 with for_backward = 1 is one). */
 size_t path_attn_workspace_bytes(int B, int H, int L, int d, path_dtype_t dt, int has_gate,
                                  int for_backward);
 

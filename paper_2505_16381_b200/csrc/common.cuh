@@ -153,5 +153,8 @@ cudaError_t launch_fa_bwd(const BwdTensorMaps& tm, const BwdParams& p, int hd, i
 cudaError_t launch_rowstats(const void* o, const void* d_o, const float* lse, const float* G, float* delta, float* lse2,
                             int S, int L, int Lp, int hd, cudaStream_t st);
 cudaError_t launch_fa_fwd(const FwdTensorMaps& tm, const FwdParams& p, int hd, cudaStream_t st);
+// Float32 forward by the definition (PATH_FP32): q, k, v, w, o are [S][L][hd] float, G the gate prefix [S][ldG] or nullptr.
+cudaError_t launch_fp32_fwd(const float* q, const float* k, const float* v, const float* w, const float* beta, const float* G,
+                            float* o, float* lse, int S, int L, int ldG, int hd, float scale, cudaStream_t st);
 
 }  // namespace path

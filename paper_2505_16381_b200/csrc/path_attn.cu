@@ -145,6 +145,12 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
     size_t cur = 0;
     const size_t SLd = (size_t)S * Lp * d, SL = (size_t)S * Lp, SNBB = (size_t)S * p.N * CHUNK * CHUNK;
     p.status = bump(cur, 256);
+    if (dt == PATH_FP32) {   // float32 tensors: forward only, computed from the definition; needs the gate prefix alone
+        if (bwd) return false;
+        p.G = bump(cur, gate ? SL * 4 : 0);
+        p.total = cur;
+        return true;
+    }
     if (p.ragged) {
         p.qp = bump(cur, SLd * 2); p.kp = bump(cur, SLd * 2); p.vp = bump(cur, SLd * 2); p.wp = bump(cur, SLd * 2);
     }
@@ -401,7 +407,25 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     Plan p;
     if (dt != PATH_BF16 && dt != PATH_FP32) return PATH_ERR_DTYPE;
     if (!make_plan(B, H, L, d, (int)dt, log_f ? 1 : 0, 0, p)) return PATH_ERR_SHAPE;
-    if (dt != PATH_BF16) return PATH_ERR_DTYPE;
+    if (dt == PATH_FP32) {
+        if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(w) || !aligned16(beta) || !aligned16(o) ||
+            !aligned16(lse) || (log_f && !aligned16(log_f)) || ((uintptr_t)workspace & 255))
+            return PATH_ERR_ALIGN;
+        if (workspace_bytes < p.total) return PATH_ERR_WORKSPACE;
+        int rc32 = check_arch();
+        if (rc32 != PATH_OK) return rc32;
+        cudaStream_t st32 = (cudaStream_t)cuda_stream;
+        CK(cudaMemsetAsync(workspace, 0, 256, st32));
+        tag_store(StateTag{workspace, q, k, v, w, beta, log_f, B, H, L, d}, false);   // this call overwrites the workspace
+        float* G = nullptr;
+        if (log_f) {
+            G = at<float>(workspace, p.G);
+            LAUNCH(launch_gate_prefix(log_f, G, p.S, L, p.Lp, st32));
+        }
+        LAUNCH(launch_fp32_fwd((const float*)q, (const float*)k, (const float*)v, (const float*)w, beta, G, (float*)o, lse,
+                               p.S, L, p.Lp, d, scale, st32));
+        return PATH_OK;
+    }
     // A workspace large enough for the backward gets the backward's layout: the chunk preparation then also keeps
     // the tiles the chain rule needs, and path_attn_bwd on the same workspace and inputs does not redo it.
     const StateTag tag{workspace, q, k, v, w, beta, log_f, B, H, L, d};
@@ -455,8 +479,8 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
     if ((log_f == nullptr) != (dlog_f == nullptr)) return PATH_ERR_NULL;
     if (dt != PATH_BF16 && dt != PATH_FP32) return PATH_ERR_DTYPE;
     Plan p;
+    if (dt != PATH_BF16) return PATH_ERR_DTYPE;   // float32 tensors: forward only
     if (!make_plan(B, H, L, d, (int)dt, log_f ? 1 : 0, 1, p)) return PATH_ERR_SHAPE;
-    if (dt != PATH_BF16) return PATH_ERR_DTYPE;
     const void* ptrs[] = {q, k, v, w, beta, log_f, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f};
     for (const void* x : ptrs)
         if (x && !aligned16(x)) return PATH_ERR_ALIGN;

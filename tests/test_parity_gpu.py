@@ -110,14 +110,58 @@ def test_persistent_scheduling_shapes(binding, oracle, B, H, L, d, gate):
 
 
 def test_c1_workload_shape_and_distribution_in_bf16(binding, oracle):
-    """Workload C1 (B=1, H=2, L=256, d=64, q, k, v ~ N(0,1) unscaled: logits of standard deviation 8) with bf16 I/O.
-    The float32 I/O dtype of C1 itself is not built (PATH_FP32 is rejected with PATH_ERR_DTYPE)."""
+    """Workload C1's shape and distributions (B=1, H=2, L=256, d=64, q, k, v ~ N(0,1) unscaled: logits of standard
+    deviation 8) through the bf16 tensor-core path."""
     c = synth.CONFIGS["C1"]
     inp = synth.make_inputs(c["B"], c["H"], c["L"], c["d"], "bf16", qk_scaled=False, gate=False, seed=synth.BASE_SEED)
     compare_all(binding, oracle, inp, backward=False)      # C1 is a forward-only workload
-    q = inp["q"].cuda().float()
+
+
+# ---------------------------------------------------------------- float32 tensors (PATH_FP32): forward only
+
+F32_REL, F32_ABS = 2e-5, 2e-5     # float32 arithmetic end to end: dot products of d terms, chains of up to L steps
+
+
+def compare_f32(b, oracle, inp, scale=1.0):
+    dev = to_dev(inp)
+    assert dev["q"].dtype == torch.float32
+    o, lse = gpu_forward(b, dev, scale)
+    assert o.dtype == torch.float32
+    S = inp["q"].shape[0] * inp["q"].shape[1]
+    x = slices(inp, list(range(S)))
+    o_ref, lse_ref = oracle.forward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["log_f"], scale=scale)
+    check("o", o.reshape(-1, *o.shape[2:]), o_ref, rel=F32_REL, mx=F32_ABS)
+    assert np.abs(lse.reshape(S, -1).cpu().double().numpy() - lse_ref).max() <= 2e-5 * max(1.0, np.abs(lse_ref).max())
+    return o, lse
+
+
+def test_c1_workload_float32(binding, oracle):
+    """Workload C1 as stated: float32 tensors, forward only, against the float64 oracle on the same float32 values."""
+    inp = synth.make_config("C1")
+    assert inp["q"].dtype == torch.float32 and tuple(inp["q"].shape) == (1, 2, 256, 64)
+    o, lse = compare_f32(binding, oracle, inp)
+    o2, lse2 = gpu_forward(binding, to_dev(inp), 1.0)
+    assert torch.equal(o, o2) and torch.equal(lse, lse2)          # bitwise reproducible
+
+
+@pytest.mark.parametrize("B,H,L,d,gate,scale", [
+    (2, 3, 333, 128, True, 0.25),     # ragged length, gate, d = 128
+    (1, 1, 1, 64, False, 1.0),
+    (1, 2, 1100, 64, True, -0.125),
+])
+def test_float32_shapes(binding, oracle, B, H, L, d, gate, scale):
+    inp = synth.make_inputs(B, H, L, d, "fp32", gate=gate, seed=900 + L)
+    compare_f32(binding, oracle, inp, scale=scale)
+
+
+def test_float32_is_forward_only(binding):
+    inp = to_dev(synth.make_inputs(1, 1, 128, 64, "fp32", seed=3))
+    assert binding.workspace_bytes(1, 1, 128, 64, binding.PATH_FP32, False, True) == 0
+    assert binding.workspace_bytes(1, 1, 128, 64, binding.PATH_FP32, True, False) > 0
+    o, lse = binding.path_attn_fwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"])
     with pytest.raises(binding.PathAttnError) as e:
-        binding.path_attn_fwd(q, q, q, q, inp["beta"].cuda())
+        ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+        binding.path_attn_bwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"], o, lse, inp["d_o"], workspace=ws)
     assert e.value.status == -3
 
 
