@@ -168,6 +168,31 @@ int path_oracle_uchain(const double* q, const double* w, const double* beta, int
 }
 
 /*
+ * Key cache of the decoding recurrence (paper Sec. 3.4): after n tokens every cached key has been hit by the
+ * transitions that followed it, kc[j] = H_{n-1} H_{n-2} ... H_{j+1} k_j, j = 0..n-1, so that the logit of a
+ * later query is the plain dot product with the cached key.  Here written as that recurrence itself: token t
+ * arrives, every earlier key gets k <- H_t k, then k_t is appended untouched.  [S, n, d] out.
+ */
+int path_oracle_key_cache(const double* k, const double* w, const double* beta, int S, int L, int d, int n,
+                          double* kc) {
+    for (int s = 0; s < S; ++s) {
+        const double* ks = k + (size_t)s * L * d;
+        const double* ws = w + (size_t)s * L * d;
+        const double* bs = beta + (size_t)s * L;
+        double* cs = kc + (size_t)s * n * d;
+        for (int t = 0; t < n; ++t) {
+            for (int j = 0; j < t; ++j) {
+                double* x = cs + (size_t)j * d;
+                const double c = bs[t] * dot(ws + (size_t)t * d, x, d);
+                for (int e = 0; e < d; ++e) x[e] -= c * ws[(size_t)t * d + e];
+            }
+            memcpy(cs + (size_t)t * d, ks + (size_t)t * d, sizeof(double) * d);
+        }
+    }
+    return 0;
+}
+
+/*
  * Backward.  Given dO, returns the gradient of  sum(O * dO)  with respect to
  * q, k, v, w, beta and (if g != NULL) g.  Per row i:
  *

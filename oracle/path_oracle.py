@@ -49,6 +49,7 @@ def _load():
         lib.path_oracle_fwd.argtypes = [P, P, P, P, P, P, I, I, I, D, P, P]
         lib.path_oracle_logits.argtypes = [P, P, P, P, P, I, I, D, P]
         lib.path_oracle_uchain.argtypes = [P, P, P, I, I, I, P]
+        lib.path_oracle_key_cache.argtypes = [P, P, P, I, I, I, I, P]
         lib.path_oracle_bwd.argtypes = [P, P, P, P, P, P, P, I, I, I, D, P, P, P, P, P, P]
         _lib = lib
     return _lib
@@ -126,6 +127,22 @@ def uchain(q, w, beta, i: int):
     if rc != 0:
         raise MemoryError("path_oracle_uchain failed")
     return U
+
+
+def key_cache(k, w, beta, n=None):
+    """Decoding key cache after the first ``n`` tokens (default: all): ``kc[..., j, :] = H_{n-1} ... H_{j+1} k_j``,
+    built by the recurrence itself (every earlier key gets ``k <- H_t k`` when token t arrives).  ``[..., n, d]``."""
+    k, w, beta = map(_f64, (k, w, beta))
+    L, d = k.shape[-2:]
+    S = int(np.prod(k.shape[:-2], dtype=np.int64)) if k.ndim > 2 else 1
+    assert w.shape == k.shape and beta.shape == k.shape[:-1]
+    n = L if n is None else int(n)
+    assert 0 <= n <= L
+    kc = np.empty(k.shape[:-2] + (n, d))
+    rc = _load().path_oracle_key_cache(_ptr(k), _ptr(w), _ptr(beta), S, L, d, n, _ptr(kc))
+    if rc != 0:
+        raise MemoryError("path_oracle_key_cache failed")
+    return kc
 
 
 def backward(q, k, v, w, beta, d_o, log_f=None, scale: float = 1.0):

@@ -112,6 +112,36 @@ def test_key_cache_recurrence(oracle):
         assert np.abs(cache @ q[t] - a[t, :t + 1]).max() < 1e-11
 
 
+def test_key_cache_function_against_logits_products_and_special_cases(oracle):
+    """The oracle's key cache (Sec. 3.4): its dot product with a query is that query's logit row; it equals the explicit
+    matrix products H_{n-1} ... H_{j+1} k_j; beta = 0 leaves the keys alone; beta = 2 with unit w preserves their norms;
+    a cache of n tokens extended by hand by one more transition equals the cache of n + 1 tokens."""
+    rng = np.random.default_rng(41)
+    L, d = 24, 6
+    q, k, v, w, beta, _ = rand_problem(rng, L, d)
+    a = oracle.logits(q, k, w, beta)
+    for n in (1, 2, 9, L):
+        kc = oracle.key_cache(k, w, beta, n)
+        assert kc.shape == (n, d)
+        assert np.abs(kc @ q[n - 1] - a[n - 1, :n]).max() < 1e-11          # logits of the last cached position
+        for j in range(n):                                                 # explicit d x d products
+            M = np.eye(d)
+            for t in range(j + 1, n):
+                M = householder(w[t], beta[t]) @ M
+            assert np.abs(M @ k[j] - kc[j]).max() < 1e-11
+    kc9, kc10 = oracle.key_cache(k, w, beta, 9), oracle.key_cache(k, w, beta, 10)
+    step = np.vstack([kc9 @ householder(w[9], beta[9]).T, k[9][None]])
+    assert np.abs(step - kc10).max() < 1e-12
+    assert np.array_equal(oracle.key_cache(k, w, 0 * beta), k)
+    wn = w / np.linalg.norm(w, axis=-1, keepdims=True)
+    kc = oracle.key_cache(k, wn, 2.0 + 0 * beta)
+    assert np.abs(np.linalg.norm(kc, axis=-1) - np.linalg.norm(k, axis=-1)).max() < 1e-12
+    # batched call = per-slice calls
+    kb = np.stack([k, 2 * k]); wb = np.stack([w, w[::-1]]); bb = np.stack([beta, beta[::-1]])
+    kcb = oracle.key_cache(kb, wb, bb)
+    assert np.array_equal(kcb[0], oracle.key_cache(k, w, beta)) and np.array_equal(kcb[1], oracle.key_cache(2 * k, w[::-1], beta[::-1]))
+
+
 # ---------------------------------------------------------------- worked constructions
 
 def _read_swaps():
