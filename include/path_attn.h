@@ -142,6 +142,33 @@ int path_attn_fwd_static(const void* q, const void* k, const void* v, const void
                          const float* log_f, void* o, float* lse, int B, int H, int L, int d, float scale,
                          path_dtype_t dt, void* cuda_stream, void** scratch_out);
 
+/*
+ * Inference with a key cache (paper Sec. 3.4).  For every past position j the cache holds the key as the transitions
+ * after it have left it, kc_j = H_{t-1} ... H_{j+1} k_j, so that a new query needs plain dot products:
+ *   kc : [B,H,cap,d] float32 (float32 because every decoding step rewrites the whole cache in place)
+ *   vc : [B,H,cap,d] bf16 values as given          gc : [B,H,cap] float32 gate prefix sums (PaTH-FoX), or NULL
+ * cap >= 1 is the capacity in tokens; dt must be PATH_BF16 (dtype of the per-token inputs and of o).
+ *
+ * path_attn_prefill_cache fills positions 0..L-1 from a whole prompt: kc[.,.,j,:] = H_{L-1} ... H_{j+1} k_j, vc <- v
+ * and, when log_f and gc are given (both or neither), gc <- inclusive prefix sums of log_f.  Needs
+ * path_attn_workspace_bytes(B, H, L, d, PATH_BF16, has_gate, 0) bytes of workspace, which it overwrites.
+ *
+ * path_attn_decode_step processes the token at position t = number of cached tokens (0 <= t < cap):
+ *   kc_j <- kc_j - beta_t w_t (w_t . kc_j) for j < t;  kc_t <- k_t, vc_t <- v_t, gc_t <- gc_{t-1} + log_f_t;
+ *   o_t = sum_{j<=t} softmax_j(scale * q_t . kc_j + gc_t - gc_j) vc_j,   lse_t = log of the softmax's normaliser.
+ * q_t, k_t, v_t, w_t, o_t : [B,H,d] bf16;  beta_t, log_f_t, lse_t : [B,H] float32 (log_f_t NULL iff gc NULL).
+ * One pass over the cache (memory-bound).  Needs path_attn_decode_workspace_bytes(B, H, cap, d) bytes.
+ * Same conventions as the entry points above: device pointers, asynchronous on cuda_stream, no allocation.
+ */
+int path_attn_prefill_cache(const void* k, const void* v, const void* w, const float* beta, const float* log_f,
+                            float* kc, void* vc, float* gc, int B, int H, int L, int d, int cap, path_dtype_t dt,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t path_attn_decode_workspace_bytes(int B, int H, int cap, int d);
+int path_attn_decode_step(const void* q_t, const void* k_t, const void* v_t, const void* w_t, const float* beta_t,
+                          const float* log_f_t, float* kc, void* vc, float* gc, int t, int cap, void* o_t,
+                          float* lse_t, int B, int H, int d, float scale, path_dtype_t dt, void* workspace,
+                          size_t workspace_bytes, void* cuda_stream);
+
 /* Reads the device status word the last call on this workspace left behind.
  * Synchronises `cuda_stream`.  Returns PATH_OK, PATH_ERR_TIMEOUT, or
  * PATH_ERR_LAUNCH if the copy itself failed.  If `detail` is not NULL it

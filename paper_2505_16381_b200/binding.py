@@ -18,6 +18,7 @@ _lib = None
 PATH_BF16, PATH_FP32 = 0, 1
 PATH_OK = 0
 EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_attn_fwd_static", "path_attn_device_status",
+           "path_attn_prefill_cache", "path_attn_decode_workspace_bytes", "path_attn_decode_step",
            "path_attn_strerror", "path_attn_last_cuda_error", "path_attn_last_launch_count",
            "path_attn_profile_enable", "path_attn_profile_read", "path_attn_profile_stage_name"]
 
@@ -48,6 +49,12 @@ def load():
         lib.path_attn_fwd_static.argtypes = [P, P, P, P, P, P, P, P, I, I, I, I, F, I, P, ctypes.POINTER(P)]
         lib.path_attn_bwd.restype = I
         lib.path_attn_bwd.argtypes = [P] * 15 + [I, I, I, I, F, I, P, Z, P]
+        lib.path_attn_prefill_cache.restype = I
+        lib.path_attn_prefill_cache.argtypes = [P] * 8 + [I, I, I, I, I, I, P, Z, P]
+        lib.path_attn_decode_workspace_bytes.restype = Z
+        lib.path_attn_decode_workspace_bytes.argtypes = [I, I, I, I]
+        lib.path_attn_decode_step.restype = I
+        lib.path_attn_decode_step.argtypes = [P] * 9 + [I, I, P, P, I, I, I, F, I, P, Z, P]
         lib.path_attn_device_status.restype = I
         lib.path_attn_device_status.argtypes = [P, P, ctypes.POINTER(ctypes.c_uint)]
         lib.path_attn_strerror.restype = ctypes.c_char_p
@@ -193,3 +200,61 @@ def profile_read() -> dict:
     if n < 0:
         raise PathAttnError(n, "path_attn_profile_read")
     return {lib.path_attn_profile_stage_name(i).decode(): float(buf[i]) for i in range(n) if buf[i] >= 0}
+
+
+# ----------------------------------------------------------------------------------------- inference (key cache)
+
+def alloc_cache(B, H, cap, d, gate=False, device="cuda"):
+    """Empty caches for ``cap`` tokens: ``kc`` float32 and ``vc`` bf16 ``[B,H,cap,d]``, ``gc`` float32 ``[B,H,cap]`` or None."""
+    return {"kc": torch.zeros(B, H, cap, d, dtype=torch.float32, device=device),
+            "vc": torch.zeros(B, H, cap, d, dtype=torch.bfloat16, device=device),
+            "gc": torch.zeros(B, H, cap, dtype=torch.float32, device=device) if gate else None}
+
+
+def path_attn_prefill_cache(k, v, w, beta, cache, log_f=None, workspace=None):
+    """Fills positions ``0..L-1`` of ``cache`` from a prompt: ``kc_j = H_{L-1} ... H_{j+1} k_j``, ``vc = v``, gate prefix."""
+    _check(k, k, v, w, beta, log_f)
+    lib = load()
+    B, H, L, d = k.shape
+    cap = cache["kc"].shape[2]
+    if workspace is None:
+        workspace = alloc_workspace(k, log_f is not None, False)
+    st = torch.cuda.current_stream(k.device).cuda_stream
+    with torch.cuda.device(k.device):
+        rc = lib.path_attn_prefill_cache(_ptr(k), _ptr(v), _ptr(w), _ptr(beta), _ptr(log_f), _ptr(cache["kc"]),
+                                         _ptr(cache["vc"]), _ptr(cache["gc"]), B, H, L, d, cap, _dt(k), _ptr(workspace),
+                                         workspace.numel(), ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_prefill_cache")
+    return workspace
+
+
+def decode_workspace(B, H, cap, d, device="cuda"):
+    n = int(load().path_attn_decode_workspace_bytes(B, H, cap, d))
+    if n == 0:
+        raise PathAttnError(-2, "path_attn_decode_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def path_attn_decode_step(q_t, k_t, v_t, w_t, beta_t, cache, t, log_f_t=None, scale=1.0, workspace=None, out=None):
+    """One decoding step at position ``t`` (= number of cached tokens): updates ``cache`` in place, returns ``(o_t, lse_t)``.
+    ``q_t, k_t, v_t, w_t``: ``[B,H,d]`` bf16; ``beta_t, log_f_t``: ``[B,H]`` float32."""
+    for x in (q_t, k_t, v_t, w_t, beta_t):
+        if not (x.is_cuda and x.is_contiguous()):
+            raise ValueError("decode inputs must be contiguous CUDA tensors")
+    lib = load()
+    B, H, d = q_t.shape
+    cap = cache["kc"].shape[2]
+    if workspace is None:
+        workspace = decode_workspace(B, H, cap, d, q_t.device)
+    o = torch.empty_like(q_t) if out is None else out[0]
+    lse = torch.empty(B, H, dtype=torch.float32, device=q_t.device) if out is None else out[1]
+    st = torch.cuda.current_stream(q_t.device).cuda_stream
+    with torch.cuda.device(q_t.device):
+        rc = lib.path_attn_decode_step(_ptr(q_t), _ptr(k_t), _ptr(v_t), _ptr(w_t), _ptr(beta_t), _ptr(log_f_t),
+                                       _ptr(cache["kc"]), _ptr(cache["vc"]), _ptr(cache["gc"]), int(t), cap, _ptr(o),
+                                       _ptr(lse), B, H, d, float(scale), _dt(q_t), _ptr(workspace), workspace.numel(),
+                                       ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_decode_step")
+    return o, lse

@@ -75,11 +75,13 @@ struct LevelParams {
     int S, N, Lp;
     __nv_bfloat16 *dyh, *dyl, *qv, *kv;
     float *dqv, *dkv, *ddy;
+    float* kc;                    // key-cache kernel: [S][cap][d] float32 out (rows < L of every slice)
+    int cap, L;
     __nv_bfloat16 *dq16, *dk16;   // [S*Lp][d] final gradients of the slot-0 versions, rounded once (the chain rule's operands)
     uint32_t* status;
 };
 
-enum { LEVEL_DYADIC_FWD = 0, LEVEL_VERSION_FWD, LEVEL_VERSION_BWD, LEVEL_DYADIC_BWD };
+enum { LEVEL_DYADIC_FWD = 0, LEVEL_VERSION_FWD, LEVEL_VERSION_BWD, LEVEL_DYADIC_BWD, LEVEL_KEY_CACHE };
 cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const LevelParams& p, int hd, cudaStream_t st);
 
 struct PrepTensorMaps {
@@ -153,6 +155,11 @@ cudaError_t launch_fa_bwd(const BwdTensorMaps& tm, const BwdParams& p, int hd, i
 cudaError_t launch_rowstats(const void* o, const void* d_o, const float* lse, const float* G, float* delta, float* lse2,
                             int S, int L, int Lp, int hd, cudaStream_t st);
 cudaError_t launch_fa_fwd(const FwdTensorMaps& tm, const FwdParams& p, int hd, cudaStream_t st);
+// One decoding step over an in-place float32 key cache (paper Sec. 3.4); `part` holds decode_partials_bytes(S, cap, hd).
+size_t decode_partials_bytes(int S, int cap, int hd);
+cudaError_t launch_decode_step(const void* q_t, const void* k_t, const void* v_t, const void* w_t, const float* beta_t,
+                               const float* log_f_t, float* kc, void* vc, float* gc, int t, int cap, void* o_t, float* lse_t,
+                               int S, int hd, float scale, float* part, cudaStream_t st);
 // Float32 forward by the definition (PATH_FP32): q, k, v, w, o are [S][L][hd] float, G the gate prefix [S][ldG] or nullptr.
 cudaError_t launch_fp32_fwd(const float* q, const float* k, const float* v, const float* w, const float* beta, const float* G,
                             float* o, float* lse, int S, int L, int ldG, int hd, float scale, cudaStream_t st);

@@ -447,6 +447,75 @@ __global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constan
     teardown<256>(c, p.status);
 }
 
+// ---------------------------------------------------------------------------------------------- key cache after a prefill
+// grid.x = S.  Paper Sec. 3.4: after L tokens the cached key of position j is H_{L-1} ... H_{j+1} k_j.  In chunk form
+// that is  kc_J = Kright_J R_J  with  R_J = P_{J+1}^T ... P_{N-1}^T,  so one CTA walks the chunks of its slice from the
+// last to the first carrying R (d x d, bf16 hi + lo in shared memory):  kc_J = Kright_J R  (float32 out),  R <- P_J^T R.
+template <int HD>
+__global__ void __launch_bounds__(256, 1) key_cache_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    Ctx c;
+    setup<256>(c, smem_raw, kBar5);
+    const int s = blockIdx.x;
+    uint8_t* sm = c.smem;   // slots: 0 Kright_J, 1 P hi, 2 P lo, 3 R hi, 4 R lo
+    {   // R = I; the tiles' unused parts read as zeros (P^T enters with M = 128: its second 64-column panel when d = 64)
+        for (int i = c.tid; i < (int)(4 * kTileB / 16); i += 256) reinterpret_cast<uint4*>(sm + kTileB)[i] = make_uint4(0, 0, 0, 0);
+        __syncthreads();
+        if (c.tid < HD) {
+            uint8_t* panel = sm + 3 * kTileB + (c.tid >> 6) * kPanelB;
+            *reinterpret_cast<__nv_bfloat16*>(panel + sw128_off((uint32_t)c.tid, (uint32_t)((c.tid & 63) >> 3)) + (c.tid & 7) * 2) =
+                __float2bfloat16_rn(1.f);
+        }
+        fence_proxy_async_smem();
+        __syncthreads();
+    }
+    auto issue = [&](int J) {
+        const long mat = p.lv.dy_off[0] / (HD * HD) + (long)s * p.lv.dy_cnt[0] + J;
+        mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2);
+        tma_tile(sm, &tm.kv, &c.bars[0], HD, (int)((long)s * p.Lp + (long)J * kT));   // version slot 0 = Kright
+        tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
+        tma_tile(sm + 2 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
+    };
+    if (c.tid == 0) issue(p.N - 1);
+#pragma unroll 1
+    for (int J = p.N - 1; J >= 0 && c.ok; --J) {
+        loads_wait(c);
+        publish();
+        if (c.tid == 0 && c.ok) {
+            tc_fence_after_sync();
+            const uint32_t a = smem_u32(sm);
+            mma(c.tmem, a, OP_K, a + 3 * kTileB, OP_MN, HD / 16, HD, false);                       // Kright R
+            mma(c.tmem, a, OP_K, a + 4 * kTileB, OP_MN, HD / 16, HD, true);
+            if (J > 0) {
+                mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a + 3 * kTileB, OP_MN, HD / 16, HD, false);   // P^T R
+                mma(c.tmem + 128, a + 2 * kTileB, OP_MN, a + 3 * kTileB, OP_MN, HD / 16, HD, true);
+                mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a + 4 * kTileB, OP_MN, HD / 16, HD, true);
+            }
+            umma_commit(&c.bars[1]);
+        }
+        mma_wait(c);
+        if (!c.ok) break;
+        if (c.tid == 0 && J > 0) issue(J - 1);   // every product has retired: the operand slots are free again
+        const int pos = J * kT + c.row;
+        float v[32];
+        uint32_t hi[16], lo[16];
+        for (int i = 0; i < HD / 64; ++i) {
+            const int c0 = c.half * (HD / 2) + i * 32;
+            tmem_row32(c.tl + c0, v);
+            gstore_f32x32(p.kc + ((size_t)s * p.cap + pos) * HD + c0, v, pos < p.L);
+            if (J > 0) {
+                tmem_row32(c.tl + 128 + c0, v);
+                if (c.row < HD) {
+                    split32(v, hi, lo);
+                    tile_store_w16(sm + 3 * kTileB, c.row, c0, hi);
+                    tile_store_w16(sm + 4 * kTileB, c.row, c0, lo);
+                }
+            }
+        }
+    }
+    teardown<256>(c, p.status);
+}
+
 template <class K>
 cudaError_t launch(K kern, dim3 grid, uint32_t slots, const LevelTensorMaps& tm, const LevelParams& p, cudaStream_t st) {
     const uint32_t bytes = smem_bytes(slots);
@@ -471,6 +540,10 @@ cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const Leve
         case LEVEL_VERSION_BWD: {
             dim3 g(p.S * p.N, 2);
             return hd == 64 ? launch(version_bwd_kernel<64>, g, 7, tm, p, st) : launch(version_bwd_kernel<128>, g, 7, tm, p, st);
+        }
+        case LEVEL_KEY_CACHE: {
+            dim3 g(p.S);
+            return hd == 64 ? launch(key_cache_kernel<64>, g, 5, tm, p, st) : launch(key_cache_kernel<128>, g, 5, tm, p, st);
         }
         default: {
             dim3 g(p.S * p.lv.dy_cnt[p.l]);

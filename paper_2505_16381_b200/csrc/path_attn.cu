@@ -213,7 +213,7 @@ static LevelParams level_params(const Plan& p, void* ws) {
 
 // Chunk preparation + dyadic run products + version chains (paper Sec. 3.1, 3.3).  Shared by forward and backward.
 static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const void* w, bool in_backward,
-                    cudaStream_t st) {
+                    cudaStream_t st, bool with_levels = true) {
     const int d = p.d, nch = p.S * p.N;
     const int stg_prep = in_backward ? STG_PREP_BWD : STG_PREP, stg_lev = in_backward ? STG_LEVELS_BWDPREP : STG_LEVELS;
     // fused per-chunk kernel: UT transform, boundary-adjusted tiles (version slot 0), chunk products (level 0)
@@ -244,7 +244,7 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
         LAUNCH(launch_chunk_prep(tm, pp, d, p.bwd, nch, st));
         prof_mark(stg_prep, 1, st);
     }
-    if (p.nlev < 2) return PATH_OK;
+    if (p.nlev < 2 || !with_levels) return PATH_OK;
     LevelTensorMaps tm;
     if (!make_level_maps(p, ws, tm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
     LevelParams lp = level_params(p, ws);
@@ -554,6 +554,70 @@ int path_attn_fwd_static(const void* q, const void* k, const void* v, const void
     path::g_prof.on = timing;
     if (scratch_out) *scratch_out = scratch;
     return rc;
+}
+
+int path_attn_prefill_cache(const void* k, const void* v, const void* w, const float* beta, const float* log_f, float* kc,
+                            void* vc, float* gc, int B, int H, int L, int d, int cap, path_dtype_t dt, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream) {
+    g_launches = 0;
+    if (!k || !v || !w || !beta || !kc || !vc || !workspace) return PATH_ERR_NULL;
+    if ((log_f == nullptr) != (gc == nullptr)) return PATH_ERR_NULL;
+    if (dt != PATH_BF16) return PATH_ERR_DTYPE;
+    Plan p;
+    if (cap < L || !make_plan(B, H, L, d, (int)dt, log_f ? 1 : 0, 0, p)) return PATH_ERR_SHAPE;
+    if (!aligned16(k) || !aligned16(v) || !aligned16(w) || !aligned16(beta) || !aligned16(kc) || !aligned16(vc) ||
+        (log_f && (!aligned16(log_f) || !aligned16(gc))) || ((uintptr_t)workspace & 255))
+        return PATH_ERR_ALIGN;
+    if (workspace_bytes < p.total) return PATH_ERR_WORKSPACE;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CK(cudaMemsetAsync(workspace, 0, 256, st));
+    tag_store(StateTag{workspace, k, k, v, w, beta, log_f, B, H, L, d}, false);   // this call overwrites the workspace
+    // the chunk preparation needs no queries for the key side: the keys stand in for them
+    const void* qd = k; const void* kd = k; const void* vd = v; const void* wd = w;
+    rc = stage_inputs(p, workspace, qd, kd, vd, wd, beta, log_f, true, st);
+    if (rc != PATH_OK) return rc;
+    rc = run_prep(p, workspace, qd, kd, wd, false, st, false);
+    if (rc != PATH_OK) return rc;
+    LevelTensorMaps tm;
+    if (!make_level_maps(p, workspace, tm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+    LevelParams lp = level_params(p, workspace);
+    lp.kc = kc; lp.cap = cap; lp.L = L;
+    LAUNCH(launch_level_kernel(LEVEL_KEY_CACHE, tm, lp, d, st));
+    CK(cudaMemcpy2DAsync(vc, (size_t)cap * d * 2, v, (size_t)L * d * 2, (size_t)L * d * 2, (size_t)p.S, cudaMemcpyDeviceToDevice, st));
+    if (gc)
+        CK(cudaMemcpy2DAsync(gc, (size_t)cap * 4, at<float>(workspace, p.G), (size_t)p.Lp * 4, (size_t)L * 4, (size_t)p.S,
+                             cudaMemcpyDeviceToDevice, st));
+    return PATH_OK;
+}
+
+size_t path_attn_decode_workspace_bytes(int B, int H, int cap, int d) {
+    if (B < 1 || H < 1 || cap < 1 || (d != 64 && d != 128) || (long long)B * H > (1 << 20)) return 0;
+    return 256 + ((decode_partials_bytes(B * H, cap, d) + 255) & ~(size_t)255);
+}
+
+int path_attn_decode_step(const void* q_t, const void* k_t, const void* v_t, const void* w_t, const float* beta_t,
+                          const float* log_f_t, float* kc, void* vc, float* gc, int t, int cap, void* o_t, float* lse_t,
+                          int B, int H, int d, float scale, path_dtype_t dt, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream) {
+    g_launches = 0;
+    if (!q_t || !k_t || !v_t || !w_t || !beta_t || !kc || !vc || !o_t || !lse_t || !workspace) return PATH_ERR_NULL;
+    if ((log_f_t == nullptr) != (gc == nullptr)) return PATH_ERR_NULL;
+    if (dt != PATH_BF16) return PATH_ERR_DTYPE;
+    const size_t need = path_attn_decode_workspace_bytes(B, H, cap, d);
+    if (need == 0 || t < 0 || t >= cap) return PATH_ERR_SHAPE;
+    const void* ptrs[] = {q_t, k_t, v_t, w_t, kc, vc, o_t};
+    for (const void* x : ptrs)
+        if (!aligned16(x)) return PATH_ERR_ALIGN;
+    if ((uintptr_t)workspace & 255) return PATH_ERR_ALIGN;
+    if (workspace_bytes < need) return PATH_ERR_WORKSPACE;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    LAUNCH(launch_decode_step(q_t, k_t, v_t, w_t, beta_t, log_f_t, kc, vc, gc, t, cap, o_t, lse_t, B * H, d, scale,
+                              (float*)((uint8_t*)workspace + 256), st));
+    return PATH_OK;
 }
 
 int path_attn_device_status(const void* workspace, void* cuda_stream, unsigned int* detail) {
