@@ -16,7 +16,7 @@ namespace path {
 
 namespace {
 
-constexpr int kKeysPerCta = 256, kWarps = 8;
+constexpr int kKeysPerCta = 256, kWarps = 8, kInFlight = 1;   // positions a warp has in flight at once
 
 template <int E>
 __device__ __forceinline__ void load_bf16(const __nv_bfloat16* p, int lane, float (&x)[E]) {
@@ -77,12 +77,12 @@ __global__ void __launch_bounds__(32 * kWarps) decode_update_kernel(
 #pragma unroll
     for (int e = 0; e < E; ++e) acc[e] = 0.f;
 
-    // two positions per iteration, so that a warp has two rows of keys and values in flight
-    for (int i0 = lo + warp; i0 < hi; i0 += 2 * kWarps) {
-        float kk[2][E], vv[2][E], Gi[2], sc[2];
-        bool live[2];
+    // several positions per iteration, so that a warp has that many rows of keys and values in flight
+    for (int i0 = lo + warp; i0 < hi; i0 += kInFlight * kWarps) {
+        float kk[kInFlight][E], vv[kInFlight][E], Gi[kInFlight], sc[kInFlight];
+        bool live[kInFlight];
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
+        for (int x = 0; x < kInFlight; ++x) {
             const int i = i0 + x * kWarps;
             live[x] = i < hi;
             Gi[x] = 0.f;
@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(32 * kWarps) decode_update_kernel(
             }
         }
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
+        for (int x = 0; x < kInFlight; ++x) {
             if (!live[x]) continue;
             const int i = i0 + x * kWarps;
             float a = 0.f, c = 0.f;
