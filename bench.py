@@ -403,6 +403,65 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def run_decode(args):
+    """Inference arm (paper Sec. 3.4), 1 GPU: prefill of the key cache for the C5 prompt shape, then `--steps` decoding
+    steps on top of it.  One JSON line: decoding throughput and the step's algorithmic cache bytes against the measured
+    copy bandwidth (the step is one read-modify-write pass over the float32 key cache plus a read of the bf16 values)."""
+    from paper_2505_16381_b200 import binding
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    c = synth.CONFIGS["C5"]
+    B, H, L, d = (args.batch or c["B"]), c["H"], c["L"], c["d"]
+    g = torch.Generator(device=dev); g.manual_seed(synth.BASE_SEED)
+    rn = lambda *sh: torch.randn(*sh, device=dev, generator=g)
+    k = (rn(B, H, L, d) / d ** 0.5).bfloat16(); v = rn(B, H, L, d).bfloat16()
+    w = rn(B, H, L, d); w = (w / w.norm(dim=-1, keepdim=True)).bfloat16(); beta = 2 * torch.sigmoid(rn(B, H, L))
+    n_tok = args.warmup + args.steps
+    cache = binding.alloc_cache(B, H, L + n_tok, d, False, dev)
+    ws = binding.alloc_workspace(k, False, False)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    binding.path_attn_prefill_cache(k, v, w, beta, cache, workspace=ws)
+    torch.cuda.synchronize()
+    p0, p1 = ev(), ev()
+    p0.record()
+    binding.path_attn_prefill_cache(k, v, w, beta, cache, workspace=ws)
+    p1.record()
+    torch.cuda.synchronize()
+    assert binding.device_status(ws) == 0
+    tok = [(rn(B, H, d) / d ** 0.5).bfloat16() for _ in range(2)] + [rn(B, H, d).bfloat16()]
+    wt = rn(B, H, d); wt = (wt / wt.norm(dim=-1, keepdim=True)).bfloat16(); bt = 2 * torch.sigmoid(rn(B, H))
+    dws = binding.decode_workspace(B, H, L + n_tok, d, dev)
+    out = (torch.empty(B, H, d, dtype=torch.bfloat16, device=dev), torch.empty(B, H, dtype=torch.float32, device=dev))
+    for i in range(args.warmup):
+        binding.path_attn_decode_step(tok[0], tok[1], tok[2], wt, bt, cache, L + i, workspace=dws, out=out)
+    sampler = ClockSampler(physical_gpu_index(0))
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = ev(), ev()
+    e0.record()
+    for i in range(args.steps):      # the cache (5.4 GB at the default shape) exceeds L2: no flush needed
+        binding.path_attn_decode_step(tok[0], tok[1], tok[2], wt, bt, cache, L + args.warmup + i, workspace=dws, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    peaks = load_peaks()
+    T = L + args.warmup + (args.steps - 1) / 2.0            # mean number of cached tokens over the timed steps
+    byt = B * H * T * (2 * 4 * d + 2 * d)
+    gbs = byt / (ms * 1e-3) / 1e9
+    line = {"metric": "PaTH decode steps/s per sequence at 32k cached tokens (B*H = %d heads)" % (B * H), "value": 1e3 / ms,
+            "unit": "steps/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"decode: B={B} H={H} cached tokens={L} d={d}, float32 key cache, bf16 values",
+                       "l2_policy": "cache exceeds L2 (no flush needed)"},
+            "clocks": clocks, "gpu_launches": 2 * args.steps,
+            "roofline": {"kernel": "decode_update_kernel", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm"], "traffic": None, "peak_source": f"{peaks['source']} copy bandwidth",
+                         "bytes_per_launch": byt},
+            "detail": {"prefill_cache_ms": p0.elapsed_time(p1), "prefill_tokens": B * L}}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -412,7 +471,12 @@ def main():
     ap.add_argument("--workload", default="C3", choices=[n for n, c in synth.CONFIGS.items() if c["backward"]])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling captures)")
+    ap.add_argument("--path", choices=["train", "decode"], default="train",
+                    help="train: the fwd+bwd step (the headline); decode: the inference arm (1 GPU, not part of the headline)")
     args = ap.parse_args()
+    if args.path == "decode":
+        args.warmup = max(args.warmup, 3)
+        return run_decode(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = dict(synth.CONFIGS[args.workload])
     if args.batch > 0:
