@@ -48,9 +48,15 @@ struct PrepSmem {
 enum { B_LOAD = 0, B_GM, B_XQK, B_U, B_Y, B_G3A, B_G3B, R_TT, R_XK, R_U, R_Y, R_E3, B_COUNT };
 constexpr int kWorkers = 256, kThreads = 384;   // warps 8..11: the issuer's warpgroup (one active lane)
 
-__device__ __forceinline__ void wsync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// Barriers over the eight worker warps.  bar.sync / bar.red are warp-aligned instructions: a warp whose lanes left a
+// loop at different times must reconverge first, or the part that runs ahead is taken for the whole warp.
+__device__ __forceinline__ void wsync() {
+    __syncwarp();
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+}
 __device__ __forceinline__ bool wsync_and(bool ok) {   // barrier over the worker warps + AND of `ok`
     uint32_t r;
+    __syncwarp();
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %1, 0;\n\t"

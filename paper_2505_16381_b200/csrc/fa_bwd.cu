@@ -449,9 +449,9 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
             tc_fence_after_sync();
             if (GATE) {   // the two threads of a key row add their halves of the column sum
                 if (h == 1) dsum_x[row] = dsum;
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+                { __syncwarp(); asm volatile("bar.sync 1, 256;" ::: "memory"); }
                 if (h == 0 && ok) p.dG[(size_t)s * p.Lp + kj] = -(dsum + dsum_x[row]);
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+                { __syncwarp(); asm volatile("bar.sync 1, 256;" ::: "memory"); }
             }
             if (!ok) {
                 mbar_arrive(&bars[K_ACCFREE]);
@@ -765,9 +765,9 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
             tc_fence_after_sync();
             if (GATE) {
                 if (h == 1) dsum_x[row] = dsum;
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+                { __syncwarp(); asm volatile("bar.sync 1, 256;" ::: "memory"); }
                 if (h == 0 && ok) p.dGrow[qi] = dsum + dsum_x[row];
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+                { __syncwarp(); asm volatile("bar.sync 1, 256;" ::: "memory"); }
             }
             if (ok) flush_dq(level(T - 1));
             tc_fence_before_sync();

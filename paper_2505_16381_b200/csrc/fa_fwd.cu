@@ -307,6 +307,7 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
         int item = 0;
         float2* statx = stat + x * kTile;
         auto wg_sync = [&]() {
+            __syncwarp();   // bar.sync is warp-aligned: reconverge first
             if (x == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
             else asm volatile("bar.sync 2, 128;" ::: "memory");
         };
@@ -428,6 +429,7 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
             // ---- merge the two streams and write O, LSE: warpgroup x handles columns [x*HD/2, (x+1)*HD/2)
             if (GATE) wg_sync();
             if (TX > 0) statx[row] = make_float2(m, l);
+            __syncwarp();
             asm volatile("bar.sync 3, 256;" ::: "memory");
             const bool two = NS > 1;
             const float2 s0 = stat[row];
