@@ -332,7 +332,7 @@ def run_ours(args, cfg):
     peaks = load_peaks()
     tf = lambda fl, t_ms: fl / (t_ms * 1e-3) / 1e12
     value = world * tf(f1 + b1, ms)
-    # work models of the single-kernel stages (DESIGN.md section 7): FLOPs for the attention sweeps (tensor-bound),
+    # work models of the single-kernel stages: FLOPs for the attention sweeps (tensor-bound),
     # algorithmic bytes for the per-chunk kernels (HBM-bound)
     nch = B * H * (-(-L // CHUNK))
     diag = nch * 2 * CHUNK ** 3

@@ -38,19 +38,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Non-blocking test of the phase with the given parity (for threads that watch several barriers).
-__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
 // Limit of one wait, in clock64() ticks (about one second at B200 clocks).
 constexpr long long kWaitTicks = 2000000000LL;
 
@@ -262,24 +249,4 @@ __device__ __forceinline__ void warp_store_rows128(void* base, size_t stride, ui
         }
     }
 }
-// Counterpart of the store: rows >= nrows read as zero.
-__device__ __forceinline__ void warp_load_rows128(const void* base, size_t stride, uint32_t (&w)[32], int nrows = 32) {
-    const int lane = threadIdx.x & 31, j = lane & 3, g4 = lane & ~3;
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        uint32_t v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-        const int row = g4 + (j ^ r);
-        if (row < nrows) {
-            const uint8_t* src = (const uint8_t*)base + (size_t)row * stride + 32 * j;
-            asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-                         : "l"(src)
-                         : "memory");
-        }
-#pragma unroll
-        for (int x = 0; x < 8; ++x) w[8 * r + x] = r == 0 ? v[x] : __shfl_xor_sync(0xffffffffu, v[x], r);
-    }
-    rot4_pieces(w, j);
-}
-
 }  // namespace tc5

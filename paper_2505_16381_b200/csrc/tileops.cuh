@@ -147,19 +147,6 @@ __device__ __forceinline__ void tile_store_w16(uint8_t* t, int row, int c0, cons
         *reinterpret_cast<uint4*>(panel + sw128_off((uint32_t)row, (uint32_t)(ch0 + ch))) =
             make_uint4(w[4 * ch], w[4 * ch + 1], w[4 * ch + 2], w[4 * ch + 3]);
 }
-__device__ __forceinline__ void gload_bf16x32(const __nv_bfloat16* src, float (&v)[32]) {
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-        const uint4 u = reinterpret_cast<const uint4*>(src)[x];
-        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-        for (int y = 0; y < 4; ++y) {
-            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[y]));
-            v[8 * x + 2 * y] = f.x;
-            v[8 * x + 2 * y + 1] = f.y;
-        }
-    }
-}
 __device__ __forceinline__ void unpack_bf16x32(const uint4 (&u4)[4], float (&v)[32]) {
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
