@@ -123,11 +123,25 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
             tile_store32(dst, row, c0, v);
         }
     };
+    // the same, both parts from one read of the accumulator
+    auto split_both = [&](uint32_t col, uint8_t* dst_hi, uint8_t* dst_lo, auto&& f) {
+        for (int c = 0; c < 2; ++c) {
+            const int c0 = half * 64 + c * 32;
+            uint32_t hi[16], lo[16];
+            tmem_row32(tl + col + c0, v);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) v[x] = f(v[x], c0 + x);
+            split32(v, hi, lo);
+            tile_store_w16(dst_hi, row, c0, hi);
+            tile_store_w16(dst_lo, row, c0, lo);
+        }
+    };
     auto f_dT = [&](float x, int col) { return col <= row ? x : 0.f; };
     auto f_tmp = [&](float x, int col) { return x * bt[col]; };
     auto f_dGm = [&](float x, int col) { return col < row ? -bt[row] * x : 0.f; };
 
-    // slots: 0 U->W   1 dQl->dT->tmp->dGm   2 Y^T->-Xq->Xk->T->Ah   3 dSd   4 dXq   5 dKr->dY->dXk   6 dP->dU->Al..K/Q
+    // slots: 0 U->W   1 dQl->dT->tmp->dGm   2 Y^T->-Xq->Xk->T->Ah->K   3 dSd->T lo->dT lo->tmp lo->dSd   4 dXq   5 dKr->dY->dXk
+    //        6 dP->dU->Al->Q
     // first tiles of a chunk: U, Y, (s dSd)^T (every use below takes the transposed view), dQl, dKr
     auto first_loads = [&](int ch) {
         mbar_expect_tx(&bars[0], 3 * kT * HD * 2 + 2 * kTileB);
@@ -203,29 +217,27 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     mma_wait();
     if (!ok) break;
-    // ---- phase 3: dXk = strictLower(T~^T dY) -> cB,  dw += T~^T dU   (hi, then lo through the same slot)
+    // ---- phase 3: dXk = strictLower(T~^T dY) -> cB,  dw += T~^T dU.  (s dSd)^T is not needed again before phase 5, where
+    // it is loaded once more: until then its slot (3) takes the lo parts of the bf16 pairs, so that the hi and lo products
+    // of a pair go out as one group.
     if (tid == 0) {
-        mbar_expect_tx(&bars[0], kTileB);
+        mbar_expect_tx(&bars[0], 2 * kTileB);
         tma_tile(slot(2), &tm.th, &bars[0], kT, r0);
+        tma_tile(slot(3), &tm.tl, &bars[0], kT, r0);
     }
     // dT stays in tensor memory (cA); its bf16 hi part goes to slot 1 now, the lo part follows in phase 4
     split_to_tile(cA, slot(1), false, f_dT);
-    for (int part = 0; part < 2; ++part) {
-        if (tid == 0 && part == 1) {
-            mbar_expect_tx(&bars[0], kTileB);
-            tma_tile(slot(2), &tm.tl, &bars[0], kT, r0);
-        }
-        loads_wait();
-        publish();
-        if (tid == 0) {
-            tc_fence_after_sync();
-            mma_call(tmem + cB, sa(2), OP_MN, sa(5), OP_MN, K8, 128, part > 0);
-            mma_call(tmem + cDW, sa(2), OP_MN, sa(6), OP_MN, K8, HD, true);
-            umma_commit(&bars[1]);
-        }
-        mma_wait();
-        if (!ok) break;
+    loads_wait();
+    publish();
+    if (tid == 0) {
+        tc_fence_after_sync();
+        mma_call(tmem + cB, sa(2), OP_MN, sa(5), OP_MN, K8, 128, false);
+        mma_call(tmem + cB, sa(3), OP_MN, sa(5), OP_MN, K8, 128, true);
+        mma_call(tmem + cDW, sa(2), OP_MN, sa(6), OP_MN, K8, HD, true);
+        mma_call(tmem + cDW, sa(3), OP_MN, sa(6), OP_MN, K8, HD, true);
+        umma_commit(&bars[1]);
     }
+    mma_wait();
     if (!ok) break;
     // ---- phase 4: M = Ainv^T dT -> cB;  dbeta_c = M_cc;  tmp = M D;  dA = strictLower(-tmp Ainv^T) -> cA
     if (tid == 0) {
@@ -234,21 +246,14 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         tma_tile(slot(6), &tm.al, &bars[0], kT, r0);
     }
     acc_to_tile(cB, kT, slot(5), 1.f, M_STRICT);                    // dXk (over dY)
+    split_to_tile(cA, slot(3), true, f_dT);                         // dT lo (over T~ lo)
     loads_wait();
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, 128, false);
         mma_call(tmem + cB, sa(6), OP_MN, sa(1), OP_MN, K8, 128, true);
-        umma_commit(&bars[1]);
-    }
-    mma_wait();
-    if (!ok) break;
-    split_to_tile(cA, slot(1), true, f_dT);                         // dT lo
-    publish();
-    if (tid == 0) {
-        tc_fence_after_sync();
-        mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, 128, true);
+        mma_call(tmem + cB, sa(2), OP_MN, sa(3), OP_MN, K8, 128, true);
         umma_commit(&bars[1]);
     }
     mma_wait();
@@ -262,29 +267,22 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
                 if (c0 + x == row) t1[row] = v[x];
         }
     }
-    split_to_tile(cB, slot(1), false, f_tmp);                       // tmp = M D, hi
+    split_both(cB, slot(1), slot(3), f_tmp);                        // tmp = M D, hi (over dT hi) and lo (over dT lo)
     publish();
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(1), OP_K, sa(2), OP_K, K8, 128, false);
         mma_call(tmem + cA, sa(1), OP_K, sa(6), OP_K, K8, 128, true);
+        mma_call(tmem + cA, sa(3), OP_K, sa(2), OP_K, K8, 128, true);
         umma_commit(&bars[1]);
     }
     mma_wait();
     if (!ok) break;
-    split_to_tile(cB, slot(1), true, f_tmp);                        // tmp lo
-    publish();
-    if (tid == 0) {
-        tc_fence_after_sync();
-        mma_call(tmem + cA, sa(1), OP_K, sa(2), OP_K, K8, 128, true);
-        umma_commit(&bars[1]);
-    }
-    mma_wait();
-    if (!ok) break;
-    if (tid == 0) {   // phase 5's K and Q replace Ainv hi / lo, whose last products have just retired
-        mbar_expect_tx(&bars[0], 2 * kT * HD * 2);
+    if (tid == 0) {   // phase 5's K and Q replace Ainv hi / lo, whose last products have just retired; (s dSd)^T returns
+        mbar_expect_tx(&bars[0], 2 * kT * HD * 2 + kTileB);
         tma_tile(slot(2), &tm.k, &bars[0], HD, r0);
         tma_tile(slot(6), &tm.q, &bars[0], HD, r0);
+        tma_tile(slot(3), &tm.dsdt, &bars[0], kT, r0);
     }
     {   // dA = strictLower(-cA);  dbeta_r = t1_r + sum_c dA_rc Gm_rc
         float part = 0.f;
