@@ -46,7 +46,7 @@ NCU_TRAFFIC_BYTES_PER_SLICE = {
     "fa_fwd": (168.90e6 + 8.16e6) / 16,
     "fa_bwd_dkv": (187.93e6 + 156.76e6) / 16,       # includes clearing the run-product gradient buffer on the side
     "fa_bwd_dq": (117.81e6 + 49.14e6) / 16,
-    "bwd_chunk_chain": (278.71e6 + 32.33e6) / 16,
+    "bwd_chunk_chain": (283.76e6 + 31.74e6) / 16,
 }
 
 
