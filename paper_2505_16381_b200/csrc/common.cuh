@@ -74,10 +74,10 @@ struct LevelParams {
     int l;                  // dyadic kernels: level being produced (fwd: l -> l + 1) / consumed (bwd); version kernels: number of levels
     int S, N, Lp;
     __nv_bfloat16 *dyh, *dyl, *qv, *kv;
-    float *dqv, *dkv, *ddy;
+    __nv_bfloat16 *dqv, *dkv;     // [slots][S][Lp][d] gradients of the versions; slot 0 ends up holding the final sums
+    float* ddy;
     float* kc;                    // key-cache kernel: [S][cap][d] float32 out (rows < L of every slice)
     int cap, L;
-    __nv_bfloat16 *dq16, *dk16;   // [S*Lp][d] final gradients of the slot-0 versions, rounded once (the chain rule's operands)
     uint32_t* status;
 };
 
@@ -134,8 +134,8 @@ struct BwdTensorMaps {
 };
 
 struct BwdParams {
-    float* dqv;          // [slots][S][Lp][d] gradients of the query versions (slot convention as the versions)
-    float* dkv;          // same for the key versions
+    __nv_bfloat16* dqv;  // [slots][S][Lp][d] gradients of the query versions (slot convention as the versions), bf16
+    __nv_bfloat16* dkv;  // same for the key versions
     void* dv;            // [S, L, d] bf16, final
     float* dsd;          // [S*N][128 q][128 k] lower(dS) of the diagonal chunks, unscaled; written for gated problems only
     __nv_bfloat16* dsdt; // [S*N][128 k][128 q] (scale * lower(dS))^T in bf16: the chain rule's operand

@@ -25,6 +25,7 @@
 #include <type_traits>
 #include "common.cuh"
 #include "tc5.cuh"
+#include "tileops.cuh"
 
 namespace path {
 using namespace tc5;
@@ -66,6 +67,21 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+// A warp writes its 32 accumulator rows as bf16: lane L holds CW consecutive columns of row L, scaled by `mul`; `dst`
+// is the first of them in the lane's own row.  One 32-column piece at a time (this runs inside the sweeps' hot loops).
+template <int CW>
+__device__ __forceinline__ void store_acc_bf16(__nv_bfloat16* dst, uint32_t tcol, float mul) {
+#pragma unroll 1
+    for (int c = 0; c < CW / 32; ++c) {
+        uint32_t r[32], w[16];
+        tmem_ld32(tcol + c * 32, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int x = 0; x < 16; ++x) w[x] = pack_bf16(__uint_as_float(r[2 * x]) * mul, __uint_as_float(r[2 * x + 1]) * mul);
+        tile::gstore_bf16_w16(dst + c * 32, w);
+    }
+}
+
 // Plain (untiled) bulk copy global -> shared, completion counted in bytes on `bar`; 16-byte aligned, size % 16 == 0.
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -305,10 +321,10 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
         } else if (warp >= 2) {
             // The two spare warps clear this CTA's share of the run-product gradient buffer, which later kernels
             // accumulate into: the sweep leaves most of the memory bandwidth unused.
-            const size_t n32 = p.zero_bytes / 32, per = (n32 + gridDim.x - 1) / gridDim.x;
-            const size_t lo = (size_t)blockIdx.x * per, hi = lo + per < n32 ? lo + per : n32;
-            for (size_t i = lo + (threadIdx.x - 64); i < hi; i += 64) {   // paced, so that the sweep's own stores are not delayed
-                asm volatile("st.global.v8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"l"((uint8_t*)p.zero_ptr + i * 32), "r"(0u)
+            const uint32_t n32 = (uint32_t)(p.zero_bytes / 32), per = (n32 + gridDim.x - 1) / gridDim.x;   // < 2^32 pieces of 32 bytes
+            const uint32_t lo = blockIdx.x * per, hi = lo + per < n32 ? lo + per : n32;
+            for (uint32_t i = lo + (threadIdx.x - 64); i < hi; i += 64) {   // paced, so that the sweep's own stores are not delayed
+                asm volatile("st.global.v8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"l"((uint8_t*)p.zero_ptr + (size_t)i * 32), "r"(0u)
                              : "memory");
                 __nanosleep(300);
             }
@@ -324,17 +340,8 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
         bool ok = true;
         int g = 0;                               // steps before the current item
         constexpr int CW = HD / 2;               // accumulator columns per thread when flushing
-        auto flush_dk = [&](int lvl) {
-            float* dst = p.dkv + ((size_t)ver_row(kslot(lvl, J), J) + q4 * 32) * HD + h * CW;   // the warp's 32 rows
-#pragma unroll 1
-            for (int c = 0; c < CW / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tlane + colDK + h * CW + c * 32, r);
-                tmem_ld_wait();
-#pragma unroll
-                for (int x = 0; x < 32; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * p.scale);
-                warp_store_rows128(dst + c * 32, (size_t)HD * 4, r);
-            }
+        auto flush_dk = [&](int lvl) {   // the version's gradient leaves as bf16, the form the version chain rule multiplies
+            store_acc_bf16<CW>(p.dkv + ((size_t)ver_row(kslot(lvl, J), J) + row) * HD + h * CW, tlane + colDK + h * CW, p.scale);
         };
         auto step = [&](auto first_tag, const int t) {
             constexpr bool FIRST = decltype(first_tag)::value;   // the diagonal chunk: causal mask, dSd written out
@@ -459,8 +466,8 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
             }
             if (T > 1) flush_dk(level(T - 1));
             else {  // last chunk: no later query chunk, the boundary-adjusted keys get a zero gradient from the sweep
-                float4* dst = reinterpret_cast<float4*>(p.dkv + ((size_t)ver_row(0, J) + row) * HD + h * CW);
-                for (int x = 0; x < CW / 4; ++x) dst[x] = make_float4(0.f, 0.f, 0.f, 0.f);
+                uint4* dst = reinterpret_cast<uint4*>(p.dkv + ((size_t)ver_row(0, J) + row) * HD + h * CW);
+                for (int x = 0; x < CW / 8; ++x) dst[x] = make_uint4(0u, 0u, 0u, 0u);
             }
             if (CW == 64) {   // 64 bf16 = one 128-byte line per row: coalesced exchange
                 uint32_t r0[32], r1[32], w[32];
@@ -672,23 +679,14 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
         int g = 0, na = 0;
         constexpr int CW = HD / 2;
         auto flush_dq = [&](int lvl) {
-            float* dst = p.dqv + ((size_t)ver_row(qslot(lvl, I), I) + q4 * 32) * HD + h * CW;   // the warp's 32 rows
-#pragma unroll 1
-            for (int c = 0; c < CW / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tlane + colDQ + h * CW + c * 32, r);
-                tmem_ld_wait();
-#pragma unroll
-                for (int x = 0; x < 32; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * p.scale);
-                warp_store_rows128(dst + c * 32, (size_t)HD * 4, r);
-            }
+            store_acc_bf16<CW>(p.dqv + ((size_t)ver_row(qslot(lvl, I), I) + row) * HD + h * CW, tlane + colDQ + h * CW, p.scale);
         };
 #pragma unroll 1
         for (int it = 0; item_of(it, I, s); ++it) {
             const int T = I;
             if (T == 0) {  // chunk 0 has no earlier keys: its boundary-adjusted queries get a zero gradient from the sweep
-                float4* dst = reinterpret_cast<float4*>(p.dqv + (size_t)s * p.Lp * HD);
-                for (int i = threadIdx.x - 128; i < kTile * HD / 4; i += 256) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                uint4* dst = reinterpret_cast<uint4*>(p.dqv + (size_t)s * p.Lp * HD);
+                for (int i = threadIdx.x - 128; i < kTile * HD / 8; i += 256) dst[i] = make_uint4(0u, 0u, 0u, 0u);
                 continue;
             }
             const size_t qi = (size_t)s * p.Lp + I * kTile + row;

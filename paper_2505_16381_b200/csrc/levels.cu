@@ -240,7 +240,8 @@ __global__ void __launch_bounds__(256, 2) version_fwd_kernel(const __grid_consta
 // g = dXv[l2][chunk] (what the sweeps wrote there plus what arrived from the level above, which stays in tensor memory):
 //     dXv[l1][chunk] += g Dy^T (queries) or g Dy (keys);
 //     dDy[l1][b]     += Xv[l1]^T g (queries) or g^T Xv[l1] (keys), atomically.
-// Only the bottom of the chain (always slot 0) leaves the CTA: as the bf16 tile the chunk chain rule loads.  The next step's operands are fetched while the
+// Gradients of the versions are bf16 (written by the sweeps).  Only the bottom of the chain (always slot 0) leaves the
+// CTA: added in place to the slot-0 gradient, which the chunk chain rule then loads as a tile.  The next step's operands are fetched while the
 // current one runs.
 template <int HD>
 __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
@@ -252,26 +253,8 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
         return 0;
     };
     int l2 = next_step(p.l - 1);
-    float* dxv = is_key ? p.dkv : p.dqv;
-    __nv_bfloat16* dx16 = (is_key ? p.dk16 : p.dq16) + ((size_t)s * p.Lp + (size_t)ch * kT) * HD;   // this chunk's rows
-    if (l2 == 0) {   // no chain: what the sweeps left in slot 0 is final
-        const float* src = dxv + ((size_t)s * p.Lp + (size_t)ch * kT) * HD;
-        constexpr int NIT = kT * HD / (256 * 8);   // every load of the thread is in flight before the first store
-        float4 a[NIT], b4[NIT];
-#pragma unroll
-        for (int it = 0; it < NIT; ++it) {
-            const int i = (it * 256 + threadIdx.x) * 8;
-            a[it] = *reinterpret_cast<const float4*>(src + i);
-            b4[it] = *reinterpret_cast<const float4*>(src + i + 4);
-        }
-#pragma unroll
-        for (int it = 0; it < NIT; ++it) {
-            const int i = (it * 256 + threadIdx.x) * 8;
-            *reinterpret_cast<uint4*>(dx16 + i) = make_uint4(pack_bf16(a[it].x, a[it].y), pack_bf16(a[it].z, a[it].w),
-                                                             pack_bf16(b4[it].x, b4[it].y), pack_bf16(b4[it].z, b4[it].w));
-        }
-        return;
-    }
+    if (l2 == 0) return;   // no chain: what the sweeps left in slot 0 is final
+    __nv_bfloat16* dxv = is_key ? p.dkv : p.dqv;
     extern __shared__ uint8_t smem_raw[];
     Ctx c;
     setup<256>(c, smem_raw, 7 * kTileB);
@@ -291,13 +274,24 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
     // The gradient stored in global memory at the level a step consumes is requested one step ahead (the first one
     // here), so that its latency hides behind the previous step's products and atomics.
     constexpr int NI = HD / 64;
-    uint32_t pend[NI][4][8];
-    {
-        const long row_top = ((long)l2 * p.S + s) * p.Lp + (long)ch * kT;
+    uint32_t pend[NI][2][8];   // 32 bf16 = 64 bytes per piece
+    auto request = [&](long row0) {
 #pragma unroll
-        for (int i = 0; i < NI; ++i)
-            gload_f32x32_issue(dxv + ((size_t)row_top + c.row) * HD + c.half * (HD / 2) + i * 32, pend[i]);
-    }
+        for (int i = 0; i < NI; ++i) {
+            const __nv_bfloat16* src = dxv + ((size_t)row0 + c.row) * HD + c.half * (HD / 2) + i * 32;
+            ld_global_v8(src, pend[i][0]);
+            ld_global_v8(src + 16, pend[i][1]);
+        }
+    };
+    auto arrived = [&](int i, float (&v)[32]) {
+#pragma unroll
+        for (int x = 0; x < 16; ++x) {
+            const uint32_t w = pend[i][x >> 3][x & 7];
+            v[2 * x] = __uint_as_float(w << 16);
+            v[2 * x + 1] = __uint_as_float(w & 0xffff0000u);
+        }
+    };
+    request(((long)l2 * p.S + s) * p.Lp + (long)ch * kT);
 #pragma unroll 1
     while (l2 >= 1 && c.ok) {
         version_step(is_key, ch, l2, p.N, l1, b, src);
@@ -309,7 +303,7 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
 #pragma unroll
             for (int i = 0; i < NI; ++i) {
                 const int c0 = c.half * (HD / 2) + i * 32;
-                gload_f32x32_finish(pend[i], v);
+                arrived(i, v);
                 if (have_acc) {
                     tmem_row32(c.tl + c0, a);
 #pragma unroll
@@ -318,9 +312,7 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
                 tile_store32(sm, c.row, c0, v);
             }
             // what is stored at the level this step contributes to: the next step's input, or the chain's final sum
-#pragma unroll
-            for (int i = 0; i < NI; ++i)
-                gload_f32x32_issue(dxv + ((size_t)row_src + c.row) * HD + c.half * (HD / 2) + i * 32, pend[i]);
+            request(row_src);
         }
         // the step after this one (its description replaces l1, b, src only after this step's were copied above)
         const int l2n = next_step(l2 - 1);
@@ -371,11 +363,12 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
             const int c0 = c.half * (HD / 2) + i * 32;
-            gload_f32x32_finish(pend[i], v);
+            arrived(i, v);
             tmem_row32(c.tl + c0, a);
 #pragma unroll
             for (int x = 0; x < 32; ++x) v[x] += a[x];
-            gstore_bf16x32(dx16 + (size_t)c.row * HD + c0, v);   // the chain's bottom is always slot 0
+            // the chain's bottom is always slot 0: its rows now hold the final sum, which the chunk chain rule loads
+            gstore_bf16x32(dxv + ((size_t)s * p.Lp + (size_t)ch * kT + c.row) * HD + c0, v);
         }
     }
     tma_store_wait_all();

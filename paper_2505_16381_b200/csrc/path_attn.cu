@@ -120,7 +120,7 @@ struct Plan {
     // offsets (bytes)
     size_t status, qp, kp, vp, wp, betap, G, Dyh, Dyl, Xqn, Yt, Qv16, Kv16;
     // backward only
-    size_t dop, delta, lse2, dQv, dKv, dQl16, dKr16, dSd, dSdT, dG, dGrow, dGdiag, dDy;
+    size_t dop, delta, lse2, dQv, dKv, dSd, dSdT, dG, dGrow, dGdiag, dDy;
     size_t sTh, sTl, sAh, sAl, sXk, sU;   // bf16 tiles kept by the chunk preparation for the chain rule
     size_t dy_bytes, dy_mats;
 };
@@ -178,8 +178,7 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
     if (bwd) {
         if (p.ragged) p.dop = bump(cur, SLd * 2);
         p.delta = bump(cur, SL * 4); p.lse2 = bump(cur, SL * 4);
-        p.dQv = bump(cur, SLd * 4 * p.nslot); p.dKv = bump(cur, SLd * 4 * p.nslot);
-        p.dQl16 = bump(cur, SLd * 2); p.dKr16 = bump(cur, SLd * 2);
+        p.dQv = bump(cur, SLd * 2 * p.nslot); p.dKv = bump(cur, SLd * 2 * p.nslot);   // bf16
         p.dSd = bump(cur, gate ? SNBB * 4 : 0); p.dSdT = bump(cur, SNBB * 2); p.dG = bump(cur, SL * 4);
         p.dGrow = bump(cur, gate ? SL * 4 : 0); p.dGdiag = bump(cur, gate ? SL * 4 : 0);
         p.dDy = bump(cur, dy_elems * 4);
@@ -204,8 +203,7 @@ static LevelParams level_params(const Plan& p, void* ws) {
     lp.dyh = at<__nv_bfloat16>(ws, p.Dyh); lp.dyl = at<__nv_bfloat16>(ws, p.Dyl);
     lp.qv = at<__nv_bfloat16>(ws, p.Qv16); lp.kv = at<__nv_bfloat16>(ws, p.Kv16);
     if (p.bwd) {
-        lp.dqv = at<float>(ws, p.dQv); lp.dkv = at<float>(ws, p.dKv); lp.ddy = at<float>(ws, p.dDy);
-        lp.dq16 = at<__nv_bfloat16>(ws, p.dQl16); lp.dk16 = at<__nv_bfloat16>(ws, p.dKr16);
+        lp.dqv = at<__nv_bfloat16>(ws, p.dQv); lp.dkv = at<__nv_bfloat16>(ws, p.dKv); lp.ddy = at<float>(ws, p.dDy);
     }
     lp.status = at<uint32_t>(ws, p.status);
     return lp;
@@ -305,10 +303,10 @@ static int run_chunk_chain(const Plan& p, void* ws, const void* q, const void* k
               make_map(&tm.th, at<void>(ws, p.sTh), rows, CHUNK) && make_map(&tm.tl, at<void>(ws, p.sTl), rows, CHUNK) &&
               make_map(&tm.ah, at<void>(ws, p.sAh), rows, CHUNK) && make_map(&tm.al, at<void>(ws, p.sAl), rows, CHUNK) &&
               make_map(&tm.dsdt, at<void>(ws, p.dSdT), (uint64_t)p.S * p.N * CHUNK, CHUNK) &&
-              make_map(&tm.dql, at<void>(ws, p.dQl16), rows, d) && make_map(&tm.dkr, at<void>(ws, p.dKr16), rows, d);
+              make_map(&tm.dql, at<void>(ws, p.dQv), rows, d) && make_map(&tm.dkr, at<void>(ws, p.dKv), rows, d);
     if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
     ChainParams cp{};
-    cp.dql = at<__nv_bfloat16>(ws, p.dQl16); cp.dkr = at<__nv_bfloat16>(ws, p.dKr16);   // slot 0 of the version gradients, final
+    cp.dql = at<__nv_bfloat16>(ws, p.dQv); cp.dkr = at<__nv_bfloat16>(ws, p.dKv);   // slot 0 of the version gradients: the final sums
     cp.dp = at<float>(ws, p.dDy);                                   // level 0 of the run-product gradients
     cp.beta = at<float>(ws, p.betap);
     cp.dq = (__nv_bfloat16*)dq; cp.dk = (__nv_bfloat16*)dk; cp.dw = (__nv_bfloat16*)dw; cp.dbeta = dbeta;
@@ -323,7 +321,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
                         float* dbeta, float* dlog_f, float scale, cudaStream_t st) {
     const int d = p.d;
     float* dDy = at<float>(ws, p.dDy);
-    float* dQv = at<float>(ws, p.dQv); float* dKv = at<float>(ws, p.dKv);
+    __nv_bfloat16* dQv = at<__nv_bfloat16>(ws, p.dQv); __nv_bfloat16* dKv = at<__nv_bfloat16>(ws, p.dKv);
 
     prof_mark(STG_ROWSTATS, 0, st);
     LAUNCH(launch_rowstats(o, d_o, lse, p.gate ? at<float>(ws, p.G) : nullptr, at<float>(ws, p.delta), at<float>(ws, p.lse2),
@@ -359,8 +357,8 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     prof_mark(STG_FA_DQ, 1, st);
     prof_mark(STG_LEVELS_BWD, 0, st);
 
-    // version chains, top level first (this also rounds the final slot-0 gradients to bf16 for the chain rule, for
-    // every chunk, with or without a chain), then the run products top-down
+    // version chains, top level first (they leave the final sums in slot 0 of the bf16 version gradients, which the chunk
+    // chain rule loads), then the run products top-down
     {
         LevelTensorMaps ltm;
         if (!make_level_maps(p, ws, ltm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
