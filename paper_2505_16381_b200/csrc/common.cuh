@@ -67,6 +67,7 @@ struct LevelTable {
 struct LevelTensorMaps {
     CUtensorMap dyh, dyl;   // [matrices * d][d] bf16 hi / lo planes of the run products
     CUtensorMap qv, kv;     // [slots * S * Lp][d] bf16 versions
+    CUtensorMap dqv, dkv;   // same shape: bf16 gradients of the versions (backward only)
 };
 
 struct LevelParams {

@@ -259,16 +259,20 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
     Ctx c;
     setup<256>(c, smem_raw, 7 * kTileB);
     uint8_t* sm = c.smem;   // slot 0: g; two buffers of three slots: Dy hi, Dy lo, Xv[l1]
-    auto issue_loads = [&](int buf) {   // operands of the step described by (l1, b, src)
+    auto issue_loads = [&](int buf, uint32_t more_bytes = 0) {   // operands of the step described by (l1, b, src)
         const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
         const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
         uint8_t* base = sm + (1 + 3 * buf) * kTileB;
-        mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2);
+        mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2 + more_bytes);   // one arrival per phase: every byte is announced here
         tma_tile(base, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
         tma_tile(base + kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
         tma_tile(base + 2 * kTileB, is_key ? &tm.kv : &tm.qv, &c.bars[0], HD, (int)row_src);
     };
-    if (c.tid == 0) issue_loads(0);
+    // the top level's gradient needs nothing added: it goes into the g slot as a tile, next to the first operands
+    if (c.tid == 0) {
+        issue_loads(0, kT * HD * 2);
+        tma_tile(sm, is_key ? &tm.dkv : &tm.dqv, &c.bars[0], HD, (int)(((long)l2 * p.S + s) * p.Lp + (long)ch * kT));
+    }
     int buf = 0;
     bool have_acc = false;
     // The gradient stored in global memory at the level a step consumes is requested one step ahead (the first one
@@ -291,25 +295,25 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
             v[2 * x + 1] = __uint_as_float(w & 0xffff0000u);
         }
     };
-    request(((long)l2 * p.S + s) * p.Lp + (long)ch * kT);
+
 #pragma unroll 1
     while (l2 >= 1 && c.ok) {
         version_step(is_key, ch, l2, p.N, l1, b, src);
         const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
         const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
-        // g = gradient stored at this level (+ the contribution from above) -> bf16 tile
+        // g = gradient stored at this level + the contribution from above -> bf16 tile (the first step's g is loaded as a tile)
         {
-            float v[32], a[32];
+            if (have_acc) {
+                float v[32], a[32];
 #pragma unroll
-            for (int i = 0; i < NI; ++i) {
-                const int c0 = c.half * (HD / 2) + i * 32;
-                arrived(i, v);
-                if (have_acc) {
+                for (int i = 0; i < NI; ++i) {
+                    const int c0 = c.half * (HD / 2) + i * 32;
+                    arrived(i, v);
                     tmem_row32(c.tl + c0, a);
 #pragma unroll
                     for (int x = 0; x < 32; ++x) v[x] += a[x];
+                    tile_store32(sm, c.row, c0, v);
                 }
-                tile_store32(sm, c.row, c0, v);
             }
             // what is stored at the level this step contributes to: the next step's input, or the chain's final sum
             request(row_src);

@@ -191,10 +191,12 @@ template <class T>
 static T* at(void* ws, size_t off) { return reinterpret_cast<T*>((char*)ws + off); }
 
 static bool make_level_maps(const Plan& p, void* ws, LevelTensorMaps& tm) {
+    memset(&tm, 0, sizeof(tm));
     const uint64_t rows = (uint64_t)p.S * p.Lp * p.nslot;
     return make_map(&tm.dyh, at<void>(ws, p.Dyh), (uint64_t)p.dy_mats * p.d, p.d) &&
            make_map(&tm.dyl, at<void>(ws, p.Dyl), (uint64_t)p.dy_mats * p.d, p.d) &&
-           make_map(&tm.qv, at<void>(ws, p.Qv16), rows, p.d) && make_map(&tm.kv, at<void>(ws, p.Kv16), rows, p.d);
+           make_map(&tm.qv, at<void>(ws, p.Qv16), rows, p.d) && make_map(&tm.kv, at<void>(ws, p.Kv16), rows, p.d) &&
+           (!p.bwd || (make_map(&tm.dqv, at<void>(ws, p.dQv), rows, p.d) && make_map(&tm.dkv, at<void>(ws, p.dKv), rows, p.d)));
 }
 
 static LevelParams level_params(const Plan& p, void* ws) {
