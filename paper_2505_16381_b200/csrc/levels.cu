@@ -240,7 +240,9 @@ __global__ void __launch_bounds__(256, 2) version_fwd_kernel(const __grid_consta
 // g = dXv[l2][chunk] (what the sweeps wrote there plus what arrived from the level above, which stays in tensor memory):
 //     dXv[l1][chunk] += g Dy^T (queries) or g Dy (keys);
 //     dDy[l1][b]     += Xv[l1]^T g (queries) or g^T Xv[l1] (keys), atomically.
-// Gradients of the versions are bf16 (written by the sweeps).  Only the bottom of the chain (always slot 0) leaves the
+// The run products enter the backward as single bf16 operands (their hi plane), like every other operand of a gradient
+// product; the lo plane only matters where products are chained (forward).  Gradients of the versions are bf16 (written
+// by the sweeps).  Only the bottom of the chain (always slot 0) leaves the
 // CTA: added in place to the slot-0 gradient, which the chunk chain rule then loads as a tile.  The next step's operands are fetched while the
 // current one runs.
 template <int HD>
@@ -258,14 +260,13 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
     extern __shared__ uint8_t smem_raw[];
     Ctx c;
     setup<256>(c, smem_raw, 7 * kTileB);
-    uint8_t* sm = c.smem;   // slot 0: g; two buffers of three slots: Dy hi, Dy lo, Xv[l1]
+    uint8_t* sm = c.smem;   // slot 0: g; two buffers of three slots: Dy (hi plane), -, Xv[l1]; a buffer is also the staging area
     auto issue_loads = [&](int buf, uint32_t more_bytes = 0) {   // operands of the step described by (l1, b, src)
         const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
         const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
         uint8_t* base = sm + (1 + 3 * buf) * kTileB;
-        mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2 + more_bytes);   // one arrival per phase: every byte is announced here
+        mbar_expect_tx(&c.bars[0], 2 * kT * HD * 2 + more_bytes);   // one arrival per phase: every byte is announced here
         tma_tile(base, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
-        tma_tile(base + kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
         tma_tile(base + 2 * kTileB, is_key ? &tm.kv : &tm.qv, &c.bars[0], HD, (int)row_src);
     };
     // the top level's gradient needs nothing added: it goes into the g slot as a tile, next to the first operands
@@ -329,7 +330,6 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
             const uint32_t g = smem_u32(sm), o = smem_u32(sm + (1 + 3 * buf) * kTileB);
             const int bop = is_key ? OP_MN : OP_K;
             mma(c.tmem, g, OP_K, o, bop, HD / 16, HD, false);
-            mma(c.tmem, g, OP_K, o + kTileB, bop, HD / 16, HD, true);
             if (!is_key) mma(c.tmem + 128, o + 2 * kTileB, OP_MN, g, OP_MN, 8, HD, false);
             else         mma(c.tmem + 128, g, OP_MN, o + 2 * kTileB, OP_MN, 8, HD, false);
             umma_commit(&c.bars[1]);
@@ -380,7 +380,8 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
 }
 
 // ---------------------------------------------------------------------------------------------- dyadic backward
-// grid.x = S * cnt(l).  With dC = dDy[l][b], A = Dy[l-1][2b+1], B = Dy[l-1][2b]:  dA += dC B^T,  dB += A^T dC.
+// grid.x = S * cnt(l).  With dC = dDy[l][b], A = Dy[l-1][2b+1], B = Dy[l-1][2b]:  dA += dC B^T,  dB += A^T dC
+// (A, B: the hi planes of the run products).
 template <int HD>
 __global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -390,13 +391,11 @@ __global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constan
     const int s = blockIdx.x / cnt, b = blockIdx.x % cnt;
     const long mat_up = p.lv.dy_off[p.l] / (HD * HD) + (long)s * cnt + b;
     const long mat_lo = p.lv.dy_off[p.l - 1] / (HD * HD) + (long)s * cntl + 2 * b;   // B; A is +1
-    uint8_t* sm = c.smem;   // slots: 0 dC, 1 A hi, 2 A lo, 3 B hi, 4 B lo
+    uint8_t* sm = c.smem;   // slots: 0 dC, 1 A, 3 B (2 and 4 are only part of the staging area below)
     if (c.tid == 0) {
-        mbar_expect_tx(&c.bars[0], 4 * kT * HD * 2);
+        mbar_expect_tx(&c.bars[0], 2 * kT * HD * 2);
         tma_tile(sm + 1 * kTileB, &tm.dyh, &c.bars[0], HD, (int)((mat_lo + 1) * HD));
-        tma_tile(sm + 2 * kTileB, &tm.dyl, &c.bars[0], HD, (int)((mat_lo + 1) * HD));
         tma_tile(sm + 3 * kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat_lo * HD));
-        tma_tile(sm + 4 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat_lo * HD));
     }
     conv(c, p.ddy + (size_t)mat_up * HD * HD, HD, HD, sm);
     constexpr int NI = HD / 64;
@@ -406,9 +405,7 @@ __global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constan
         tc_fence_after_sync();
         const uint32_t a = smem_u32(sm);
         mma(c.tmem, a, OP_K, a + 3 * kTileB, OP_K, HD / 16, HD, false);            // dC B^T
-        mma(c.tmem, a, OP_K, a + 4 * kTileB, OP_K, HD / 16, HD, true);
         mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a, OP_MN, HD / 16, HD, false);    // A^T dC
-        mma(c.tmem + 128, a + 2 * kTileB, OP_MN, a, OP_MN, HD / 16, HD, true);
         umma_commit(&c.bars[1]);
     }
     mma_wait(c);
