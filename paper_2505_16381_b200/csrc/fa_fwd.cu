@@ -450,7 +450,8 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
             const float f0 = w0 * inv, f1 = w1 * inv;
             const bool live = qi < p.L;
             const size_t orow = ((size_t)s * p.L + (live ? qi : 0)) * HD;
-#pragma unroll 1
+            uint32_t wrow[CW == 64 ? 32 : 1];   // d = 128: this thread's 64 outputs as one 128-byte row piece
+#pragma unroll
             for (int c = 0; c < CW / 32; ++c) {
                 const int c0 = x * CW + c * 32;
                 uint32_t oa[32], ob[32];
@@ -468,6 +469,11 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
                     if (two) v += __uint_as_float(ob[e]) * f1;
                     o[e] = v;
                 }
+                if (CW == 64 && !p.out_fp32) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) wrow[(CW == 64 ? c * 16 : 0) + (CW == 64 ? e : 0)] = pack_bf16(o[2 * e], o[2 * e + 1]);
+                    continue;
+                }
                 if (!live) continue;
                 if (p.out_fp32) {
                     float4* dst = reinterpret_cast<float4*>((float*)p.o + orow + c0);
@@ -480,6 +486,12 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
                         dst[e] = make_uint4(pack_bf16(o[8 * e], o[8 * e + 1]), pack_bf16(o[8 * e + 2], o[8 * e + 3]),
                                             pack_bf16(o[8 * e + 4], o[8 * e + 5]), pack_bf16(o[8 * e + 6], o[8 * e + 7]));
                 }
+            }
+            if (CW == 64 && !p.out_fp32) {   // the warp's 32 rows, whole 128-byte pieces per store instruction
+                const int row0 = I * kTile + q4 * 32;
+                if (CW == 64)
+                    warp_store_rows128((__nv_bfloat16*)p.o + ((size_t)s * p.L + row0) * HD + x * CW, (size_t)HD * 2,
+                                       reinterpret_cast<uint32_t(&)[32]>(wrow), p.L - row0);
             }
             if (live) {
                 if (x == 0) p.lse[(size_t)s * p.L + qi] = (mm + log2f(lsum)) * 0.6931471805599453f;
