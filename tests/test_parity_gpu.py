@@ -109,6 +109,24 @@ def test_persistent_scheduling_shapes(binding, oracle, B, H, L, d, gate):
     compare_all(binding, oracle, inp)
 
 
+def _random_cases(n, seed=20250516):
+    """Seeded list of small problems: lengths below, at and across chunk boundaries, both head sizes, gate, scale sign."""
+    import random
+    rng = random.Random(seed)
+    out = []
+    for i in range(n):
+        L = rng.choice([rng.randint(1, 130), rng.randint(130, 700), rng.choice([256, 384, 512, 640, 1024, 1152])])
+        out.append((rng.choice([1, 1, 2, 3]), rng.choice([1, 2, 3, 5]), L, rng.choice([64, 128]), rng.random() < 0.5,
+                    rng.random() < 0.3, rng.choice([1.0, 1.0, 0.5, -0.25]), 4000 + i))
+    return out
+
+
+@pytest.mark.parametrize("B,H,L,d,gate,sharp,scale,seed", _random_cases(16))
+def test_random_small_problems(binding, oracle, B, H, L, d, gate, sharp, scale, seed):
+    inp = synth.make_inputs(B, H, L, d, "bf16", gate=gate, seed=seed, sharp=sharp)
+    compare_all(binding, oracle, inp, scale=scale)
+
+
 def test_c1_workload_shape_and_distribution_in_bf16(binding, oracle):
     """Workload C1's shape and distributions (B=1, H=2, L=256, d=64, q, k, v ~ N(0,1) unscaled: logits of standard
     deviation 8) through the bf16 tensor-core path."""
