@@ -7,161 +7,161 @@
 // step is bound by memory bandwidth: 2 * 4 d bytes per cached key plus 2 d for its value.  The cache is float32
 // because it is rewritten at every step: a bf16 cache would be rounded t times.
 //
-// One warp handles one cached key at a time, the head dimension spread over its lanes; a CTA covers 256 consecutive
-// positions of one (batch, head) slice and leaves a partial softmax state (max, sum, weighted values), which a small
-// second kernel merges over the CTAs of the slice.
+// One half-warp handles one cached key at a time, the head dimension spread over its 16 lanes; a CTA covers 256
+// consecutive positions of one (batch, head) slice and leaves a partial softmax state (max, sum, weighted values), which
+// a small second kernel merges over the CTAs of the slice.
 #include "common.cuh"
 
 namespace path {
 
 namespace {
 
-constexpr int kKeysPerCta = 256, kWarps = 8, kInFlight = 1;   // positions a warp has in flight at once
-
-template <int E>
-__device__ __forceinline__ void load_bf16(const __nv_bfloat16* p, int lane, float (&x)[E]) {
-    if (E == 2) {
-        const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p + lane * 2));
-        x[0] = f.x; x[1] = f.y;
-    } else {
-        const uint2 u = *reinterpret_cast<const uint2*>(p + lane * 4);
-        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.x));
-        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.y));
-        x[0] = a.x; x[1] = a.y; x[E - 2] = b.x; x[E - 1] = b.y;
-    }
-}
-template <int E>
-__device__ __forceinline__ void load_f32(const float* p, int lane, float (&x)[E]) {
-    if (E == 2) {
-        const float2 f = *reinterpret_cast<const float2*>(p + lane * 2);
-        x[0] = f.x; x[1] = f.y;
-    } else {
-        const float4 f = *reinterpret_cast<const float4*>(p + lane * 4);
-        x[0] = f.x; x[1] = f.y; x[E - 2] = f.z; x[E - 1] = f.w;
-    }
-}
-template <int E>
-__device__ __forceinline__ void store_f32(float* p, int lane, const float (&x)[E]) {
-    if (E == 2) *reinterpret_cast<float2*>(p + lane * 2) = make_float2(x[0], x[1]);
-    else *reinterpret_cast<float4*>(p + lane * 4) = make_float4(x[0], x[1], x[E - 2], x[E - 1]);
-}
-__device__ __forceinline__ float warp_sum(float a) {
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
-    return a;
-}
+constexpr int kKeysPerCta = 256, kWarps = 8;
 
 // part: [S][nsplit][HD + 2] = (max, sum, weighted values) of each CTA's positions
+//
+// A half-warp (16 lanes) owns one cached position at a time: lane j of the half holds the elements
+// [4j, 4j+4) of every 64-element panel of the row (16-byte loads, a half-warp covers 256 contiguous bytes per
+// instruction), so a warp has two key rows and two value rows in flight.
 template <int HD>
 __global__ void __launch_bounds__(32 * kWarps) decode_update_kernel(
     const __nv_bfloat16* __restrict__ q_t, const __nv_bfloat16* __restrict__ k_t, const __nv_bfloat16* __restrict__ v_t,
     const __nv_bfloat16* __restrict__ w_t, const float* __restrict__ beta_t, const float* __restrict__ log_f_t, float* kc,
     __nv_bfloat16* vc, float* gc, int t, int cap, float scale, float* __restrict__ part) {
-    constexpr int E = HD / 32;
-    __shared__ float sm_m[kWarps], sm_l[kWarps], sm_acc[kWarps][HD];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int NP = HD / 64;          // 64-element panels per row
+    constexpr int NH = 2 * kWarps;       // half-warps per CTA
+    __shared__ float sm_m[NH], sm_l[NH], sm_acc[NH][HD];
+    const int lane = threadIdx.x & 31, hl = lane & 15, hw = threadIdx.x >> 4;   // lane in the half-warp, half-warp in the CTA
     const int s = blockIdx.y, nsplit = gridDim.x;
     const int lo = blockIdx.x * kKeysPerCta, hi = min(lo + kKeysPerCta, t + 1);
-    float q[E], w[E];
-    load_bf16<E>(q_t + (size_t)s * HD, lane, q);
-    load_bf16<E>(w_t + (size_t)s * HD, lane, w);
+    auto ld_bf16 = [&](const __nv_bfloat16* row, float (&x)[NP][4]) {
+#pragma unroll
+        for (int pn = 0; pn < NP; ++pn) {
+            const uint2 u = *reinterpret_cast<const uint2*>(row + pn * 64 + hl * 4);
+            const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.x));
+            const float2 b2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.y));
+            x[pn][0] = a.x; x[pn][1] = a.y; x[pn][2] = b2.x; x[pn][3] = b2.y;
+        }
+    };
+    float q[NP][4], w[NP][4];
+    ld_bf16(q_t + (size_t)s * HD, q);
+    ld_bf16(w_t + (size_t)s * HD, w);
     const float b = beta_t[s];
     float qw = 0.f;
 #pragma unroll
-    for (int e = 0; e < E; ++e) qw = fmaf(q[e], w[e], qw);
-    qw = warp_sum(qw);
+    for (int pn = 0; pn < NP; ++pn)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) qw = fmaf(q[pn][e], w[pn][e], qw);
+#pragma unroll
+    for (int off = 8; off >= 1; off >>= 1) qw += __shfl_xor_sync(0xffffffffu, qw, off);
     const float Gt = gc ? ((t > 0 ? gc[(size_t)s * cap + t - 1] : 0.f) + log_f_t[s]) : 0.f;
     float* kcs = kc + (size_t)s * cap * HD;
     __nv_bfloat16* vcs = vc + (size_t)s * cap * HD;
-    float m = -INFINITY, l = 0.f, acc[E];
+    float m = -INFINITY, l = 0.f, acc[NP][4];
 #pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+    for (int pn = 0; pn < NP; ++pn)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[pn][e] = 0.f;
 
-    // several positions per iteration, so that a warp has that many rows of keys and values in flight
-    for (int i0 = lo + warp; i0 < hi; i0 += kInFlight * kWarps) {
-        float kk[kInFlight][E], vv[kInFlight][E], Gi[kInFlight], sc[kInFlight];
-        bool live[kInFlight];
-#pragma unroll
-        for (int x = 0; x < kInFlight; ++x) {
-            const int i = i0 + x * kWarps;
-            live[x] = i < hi;
-            Gi[x] = 0.f;
-            if (!live[x]) continue;
+    // both halves of a warp run the same number of iterations (the shuffles below name all 32 lanes)
+    for (int i0 = lo; i0 < hi; i0 += NH) {
+        const int i = i0 + hw;
+        const bool live = i < hi;
+        float kk[NP][4], vv[NP][4], Gi = 0.f;
+        if (live) {
             if (i < t) {
-                load_f32<E>(kcs + (size_t)i * HD, lane, kk[x]);
-                load_bf16<E>(vcs + (size_t)i * HD, lane, vv[x]);
-                if (gc) Gi[x] = gc[(size_t)s * cap + i];
-            } else {   // the new token: appended as it is
-                load_bf16<E>(k_t + (size_t)s * HD, lane, kk[x]);
-                load_bf16<E>(v_t + (size_t)s * HD, lane, vv[x]);
-            }
-        }
 #pragma unroll
-        for (int x = 0; x < kInFlight; ++x) {
-            if (!live[x]) continue;
-            const int i = i0 + x * kWarps;
-            float a = 0.f, c = 0.f;
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-                a = fmaf(q[e], kk[x][e], a);
-                c = fmaf(w[e], kk[x][e], c);
-            }
-#pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) {
-                a += __shfl_xor_sync(0xffffffffu, a, off);
-                c += __shfl_xor_sync(0xffffffffu, c, off);
-            }
-            if (i < t) {   // kc_i <- H_t kc_i; its logit follows from the two dot products already known
-                const float coef = b * c;
-#pragma unroll
-                for (int e = 0; e < E; ++e) kk[x][e] = fmaf(-coef, w[e], kk[x][e]);
-                store_f32<E>(kcs + (size_t)i * HD, lane, kk[x]);
-                sc[x] = fmaf(scale, a - coef * qw, Gt - Gi[x]);
-            } else {
-                store_f32<E>(kcs + (size_t)i * HD, lane, kk[x]);
-                if (E == 2) {
-                    *reinterpret_cast<__nv_bfloat162*>(vcs + (size_t)i * HD + lane * 2) = __floats2bfloat162_rn(vv[x][0], vv[x][1]);
-                } else {
-                    __nv_bfloat162 p0 = __floats2bfloat162_rn(vv[x][0], vv[x][1]), p1 = __floats2bfloat162_rn(vv[x][E - 2], vv[x][E - 1]);
-                    uint2 u;
-                    u.x = *reinterpret_cast<uint32_t*>(&p0); u.y = *reinterpret_cast<uint32_t*>(&p1);
-                    *reinterpret_cast<uint2*>(vcs + (size_t)i * HD + lane * 4) = u;
+                for (int pn = 0; pn < NP; ++pn) {
+                    const float4 f = *reinterpret_cast<const float4*>(kcs + (size_t)i * HD + pn * 64 + hl * 4);
+                    kk[pn][0] = f.x; kk[pn][1] = f.y; kk[pn][2] = f.z; kk[pn][3] = f.w;
                 }
-                if (gc && lane == 0) gc[(size_t)s * cap + i] = Gt;
-                sc[x] = scale * a;
+                ld_bf16(vcs + (size_t)i * HD, vv);
+                if (gc) Gi = gc[(size_t)s * cap + i];
+            } else {   // the new token: appended as it is
+                ld_bf16(k_t + (size_t)s * HD, kk);
+                ld_bf16(v_t + (size_t)s * HD, vv);
             }
-            if (sc[x] > m) {   // warp-uniform
-                const float r = expf(m - sc[x]);
-                l *= r;
+        } else {
 #pragma unroll
-                for (int e = 0; e < E; ++e) acc[e] *= r;
-                m = sc[x];
-            }
-            const float pj = expf(sc[x] - m);
-            l += pj;
+            for (int pn = 0; pn < NP; ++pn)
 #pragma unroll
-            for (int e = 0; e < E; ++e) acc[e] = fmaf(pj, vv[x][e], acc[e]);
+                for (int e = 0; e < 4; ++e) kk[pn][e] = vv[pn][e] = 0.f;
         }
-    }
-    // merge the warps of the CTA
-    if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+        float a = 0.f, c = 0.f;
 #pragma unroll
-    for (int e = 0; e < E; ++e) sm_acc[warp][lane * E + e] = acc[e];
+        for (int pn = 0; pn < NP; ++pn)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                a = fmaf(q[pn][e], kk[pn][e], a);
+                c = fmaf(w[pn][e], kk[pn][e], c);
+            }
+#pragma unroll
+        for (int off = 8; off >= 1; off >>= 1) {   // within the half-warp
+            a += __shfl_xor_sync(0xffffffffu, a, off);
+            c += __shfl_xor_sync(0xffffffffu, c, off);
+        }
+        if (!live) continue;
+        float sc;
+        if (i < t) {   // kc_i <- H_t kc_i; its logit follows from the two dot products already known
+            const float coef = b * c;
+#pragma unroll
+            for (int pn = 0; pn < NP; ++pn) {
+                float4 f;
+                f.x = fmaf(-coef, w[pn][0], kk[pn][0]); f.y = fmaf(-coef, w[pn][1], kk[pn][1]);
+                f.z = fmaf(-coef, w[pn][2], kk[pn][2]); f.w = fmaf(-coef, w[pn][3], kk[pn][3]);
+                *reinterpret_cast<float4*>(kcs + (size_t)i * HD + pn * 64 + hl * 4) = f;
+            }
+            sc = fmaf(scale, a - coef * qw, Gt - Gi);
+        } else {
+#pragma unroll
+            for (int pn = 0; pn < NP; ++pn) {
+                *reinterpret_cast<float4*>(kcs + (size_t)i * HD + pn * 64 + hl * 4) =
+                    make_float4(kk[pn][0], kk[pn][1], kk[pn][2], kk[pn][3]);
+                __nv_bfloat162 p0 = __floats2bfloat162_rn(vv[pn][0], vv[pn][1]), p1 = __floats2bfloat162_rn(vv[pn][2], vv[pn][3]);
+                uint2 u;
+                u.x = *reinterpret_cast<uint32_t*>(&p0); u.y = *reinterpret_cast<uint32_t*>(&p1);
+                *reinterpret_cast<uint2*>(vcs + (size_t)i * HD + pn * 64 + hl * 4) = u;
+            }
+            if (gc && hl == 0) gc[(size_t)s * cap + i] = Gt;
+            sc = scale * a;
+        }
+        if (sc > m) {   // uniform over the half-warp
+            const float r = expf(m - sc);
+            l *= r;
+#pragma unroll
+            for (int pn = 0; pn < NP; ++pn)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[pn][e] *= r;
+            m = sc;
+        }
+        const float pj = expf(sc - m);
+        l += pj;
+#pragma unroll
+        for (int pn = 0; pn < NP; ++pn)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[pn][e] = fmaf(pj, vv[pn][e], acc[pn][e]);
+    }
+    // merge the half-warps of the CTA
+    if (hl == 0) { sm_m[hw] = m; sm_l[hw] = l; }
+#pragma unroll
+    for (int pn = 0; pn < NP; ++pn)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sm_acc[hw][pn * 64 + hl * 4 + e] = acc[pn][e];
     __syncthreads();
     float M = -INFINITY;
 #pragma unroll
-    for (int x = 0; x < kWarps; ++x) M = fmaxf(M, sm_m[x]);
+    for (int x = 0; x < NH; ++x) M = fmaxf(M, sm_m[x]);
     float* out = part + ((size_t)s * nsplit + blockIdx.x) * (HD + 2);
     if (threadIdx.x < HD) {
         float a = 0.f;
 #pragma unroll
-        for (int x = 0; x < kWarps; ++x) a += sm_acc[x][threadIdx.x] * expf(sm_m[x] - M);   // an idle warp has max = -inf: factor 0
+        for (int x = 0; x < NH; ++x) a += sm_acc[x][threadIdx.x] * expf(sm_m[x] - M);   // an idle half-warp has max = -inf: factor 0
         out[2 + threadIdx.x] = a;
     }
     if (threadIdx.x == 0) {
         float a = 0.f;
 #pragma unroll
-        for (int x = 0; x < kWarps; ++x) a += sm_l[x] * expf(sm_m[x] - M);
+        for (int x = 0; x < NH; ++x) a += sm_l[x] * expf(sm_m[x] - M);
         out[0] = M; out[1] = a;
     }
 }
