@@ -24,7 +24,7 @@ constexpr int kKeysPerCta = 256, kWarps = 8;
 // [4j, 4j+4) of every 64-element panel of the row (16-byte loads, a half-warp covers 256 contiguous bytes per
 // instruction), so a warp has two key rows and two value rows in flight.
 template <int HD>
-__global__ void __launch_bounds__(32 * kWarps) decode_update_kernel(
+__global__ void __launch_bounds__(32 * kWarps, 4) decode_update_kernel(
     const __nv_bfloat16* __restrict__ q_t, const __nv_bfloat16* __restrict__ k_t, const __nv_bfloat16* __restrict__ v_t,
     const __nv_bfloat16* __restrict__ w_t, const float* __restrict__ beta_t, const float* __restrict__ log_f_t, float* kc,
     __nv_bfloat16* vc, float* gc, int t, int cap, float scale, float* __restrict__ part) {
