@@ -442,23 +442,26 @@ __global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------- key cache after a prefill
-// grid.x = S.  Paper Sec. 3.4: after L tokens the cached key of position j is H_{L-1} ... H_{j+1} k_j.  In chunk form
-// that is  kc_J = Kright_J R_J  with  R_J = P_{J+1}^T ... P_{N-1}^T,  so one CTA walks the chunks of its slice from the
-// last to the first carrying R (d x d, bf16 hi + lo in shared memory):  kc_J = Kright_J R  (float32 out),  R <- P_J^T R.
+// grid = (S, d / 64).  Paper Sec. 3.4: after L tokens the cached key of position j is H_{L-1} ... H_{j+1} k_j.  In chunk
+// form that is  kc_J = Kright_J R_J  with  R_J = P_{J+1}^T ... P_{N-1}^T,  so a CTA walks the chunks of its slice from the
+// last to the first carrying R (bf16 hi + lo in shared memory):  kc_J = Kright_J R  (float32 out),  R <- P_J^T R.
+// Both products act on the columns of R independently, so a CTA carries only 64 columns of R (and writes those columns
+// of the cache): at d = 128 two CTAs share a slice (four with 32 columns each were no faster per step and, at 4096 tokens,
+// more CTAs than SMs).
 template <int HD>
 __global__ void __launch_bounds__(256, 1) key_cache_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
     extern __shared__ uint8_t smem_raw[];
     Ctx c;
     setup<256>(c, smem_raw, kBar5);
-    const int s = blockIdx.x;
-    uint8_t* sm = c.smem;   // slots: 0 Kright_J, 1 P hi, 2 P lo, 3 R hi, 4 R lo
-    {   // R = I; the tiles' unused parts read as zeros (P^T enters with M = 128: its second 64-column panel when d = 64)
+    constexpr int NC = 64;                      // columns of R per CTA
+    const int s = blockIdx.x, col0 = blockIdx.y * NC;
+    uint8_t* sm = c.smem;   // slots: 0 Kright_J, 1 P hi, 2 P lo, 3 R hi, 4 R lo ([d x 64] in the first panel)
+    {   // R = I[:, col0 .. col0+63]; the tiles' unused parts read as zeros (P^T enters with M = 128: its second panel when d = 64)
         for (int i = c.tid; i < (int)(4 * kTileB / 16); i += 256) reinterpret_cast<uint4*>(sm + kTileB)[i] = make_uint4(0, 0, 0, 0);
         __syncthreads();
-        if (c.tid < HD) {
-            uint8_t* panel = sm + 3 * kTileB + (c.tid >> 6) * kPanelB;
-            *reinterpret_cast<__nv_bfloat16*>(panel + sw128_off((uint32_t)c.tid, (uint32_t)((c.tid & 63) >> 3)) + (c.tid & 7) * 2) =
-                __float2bfloat16_rn(1.f);
+        if (c.tid < NC) {
+            const uint32_t r = (uint32_t)(col0 + c.tid), j = (uint32_t)c.tid;
+            *reinterpret_cast<__nv_bfloat16*>(sm + 3 * kTileB + sw128_off(r, j >> 3) + (j & 7) * 2) = __float2bfloat16_rn(1.f);
         }
         fence_proxy_async_smem();
         __syncthreads();
@@ -478,32 +481,29 @@ __global__ void __launch_bounds__(256, 1) key_cache_kernel(const __grid_constant
         if (c.tid == 0 && c.ok) {
             tc_fence_after_sync();
             const uint32_t a = smem_u32(sm);
-            mma(c.tmem, a, OP_K, a + 3 * kTileB, OP_MN, HD / 16, HD, false);                       // Kright R
-            mma(c.tmem, a, OP_K, a + 4 * kTileB, OP_MN, HD / 16, HD, true);
+            mma(c.tmem, a, OP_K, a + 3 * kTileB, OP_MN, HD / 16, NC, false);                       // Kright R
+            mma(c.tmem, a, OP_K, a + 4 * kTileB, OP_MN, HD / 16, NC, true);
             if (J > 0) {
-                mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a + 3 * kTileB, OP_MN, HD / 16, HD, false);   // P^T R
-                mma(c.tmem + 128, a + 2 * kTileB, OP_MN, a + 3 * kTileB, OP_MN, HD / 16, HD, true);
-                mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a + 4 * kTileB, OP_MN, HD / 16, HD, true);
+                mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a + 3 * kTileB, OP_MN, HD / 16, NC, false);   // P^T R
+                mma(c.tmem + 128, a + 2 * kTileB, OP_MN, a + 3 * kTileB, OP_MN, HD / 16, NC, true);
+                mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a + 4 * kTileB, OP_MN, HD / 16, NC, true);
             }
             umma_commit(&c.bars[1]);
         }
         mma_wait(c);
         if (!c.ok) break;
         if (c.tid == 0 && J > 0) issue(J - 1);   // every product has retired: the operand slots are free again
-        const int pos = J * kT + c.row;
+        const int pos = J * kT + c.row, c0 = c.half * 32;
         float v[32];
         uint32_t hi[16], lo[16];
-        for (int i = 0; i < HD / 64; ++i) {
-            const int c0 = c.half * (HD / 2) + i * 32;
-            tmem_row32(c.tl + c0, v);
-            gstore_f32x32(p.kc + ((size_t)s * p.cap + pos) * HD + c0, v, pos < p.L);
-            if (J > 0) {
-                tmem_row32(c.tl + 128 + c0, v);
-                if (c.row < HD) {
-                    split32(v, hi, lo);
-                    tile_store_w16(sm + 3 * kTileB, c.row, c0, hi);
-                    tile_store_w16(sm + 4 * kTileB, c.row, c0, lo);
-                }
+        tmem_row32(c.tl + c0, v);
+        gstore_f32x32(p.kc + ((size_t)s * p.cap + pos) * HD + col0 + c0, v, pos < p.L);
+        if (J > 0) {
+            tmem_row32(c.tl + 128 + c0, v);
+            if (c.row < HD) {
+                split32(v, hi, lo);
+                tile_store_w16(sm + 3 * kTileB, c.row, c0, hi);
+                tile_store_w16(sm + 4 * kTileB, c.row, c0, lo);
             }
         }
     }
@@ -536,7 +536,7 @@ cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const Leve
             return hd == 64 ? launch(version_bwd_kernel<64>, g, 7, tm, p, st) : launch(version_bwd_kernel<128>, g, 7, tm, p, st);
         }
         case LEVEL_KEY_CACHE: {
-            dim3 g(p.S);
+            dim3 g(p.S, hd / 64);
             return hd == 64 ? launch(key_cache_kernel<64>, g, 5, tm, p, st) : launch(key_cache_kernel<128>, g, 5, tm, p, st);
         }
         default: {
