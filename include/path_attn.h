@@ -169,6 +169,30 @@ int path_attn_decode_step(const void* q_t, const void* k_t, const void* v_t, con
                           float* lse_t, int B, int H, int d, float scale, path_dtype_t dt, void* workspace,
                           size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * Layer front-end: how a PaTH layer obtains the operator's w, beta and log_f (paper Sec. 2.2, footnote to the
+ * definition of H_t; gate of Sec. 2.4).  The linear maps in front (the low-rank layer giving z, and u^T x + b for the
+ * two logits) are plain matrix products and stay with the caller's GEMM library; these two calls are the rest:
+ *   y_t[c]  = conv_w[c][0] z_{t-2}[c] + conv_w[c][1] z_{t-1}[c] + conv_w[c][2] z_t[c]   (causal, depthwise, z = 0 before t = 0)
+ *   w_t     = y_t / sqrt(sum over the head's d channels of y_t^2 + eps)               (per head)
+ *   beta_t  = 2 sigmoid(beta_logit_t),      log_f_t = log sigmoid(gate_logit_t)
+ * Layouts: z, dz : [B,L,H*d] bf16 (head h owns channels h*d .. h*d+d-1);  conv_w, dconv_w : [H*d,3] float32;
+ *   beta_logit, gate_logit and their gradients : [B,L,H] float32;  w, dw : [B,H,L,d] bf16;
+ *   beta, log_f, dbeta, dlog_f : [B,H,L] float32  (the operator's layouts: the calls also do the change of layout).
+ * gate_logit, log_f, dlog_f, dgate_logit are all NULL for plain PaTH and all given for PaTH-FoX.  eps >= 0.
+ * path_attn_frontend_bwd returns the gradients of sum(w*dw) + sum(beta*dbeta) + sum(log_f*dlog_f); dconv_w is
+ * summed with float32 atomics (reproducible to rounding, not bitwise).  Float32 arithmetic, one pass over the
+ * tensors (memory-bound), no workspace.  Same conventions as above: device pointers, outputs fully overwritten,
+ * asynchronous on cuda_stream, argument errors detected on the host.
+ */
+int path_attn_frontend_fwd(const void* z, const float* conv_w, const float* beta_logit, const float* gate_logit,
+                           void* w, float* beta, float* log_f, int B, int H, int L, int d, float eps,
+                           void* cuda_stream);
+int path_attn_frontend_bwd(const void* z, const float* conv_w, const float* beta_logit, const float* gate_logit,
+                           const void* dw, const float* dbeta, const float* dlog_f, void* dz, float* dconv_w,
+                           float* dbeta_logit, float* dgate_logit, int B, int H, int L, int d, float eps,
+                           void* cuda_stream);
+
 /* Reads the device status word the last call on this workspace left behind.
  * Synchronises `cuda_stream`.  Returns PATH_OK, PATH_ERR_TIMEOUT, or
  * PATH_ERR_LAUNCH if the copy itself failed.  If `detail` is not NULL it

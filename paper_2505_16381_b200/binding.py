@@ -19,6 +19,7 @@ PATH_BF16, PATH_FP32 = 0, 1
 PATH_OK = 0
 EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_attn_fwd_static", "path_attn_device_status",
            "path_attn_prefill_cache", "path_attn_decode_workspace_bytes", "path_attn_decode_step",
+           "path_attn_frontend_fwd", "path_attn_frontend_bwd",
            "path_attn_strerror", "path_attn_last_cuda_error", "path_attn_last_launch_count",
            "path_attn_profile_enable", "path_attn_profile_read", "path_attn_profile_stage_name"]
 
@@ -55,6 +56,10 @@ def load():
         lib.path_attn_decode_workspace_bytes.argtypes = [I, I, I, I]
         lib.path_attn_decode_step.restype = I
         lib.path_attn_decode_step.argtypes = [P] * 9 + [I, I, P, P, I, I, I, F, I, P, Z, P]
+        lib.path_attn_frontend_fwd.restype = I
+        lib.path_attn_frontend_fwd.argtypes = [P] * 7 + [I, I, I, I, F, P]
+        lib.path_attn_frontend_bwd.restype = I
+        lib.path_attn_frontend_bwd.argtypes = [P] * 11 + [I, I, I, I, F, P]
         lib.path_attn_device_status.restype = I
         lib.path_attn_device_status.argtypes = [P, P, ctypes.POINTER(ctypes.c_uint)]
         lib.path_attn_strerror.restype = ctypes.c_char_p
@@ -258,3 +263,64 @@ def path_attn_decode_step(q_t, k_t, v_t, w_t, beta_t, cache, t, log_f_t=None, sc
     if rc != PATH_OK:
         raise PathAttnError(rc, "path_attn_decode_step")
     return o, lse
+
+
+# ----------------------------------------------------------------------------------------- layer front-end
+
+def _frontend_check(z, conv_w, beta_logit, gate_logit, H):
+    B, L, C = z.shape
+    if C % H:
+        raise ValueError("z's channel count must be a multiple of H")
+    d = C // H
+    if z.dtype != torch.bfloat16:
+        raise ValueError("z must be bf16")
+    if conv_w.shape != (C, 3) or conv_w.dtype != torch.float32:
+        raise ValueError("conv_w must be float32 [H*d, 3]")
+    for x in (beta_logit, gate_logit):
+        if x is not None and (x.shape != (B, L, H) or x.dtype != torch.float32):
+            raise ValueError("logits must be float32 [B, L, H]")
+    for x in (z, conv_w, beta_logit, gate_logit):
+        if x is not None and not (x.is_cuda and x.is_contiguous()):
+            raise ValueError("front-end inputs must be contiguous CUDA tensors")
+    return B, L, d
+
+
+def path_attn_frontend_fwd(z, conv_w, beta_logit, gate_logit=None, H=1, eps=1e-6):
+    """``z`` ``[B,L,H*d]`` bf16, ``conv_w`` ``[H*d,3]``, logits ``[B,L,H]`` float32 -> ``(w [B,H,L,d] bf16, beta, log_f [B,H,L])``."""
+    B, L, d = _frontend_check(z, conv_w, beta_logit, gate_logit, H)
+    lib = load()
+    w = torch.empty(B, H, L, d, dtype=torch.bfloat16, device=z.device)
+    beta = torch.empty(B, H, L, dtype=torch.float32, device=z.device)
+    log_f = torch.empty_like(beta) if gate_logit is not None else None
+    st = torch.cuda.current_stream(z.device).cuda_stream
+    with torch.cuda.device(z.device):
+        rc = lib.path_attn_frontend_fwd(_ptr(z), _ptr(conv_w), _ptr(beta_logit), _ptr(gate_logit), _ptr(w), _ptr(beta),
+                                        _ptr(log_f), B, H, L, d, float(eps), ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_frontend_fwd")
+    return w, beta, log_f
+
+
+def path_attn_frontend_bwd(z, conv_w, beta_logit, dw, dbeta, gate_logit=None, dlog_f=None, H=1, eps=1e-6):
+    """Backward of :func:`path_attn_frontend_fwd`: returns ``(dz, dconv_w, dbeta_logit, dgate_logit or None)``."""
+    B, L, d = _frontend_check(z, conv_w, beta_logit, gate_logit, H)
+    if dw.shape != (B, H, L, d) or dw.dtype != torch.bfloat16 or dbeta.shape != (B, H, L) or dbeta.dtype != torch.float32:
+        raise ValueError("dw must be bf16 [B,H,L,d] and dbeta float32 [B,H,L]")
+    if (gate_logit is None) != (dlog_f is None):
+        raise ValueError("gate_logit and dlog_f go together")
+    for x in (dw, dbeta, dlog_f):
+        if x is not None and not (x.is_cuda and x.is_contiguous()):
+            raise ValueError("front-end gradients must be contiguous CUDA tensors")
+    lib = load()
+    dz = torch.empty_like(z)
+    dcw = torch.empty_like(conv_w)
+    dbl = torch.empty_like(beta_logit)
+    dgl = torch.empty_like(gate_logit) if gate_logit is not None else None
+    st = torch.cuda.current_stream(z.device).cuda_stream
+    with torch.cuda.device(z.device):
+        rc = lib.path_attn_frontend_bwd(_ptr(z), _ptr(conv_w), _ptr(beta_logit), _ptr(gate_logit), _ptr(dw), _ptr(dbeta),
+                                        _ptr(dlog_f), _ptr(dz), _ptr(dcw), _ptr(dbl), _ptr(dgl), B, H, L, d, float(eps),
+                                        ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_frontend_bwd")
+    return dz, dcw, dbl, dgl

@@ -164,5 +164,12 @@ cudaError_t launch_decode_step(const void* q_t, const void* k_t, const void* v_t
 // Float32 forward by the definition (PATH_FP32): q, k, v, w, o are [S][L][hd] float, G the gate prefix [S][ldG] or nullptr.
 cudaError_t launch_fp32_fwd(const float* q, const float* k, const float* v, const float* w, const float* beta, const float* G,
                             float* o, float* lse, int S, int L, int ldG, int hd, float scale, cudaStream_t st);
+// Layer front-end (paper Sec. 2.2 footnote, Sec. 2.4 gate): z [B][L][H*hd] bf16 and logits [B][L][H] -> w [B][H][L][hd] bf16,
+// beta / log f [B][H][L]; and the backward (dcw must be zero on entry: CTAs add into it).
+cudaError_t launch_frontend_fwd(const void* z, const float* cw, const float* bl, const float* gl, void* w, float* beta,
+                                float* logf, int B, int H, int L, int hd, float eps, cudaStream_t st);
+cudaError_t launch_frontend_bwd(const void* z, const float* cw, const float* bl, const float* gl, const void* dw,
+                                const float* dbeta, const float* dlogf, void* dz, float* dcw, float* dbl, float* dgl, int B,
+                                int H, int L, int hd, float eps, cudaStream_t st);
 
 }  // namespace path

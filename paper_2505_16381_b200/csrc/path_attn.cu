@@ -620,6 +620,43 @@ int path_attn_decode_step(const void* q_t, const void* k_t, const void* v_t, con
     return PATH_OK;
 }
 
+// ------------------------------------------------------------------------------------------- layer front-end
+static int frontend_shape_ok(int B, int H, int L, int d) {
+    if (B < 1 || H < 1 || L < 1 || (d != 64 && d != 128)) return 0;
+    const size_t blocks = ((size_t)L + 127) / 128 * (size_t)B * H;
+    return blocks <= 0x7fffffffull;
+}
+
+int path_attn_frontend_fwd(const void* z, const float* conv_w, const float* beta_logit, const float* gate_logit, void* w,
+                           float* beta, float* log_f, int B, int H, int L, int d, float eps, void* cuda_stream) {
+    g_launches = 0;
+    if (!z || !conv_w || !beta_logit || !w || !beta) return PATH_ERR_NULL;
+    if ((gate_logit == nullptr) != (log_f == nullptr)) return PATH_ERR_NULL;
+    if (!frontend_shape_ok(B, H, L, d) || !(eps >= 0.f)) return PATH_ERR_SHAPE;
+    if (!aligned16(z) || !aligned16(w)) return PATH_ERR_ALIGN;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    LAUNCH(launch_frontend_fwd(z, conv_w, beta_logit, gate_logit, w, beta, log_f, B, H, L, d, eps, (cudaStream_t)cuda_stream));
+    return PATH_OK;
+}
+
+int path_attn_frontend_bwd(const void* z, const float* conv_w, const float* beta_logit, const float* gate_logit, const void* dw,
+                           const float* dbeta, const float* dlog_f, void* dz, float* dconv_w, float* dbeta_logit,
+                           float* dgate_logit, int B, int H, int L, int d, float eps, void* cuda_stream) {
+    g_launches = 0;
+    if (!z || !conv_w || !beta_logit || !dw || !dbeta || !dz || !dconv_w || !dbeta_logit) return PATH_ERR_NULL;
+    if ((gate_logit == nullptr) != (dlog_f == nullptr) || (gate_logit == nullptr) != (dgate_logit == nullptr)) return PATH_ERR_NULL;
+    if (!frontend_shape_ok(B, H, L, d) || !(eps >= 0.f)) return PATH_ERR_SHAPE;
+    if (!aligned16(z) || !aligned16(dw) || !aligned16(dz)) return PATH_ERR_ALIGN;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CK(cudaMemsetAsync(dconv_w, 0, (size_t)H * d * 3 * sizeof(float), st));
+    LAUNCH(launch_frontend_bwd(z, conv_w, beta_logit, gate_logit, dw, dbeta, dlog_f, dz, dconv_w, dbeta_logit, dgate_logit, B, H,
+                               L, d, eps, st));
+    return PATH_OK;
+}
+
 int path_attn_device_status(const void* workspace, void* cuda_stream, unsigned int* detail) {
     if (!workspace) return PATH_ERR_NULL;
     unsigned int word = 0;

@@ -68,6 +68,30 @@ def make_inputs(B, H, L, d, dtype="bf16", qk_scaled=True, gate=False, seed=BASE_
     }
 
 
+def make_frontend_inputs(B, H, L, d, gate=False, seed=BASE_SEED):
+    """Random inputs of the layer front-end (CPU tensors): z ``[B,L,H*d]`` bf16 ~ N(0,1), conv_w ``[H*d,3]`` float32
+    ~ N(0,1/3), beta_logit ``[B,L,H]`` ~ N(0,1), gate_logit ~ N(3,1) or None, and upstream gradients dw ``[B,H,L,d]``
+    bf16, dbeta, dlog_f ``[B,H,L]`` float32 ~ N(0,1).  Draw order as listed."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(int(seed))
+
+    def draw(*shape):
+        return torch.randn(*shape, generator=gen, dtype=torch.float32)
+
+    z = draw(B, L, H * d)
+    conv_w = draw(H * d, 3) / 3 ** 0.5
+    beta_logit = draw(B, L, H)
+    gate_logit = draw(B, L, H) + 3.0
+    dw = draw(B, H, L, d)
+    dbeta = draw(B, H, L)
+    dlog_f = draw(B, H, L)
+    return {
+        "z": z.to(torch.bfloat16).contiguous(), "conv_w": conv_w.contiguous(), "beta_logit": beta_logit.contiguous(),
+        "gate_logit": gate_logit.contiguous() if gate else None, "dw": dw.to(torch.bfloat16).contiguous(),
+        "dbeta": dbeta.contiguous(), "dlog_f": dlog_f.contiguous() if gate else None,
+    }
+
+
 def make_config(name: str):
     """Inputs of one of the named workloads (seed = BASE_SEED + its index)."""
     c = CONFIGS[name]
