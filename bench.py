@@ -461,6 +461,63 @@ def run_decode(args):
     print(json.dumps(line), flush=True)
 
 
+def run_frontend(args):
+    """Layer front-end arm (paper Sec. 2.2 footnote, Sec. 2.4 gate), 1 GPU: one step = forward (z, logits -> w, beta, log f)
+    plus backward (dw, dbeta, dlog f -> dz, dconv_w, dlogits) at the paper's benchmark shape B=32, H=32, L=4096, d=64
+    with the gate.  One JSON line; the roofline entry is the backward kernel (the longer of the two): algorithmic bytes
+    per (b, h, t) row = 2d (z) + 2d (dw) + 2d (dz) + 24 (six float32 scalars) against the measured copy bandwidth."""
+    from paper_2505_16381_b200 import binding
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    B, H, L, d, gate = (args.batch or 32), 32, 4096, 64, True
+    inp = synth.make_frontend_inputs(B, H, L, d, gate, seed=synth.BASE_SEED)
+    x = {n: (t.to(dev) if torch.is_tensor(t) else t) for n, t in inp.items()}
+    fwd = lambda: binding.path_attn_frontend_fwd(x["z"], x["conv_w"], x["beta_logit"], x["gate_logit"], H=H)
+    bwd = lambda: binding.path_attn_frontend_bwd(x["z"], x["conv_w"], x["beta_logit"], x["dw"], x["dbeta"], x["gate_logit"],
+                                                 x["dlog_f"], H=H)
+    for _ in range(args.warmup):
+        fwd(); bwd()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    marks = [(ev(), ev(), ev()) for _ in range(args.steps)]
+    sampler = ClockSampler(physical_gpu_index(0))
+    torch.cuda.synchronize()
+    sampler.start()
+    for a, b, c in marks:      # the tensors of one step (2.9 GB at the default shape) exceed L2: no flush needed
+        a.record(); fwd(); b.record(); bwd(); c.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = marks[0][0].elapsed_time(marks[-1][2]) / args.steps
+    ms_f = sum(a.elapsed_time(b) for a, b, _ in marks) / args.steps
+    ms_b = sum(b.elapsed_time(c) for _, b, c in marks) / args.steps
+    rows = B * H * L
+    byt_f, byt_b = rows * (4 * d + 16), rows * (6 * d + 24)
+    peaks = load_peaks()
+    gbs = byt_b / (ms_b * 1e-3) / 1e9
+    line = {"metric": "PaTH layer front-end positions/s (forward + backward, all heads)", "value": B * L / (ms * 1e-3),
+            "unit": "positions/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"front-end: B={B} H={H} L={L} d={d} gate={gate}, bf16 z / w / dw / dz, float32 scalars",
+                       "l2_policy": "tensors exceed L2 (no flush needed)"},
+            "clocks": clocks, "gpu_launches": 2 * args.steps,
+            "roofline": {"kernel": "frontend_bwd_kernel", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm"], "traffic": None, "peak_source": f"{peaks['source']} copy bandwidth",
+                         "bytes_per_launch": byt_b},
+            "detail": {"fwd_ms": ms_f, "bwd_ms": ms_b, "fwd_GBps": byt_f / (ms_f * 1e-3) / 1e9, "fwd_bytes_per_launch": byt_f}}
+    if not args.no_cpu_baseline:
+        from oracle import frontend_oracle as fo
+        import time
+        Ls = 256                                             # one batch row, the first 256 positions, all heads
+        f64 = lambda t: None if t is None else synth.to_f64(t[:1, :Ls] if t.shape[1] == L else t[:1, :, :Ls])
+        t0 = time.perf_counter()
+        fo.frontend_fwd(f64(inp["z"]), synth.to_f64(inp["conv_w"]), f64(inp["beta_logit"]), f64(inp["gate_logit"]), H, 1e-6)
+        fo.frontend_bwd(f64(inp["z"]), synth.to_f64(inp["conv_w"]), f64(inp["beta_logit"]), f64(inp["gate_logit"]),
+                        f64(inp["dw"]), f64(inp["dbeta"]), f64(inp["dlog_f"]), H, 1e-6)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": Ls / dt, "unit": "positions/s", "cores": 1, "kind": "oracle",
+                                "sample": f"B=1, first {Ls} positions, all {H} heads, forward + backward"}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -470,12 +527,16 @@ def main():
     ap.add_argument("--workload", default="C3", choices=[n for n, c in synth.CONFIGS.items() if c["backward"]])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling captures)")
-    ap.add_argument("--path", choices=["train", "decode"], default="train",
-                    help="train: the fwd+bwd step (the headline); decode: the inference arm (1 GPU, not part of the headline)")
+    ap.add_argument("--path", choices=["train", "decode", "frontend"], default="train",
+                    help="train: the fwd+bwd step (the headline); decode: the inference arm; frontend: the layer front-end "
+                         "kernels (both 1 GPU, not part of the headline)")
     args = ap.parse_args()
     if args.path == "decode":
         args.warmup = max(args.warmup, 3)
         return run_decode(args)
+    if args.path == "frontend":
+        args.warmup = max(args.warmup, 3)
+        return run_frontend(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = dict(synth.CONFIGS[args.workload])
     if args.batch > 0:
