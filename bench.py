@@ -49,6 +49,10 @@ NCU_TRAFFIC_BYTES_PER_SLICE = {
     "bwd_chunk_chain": (283.98e6 + 33.74e6) / 16,
 }
 
+# DRAM bytes per launch of frontend_bwd_kernel PER BATCH ROW at H=32, L=4096, d=64 with the gate, from the ncu capture at
+# batch 16 summarised under profiles/ (573.75 MB read + 255.09 MB written); batch rows are independent.
+NCU_FRONTEND_BWD_TRAFFIC_PER_BATCH_ROW = (573.75e6 + 255.09e6) / 16
+
 
 # ----------------------------------------------------------------------------------------- FLOP models
 def flops_m1(B, H, L, d):
@@ -500,8 +504,8 @@ def run_frontend(args):
                        "l2_policy": "tensors exceed L2 (no flush needed)"},
             "clocks": clocks, "gpu_launches": 2 * args.steps,
             "roofline": {"kernel": "frontend_bwd_kernel", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm"], "traffic": None, "peak_source": f"{peaks['source']} copy bandwidth",
-                         "bytes_per_launch": byt_b},
+                         "frac": gbs / peaks["hbm"], "traffic": NCU_FRONTEND_BWD_TRAFFIC_PER_BATCH_ROW * B,
+                         "peak_source": f"{peaks['source']} copy bandwidth", "bytes_per_launch": byt_b},
             "detail": {"fwd_ms": ms_f, "bwd_ms": ms_b, "fwd_GBps": byt_f / (ms_f * 1e-3) / 1e9, "fwd_bytes_per_launch": byt_f}}
     if not args.no_cpu_baseline:
         from oracle import frontend_oracle as fo
