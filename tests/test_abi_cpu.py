@@ -79,6 +79,29 @@ def test_backward_rejects_bad_arguments_on_the_host(lib):
     assert bwd(n=4096) == -5
 
 
+def test_frontend_rejects_bad_arguments_on_the_host(lib):
+    P = 0x2000
+    def fwd(**kw):
+        a = dict(z=P, cw=P, bl=P, gl=None, w=P, beta=P, log_f=None, B=1, H=2, L=16, d=64, eps=1e-6)
+        a.update(kw)
+        return lib.path_attn_frontend_fwd(a["z"], a["cw"], a["bl"], a["gl"], a["w"], a["beta"], a["log_f"], a["B"], a["H"],
+                                          a["L"], a["d"], a["eps"], None)
+    def bwd(**kw):
+        a = dict(z=P, cw=P, bl=P, gl=None, dw=P, dbeta=P, dlog_f=None, dz=P, dcw=P, dbl=P, dgl=None, B=1, H=2, L=16, d=128,
+                 eps=1e-6)
+        a.update(kw)
+        return lib.path_attn_frontend_bwd(a["z"], a["cw"], a["bl"], a["gl"], a["dw"], a["dbeta"], a["dlog_f"], a["dz"],
+                                          a["dcw"], a["dbl"], a["dgl"], a["B"], a["H"], a["L"], a["d"], a["eps"], None)
+    assert fwd(z=None) == -1 and fwd(beta=None) == -1
+    assert fwd(gl=P) == -1 and fwd(log_f=P) == -1          # gate logits and log_f go together
+    assert fwd(d=96) == -2 and fwd(L=0) == -2 and fwd(H=0) == -2 and fwd(eps=-1.0) == -2
+    assert fwd(z=P + 8) == -4 and fwd(w=P + 2) == -4
+    assert bwd(dw=None) == -1 and bwd(dcw=None) == -1
+    assert bwd(gl=P) == -1 and bwd(gl=P, dlog_f=P) == -1 and bwd(dgl=P) == -1
+    assert bwd(d=32) == -2 and bwd(B=0) == -2
+    assert bwd(dz=P + 8) == -4
+
+
 def test_strerror_and_counters(lib):
     seen = set()
     for code in range(0, -9, -1):
