@@ -50,8 +50,8 @@ NCU_TRAFFIC_BYTES_PER_SLICE = {
 }
 
 # DRAM bytes per launch of frontend_bwd_kernel PER BATCH ROW at H=32, L=4096, d=64 with the gate, from the ncu capture at
-# batch 16 summarised under profiles/ (573.75 MB read + 255.09 MB written); batch rows are independent.
-NCU_FRONTEND_BWD_TRAFFIC_PER_BATCH_ROW = (573.75e6 + 255.09e6) / 16
+# batch 16 summarised under profiles/ (573.76 MB read + 255.33 MB written); batch rows are independent.
+NCU_FRONTEND_BWD_TRAFFIC_PER_BATCH_ROW = (573.76e6 + 255.33e6) / 16
 
 
 # ----------------------------------------------------------------------------------------- FLOP models

@@ -7,12 +7,12 @@
 // change of layout that the operator wants, so no separate transpose pass exists.
 //
 // Work split.  A lane holds 8 adjacent channels of a row (one 16-byte load), so a row of a head takes d/8 lanes and a
-// warp holds 32/(d/8) lane groups.  Each group walks over 8 consecutive positions with the filter's window in
-// registers.  The rows a lane will need are fetched by 16-byte asynchronous copies into a slot of shared memory that only
-// this lane reads back (a per-lane queue, so no barrier is involved: the lane waits for its own copy group), several
-// position blocks ahead of the one being computed: the bytes in flight, which is what a bandwidth-bound kernel lives on,
-// sit in shared memory instead of registers.  A CTA is 4 warps = 128 (d = 64) or 64 (d = 128) consecutive positions of one head; CTAs are numbered
-// with the head fastest, so the CTAs that run at the same time read whole contiguous rows of z between them, and each
+// warp holds 32/(d/8) lane groups.  Each group walks over R consecutive positions (5 or 8, see FwdR / BwdR) with the
+// filter's window in registers.  The rows a lane will need are fetched by 16-byte asynchronous copies into a slot of
+// shared memory that only this lane reads back (a per-lane queue, so no barrier is involved: the lane waits for its own
+// copy group), one position block ahead of the one being computed: the bytes in flight, which is what a
+// bandwidth-bound kernel lives on, sit in shared memory instead of registers.  A CTA is 4 warps = 4 * (256 / d) * R
+// consecutive positions of one head; CTAs are numbered with the head fastest, so the CTAs that run at the same time read whole contiguous rows of z between them, and each
 // loops over the position blocks of its head with a stride (the backward keeps its filter-gradient sums in registers
 // across that loop and adds them to global memory once).
 #include "common.cuh"
@@ -21,15 +21,21 @@ namespace path {
 
 namespace {
 
-constexpr int kR = 8, kWarps = 4;   // positions per lane group, warps per CTA
+constexpr int kWarps = 4;   // warps per CTA
 
-template <int HD>
+template <int HD, int R>   // R = consecutive positions per lane group
 struct Geo {
     static constexpr int LPR = HD / 8;        // lanes per row
     static constexpr int G = 32 / LPR;        // lane groups per warp
-    static constexpr int ROWS_W = G * kR;     // positions per warp
+    static constexpr int ROWS_W = G * R;      // positions per warp
     static constexpr int ROWS_CTA = kWarps * ROWS_W;
+    static_assert(ROWS_W <= 32, "one lane per position fetches its scalars");
 };
+// Positions per lane group, by measurement (TB/s of algorithmic bytes at B=32 H=32 L=4096 d=64 / B=8 H=32 L=8192 d=128):
+// forward d = 64: 5.3 / 5.7 / 4.9 at 4 / 5 / 8;  forward d = 128: 5.5 / 5.9 / 5.8 at 5 / 6 / 8;
+// backward d = 64: 3.4 / 3.9 / 4.2 at 5 / 6 / 8;  backward d = 128: 3.7 / 4.0 / 4.0 at 5 / 8 / 10.
+template <int HD> struct FwdR { static constexpr int value = HD == 64 ? 5 : 8; };
+template <int HD> struct BwdR { static constexpr int value = 8; };
 
 // 16-byte asynchronous copy global -> shared; copies nothing and writes zeros when `valid` is false
 __device__ __forceinline__ void cp_async16(uint4* dst, const void* src, bool valid) {
@@ -86,14 +92,16 @@ __device__ __forceinline__ void st16(__nv_bfloat16* p, const float2 (&x)[4]) {
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
 
 constexpr int kThreads = 32 * kWarps;
-constexpr int kFwdRows = kR + 2, kFwdStages = 2;          // z rows t0-2 .. t0+7 per lane and block
-constexpr int kBwdRows = (kR + 4) + (kR + 2), kBwdStages = 2;   // z rows t0-2 .. t0+9, then dw rows t0 .. t0+9
+constexpr int kFwdStages = 2, kBwdStages = 2;
+__host__ __device__ constexpr int fwd_rows(int R) { return R + 2; }               // z rows t0-2 .. t0+R-1 per lane and block
+__host__ __device__ constexpr int bwd_rows(int R) { return (R + 4) + (R + 2); }   // z rows t0-2 .. t0+R+1, then dw rows t0 .. t0+R+1
 
 template <int HD>
 __global__ void __launch_bounds__(kThreads, 4) frontend_fwd_kernel(
     const __nv_bfloat16* __restrict__ z, const float* __restrict__ cw, const float* __restrict__ bl, const float* __restrict__ gl,
     __nv_bfloat16* __restrict__ w, float* __restrict__ beta, float* __restrict__ logf, int B, int H, int L, int nblk, float eps) {
-    typedef Geo<HD> Ge;
+    constexpr int kR = FwdR<HD>::value, kFwdRows = fwd_rows(kR);
+    typedef Geo<HD, kR> Ge;
     extern __shared__ uint4 queue[];   // [stage][row][thread]: every slot is written and read by the same thread
     float* lq = reinterpret_cast<float*>(queue + kFwdStages * kFwdRows * kThreads);   // [stage][beta, gate logit][thread]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, grp = lane / Ge::LPR, li = lane % Ge::LPR;
@@ -184,7 +192,8 @@ __global__ void __launch_bounds__(kThreads, 2) frontend_bwd_kernel(
     const __nv_bfloat16* __restrict__ dw, const float* __restrict__ dbeta, const float* __restrict__ dlogf,
     __nv_bfloat16* __restrict__ dz, float* dcw, float* __restrict__ dbl, float* __restrict__ dgl, int B, int H, int L, int nblk,
     float eps) {
-    typedef Geo<HD> Ge;
+    constexpr int kR = BwdR<HD>::value, kBwdRows = bwd_rows(kR);
+    typedef Geo<HD, kR> Ge;
     extern __shared__ uint4 queue[];   // [stage][row][thread]; reused for the reduction of the filter gradient at the end
     float* lq = reinterpret_cast<float*>(queue + kBwdStages * kBwdRows * kThreads);   // [stage][4 scalars][thread]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, grp = lane / Ge::LPR, li = lane % Ge::LPR;
@@ -335,12 +344,14 @@ cudaError_t ctas_per_head(int B, int H, int nblk, int per_sm, int* out) {
 cudaError_t launch_frontend_fwd(const void* z, const float* cw, const float* bl, const float* gl, void* w, float* beta,
                                 float* logf, int B, int H, int L, int hd, float eps, cudaStream_t st) {
     typedef __nv_bfloat16 bf;
-    const int rows = hd == 64 ? Geo<64>::ROWS_CTA : Geo<128>::ROWS_CTA, nblk = (L + rows - 1) / rows;
+    const int rows = hd == 64 ? Geo<64, FwdR<64>::value>::ROWS_CTA : Geo<128, FwdR<128>::value>::ROWS_CTA;
+    const int nblk = (L + rows - 1) / rows;
     int W = 1;
     cudaError_t e = ctas_per_head(B, H, nblk, 4, &W);
     if (e != cudaSuccess) return e;
     const dim3 grid((unsigned)((size_t)H * W));
-    constexpr int smem = kFwdStages * (kFwdRows * (int)sizeof(uint4) + 2 * (int)sizeof(float)) * kThreads;
+    auto smem_of = [](int R) { return kFwdStages * (fwd_rows(R) * (int)sizeof(uint4) + 2 * (int)sizeof(float)) * kThreads; };
+    const int smem = smem_of(hd == 64 ? FwdR<64>::value : FwdR<128>::value);
     if (hd == 64) {
         e = cudaFuncSetAttribute(frontend_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
@@ -357,13 +368,17 @@ cudaError_t launch_frontend_bwd(const void* z, const float* cw, const float* bl,
                                 const float* dbeta, const float* dlogf, void* dz, float* dcw, float* dbl, float* dgl, int B,
                                 int H, int L, int hd, float eps, cudaStream_t st) {
     typedef __nv_bfloat16 bf;
-    const int rows = hd == 64 ? Geo<64>::ROWS_CTA : Geo<128>::ROWS_CTA, nblk = (L + rows - 1) / rows;
+    const int rows = hd == 64 ? Geo<64, BwdR<64>::value>::ROWS_CTA : Geo<128, BwdR<128>::value>::ROWS_CTA;
+    const int nblk = (L + rows - 1) / rows;
     int W = 1;
     cudaError_t e = ctas_per_head(B, H, nblk, 2, &W);
     if (e != cudaSuccess) return e;
     const dim3 grid((unsigned)((size_t)H * W));
-    constexpr int smem = kBwdStages * (kBwdRows * (int)sizeof(uint4) + 4 * (int)sizeof(float)) * kThreads;
-    static_assert(smem >= kWarps * 4 * 128 * 3 * (int)sizeof(float), "the queue also holds the filter-gradient partials");
+    auto smem_of = [](int R) { return kBwdStages * (bwd_rows(R) * (int)sizeof(uint4) + 4 * (int)sizeof(float)) * kThreads; };
+    const int smem = smem_of(hd == 64 ? BwdR<64>::value : BwdR<128>::value);
+    static_assert(kBwdStages * bwd_rows(1) * (int)sizeof(uint4) * kThreads >= kWarps * 4 * 64 * 3 * (int)sizeof(float) &&
+                      kBwdStages * bwd_rows(1) * (int)sizeof(uint4) * kThreads >= kWarps * 2 * 128 * 3 * (int)sizeof(float),
+                  "the queue also holds the filter-gradient partials");
     if (hd == 64) {
         e = cudaFuncSetAttribute(frontend_bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
