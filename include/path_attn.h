@@ -193,6 +193,19 @@ int path_attn_frontend_bwd(const void* z, const float* conv_w, const float* beta
                            float* dbeta_logit, float* dgate_logit, int B, int H, int L, int d, float eps,
                            void* cuda_stream);
 
+/*
+ * Block skipping in gated problems (the paper notes, Sec. 2.4, that PaTH-FoX stays compatible with FoX's pruning of
+ * negligible blocks).  When log_f is given, path_attn_fwd leaves out every (query chunk, key chunk) pair of 128 x 128
+ * positions whose logits are all provably more than 30 nats below the largest logit of their rows (the bound uses
+ * |k| |q|, the norm bounds of the H_t in between and the accumulated gate; exp(-30) is far below bf16 resolution), and
+ * with it every farther key chunk of that query chunk.  Results are unchanged within the stated tolerances; plain PaTH
+ * (log_f == NULL) never skips.  This call reports, for the last gated path_attn_fwd on `workspace` (until another call
+ * uses the workspace), how many chunk pairs were computed and how many a full causal sweep has.  Synchronises
+ * `cuda_stream`.
+ */
+int path_attn_skipped_chunk_pairs(const void* workspace, void* cuda_stream, unsigned long long* kept,
+                                  unsigned long long* all);
+
 /* Reads the device status word the last call on this workspace left behind.
  * Synchronises `cuda_stream`.  Returns PATH_OK, PATH_ERR_TIMEOUT, or
  * PATH_ERR_LAUNCH if the copy itself failed.  If `detail` is not NULL it

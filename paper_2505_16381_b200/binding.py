@@ -19,7 +19,7 @@ PATH_BF16, PATH_FP32 = 0, 1
 PATH_OK = 0
 EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_attn_fwd_static", "path_attn_device_status",
            "path_attn_prefill_cache", "path_attn_decode_workspace_bytes", "path_attn_decode_step",
-           "path_attn_frontend_fwd", "path_attn_frontend_bwd",
+           "path_attn_frontend_fwd", "path_attn_frontend_bwd", "path_attn_skipped_chunk_pairs",
            "path_attn_strerror", "path_attn_last_cuda_error", "path_attn_last_launch_count",
            "path_attn_profile_enable", "path_attn_profile_read", "path_attn_profile_stage_name"]
 
@@ -60,6 +60,8 @@ def load():
         lib.path_attn_frontend_fwd.argtypes = [P] * 7 + [I, I, I, I, F, P]
         lib.path_attn_frontend_bwd.restype = I
         lib.path_attn_frontend_bwd.argtypes = [P] * 11 + [I, I, I, I, F, P]
+        lib.path_attn_skipped_chunk_pairs.restype = I
+        lib.path_attn_skipped_chunk_pairs.argtypes = [P, P, ctypes.POINTER(ctypes.c_ulonglong), ctypes.POINTER(ctypes.c_ulonglong)]
         lib.path_attn_device_status.restype = I
         lib.path_attn_device_status.argtypes = [P, P, ctypes.POINTER(ctypes.c_uint)]
         lib.path_attn_strerror.restype = ctypes.c_char_p
@@ -186,6 +188,18 @@ def device_status(workspace) -> int:
     if rc != PATH_OK:
         raise PathAttnError(rc, f"path_attn_device_status (word 0x{detail.value:x})")
     return int(detail.value)
+
+
+def skipped_chunk_pairs(workspace):
+    """(kept, all) chunk pairs of the last gated forward on ``workspace`` (block skipping; synchronises the stream)."""
+    lib = load()
+    kept, total = ctypes.c_ulonglong(0), ctypes.c_ulonglong(0)
+    st = torch.cuda.current_stream(workspace.device).cuda_stream
+    with torch.cuda.device(workspace.device):
+        rc = lib.path_attn_skipped_chunk_pairs(_ptr(workspace), ctypes.c_void_p(st), ctypes.byref(kept), ctypes.byref(total))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_skipped_chunk_pairs")
+    return kept.value, total.value
 
 
 def last_launch_count() -> int:

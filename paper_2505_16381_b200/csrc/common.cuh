@@ -51,6 +51,7 @@ struct FwdParams {
     void* o;            // [S, L, HD] bf16 or f32
     float* lse;         // [S, L]
     const float* G;     // [S, Lp] inclusive prefix of the log gate, or nullptr
+    const int* nkeep;   // [S, N] key chunks each query chunk has to visit (gated problems), or nullptr = all
     uint32_t* status;   // device status word
     int S, L, Lp, N;
     float scale;

@@ -134,6 +134,9 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
         I = (j & 1) ? (j >> 1) : p.N - 1 - (j >> 1);
         return true;
     };
+    // key chunks a work item visits, counted from the diagonal: all I + 1 of them, or fewer when the gate has made the
+    // far ones negligible (every warp role reads the same precomputed number)
+    auto steps_of = [&](int I, int s) { return p.nkeep ? min(I + 1, p.nkeep[s * p.N + I]) : I + 1; };
     auto ver_row = [&](int s, int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
 
     if (warp < 4) {
@@ -166,7 +169,7 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
             };
             int I, s;
             for (int it = 0; ok && item_of(it, I, s); ++it) {
-                const int NS = I + 1;
+                const int NS = steps_of(I, s);
                 const int rowRaw = s * p.Lp + I * kTile;
                 // diagonal chunk: raw q, k and the correction operands (both K slots), V of chunk I
                 load_q(&tm.q_raw, HD, rowRaw);
@@ -215,9 +218,9 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
             auto release_q = [&](int upto) {
                 for (; released < upto; ++released) umma_commit(&bars[B_QEMPTY + released % 3]);
             };
-            int I, s_unused;
-            for (; ok && item_of(item, I, s_unused); ++item) {
-                const int NS = I + 1;
+            int I, s_it;
+            for (; ok && item_of(item, I, s_it); ++item) {
+                const int NS = steps_of(I, s_it);
                 int cur_level = -1;
                 int q_of0, q_of1;              // operand index used by each stream's most recent S product
                 auto advance_q = [&](int n) {  // operand index of step n >= 1 (waits for a newly needed one)
@@ -314,7 +317,7 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
 
         int I, s;
         for (; item_of(item, I, s); ++item) {
-            const int NS = I + 1;
+            const int NS = steps_of(I, s);
             const int qi = I * kTile + row;     // position within the slice (may be >= L in the ragged tail)
             const int TX = (NS - x + 1) >> 1;   // steps of this stream: n = 2t + x
             float gi2 = 0.f;

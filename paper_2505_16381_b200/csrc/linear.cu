@@ -88,6 +88,80 @@ __global__ void __launch_bounds__(1024) gate_suffix_kernel(const float* __restri
     }
 }
 
+// ---- block skipping for gated problems (the paper notes that PaTH-FoX keeps FoX's pruning of negligible blocks)
+//
+// |k_j^T (H_{j+1} ... H_i) q_i| <= |k_j| |q_i| prod_s max(1, |1 - beta_s |w_s|^2|)   (each factor bounds the 2-norm of H_s;
+// it is 1 whenever 0 <= beta_s |w_s|^2 <= 2), and every row's largest logit is at least its own diagonal one,
+// s_ii = scale q_i . k_i.  So if for a pair of chunks (I, J)
+//     |scale| max_I|q| max_J|k| exp(sum of the log factors over chunks J..I) + max_I G - min_J G  <  min_I s_ii - kSkipMargin
+// every probability of the pair is below exp(-kSkipMargin) of its row's normaliser and the pair can be left out.  A
+// query chunk keeps the key chunks up to the farthest one that fails this test.
+constexpr float kSkipMargin = 30.f;   // exp(-30) ~ 1e-13 per logit, far below bf16 resolution even summed over a long row
+
+// stats[tile] = {max|q|, max|k|, max G, min G, min s_ii over real rows, sum of log factors, 0, 0}
+__global__ void __launch_bounds__(256) tile_stats_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                                                        const __nv_bfloat16* __restrict__ w, const float* __restrict__ beta,
+                                                        const float* __restrict__ G, float* __restrict__ stats, int L, int Lp,
+                                                        int hd, float scale) {
+    __shared__ float red[8][6];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int N = Lp / CHUNK, sl = blockIdx.x / N, c = blockIdx.x % N;
+    float qn = 0.f, kn = 0.f, gmax = -INFINITY, gmin = INFINITY, mlo = INFINITY, gam = 0.f;
+    for (int r = warp; r < CHUNK; r += 8) {
+        const int t = c * CHUNK + r;
+        const size_t row = (size_t)sl * Lp + t;
+        float qq = 0.f, kk = 0.f, qk = 0.f, ww = 0.f;
+        for (int e = lane; e < hd / 2; e += 32) {
+            const float2 a = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(q + row * hd)[e]);
+            const float2 b = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(k + row * hd)[e]);
+            const float2 x = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(w + row * hd)[e]);
+            qq += a.x * a.x + a.y * a.y; kk += b.x * b.x + b.y * b.y; qk += a.x * b.x + a.y * b.y; ww += x.x * x.x + x.y * x.y;
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            qq += __shfl_xor_sync(0xffffffffu, qq, off); kk += __shfl_xor_sync(0xffffffffu, kk, off);
+            qk += __shfl_xor_sync(0xffffffffu, qk, off); ww += __shfl_xor_sync(0xffffffffu, ww, off);
+        }
+        const float g = G[row];
+        qn = fmaxf(qn, sqrtf(qq)); kn = fmaxf(kn, sqrtf(kk));
+        gmax = fmaxf(gmax, g); gmin = fminf(gmin, g);
+        if (t < L) mlo = fminf(mlo, scale * qk);
+        gam += logf(fmaxf(1.f, fabsf(1.f - beta[row] * ww)));
+    }
+    if (lane == 0) { red[warp][0] = qn; red[warp][1] = kn; red[warp][2] = gmax; red[warp][3] = gmin; red[warp][4] = mlo; red[warp][5] = gam; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int x = 1; x < 8; ++x) {
+            qn = fmaxf(qn, red[x][0]); kn = fmaxf(kn, red[x][1]); gmax = fmaxf(gmax, red[x][2]); gmin = fminf(gmin, red[x][3]);
+            mlo = fminf(mlo, red[x][4]); gam += red[x][5];
+        }
+        float* o = stats + (size_t)blockIdx.x * 8;
+        // the norms and the growth go up, the row maximum goes down by a rounding margin: the test must err towards keeping
+        o[0] = qn * 1.001f; o[1] = kn * 1.001f; o[2] = gmax; o[3] = gmin; o[4] = mlo - 1e-3f * fabsf(mlo); o[5] = gam * 1.001f + 1e-6f;
+        o[6] = o[7] = 0.f;
+    }
+}
+
+__global__ void __launch_bounds__(128) tile_keep_kernel(const float* __restrict__ stats, int* __restrict__ nkeep,
+                                                       unsigned long long* counters, int S, int N, float ascale) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= S * N) return;
+    const int sl = idx / N, I = idx % N;
+    const float* me = stats + (size_t)idx * 8;
+    const float qn = me[0], gmax = me[2], need = me[4] - kSkipMargin;
+    float acc = 0.f;
+    int keep = 1;
+    for (int n = 0; n <= I; ++n) {
+        const float* o = stats + ((size_t)sl * N + I - n) * 8;
+        acc += o[5];
+        const float bound = ascale * qn * o[1] * expf(acc) + gmax - o[3];
+        if (!(bound < need)) keep = n + 1;   // also keeps everything when a NaN or an infinity is around
+    }
+    nkeep[idx] = keep;
+    atomicAdd(&counters[0], (unsigned long long)keep);
+    atomicAdd(&counters[1], (unsigned long long)(I + 1));
+}
+
 }  // namespace
 
 cudaError_t launch_gate_suffix(const float* dGa, const float* dGb, const float* dGc, float* out, int S, int L, int Lp,
@@ -116,6 +190,18 @@ cudaError_t launch_pad_vec(const float* src, float* dst, int S, int L, int Lp, c
 
 cudaError_t launch_gate_prefix(const float* g, float* G, int S, int L, int Lp, cudaStream_t st) {
     gate_prefix_kernel<<<S, 1024, 0, st>>>(g, G, L, Lp);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gate_skip(const void* q, const void* k, const void* w, const float* beta, const float* G, float* stats,
+                             int* nkeep, unsigned long long* counters, int S, int L, int Lp, int hd, float scale,
+                             cudaStream_t st) {
+    typedef __nv_bfloat16 bf;
+    const int N = Lp / CHUNK;
+    tile_stats_kernel<<<S * N, 256, 0, st>>>((const bf*)q, (const bf*)k, (const bf*)w, beta, G, stats, L, Lp, hd, scale);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    tile_keep_kernel<<<(S * N + 127) / 128, 128, 0, st>>>(stats, nkeep, counters, S, N, fabsf(scale));
     return cudaGetLastError();
 }
 

@@ -18,4 +18,11 @@ cudaError_t launch_gate_suffix(const float* dGa, const float* dGb, const float* 
 // rs[chunk][i] = sum_k dsd[chunk][i][k]
 cudaError_t launch_dsd_rowsum(const float* dsd, float* rs, int nchunks, cudaStream_t st);
 
+// Gated problems (PaTH-FoX): which key chunks a query chunk can skip because the accumulated gate has made every logit
+// of the pair negligible.  stats: [S*N][8] floats of scratch, nkeep: [S*N], counters: {kept pairs, all pairs} (zeroed
+// by the caller).  q, k, w: [S][Lp][hd] bf16 (padded), beta, G: [S][Lp].
+cudaError_t launch_gate_skip(const void* q, const void* k, const void* w, const float* beta, const float* G, float* stats,
+                             int* nkeep, unsigned long long* counters, int S, int L, int Lp, int hd, float scale,
+                             cudaStream_t st);
+
 }  // namespace path

@@ -24,6 +24,10 @@ static thread_local int g_launches = 0;
     } while (0)
 #define LAUNCH(expr) do { CK(expr); ++g_launches; } while (0)
 
+// Status block (the first 256 bytes of a workspace): word 0 = device status; bytes 32..47 = {kept, all} chunk pairs of the
+// last gated forward (two 64-bit counters).
+constexpr size_t kSkipCounterOffset = 32;
+
 // ------------------------------------------------------------------------------------------- stage timing
 // Optional per-thread instrumentation: CUDA events around groups of launches of the most recent call.
 enum Stage { STG_PREP = 0, STG_LEVELS, STG_FA_FWD, STG_PREP_BWD, STG_LEVELS_BWDPREP, STG_ROWSTATS, STG_FA_DKV, STG_FA_DQ,
@@ -118,7 +122,7 @@ struct Plan {
     LevelTable lv;
     size_t total;
     // offsets (bytes)
-    size_t status, qp, kp, vp, wp, betap, G, Dyh, Dyl, Xqn, Yt, Qv16, Kv16;
+    size_t status, qp, kp, vp, wp, betap, G, tstats, nkeep, Dyh, Dyl, Xqn, Yt, Qv16, Kv16;
     // backward only
     size_t dop, delta, lse2, dQv, dKv, dSd, dSdT, dG, dGrow, dGdiag, dDy;
     size_t sTh, sTl, sAh, sAl, sXk, sU;   // bf16 tiles kept by the chunk preparation for the chain rule
@@ -155,7 +159,11 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
         p.qp = bump(cur, SLd * 2); p.kp = bump(cur, SLd * 2); p.vp = bump(cur, SLd * 2); p.wp = bump(cur, SLd * 2);
     }
     p.betap = bump(cur, SL * 4);
-    if (gate) p.G = bump(cur, SL * 4);
+    if (gate) {
+        p.G = bump(cur, SL * 4);
+        p.tstats = bump(cur, (size_t)S * p.N * 8 * 4);   // per-chunk bounds and the resulting key-chunk counts: block skipping
+        p.nkeep = bump(cur, (size_t)S * p.N * 4);
+    }
     const size_t keep = bwd ? 1 : 0;   // bf16 intermediates of the chunk preparation, kept for the chain rule
     p.sTh = bump(cur, keep * SNBB * 2); p.sTl = bump(cur, keep * SNBB * 2);
     p.sAh = bump(cur, keep * SNBB * 2); p.sAl = bump(cur, keep * SNBB * 2);
@@ -463,6 +471,12 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     fp.status = at<uint32_t>(workspace, p.status);
     fp.S = p.S; fp.L = L; fp.Lp = p.Lp; fp.N = p.N; fp.scale = scale; fp.out_fp32 = 0;
     prof_mark(STG_FA_FWD, 0, st);
+    if (log_f) {   // which far key chunks the gate has made negligible (two small kernels, counted with the sweep)
+        fp.nkeep = at<int>(workspace, p.nkeep);
+        LAUNCH(launch_gate_skip(q, k, w, at<float>(workspace, p.betap), fp.G, at<float>(workspace, p.tstats), at<int>(workspace, p.nkeep),
+                                at<unsigned long long>(workspace, p.status + kSkipCounterOffset), p.S, L, p.Lp, d, scale, st));
+        ++g_launches;   // the call above is two launches
+    }
     LAUNCH(launch_fa_fwd(tm, fp, d, st));
     prof_mark(STG_FA_FWD, 1, st);
     if (keep_state) tag_store(tag, true);
@@ -668,6 +682,20 @@ int path_attn_device_status(const void* workspace, void* cuda_stream, unsigned i
     }
     if (detail) *detail = word;
     return word == 0 ? PATH_OK : PATH_ERR_TIMEOUT;
+}
+
+int path_attn_skipped_chunk_pairs(const void* workspace, void* cuda_stream, unsigned long long* kept,
+                                  unsigned long long* all) {
+    if (!workspace || !kept || !all) return PATH_ERR_NULL;
+    unsigned long long c[2] = {0, 0};
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(c, (const uint8_t*)workspace + kSkipCounterOffset, sizeof(c), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        g_last_cuda_error = (int)cudaGetLastError();
+        return PATH_ERR_LAUNCH;
+    }
+    *kept = c[0]; *all = c[1];
+    return PATH_OK;
 }
 
 const char* path_attn_strerror(int status) {

@@ -291,3 +291,64 @@ def test_c5_long_prefill_forward_sampled_rows(binding, oracle):
     lg = lse.reshape(-1, L)[idx][:, rows].cpu().double().numpy()
     assert np.abs(lg - lse_ref).max() <= 2e-3 * max(1.0, np.abs(lse_ref).max())
     assert torch.isfinite(o).all()
+
+
+# ---------------------------------------------------------------- block skipping in gated problems (paper Sec. 2.4 remark)
+
+@pytest.mark.parametrize("L,d,shift,expect", [
+    (2048, 64, -1.0, "most"),     # log f ~ -1.3 per token: only the diagonal and the neighbouring chunk matter
+    (2304, 128, 3.0, "some"),     # the workloads' gate (log f ~ -0.07 per token): a band of a few chunks
+    (1024, 64, 9.0, "none"),      # log f ~ -1e-4 per token: nothing is negligible, nothing may be skipped
+])
+def test_gate_block_skipping_keeps_parity(binding, oracle, L, d, shift, expect):
+    inp = synth.make_inputs(1, 2, L, d, "bf16", gate=True, seed=4000 + L)
+    gen = torch.Generator().manual_seed(4100 + L)
+    inp["log_f"] = torch.nn.functional.logsigmoid(torch.randn(1, 2, L, generator=gen) + shift).contiguous()
+    dev = to_dev(inp)
+    ws = binding.alloc_workspace(dev["q"], True, False)
+    o, lse = binding.path_attn_fwd(dev["q"], dev["k"], dev["v"], dev["w"], dev["beta"], dev["log_f"], workspace=ws)
+    assert binding.device_status(ws) == 0
+    kept, total = binding.skipped_chunk_pairs(ws)
+    N = (L + 127) // 128
+    assert total == 2 * N * (N + 1) // 2
+    if expect == "most":
+        assert 2 * N <= kept <= 2 * 3 * N
+    elif expect == "some":
+        assert 2 * 2 * N <= kept < total
+    else:
+        assert kept == total
+    x = slices(inp, [0, 1])
+    o_ref, lse_ref = oracle.forward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["log_f"])
+    check("o", o.reshape(-1, L, d), o_ref)
+    assert np.abs(lse.reshape(-1, L).cpu().double().numpy() - lse_ref).max() <= 2e-3 * max(1.0, np.abs(lse_ref).max())
+    # the backward after a skipping forward
+    g = gpu_backward(binding, dev, o, lse, 1.0)
+    ref = oracle.backward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["d_o"], x["log_f"])
+    for name, r in ref.items():
+        check(name, g[name].reshape(-1, *g[name].shape[2:]), r)
+
+
+def test_block_skipping_respects_large_logits_and_growing_transitions(binding, oracle):
+    """Keys with a large norm, or transitions with |1 - beta |w|^2| > 1, can outweigh the gate: the bound must see both."""
+    L, d = 1024, 64
+    inp = synth.make_inputs(1, 2, L, d, "bf16", gate=True, seed=4500, qk_scaled=False)   # |q|, |k| ~ 8: logits of +-60
+    gen = torch.Generator().manual_seed(4501)
+    inp["log_f"] = torch.nn.functional.logsigmoid(torch.randn(1, 2, L, generator=gen) + 2.0).contiguous()
+    inp["w"][0, 1] = (inp["w"][0, 1].float() * 1.05).to(torch.bfloat16)     # head 1: |w|^2 = 1.1, growth where beta > 1.8
+    dev = to_dev(inp)
+    ws = binding.alloc_workspace(dev["q"], True, False)
+    o, lse = binding.path_attn_fwd(dev["q"], dev["k"], dev["v"], dev["w"], dev["beta"], dev["log_f"], scale=0.25, workspace=ws)
+    assert binding.device_status(ws) == 0
+    kept, total = binding.skipped_chunk_pairs(ws)
+    assert 0 < kept <= total
+    x = slices(inp, [0, 1])
+    o_ref, lse_ref = oracle.forward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["log_f"], scale=0.25)
+    check("o", o.reshape(-1, L, d), o_ref)
+    assert np.abs(lse.reshape(-1, L).cpu().double().numpy() - lse_ref).max() <= 2e-3 * max(1.0, np.abs(lse_ref).max())
+
+
+def test_plain_path_never_skips(binding):
+    inp = to_dev(synth.make_inputs(1, 2, 1024, 64, "bf16", gate=False, seed=4600))
+    ws = binding.alloc_workspace(inp["q"], False, False)
+    binding.path_attn_fwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"], None, workspace=ws)
+    assert binding.skipped_chunk_pairs(ws) == (0, 0)
