@@ -80,6 +80,7 @@ struct LevelParams {
     float* ddy;
     float* kc;                    // key-cache kernel: [S][cap][d] float32 out (rows < L of every slice)
     int cap, L;
+    const int *nkeep, *nvisit;    // version backward: chunk counts of a sweep shortened by block skipping ([S][N]), or nullptr
     uint32_t* status;
 };
 
@@ -146,6 +147,8 @@ struct BwdParams {
     const float* lse2;   // [S][Lp] (gate prefix - lse) * log2(e)
     const float* delta;  // [S][Lp] -(dO . O)
     const float* G;      // [S][Lp] gate prefix or nullptr
+    const int* nkeep;    // [S][N] key chunks a query chunk has to visit / nvisit: query chunks a key chunk has to meet
+    const int* nvisit;   //        (block skipping in gated problems), or nullptr = all
     void* zero_ptr;      // dK/dV sweep: buffer it clears on the side (32-byte aligned, zero_bytes % 32 == 0), or zero_bytes = 0
     size_t zero_bytes;
     uint32_t* status;

@@ -175,6 +175,9 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
     int J = 0, s = 0;   // current item of this thread's role
     auto ver_row = [&](int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
     auto level = [&](int t) { return t == 0 ? -1 : msb32((unsigned)((J + t) ^ J)); };
+    // query chunks this key chunk meets (I = J .. J + T - 1): all later ones, or fewer when the gate has made the far
+    // pairs negligible (every warp role reads the same precomputed number)
+    auto steps_of = [&](int J, int s) { return p.nvisit ? min(p.N - J, p.nvisit[s * p.N + J]) : p.N - J; };
 
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
@@ -202,7 +205,7 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
             };
 #pragma unroll 1
             for (int it = 0; ok && item_of(it, J, s); ++it) {
-                const int T = p.N - J, rowJ = s * p.Lp + J * kTile;
+                const int T = steps_of(J, s), rowJ = s * p.Lp + J * kTile;
 #pragma unroll 1
                 for (int t = 0; t < T && ok; ++t) {
                     const int I = J + t, l = level(t);
@@ -252,7 +255,7 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
             auto do_addr = [&](int e) { return smem_u32(sDO + (e & 1) * kSlotBytes); };
 #pragma unroll 1
             for (int it = 0; ok && item_of(it, J, s); ++it) {
-                const int T = p.N - J;
+                const int T = steps_of(J, s);
                 // step 0: S^T of the diagonal chunk (two contractions) and its dP^T
                 wait(K_KFULL, nk); ++nk;
                 q_wait(qb);
@@ -323,10 +326,13 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
             // accumulate into: the sweep leaves most of the memory bandwidth unused.
             const uint32_t n32 = (uint32_t)(p.zero_bytes / 32), per = (n32 + gridDim.x - 1) / gridDim.x;   // < 2^32 pieces of 32 bytes
             const uint32_t lo = blockIdx.x * per, hi = lo + per < n32 ? lo + per : n32;
-            for (uint32_t i = lo + (threadIdx.x - 64); i < hi; i += 64) {   // paced, so that the sweep's own stores are not delayed
+            // paced, so that the sweep's own stores are not delayed; a sweep shortened by block skipping would end up
+            // waiting for the pacing instead, so there the clearing runs at full speed
+            const bool paced = p.nvisit == nullptr;
+            for (uint32_t i = lo + (threadIdx.x - 64); i < hi; i += 64) {
                 asm volatile("st.global.v8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"l"((uint8_t*)p.zero_ptr + (size_t)i * 32), "r"(0u)
                              : "memory");
-                __nanosleep(300);
+                if (paced) __nanosleep(300);
             }
         }
     } else {
@@ -440,7 +446,7 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
         };
 #pragma unroll 1
         for (int it = 0; item_of(it, J, s); ++it) {
-            const int T = p.N - J;
+            const int T = steps_of(J, s);
             const int kj = J * kTile + row;          // key position of this thread's row
             if (GATE) {
                 const float gj2 = p.G[(size_t)s * p.Lp + kj] * kLog2e;
@@ -464,11 +470,14 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
                 mbar_arrive(&bars[K_ACCFREE]);
                 break;
             }
-            if (T > 1) flush_dk(level(T - 1));
-            else {  // last chunk: no later query chunk, the boundary-adjusted keys get a zero gradient from the sweep
-                uint4* dst = reinterpret_cast<uint4*>(p.dkv + ((size_t)ver_row(0, J) + row) * HD + h * CW);
+            auto zero_dk = [&](int slot) {
+                uint4* dst = reinterpret_cast<uint4*>(p.dkv + ((size_t)ver_row(slot, J) + row) * HD + h * CW);
                 for (int x = 0; x < CW / 8; ++x) dst[x] = make_uint4(0u, 0u, 0u, 0u);
-            }
+            };
+            if (T > 1) flush_dk(level(T - 1));
+            else zero_dk(0);   // no later query chunk met: the boundary-adjusted keys get a zero gradient from the sweep
+            // (levels that a sweep shortened by block skipping did not reach stay unwritten: the version chain rule starts
+            // at the highest level reached)
             if (CW == 64) {   // 64 bf16 = one 128-byte line per row: coalesced exchange
                 uint32_t r0[32], r1[32], w[32];
                 tmem_ld32(tlane + colDV + h * CW, r0);
@@ -565,6 +574,9 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
     int I = 0, s = 0;
     auto ver_row = [&](int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
     auto level = [&](int t) { return msb32((unsigned)(I ^ (I - 1 - t))); };
+    // earlier key chunks this query chunk visits (J = I-1 .. I-T): all of them, or fewer when the gate has made the far
+    // ones negligible (every warp role reads the same precomputed number; the diagonal chunk is not part of this sweep)
+    auto steps_of = [&](int I, int s) { return p.nkeep ? min(I, p.nkeep[s * p.N + I] - 1) : I; };
 
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
@@ -576,7 +588,7 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
             };
 #pragma unroll 1
             for (int it = 0; ok && item_of(it, I, s); ++it) {
-                const int T = I;
+                const int T = steps_of(I, s);
                 if (T == 0) continue;
                 wait_empty(Q_DOEMPTY, nd);
                 if (!ok) break;
@@ -643,7 +655,7 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
             };
 #pragma unroll 1
             for (int it = 0; ok && item_of(it, I, s); ++it) {
-                T = I;
+                T = steps_of(I, s);
                 if (T == 0) continue;
                 wait(Q_DOFULL, nd); ++nd;
                 issue_s(0);
@@ -683,10 +695,16 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
         };
 #pragma unroll 1
         for (int it = 0; item_of(it, I, s); ++it) {
-            const int T = I;
-            if (T == 0) {  // chunk 0 has no earlier keys: its boundary-adjusted queries get a zero gradient from the sweep
-                uint4* dst = reinterpret_cast<uint4*>(p.dqv + (size_t)s * p.Lp * HD);
+            const int T = steps_of(I, s);
+            auto zero_dq = [&](int slot) {   // a whole [128 x HD] version gradient tile, by the 256 math threads
+                uint4* dst = reinterpret_cast<uint4*>(p.dqv + (size_t)ver_row(slot, I) * HD);
                 for (int i = threadIdx.x - 128; i < kTile * HD / 8; i += 256) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+            };
+            // no key chunk visited (chunk 0, or block skipping left only the diagonal): the boundary-adjusted queries get a
+            // zero gradient from the sweep.  Levels that a shortened sweep does not reach stay unwritten: the version
+            // chain rule starts at the highest level reached.
+            if (T == 0) {
+                zero_dq(0);
                 continue;
             }
             const size_t qi = (size_t)s * p.Lp + I * kTile + row;

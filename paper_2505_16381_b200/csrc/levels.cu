@@ -254,7 +254,21 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
             if (version_step(is_key, ch, l, p.N, l1, b, src)) return l;
         return 0;
     };
-    int l2 = next_step(p.l - 1);
+    // A sweep shortened by block skipping has written the gradients of the levels it reached only (the near ones); the
+    // chain starts at the highest of them instead of the top (everything above would have been zero).
+    int top = p.l - 1;
+    if (p.nkeep) {
+        int reached = 0;
+        if (is_key) {
+            const int T = min(p.N - ch, p.nvisit[s * p.N + ch]);          // query chunks ch .. ch + T - 1 were met
+            if (T > 1) reached = msb32((unsigned)((ch + T - 1) ^ ch));
+        } else {
+            const int T = min(ch, p.nkeep[s * p.N + ch] - 1);             // key chunks ch - 1 .. ch - T were visited
+            if (T > 0) reached = msb32((unsigned)(ch ^ (ch - T)));
+        }
+        top = min(top, reached);
+    }
+    int l2 = next_step(top);
     if (l2 == 0) return;   // no chain: what the sweeps left in slot 0 is final
     __nv_bfloat16* dxv = is_key ? p.dkv : p.dqv;
     extern __shared__ uint8_t smem_raw[];

@@ -99,26 +99,34 @@ __global__ void __launch_bounds__(1024) gate_suffix_kernel(const float* __restri
 constexpr float kSkipMargin = 30.f;   // exp(-30) ~ 1e-13 per logit, far below bf16 resolution even summed over a long row
 
 // stats[tile] = {max|q|, max|k|, max G, min G, min s_ii over real rows, sum of log factors, 0, 0}
+// A row takes hd/8 lanes (16-byte loads), so a warp works on 2 (hd = 128) or 4 (hd = 64) rows at a time.
 __global__ void __launch_bounds__(256) tile_stats_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                                                         const __nv_bfloat16* __restrict__ w, const float* __restrict__ beta,
                                                         const float* __restrict__ G, float* __restrict__ stats, int L, int Lp,
                                                         int hd, float scale) {
     __shared__ float red[8][6];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lpr = hd / 8, grp = lane / lpr, li = lane % lpr, rows_w = 32 / lpr;
     const int N = Lp / CHUNK, sl = blockIdx.x / N, c = blockIdx.x % N;
     float qn = 0.f, kn = 0.f, gmax = -INFINITY, gmin = INFINITY, mlo = INFINITY, gam = 0.f;
-    for (int r = warp; r < CHUNK; r += 8) {
+    auto dot8 = [](const uint4& a, const uint4& b) {
+        const uint32_t x[4] = {a.x, a.y, a.z, a.w}, y[4] = {b.x, b.y, b.z, b.w};
+        float acc = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            acc = fmaf(__uint_as_float(x[i] << 16), __uint_as_float(y[i] << 16), acc);
+            acc = fmaf(__uint_as_float(x[i] & 0xffff0000u), __uint_as_float(y[i] & 0xffff0000u), acc);
+        }
+        return acc;
+    };
+    for (int r = warp * rows_w + grp; r < CHUNK; r += 8 * rows_w) {
         const int t = c * CHUNK + r;
         const size_t row = (size_t)sl * Lp + t;
-        float qq = 0.f, kk = 0.f, qk = 0.f, ww = 0.f;
-        for (int e = lane; e < hd / 2; e += 32) {
-            const float2 a = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(q + row * hd)[e]);
-            const float2 b = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(k + row * hd)[e]);
-            const float2 x = __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(w + row * hd)[e]);
-            qq += a.x * a.x + a.y * a.y; kk += b.x * b.x + b.y * b.y; qk += a.x * b.x + a.y * b.y; ww += x.x * x.x + x.y * x.y;
-        }
-#pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) {
+        const uint4 a = *reinterpret_cast<const uint4*>(q + row * hd + li * 8);
+        const uint4 b = *reinterpret_cast<const uint4*>(k + row * hd + li * 8);
+        const uint4 x = *reinterpret_cast<const uint4*>(w + row * hd + li * 8);
+        float qq = dot8(a, a), kk = dot8(b, b), qk = dot8(a, b), ww = dot8(x, x);
+        for (int off = lpr / 2; off >= 1; off >>= 1) {
             qq += __shfl_xor_sync(0xffffffffu, qq, off); kk += __shfl_xor_sync(0xffffffffu, kk, off);
             qk += __shfl_xor_sync(0xffffffffu, qk, off); ww += __shfl_xor_sync(0xffffffffu, ww, off);
         }
@@ -127,6 +135,12 @@ __global__ void __launch_bounds__(256) tile_stats_kernel(const __nv_bfloat16* __
         gmax = fmaxf(gmax, g); gmin = fminf(gmin, g);
         if (t < L) mlo = fminf(mlo, scale * qk);
         gam += logf(fmaxf(1.f, fabsf(1.f - beta[row] * ww)));
+    }
+    // the lanes of a group hold the same values; combine the groups of the warp (the growth sum counts each group once)
+    for (int off = lpr; off < 32; off <<= 1) {
+        qn = fmaxf(qn, __shfl_xor_sync(0xffffffffu, qn, off)); kn = fmaxf(kn, __shfl_xor_sync(0xffffffffu, kn, off));
+        gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, off)); gmin = fminf(gmin, __shfl_xor_sync(0xffffffffu, gmin, off));
+        mlo = fminf(mlo, __shfl_xor_sync(0xffffffffu, mlo, off)); gam += __shfl_xor_sync(0xffffffffu, gam, off);
     }
     if (lane == 0) { red[warp][0] = qn; red[warp][1] = kn; red[warp][2] = gmax; red[warp][3] = gmin; red[warp][4] = mlo; red[warp][5] = gam; }
     __syncthreads();
@@ -162,6 +176,18 @@ __global__ void __launch_bounds__(128) tile_keep_kernel(const float* __restrict_
     atomicAdd(&counters[1], (unsigned long long)(I + 1));
 }
 
+// nvisit[s][J] = query chunks the key chunk J has to meet in a sweep over I = J, J+1, ...: up to the farthest query chunk
+// whose kept range still reaches J (the chunks in between are visited too: a superset is always safe)
+__global__ void __launch_bounds__(128) tile_visit_kernel(const int* __restrict__ nkeep, int* __restrict__ nvisit, int S, int N) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= S * N) return;
+    const int sl = idx / N, J = idx % N;
+    int far = J;
+    for (int I = N - 1; I > J; --I)
+        if (I - nkeep[sl * N + I] + 1 <= J) { far = I; break; }
+    nvisit[idx] = far - J + 1;
+}
+
 }  // namespace
 
 cudaError_t launch_gate_suffix(const float* dGa, const float* dGb, const float* dGc, float* out, int S, int L, int Lp,
@@ -194,14 +220,20 @@ cudaError_t launch_gate_prefix(const float* g, float* G, int S, int L, int Lp, c
 }
 
 cudaError_t launch_gate_skip(const void* q, const void* k, const void* w, const float* beta, const float* G, float* stats,
-                             int* nkeep, unsigned long long* counters, int S, int L, int Lp, int hd, float scale,
+                             int* nkeep, int* nvisit, unsigned long long* counters, int S, int L, int Lp, int hd, float scale,
                              cudaStream_t st) {
     typedef __nv_bfloat16 bf;
     const int N = Lp / CHUNK;
-    tile_stats_kernel<<<S * N, 256, 0, st>>>((const bf*)q, (const bf*)k, (const bf*)w, beta, G, stats, L, Lp, hd, scale);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    tile_keep_kernel<<<(S * N + 127) / 128, 128, 0, st>>>(stats, nkeep, counters, S, N, fabsf(scale));
+    cudaError_t e = cudaSuccess;
+    if (stats != nullptr) {   // otherwise nkeep is already there (the forward of this problem computed it)
+        tile_stats_kernel<<<S * N, 256, 0, st>>>((const bf*)q, (const bf*)k, (const bf*)w, beta, G, stats, L, Lp, hd, scale);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        tile_keep_kernel<<<(S * N + 127) / 128, 128, 0, st>>>(stats, nkeep, counters, S, N, fabsf(scale));
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess || nvisit == nullptr) return e;
+    tile_visit_kernel<<<(S * N + 127) / 128, 128, 0, st>>>(nkeep, nvisit, S, N);
     return cudaGetLastError();
 }
 

@@ -62,6 +62,7 @@ static void prof_mark(int stage, int end, cudaStream_t st) {
 struct StateTag {
     const void *ws, *q, *k, *v, *w, *beta, *log_f;
     int B, H, L, d;
+    float scale;   // not part of the identity (the chunk preparation does not depend on it); the block-skipping counts do
 };
 static std::mutex g_tag_mutex;
 static StateTag g_tags[64];
@@ -79,10 +80,13 @@ static void tag_store(const StateTag& t, bool valid) {   // valid = false: forge
     g_tags[g_tag_next] = t;
     g_tag_next = (g_tag_next + 1) % 64;
 }
-static bool tag_matches(const StateTag& t) {
+static bool tag_matches(const StateTag& t, bool* same_scale = nullptr) {
     std::lock_guard<std::mutex> lock(g_tag_mutex);
     for (const auto& e : g_tags)
-        if (e.ws == t.ws) return tag_equal(e, t);
+        if (e.ws == t.ws) {
+            if (same_scale) *same_scale = e.scale == t.scale;
+            return tag_equal(e, t);
+        }
     return false;
 }
 
@@ -122,7 +126,7 @@ struct Plan {
     LevelTable lv;
     size_t total;
     // offsets (bytes)
-    size_t status, qp, kp, vp, wp, betap, G, tstats, nkeep, Dyh, Dyl, Xqn, Yt, Qv16, Kv16;
+    size_t status, qp, kp, vp, wp, betap, G, tstats, nkeep, nvisit, Dyh, Dyl, Xqn, Yt, Qv16, Kv16;
     // backward only
     size_t dop, delta, lse2, dQv, dKv, dSd, dSdT, dG, dGrow, dGdiag, dDy;
     size_t sTh, sTl, sAh, sAl, sXk, sU;   // bf16 tiles kept by the chunk preparation for the chain rule
@@ -163,6 +167,7 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
         p.G = bump(cur, SL * 4);
         p.tstats = bump(cur, (size_t)S * p.N * 8 * 4);   // per-chunk bounds and the resulting key-chunk counts: block skipping
         p.nkeep = bump(cur, (size_t)S * p.N * 4);
+        p.nvisit = bump(cur, (size_t)S * p.N * 4);
     }
     const size_t keep = bwd ? 1 : 0;   // bf16 intermediates of the chunk preparation, kept for the chain rule
     p.sTh = bump(cur, keep * SNBB * 2); p.sTl = bump(cur, keep * SNBB * 2);
@@ -328,7 +333,7 @@ static int run_chunk_chain(const Plan& p, void* ws, const void* q, const void* k
 
 static int run_backward(const Plan& p, void* ws, const void* q, const void* k, const void* v, const void* w,
                         const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
-                        float* dbeta, float* dlog_f, float scale, cudaStream_t st) {
+                        float* dbeta, float* dlog_f, float scale, bool reuse_keep, cudaStream_t st) {
     const int d = p.d;
     float* dDy = at<float>(ws, p.dDy);
     __nv_bfloat16* dQv = at<__nv_bfloat16>(ws, p.dQv); __nv_bfloat16* dKv = at<__nv_bfloat16>(ws, p.dKv);
@@ -358,6 +363,15 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     bp.status = at<uint32_t>(ws, p.status);
     bp.zero_ptr = dDy; bp.zero_bytes = p.dy_bytes;   // cleared by the dK/dV sweep, first accumulated into by the version chains
     bp.S = p.S; bp.L = p.L; bp.Lp = p.Lp; bp.N = p.N; bp.scale = scale;
+    if (p.gate) {   // chunk pairs the gate has made negligible are left out of both sweeps (three small kernels)
+        bp.nkeep = at<int>(ws, p.nkeep); bp.nvisit = at<int>(ws, p.nvisit);
+        // (a forward whose preparation is being reused has left its per-query-chunk counts, and the counters, in place)
+        if (!reuse_keep) CK(cudaMemsetAsync(at<uint8_t>(ws, p.status + kSkipCounterOffset), 0, 16, st));
+        LAUNCH(launch_gate_skip(q, k, w, at<float>(ws, p.betap), bp.G, reuse_keep ? nullptr : at<float>(ws, p.tstats),
+                                at<int>(ws, p.nkeep), at<int>(ws, p.nvisit),
+                                at<unsigned long long>(ws, p.status + kSkipCounterOffset), p.S, p.L, p.Lp, d, scale, st));
+        if (!reuse_keep) g_launches += 2;
+    }
     prof_mark(STG_ROWSTATS, 1, st);
     prof_mark(STG_FA_DKV, 0, st);
     LAUNCH(launch_fa_bwd(tm, bp, d, 0, st));
@@ -373,6 +387,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
         LevelTensorMaps ltm;
         if (!make_level_maps(p, ws, ltm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
         LevelParams lp = level_params(p, ws);
+        if (p.gate) { lp.nkeep = at<int>(ws, p.nkeep); lp.nvisit = at<int>(ws, p.nvisit); }
         lp.l = p.nlev;
         LAUNCH(launch_level_kernel(LEVEL_VERSION_BWD, ltm, lp, d, st));
         for (int l = p.nlev - 2; l >= 1; --l) {
@@ -424,7 +439,7 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
         if (rc32 != PATH_OK) return rc32;
         cudaStream_t st32 = (cudaStream_t)cuda_stream;
         CK(cudaMemsetAsync(workspace, 0, 256, st32));
-        tag_store(StateTag{workspace, q, k, v, w, beta, log_f, B, H, L, d}, false);   // this call overwrites the workspace
+        tag_store(StateTag{workspace, q, k, v, w, beta, log_f, B, H, L, d, scale}, false);   // this call overwrites the workspace
         float* G = nullptr;
         if (log_f) {
             G = at<float>(workspace, p.G);
@@ -436,7 +451,7 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     }
     // A workspace large enough for the backward gets the backward's layout: the chunk preparation then also keeps
     // the tiles the chain rule needs, and path_attn_bwd on the same workspace and inputs does not redo it.
-    const StateTag tag{workspace, q, k, v, w, beta, log_f, B, H, L, d};
+    const StateTag tag{workspace, q, k, v, w, beta, log_f, B, H, L, d, scale};
     bool keep_state = false;
     {
         Plan pb;
@@ -474,7 +489,8 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     if (log_f) {   // which far key chunks the gate has made negligible (two small kernels, counted with the sweep)
         fp.nkeep = at<int>(workspace, p.nkeep);
         LAUNCH(launch_gate_skip(q, k, w, at<float>(workspace, p.betap), fp.G, at<float>(workspace, p.tstats), at<int>(workspace, p.nkeep),
-                                at<unsigned long long>(workspace, p.status + kSkipCounterOffset), p.S, L, p.Lp, d, scale, st));
+                                nullptr, at<unsigned long long>(workspace, p.status + kSkipCounterOffset), p.S, L, p.Lp, d, scale,
+                                st));
         ++g_launches;   // the call above is two launches
     }
     LAUNCH(launch_fa_fwd(tm, fp, d, st));
@@ -503,10 +519,11 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
     int rc = check_arch();
     if (rc != PATH_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    CK(cudaMemsetAsync(workspace, 0, 256, st));
+    CK(cudaMemsetAsync(workspace, 0, kSkipCounterOffset, st));   // the status word; the block-skipping counters may be reused
     prof_reset(STG_PREP_BWD, STG_COUNT);
-    const StateTag tag{workspace, q, k, v, w, beta, log_f, B, H, L, d};
-    const bool reuse = tag_matches(tag);   // the forward of this very problem left its preparation in this workspace
+    const StateTag tag{workspace, q, k, v, w, beta, log_f, B, H, L, d, scale};
+    bool same_scale = false;
+    const bool reuse = tag_matches(tag, &same_scale);   // the forward of this very problem left its preparation in this workspace
     if (!reuse) tag_store(tag, false);
     rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, !reuse, st);
     if (rc != PATH_OK) return rc;
@@ -515,7 +532,7 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
         if (rc != PATH_OK) return rc;
         tag_store(tag, true);
     }
-    return run_backward(p, workspace, q, k, v, w, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, scale, st);
+    return run_backward(p, workspace, q, k, v, w, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, scale, reuse && same_scale, st);
 }
 
 }  // extern "C"

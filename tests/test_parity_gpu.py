@@ -352,3 +352,26 @@ def test_plain_path_never_skips(binding):
     ws = binding.alloc_workspace(inp["q"], False, False)
     binding.path_attn_fwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"], None, workspace=ws)
     assert binding.skipped_chunk_pairs(ws) == (0, 0)
+
+
+def test_backward_recomputes_the_skip_counts_when_the_scale_differs(binding, oracle):
+    """A forward at one scale leaves its chunk counts in the workspace; a backward at another scale on the same workspace
+    and tensors may reuse the chunk preparation but not those counts (the bound depends on the scale)."""
+    L, d = 1536, 64
+    inp = synth.make_inputs(1, 2, L, d, "bf16", gate=True, seed=4700, qk_scaled=False)
+    gen = torch.Generator().manual_seed(4701)
+    inp["log_f"] = torch.nn.functional.logsigmoid(torch.randn(1, 2, L, generator=gen) + 1.0).contiguous()
+    dev = to_dev(inp)
+    ws = binding.alloc_workspace(dev["q"], True, True)
+    args = (dev["q"], dev["k"], dev["v"], dev["w"], dev["beta"])
+    binding.path_attn_fwd(*args, dev["log_f"], scale=0.01, workspace=ws)       # tiny logits: short kept ranges
+    small = binding.skipped_chunk_pairs(ws)[0]
+    ws2 = binding.alloc_workspace(dev["q"], True, False)
+    o, lse = binding.path_attn_fwd(*args, dev["log_f"], scale=0.5, workspace=ws2)   # logits of +-30: longer ranges
+    assert binding.skipped_chunk_pairs(ws2)[0] > small
+    g = binding.path_attn_bwd(*args, o, lse, dev["d_o"], dev["log_f"], scale=0.5, workspace=ws)
+    assert binding.device_status(ws) == 0
+    x = slices(inp, [0, 1])
+    ref = oracle.backward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["d_o"], x["log_f"], scale=0.5)
+    for name, r in ref.items():
+        check(name, g[name].reshape(-1, *g[name].shape[2:]), r)
