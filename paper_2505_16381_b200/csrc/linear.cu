@@ -48,16 +48,23 @@ __global__ void __launch_bounds__(1024) gate_prefix_kernel(const float* __restri
     }
 }
 
-// rs[chunk*128 + i] = sum_k dsd[chunk][i][k]; one warp per row.
+// rs[chunk*128 + i] = sum_k dsd[chunk][i][k]; one warp per row (a lane reads four adjacent entries), four rows in flight.
 __global__ void __launch_bounds__(256) dsd_rowsum_kernel(const float* __restrict__ dsd, float* __restrict__ rs) {
-    const size_t base = (size_t)blockIdx.x * CHUNK * CHUNK;
+    const float4* base = reinterpret_cast<const float4*>(dsd + (size_t)blockIdx.x * CHUNK * CHUNK);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int r = warp; r < CHUNK; r += 8) {
-        float acc = 0.f;
-        for (int c = lane; c < CHUNK; c += 32) acc += dsd[base + r * CHUNK + c];
+#pragma unroll 1
+    for (int r0 = warp * 16; r0 < warp * 16 + 16; r0 += 4) {
+        float4 v[4];
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (lane == 0) rs[(size_t)blockIdx.x * CHUNK + r] = acc;
+        for (int x = 0; x < 4; ++x) v[x] = base[(r0 + x) * (CHUNK / 4) + lane];
+        float acc[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) acc[x] = (v[x].x + v[x].y) + (v[x].z + v[x].w);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) acc[x] += __shfl_xor_sync(0xffffffffu, acc[x], off);
+        if (lane < 4) rs[(size_t)blockIdx.x * CHUNK + r0 + lane] = lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3];
     }
 }
 
