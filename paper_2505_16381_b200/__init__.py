@@ -6,4 +6,4 @@ the library; the first call does, and fails loudly if it has not been built.
 """
 from . import synth  # noqa: F401
 
-__all__ = ["synth", "binding", "build"]
+__all__ = ["synth", "binding", "build", "autograd"]
