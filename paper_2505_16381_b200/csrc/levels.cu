@@ -183,20 +183,34 @@ __global__ void __launch_bounds__(256, 1) dyadic_fwd_kernel(const __grid_constan
 // grid = (S * N, 2): y = 0 queries, y = 1 keys; p.l = number of levels.  One CTA walks the whole chain of its chunk,
 // bottom level first:  Xv[l2] = Xv[l1] * Dy (queries) or Dy^T (keys).  The version just produced stays in shared
 // memory as the next step's left operand (the same bf16 values that go to global memory).
+// Highest dyadic level at which chunk `ch` of slice `s` takes part in a chunk pair the sweeps compute: every level for a
+// plain problem; for a gated one the level of the farthest kept pair (0 = only level 0 or none: no version chain).
+__device__ __forceinline__ int highest_level_reached(const LevelParams& p, int is_key, int s, int ch) {
+    if (!p.nkeep) return 30;
+    if (is_key) {
+        const int T = min(p.N - ch, p.nvisit[s * p.N + ch]);          // query chunks ch .. ch + T - 1 meet this key chunk
+        return T > 1 ? msb32((unsigned)((ch + T - 1) ^ ch)) : 0;
+    }
+    const int T = min(ch, p.nkeep[s * p.N + ch] - 1);                 // key chunks ch - 1 .. ch - T are visited
+    return T > 0 ? msb32((unsigned)(ch ^ (ch - T))) : 0;
+}
+
 template <int HD>
 __global__ void __launch_bounds__(256, 2) version_fwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
     const int is_key = blockIdx.y, s = blockIdx.x / p.N, ch = blockIdx.x % p.N;
+    // levels to build: all of them, or for a gated problem up to the highest one a kept chunk pair uses (see version_bwd)
+    const int lim = min(p.l, highest_level_reached(p, is_key, s, ch) + 1);
     int l1, b, src, l2 = 1;
-    for (; l2 < p.l; ++l2)
+    for (; l2 < lim; ++l2)
         if (version_step(is_key, ch, l2, p.N, l1, b, src)) break;
-    if (l2 >= p.l) return;
+    if (l2 >= lim) return;
     extern __shared__ uint8_t smem_raw[];
     Ctx c;
     setup<128>(c, smem_raw, kBar3);
     uint8_t* sm = c.smem;   // slots: 0 current version, 1 Dy hi, 2 Dy lo
     bool first = true;
 #pragma unroll 1
-    for (; l2 < p.l && c.ok; ++l2) {
+    for (; l2 < lim && c.ok; ++l2) {
         if (!version_step(is_key, ch, l2, p.N, l1, b, src)) continue;
         const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
         const long row_dst = ((long)l2 * p.S + s) * p.Lp + (long)ch * kT;
@@ -256,18 +270,7 @@ __global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_consta
     };
     // A sweep shortened by block skipping has written the gradients of the levels it reached only (the near ones); the
     // chain starts at the highest of them instead of the top (everything above would have been zero).
-    int top = p.l - 1;
-    if (p.nkeep) {
-        int reached = 0;
-        if (is_key) {
-            const int T = min(p.N - ch, p.nvisit[s * p.N + ch]);          // query chunks ch .. ch + T - 1 were met
-            if (T > 1) reached = msb32((unsigned)((ch + T - 1) ^ ch));
-        } else {
-            const int T = min(ch, p.nkeep[s * p.N + ch] - 1);             // key chunks ch - 1 .. ch - T were visited
-            if (T > 0) reached = msb32((unsigned)(ch ^ (ch - T)));
-        }
-        top = min(top, reached);
-    }
+    const int top = min(p.l - 1, highest_level_reached(p, is_key, s, ch));
     int l2 = next_step(top);
     if (l2 == 0) return;   // no chain: what the sweeps left in slot 0 is final
     __nv_bfloat16* dxv = is_key ? p.dkv : p.dqv;

@@ -163,8 +163,8 @@ __global__ void __launch_bounds__(256) tile_stats_kernel(const __nv_bfloat16* __
     }
 }
 
-__global__ void __launch_bounds__(128) tile_keep_kernel(const float* __restrict__ stats, int* __restrict__ nkeep,
-                                                       unsigned long long* counters, int S, int N, float ascale) {
+__global__ void __launch_bounds__(128) tile_keep_kernel(const float* __restrict__ stats, int* __restrict__ nkeep, int S, int N,
+                                                       float ascale) {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= S * N) return;
     const int sl = idx / N, I = idx % N;
@@ -179,20 +179,62 @@ __global__ void __launch_bounds__(128) tile_keep_kernel(const float* __restrict_
         if (!(bound < need)) keep = n + 1;   // also keeps everything when a NaN or an infinity is around
     }
     nkeep[idx] = keep;
-    atomicAdd(&counters[0], (unsigned long long)keep);
-    atomicAdd(&counters[1], (unsigned long long)(I + 1));
 }
 
-// nvisit[s][J] = query chunks the key chunk J has to meet in a sweep over I = J, J+1, ...: up to the farthest query chunk
-// whose kept range still reaches J (the chunks in between are visited too: a superset is always safe)
-__global__ void __launch_bounds__(128) tile_visit_kernel(const int* __restrict__ nkeep, int* __restrict__ nvisit, int S, int N) {
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= S * N) return;
-    const int sl = idx / N, J = idx % N;
-    int far = J;
-    for (int I = N - 1; I > J; --I)
-        if (I - nkeep[sl * N + I] + 1 <= J) { far = I; break; }
-    nvisit[idx] = far - J + 1;
+// One CTA per slice.  First the kept ranges are made a staircase: the first kept key chunk of a query chunk never lies
+// after that of a later query chunk (ranges only grow, which is always safe).  Then "key chunk J is kept by query chunk I"
+// holds for exactly the I in J .. far(J), so the key-major sweep of the backward (nvisit[J] = far(J) - J + 1 query chunks)
+// computes the same pairs as the query-major sweeps, and every version a sweep asks for lies within the levels its chunk
+// reaches.  Also counts the kept pairs.
+__global__ void __launch_bounds__(128) tile_stair_kernel(int* __restrict__ nkeep, int* __restrict__ nvisit,
+                                                        unsigned long long* counters, int S, int N) {
+    // one CTA per slice; the two serial scans run on a copy in shared memory when it fits (N <= kStairMax chunks, i.e.
+    // sequences up to a million tokens), else directly on global memory
+    constexpr int kStairMax = 8192;
+    __shared__ int snk[kStairMax];
+    const int sl = blockIdx.x;
+    int* gk = nkeep + (size_t)sl * N;
+    int* gv = nvisit + (size_t)sl * N;
+    const bool in_smem = N <= kStairMax;
+    if (in_smem) {
+        for (int i = threadIdx.x; i < N; i += blockDim.x) snk[i] = gk[i];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        int* nk = in_smem ? snk : gk;
+        unsigned long long kept = 0;
+        int start = N;
+        for (int I = N - 1; I >= 0; --I) {
+            start = min(start, I - nk[I] + 1);
+            nk[I] = I - start + 1;
+            kept += (unsigned long long)nk[I];
+        }
+        if (in_smem) {   // nvisit is written below by all threads from the staircase
+            atomicAdd(&counters[0], kept);
+        } else {
+            int far = 0;
+            for (int J = 0; J < N; ++J) {
+                far = max(far, J);
+                while (far + 1 < N && far + 1 - nk[far + 1] + 1 <= J) ++far;
+                gv[J] = far - J + 1;
+            }
+            atomicAdd(&counters[0], kept);
+        }
+        atomicAdd(&counters[1], (unsigned long long)N * (N + 1) / 2);
+    }
+    if (!in_smem) return;
+    __syncthreads();
+    // far(J) = the last I whose first kept key chunk I - nk[I] + 1 is <= J; those first chunks do not decrease with I, so a
+    // binary search per J finds it
+    for (int J = threadIdx.x; J < N; J += blockDim.x) {
+        int lo = J, hi = N - 1;   // invariant: chunk lo keeps J (a chunk always keeps itself)
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (mid - snk[mid] + 1 <= J) lo = mid; else hi = mid - 1;
+        }
+        gv[J] = lo - J + 1;
+        gk[J] = snk[J];
+    }
 }
 
 }  // namespace
@@ -231,16 +273,13 @@ cudaError_t launch_gate_skip(const void* q, const void* k, const void* w, const 
                              cudaStream_t st) {
     typedef __nv_bfloat16 bf;
     const int N = Lp / CHUNK;
-    cudaError_t e = cudaSuccess;
-    if (stats != nullptr) {   // otherwise nkeep is already there (the forward of this problem computed it)
-        tile_stats_kernel<<<S * N, 256, 0, st>>>((const bf*)q, (const bf*)k, (const bf*)w, beta, G, stats, L, Lp, hd, scale);
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-        tile_keep_kernel<<<(S * N + 127) / 128, 128, 0, st>>>(stats, nkeep, counters, S, N, fabsf(scale));
-        e = cudaGetLastError();
-    }
-    if (e != cudaSuccess || nvisit == nullptr) return e;
-    tile_visit_kernel<<<(S * N + 127) / 128, 128, 0, st>>>(nkeep, nvisit, S, N);
+    tile_stats_kernel<<<S * N, 256, 0, st>>>((const bf*)q, (const bf*)k, (const bf*)w, beta, G, stats, L, Lp, hd, scale);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    tile_keep_kernel<<<(S * N + 127) / 128, 128, 0, st>>>(stats, nkeep, S, N, fabsf(scale));
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    tile_stair_kernel<<<S, 128, 0, st>>>(nkeep, nvisit, counters, S, N);
     return cudaGetLastError();
 }
 

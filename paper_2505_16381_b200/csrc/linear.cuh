@@ -19,10 +19,9 @@ cudaError_t launch_gate_suffix(const float* dGa, const float* dGb, const float* 
 cudaError_t launch_dsd_rowsum(const float* dsd, float* rs, int nchunks, cudaStream_t st);
 
 // Gated problems (PaTH-FoX): which key chunks a query chunk can skip because the accumulated gate has made every logit
-// of the pair negligible.  stats: [S*N][8] floats of scratch, nkeep: [S*N], counters: {kept pairs, all pairs} (zeroed
-// by the caller).  q, k, w: [S][Lp][hd] bf16 (padded), beta, G: [S][Lp].  nvisit: [S*N] or nullptr: the same knowledge
-// seen from the key chunks (how many query chunks each has to meet), for the backward's key-major sweep.  stats ==
-// nullptr: nkeep is taken as given (an earlier call on the same problem computed it) and only nvisit is produced.
+// of the pair negligible.  stats: [S*N][8] floats of scratch; nkeep: [S*N] key chunks each query chunk visits (counted
+// from the diagonal); nvisit: [S*N] query chunks each key chunk meets (the same pairs, key-major); counters: {kept pairs,
+// all pairs}, added to (zeroed by the caller).  q, k, w: [S][Lp][hd] bf16 (padded), beta, G: [S][Lp].
 cudaError_t launch_gate_skip(const void* q, const void* k, const void* w, const float* beta, const float* G, float* stats,
                              int* nkeep, int* nvisit, unsigned long long* counters, int S, int L, int Lp, int hd, float scale,
                              cudaStream_t st);

@@ -220,8 +220,20 @@ static LevelParams level_params(const Plan& p, void* ws) {
     if (p.bwd) {
         lp.dqv = at<__nv_bfloat16>(ws, p.dQv); lp.dkv = at<__nv_bfloat16>(ws, p.dKv); lp.ddy = at<float>(ws, p.dDy);
     }
+    if (p.gate) { lp.nkeep = at<int>(ws, p.nkeep); lp.nvisit = at<int>(ws, p.nvisit); }   // block skipping (see run_gate_skip)
     lp.status = at<uint32_t>(ws, p.status);
     return lp;
+}
+
+// Gated problems: which chunk pairs the sweeps can leave out (counts per query chunk and per key chunk, three small
+// kernels).  Runs before the chunk preparation: the version chains stop at the highest level a kept pair uses.
+static int run_gate_skip(const Plan& p, void* ws, const void* q, const void* k, const void* w, float scale, cudaStream_t st) {
+    CK(cudaMemsetAsync(at<uint8_t>(ws, p.status + kSkipCounterOffset), 0, 16, st));
+    LAUNCH(launch_gate_skip(q, k, w, at<float>(ws, p.betap), at<float>(ws, p.G), at<float>(ws, p.tstats), at<int>(ws, p.nkeep),
+                            at<int>(ws, p.nvisit), at<unsigned long long>(ws, p.status + kSkipCounterOffset), p.S, p.L, p.Lp,
+                            p.d, scale, st));
+    g_launches += 2;
+    return PATH_OK;
 }
 
 // Chunk preparation + dyadic run products + version chains (paper Sec. 3.1, 3.3).  Shared by forward and backward.
@@ -333,7 +345,7 @@ static int run_chunk_chain(const Plan& p, void* ws, const void* q, const void* k
 
 static int run_backward(const Plan& p, void* ws, const void* q, const void* k, const void* v, const void* w,
                         const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
-                        float* dbeta, float* dlog_f, float scale, bool reuse_keep, cudaStream_t st) {
+                        float* dbeta, float* dlog_f, float scale, cudaStream_t st) {
     const int d = p.d;
     float* dDy = at<float>(ws, p.dDy);
     __nv_bfloat16* dQv = at<__nv_bfloat16>(ws, p.dQv); __nv_bfloat16* dKv = at<__nv_bfloat16>(ws, p.dKv);
@@ -363,15 +375,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     bp.status = at<uint32_t>(ws, p.status);
     bp.zero_ptr = dDy; bp.zero_bytes = p.dy_bytes;   // cleared by the dK/dV sweep, first accumulated into by the version chains
     bp.S = p.S; bp.L = p.L; bp.Lp = p.Lp; bp.N = p.N; bp.scale = scale;
-    if (p.gate) {   // chunk pairs the gate has made negligible are left out of both sweeps (three small kernels)
-        bp.nkeep = at<int>(ws, p.nkeep); bp.nvisit = at<int>(ws, p.nvisit);
-        // (a forward whose preparation is being reused has left its per-query-chunk counts, and the counters, in place)
-        if (!reuse_keep) CK(cudaMemsetAsync(at<uint8_t>(ws, p.status + kSkipCounterOffset), 0, 16, st));
-        LAUNCH(launch_gate_skip(q, k, w, at<float>(ws, p.betap), bp.G, reuse_keep ? nullptr : at<float>(ws, p.tstats),
-                                at<int>(ws, p.nkeep), at<int>(ws, p.nvisit),
-                                at<unsigned long long>(ws, p.status + kSkipCounterOffset), p.S, p.L, p.Lp, d, scale, st));
-        if (!reuse_keep) g_launches += 2;
-    }
+    if (p.gate) { bp.nkeep = at<int>(ws, p.nkeep); bp.nvisit = at<int>(ws, p.nvisit); }   // block skipping: see run_gate_skip
     prof_mark(STG_ROWSTATS, 1, st);
     prof_mark(STG_FA_DKV, 0, st);
     LAUNCH(launch_fa_bwd(tm, bp, d, 0, st));
@@ -387,7 +391,6 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
         LevelTensorMaps ltm;
         if (!make_level_maps(p, ws, ltm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
         LevelParams lp = level_params(p, ws);
-        if (p.gate) { lp.nkeep = at<int>(ws, p.nkeep); lp.nvisit = at<int>(ws, p.nvisit); }
         lp.l = p.nlev;
         LAUNCH(launch_level_kernel(LEVEL_VERSION_BWD, ltm, lp, d, st));
         for (int l = p.nlev - 2; l >= 1; --l) {
@@ -470,6 +473,10 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     tag_store(tag, false);
     rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, true, st);
     if (rc != PATH_OK) return rc;
+    if (log_f) {
+        rc = run_gate_skip(p, workspace, q, k, w, scale, st);
+        if (rc != PATH_OK) return rc;
+    }
     rc = run_prep(p, workspace, q, k, w, false, st);
     if (rc != PATH_OK) return rc;
 
@@ -486,13 +493,7 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     fp.status = at<uint32_t>(workspace, p.status);
     fp.S = p.S; fp.L = L; fp.Lp = p.Lp; fp.N = p.N; fp.scale = scale; fp.out_fp32 = 0;
     prof_mark(STG_FA_FWD, 0, st);
-    if (log_f) {   // which far key chunks the gate has made negligible (two small kernels, counted with the sweep)
-        fp.nkeep = at<int>(workspace, p.nkeep);
-        LAUNCH(launch_gate_skip(q, k, w, at<float>(workspace, p.betap), fp.G, at<float>(workspace, p.tstats), at<int>(workspace, p.nkeep),
-                                nullptr, at<unsigned long long>(workspace, p.status + kSkipCounterOffset), p.S, L, p.Lp, d, scale,
-                                st));
-        ++g_launches;   // the call above is two launches
-    }
+    if (log_f) fp.nkeep = at<int>(workspace, p.nkeep);   // block skipping: see run_gate_skip
     LAUNCH(launch_fa_fwd(tm, fp, d, st));
     prof_mark(STG_FA_FWD, 1, st);
     if (keep_state) tag_store(tag, true);
@@ -523,16 +524,22 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
     prof_reset(STG_PREP_BWD, STG_COUNT);
     const StateTag tag{workspace, q, k, v, w, beta, log_f, B, H, L, d, scale};
     bool same_scale = false;
-    const bool reuse = tag_matches(tag, &same_scale);   // the forward of this very problem left its preparation in this workspace
+    // the forward of this very problem left its preparation in this workspace (for a gated problem the scale has to be
+    // the same too: the block-skipping counts, and with them the levels the version chains were built up to, depend on it)
+    const bool reuse = tag_matches(tag, &same_scale) && (log_f == nullptr || same_scale);
     if (!reuse) tag_store(tag, false);
     rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, !reuse, st);
     if (rc != PATH_OK) return rc;
     if (!reuse) {
+        if (log_f) {
+            rc = run_gate_skip(p, workspace, q, k, w, scale, st);
+            if (rc != PATH_OK) return rc;
+        }
         rc = run_prep(p, workspace, q, k, w, true, st);
         if (rc != PATH_OK) return rc;
         tag_store(tag, true);
     }
-    return run_backward(p, workspace, q, k, v, w, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, scale, reuse && same_scale, st);
+    return run_backward(p, workspace, q, k, v, w, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, scale, st);
 }
 
 }  // extern "C"
