@@ -93,7 +93,7 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
  * rounding, not bitwise.
  *
  * Reuse of the forward's work: if path_attn_fwd ran on this same workspace with
- * these same input pointers and shape, and the workspace was at least
+ * these same input pointers and shape (and, when log_f is given, the same scale), and the workspace was at least
  * path_attn_workspace_bytes(..., for_backward = 1) bytes, the chunk preparation
  * it left there (Sec. 3.1 / 3.3 quantities) is reused instead of recomputed.
  * Any other call on the workspace in between, or different pointers, makes the

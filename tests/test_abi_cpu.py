@@ -102,6 +102,13 @@ def test_frontend_rejects_bad_arguments_on_the_host(lib):
     assert bwd(dz=P + 8) == -4
 
 
+def test_skipped_chunk_pairs_rejects_null_arguments(lib):
+    import ctypes
+    a, b = ctypes.c_ulonglong(0), ctypes.c_ulonglong(0)
+    assert lib.path_attn_skipped_chunk_pairs(None, None, ctypes.byref(a), ctypes.byref(b)) == -1
+    assert lib.path_attn_skipped_chunk_pairs(0x2000, None, None, ctypes.byref(b)) == -1
+
+
 def test_strerror_and_counters(lib):
     seen = set()
     for code in range(0, -9, -1):
