@@ -807,7 +807,7 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
 
 // Per-row constants of the backward sweeps, stored negated so that they enter as addends:
 //   delta[i] = -(dO_i . O_i),   lse2[i] = (G_i - lse_i) * log2(e)   (G: gate prefix, absent = 0),
-// padded to Lp (tail rows: 0).  One warp per row.
+// padded to Lp (tail rows: delta 0, lse2 -1e30 so that their probabilities vanish).  One warp per row.
 template <int HD>
 __global__ void rowstats_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                                 const float* __restrict__ lse, const float* __restrict__ G, float* __restrict__ delta,
@@ -832,7 +832,10 @@ __global__ void rowstats_kernel(const __nv_bfloat16* __restrict__ o, const __nv_
     for (int off = TPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     if (sub == 0 && i < Lp) {
         delta[(size_t)s * Lp + i] = -acc;
-        float v = 0.f;
+        // rows of the zero-padded tail get a huge negative value: their probabilities must come out as exact zeros.  (A
+        // plain 0 would do without a gate; with one, exp2(0 - G_j log2 e) of a strongly decayed key overflows and the
+        // product with the row's zero dP - delta is a NaN.)
+        float v = -1e30f;
         if (i < L) v = ((G ? G[(size_t)s * Lp + i] : 0.f) - lse[(size_t)s * L + i]) * kLog2e;
         lse2[(size_t)s * Lp + i] = v;
     }

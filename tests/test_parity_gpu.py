@@ -375,3 +375,13 @@ def test_backward_recomputes_the_skip_counts_when_the_scale_differs(binding, ora
     ref = oracle.backward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["d_o"], x["log_f"], scale=0.5)
     for name, r in ref.items():
         check(name, g[name].reshape(-1, *g[name].shape[2:]), r)
+
+
+@pytest.mark.parametrize("L,d,shift", [(201, 128, 0.0), (130, 64, -1.0), (700, 64, 0.0)])
+def test_strong_gate_with_a_ragged_tail(binding, oracle, L, d, shift):
+    """A gate that decays by e^-100 within one chunk, on a length that leaves padded rows in the last chunk: the padded
+    query rows must drop out exactly (their exponent used to overflow against a strongly decayed key: NaN gradients)."""
+    inp = synth.make_inputs(2, 2, L, d, "bf16", gate=True, seed=4800 + L)
+    gen = torch.Generator().manual_seed(4801 + L)
+    inp["log_f"] = torch.nn.functional.logsigmoid(torch.randn(2, 2, L, generator=gen) + shift).contiguous()
+    compare_all(binding, oracle, inp)
