@@ -127,6 +127,31 @@ def test_random_small_problems(binding, oracle, B, H, L, d, gate, sharp, scale, 
     compare_all(binding, oracle, inp, scale=scale)
 
 
+def _random_gated_cases(n, seed=20250517):
+    """Seeded gated problems whose decay ranges from negligible to e^-100 per chunk (block skipping from none to nearly
+    all), lengths of at least 16 tokens, some with |w| up to 1.15 and beta up to 2.4 (transitions that can grow)."""
+    import random
+    rng = random.Random(seed)
+    out = []
+    for i in range(n):
+        L = rng.choice([rng.randint(16, 130), rng.randint(130, 700), rng.choice([256, 512, 1024, 1536, 2304])])
+        out.append((rng.choice([1, 2]), rng.choice([1, 2, 3]), L, rng.choice([64, 128]),
+                    rng.choice([-2.0, -1.0, 0.0, 1.0, 3.0, 5.0]), rng.random() < 0.3 and L <= 512,
+                    rng.choice([1.0, 0.5, -0.25]), 4900 + i))
+    return out
+
+
+@pytest.mark.parametrize("B,H,L,d,shift,wild,scale,seed", _random_gated_cases(12))
+def test_random_gated_problems(binding, oracle, B, H, L, d, shift, wild, scale, seed):
+    inp = synth.make_inputs(B, H, L, d, "bf16", gate=True, seed=seed)
+    gen = torch.Generator().manual_seed(seed + 7)
+    inp["log_f"] = torch.nn.functional.logsigmoid(torch.randn(B, H, L, generator=gen) + shift).contiguous()
+    if wild:
+        inp["w"] = (inp["w"].float() * (1.0 + 0.15 * torch.rand(B, H, L, 1, generator=gen))).to(torch.bfloat16).contiguous()
+        inp["beta"] = (inp["beta"] * 1.2).contiguous()
+    compare_all(binding, oracle, inp, scale=scale)
+
+
 def test_c1_workload_shape_and_distribution_in_bf16(binding, oracle):
     """Workload C1's shape and distributions (B=1, H=2, L=256, d=64, q, k, v ~ N(0,1) unscaled: logits of standard
     deviation 8) through the bf16 tensor-core path."""
