@@ -42,11 +42,11 @@ UNIT = "TFLOP/s"
 # DRAM bytes per launch PER (batch, head) SLICE at the C3 shape (L=4096, d=128), from the ncu captures at batch 1
 # (16 slices) summarised under profiles/; slices are independent, so a launch over S slices moves S times this.
 NCU_TRAFFIC_BYTES_PER_SLICE = {
-    "chunk_prep": (52.89e6 + 148.07e6) / 16,        # backward instance (the step's forward runs on the shared workspace)
-    "fa_fwd": (168.88e6 + 10.15e6) / 16,
-    "fa_bwd_dkv": (187.54e6 + 123.63e6) / 16,       # includes clearing the run-product gradient buffer on the side
-    "fa_bwd_dq": (117.30e6 + 20.53e6) / 16,
-    "bwd_chunk_chain": (283.98e6 + 33.74e6) / 16,
+    "chunk_prep": (54.62e6 + 146.33e6) / 16,        # backward instance (the step's forward runs on the shared workspace)
+    "fa_fwd": (169.10e6 + 10.06e6) / 16,
+    "fa_bwd_dkv": (187.31e6 + 122.91e6) / 16,       # includes clearing the run-product gradient buffer on the side
+    "fa_bwd_dq": (117.25e6 + 20.75e6) / 16,
+    "bwd_chunk_chain": (282.82e6 + 33.00e6) / 16,
 }
 
 # DRAM bytes per launch of frontend_bwd_kernel PER BATCH ROW at H=32, L=4096, d=64 with the gate, from the ncu capture at
