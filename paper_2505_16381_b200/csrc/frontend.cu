@@ -12,9 +12,9 @@
 // shared memory that only this lane reads back (a per-lane queue, so no barrier is involved: the lane waits for its own
 // copy group), one position block ahead of the one being computed: the bytes in flight, which is what a
 // bandwidth-bound kernel lives on, sit in shared memory instead of registers.  A CTA is 4 warps = 4 * (256 / d) * R
-// consecutive positions of one head; CTAs are numbered with the head fastest, so the CTAs that run at the same time read whole contiguous rows of z between them, and each
-// loops over the position blocks of its head with a stride (the backward keeps its filter-gradient sums in registers
-// across that loop and adds them to global memory once).
+// consecutive positions of one head; CTAs are numbered with the head fastest, so the CTAs that run at the same time
+// read whole contiguous rows of z between them, and each loops over the position blocks of its head with a stride (the
+// backward keeps its filter-gradient sums in registers across that loop and adds them to global memory once).
 #include "common.cuh"
 
 namespace path {

@@ -64,7 +64,8 @@ __global__ void __launch_bounds__(256) dsd_rowsum_kernel(const float* __restrict
         for (int off = 16; off > 0; off >>= 1)
 #pragma unroll
             for (int x = 0; x < 4; ++x) acc[x] += __shfl_xor_sync(0xffffffffu, acc[x], off);
-        if (lane < 4) rs[(size_t)blockIdx.x * CHUNK + r0 + lane] = lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3];
+        if (lane < 4)
+            rs[(size_t)blockIdx.x * CHUNK + r0 + lane] = lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3];
     }
 }
 
@@ -149,7 +150,10 @@ __global__ void __launch_bounds__(256) tile_stats_kernel(const __nv_bfloat16* __
         gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, off)); gmin = fminf(gmin, __shfl_xor_sync(0xffffffffu, gmin, off));
         mlo = fminf(mlo, __shfl_xor_sync(0xffffffffu, mlo, off)); gam += __shfl_xor_sync(0xffffffffu, gam, off);
     }
-    if (lane == 0) { red[warp][0] = qn; red[warp][1] = kn; red[warp][2] = gmax; red[warp][3] = gmin; red[warp][4] = mlo; red[warp][5] = gam; }
+    if (lane == 0) {
+        red[warp][0] = qn; red[warp][1] = kn; red[warp][2] = gmax;
+        red[warp][3] = gmin; red[warp][4] = mlo; red[warp][5] = gam;
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int x = 1; x < 8; ++x) {
@@ -158,7 +162,8 @@ __global__ void __launch_bounds__(256) tile_stats_kernel(const __nv_bfloat16* __
         }
         float* o = stats + (size_t)blockIdx.x * 8;
         // the norms and the growth go up, the row maximum goes down by a rounding margin: the test must err towards keeping
-        o[0] = qn * 1.001f; o[1] = kn * 1.001f; o[2] = gmax; o[3] = gmin; o[4] = mlo - 1e-3f * fabsf(mlo); o[5] = gam * 1.001f + 1e-6f;
+        o[0] = qn * 1.001f; o[1] = kn * 1.001f; o[2] = gmax; o[3] = gmin;
+        o[4] = mlo - 1e-3f * fabsf(mlo); o[5] = gam * 1.001f + 1e-6f;
         o[6] = o[7] = 0.f;
     }
 }
