@@ -35,6 +35,11 @@ from paper_2505_16381_b200 import synth  # noqa: E402
 
 CHUNK = 128
 METRIC = "PaTH attn fwd+bwd TFLOP/s (attention-equivalent FLOPs) at L=4096, d=128"
+
+
+def metric_name(cfg):
+    """The headline metric's name; the other workloads (--workload) carry their own length and head size in it."""
+    return METRIC.replace("L=4096, d=128", f"L={cfg['L']}, d={cfg['d']}")
 UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the kernel named by `roofline.kernel`,
@@ -194,7 +199,7 @@ def run_reference(args, cfg):
     val = (f1 + b1) / (ms * 1e-3) / 1e12
     sample = f"1 of {cfg['B'] * cfg['H']} (batch, head) slices of {args.workload} per step, forward + backward, float64"
     line = {
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "impl": "reference", "metric": metric_name(cfg), "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
         "config": {"workload": f"{args.workload}: B={cfg['B']} H={cfg['H']} L={cfg['L']} d={cfg['d']} fwd+bwd",
@@ -373,7 +378,7 @@ def run_ours(args, cfg):
         skipping = {"kept_chunk_pairs": kept, "all_chunk_pairs": total,
                     "note": "TFLOP/s are attention-equivalent FLOPs of the full causal problem per second, skipped pairs included"}
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": metric_name(cfg), "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": f"{args.workload}: B={B} H={H} L={L} d={d} bf16 fwd+bwd per GPU", "global_batch": B * world,
