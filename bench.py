@@ -246,7 +246,7 @@ def run_ours(args, cfg):
                               out=(o, lse))
         n = binding.last_launch_count()
         binding.path_attn_bwd(t["q"], t["k"], t["v"], t["w"], t["beta"], o, lse, t["d_o"], t["log_f"], scale=scale,
-                              workspace=ws, out=gout)
+                              workspace=ws, out=gout, reuse=True)
         launches[0] = n + binding.last_launch_count()
 
     def barrier():
@@ -315,7 +315,7 @@ def run_ours(args, cfg):
                 binding.path_attn_fwd(t["q"], t["k"], t["v"], t["w"], t["beta"], t["log_f"], scale=scale, workspace=ws,
                                       out=(o, lse))
                 binding.path_attn_bwd(t["q"], t["k"], t["v"], t["w"], t["beta"], o, lse, t["d_o"], t["log_f"],
-                                      scale=scale, workspace=ws, out=gouts[b])
+                                      scale=scale, workspace=ws, out=gouts[b], reuse=True)
                 in_free[b].record(s_cmp)
                 out_ready[b].record(s_cmp)
             with torch.cuda.stream(s_out):

@@ -60,7 +60,9 @@ typedef enum {
     PATH_ERR_ARCH = -6,      /* current device is not compute capability 10.x */
     PATH_ERR_LAUNCH = -7,    /* a CUDA runtime / driver call failed (see path_attn_last_cuda_error) */
     PATH_ERR_TIMEOUT = -8,   /* reported by path_attn_device_status: a bounded device wait ran out */
-    PATH_ERR_STATIC_LIMIT = -9 /* path_attn_fwd_static: the problem needs more scratch than the built-in buffer holds */
+    PATH_ERR_STATIC_LIMIT = -9, /* path_attn_fwd_static: the problem needs more scratch than the built-in buffer holds */
+    PATH_ERR_STATE = -10     /* reported by path_attn_device_status after path_attn_bwd_reuse: the workspace does not
+                                hold the forward state of this problem; the gradients of that call are invalid */
 } path_status_t;
 
 /* Bytes of scratch memory path_attn_fwd (for_backward = 0) or path_attn_bwd
@@ -92,18 +94,36 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
  * dt must be PATH_BF16.  Uses float32 atomics: results are reproducible to
  * rounding, not bitwise.
  *
- * Reuse of the forward's work: if path_attn_fwd ran on this same workspace with
- * these same input pointers and shape (and, when log_f is given, the same scale), and the workspace was at least
- * path_attn_workspace_bytes(..., for_backward = 1) bytes, the chunk preparation
- * it left there (Sec. 3.1 / 3.3 quantities) is reused instead of recomputed.
- * Any other call on the workspace in between, or different pointers, makes the
- * backward recompute it.  (As always, o and lse must belong to the inputs.)
+ * path_attn_bwd always recomputes the chunk preparation (Sec. 3.1 / 3.3
+ * quantities) from q, k, w, beta, log_f: it depends on nothing a previous call
+ * left in the workspace.
+ *
+ * path_attn_bwd_reuse (same arguments) is the explicit request to skip that
+ * recomputation.  Contract: the last call on `workspace` was path_attn_fwd for
+ * this very problem (same pointers q, k, v, w, beta, log_f, same shape and,
+ * when log_f is given, the same scale), the workspace was at least
+ * path_attn_workspace_bytes(..., for_backward = 1) bytes in that call too, and
+ * since then neither the workspace nor the contents of q, k, w, beta, log_f
+ * have been written to.  A forward that runs on a backward-sized workspace ends
+ * by writing a record of its problem into the workspace; path_attn_bwd_reuse
+ * compares that record on the device before anything reads the state, and a
+ * mismatch (another problem, a forward-sized forward, a call in between) is
+ * reported by path_attn_device_status as PATH_ERR_STATE, in which case the
+ * outputs of the call are invalid.  The record cannot see a caller that
+ * rewrites an input buffer in place: that is the caller's side of the contract.
+ * Holding the state costs the whole backward-sized workspace from forward to
+ * backward; recomputing costs the preparation stages once more.
  */
 int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, const float* beta,
                   const float* log_f, const void* o, const float* lse, const void* d_o, void* dq,
                   void* dk, void* dv, void* dw, float* dbeta, float* dlog_f, int B, int H, int L,
                   int d, float scale, path_dtype_t dt, void* workspace, size_t workspace_bytes,
                   void* cuda_stream);
+int path_attn_bwd_reuse(const void* q, const void* k, const void* v, const void* w, const float* beta,
+                        const float* log_f, const void* o, const float* lse, const void* d_o, void* dq,
+                        void* dk, void* dv, void* dw, float* dbeta, float* dlog_f, int B, int H, int L,
+                        int d, float scale, path_dtype_t dt, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream);
 
 /*
  * Forward pass for callers that cannot allocate device memory (the paper has no
@@ -207,10 +227,28 @@ int path_attn_skipped_chunk_pairs(const void* workspace, void* cuda_stream, unsi
                                   unsigned long long* all);
 
 /* Reads the device status word the last call on this workspace left behind.
- * Synchronises `cuda_stream`.  Returns PATH_OK, PATH_ERR_TIMEOUT, or
- * PATH_ERR_LAUNCH if the copy itself failed.  If `detail` is not NULL it
- * receives the raw status word (0 = clean; otherwise a code naming the wait). */
+ * Synchronises `cuda_stream`.  Returns PATH_OK, PATH_ERR_TIMEOUT (a bounded
+ * wait ran out), PATH_ERR_STATE (path_attn_bwd_reuse found no matching forward
+ * state), or PATH_ERR_LAUNCH if the copy itself failed.  If `detail` is not
+ * NULL it receives the raw status word (0 = clean; otherwise a code naming the
+ * wait: 0x1xx forward sweep, 0x2xx dK/dV sweep, 0x3xx dQ sweep, 0x401 chunk
+ * preparation, 0x501 chunk chain rule, 0x601 level kernels, 0x701 state
+ * mismatch, 0x7f1 the self-test below). */
 int path_attn_device_status(const void* workspace, void* cuda_stream, unsigned int* detail);
+
+/*
+ * Self-test of the bounded-wait machinery (no counterpart in the paper).  Every
+ * device-side wait of the library (on an mbarrier fed by TMA or by tcgen05
+ * commits) gives up after a time limit, raises its CTA's abort flag, lets the
+ * kernel wind down and leaves a code in the status word.  This call runs that
+ * very wait routine on a barrier nothing ever arrives on, with a limit of
+ * `limit_us` microseconds (1 .. 100000) instead of the library's ~1 s, so that
+ * the path from an expired wait to PATH_ERR_TIMEOUT can be exercised without a
+ * fault or a hang: afterwards path_attn_device_status(workspace, ...) returns
+ * PATH_ERR_TIMEOUT with detail 0x7f1.  Only the first 256 bytes of `workspace`
+ * (256-byte aligned) are written.  Asynchronous on cuda_stream.
+ */
+int path_attn_selftest_timeout(void* workspace, unsigned int limit_us, void* cuda_stream);
 
 /* Static description of a status code. */
 const char* path_attn_strerror(int status);

@@ -206,11 +206,14 @@ int path_oracle_key_cache(const double* k, const double* w, const double* beta, 
  *       dw_j    -= beta_j [ (w_j.x) gbar + (w_j.gbar) x ],
  *       gbar    <- H_j gbar + da_ij k_j      (gbar becomes d/du_{i,j}),
  *   dq_i = gbar after j = i.
+ *
+ * path_oracle_bwd_lse is the same for the loss  sum(O * dO) + sum(lse * d_lse)  (d_lse: [S, L], may be
+ * NULL): since d lse_i / d s_ij = p_ij, the only change is  ds_ij = p_ij (dp_ij - delta_i + d_lse_i).
  */
-int path_oracle_bwd(const double* q, const double* k, const double* v, const double* w,
-                    const double* beta, const double* g, const double* d_o, int S, int L, int d,
-                    double scale, double* dq, double* dk, double* dv, double* dw, double* dbeta,
-                    double* dg) {
+int path_oracle_bwd_lse(const double* q, const double* k, const double* v, const double* w,
+                        const double* beta, const double* g, const double* d_o, const double* d_lse, int S, int L,
+                        int d, double scale, double* dq, double* dk, double* dv, double* dw, double* dbeta,
+                        double* dg) {
     size_t nLd = (size_t)L * d;
     int fail = 0;
     memset(dq, 0, sizeof(double) * S * nLd);
@@ -259,10 +262,11 @@ int path_oracle_bwd(const double* q, const double* k, const double* v, const dou
                         for (int x = 0; x < d; ++x) o[x] += s[j] * vj[x];
                     }
                     double delta = dot(doi, o, d);
+                    double dl = d_lse ? d_lse[(size_t)sl * L + i] : 0.0;
                     for (int j = 0; j <= i; ++j) {
                         double p = s[j];
                         double dp = dot(doi, vs + (size_t)j * d, d);
-                        double ds = p * (dp - delta);
+                        double ds = p * (dp - delta + dl);
                         double* dvj = tdv + (size_t)j * d;
                         for (int x = 0; x < d; ++x) dvj[x] += p * doi[x];
                         tdG[i] += ds;
@@ -307,4 +311,11 @@ int path_oracle_bwd(const double* q, const double* k, const double* v, const dou
         free(G); free(dG);
     }
     return fail ? -1 : 0;
+}
+
+int path_oracle_bwd(const double* q, const double* k, const double* v, const double* w,
+                    const double* beta, const double* g, const double* d_o, int S, int L, int d,
+                    double scale, double* dq, double* dk, double* dv, double* dw, double* dbeta,
+                    double* dg) {
+    return path_oracle_bwd_lse(q, k, v, w, beta, g, d_o, NULL, S, L, d, scale, dq, dk, dv, dw, dbeta, dg);
 }

@@ -51,6 +51,8 @@ def _load():
         lib.path_oracle_uchain.argtypes = [P, P, P, I, I, I, P]
         lib.path_oracle_key_cache.argtypes = [P, P, P, I, I, I, I, P]
         lib.path_oracle_bwd.argtypes = [P, P, P, P, P, P, P, I, I, I, D, P, P, P, P, P, P]
+        lib.path_oracle_bwd_lse.restype = ctypes.c_int
+        lib.path_oracle_bwd_lse.argtypes = [P, P, P, P, P, P, P, P, I, I, I, D, P, P, P, P, P, P]
         _lib = lib
     return _lib
 
@@ -145,17 +147,20 @@ def key_cache(k, w, beta, n=None):
     return kc
 
 
-def backward(q, k, v, w, beta, d_o, log_f=None, scale: float = 1.0):
-    """Gradients of sum(O * d_o): dict with dq, dk, dv, dw, dbeta and (if gated) dlog_f."""
+def backward(q, k, v, w, beta, d_o, log_f=None, scale: float = 1.0, d_lse=None):
+    """Gradients of sum(O * d_o) (+ sum(lse * d_lse) when ``d_lse`` is given): dict with dq, dk, dv, dw, dbeta and
+    (if gated) dlog_f."""
     q, k, v, w, beta, g, S, L, d = _flatten(q, k, v, w, beta, log_f)
     d_o = _f64(d_o)
     assert d_o.shape == q.shape
+    d_lse = None if d_lse is None else _f64(d_lse)
+    assert d_lse is None or d_lse.shape == beta.shape
     dq, dk, dv, dw = (np.empty_like(q) for _ in range(4))
     dbeta = np.empty_like(beta)
     dg = None if g is None else np.empty_like(beta)
-    rc = _load().path_oracle_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(beta), _ptr(g), _ptr(d_o),
-                                 S, L, d, float(scale), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dw),
-                                 _ptr(dbeta), _ptr(dg))
+    rc = _load().path_oracle_bwd_lse(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(beta), _ptr(g), _ptr(d_o), _ptr(d_lse),
+                                     S, L, d, float(scale), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dw),
+                                     _ptr(dbeta), _ptr(dg))
     if rc != 0:
         raise MemoryError("path_oracle_bwd failed")
     out = {"dq": dq, "dk": dk, "dv": dv, "dw": dw, "dbeta": dbeta}

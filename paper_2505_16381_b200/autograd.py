@@ -15,30 +15,38 @@ from . import binding
 
 class _PathAttention(torch.autograd.Function):
     @staticmethod
-    def forward(ctx, q, k, v, w, beta, log_f, scale):
+    def forward(ctx, q, k, v, w, beta, log_f, scale, retain_state):
+        # (requires_grad of the copies .contiguous() makes is always False here: ask autograd itself)
+        need_grad = any(ctx.needs_input_grad[:6])
         q, k, v, w = (t.contiguous() for t in (q, k, v, w))
         beta = beta.contiguous()
         log_f = None if log_f is None else log_f.contiguous()
-        need_grad = any(t is not None and t.requires_grad for t in (q, k, v, w, beta, log_f))
-        # a backward-sized workspace lets the backward reuse the forward's chunk preparation
-        ws = binding.alloc_workspace(q, log_f is not None, need_grad)
+        # Default: a forward-sized workspace that is released right away; the backward recomputes the chunk preparation.
+        # retain_state keeps a backward-sized workspace (about ten times the size of q, k, v, w together) alive from
+        # forward to backward so that the backward can skip that recomputation.
+        keep = bool(retain_state) and need_grad
+        ws = binding.alloc_workspace(q, log_f is not None, keep)
         o, lse = binding.path_attn_fwd(q, k, v, w, beta, log_f, scale=scale, workspace=ws)
         ctx.save_for_backward(q, k, v, w, beta, log_f, o, lse)
-        ctx.scale, ctx.ws = scale, ws
+        ctx.scale, ctx.ws = scale, (ws if keep else None)
         ctx.mark_non_differentiable(lse)
         return o, lse
 
     @staticmethod
     def backward(ctx, d_o, _d_lse):
         q, k, v, w, beta, log_f, o, lse = ctx.saved_tensors
-        g = binding.path_attn_bwd(q, k, v, w, beta, o, lse, d_o.contiguous(), log_f, scale=ctx.scale, workspace=ctx.ws)
+        g = binding.path_attn_bwd(q, k, v, w, beta, o, lse, d_o.contiguous(), log_f, scale=ctx.scale, workspace=ctx.ws,
+                                  reuse=ctx.ws is not None)
         ctx.ws = None
-        return g["dq"], g["dk"], g["dv"], g["dw"], g["dbeta"], g.get("dlog_f"), None
+        return g["dq"], g["dk"], g["dv"], g["dw"], g["dbeta"], g.get("dlog_f"), None, None
 
 
-def path_attention(q, k, v, w, beta, log_f=None, scale: float = 1.0, return_lse: bool = False):
-    """PaTH attention (paper Sec. 2.2; PaTH-FoX when ``log_f`` is given), differentiable in q, k, v, w, beta, log_f."""
-    o, lse = _PathAttention.apply(q, k, v, w, beta, log_f, float(scale))
+def path_attention(q, k, v, w, beta, log_f=None, scale: float = 1.0, return_lse: bool = False, retain_state: bool = False):
+    """PaTH attention (paper Sec. 2.2; PaTH-FoX when ``log_f`` is given), differentiable in q, k, v, w, beta, log_f.
+
+    ``retain_state=True`` trades memory for time: the forward's chunk preparation stays in a backward-sized workspace
+    until the backward has used it (see ``path_attn_bwd_reuse``)."""
+    o, lse = _PathAttention.apply(q, k, v, w, beta, log_f, float(scale), bool(retain_state))
     return (o, lse) if return_lse else o
 
 

@@ -17,7 +17,8 @@ _lib = None
 
 PATH_BF16, PATH_FP32 = 0, 1
 PATH_OK = 0
-EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_attn_fwd_static", "path_attn_device_status",
+EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_attn_bwd_reuse", "path_attn_fwd_static",
+           "path_attn_device_status", "path_attn_selftest_timeout",
            "path_attn_prefill_cache", "path_attn_decode_workspace_bytes", "path_attn_decode_step",
            "path_attn_frontend_fwd", "path_attn_frontend_bwd", "path_attn_skipped_chunk_pairs",
            "path_attn_strerror", "path_attn_last_cuda_error", "path_attn_last_launch_count",
@@ -50,6 +51,10 @@ def load():
         lib.path_attn_fwd_static.argtypes = [P, P, P, P, P, P, P, P, I, I, I, I, F, I, P, ctypes.POINTER(P)]
         lib.path_attn_bwd.restype = I
         lib.path_attn_bwd.argtypes = [P] * 15 + [I, I, I, I, F, I, P, Z, P]
+        lib.path_attn_bwd_reuse.restype = I
+        lib.path_attn_bwd_reuse.argtypes = [P] * 15 + [I, I, I, I, F, I, P, Z, P]
+        lib.path_attn_selftest_timeout.restype = I
+        lib.path_attn_selftest_timeout.argtypes = [P, ctypes.c_uint, P]
         lib.path_attn_prefill_cache.restype = I
         lib.path_attn_prefill_cache.argtypes = [P] * 8 + [I, I, I, I, I, I, P, Z, P]
         lib.path_attn_decode_workspace_bytes.restype = Z
@@ -154,11 +159,17 @@ def path_attn_fwd_static(q, k, v, w, beta, log_f=None, scale=1.0, out=None):
     return o, lse, addr.value
 
 
-def path_attn_bwd(q, k, v, w, beta, o, lse, d_o, log_f=None, scale=1.0, workspace=None, out=None):
-    """Backward.  Returns a dict dq, dk, dv, dw, dbeta (and dlog_f when gated)."""
+def path_attn_bwd(q, k, v, w, beta, o, lse, d_o, log_f=None, scale=1.0, workspace=None, out=None, reuse=False):
+    """Backward.  Returns a dict dq, dk, dv, dw, dbeta (and dlog_f when gated).
+
+    ``reuse=True`` calls ``path_attn_bwd_reuse``: the chunk preparation is taken from ``workspace``, where the forward of
+    this very problem must have left it (backward-sized workspace, nothing written in between); a mismatch shows up as
+    status -10 from :func:`device_status`."""
     _check(q, k, v, w, beta, log_f, o, lse, d_o)
     lib = load()
     B, H, L, d = q.shape
+    if reuse and workspace is None:
+        raise ValueError("reuse=True needs the workspace the forward ran on")
     if workspace is None:
         workspace = alloc_workspace(q, log_f is not None, True)
     if out is None:
@@ -167,11 +178,12 @@ def path_attn_bwd(q, k, v, w, beta, o, lse, d_o, log_f=None, scale=1.0, workspac
         if log_f is not None:
             out["dlog_f"] = torch.empty_like(log_f)
     st = torch.cuda.current_stream(q.device).cuda_stream
+    fn = lib.path_attn_bwd_reuse if reuse else lib.path_attn_bwd
     with torch.cuda.device(q.device):
-        rc = lib.path_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(beta), _ptr(log_f), _ptr(o), _ptr(lse),
-                               _ptr(d_o), _ptr(out["dq"]), _ptr(out["dk"]), _ptr(out["dv"]), _ptr(out["dw"]),
-                               _ptr(out["dbeta"]), _ptr(out.get("dlog_f")), B, H, L, d, float(scale), _dt(q),
-                               _ptr(workspace), workspace.numel(), ctypes.c_void_p(st))
+        rc = fn(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(beta), _ptr(log_f), _ptr(o), _ptr(lse),
+                _ptr(d_o), _ptr(out["dq"]), _ptr(out["dk"]), _ptr(out["dv"]), _ptr(out["dw"]),
+                _ptr(out["dbeta"]), _ptr(out.get("dlog_f")), B, H, L, d, float(scale), _dt(q),
+                _ptr(workspace), workspace.numel(), ctypes.c_void_p(st))
     if rc != PATH_OK:
         raise PathAttnError(rc, "path_attn_bwd")
     return out
@@ -188,6 +200,17 @@ def device_status(workspace) -> int:
     if rc != PATH_OK:
         raise PathAttnError(rc, f"path_attn_device_status (word 0x{detail.value:x})")
     return int(detail.value)
+
+
+def selftest_timeout(workspace, limit_us=1000) -> None:
+    """Launches the library's wait self-test on ``workspace``: a bounded wait that runs out after ``limit_us``
+    microseconds and reports itself through the status word (read it with :func:`device_status`)."""
+    lib = load()
+    st = torch.cuda.current_stream(workspace.device).cuda_stream
+    with torch.cuda.device(workspace.device):
+        rc = lib.path_attn_selftest_timeout(_ptr(workspace), int(limit_us), ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_selftest_timeout")
 
 
 def skipped_chunk_pairs(workspace):

@@ -16,6 +16,20 @@ enum : uint32_t {
     ST_DKV_PRODUCER = 0x201, ST_DKV_MMA = 0x202, ST_DKV_COMPUTE = 0x203,
     ST_DQ_PRODUCER = 0x301, ST_DQ_MMA = 0x302, ST_DQ_COMPUTE = 0x303,
     ST_PREP = 0x401, ST_CHAIN = 0x501, ST_LEVELS = 0x601,
+    ST_STATE = 0x701,      // path_attn_bwd_reuse: the workspace does not hold the forward state of this problem
+    ST_SELFTEST = 0x7f1,   // path_attn_selftest_timeout: the wait it makes run out
+};
+
+// What a forward that ran on a backward-sized workspace leaves at byte kStateRecordOffset of the status block: which
+// problem the chunk preparation in the workspace belongs to.  path_attn_bwd_reuse compares it on the device.
+constexpr size_t kStateRecordOffset = 64;
+constexpr unsigned long long kStateMagic = 0x50615448537461ull;
+struct StateRecord {
+    unsigned long long magic;
+    const void *q, *k, *v, *w, *beta, *log_f;
+    int B, H, L, d;
+    float scale;   // compared for gated problems only (the block-skipping counts depend on it)
+    int gate;
 };
 
 __host__ __device__ inline int msb32(unsigned x) {

@@ -1,6 +1,7 @@
 // Memory-bound helpers: zero-padding of ragged inputs, prefix sum of the log gate (PaTH-FoX, paper Sec. 2.2),
 // suffix sum of its gradient, row sums of the diagonal-chunk dS.
 #include "linear.cuh"
+#include "tc5.cuh"
 
 namespace path {
 
@@ -242,6 +243,37 @@ __global__ void __launch_bounds__(128) tile_stair_kernel(int* __restrict__ nkeep
     }
 }
 
+// ---- forward-state record and the wait self-test
+__global__ void state_write_kernel(StateRecord* dst, const StateRecord rec) {
+    if (threadIdx.x == 0) *dst = rec;
+}
+__global__ void state_check_kernel(const StateRecord* have, const StateRecord want, uint32_t* status) {
+    if (threadIdx.x != 0) return;
+    const StateRecord h = *have;
+    const bool same = h.magic == want.magic && h.q == want.q && h.k == want.k && h.v == want.v && h.w == want.w &&
+                      h.beta == want.beta && h.log_f == want.log_f && h.B == want.B && h.H == want.H && h.L == want.L &&
+                      h.d == want.d && h.gate == want.gate && (!want.gate || h.scale == want.scale);
+    if (!same) atomicCAS(status, 0u, (uint32_t)ST_STATE);
+}
+// The same bounded wait every kernel of the library uses, on a barrier that never completes: after `ticks` cycles it
+// gives up, raises the CTA's abort flag with its code, and the kernel forwards the flag to the status word and returns.
+__global__ void selftest_wait_kernel(uint32_t* status, long long ticks) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_word;
+    volatile uint32_t* abort_flag = &abort_word;
+    if (threadIdx.x == 0) {
+        tc5::mbar_init(&bar, 1);
+        *abort_flag = 0;
+        tc5::mbar_fence_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bool ok = tc5::mbar_try_wait(&bar, 0);
+        if (!ok) ok = tc5::mbar_wait_slow(&bar, 0, abort_flag, ST_SELFTEST, ticks);
+        if (!ok && *abort_flag != 0) atomicCAS(status, 0u, *abort_flag);
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_gate_suffix(const float* dGa, const float* dGb, const float* dGc, float* out, int S, int L, int Lp,
@@ -285,6 +317,19 @@ cudaError_t launch_gate_skip(const void* q, const void* k, const void* w, const 
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     tile_stair_kernel<<<S, 128, 0, st>>>(nkeep, nvisit, counters, S, N);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_state_write(void* record, const StateRecord& rec, cudaStream_t st) {
+    state_write_kernel<<<1, 32, 0, st>>>((StateRecord*)record, rec);
+    return cudaGetLastError();
+}
+cudaError_t launch_state_check(const void* record, const StateRecord& want, uint32_t* status, cudaStream_t st) {
+    state_check_kernel<<<1, 32, 0, st>>>((const StateRecord*)record, want, status);
+    return cudaGetLastError();
+}
+cudaError_t launch_selftest_wait(uint32_t* status, long long ticks, cudaStream_t st) {
+    selftest_wait_kernel<<<1, 32, 0, st>>>(status, ticks);
     return cudaGetLastError();
 }
 

@@ -26,4 +26,12 @@ cudaError_t launch_gate_skip(const void* q, const void* k, const void* w, const 
                              int* nkeep, int* nvisit, unsigned long long* counters, int S, int L, int Lp, int hd, float scale,
                              cudaStream_t st);
 
+// Forward-state record in the status block of a workspace (see StateRecord): written at the end of a forward that kept its
+// chunk preparation, compared by the backward that wants to reuse it (a mismatch raises ST_STATE in the status word).
+cudaError_t launch_state_write(void* record, const StateRecord& rec, cudaStream_t st);
+cudaError_t launch_state_check(const void* record, const StateRecord& want, uint32_t* status, cudaStream_t st);
+// One thread waits on an mbarrier that nothing arrives on, with a limit of `ticks` clock cycles, then reports
+// ST_SELFTEST through the status word like every bounded wait of the library does.
+cudaError_t launch_selftest_wait(uint32_t* status, long long ticks, cudaStream_t st);
+
 }  // namespace path

@@ -57,37 +57,16 @@ static void prof_mark(int stage, int end, cudaStream_t st) {
 
 // ------------------------------------------------------------------------------------------- forward state reuse
 // A forward that ran on a backward-sized workspace leaves the chunk preparation (with the tiles the chain rule needs)
-// in it.  The table remembers, per workspace pointer, which problem that state belongs to, so that the backward of
-// the same problem can skip recomputing it.  Host-side only; entries are overwritten by any later call on the workspace.
-struct StateTag {
-    const void *ws, *q, *k, *v, *w, *beta, *log_f;
-    int B, H, L, d;
-    float scale;   // not part of the identity (the chunk preparation does not depend on it); the block-skipping counts do
-};
-static std::mutex g_tag_mutex;
-static StateTag g_tags[64];
-static int g_tag_next = 0;
-
-static bool tag_equal(const StateTag& a, const StateTag& b) {
-    return a.ws == b.ws && a.q == b.q && a.k == b.k && a.v == b.v && a.w == b.w && a.beta == b.beta &&
-           a.log_f == b.log_f && a.B == b.B && a.H == b.H && a.L == b.L && a.d == b.d;
-}
-static void tag_store(const StateTag& t, bool valid) {   // valid = false: forget whatever was known about t.ws
-    std::lock_guard<std::mutex> lock(g_tag_mutex);
-    for (auto& e : g_tags)
-        if (e.ws == t.ws) { if (valid) e = t; else e = StateTag{}; return; }
-    if (!valid) return;
-    g_tags[g_tag_next] = t;
-    g_tag_next = (g_tag_next + 1) % 64;
-}
-static bool tag_matches(const StateTag& t, bool* same_scale = nullptr) {
-    std::lock_guard<std::mutex> lock(g_tag_mutex);
-    for (const auto& e : g_tags)
-        if (e.ws == t.ws) {
-            if (same_scale) *same_scale = e.scale == t.scale;
-            return tag_equal(e, t);
-        }
-    return false;
+// in it, and ends by writing a record of the problem into the status block.  path_attn_bwd_reuse, the explicit request
+// to skip the preparation, compares that record on the device before its first kernel reads the state; nothing is
+// remembered on the host.
+static StateRecord make_record(const void* q, const void* k, const void* v, const void* w, const float* beta,
+                               const float* log_f, int B, int H, int L, int d, float scale) {
+    StateRecord r{};
+    r.magic = kStateMagic;
+    r.q = q; r.k = k; r.v = v; r.w = w; r.beta = beta; r.log_f = log_f;
+    r.B = B; r.H = H; r.L = L; r.d = d; r.scale = scale; r.gate = log_f ? 1 : 0;
+    return r;
 }
 
 // ------------------------------------------------------------------------------------------- tensor maps
@@ -442,7 +421,6 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
         if (rc32 != PATH_OK) return rc32;
         cudaStream_t st32 = (cudaStream_t)cuda_stream;
         CK(cudaMemsetAsync(workspace, 0, 256, st32));
-        tag_store(StateTag{workspace, q, k, v, w, beta, log_f, B, H, L, d, scale}, false);   // this call overwrites the workspace
         float* G = nullptr;
         if (log_f) {
             G = at<float>(workspace, p.G);
@@ -454,7 +432,7 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     }
     // A workspace large enough for the backward gets the backward's layout: the chunk preparation then also keeps
     // the tiles the chain rule needs, and path_attn_bwd on the same workspace and inputs does not redo it.
-    const StateTag tag{workspace, q, k, v, w, beta, log_f, B, H, L, d, scale};
+    const StateRecord rec = make_record(q, k, v, w, beta, log_f, B, H, L, d, scale);   // (the caller's pointers, before padding)
     bool keep_state = false;
     {
         Plan pb;
@@ -470,7 +448,6 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     CK(cudaMemsetAsync(workspace, 0, 256, st));
 
     prof_reset(STG_PREP, STG_PREP_BWD);
-    tag_store(tag, false);
     rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, true, st);
     if (rc != PATH_OK) return rc;
     if (log_f) {
@@ -496,14 +473,14 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     if (log_f) fp.nkeep = at<int>(workspace, p.nkeep);   // block skipping: see run_gate_skip
     LAUNCH(launch_fa_fwd(tm, fp, d, st));
     prof_mark(STG_FA_FWD, 1, st);
-    if (keep_state) tag_store(tag, true);
+    if (keep_state) LAUNCH(launch_state_write(at<void>(workspace, p.status + kStateRecordOffset), rec, st));
     return PATH_OK;
 }
 
-int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, const float* beta, const float* log_f,
-                  const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
-                  float* dbeta, float* dlog_f, int B, int H, int L, int d, float scale, path_dtype_t dt,
-                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+static int backward_entry(const void* q, const void* k, const void* v, const void* w, const float* beta, const float* log_f,
+                          const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
+                          float* dbeta, float* dlog_f, int B, int H, int L, int d, float scale, path_dtype_t dt,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream, bool reuse) {
     g_launches = 0;
     if (!q || !k || !v || !w || !beta || !o || !lse || !d_o || !dq || !dk || !dv || !dw || !dbeta || !workspace)
         return PATH_ERR_NULL;
@@ -522,12 +499,14 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
     cudaStream_t st = (cudaStream_t)cuda_stream;
     CK(cudaMemsetAsync(workspace, 0, kSkipCounterOffset, st));   // the status word; the block-skipping counters may be reused
     prof_reset(STG_PREP_BWD, STG_COUNT);
-    const StateTag tag{workspace, q, k, v, w, beta, log_f, B, H, L, d, scale};
-    bool same_scale = false;
-    // the forward of this very problem left its preparation in this workspace (for a gated problem the scale has to be
-    // the same too: the block-skipping counts, and with them the levels the version chains were built up to, depend on it)
-    const bool reuse = tag_matches(tag, &same_scale) && (log_f == nullptr || same_scale);
-    if (!reuse) tag_store(tag, false);
+    if (reuse) {
+        // the record the forward left must describe this very problem (for a gated one the scale too: the block-skipping
+        // counts, and with them the levels the version chains were built up to, depend on it)
+        LAUNCH(launch_state_check(at<void>(workspace, p.status + kStateRecordOffset),
+                                  make_record(q, k, v, w, beta, log_f, B, H, L, d, scale), at<uint32_t>(workspace, p.status), st));
+    } else {
+        CK(cudaMemsetAsync(at<uint8_t>(workspace, p.status + kStateRecordOffset), 0, sizeof(StateRecord), st));
+    }
     rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, !reuse, st);
     if (rc != PATH_OK) return rc;
     if (!reuse) {
@@ -537,9 +516,37 @@ int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, co
         }
         rc = run_prep(p, workspace, q, k, w, true, st);
         if (rc != PATH_OK) return rc;
-        tag_store(tag, true);
     }
     return run_backward(p, workspace, q, k, v, w, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, scale, st);
+}
+
+int path_attn_bwd(const void* q, const void* k, const void* v, const void* w, const float* beta, const float* log_f,
+                  const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
+                  float* dbeta, float* dlog_f, int B, int H, int L, int d, float scale, path_dtype_t dt,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return backward_entry(q, k, v, w, beta, log_f, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, B, H, L, d, scale, dt,
+                          workspace, workspace_bytes, cuda_stream, false);
+}
+
+int path_attn_bwd_reuse(const void* q, const void* k, const void* v, const void* w, const float* beta, const float* log_f,
+                        const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
+                        float* dbeta, float* dlog_f, int B, int H, int L, int d, float scale, path_dtype_t dt,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return backward_entry(q, k, v, w, beta, log_f, o, lse, d_o, dq, dk, dv, dw, dbeta, dlog_f, B, H, L, d, scale, dt,
+                          workspace, workspace_bytes, cuda_stream, true);
+}
+
+int path_attn_selftest_timeout(void* workspace, unsigned int limit_us, void* cuda_stream) {
+    g_launches = 0;
+    if (!workspace) return PATH_ERR_NULL;
+    if ((uintptr_t)workspace & 255) return PATH_ERR_ALIGN;
+    if (limit_us < 1 || limit_us > 100000) return PATH_ERR_SHAPE;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CK(cudaMemsetAsync(workspace, 0, 256, st));
+    LAUNCH(launch_selftest_wait((uint32_t*)workspace, (long long)limit_us * 2000LL, st));   // ~2 clock ticks per ns
+    return PATH_OK;
 }
 
 }  // extern "C"
@@ -587,8 +594,8 @@ int path_attn_fwd_static(const void* q, const void* k, const void* v, const void
     if (rc != PATH_OK) return rc;
     const bool timing = path::g_prof.on;   // stage timing would create CUDA events on first use
     path::g_prof.on = false;
-    rc = path_attn_fwd(q, k, v, w, beta, log_f, o, lse, B, H, L, d, scale, dt, scratch,
-                       (size_t)PATH_ATTN_STATIC_SCRATCH_BYTES, cuda_stream);
+    // (the forward's own size, not the buffer's: a larger figure would select the backward's layout and keep its state)
+    rc = path_attn_fwd(q, k, v, w, beta, log_f, o, lse, B, H, L, d, scale, dt, scratch, need, cuda_stream);
     path::g_prof.on = timing;
     if (scratch_out) *scratch_out = scratch;
     return rc;
@@ -611,7 +618,6 @@ int path_attn_prefill_cache(const void* k, const void* v, const void* w, const f
     if (rc != PATH_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     CK(cudaMemsetAsync(workspace, 0, 256, st));
-    tag_store(StateTag{workspace, k, k, v, w, beta, log_f, B, H, L, d}, false);   // this call overwrites the workspace
     // the chunk preparation needs no queries for the key side: the keys stand in for them
     const void* qd = k; const void* kd = k; const void* vd = v; const void* wd = w;
     rc = stage_inputs(p, workspace, qd, kd, vd, wd, beta, log_f, true, st);
@@ -705,7 +711,7 @@ int path_attn_device_status(const void* workspace, void* cuda_stream, unsigned i
         return PATH_ERR_LAUNCH;
     }
     if (detail) *detail = word;
-    return word == 0 ? PATH_OK : PATH_ERR_TIMEOUT;
+    return word == 0 ? PATH_OK : (word == ST_STATE ? PATH_ERR_STATE : PATH_ERR_TIMEOUT);
 }
 
 int path_attn_skipped_chunk_pairs(const void* workspace, void* cuda_stream, unsigned long long* kept,
@@ -734,6 +740,7 @@ const char* path_attn_strerror(int status) {
         case PATH_ERR_LAUNCH: return "a CUDA call failed";
         case PATH_ERR_TIMEOUT: return "a bounded device-side wait ran out";
         case PATH_ERR_STATIC_LIMIT: return "problem needs more scratch than the built-in static buffer holds";
+        case PATH_ERR_STATE: return "the workspace does not hold the forward state of this problem (path_attn_bwd_reuse)";
         default: return "unknown status";
     }
 }

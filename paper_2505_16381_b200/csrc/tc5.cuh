@@ -43,7 +43,8 @@ constexpr long long kWaitTicks = 2000000000LL;
 
 // Waits for the phase with the given parity.  Returns false (and raises *abort_flag with
 // `code`) if the limit ran out or another thread of the CTA already gave up.
-__device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code) {
+__device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code,
+                                               long long limit_ticks = kWaitTicks) {
     long long t0 = clock64();
 #pragma unroll 1
     for (;;) {
@@ -51,7 +52,7 @@ __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, v
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag != 0) return false;
-        if (clock64() - t0 > kWaitTicks) {
+        if (clock64() - t0 > limit_ticks) {
             atomicCAS((uint32_t*)abort_flag, 0u, code);
             return false;
         }

@@ -35,6 +35,26 @@ def test_path_attention_autograd_matches_oracle(oracle, gate):
         assert rel_fro(f64(log_f.grad).reshape(ref["dlog_f"].shape), ref["dlog_f"]) <= 1e-2
 
 
+@pytest.mark.parametrize("retain", [False, True])
+def test_path_attention_autograd_takes_transposed_views(oracle, retain):
+    """The usual layer layout: q, k, v, w arrive as [B, L, H, d].transpose(1, 2) and beta, log_f as [B, L, H].transpose(1, 2):
+    none of them contiguous, all of them requiring grad."""
+    from paper_2505_16381_b200.autograd import path_attention
+    B, H, L, d = 1, 2, 200, 64
+    inp = synth.make_inputs(B, H, L, d, "bf16", gate=True, seed=8150)
+    base = {n: inp[n].transpose(1, 2).contiguous().cuda().requires_grad_(True) for n in ("q", "k", "v", "w", "beta", "log_f")}
+    view = {n: t.transpose(1, 2) for n, t in base.items()}
+    assert not view["q"].is_contiguous() and not view["beta"].is_contiguous()
+    o = path_attention(view["q"], view["k"], view["v"], view["w"], view["beta"], view["log_f"], retain_state=retain)
+    o.backward(inp["d_o"].cuda())
+    f64 = synth.to_f64
+    ref = oracle.backward(f64(inp["q"]), f64(inp["k"]), f64(inp["v"]), f64(inp["w"]), f64(inp["beta"]), f64(inp["d_o"]),
+                          f64(inp["log_f"]))
+    for n, r in (("q", "dq"), ("k", "dk"), ("v", "dv"), ("w", "dw"), ("beta", "dbeta"), ("log_f", "dlog_f")):
+        got = f64(base[n].grad.transpose(1, 2)).reshape(ref[r].shape)
+        assert rel_fro(got, ref[r]) <= 1e-2, r
+
+
 def test_frontend_then_operator_autograd_chain(oracle):
     from paper_2505_16381_b200.autograd import path_attention, path_frontend
     B, H, L, d = 1, 2, 300, 64

@@ -326,6 +326,41 @@ def test_backward_matches_central_differences(oracle, gate):
         assert err < 2e-7 * max(1.0, np.abs(num).max()), (name, err)
 
 
+@pytest.mark.parametrize("gate", [False, True])
+def test_backward_with_an_lse_gradient_matches_central_differences(oracle, gate):
+    """Loss sum(O dO) + sum(lse dlse): the lse term alone, against central differences of the forward's lse, and
+    the sum rule (gradients add)."""
+    rng = np.random.default_rng(15)
+    L, d, scale = 9, 4, 0.7
+    q, k, v, w, beta, g = rand_problem(rng, L, d, unit_w=False, gate=gate)
+    d_o = rng.standard_normal((L, d))
+    d_lse = rng.standard_normal(L)
+    both = oracle.backward(q, k, v, w, beta, d_o, g, scale=scale, d_lse=d_lse)
+    only_o = oracle.backward(q, k, v, w, beta, d_o, g, scale=scale)
+    only_l = oracle.backward(q, k, v, w, beta, np.zeros_like(d_o), g, scale=scale, d_lse=d_lse)
+    for n in both:
+        assert np.abs(both[n] - (only_o[n] + only_l[n])).max() < 1e-12, n
+    assert np.abs(only_l["dv"]).max() == 0.0                      # lse does not depend on v
+    lse_loss = lambda: float(np.sum(oracle.forward(q, k, v, w, beta, g, scale=scale)[1] * d_lse))
+    args = {"q": q, "k": k, "w": w, "beta": beta}
+    names = {"q": "dq", "k": "dk", "w": "dw", "beta": "dbeta"}
+    if gate:
+        args["g"] = g; names["g"] = "dlog_f"
+    eps = 1e-6
+    for name, arr in args.items():
+        num = np.zeros_like(arr)
+        it = np.nditer(arr, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            old = arr[idx]
+            arr[idx] = old + eps; lp = lse_loss()
+            arr[idx] = old - eps; lm = lse_loss()
+            arr[idx] = old
+            num[idx] = (lp - lm) / (2 * eps)
+        err = np.abs(num - only_l[names[name]]).max()
+        assert err < 2e-7 * max(1.0, np.abs(num).max()), (name, err)
+
+
 def _boxed_forward_torch(q, k, v, w, beta, g, scale):
     """The paper's closed matrix form (Sec. 3.2) in torch float64, differentiable by autograd."""
     L = q.shape[0]

@@ -37,20 +37,24 @@ def gpu_forward(b, dev, scale):
 
 def gpu_backward(b, dev, o, lse, scale):
     ws = b.alloc_workspace(dev["q"], dev["log_f"] is not None, True)
+    ws.fill_(0xFF)      # (NaN patterns) whatever an earlier problem left at these addresses must not matter: the backward recomputes
     g = b.path_attn_bwd(dev["q"], dev["k"], dev["v"], dev["w"], dev["beta"], o, lse, dev["d_o"], dev["log_f"],
                         scale=scale, workspace=ws)
     assert b.device_status(ws) == 0
     return g
 
 
-def check(name, got, ref, rel=REL_FRO, mx=MAX_ABS):
+def check(name, got, ref, rel=REL_FRO, mx=MAX_ABS, unscaled_below=1.0):
+    """rel-Fro <= rel and max-abs <= mx, the latter scaled by max|ref| only where max|ref| exceeds `unscaled_below`
+    (the named workloads pass 4.0: up to that magnitude half a bf16 ulp, 2^-9 |ref|, still leaves room under 2e-2)."""
     got = got.detach().float().cpu().double().numpy() if torch.is_tensor(got) else got
     err = np.abs(got - ref).max()
     nrm = np.linalg.norm(ref)
+    top = np.abs(ref).max()
     relerr = np.linalg.norm(got - ref) / nrm if nrm > 0 else np.linalg.norm(got)
     assert np.isfinite(got).all(), name
     assert relerr <= rel, (name, "rel-fro", relerr)
-    assert err <= mx * max(1.0, np.abs(ref).max()), (name, "max-abs", err)
+    assert err <= mx * (1.0 if top <= unscaled_below else top), (name, "max-abs", err, "max|ref|", top)
 
 
 def slices(inp, idx):
@@ -60,7 +64,7 @@ def slices(inp, idx):
     return {n: pick(inp[n]) for n in ("q", "k", "v", "w", "beta", "d_o", "log_f")}
 
 
-def compare_all(b, oracle, inp, scale=1.0, idx=None, backward=True):
+def compare_all(b, oracle, inp, scale=1.0, idx=None, backward=True, unscaled_below=1.0):
     dev = to_dev(inp)
     S = inp["q"].shape[0] * inp["q"].shape[1]
     idx = list(range(S)) if idx is None else idx
@@ -68,14 +72,14 @@ def compare_all(b, oracle, inp, scale=1.0, idx=None, backward=True):
     x = slices(inp, idx)
     o_ref, lse_ref = oracle.forward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["log_f"], scale=scale)
     flat = lambda t: t.reshape(-1, *t.shape[2:])[idx]
-    check("o", flat(o), o_ref)
+    check("o", flat(o), o_ref, unscaled_below=unscaled_below)
     assert np.abs(flat(lse).cpu().double().numpy() - lse_ref).max() <= 2e-3 * max(1.0, np.abs(lse_ref).max())
     if not backward:
         return o, lse, None
     g = gpu_backward(b, dev, o, lse, scale)
     ref = oracle.backward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["d_o"], x["log_f"], scale=scale)
     for name, r in ref.items():
-        check(name, flat(g[name]), r)
+        check(name, flat(g[name]), r, unscaled_below=unscaled_below)
     return o, lse, g
 
 
@@ -150,6 +154,51 @@ def test_random_gated_problems(binding, oracle, B, H, L, d, shift, wild, scale, 
         inp["w"] = (inp["w"].float() * (1.0 + 0.15 * torch.rand(B, H, L, 1, generator=gen))).to(torch.bfloat16).contiguous()
         inp["beta"] = (inp["beta"] * 1.2).contiguous()
     compare_all(binding, oracle, inp, scale=scale)
+
+
+def test_short_gated_problems_down_to_one_token(binding, oracle):
+    """300 seeded PaTH-FoX problems of 1 to 15 tokens, gates from negligible to e^-2 per token, three scales.
+
+    Two things set these apart from the workloads, and the criterion says so instead of leaving them out:
+    (1) The backward's input `o` is bf16 (the ABI's dtype), so delta_i = dO_i . o_i is off by eps_i = dO_i . (o_i - O_i) and
+        every ds_ij moves by -p_ij eps_i, whatever the kernels do.  Under a strong gate on a handful of tokens the attention
+        is nearly the identity, the exact ds is nearly zero and this term is all there is.  d lse_i / d s_ij = p_ij, so
+        that perturbation is exactly an upstream gradient -eps_i on lse_i: the reference here is the oracle's backward
+        for  sum(O dO) - sum(eps lse),  i.e. the gradient the definition gives for the o the call was handed.
+    (2) dbeta / dw of such a problem can be carried by one or two entries of magnitude 1e-3; each comes out of four to five
+        products of bf16-rounded operands (2^-9 relative each), which average out over a workload's thousands of
+        entries but not here.  A tensor whose largest reference entry is below 0.05 is therefore judged by
+        max-abs <= 1e-3 (the absolute bound 2e-2 scaled to that floor) where it misses the relative bound.
+    Against the plain oracle every tensor still meets the absolute bound."""
+    import random
+    rng = random.Random(3)
+    f = synth.to_f64
+    worst = {}
+    for i in range(300):
+        B, H, d = rng.choice([1, 2, 3]), rng.choice([1, 2, 3]), rng.choice([64, 128])
+        L = rng.randint(1, 15)
+        shift, scale = rng.choice([-2.0, -1.0, 0.0, 1.0, 3.0, 5.0]), rng.choice([1.0, 0.5, -0.25])
+        inp = synth.make_inputs(B, H, L, d, "bf16", gate=True, seed=7000 + i)
+        gen = torch.Generator().manual_seed(7007 + i)
+        inp["log_f"] = torch.nn.functional.logsigmoid(torch.randn(B, H, L, generator=gen) + shift).contiguous()
+        dev = to_dev(inp)
+        o, lse = gpu_forward(binding, dev, scale)
+        g = gpu_backward(binding, dev, o, lse, scale)
+        x = {n: f(inp[n]) for n in ("q", "k", "v", "w", "beta", "d_o", "log_f")}
+        o_ref, lse_ref = oracle.forward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["log_f"], scale=scale)
+        check("o", o, o_ref)
+        eps = np.sum(x["d_o"] * (f(o) - o_ref), -1)
+        ref = oracle.backward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["d_o"], x["log_f"], scale=scale, d_lse=-eps)
+        plain = oracle.backward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["d_o"], x["log_f"], scale=scale)
+        for name, r in ref.items():
+            got = f(g[name]).reshape(r.shape)
+            assert np.isfinite(got).all(), (i, name)
+            err, nrm, top = np.abs(got - r).max(), np.linalg.norm(plain[name]), np.abs(plain[name]).max()
+            rel = np.linalg.norm(got - r) / nrm if nrm > 0 else np.linalg.norm(got - r)
+            assert rel <= REL_FRO or (top < 0.05 and err <= 1e-3), (i, name, L, d, shift, scale, rel, err, top)
+            assert np.abs(got - plain[name]).max() <= MAX_ABS * max(1.0, top), (i, name, "max-abs vs the plain oracle")
+            worst[name] = max(worst.get(name, 0.0), rel if top >= 0.05 else 0.0)
+    assert max(worst.values()) <= REL_FRO
 
 
 def test_c1_workload_shape_and_distribution_in_bf16(binding, oracle):
@@ -234,20 +283,25 @@ def test_forward_is_bitwise_reproducible_and_workspace_is_reusable(binding):
     inp = to_dev(synth.make_inputs(2, 2, 1024, 128, "bf16", gate=True, seed=3))
     ws = binding.alloc_workspace(inp["q"], True, True)   # backward-sized: shared by both directions
     run = lambda: binding.path_attn_fwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"], inp["log_f"], workspace=ws)
+    bwd = lambda o, l, reuse: binding.path_attn_bwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"], o, l, inp["d_o"],
+                                                    inp["log_f"], workspace=ws, reuse=reuse)
     o1, l1 = run()
-    g1 = binding.path_attn_bwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"], o1, l1, inp["d_o"], inp["log_f"],
-                               workspace=ws)
+    g1 = bwd(o1, l1, True)
+    assert binding.device_status(ws) == 0
     o2, l2 = run()
     assert torch.equal(o1, o2) and torch.equal(l1, l2)
-    g2 = binding.path_attn_bwd(inp["q"], inp["k"], inp["v"], inp["w"], inp["beta"], o1, l1, inp["d_o"], inp["log_f"],
-                               workspace=ws)
+    g2 = bwd(o1, l1, True)
+    g3 = bwd(o1, l1, False)
     for n in g1:  # float atomics in the run-product gradients: equal to rounding, not bitwise
         assert torch.allclose(g1[n].float(), g2[n].float(), rtol=2e-2, atol=1e-3), n
-    assert torch.equal(g1["dv"], g2["dv"])
+        assert torch.allclose(g1[n].float(), g3[n].float(), rtol=2e-2, atol=1e-3), n
+    assert torch.equal(g1["dv"], g2["dv"]) and torch.equal(g1["dv"], g3["dv"])
     assert binding.device_status(ws) == 0
 
 
-def test_backward_reuses_forward_state_only_for_the_same_problem(binding):
+def test_backward_reuse_is_explicit_and_checked_on_the_device(binding, oracle):
+    """path_attn_bwd never depends on what is in the workspace; path_attn_bwd_reuse takes the forward's chunk preparation
+    and reports PATH_ERR_STATE (-10) when the workspace holds no forward state of this very problem."""
     a = to_dev(synth.make_inputs(1, 2, 700, 128, "bf16", gate=True, seed=31))
     b_ = to_dev(synth.make_inputs(1, 2, 700, 128, "bf16", gate=True, seed=32))
     args = lambda t: (t["q"], t["k"], t["v"], t["w"], t["beta"])
@@ -255,32 +309,72 @@ def test_backward_reuses_forward_state_only_for_the_same_problem(binding):
     fresh = lambda t, o, lse: binding.path_attn_bwd(*args(t), o, lse, t["d_o"], t["log_f"],
                                                     workspace=binding.alloc_workspace(t["q"], True, True))
     o_a, lse_a = binding.path_attn_fwd(*args(a), a["log_f"], workspace=ws)          # leaves its preparation in ws
-    g_reuse = binding.path_attn_bwd(*args(a), o_a, lse_a, a["d_o"], a["log_f"], workspace=ws)
+    g_reuse = binding.path_attn_bwd(*args(a), o_a, lse_a, a["d_o"], a["log_f"], workspace=ws, reuse=True)
     n_reuse = binding.last_launch_count()
+    assert binding.device_status(ws) == 0
     g_fresh = fresh(a, o_a, lse_a)
     assert n_reuse < binding.last_launch_count()                                   # the preparation was skipped
     for n in g_fresh:
         assert torch.allclose(g_reuse[n].float(), g_fresh[n].float(), rtol=2e-2, atol=1e-3), n
-    # same workspace, other problem: nothing stale may be reused
+
+    def state_error(call):
+        call()
+        with pytest.raises(binding.PathAttnError) as e:
+            binding.device_status(ws)
+        assert e.value.status == -10
+
+    # the workspace holds problem a's state: reuse for problem b is refused
     o_b, lse_b = binding.path_attn_fwd(*args(b_), b_["log_f"])
-    binding.path_attn_fwd(*args(a), a["log_f"], workspace=ws)
-    g_b = binding.path_attn_bwd(*args(b_), o_b, lse_b, b_["d_o"], b_["log_f"], workspace=ws)
-    g_b_fresh = fresh(b_, o_b, lse_b)
-    for n in g_b_fresh:
-        assert torch.allclose(g_b[n].float(), g_b_fresh[n].float(), rtol=2e-2, atol=1e-3), n
+    state_error(lambda: binding.path_attn_bwd(*args(b_), o_b, lse_b, b_["d_o"], b_["log_f"], workspace=ws, reuse=True))
+    # a plain backward consumed the workspace: its record is gone
+    binding.path_attn_bwd(*args(b_), o_b, lse_b, b_["d_o"], b_["log_f"], workspace=ws)
     assert binding.device_status(ws) == 0
+    state_error(lambda: binding.path_attn_bwd(*args(a), o_a, lse_a, a["d_o"], a["log_f"], workspace=ws, reuse=True))
+    # a gated problem's state belongs to one scale
+    binding.path_attn_fwd(*args(a), a["log_f"], scale=0.5, workspace=ws)
+    state_error(lambda: binding.path_attn_bwd(*args(a), o_a, lse_a, a["d_o"], a["log_f"], scale=1.0, workspace=ws, reuse=True))
+    # a forward on a forward-sized workspace keeps no state
+    small = binding.alloc_workspace(a["q"], True, False)
+    binding.path_attn_fwd(*args(a), a["log_f"], workspace=small)
+    ws.zero_()
+    state_error(lambda: binding.path_attn_bwd(*args(a), o_a, lse_a, a["d_o"], a["log_f"], workspace=ws, reuse=True))
+    # and the plain backward on that same workspace is clean and right
+    g = binding.path_attn_bwd(*args(a), o_a, lse_a, a["d_o"], a["log_f"], workspace=ws)
+    assert binding.device_status(ws) == 0
+    for n in g_fresh:
+        assert torch.allclose(g[n].float(), g_fresh[n].float(), rtol=2e-2, atol=1e-3), n
+
+
+def test_backward_after_an_in_place_rewrite_of_the_inputs(binding, oracle):
+    """Forward, then q, k, w, beta rewritten in place (same addresses), then the plain backward on the same workspace:
+    the gradients are those of the new contents, checked against the oracle."""
+    a = synth.make_inputs(1, 2, 640, 64, "bf16", gate=False, seed=41)
+    b_ = synth.make_inputs(1, 2, 640, 64, "bf16", gate=False, seed=42)
+    dev = to_dev(a)
+    ws = binding.alloc_workspace(dev["q"], False, True)
+    args = (dev["q"], dev["k"], dev["v"], dev["w"], dev["beta"])
+    binding.path_attn_fwd(*args, None, workspace=ws)
+    for n in ("q", "k", "v", "w", "beta", "d_o"):
+        dev[n].copy_(b_[n])
+    o, lse = binding.path_attn_fwd(*args, None)                     # forward of the new contents, elsewhere
+    g = binding.path_attn_bwd(*args, o, lse, dev["d_o"], None, workspace=ws)
+    assert binding.device_status(ws) == 0
+    x = slices(b_, [0, 1])
+    ref = oracle.backward(x["q"], x["k"], x["v"], x["w"], x["beta"], x["d_o"], None)
+    for name, r in ref.items():
+        check(name, g[name].reshape(-1, *g[name].shape[2:]), r)
 
 
 # ---------------------------------------------------------------- the named workloads at full size
 
 def test_c2_full_size_sampled_slices(binding, oracle):
     inp = synth.make_config("C2")
-    compare_all(binding, oracle, inp, idx=[0, 37, 127])
+    compare_all(binding, oracle, inp, idx=[0, 37, 64, 127], unscaled_below=4.0)
 
 
 def test_c3_headline_full_size_sampled_slices_and_invariants(binding, oracle):
     inp = synth.make_config("C3")
-    o, lse, g = compare_all(binding, oracle, inp, idx=[0, 63])
+    o, lse, g = compare_all(binding, oracle, inp, idx=[0, 5, 17, 22, 31, 40, 54, 63], unscaled_below=4.0)
     # exact invariants that hold at any size (all slices)
     w, beta = inp["w"].double(), inp["beta"].double()
     dw, dbeta = g["dw"].cpu().double(), g["dbeta"].cpu().double()
@@ -293,9 +387,9 @@ def test_c3_headline_full_size_sampled_slices_and_invariants(binding, oracle):
     assert torch.isfinite(g["dq"]).all() and torch.isfinite(o).all()
 
 
-def test_c4_path_fox_full_size_one_slice(binding, oracle):
+def test_c4_path_fox_full_size_sampled_slices(binding, oracle):
     inp = synth.make_config("C4")
-    compare_all(binding, oracle, inp, idx=[17])
+    compare_all(binding, oracle, inp, idx=[0, 9, 17, 31], unscaled_below=4.0)
 
 
 def test_c5_long_prefill_forward_sampled_rows(binding, oracle):
@@ -312,7 +406,7 @@ def test_c5_long_prefill_forward_sampled_rows(binding, oracle):
     o_ref, lse_ref = oracle.forward(pick(inp["q"]), pick(inp["k"]), pick(inp["v"]), pick(inp["w"]), pick(inp["beta"]),
                                     None, scale=1.0, rows=rows)
     og = o.reshape(-1, L, o.shape[-1])[idx][:, rows]
-    check("o", og, o_ref)
+    check("o", og, o_ref, unscaled_below=4.0)
     lg = lse.reshape(-1, L)[idx][:, rows].cpu().double().numpy()
     assert np.abs(lg - lse_ref).max() <= 2e-3 * max(1.0, np.abs(lse_ref).max())
     assert torch.isfinite(o).all()
