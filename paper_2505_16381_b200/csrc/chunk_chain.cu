@@ -84,15 +84,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         ok = __syncthreads_and(ok);
         tc_fence_after_sync();
     };
-    // float rows of a [nrows][ncols] global matrix -> bf16 tile (rows >= nrows read as zero)
-    auto conv = [&](const float* src, int ncols, int nrows, uint8_t* dst) {
-        const int per = ncols / 2;
-        for (int c = 0; c < per / 32; ++c) {
-            const int c0 = half * per + c * 32;
-            gload_f32x32(src + (size_t)row * ncols + c0, v, row < nrows);
-            tile_store32(dst, row, c0, v);
-        }
-    };
     // accumulator [128][ncols] -> f(row values) -> bf16 tile
     enum { M_NONE = 0, M_LOWER = 1, M_STRICT = 2 };
     auto acc_to_tile = [&](uint32_t col, int ncols, uint8_t* dst, float mul, int mask) {
@@ -142,9 +133,10 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
 
     // slots: 0 U->W   1 dQl->dT->tmp->dGm   2 Y^T->-Xq->Xk->T->Ah->K   3 dSd->T lo->dT lo->tmp lo->dSd   4 dXq   5 dKr->dY->dXk
     //        6 dP->dU->Al->Q
-    // first tiles of a chunk: U, Y, (s dSd)^T (every use below takes the transposed view), dQl, dKr
+    // first tiles of a chunk: U, Y, (s dSd)^T (every use below takes the transposed view), dQl, dKr, dP
     auto first_loads = [&](int ch) {
-        mbar_expect_tx(&bars[0], 3 * kT * HD * 2 + 2 * kTileB);
+        mbar_expect_tx(&bars[0], 4 * kT * HD * 2 + 2 * kTileB);
+        tma_tile(slot(6), &tm.dp, &bars[0], HD, ch * HD);
         tma_tile(slot(0), &tm.u, &bars[0], HD, ch * kT);
         tma_tile(slot(2), &tm.yt, &bars[0], kT, ch * kT);
         tma_tile(slot(3), &tm.dsdt, &bars[0], kT, ch * kT);
@@ -160,11 +152,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     const size_t urow = (size_t)s_idx * p.L + pos;                   // row in the caller's [S][L][.] tensors
     const __nv_bfloat16* g_dql = p.dql + ((size_t)chunk * kT + row) * HD;
     const __nv_bfloat16* g_dkr = p.dkr + ((size_t)chunk * kT + row) * HD;
-    const float* g_dp = p.dp + (size_t)chunk * HD * HD;
     const int r0 = chunk * kT;
     if (tid < kT) bt[tid] = p.beta[(size_t)chunk * kT + tid];   // first read after several barriers (phase 4)
     // ---- phase 0a: dXq = lower(-(dQl U^T + s dSd Y^T))
-    conv(g_dp, HD, HD, slot(6));
     loads_wait();
     publish();
     if (tid == 0) {

@@ -83,22 +83,25 @@ struct LevelTensorMaps {
     CUtensorMap dyh, dyl;   // [matrices * d][d] bf16 hi / lo planes of the run products
     CUtensorMap qv, kv;     // [slots * S * Lp][d] bf16 versions
     CUtensorMap dqv, dkv;   // same shape: bf16 gradients of the versions (backward only)
+    CUtensorMap ddy;        // [matrices * d][d] bf16 gradients of the run products (backward only)
 };
 
 struct LevelParams {
     LevelTable lv;
-    int l;                  // dyadic kernels: level being produced (fwd: l -> l + 1) / consumed (bwd); version kernels: number of levels
+    int l;                  // dyadic forward: level consumed (l -> l + 1); version forward: number of levels; level backward: the
+                            // level of the run products whose gradients the launch finishes
+    int nlev;               // number of levels (level backward)
     int S, N, Lp;
     __nv_bfloat16 *dyh, *dyl, *qv, *kv;
     __nv_bfloat16 *dqv, *dkv;     // [slots][S][Lp][d] gradients of the versions; slot 0 ends up holding the final sums
-    float* ddy;
+    __nv_bfloat16* ddy16;         // gradients of the run products, same placement as the run products themselves
     float* kc;                    // key-cache kernel: [S][cap][d] float32 out (rows < L of every slice)
     int cap, L;
     const int *nkeep, *nvisit;    // version backward: chunk counts of a sweep shortened by block skipping ([S][N]), or nullptr
     uint32_t* status;
 };
 
-enum { LEVEL_DYADIC_FWD = 0, LEVEL_VERSION_FWD, LEVEL_VERSION_BWD, LEVEL_DYADIC_BWD, LEVEL_KEY_CACHE };
+enum { LEVEL_DYADIC_FWD = 0, LEVEL_VERSION_FWD, LEVEL_BWD, LEVEL_KEY_CACHE };
 cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const LevelParams& p, int hd, cudaStream_t st);
 
 struct PrepTensorMaps {
@@ -130,12 +133,12 @@ struct ChainTensorMaps {
     CUtensorMap yt, xqn, xk, th, tl, ah, al;      // [S*Lp][128]; yt = Y^T and xqn = -Xq are the attention sweep's operands
     CUtensorMap dsdt;                             // [S*N*128][128] bf16: (scale * lower(dS))^T of the diagonal chunks
     CUtensorMap dql, dkr;                         // [S*Lp][d] bf16 gradients of the boundary-adjusted queries / keys
+    CUtensorMap dp;                               // [S*N*d][d] bf16 gradients of the chunk products
 };
 
 struct ChainParams {
     const __nv_bfloat16* dql;   // [S*Lp][d]  gradient of the boundary-adjusted queries (version slot 0), bf16
     const __nv_bfloat16* dkr;   // [S*Lp][d]  gradient of the boundary-adjusted keys, bf16
-    const float* dp;      // [S*N][d][d] gradient of the chunk products
     const float* beta;    // [S*Lp]
     __nv_bfloat16 *dq, *dk, *dw;   // [S][L][d] outputs
     float* dbeta;         // [S][L]

@@ -8,7 +8,7 @@
 //     Dy[l+1][b] = Dy[l][2b+1] Dy[l][2b]                                                (dyadic_fwd)
 //     Qv[l2][I]  = Qv[l1][I] Dy[l1][(I >> l2 << l2) >> l1]      l1 < l2 consecutive set bits of I     (version_fwd)
 //     Kv[l2][J]  = Kv[l1][J] Dy[l1][(J >> l1) + 1]^T            l1 < l2 consecutive clear bits of J
-// and the backward kernels apply the chain rule to exactly these products.  Run products are stored as bf16
+// and the backward kernel (level_bwd) applies the chain rule to exactly these products, level by level.  Run products are stored as bf16
 // hi + lo pairs (they are multiplied up to log2(N) times); versions are bf16, the values the sweep consumes.
 #include "tileops.cuh"
 
@@ -75,41 +75,6 @@ __device__ __forceinline__ void mma_wait(Ctx& c) {
     c.ok = __syncthreads_and(c.ok);
     tc_fence_after_sync();
 }
-// float rows [nrows][ncols] of a global matrix -> bf16 tile (rows >= nrows are zero-filled)
-__device__ __forceinline__ void conv(const Ctx& c, const float* src, int ncols, int nrows, uint8_t* dst) {
-    const int per = ncols / 2;
-    float v[32];
-    for (int i = 0; i < per / 32; ++i) {
-        const int c0 = c.half * per + i * 32;
-        gload_f32x32(src + (size_t)c.row * ncols + c0, v, c.row < nrows);
-        tile_store32(dst, c.row, c0, v);
-    }
-}
-// accumulator rows -> global float matrix [nrows][ncols]: dst += acc (plain or atomic)
-template <bool ATOMIC>
-__device__ __forceinline__ void acc_add_global(const Ctx& c, uint32_t col, int ncols, int nrows, float* dst) {
-    const int per = ncols / 2;
-    float v[32];
-    for (int i = 0; i < per / 32; ++i) {
-        const int c0 = c.half * per + i * 32;
-        tmem_row32(c.tl + col + c0, v);
-        const bool live = c.row < nrows;
-        float* d = dst + (size_t)c.row * ncols + c0;
-        if (ATOMIC) {
-            if (live) {
-#pragma unroll
-                for (int x = 0; x < 32; ++x) atomicAdd(d + x, v[x]);
-            }
-        } else {
-            float o[32];
-            gload_f32x32(d, o, live);
-#pragma unroll
-            for (int x = 0; x < 32; ++x) o[x] += v[x];
-            gstore_f32x32(d, o, live);
-        }
-    }
-}
-
 // Resolves the version-chain step of chunk c at level l2.  Returns false if there is none.
 __device__ __forceinline__ bool version_step(int is_key, int c, int l2, int N, int& l1, int& b, int& src_slot) {
     if (!is_key) {
@@ -198,7 +163,7 @@ __device__ __forceinline__ int highest_level_reached(const LevelParams& p, int i
 template <int HD>
 __global__ void __launch_bounds__(256, 2) version_fwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
     const int is_key = blockIdx.y, s = blockIdx.x / p.N, ch = blockIdx.x % p.N;
-    // levels to build: all of them, or for a gated problem up to the highest one a kept chunk pair uses (see version_bwd)
+    // levels to build: all of them, or for a gated problem up to the highest one a kept chunk pair uses (see level_bwd)
     const int lim = min(p.l, highest_level_reached(p, is_key, s, ch) + 1);
     int l1, b, src, l2 = 1;
     for (; l2 < lim; ++l2)
@@ -249,210 +214,165 @@ __global__ void __launch_bounds__(256, 2) version_fwd_kernel(const __grid_consta
     teardown<128>(c, p.status);
 }
 
-// ---------------------------------------------------------------------------------------------- version backward
-// grid = (S * N, 2), p.l = number of levels.  One CTA walks the chain of its chunk top level first.  With
-// g = dXv[l2][chunk] (what the sweeps wrote there plus what arrived from the level above, which stays in tensor memory):
-//     dXv[l1][chunk] += g Dy^T (queries) or g Dy (keys);
-//     dDy[l1][b]     += Xv[l1]^T g (queries) or g^T Xv[l1] (keys), atomically.
-// The run products enter the backward as single bf16 operands (their hi plane), like every other operand of a gradient
-// product; the lo plane only matters where products are chained (forward).  Gradients of the versions are bf16 (written
-// by the sweeps).  Only the bottom of the chain (always slot 0) leaves the
-// CTA: added in place to the slot-0 gradient, which the chunk chain rule then loads as a tile.  The next step's operands are fetched while the
-// current one runs.
+// ---------------------------------------------------------------------------------------------- level backward
+// Chain rule of the version chains and of the run products, one launch per level l1 = nlev-2, ..., 0 (p.l = l1),
+// grid.x = S * cnt(l1).  A CTA owns ONE run product Dy[l1][b] and gathers its whole gradient in tensor memory, so nothing
+// is added atomically and nothing has to be cleared beforehand:
+//   (1) the level above (Dy[l1+1][b'] = Dy[l1][2b'+1] Dy[l1][2b'], finished by the previous launch), dC = dDy[l1+1][b >> 1]:
+//         b odd:  dDy = dC Dy[l1][b-1]^T          b even:  dDy = Dy[l1][b+1]^T dC
+//   (2) every version step that multiplies by Dy[l1][b]: the 2^l1 chunks ch of one aligned run, all at the same
+//       target level l2 > l1, with g = dXv[l2][ch] (what the sweeps wrote there plus what earlier launches added):
+//         queries (b even, b >= 2, ch = (b << l1) + 2^l1 + x):   dDy += Qv[l1][ch]^T g,   dQv[l1][ch] += g Dy^T
+//         keys    (b odd,          ch = ((b-1) << l1) + x):      dDy += g^T Kv[l1][ch],   dKv[l1][ch] += g Dy
+//       (the second product is the chain's carry: added in place to the gradient the sweep left at level l1, which the
+//       launch of level l1's own source level, or the chunk chain rule for slot 0, reads next).
+// The run products enter as single bf16 operands (their hi plane), like every other operand of a gradient product.
+// dDy is written once, as bf16: it is only ever read as an MMA operand (by the next launch and, at level 0, by the
+// chunk chain rule as dP).  Runs with b = 0 multiply nothing (no boundary lies before chunk 0): only level 0 writes them.
 template <int HD>
-__global__ void __launch_bounds__(256, 1) version_bwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
-    const int is_key = blockIdx.y, s = blockIdx.x / p.N, ch = blockIdx.x % p.N;
-    int l1, b, src;
-    auto next_step = [&](int from) {   // highest level <= from with a version step, 0 if none
-        for (int l = from; l >= 1; --l)
-            if (version_step(is_key, ch, l, p.N, l1, b, src)) return l;
-        return 0;
+__global__ void __launch_bounds__(256, 1) level_bwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
+    const int l1 = p.l, cnt = p.lv.dy_cnt[l1];
+    const int s = blockIdx.x / cnt, b = blockIdx.x % cnt;
+    const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * cnt + b;
+    const int is_key = b & 1;
+    // the chunks of this run's version steps and their common target level
+    const int c0 = is_key ? ((b - 1) << l1) : ((b << l1) + (1 << l1));
+    int l2 = 0;
+    bool role = is_key || b >= 2;
+    if (role) {
+        if (!is_key) l2 = lowest_set((unsigned)(b << l1));
+        else l2 = l1 + 1 + lowest_set(~((unsigned)c0 >> (l1 + 1)));
+        role = l2 < p.nlev;
+    }
+    int src = 0;
+    auto valid = [&](int ch) {   // does chunk ch take the step l1 -> l2 through this run product?
+        if (!role || ch >= p.N) return false;
+        int l1x, bx;
+        if (!version_step(is_key, ch, l2, p.N, l1x, bx, src) || l1x != l1) return false;
+        return l2 <= highest_level_reached(p, is_key, s, ch);   // block skipping: levels the sweeps did not reach hold nothing
     };
-    // A sweep shortened by block skipping has written the gradients of the levels it reached only (the near ones); the
-    // chain starts at the highest of them instead of the top (everything above would have been zero).
-    const int top = min(p.l - 1, highest_level_reached(p, is_key, s, ch));
-    int l2 = next_step(top);
-    if (l2 == 0) return;   // no chain: what the sweeps left in slot 0 is final
+    auto next_chunk = [&](int from) {
+        for (int ch = from; ch < c0 + (1 << l1); ++ch)
+            if (valid(ch)) return ch;
+        return -1;
+    };
+    const bool parent = l1 + 1 <= p.nlev - 2 && (b >> 1) >= 1 && (b >> 1) < p.lv.dy_cnt[l1 + 1];
+    int ch = next_chunk(c0);
+    __nv_bfloat16* out = p.ddy16 + (size_t)mat * HD * HD;
+    if (ch < 0 && !parent) {   // nothing multiplies by this run product
+        if (b >= 1 || l1 == 0)
+            for (int i = threadIdx.x; i < HD * HD / 8; i += 256) reinterpret_cast<uint4*>(out)[i] = make_uint4(0u, 0u, 0u, 0u);
+        return;
+    }
     __nv_bfloat16* dxv = is_key ? p.dkv : p.dqv;
     extern __shared__ uint8_t smem_raw[];
     Ctx c;
     setup<256>(c, smem_raw, 7 * kTileB);
-    uint8_t* sm = c.smem;   // slot 0: g; two buffers of three slots: Dy (hi plane), -, Xv[l1]; a buffer is also the staging area
-    auto issue_loads = [&](int buf, uint32_t more_bytes = 0) {   // operands of the step described by (l1, b, src)
-        const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
-        const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
-        uint8_t* base = sm + (1 + 3 * buf) * kTileB;
-        mbar_expect_tx(&c.bars[0], 2 * kT * HD * 2 + more_bytes);   // one arrival per phase: every byte is announced here
-        tma_tile(base, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
-        tma_tile(base + 2 * kTileB, is_key ? &tm.kv : &tm.qv, &c.bars[0], HD, (int)row_src);
+    uint8_t* sm = c.smem;   // slots: 0 Dy, 1 dC, 2 the other factor of the level above, (3, 4) and (5, 6): g and Xv[l1] of a chunk
+    constexpr uint32_t colCarry = 0, colAcc = 128;
+    auto chunk_loads = [&](int chx, int buf) {   // (valid(chx) has left the chunk's source slot in `src`)
+        uint8_t* base = sm + (3 + 2 * buf) * kTileB;
+        const CUtensorMap* gm = is_key ? &tm.dkv : &tm.dqv;
+        const CUtensorMap* xm = is_key ? &tm.kv : &tm.qv;
+        tma_tile(base, gm, &c.bars[0], HD, (int)(((long)l2 * p.S + s) * p.Lp + (long)chx * kT));
+        tma_tile(base + kTileB, xm, &c.bars[0], HD, (int)(((long)src * p.S + s) * p.Lp + (long)chx * kT));
     };
-    // the top level's gradient needs nothing added: it goes into the g slot as a tile, next to the first operands
-    if (c.tid == 0) {
-        issue_loads(0, kT * HD * 2);
-        tma_tile(sm, is_key ? &tm.dkv : &tm.dqv, &c.bars[0], HD, (int)(((long)l2 * p.S + s) * p.Lp + (long)ch * kT));
+    if (c.tid == 0) {   // first group: the run product itself, the operands of the level above, the first chunk
+        const uint32_t tile = kT * HD * 2;
+        mbar_expect_tx(&c.bars[0], (ch >= 0 ? 3 : 0) * tile + (parent ? 2 : 0) * tile);
+        if (ch >= 0) {
+            tma_tile(sm, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
+            valid(ch);
+            chunk_loads(ch, 0);
+        }
+        if (parent) {
+            const long up = p.lv.dy_off[l1 + 1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1 + 1] + (b >> 1);
+            tma_tile(sm + kTileB, &tm.ddy, &c.bars[0], HD, (int)(up * HD));
+            tma_tile(sm + 2 * kTileB, &tm.dyh, &c.bars[0], HD, (int)((mat + (is_key ? -1 : 1)) * HD));
+        }
     }
-    int buf = 0;
-    bool have_acc = false;
-    // The gradient stored in global memory at the level a step consumes is requested one step ahead (the first one
-    // here), so that its latency hides behind the previous step's products and atomics.
     constexpr int NI = HD / 64;
-    uint32_t pend[NI][2][8];   // 32 bf16 = 64 bytes per piece
+    uint32_t pend[NI][2][8];   // the gradient stored at level l1 for the current chunk (32 bf16 = 64 bytes per piece)
     auto request = [&](long row0) {
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
-            const __nv_bfloat16* src = dxv + ((size_t)row0 + c.row) * HD + c.half * (HD / 2) + i * 32;
-            ld_global_v8(src, pend[i][0]);
-            ld_global_v8(src + 16, pend[i][1]);
+            const __nv_bfloat16* g = dxv + ((size_t)row0 + c.row) * HD + c.half * (HD / 2) + i * 32;
+            ld_global_v8(g, pend[i][0]);
+            ld_global_v8(g + 16, pend[i][1]);
         }
     };
-    auto arrived = [&](int i, float (&v)[32]) {
-#pragma unroll
-        for (int x = 0; x < 16; ++x) {
-            const uint32_t w = pend[i][x >> 3][x & 7];
-            v[2 * x] = __uint_as_float(w << 16);
-            v[2 * x + 1] = __uint_as_float(w & 0xffff0000u);
-        }
+    auto issue_parent = [&](uint32_t a) {
+        if (is_key) mma(c.tmem + colAcc, a + kTileB, OP_K, a + 2 * kTileB, OP_K, HD / 16, HD, false);      // dC B^T
+        else        mma(c.tmem + colAcc, a + 2 * kTileB, OP_MN, a + kTileB, OP_MN, HD / 16, HD, false);   // A^T dC
     };
-
+    int buf = 0;
+    bool first = true;
 #pragma unroll 1
-    while (l2 >= 1 && c.ok) {
-        version_step(is_key, ch, l2, p.N, l1, b, src);
-        const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
-        const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
-        // g = gradient stored at this level + the contribution from above -> bf16 tile (the first step's g is loaded as a tile)
-        {
-            if (have_acc) {
-                float v[32], a[32];
-#pragma unroll
-                for (int i = 0; i < NI; ++i) {
-                    const int c0 = c.half * (HD / 2) + i * 32;
-                    arrived(i, v);
-                    tmem_row32(c.tl + c0, a);
-#pragma unroll
-                    for (int x = 0; x < 32; ++x) v[x] += a[x];
-                    tile_store32(sm, c.row, c0, v);
-                }
-            }
-            // what is stored at the level this step contributes to: the next step's input, or the chain's final sum
-            request(row_src);
-        }
-        // the step after this one (its description replaces l1, b, src only after this step's were copied above)
-        const int l2n = next_step(l2 - 1);
+    while (ch >= 0 && c.ok) {
+        valid(ch);   // refreshes `src` for this chunk
+        const long row_lo = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
+        request(row_lo);
+        const int nxt = next_chunk(ch + 1);
         loads_wait(c);
-        tma_store_wait_read();   // the previous step's reductions have read their staging area: the prefetch below refills it
-        publish();
+        // every thread has read the previous chunk's carry out of tensor memory before the next product overwrites it
+        tc_fence_before_sync();
+        __syncthreads();
         if (c.tid == 0 && c.ok) {
-            if (l2n >= 1) issue_loads(buf ^ 1);
+            if (nxt >= 0) {   // the other buffer's products retired before the previous mma_wait returned
+                mbar_expect_tx(&c.bars[0], 2 * kT * HD * 2);
+                valid(nxt);
+                chunk_loads(nxt, buf ^ 1);
+            }
             tc_fence_after_sync();
-            const uint32_t g = smem_u32(sm), o = smem_u32(sm + (1 + 3 * buf) * kTileB);
-            const int bop = is_key ? OP_MN : OP_K;
-            mma(c.tmem, g, OP_K, o, bop, HD / 16, HD, false);
-            if (!is_key) mma(c.tmem + 128, o + 2 * kTileB, OP_MN, g, OP_MN, 8, HD, false);
-            else         mma(c.tmem + 128, g, OP_MN, o + 2 * kTileB, OP_MN, 8, HD, false);
+            const uint32_t a = smem_u32(sm), g = a + (3 + 2 * buf) * kTileB, x = g + kTileB;
+            if (first && parent) issue_parent(a);
+            const bool acc = !first || parent;
+            if (!is_key) {
+                mma(c.tmem + colCarry, g, OP_K, a, OP_K, HD / 16, HD, false);     // g Dy^T
+                mma(c.tmem + colAcc, x, OP_MN, g, OP_MN, 8, HD, acc);             // Xv^T g
+            } else {
+                mma(c.tmem + colCarry, g, OP_K, a, OP_MN, HD / 16, HD, false);    // g Dy
+                mma(c.tmem + colAcc, g, OP_MN, x, OP_MN, 8, HD, acc);             // g^T Xv
+            }
             umma_commit(&c.bars[1]);
         }
         mma_wait(c);
         if (c.ok) {
-            // run-product gradient: stage the [d][d] accumulator in this step's (now dead) operand slots
-            constexpr int LDS = HD + 4;
-            float* stage = (float*)(sm + (1 + 3 * buf) * kTileB);
-            float v[32];
-            for (int i = 0; i < HD / 64; ++i) {
-                const int c0 = c.half * (HD / 2) + i * 32;
-                tmem_row32(c.tl + 128 + c0, v);
-                if (c.row < HD) {
+            float v[32], a[32];
 #pragma unroll
-                    for (int x = 0; x < 8; ++x)
-                        *reinterpret_cast<float4*>(stage + c.row * LDS + c0 + 4 * x) =
-                            make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
+            for (int i = 0; i < NI; ++i) {
+                const int col = c.half * (HD / 2) + i * 32;
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    const uint32_t w = pend[i][x >> 3][x & 7];
+                    v[2 * x] = __uint_as_float(w << 16);
+                    v[2 * x + 1] = __uint_as_float(w & 0xffff0000u);
                 }
-            }
-            fence_proxy_async_smem();
-            __syncthreads();
-            // one bulk reduction per row: the adds happen at the memory side while this CTA goes on with its next step
-            if (c.tid < HD) {
-                bulk_reduce_add_f32(p.ddy + (size_t)mat * HD * HD + (size_t)c.tid * HD, stage + c.tid * LDS, HD * 4);
-                tma_store_commit();
+                tmem_row32(c.tl + colCarry + col, a);
+#pragma unroll
+                for (int x = 0; x < 32; ++x) v[x] += a[x];
+                gstore_bf16x32(dxv + ((size_t)row_lo + c.row) * HD + col, v);
             }
         }
-        have_acc = true;
-        l2 = l2n;
+        first = false;
+        ch = nxt;
         buf ^= 1;
     }
-    if (c.ok && have_acc) {   // bottom of the chain: stored value + carried contribution
-        float v[32], a[32];
-#pragma unroll
-        for (int i = 0; i < NI; ++i) {
-            const int c0 = c.half * (HD / 2) + i * 32;
-            arrived(i, v);
-            tmem_row32(c.tl + c0, a);
-#pragma unroll
-            for (int x = 0; x < 32; ++x) v[x] += a[x];
-            // the chain's bottom is always slot 0: its rows now hold the final sum, which the chunk chain rule loads
-            gstore_bf16x32(dxv + ((size_t)s * p.Lp + (size_t)ch * kT + c.row) * HD + c0, v);
+    if (first && c.ok) {   // no version step: the level above is the only contribution
+        loads_wait(c);
+        if (c.tid == 0 && c.ok) {
+            tc_fence_after_sync();
+            issue_parent(smem_u32(sm));
+            umma_commit(&c.bars[1]);
         }
+        mma_wait(c);
     }
-    tma_store_wait_all();
-    teardown<256>(c, p.status);
-}
-
-// ---------------------------------------------------------------------------------------------- dyadic backward
-// grid.x = S * cnt(l).  With dC = dDy[l][b], A = Dy[l-1][2b+1], B = Dy[l-1][2b]:  dA += dC B^T,  dB += A^T dC
-// (A, B: the hi planes of the run products).
-template <int HD>
-__global__ void __launch_bounds__(256, 1) dyadic_bwd_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    Ctx c;
-    setup<256>(c, smem_raw, kBar5);
-    const int cnt = p.lv.dy_cnt[p.l], cntl = p.lv.dy_cnt[p.l - 1];
-    const int s = blockIdx.x / cnt, b = blockIdx.x % cnt;
-    const long mat_up = p.lv.dy_off[p.l] / (HD * HD) + (long)s * cnt + b;
-    const long mat_lo = p.lv.dy_off[p.l - 1] / (HD * HD) + (long)s * cntl + 2 * b;   // B; A is +1
-    uint8_t* sm = c.smem;   // slots: 0 dC, 1 A, 3 B (2 and 4 are only part of the staging area below)
-    if (c.tid == 0) {
-        mbar_expect_tx(&c.bars[0], 2 * kT * HD * 2);
-        tma_tile(sm + 1 * kTileB, &tm.dyh, &c.bars[0], HD, (int)((mat_lo + 1) * HD));
-        tma_tile(sm + 3 * kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat_lo * HD));
-    }
-    conv(c, p.ddy + (size_t)mat_up * HD * HD, HD, HD, sm);
-    constexpr int NI = HD / 64;
-    loads_wait(c);
-    publish();
-    if (c.tid == 0 && c.ok) {
-        tc_fence_after_sync();
-        const uint32_t a = smem_u32(sm);
-        mma(c.tmem, a, OP_K, a + 3 * kTileB, OP_K, HD / 16, HD, false);            // dC B^T
-        mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a, OP_MN, HD / 16, HD, false);    // A^T dC
-        umma_commit(&c.bars[1]);
-    }
-    mma_wait(c);
     if (c.ok) {
-        // both [d][d] accumulators are staged in the (now dead) operand slots and added to the gradients of the two
-        // factors by bulk reductions, one per row: the adds happen at the memory side
-        constexpr int LDS = HD + 4;
-        float* stage = (float*)sm;
         float v[32];
-#pragma unroll
         for (int i = 0; i < NI; ++i) {
-            const int c0 = c.half * (HD / 2) + i * 32;
-#pragma unroll
-            for (int m = 0; m < 2; ++m) {
-                tmem_row32(c.tl + m * 128 + c0, v);
-                if (c.row < HD) {
-#pragma unroll
-                    for (int x = 0; x < 8; ++x)
-                        *reinterpret_cast<float4*>(stage + (m * HD + c.row) * LDS + c0 + 4 * x) =
-                            make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
-                }
-            }
-        }
-        fence_proxy_async_smem();
-        __syncthreads();
-        if (c.tid < 2 * HD) {   // rows 0 .. d-1: dA (factor 2b+1), rows d .. 2d-1: dB (factor 2b)
-            const int m = c.tid / HD, r = c.tid % HD;
-            bulk_reduce_add_f32(p.ddy + (size_t)(mat_lo + 1 - m) * HD * HD + (size_t)r * HD, stage + c.tid * LDS, HD * 4);
-            tma_store_commit();
-            tma_store_wait_read();
+            const int col = c.half * (HD / 2) + i * 32;
+            tmem_row32(c.tl + colAcc + col, v);
+            gstore_bf16x32(out + (size_t)c.row * HD + col, v, c.row < HD);
         }
     }
     teardown<256>(c, p.status);
@@ -548,18 +468,16 @@ cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const Leve
             dim3 g(p.S * p.N, 2);
             return hd == 64 ? launch(version_fwd_kernel<64>, g, 3, tm, p, st) : launch(version_fwd_kernel<128>, g, 3, tm, p, st);
         }
-        case LEVEL_VERSION_BWD: {
-            dim3 g(p.S * p.N, 2);
-            return hd == 64 ? launch(version_bwd_kernel<64>, g, 7, tm, p, st) : launch(version_bwd_kernel<128>, g, 7, tm, p, st);
+        case LEVEL_BWD: {
+            dim3 g(p.S * p.lv.dy_cnt[p.l]);
+            return hd == 64 ? launch(level_bwd_kernel<64>, g, 7, tm, p, st) : launch(level_bwd_kernel<128>, g, 7, tm, p, st);
         }
         case LEVEL_KEY_CACHE: {
             dim3 g(p.S, hd / 64);
             return hd == 64 ? launch(key_cache_kernel<64>, g, 5, tm, p, st) : launch(key_cache_kernel<128>, g, 5, tm, p, st);
         }
-        default: {
-            dim3 g(p.S * p.lv.dy_cnt[p.l]);
-            return hd == 64 ? launch(dyadic_bwd_kernel<64>, g, 5, tm, p, st) : launch(dyadic_bwd_kernel<128>, g, 5, tm, p, st);
-        }
+        default:
+            return cudaErrorInvalidValue;
     }
 }
 

@@ -166,14 +166,14 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
     p.Yt = bump(cur, SL * CHUNK * 2);
     p.Qv16 = bump(cur, SLd * 2 * p.nslot);
     p.Kv16 = bump(cur, SLd * 2 * p.nslot);
-    p.dy_bytes = dy_elems * 4;
+    p.dy_bytes = dy_elems * 2;
     if (bwd) {
         if (p.ragged) p.dop = bump(cur, SLd * 2);
         p.delta = bump(cur, SL * 4); p.lse2 = bump(cur, SL * 4);
         p.dQv = bump(cur, SLd * 2 * p.nslot); p.dKv = bump(cur, SLd * 2 * p.nslot);   // bf16
         p.dSd = bump(cur, gate ? SNBB * 4 : 0); p.dSdT = bump(cur, SNBB * 2); p.dG = bump(cur, SL * 4);
         p.dGrow = bump(cur, gate ? SL * 4 : 0); p.dGdiag = bump(cur, gate ? SL * 4 : 0);
-        p.dDy = bump(cur, dy_elems * 4);
+        p.dDy = bump(cur, dy_elems * 2);   // bf16, each matrix written once by the CTA that owns it
     }
     p.total = cur;
     return true;
@@ -188,16 +188,17 @@ static bool make_level_maps(const Plan& p, void* ws, LevelTensorMaps& tm) {
     return make_map(&tm.dyh, at<void>(ws, p.Dyh), (uint64_t)p.dy_mats * p.d, p.d) &&
            make_map(&tm.dyl, at<void>(ws, p.Dyl), (uint64_t)p.dy_mats * p.d, p.d) &&
            make_map(&tm.qv, at<void>(ws, p.Qv16), rows, p.d) && make_map(&tm.kv, at<void>(ws, p.Kv16), rows, p.d) &&
-           (!p.bwd || (make_map(&tm.dqv, at<void>(ws, p.dQv), rows, p.d) && make_map(&tm.dkv, at<void>(ws, p.dKv), rows, p.d)));
+           (!p.bwd || (make_map(&tm.dqv, at<void>(ws, p.dQv), rows, p.d) && make_map(&tm.dkv, at<void>(ws, p.dKv), rows, p.d) &&
+                       make_map(&tm.ddy, at<void>(ws, p.dDy), (uint64_t)p.dy_mats * p.d, p.d)));
 }
 
 static LevelParams level_params(const Plan& p, void* ws) {
     LevelParams lp{};
-    lp.lv = p.lv; lp.S = p.S; lp.N = p.N; lp.Lp = p.Lp;
+    lp.lv = p.lv; lp.S = p.S; lp.N = p.N; lp.Lp = p.Lp; lp.nlev = p.nlev;
     lp.dyh = at<__nv_bfloat16>(ws, p.Dyh); lp.dyl = at<__nv_bfloat16>(ws, p.Dyl);
     lp.qv = at<__nv_bfloat16>(ws, p.Qv16); lp.kv = at<__nv_bfloat16>(ws, p.Kv16);
     if (p.bwd) {
-        lp.dqv = at<__nv_bfloat16>(ws, p.dQv); lp.dkv = at<__nv_bfloat16>(ws, p.dKv); lp.ddy = at<float>(ws, p.dDy);
+        lp.dqv = at<__nv_bfloat16>(ws, p.dQv); lp.dkv = at<__nv_bfloat16>(ws, p.dKv); lp.ddy16 = at<__nv_bfloat16>(ws, p.dDy);
     }
     if (p.gate) { lp.nkeep = at<int>(ws, p.nkeep); lp.nvisit = at<int>(ws, p.nvisit); }   // block skipping (see run_gate_skip)
     lp.status = at<uint32_t>(ws, p.status);
@@ -309,11 +310,11 @@ static int run_chunk_chain(const Plan& p, void* ws, const void* q, const void* k
               make_map(&tm.th, at<void>(ws, p.sTh), rows, CHUNK) && make_map(&tm.tl, at<void>(ws, p.sTl), rows, CHUNK) &&
               make_map(&tm.ah, at<void>(ws, p.sAh), rows, CHUNK) && make_map(&tm.al, at<void>(ws, p.sAl), rows, CHUNK) &&
               make_map(&tm.dsdt, at<void>(ws, p.dSdT), (uint64_t)p.S * p.N * CHUNK, CHUNK) &&
-              make_map(&tm.dql, at<void>(ws, p.dQv), rows, d) && make_map(&tm.dkr, at<void>(ws, p.dKv), rows, d);
+              make_map(&tm.dql, at<void>(ws, p.dQv), rows, d) && make_map(&tm.dkr, at<void>(ws, p.dKv), rows, d) &&
+              make_map(&tm.dp, at<void>(ws, p.dDy), (uint64_t)p.S * p.N * d, d);   // level 0 of the run-product gradients
     if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
     ChainParams cp{};
     cp.dql = at<__nv_bfloat16>(ws, p.dQv); cp.dkr = at<__nv_bfloat16>(ws, p.dKv);   // slot 0 of the version gradients: the final sums
-    cp.dp = at<float>(ws, p.dDy);                                   // level 0 of the run-product gradients
     cp.beta = at<float>(ws, p.betap);
     cp.dq = (__nv_bfloat16*)dq; cp.dk = (__nv_bfloat16*)dk; cp.dw = (__nv_bfloat16*)dw; cp.dbeta = dbeta;
     cp.status = at<uint32_t>(ws, p.status);
@@ -326,7 +327,6 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
                         const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* dw,
                         float* dbeta, float* dlog_f, float scale, cudaStream_t st) {
     const int d = p.d;
-    float* dDy = at<float>(ws, p.dDy);
     __nv_bfloat16* dQv = at<__nv_bfloat16>(ws, p.dQv); __nv_bfloat16* dKv = at<__nv_bfloat16>(ws, p.dKv);
 
     prof_mark(STG_ROWSTATS, 0, st);
@@ -352,7 +352,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     bp.lse2 = at<float>(ws, p.lse2); bp.delta = at<float>(ws, p.delta);
     bp.G = p.gate ? at<float>(ws, p.G) : nullptr;
     bp.status = at<uint32_t>(ws, p.status);
-    bp.zero_ptr = dDy; bp.zero_bytes = p.dy_bytes;   // cleared by the dK/dV sweep, first accumulated into by the version chains
+    bp.zero_ptr = nullptr; bp.zero_bytes = 0;
     bp.S = p.S; bp.L = p.L; bp.Lp = p.Lp; bp.N = p.N; bp.scale = scale;
     if (p.gate) { bp.nkeep = at<int>(ws, p.nkeep); bp.nvisit = at<int>(ws, p.nvisit); }   // block skipping: see run_gate_skip
     prof_mark(STG_ROWSTATS, 1, st);
@@ -364,17 +364,16 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     prof_mark(STG_FA_DQ, 1, st);
     prof_mark(STG_LEVELS_BWD, 0, st);
 
-    // version chains, top level first (they leave the final sums in slot 0 of the bf16 version gradients, which the chunk
-    // chain rule loads), then the run products top-down
+    // version chains and run products, top level first: one launch per level finishes the gradients of that level's run
+    // products and adds the chains' carries to the version gradients one level down (slot 0 ends up holding the final
+    // sums the chunk chain rule loads; level 0 of the run-product gradients is its dP)
     {
         LevelTensorMaps ltm;
         if (!make_level_maps(p, ws, ltm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
         LevelParams lp = level_params(p, ws);
-        lp.l = p.nlev;
-        LAUNCH(launch_level_kernel(LEVEL_VERSION_BWD, ltm, lp, d, st));
-        for (int l = p.nlev - 2; l >= 1; --l) {
+        for (int l = p.nlev - 2 > 0 ? p.nlev - 2 : 0; l >= 0; --l) {
             lp.l = l;
-            LAUNCH(launch_level_kernel(LEVEL_DYADIC_BWD, ltm, lp, d, st));
+            LAUNCH(launch_level_kernel(LEVEL_BWD, ltm, lp, d, st));
         }
     }
     prof_mark(STG_LEVELS_BWD, 1, st);
