@@ -190,6 +190,44 @@ int path_attn_decode_step(const void* q_t, const void* k_t, const void* v_t, con
                           size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Context-parallel PaTH (paper Sec. 3.5, "Compatibility with context-parallelism"): the sequence is cut into
+ * contiguous segments, one per device; every device first handles its own segment, then the (transformed keys, values,
+ * segment product) of each EARLIER segment pass by, nearest first, and are attended by the resident queries.  These calls
+ * are the per-device arithmetic of that scheme; they run on one GPU and know nothing about how a message travels
+ * (paper_2505_16381_b200/ring.py holds a ring schedule over torch.distributed send / recv, which copies every incoming
+ * message into this GPU's own memory before a kernel reads it).
+ *
+ *   path_attn_cp_prepare   this device's segment q, k, v, w [B,H,L,d] bf16, beta, log_f (or NULL) [B,H,L] float32
+ *        -> `state`   (path_attn_cp_state_bytes): the queries pulled back to the segment's start, x_i = (H_s ... H_i q_i)
+ *                     with s the segment's first position, as bf16 tiles; their gate terms; and the running result
+ *                     (float32 O, normalised, with its LSE) initialised with the segment's own causal attention;
+ *        -> `message` (path_attn_cp_message_bytes): the keys advanced to the segment's end, H_e ... H_{j+1} k_j with e
+ *                     the segment's last position (Sec. 3.4's key transform), the values, the product of the segment's
+ *                     transitions P = H_s ... H_e as a bf16 hi + lo pair, and the gate sums from each key to the
+ *                     segment's end.  One contiguous buffer: what travels along the ring.
+ *   path_attn_cp_step      `state` (Lq positions) meets the `message` of an earlier segment (Lk positions): plain
+ *        softmax attention of x against the transformed keys (no mask: every key is earlier), merged into the
+ *        running (O, LSE); then the queries move on past that segment, x <- x P  (the paper's in-place query update),
+ *        and their gate terms grow by the segment's total.  Messages must arrive nearest segment first.
+ *   path_attn_cp_finish    o [B,H,L,d] bf16 and lse [B,H,L] float32 from the state.
+ * After prepare, step for every earlier segment and finish, (o, lse) equal path_attn_fwd's rows for this segment on
+ * the whole sequence, up to rounding (x is re-rounded to bf16 once per step; the running result is float32).
+ * Forward only.  state, message and workspace are device buffers, 256-byte aligned, caller-owned;
+ * path_attn_cp_workspace_bytes(B, H, L, d, has_gate) covers prepare and step for a state of L positions.  Segments
+ * may differ in length.  dt must be PATH_BF16.  Same conventions as above (asynchronous, no allocation, error codes;
+ * the status word is at the start of `workspace`).
+ */
+size_t path_attn_cp_state_bytes(int B, int H, int L, int d);
+size_t path_attn_cp_message_bytes(int B, int H, int L, int d);
+size_t path_attn_cp_workspace_bytes(int B, int H, int L, int d, int has_gate);
+int path_attn_cp_prepare(const void* q, const void* k, const void* v, const void* w, const float* beta,
+                         const float* log_f, void* state, void* message, int B, int H, int L, int d, float scale,
+                         path_dtype_t dt, void* workspace, size_t workspace_bytes, void* cuda_stream);
+int path_attn_cp_step(void* state, const void* message, int B, int H, int Lq, int Lk, int d, float scale,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+int path_attn_cp_finish(const void* state, void* o, float* lse, int B, int H, int L, int d, void* cuda_stream);
+
+/*
  * Layer front-end: how a PaTH layer obtains the operator's w, beta and log_f (paper Sec. 2.2, footnote to the
  * definition of H_t; gate of Sec. 2.4).  The linear maps in front (the low-rank layer giving z, and u^T x + b for the
  * two logits) are plain matrix products and stay with the caller's GEMM library; these two calls are the rest:

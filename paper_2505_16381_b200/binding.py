@@ -21,6 +21,8 @@ EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_
            "path_attn_device_status", "path_attn_selftest_timeout",
            "path_attn_prefill_cache", "path_attn_decode_workspace_bytes", "path_attn_decode_step",
            "path_attn_frontend_fwd", "path_attn_frontend_bwd", "path_attn_skipped_chunk_pairs",
+           "path_attn_cp_state_bytes", "path_attn_cp_message_bytes", "path_attn_cp_workspace_bytes",
+           "path_attn_cp_prepare", "path_attn_cp_step", "path_attn_cp_finish",
            "path_attn_strerror", "path_attn_last_cuda_error", "path_attn_last_launch_count",
            "path_attn_profile_enable", "path_attn_profile_read", "path_attn_profile_stage_name"]
 
@@ -65,6 +67,16 @@ def load():
         lib.path_attn_frontend_fwd.argtypes = [P] * 7 + [I, I, I, I, F, P]
         lib.path_attn_frontend_bwd.restype = I
         lib.path_attn_frontend_bwd.argtypes = [P] * 11 + [I, I, I, I, F, P]
+        for fn in (lib.path_attn_cp_state_bytes, lib.path_attn_cp_message_bytes):
+            fn.restype, fn.argtypes = Z, [I, I, I, I]
+        lib.path_attn_cp_workspace_bytes.restype = Z
+        lib.path_attn_cp_workspace_bytes.argtypes = [I, I, I, I, I]
+        lib.path_attn_cp_prepare.restype = I
+        lib.path_attn_cp_prepare.argtypes = [P] * 8 + [I, I, I, I, F, I, P, Z, P]
+        lib.path_attn_cp_step.restype = I
+        lib.path_attn_cp_step.argtypes = [P, P, I, I, I, I, I, F, P, Z, P]
+        lib.path_attn_cp_finish.restype = I
+        lib.path_attn_cp_finish.argtypes = [P, P, P, I, I, I, I, P]
         lib.path_attn_skipped_chunk_pairs.restype = I
         lib.path_attn_skipped_chunk_pairs.argtypes = [P, P, ctypes.POINTER(ctypes.c_ulonglong), ctypes.POINTER(ctypes.c_ulonglong)]
         lib.path_attn_device_status.restype = I
@@ -361,3 +373,66 @@ def path_attn_frontend_bwd(z, conv_w, beta_logit, dw, dbeta, gate_logit=None, dl
     if rc != PATH_OK:
         raise PathAttnError(rc, "path_attn_frontend_bwd")
     return dz, dcw, dbl, dgl
+
+
+# ----------------------------------------------------------------------------------------- context-parallel path
+
+def _u8(n, device):
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def cp_alloc(B, H, L, d, has_gate=False, device="cuda"):
+    """(state, message, workspace) buffers for a segment of L positions (paper Sec. 3.5)."""
+    lib = load()
+    sizes = (lib.path_attn_cp_state_bytes(B, H, L, d), lib.path_attn_cp_message_bytes(B, H, L, d),
+             lib.path_attn_cp_workspace_bytes(B, H, L, d, int(has_gate)))
+    if 0 in sizes:
+        raise PathAttnError(-2, "path_attn_cp_*_bytes")
+    return tuple(_u8(int(n), device) for n in sizes)
+
+
+def path_attn_cp_prepare(q, k, v, w, beta, log_f=None, scale=1.0, state=None, message=None, workspace=None):
+    """This device's segment: fills ``state`` (resident queries + running result) and ``message`` (what later segments'
+    holders need from this one).  Returns ``(state, message, workspace)``."""
+    _check(q, k, v, w, beta, log_f)
+    lib = load()
+    B, H, L, d = q.shape
+    if state is None or message is None or workspace is None:
+        s_, m_, w_ = cp_alloc(B, H, L, d, log_f is not None, q.device)
+        state = s_ if state is None else state
+        message = m_ if message is None else message
+        workspace = w_ if workspace is None else workspace
+    st = torch.cuda.current_stream(q.device).cuda_stream
+    with torch.cuda.device(q.device):
+        rc = lib.path_attn_cp_prepare(_ptr(q), _ptr(k), _ptr(v), _ptr(w), _ptr(beta), _ptr(log_f), _ptr(state), _ptr(message),
+                                      B, H, L, d, float(scale), _dt(q), _ptr(workspace), workspace.numel(), ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_cp_prepare")
+    return state, message, workspace
+
+
+def path_attn_cp_step(state, message, B, H, Lq, Lk, d, scale=1.0, workspace=None):
+    """The resident queries (``state``, Lq positions) attend an earlier segment's ``message`` (Lk positions) and move on."""
+    lib = load()
+    if workspace is None:
+        workspace = _u8(int(lib.path_attn_cp_workspace_bytes(B, H, Lq, d, 0)), state.device)
+    st = torch.cuda.current_stream(state.device).cuda_stream
+    with torch.cuda.device(state.device):
+        rc = lib.path_attn_cp_step(_ptr(state), _ptr(message), B, H, Lq, Lk, d, float(scale), _ptr(workspace),
+                                   workspace.numel(), ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_cp_step")
+    return workspace
+
+
+def path_attn_cp_finish(state, B, H, L, d):
+    """``(o [B,H,L,d] bf16, lse [B,H,L] float32)`` of the segment from its state."""
+    lib = load()
+    o = torch.empty(B, H, L, d, dtype=torch.bfloat16, device=state.device)
+    lse = torch.empty(B, H, L, dtype=torch.float32, device=state.device)
+    st = torch.cuda.current_stream(state.device).cuda_stream
+    with torch.cuda.device(state.device):
+        rc = lib.path_attn_cp_finish(_ptr(state), _ptr(o), _ptr(lse), B, H, L, d, ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_cp_finish")
+    return o, lse

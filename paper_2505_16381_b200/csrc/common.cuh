@@ -70,6 +70,10 @@ struct FwdParams {
     int S, L, Lp, N;
     float scale;
     int out_fp32;
+    // segment-against-segment sweep of the context-parallel path only (launch_fa_fwd_cross): the key segment's padded
+    // length and chunk count, and its gate terms [S, Lkp] (G then holds the query rows' terms; logit += G_i - Gk_j)
+    const float* Gk;
+    int Lkp, Nk;
 };
 
 // Placement of the dyadic run products: level l holds dy_cnt[l] = N >> l matrices per slice, starting
@@ -95,13 +99,17 @@ struct LevelParams {
     __nv_bfloat16 *dyh, *dyl, *qv, *kv;
     __nv_bfloat16 *dqv, *dkv;     // [slots][S][Lp][d] gradients of the versions; slot 0 ends up holding the final sums
     __nv_bfloat16* ddy16;         // gradients of the run products, same placement as the run products themselves
-    float* kc;                    // key-cache kernel: [S][cap][d] float32 out (rows < L of every slice)
+    float* kc;                    // edge kernels: [S][cap][d] float32 out (rows < L of every slice), or nullptr
     int cap, L;
+    __nv_bfloat16* edge16;        // edge kernels: [S][L][d] bf16 out, or nullptr
+    __nv_bfloat16* pseg;          // query-edge kernel: [S][2][d][d] product of the whole segment as bf16 hi, lo; or nullptr
+    float* gq;                    // apply-product kernel: [S][Lp] gate terms of the rows (+= gtot[slice]), or nullptr
+    const float* gtot;            // [S]
     const int *nkeep, *nvisit;    // version backward: chunk counts of a sweep shortened by block skipping ([S][N]), or nullptr
     uint32_t* status;
 };
 
-enum { LEVEL_DYADIC_FWD = 0, LEVEL_VERSION_FWD, LEVEL_BWD, LEVEL_KEY_CACHE };
+enum { LEVEL_DYADIC_FWD = 0, LEVEL_VERSION_FWD, LEVEL_BWD, LEVEL_KEY_CACHE, LEVEL_QUERY_EDGE, LEVEL_APPLY_PRODUCT };
 cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const LevelParams& p, int hd, cudaStream_t st);
 
 struct PrepTensorMaps {
@@ -177,6 +185,8 @@ cudaError_t launch_fa_bwd(const BwdTensorMaps& tm, const BwdParams& p, int hd, i
 cudaError_t launch_rowstats(const void* o, const void* d_o, const float* lse, const float* G, float* delta, float* lse2,
                             int S, int L, int Lp, int hd, cudaStream_t st);
 cudaError_t launch_fa_fwd(const FwdTensorMaps& tm, const FwdParams& p, int hd, cudaStream_t st);
+// Every query chunk of one segment against every key chunk of another (tm.qv / tm.kv / tm.v only; p.G, p.Gk required).
+cudaError_t launch_fa_fwd_cross(const FwdTensorMaps& tm, const FwdParams& p, int hd, cudaStream_t st);
 // One decoding step over an in-place float32 key cache (paper Sec. 3.4); `part` holds decode_partials_bytes(S, cap, hd).
 size_t decode_partials_bytes(int S, int cap, int hd);
 cudaError_t launch_decode_step(const void* q_t, const void* k_t, const void* v_t, const void* w_t, const float* beta_t,

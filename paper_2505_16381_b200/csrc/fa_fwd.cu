@@ -90,7 +90,12 @@ struct FwdSmem {
 enum { B_QFULL = 0, B_QEMPTY = 3, B_KFULL = 6, B_KEMPTY = 8, B_VFULL = 10, B_VEMPTY = 12,
        B_SFULL = 14, B_PFULL = 16, B_OFULL = 18, B_OFREE = 20, B_COUNT = 21 };
 
-template <int HD, bool GATE>
+// CROSS = true is the segment-against-segment variant used by the context-parallel path (paper Sec. 3.5): a work item is a
+// query chunk of one segment, it visits EVERY key chunk of another (earlier) segment, there is no diagonal chunk and no
+// causal mask, queries and keys come as one prepared tile each (tm.qv / tm.kv, no levels), the key-side gate terms are
+// their own array (whose padded tail holds a huge value, which masks the padded keys), and the result is written
+// normalised in float32 together with its LSE so that the caller can merge it into a running state.
+template <int HD, bool GATE, bool CROSS = false>
 __global__ void __launch_bounds__(384, 1)
 fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -136,7 +141,10 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
     };
     // key chunks a work item visits, counted from the diagonal: all I + 1 of them, or fewer when the gate has made the
     // far ones negligible (every warp role reads the same precomputed number)
-    auto steps_of = [&](int I, int s) { return p.nkeep ? min(I + 1, p.nkeep[s * p.N + I]) : I + 1; };
+    auto steps_of = [&](int I, int s) {
+        if (CROSS) return p.Nk;
+        return p.nkeep ? min(I + 1, p.nkeep[s * p.N + I]) : I + 1;
+    };
     auto ver_row = [&](int s, int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
 
     if (warp < 4) {
@@ -171,6 +179,15 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
             for (int it = 0; ok && item_of(it, I, s); ++it) {
                 const int NS = steps_of(I, s);
                 const int rowRaw = s * p.Lp + I * kTile;
+                if (CROSS) {   // one query tile, then every key chunk of the other segment, last chunk first
+                    load_q(&tm.qv, HD, rowRaw);
+                    for (int n = 0; n < NS && ok; ++n) {
+                        const int x = n & 1, rowK = s * p.Lkp + (NS - 1 - n) * kTile;
+                        load_kv(sK, B_KFULL, B_KEMPTY, x, kf, &tm.kv, HD, rowK);
+                        load_kv(sV, B_VFULL, B_VEMPTY, x, vf, &tm.v, HD, rowK);
+                    }
+                    continue;
+                }
                 // diagonal chunk: raw q, k and the correction operands (both K slots), V of chunk I
                 load_q(&tm.q_raw, HD, rowRaw);
                 load_kv(sK, B_KFULL, B_KEMPTY, 0, kf, &tm.k_raw, HD, rowRaw);
@@ -224,13 +241,24 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
                 int cur_level = -1;
                 int q_of0, q_of1;              // operand index used by each stream's most recent S product
                 auto advance_q = [&](int n) {  // operand index of step n >= 1 (waits for a newly needed one)
-                    const int l = msb32((unsigned)(I ^ (I - n)));
+                    const int l = CROSS ? 0 : msb32((unsigned)(I ^ (I - n)));
                     if (l != cur_level) {
                         cur_level = l;
                         take_q();
                     }
                     return qi_next - 1;
                 };
+                if (CROSS) {   // S of step 0 (stream 0): an ordinary tile product; the one query operand serves every step
+                    cur_level = 0;
+                    const int q0 = take_q();
+                    take_k(0);
+                    tc_fence_after_sync();
+                    if (!ok) break;
+                    issue_s(0, q0 % 3, 0, HD, false);
+                    umma_commit(&bars[B_SFULL + 0]);
+                    umma_commit(&bars[B_KEMPTY + 0]);
+                    q_of0 = q_of1 = q0;
+                } else {
                 // S of step 0 (diagonal, stream 0): two contractions
                 const int q0 = take_q();
                 take_k(0);
@@ -246,6 +274,7 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
                 umma_commit(&bars[B_VEMPTY + 1]);
                 release_q(q1 + 1);             // rawQ and Xqn go back once the diagonal products retire
                 q_of0 = q_of1 = q1 + 1;
+                }
                 // S of step 1 (stream 1)
                 if (NS > 1) {
                     q_of1 = advance_q(1);
@@ -329,10 +358,11 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
             auto softmax_step = [&](auto diag_tag, const int t) {
                 constexpr bool DIAG = decltype(diag_tag)::value;   // the diagonal chunk (step 0): causal mask
                 constexpr bool PRE = DIAG || GATE;                 // logits are scaled (and gated, masked) in place first
-                const int n = 2 * t + x, J = I - n;
+                const int n = 2 * t + x, J = CROSS ? NS - 1 - n : I - n;
                 if (GATE) {
                     wg_sync();   // everyone is done with the previous chunk's values
-                    statx[row].x = p.G[(size_t)s * p.Lp + J * kTile + row] * kLog2e;
+                    statx[row].x = CROSS ? p.Gk[(size_t)s * p.Lkp + J * kTile + row] * kLog2e
+                                         : p.G[(size_t)s * p.Lp + J * kTile + row] * kLog2e;
                     wg_sync();
                 }
                 if (ok && !mbar_wait(&bars[B_SFULL + x], sc & 1, abort_flag, ST_FWD_SOFTMAX)) ok = false;
@@ -422,7 +452,7 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
             };
             {
                 int t = 0;
-                if (x == 0 && TX > 0) {
+                if (!CROSS && x == 0 && TX > 0) {
                     softmax_step(std::true_type{}, 0);
                     t = 1;
                 }
@@ -535,6 +565,25 @@ static cudaError_t launch_hd(const FwdTensorMaps& tm, const FwdParams& p, cudaSt
 
 cudaError_t launch_fa_fwd(const FwdTensorMaps& tm, const FwdParams& p, int hd, cudaStream_t st) {
     return hd == 64 ? launch_hd<64>(tm, p, st) : launch_hd<128>(tm, p, st);
+}
+
+template <int HD>
+static cudaError_t launch_cross_hd(const FwdTensorMaps& tm, const FwdParams& p, cudaStream_t st) {
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    if (!p.G || !p.Gk || p.Nk < 1) return cudaErrorInvalidValue;
+    const int pairs = (p.N * p.S + 1) / 2;
+    e = cudaFuncSetAttribute(fa_fwd_kernel<HD, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem::alloc);
+    if (e != cudaSuccess) return e;
+    fa_fwd_kernel<HD, true, true><<<dim3(pairs < sms ? pairs : sms), 384, FwdSmem::alloc, st>>>(tm, p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fa_fwd_cross(const FwdTensorMaps& tm, const FwdParams& p, int hd, cudaStream_t st) {
+    return hd == 64 ? launch_cross_hd<64>(tm, p, st) : launch_cross_hd<128>(tm, p, st);
 }
 
 }  // namespace path

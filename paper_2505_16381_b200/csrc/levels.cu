@@ -378,21 +378,25 @@ __global__ void __launch_bounds__(256, 1) level_bwd_kernel(const __grid_constant
     teardown<256>(c, p.status);
 }
 
-// ---------------------------------------------------------------------------------------------- key cache after a prefill
+// ---------------------------------------------------------------------------------------------- tiles moved to a segment's edge
 // grid = (S, d / 64).  Paper Sec. 3.4: after L tokens the cached key of position j is H_{L-1} ... H_{j+1} k_j.  In chunk
 // form that is  kc_J = Kright_J R_J  with  R_J = P_{J+1}^T ... P_{N-1}^T,  so a CTA walks the chunks of its slice from the
-// last to the first carrying R (bf16 hi + lo in shared memory):  kc_J = Kright_J R  (float32 out),  R <- P_J^T R.
+// last to the first carrying R (bf16 hi + lo in shared memory):  kc_J = Kright_J R,  R <- P_J^T R.
 // Both products act on the columns of R independently, so a CTA carries only 64 columns of R (and writes those columns
-// of the cache): at d = 128 two CTAs share a slice (four with 32 columns each were no faster per step and, at 4096 tokens,
-// more CTAs than SMs).
-template <int HD>
+// of the result): at d = 128 two CTAs share a slice (four with 32 columns each were no faster per step and, at 4096
+// tokens, more CTAs than SMs).
+// QUERY = true is the mirror image for the context-parallel path (paper Sec. 3.5): the queries pulled back to the start of
+// the segment,  x_I = Qleft_I R_I  with  R_I = P_{I-1} ... P_0,  walking the chunks upwards with  R <- P_I R;  the last R is
+// the product of the whole segment, which the segment hands to the devices holding later queries.
+// Results leave as float32 rows (p.kc, the decoding cache) and / or bf16 rows (p.edge16).
+template <int HD, bool QUERY>
 __global__ void __launch_bounds__(256, 1) key_cache_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
     extern __shared__ uint8_t smem_raw[];
     Ctx c;
     setup<256>(c, smem_raw, kBar5);
     constexpr int NC = 64;                      // columns of R per CTA
     const int s = blockIdx.x, col0 = blockIdx.y * NC;
-    uint8_t* sm = c.smem;   // slots: 0 Kright_J, 1 P hi, 2 P lo, 3 R hi, 4 R lo ([d x 64] in the first panel)
+    uint8_t* sm = c.smem;   // slots: 0 Kright_J / Qleft_I, 1 P hi, 2 P lo, 3 R hi, 4 R lo ([d x 64] in the first panel)
     {   // R = I[:, col0 .. col0+63]; the tiles' unused parts read as zeros (P^T enters with M = 128: its second panel when d = 64)
         for (int i = c.tid; i < (int)(4 * kTileB / 16); i += 256) reinterpret_cast<uint4*>(sm + kTileB)[i] = make_uint4(0, 0, 0, 0);
         __syncthreads();
@@ -406,45 +410,93 @@ __global__ void __launch_bounds__(256, 1) key_cache_kernel(const __grid_constant
     auto issue = [&](int J) {
         const long mat = p.lv.dy_off[0] / (HD * HD) + (long)s * p.lv.dy_cnt[0] + J;
         mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2);
-        tma_tile(sm, &tm.kv, &c.bars[0], HD, (int)((long)s * p.Lp + (long)J * kT));   // version slot 0 = Kright
+        tma_tile(sm, QUERY ? &tm.qv : &tm.kv, &c.bars[0], HD, (int)((long)s * p.Lp + (long)J * kT));   // version slot 0
         tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
         tma_tile(sm + 2 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
     };
-    if (c.tid == 0) issue(p.N - 1);
+    const int first = QUERY ? 0 : p.N - 1, step = QUERY ? 1 : -1;
+    if (c.tid == 0) issue(first);
 #pragma unroll 1
-    for (int J = p.N - 1; J >= 0 && c.ok; --J) {
+    for (int n = 0, J = first; n < p.N && c.ok; ++n, J += step) {
+        const bool more = n + 1 < p.N;
+        const bool update = QUERY || more;         // the query side also wants the product of the whole segment
         loads_wait(c);
         publish();
         if (c.tid == 0 && c.ok) {
             tc_fence_after_sync();
             const uint32_t a = smem_u32(sm);
-            mma(c.tmem, a, OP_K, a + 3 * kTileB, OP_MN, HD / 16, NC, false);                       // Kright R
+            mma(c.tmem, a, OP_K, a + 3 * kTileB, OP_MN, HD / 16, NC, false);                       // X R
             mma(c.tmem, a, OP_K, a + 4 * kTileB, OP_MN, HD / 16, NC, true);
-            if (J > 0) {
-                mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a + 3 * kTileB, OP_MN, HD / 16, NC, false);   // P^T R
-                mma(c.tmem + 128, a + 2 * kTileB, OP_MN, a + 3 * kTileB, OP_MN, HD / 16, NC, true);
-                mma(c.tmem + 128, a + 1 * kTileB, OP_MN, a + 4 * kTileB, OP_MN, HD / 16, NC, true);
+            if (update) {
+                constexpr int pop = QUERY ? OP_K : OP_MN;                                          // P R  /  P^T R
+                mma(c.tmem + 128, a + 1 * kTileB, pop, a + 3 * kTileB, OP_MN, HD / 16, NC, false);
+                mma(c.tmem + 128, a + 2 * kTileB, pop, a + 3 * kTileB, OP_MN, HD / 16, NC, true);
+                mma(c.tmem + 128, a + 1 * kTileB, pop, a + 4 * kTileB, OP_MN, HD / 16, NC, true);
             }
             umma_commit(&c.bars[1]);
         }
         mma_wait(c);
         if (!c.ok) break;
-        if (c.tid == 0 && J > 0) issue(J - 1);   // every product has retired: the operand slots are free again
+        if (c.tid == 0 && more) issue(J + step);   // every product has retired: the operand slots are free again
         const int pos = J * kT + c.row, c0 = c.half * 32;
         float v[32];
         uint32_t hi[16], lo[16];
         tmem_row32(c.tl + c0, v);
-        gstore_f32x32(p.kc + ((size_t)s * p.cap + pos) * HD + col0 + c0, v, pos < p.L);
-        if (J > 0) {
+        if (p.kc) gstore_f32x32(p.kc + ((size_t)s * p.cap + pos) * HD + col0 + c0, v, pos < p.L);
+        if (p.edge16) gstore_bf16x32(p.edge16 + ((size_t)s * p.L + pos) * HD + col0 + c0, v, pos < p.L);
+        if (update) {
             tmem_row32(c.tl + 128 + c0, v);
+            split32(v, hi, lo);
             if (c.row < HD) {
-                split32(v, hi, lo);
                 tile_store_w16(sm + 3 * kTileB, c.row, c0, hi);
                 tile_store_w16(sm + 4 * kTileB, c.row, c0, lo);
+            }
+            if (QUERY && !more && p.pseg) {   // the segment's product, [S][2 (hi, lo)][d][d]
+                gstore_bf16_w16(p.pseg + (((size_t)s * 2 + 0) * HD + c.row) * HD + col0 + c0, hi, c.row < HD);
+                gstore_bf16_w16(p.pseg + (((size_t)s * 2 + 1) * HD + c.row) * HD + col0 + c0, lo, c.row < HD);
             }
         }
     }
     teardown<256>(c, p.status);
+}
+
+// ---------------------------------------------------------------------------------------------- segment product applied to a tile
+// grid = S * N.  x <- x M  for every 128-row tile of x ([S][Lp][d] bf16, in place), with one matrix M = hi + lo per slice
+// ([S][2][d][d] bf16): the update of the query state after a key segment has been attended (paper Sec. 3.5).  The
+// gate term of the rows moves on as well: gq[row] += gtot[slice].
+template <int HD>
+__global__ void __launch_bounds__(256, 2) apply_product_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    Ctx c;
+    setup<128>(c, smem_raw, kBar3);
+    const int s = blockIdx.x / p.N, ch = blockIdx.x % p.N;
+    uint8_t* sm = c.smem;   // slots: 0 x tile, 1 M hi, 2 M lo
+    const long row0 = (long)s * p.Lp + (long)ch * kT;
+    if (c.tid == 0) {
+        mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2);
+        tma_tile(sm, &tm.qv, &c.bars[0], HD, (int)row0);
+        tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)((long)(2 * s) * HD));
+        tma_tile(sm + 2 * kTileB, &tm.dyh, &c.bars[0], HD, (int)((long)(2 * s + 1) * HD));
+    }
+    if (p.gq && c.tid < kT) p.gq[row0 + c.tid] += p.gtot[s];
+    loads_wait(c);
+    if (c.tid == 0 && c.ok) {
+        tc_fence_after_sync();
+        const uint32_t a = smem_u32(sm);
+        mma(c.tmem, a, OP_K, a + kTileB, OP_MN, HD / 16, HD, false);
+        mma(c.tmem, a, OP_K, a + 2 * kTileB, OP_MN, HD / 16, HD, true);
+        umma_commit(&c.bars[1]);
+    }
+    mma_wait(c);
+    if (c.ok) {
+        float v[32];
+        for (int i = 0; i < HD / 64; ++i) {
+            const int c0 = c.half * (HD / 2) + i * 32;
+            tmem_row32(c.tl + c0, v);
+            gstore_bf16x32(p.qv + ((size_t)row0 + c.row) * HD + c0, v);
+        }
+    }
+    teardown<128>(c, p.status);
 }
 
 template <class K>
@@ -474,7 +526,15 @@ cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const Leve
         }
         case LEVEL_KEY_CACHE: {
             dim3 g(p.S, hd / 64);
-            return hd == 64 ? launch(key_cache_kernel<64>, g, 5, tm, p, st) : launch(key_cache_kernel<128>, g, 5, tm, p, st);
+            return hd == 64 ? launch(key_cache_kernel<64, false>, g, 5, tm, p, st) : launch(key_cache_kernel<128, false>, g, 5, tm, p, st);
+        }
+        case LEVEL_QUERY_EDGE: {
+            dim3 g(p.S, hd / 64);
+            return hd == 64 ? launch(key_cache_kernel<64, true>, g, 5, tm, p, st) : launch(key_cache_kernel<128, true>, g, 5, tm, p, st);
+        }
+        case LEVEL_APPLY_PRODUCT: {
+            dim3 g(p.S * p.N);
+            return hd == 64 ? launch(apply_product_kernel<64>, g, 3, tm, p, st) : launch(apply_product_kernel<128>, g, 3, tm, p, st);
         }
         default:
             return cudaErrorInvalidValue;

@@ -243,6 +243,42 @@ __global__ void __launch_bounds__(128) tile_stair_kernel(int* __restrict__ nkeep
     }
 }
 
+// ---- context-parallel path: gate terms of a segment, merge of partial softmax results
+__global__ void cp_gate_kernel(const float* __restrict__ G, float* __restrict__ gq, float* __restrict__ gk,
+                               float* __restrict__ gtot, int L, int Lp) {
+    const int s = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
+    const float tot = G ? G[(size_t)s * Lp + L - 1] : 0.f;
+    if (i == 0) gtot[s] = tot;
+    if (i >= Lp) return;
+    const float g = G ? G[(size_t)s * Lp + i] : 0.f;
+    gq[(size_t)s * Lp + i] = i < L ? g : 0.f;
+    gk[(size_t)s * Lp + i] = i < L ? g - tot : 1e30f;
+}
+// one thread per 4 outputs of a row
+__global__ void cp_merge_kernel(float* __restrict__ o_acc, float* __restrict__ lse_acc, const float* __restrict__ o_t,
+                                const float* __restrict__ lse_t, size_t rows, int hd4) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows * hd4) return;
+    const size_t r = i / hd4;
+    const float la = lse_acc[r], lt = lse_t[r];
+    const float m = fmaxf(la, lt);
+    const float wa = __expf(la - m), wt = __expf(lt - m), inv = 1.f / (wa + wt);
+    const float4 a = reinterpret_cast<const float4*>(o_acc)[i], t = reinterpret_cast<const float4*>(o_t)[i];
+    reinterpret_cast<float4*>(o_acc)[i] = make_float4((a.x * wa + t.x * wt) * inv, (a.y * wa + t.y * wt) * inv,
+                                                      (a.z * wa + t.z * wt) * inv, (a.w * wa + t.w * wt) * inv);
+    __syncwarp();   // (the lanes of a row read lse_acc before one of them replaces it: a row's hd4 lanes sit in one warp)
+    if (i % hd4 == 0) lse_acc[r] = m + __logf(wa + wt);
+}
+__global__ void cp_finish_kernel(const float* __restrict__ o_acc, const float* __restrict__ lse_acc, __nv_bfloat16* __restrict__ o,
+                                 float* __restrict__ lse, size_t rows, int hd4) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows * hd4) return;
+    const float4 a = reinterpret_cast<const float4*>(o_acc)[i];
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+    reinterpret_cast<uint2*>(o)[i] = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+    if (i % hd4 == 0) lse[i / hd4] = lse_acc[i / hd4];
+}
+
 // ---- forward-state record and the wait self-test
 __global__ void state_write_kernel(StateRecord* dst, const StateRecord rec) {
     if (threadIdx.x == 0) *dst = rec;
@@ -317,6 +353,23 @@ cudaError_t launch_gate_skip(const void* q, const void* k, const void* w, const 
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     tile_stair_kernel<<<S, 128, 0, st>>>(nkeep, nvisit, counters, S, N);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_cp_gate(const float* G, float* gq, float* gk, float* gtot, int S, int L, int Lp, cudaStream_t st) {
+    cp_gate_kernel<<<dim3((Lp + 255) / 256, S), 256, 0, st>>>(G, gq, gk, gtot, L, Lp);
+    return cudaGetLastError();
+}
+cudaError_t launch_cp_merge(float* o_acc, float* lse_acc, const float* o_t, const float* lse_t, size_t rows, int hd,
+                            cudaStream_t st) {
+    const size_t n = rows * (hd / 4);
+    cp_merge_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(o_acc, lse_acc, o_t, lse_t, rows, hd / 4);
+    return cudaGetLastError();
+}
+cudaError_t launch_cp_finish(const float* o_acc, const float* lse_acc, void* o, float* lse, size_t rows, int hd,
+                             cudaStream_t st) {
+    const size_t n = rows * (hd / 4);
+    cp_finish_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(o_acc, lse_acc, (__nv_bfloat16*)o, lse, rows, hd / 4);
     return cudaGetLastError();
 }
 

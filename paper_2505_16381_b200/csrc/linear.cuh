@@ -26,6 +26,18 @@ cudaError_t launch_gate_skip(const void* q, const void* k, const void* w, const 
                              int* nkeep, int* nvisit, unsigned long long* counters, int S, int L, int Lp, int hd, float scale,
                              cudaStream_t st);
 
+// Context-parallel path (paper Sec. 3.5), gate terms of a segment from its prefix sums G [S][Lp] (nullptr = no gate):
+// gq[S][Lp] <- G (the query rows' terms), gk[S][Lp] <- G - G[L-1] for positions < L and a huge value for the padded tail
+// (which masks those keys), gtot[S] <- G[L-1].
+cudaError_t launch_cp_gate(const float* G, float* gq, float* gk, float* gtot, int S, int L, int Lp, cudaStream_t st);
+// Running softmax state (o_acc [S][L][d] float32 normalised, lse_acc [S][L]) merged with a partial result of the same
+// shape (o_t, lse_t): o_acc <- (e^{lse_acc} o_acc + e^{lse_t} o_t) / (e^{lse_acc} + e^{lse_t}), lse_acc <- log of that sum.
+cudaError_t launch_cp_merge(float* o_acc, float* lse_acc, const float* o_t, const float* lse_t, size_t rows, int hd,
+                            cudaStream_t st);
+// o [rows][d] bf16 <- o_acc, lse <- lse_acc.
+cudaError_t launch_cp_finish(const float* o_acc, const float* lse_acc, void* o, float* lse, size_t rows, int hd,
+                             cudaStream_t st);
+
 // Forward-state record in the status block of a workspace (see StateRecord): written at the end of a forward that kept its
 // chunk preparation, compared by the backward that wants to reuse it (a mismatch raises ST_STATE in the status word).
 cudaError_t launch_state_write(void* record, const StateRecord& rec, cudaStream_t st);

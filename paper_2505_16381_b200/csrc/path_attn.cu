@@ -600,6 +600,167 @@ int path_attn_fwd_static(const void* q, const void* k, const void* v, const void
     return rc;
 }
 
+// ------------------------------------------------------------------------------------------- context-parallel path
+// Layouts of the two caller-owned buffers of the segment-level calls (paper Sec. 3.5); every part starts 256-byte aligned.
+struct CpLayout {
+    int S, L, Lp, N, d;
+    size_t x, gq, o_acc, lse_acc, state_total;        // state: query tiles pulled back so far, their gate terms, running result
+    size_t kend, v, pseg, gk, gtot, message_total;    // message: what a segment hands to the holders of later queries
+    size_t o_t, lse_t, step_total;                    // scratch of one step (after the 256-byte status block)
+};
+static bool cp_layout(int B, int H, int L, int d, CpLayout& c) {
+    Plan p;
+    if (!make_plan(B, H, L, d, PATH_BF16, 0, 0, p)) return false;
+    c.S = p.S; c.L = L; c.Lp = p.Lp; c.N = p.N; c.d = d;
+    const size_t SLpd = (size_t)p.S * p.Lp * d, SLp = (size_t)p.S * p.Lp, SLd = (size_t)p.S * L * d, SL = (size_t)p.S * L;
+    size_t cur = 0;
+    c.x = bump(cur, SLpd * 2); c.gq = bump(cur, SLp * 4); c.o_acc = bump(cur, SLd * 4); c.lse_acc = bump(cur, SL * 4);
+    c.state_total = cur;
+    cur = 0;
+    c.kend = bump(cur, SLpd * 2); c.v = bump(cur, SLpd * 2); c.pseg = bump(cur, (size_t)p.S * 2 * d * d * 2);
+    c.gk = bump(cur, SLp * 4); c.gtot = bump(cur, (size_t)p.S * 4);
+    c.message_total = cur;
+    cur = 256;
+    c.o_t = bump(cur, SLd * 4); c.lse_t = bump(cur, SL * 4);
+    c.step_total = cur;
+    return true;
+}
+
+size_t path_attn_cp_state_bytes(int B, int H, int L, int d) {
+    CpLayout c;
+    return cp_layout(B, H, L, d, c) ? c.state_total : 0;
+}
+size_t path_attn_cp_message_bytes(int B, int H, int L, int d) {
+    CpLayout c;
+    return cp_layout(B, H, L, d, c) ? c.message_total : 0;
+}
+size_t path_attn_cp_workspace_bytes(int B, int H, int L, int d, int has_gate) {
+    CpLayout c;
+    Plan p;
+    if (!cp_layout(B, H, L, d, c) || !make_plan(B, H, L, d, PATH_BF16, has_gate ? 1 : 0, 0, p)) return 0;
+    return p.total > c.step_total ? p.total : c.step_total;
+}
+
+int path_attn_cp_prepare(const void* q, const void* k, const void* v, const void* w, const float* beta, const float* log_f,
+                         void* state, void* message, int B, int H, int L, int d, float scale, path_dtype_t dt,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    g_launches = 0;
+    if (!q || !k || !v || !w || !beta || !state || !message || !workspace) return PATH_ERR_NULL;
+    if (dt != PATH_BF16) return PATH_ERR_DTYPE;
+    Plan p;
+    CpLayout c;
+    if (!make_plan(B, H, L, d, (int)dt, log_f ? 1 : 0, 0, p) || !cp_layout(B, H, L, d, c)) return PATH_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(w) || !aligned16(beta) || (log_f && !aligned16(log_f)) ||
+        ((uintptr_t)workspace & 255) || ((uintptr_t)state & 255) || ((uintptr_t)message & 255))
+        return PATH_ERR_ALIGN;
+    if (workspace_bytes < path_attn_cp_workspace_bytes(B, H, L, d, log_f ? 1 : 0)) return PATH_ERR_WORKSPACE;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CK(cudaMemsetAsync(workspace, 0, 256, st));
+    rc = stage_inputs(p, workspace, q, k, v, w, beta, log_f, true, st);
+    if (rc != PATH_OK) return rc;
+    if (log_f) {
+        rc = run_gate_skip(p, workspace, q, k, w, scale, st);
+        if (rc != PATH_OK) return rc;
+    }
+    rc = run_prep(p, workspace, q, k, w, false, st);
+    if (rc != PATH_OK) return rc;
+    // the segment's own (causal) attention, as a float32 running result
+    {
+        FwdTensorMaps tm;
+        const uint64_t rows = (uint64_t)p.S * p.Lp;
+        bool ok = make_map(&tm.q_raw, q, rows, d) && make_map(&tm.k_raw, k, rows, d) && make_map(&tm.v, v, rows, d) &&
+                  make_map(&tm.qv, at<void>(workspace, p.Qv16), rows * p.nslot, d) &&
+                  make_map(&tm.kv, at<void>(workspace, p.Kv16), rows * p.nslot, d) &&
+                  make_map(&tm.xqn, at<void>(workspace, p.Xqn), rows, CHUNK) && make_map(&tm.yt, at<void>(workspace, p.Yt), rows, CHUNK);
+        if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+        FwdParams fp{};
+        fp.o = at<float>(state, c.o_acc); fp.lse = at<float>(state, c.lse_acc); fp.G = log_f ? at<float>(workspace, p.G) : nullptr;
+        fp.status = at<uint32_t>(workspace, p.status);
+        fp.S = p.S; fp.L = L; fp.Lp = p.Lp; fp.N = p.N; fp.scale = scale; fp.out_fp32 = 1;
+        if (log_f) fp.nkeep = at<int>(workspace, p.nkeep);
+        LAUNCH(launch_fa_fwd(tm, fp, d, st));
+    }
+    // keys advanced to the segment's end, queries pulled back to its start, the product of the whole segment
+    {
+        LevelTensorMaps tm;
+        if (!make_level_maps(p, workspace, tm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+        LevelParams lp = level_params(p, workspace);
+        lp.L = p.Lp; lp.cap = p.Lp;   // (whole padded chunks: the padded rows of the prepared tiles are zero)
+        lp.edge16 = at<__nv_bfloat16>(message, c.kend);
+        LAUNCH(launch_level_kernel(LEVEL_KEY_CACHE, tm, lp, d, st));
+        lp.edge16 = at<__nv_bfloat16>(state, c.x);
+        lp.pseg = at<__nv_bfloat16>(message, c.pseg);
+        LAUNCH(launch_level_kernel(LEVEL_QUERY_EDGE, tm, lp, d, st));
+    }
+    CK(cudaMemcpyAsync(at<void>(message, c.v), v, (size_t)p.S * p.Lp * d * 2, cudaMemcpyDeviceToDevice, st));
+    LAUNCH(launch_cp_gate(log_f ? at<float>(workspace, p.G) : nullptr, at<float>(state, c.gq), at<float>(message, c.gk),
+                          at<float>(message, c.gtot), p.S, L, p.Lp, st));
+    return PATH_OK;
+}
+
+int path_attn_cp_step(void* state, const void* message, int B, int H, int Lq, int Lk, int d, float scale, void* workspace,
+                      size_t workspace_bytes, void* cuda_stream) {
+    g_launches = 0;
+    if (!state || !message || !workspace) return PATH_ERR_NULL;
+    CpLayout cq, ck;
+    if (!cp_layout(B, H, Lq, d, cq) || !cp_layout(B, H, Lk, d, ck)) return PATH_ERR_SHAPE;
+    if (((uintptr_t)workspace & 255) || ((uintptr_t)state & 255) || ((uintptr_t)message & 255)) return PATH_ERR_ALIGN;
+    if (workspace_bytes < cq.step_total) return PATH_ERR_WORKSPACE;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CK(cudaMemsetAsync(workspace, 0, 256, st));
+    void* msg = const_cast<void*>(message);
+    // every query chunk of this segment against every key chunk of the incoming one
+    {
+        FwdTensorMaps tm;
+        bool ok = make_map(&tm.qv, at<void>(state, cq.x), (uint64_t)cq.S * cq.Lp, d) &&
+                  make_map(&tm.kv, at<void>(msg, ck.kend), (uint64_t)ck.S * ck.Lp, d) &&
+                  make_map(&tm.v, at<void>(msg, ck.v), (uint64_t)ck.S * ck.Lp, d);
+        if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+        tm.q_raw = tm.k_raw = tm.xqn = tm.yt = tm.qv;   // unused by this sweep, but every descriptor gets prefetched
+        FwdParams fp{};
+        fp.o = at<float>(workspace, cq.o_t); fp.lse = at<float>(workspace, cq.lse_t);
+        fp.G = at<float>(state, cq.gq); fp.Gk = at<float>(msg, ck.gk);
+        fp.status = (uint32_t*)workspace;
+        fp.S = cq.S; fp.L = Lq; fp.Lp = cq.Lp; fp.N = cq.N; fp.Nk = ck.N; fp.Lkp = ck.Lp; fp.scale = scale; fp.out_fp32 = 1;
+        LAUNCH(launch_fa_fwd_cross(tm, fp, d, st));
+    }
+    LAUNCH(launch_cp_merge(at<float>(state, cq.o_acc), at<float>(state, cq.lse_acc), at<float>(workspace, cq.o_t),
+                           at<float>(workspace, cq.lse_t), (size_t)cq.S * Lq, d, st));
+    // the queries move on past the attended segment: x <- x P(segment), gate terms += the segment's total
+    {
+        LevelTensorMaps tm;
+        memset(&tm, 0, sizeof(tm));
+        bool ok = make_map(&tm.qv, at<void>(state, cq.x), (uint64_t)cq.S * cq.Lp, d) &&
+                  make_map(&tm.dyh, at<void>(msg, ck.pseg), (uint64_t)ck.S * 2 * d, d);
+        if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+        tm.dyl = tm.kv = tm.dqv = tm.dkv = tm.ddy = tm.qv;
+        LevelParams lp{};
+        lp.S = cq.S; lp.N = cq.N; lp.Lp = cq.Lp;
+        lp.qv = at<__nv_bfloat16>(state, cq.x);
+        lp.gq = at<float>(state, cq.gq); lp.gtot = at<float>(msg, ck.gtot);
+        lp.status = (uint32_t*)workspace;
+        LAUNCH(launch_level_kernel(LEVEL_APPLY_PRODUCT, tm, lp, d, st));
+    }
+    return PATH_OK;
+}
+
+int path_attn_cp_finish(const void* state, void* o, float* lse, int B, int H, int L, int d, void* cuda_stream) {
+    g_launches = 0;
+    if (!state || !o || !lse) return PATH_ERR_NULL;
+    CpLayout c;
+    if (!cp_layout(B, H, L, d, c)) return PATH_ERR_SHAPE;
+    if (((uintptr_t)state & 255) || !aligned16(o) || !aligned16(lse)) return PATH_ERR_ALIGN;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    void* st_ = const_cast<void*>(state);
+    LAUNCH(launch_cp_finish(at<float>(st_, c.o_acc), at<float>(st_, c.lse_acc), o, lse, (size_t)c.S * L, d, (cudaStream_t)cuda_stream));
+    return PATH_OK;
+}
+
 int path_attn_prefill_cache(const void* k, const void* v, const void* w, const float* beta, const float* log_f, float* kc,
                             void* vc, float* gc, int B, int H, int L, int d, int cap, path_dtype_t dt, void* workspace,
                             size_t workspace_bytes, void* cuda_stream) {
