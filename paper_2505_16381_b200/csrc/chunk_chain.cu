@@ -21,13 +21,12 @@ using namespace tile;
 
 namespace {
 
-// The kernel below is ~30 products of straight-line code that runs once per CTA; with every product inlined it
-// no longer fits the instruction cache, so the products go through one real function.
-__device__ __noinline__ void mma_call(uint32_t d_tmem, uint32_t a_tile, int a_op, uint32_t b_tile, int b_op, int ksteps, int n,
-                                      bool acc, bool negate = false) {
-    tile::mma(d_tmem, a_tile, a_op, b_tile, b_op, ksteps, n, acc, negate);
-}
-
+#ifdef CHAIN_STAMPS
+__device__ long long g_chain_stamps[32];
+#define STAMP(i) do { if (blockIdx.x == 0 && tid == 32 && chunk == (int)blockIdx.x + 3 * (int)gridDim.x) stamps[i] = clock64(); } while (0)
+#else
+#define STAMP(i) do {} while (0)
+#endif
 constexpr int kSlots = 7;
 constexpr uint32_t kBarOff = kSlots * kTileB;
 constexpr uint32_t kChainSmem = kBarOff + 64 + kT * 4 + kT * 4 + 1024;
@@ -63,6 +62,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     constexpr int KD = HD / 16, K8 = 8;
     constexpr uint32_t cDW = 0, cA = 128, cB = 256, cG = 384;   // tensor-memory columns: dw, two work accumulators, W W^T
     bool ok = true;
+#ifdef CHAIN_STAMPS
+    long long* stamps = g_chain_stamps;
+#endif
     uint32_t ph_load = 0, ph_mma = 0;
     float v[32];
 
@@ -147,6 +149,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
 
 #pragma unroll 1
     for (int chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+    STAMP(30);
     const int s_idx = chunk / p.N, pos = (chunk % p.N) * kT + row;   // slice and position of this thread's row
     const bool row_valid = pos < p.L;
     const size_t urow = (size_t)s_idx * p.L + pos;                   // row in the caller's [S][L][.] tensors
@@ -156,7 +159,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     if (tid < kT) bt[tid] = p.beta[(size_t)chunk * kT + tid];   // first read after several barriers (phase 4)
     // ---- phase 0a: dXq = lower(-(dQl U^T + s dSd Y^T))
     loads_wait();
+    STAMP(0);
     publish();
+    STAMP(1);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(1), OP_K, sa(0), OP_K, KD, 128, false);
@@ -167,6 +172,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
+    STAMP(2);
     if (!ok) break;
     // ---- phase 1: dY = -(W dKr^T + Xq^T s dSd),  dU = -(Xq^T dQl + W dP),  Gm = W W^T
     // (every group's tiles are requested as soon as the products that read the slots have retired, before the
@@ -178,7 +184,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     acc_to_tile(cA, kT, slot(4), -1.f, M_LOWER);                    // dXq
     loads_wait();
+    STAMP(3);
     publish();
+    STAMP(4);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(0), OP_K, sa(5), OP_K, KD, 128, false);
@@ -189,6 +197,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
+    STAMP(5);
     if (!ok) break;
     // ---- phase 2: dT = lower(dY Xk^T + dU W^T)
     if (tid == 0) {
@@ -198,7 +207,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     acc_to_tile(cA, kT, slot(5), -1.f, M_NONE);                     // dY (over dKr)
     acc_to_tile(cB, HD, slot(6), -1.f, M_NONE);                     // dU (over dP)
     loads_wait();
+    STAMP(6);
     publish();
+    STAMP(7);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(5), OP_K, sa(2), OP_K, K8, 128, false);
@@ -206,6 +217,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
+    STAMP(8);
     if (!ok) break;
     // ---- phase 3: dXk = strictLower(T~^T dY) -> cB,  dw += T~^T dU.  (s dSd)^T is not needed again before phase 5, where
     // it is loaded once more: until then its slot (3) takes the lo parts of the bf16 pairs, so that the hi and lo products
@@ -218,7 +230,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     // dT stays in tensor memory (cA); its bf16 hi part goes to slot 1 now, the lo part follows in phase 4
     split_to_tile(cA, slot(1), false, f_dT);
     loads_wait();
+    STAMP(9);
     publish();
+    STAMP(10);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cB, sa(2), OP_MN, sa(5), OP_MN, K8, 128, false);
@@ -228,6 +242,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
+    STAMP(11);
     if (!ok) break;
     // ---- phase 4: M = Ainv^T dT -> cB;  dbeta_c = M_cc;  tmp = M D;  dA = strictLower(-tmp Ainv^T) -> cA
     if (tid == 0) {
@@ -238,7 +253,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     acc_to_tile(cB, kT, slot(5), 1.f, M_STRICT);                    // dXk (over dY)
     split_to_tile(cA, slot(3), true, f_dT);                         // dT lo (over T~ lo)
     loads_wait();
+    STAMP(12);
     publish();
+    STAMP(13);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, 128, false);
@@ -247,6 +264,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
+    STAMP(14);
     if (!ok) break;
     {   // diagonal of M -> t1
         const int c0 = (row >> 5) << 5;
@@ -259,6 +277,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     split_both(cB, slot(1), slot(3), f_tmp);                        // tmp = M D, hi (over dT hi) and lo (over dT lo)
     publish();
+    STAMP(15);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(1), OP_K, sa(2), OP_K, K8, 128, false);
@@ -267,6 +286,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
+    STAMP(16);
     if (!ok) break;
     if (tid == 0) {   // phase 5's K and Q replace Ainv hi / lo, whose last products have just retired; (s dSd)^T returns
         mbar_expect_tx(&bars[0], 2 * kT * HD * 2 + kTileB);
@@ -294,7 +314,9 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     split_to_tile(cA, slot(1), false, f_dGm);                       // dGm = D dA, hi
     // ---- phase 5: dq -> cB, dk -> cG and the rest of dw
     loads_wait();
+    STAMP(17);
     publish();
+    STAMP(18);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cB, sa(3), OP_MN, sa(2), OP_MN, K8, HD, false);   // s dSd K
@@ -308,9 +330,11 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
+    STAMP(19);
     if (!ok) break;
     split_to_tile(cA, slot(1), true, f_dGm);                        // dGm lo
     publish();
+    STAMP(20);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cDW, sa(1), OP_K, sa(0), OP_MN, K8, HD, true);
@@ -329,6 +353,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         }
     }
     mma_wait();
+    STAMP(21);
     if (!ok) break;
     // every product of this chunk has retired: all tile slots are free for the next chunk's first tiles
     if (tid == 0 && chunk + (int)gridDim.x < nchunks) first_loads(chunk + gridDim.x);
@@ -349,6 +374,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         tmem_row32(tl + cDW + c0, v);
         gstore_bf16x32(p.dw + urow * HD + c0, v, row_valid);
     }
+    STAMP(31);
     // the next chunk's first products overwrite the accumulators read above
     tc_fence_before_sync();
     __syncthreads();
@@ -365,6 +391,12 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
 }
 
 }  // namespace
+
+#ifdef CHAIN_STAMPS
+extern "C" int path_attn_debug_chain_stamps(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_chain_stamps, sizeof(long long) * 32);
+}
+#endif
 
 cudaError_t launch_chunk_chain(const ChainTensorMaps& tm, const ChainParams& p, int hd, int nchunks, cudaStream_t st) {
     int dev = 0, sms = 0;

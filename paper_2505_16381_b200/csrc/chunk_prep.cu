@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 ok = wait(B_LOAD, 0);
                 if (ok) {
                     tc_fence_after_sync();
-                    mma(tmem + 0, aW_, OP_K, aW_, OP_K, KS, 128, false);
+                    mma_small(tmem + 0, aW_, OP_K, aW_, OP_K, KS, 128, false);
                     umma_commit(&bars[B_GM]);
                 }
             }
@@ -143,14 +143,14 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 // Xq, Xk: their columns held the previous chunk's W^T U and Xq U
                 if (it > 0 && !wait(R_E3, par ^ 1)) break;
                 tc_fence_after_sync();
-                mma(tmem + 128, aQ, OP_K, aW, OP_K, KS, 128, false);
-                mma(tmem + 256, aW, OP_K, aK, OP_K, KS, 128, false);
+                mma_small(tmem + 128, aQ, OP_K, aW, OP_K, KS, 128, false);
+                mma_small(tmem + 256, aW, OP_K, aK, OP_K, KS, 128, false);
                 umma_commit(&bars[B_XQK]);
                 // U = T~ W  (lo x lo terms are dropped everywhere)
                 if (!wait(R_TT, par)) break;
                 tc_fence_after_sync();
-                mma(tmem + 0, aQ, OP_K, aW, OP_MN, 8, HD, false);
-                mma(tmem + 0, aK, OP_K, aW, OP_MN, 8, HD, true);
+                mma_small(tmem + 0, aQ, OP_K, aW, OP_MN, 8, HD, false);
+                mma_small(tmem + 0, aK, OP_K, aW, OP_MN, 8, HD, true);
                 umma_commit(&bars[B_U]);
                 if (SAVE) {   // the tiles kept for the chain rule leave through TMA stores, straight from the operand slots
                     store(&tm.th, sQK, kT, chunk);
@@ -159,9 +159,9 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 // Y = T~ Xk
                 if (!wait(R_XK, par)) break;
                 tc_fence_after_sync();
-                mma(tmem + 384, aQ, OP_K, aBig + 2 * kTileB, OP_MN, 8, 128, false);
-                mma(tmem + 384, aK, OP_K, aBig + 2 * kTileB, OP_MN, 8, 128, true);
-                mma(tmem + 384, aQ, OP_K, aBig + 3 * kTileB, OP_MN, 8, 128, true);
+                mma_small(tmem + 384, aQ, OP_K, aBig + 2 * kTileB, OP_MN, 8, 128, false);
+                mma_small(tmem + 384, aK, OP_K, aBig + 2 * kTileB, OP_MN, 8, 128, true);
+                mma_small(tmem + 384, aQ, OP_K, aBig + 3 * kTileB, OP_MN, 8, 128, true);
                 if (SAVE) {   // B_Y lets the workers overwrite T~ (with U) and Xk (with Y): the stores must have read them
                     store(&tm.xk, sBig + 2 * kTileB, kT, chunk);
                     tma_store_commit();
@@ -171,11 +171,11 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 // Xq U and W^T U
                 if (!wait(R_U, par)) break;
                 tc_fence_after_sync();
-                mma(tmem + 256, aBig, OP_K, aQ, OP_MN, 8, HD, false);
-                mma(tmem + 256, aBig + kTileB, OP_K, aQ, OP_MN, 8, HD, true);
-                mma(tmem + 256, aBig, OP_K, aK, OP_MN, 8, HD, true);
-                mma(tmem + 128, aW, OP_MN, aQ, OP_MN, 8, HD, false);
-                mma(tmem + 128, aW, OP_MN, aK, OP_MN, 8, HD, true);
+                mma_small(tmem + 256, aBig, OP_K, aQ, OP_MN, 8, HD, false);
+                mma_small(tmem + 256, aBig + kTileB, OP_K, aQ, OP_MN, 8, HD, true);
+                mma_small(tmem + 256, aBig, OP_K, aK, OP_MN, 8, HD, true);
+                mma_small(tmem + 128, aW, OP_MN, aQ, OP_MN, 8, HD, false);
+                mma_small(tmem + 128, aW, OP_MN, aK, OP_MN, 8, HD, true);
                 umma_commit(&bars[B_G3A]);
                 if (SAVE) {
                     store(&tm.u, sQK, HD, chunk);
@@ -184,8 +184,8 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 // Y^T W
                 if (!wait(R_Y, par)) break;
                 tc_fence_after_sync();
-                mma(tmem + 384, aBig + 2 * kTileB, OP_MN, aW, OP_MN, 8, HD, false);
-                mma(tmem + 384, aBig + 3 * kTileB, OP_MN, aW, OP_MN, 8, HD, true);
+                mma_small(tmem + 384, aBig + 2 * kTileB, OP_MN, aW, OP_MN, 8, HD, false);
+                mma_small(tmem + 384, aBig + 3 * kTileB, OP_MN, aW, OP_MN, 8, HD, true);
                 umma_commit(&bars[B_G3B]);
                 // next chunk: once this chunk's last product has retired every tile slot is free
                 const int next = chunk + (int)gridDim.x;
@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                     load(next);
                     if (!wait(B_LOAD, par ^ 1)) break;
                     tc_fence_after_sync();
-                    mma(tmem + 0, aW, OP_K, aW, OP_K, KS, 128, false);
+                    mma_small(tmem + 0, aW, OP_K, aW, OP_K, KS, 128, false);
                     umma_commit(&bars[B_GM]);
                 }
             }

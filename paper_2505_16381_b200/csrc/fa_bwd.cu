@@ -98,19 +98,27 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
         : "memory");
 }
 
-// D[tmem] (+)= A B^T with both operands K-major [rows][kdim] tiles (two 64-column panels per 128 of kdim).
+// D[tmem] (+)= A B^T with both operands K-major [rows][kdim] tiles (two 64-column panels per 128 of kdim).  Descriptors
+// advance by their low word only (32 bytes per step, the next panel after four steps).
 __device__ __forceinline__ void mma_kk(uint32_t d_tmem, uint32_t a0, uint32_t b0, int kdim, uint32_t idesc, bool acc) {
+    uint32_t a_lo = umma_desc_lo(a0, 16), b_lo = umma_desc_lo(b0, 16);
+#pragma unroll
     for (int kk = 0; kk < kdim / 16; ++kk) {
-        const uint32_t off = (kk >> 2) * kPanelBytes + (kk & 3) * 32;
-        umma_ss(d_tmem, umma_desc(a0 + off, 16, 1024), umma_desc(b0 + off, 16, 1024), idesc, (acc || kk > 0) ? 1u : 0u);
+        umma_ss(d_tmem, umma_desc_join(a_lo), umma_desc_join(b_lo), idesc, (acc || kk > 0) ? 1u : 0u);
+        const uint32_t step = (kk & 3) == 3 ? (kPanelBytes - 96u) >> 4 : 2u;
+        a_lo += step;
+        b_lo += step;
     }
 }
 // D[tmem] (+)= A B with A in tensor memory (packed bf16: the 64 contraction indices [64h, 64h+64) of a row sit in the
-// 32 columns starting at a_col + 64h) and B MN-major [128 (k)][HD] in shared memory.
+// 32 columns starting at a_col + 64h) and B MN-major [128 (k)][HD] in shared memory (2048 bytes per step).
 __device__ __forceinline__ void mma_tn(uint32_t d_tmem, uint32_t a_col, uint32_t b0, uint32_t idesc, bool acc) {
-    for (int kk = 0; kk < kTile / 16; ++kk)
-        umma_ts(d_tmem, a_col + (kk >> 2) * 64 + (kk & 3) * 8, umma_desc(b0 + kk * 2048, kPanelBytes, 1024), idesc,
-                (acc || kk > 0) ? 1u : 0u);
+    uint32_t b_lo = umma_desc_lo(b0, kPanelBytes);
+#pragma unroll
+    for (int kk = 0; kk < kTile / 16; ++kk) {
+        umma_ts(d_tmem, a_col + (kk >> 2) * 64 + (kk & 3) * 8, umma_desc_join(b_lo), idesc, (acc || kk > 0) ? 1u : 0u);
+        b_lo += 128u;
+    }
 }
 
 __device__ __forceinline__ void tma_tile(uint8_t* dst, const CUtensorMap* m, uint64_t* bar, int kdim, int row0) {

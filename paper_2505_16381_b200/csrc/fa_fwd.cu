@@ -215,11 +215,13 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
                 if (ok && !mbar_wait(&bars[bar], parity & 1, abort_flag, ST_FWD_MMA)) ok = false;
             };
             auto issue_s = [&](int x, int qs, int ks, int kdim, bool acc) {   // ks >= 2: a V slot
-                const uint32_t a0 = smem_u32(sQ + qs * kSlotBytes), b0 = smem_u32(sK + ks * kSlotBytes);
+                // (descriptors advance by their low word only: 32 bytes per step, the next panel after four steps)
+                uint32_t a_lo = umma_desc_lo(smem_u32(sQ + qs * kSlotBytes), 16), b_lo = umma_desc_lo(smem_u32(sK + ks * kSlotBytes), 16);
                 for (int kk = 0; kk < kdim / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * kPanelBytes + (kk & 3) * 32;
-                    umma_ss(tmem + x * 128, umma_desc(a0 + off, 16, 1024), umma_desc(b0 + off, 16, 1024), idescS,
-                            (acc || kk > 0) ? 1u : 0u);
+                    umma_ss(tmem + x * 128, umma_desc_join(a_lo), umma_desc_join(b_lo), idescS, (acc || kk > 0) ? 1u : 0u);
+                    const uint32_t step = (kk & 3) == 3 ? (kPanelBytes - 96u) >> 4 : 2u;
+                    a_lo += step;
+                    b_lo += step;
                 }
             };
             int qi_next = 0;                   // query operands waited for so far (all work items)
@@ -296,10 +298,13 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
                     tc_fence_after_sync();
                     if (!ok) break;
                     {
-                        const uint32_t b0 = smem_u32(sV + x * kSlotBytes);
-                        for (int kk = 0; kk < kTile / 16; ++kk)
-                            umma_ts(tmem + 256 + x * 128, tmem + x * 128 + kk * 8,
-                                    umma_desc(b0 + kk * 2048, kPanelBytes, 1024), idescO, (t > 0 || kk > 0) ? 1u : 0u);
+                        uint32_t b_lo = umma_desc_lo(smem_u32(sV + x * kSlotBytes), kPanelBytes);
+#pragma unroll
+                        for (int kk = 0; kk < kTile / 16; ++kk) {
+                            umma_ts(tmem + 256 + x * 128, tmem + x * 128 + kk * 8, umma_desc_join(b_lo), idescO,
+                                    (t > 0 || kk > 0) ? 1u : 0u);
+                            b_lo += 128u;
+                        }
                         umma_commit(&bars[B_VEMPTY + x]);
                     }
                     // the stream's next S overwrites P; products issued by one thread execute in order, so it lands

@@ -182,6 +182,19 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes
     d |= (uint64_t)2 << 61;  // SWIZZLE_128B
     return d;
 }
+// The same descriptor in two words.  From one step of a product to the next only the start address changes, and it sits
+// in the low word together with the leading-dimension offset; strides, version and swizzle mode are the high word, which
+// is one constant for every tile used here (SBO = 1024, 128-byte swizzle).  The thread that issues the products is a
+// single instruction stream: the fewer instructions between two tcgen05.mma, the closer the pipe runs to its own pace.
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+constexpr uint32_t kUmmaDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint64_t umma_desc_join(uint32_t lo) {
+    uint64_t d;
+    asm volatile("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(kUmmaDescHi));
+    return d;
+}
 // Instruction descriptor for kind::f16: bf16 x bf16 -> f32, M x N tile, operand majors.
 __host__ __device__ constexpr uint32_t umma_idesc(int M, int N, int a_mn_major, int b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |

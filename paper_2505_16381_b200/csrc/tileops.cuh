@@ -20,13 +20,42 @@ __device__ __forceinline__ uint64_t desc_k(uint32_t t, int kk) {
 }
 __device__ __forceinline__ uint64_t desc_mn(uint32_t t, int kk) { return umma_desc(t + kk * 2048, kPanelB, 1024); }
 
-// D[128 x n] (+)= (+-) op(A) op(B), `ksteps` steps of 16 along the contraction.
+// D[128 x n] (+)= (+-) op(A) op(B), `ksteps` steps of 16 along the contraction.  One thread issues all of them, so the
+// instructions between two tcgen05.mma count: only the low word of a descriptor changes from step to step (the start
+// address; the strides and the swizzle mode sit in the high word), by a constant the view decides.
 __device__ __forceinline__ void mma(uint32_t d_tmem, uint32_t a_tile, int a_op, uint32_t b_tile, int b_op, int ksteps,
                                     int n, bool acc, bool negate = false) {
+    const uint32_t idesc = umma_idesc(128, n, a_op, b_op) | (negate ? (1u << 13) : 0u);
+    uint32_t a_lo = umma_desc_lo(a_tile, a_op == OP_K ? 16u : kPanelB);
+    uint32_t b_lo = umma_desc_lo(b_tile, b_op == OP_K ? 16u : kPanelB);
+    // K view: 32 bytes per step, the next 64-column panel after four; MN view: 2048 bytes per step
+    const uint32_t a_step = a_op == OP_K ? 2u : 128u, a_jump = a_op == OP_K ? (kPanelB - 96u) >> 4 : 128u;
+    const uint32_t b_step = b_op == OP_K ? 2u : 128u, b_jump = b_op == OP_K ? (kPanelB - 96u) >> 4 : 128u;
+    uint32_t accum = acc ? 1u : 0u;
+    for (int kk = 0; kk < ksteps; ++kk) {
+        umma_ss(d_tmem, umma_desc_join(a_lo), umma_desc_join(b_lo), idesc, accum);
+        accum = 1u;
+        const bool last_of_panel = (kk & 3) == 3;
+        a_lo += last_of_panel ? a_jump : a_step;
+        b_lo += last_of_panel ? b_jump : b_step;
+    }
+}
+
+// The products of a kernel whose issuing thread lives on a small register allotment (setmaxnreg): descriptors rebuilt at
+// every step, nothing carried across the loop.
+__device__ __forceinline__ void mma_small(uint32_t d_tmem, uint32_t a_tile, int a_op, uint32_t b_tile, int b_op, int ksteps,
+                                          int n, bool acc, bool negate = false) {
     const uint32_t idesc = umma_idesc(128, n, a_op, b_op) | (negate ? (1u << 13) : 0u);
     for (int kk = 0; kk < ksteps; ++kk)
         umma_ss(d_tmem, a_op == OP_K ? desc_k(a_tile, kk) : desc_mn(a_tile, kk),
                 b_op == OP_K ? desc_k(b_tile, kk) : desc_mn(b_tile, kk), idesc, (acc || kk > 0) ? 1u : 0u);
+}
+
+// The same as a real function, for kernels that issue dozens of different products from straight-line code: inlined,
+// they no longer fit the instruction cache (and the issuing thread's small register allotment).
+static __device__ __noinline__ void mma_call(uint32_t d_tmem, uint32_t a_tile, int a_op, uint32_t b_tile, int b_op, int ksteps,
+                                             int n, bool acc, bool negate = false) {
+    mma(d_tmem, a_tile, a_op, b_tile, b_op, ksteps, n, acc, negate);
 }
 
 // Stores columns c0 .. c0+31 of `row` of a swizzled bf16 tile.
