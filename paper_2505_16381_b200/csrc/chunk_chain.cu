@@ -21,12 +21,6 @@ using namespace tile;
 
 namespace {
 
-#ifdef CHAIN_STAMPS
-__device__ long long g_chain_stamps[32];
-#define STAMP(i) do { if (blockIdx.x == 0 && tid == 32 && chunk == (int)blockIdx.x + 3 * (int)gridDim.x) stamps[i] = clock64(); } while (0)
-#else
-#define STAMP(i) do {} while (0)
-#endif
 constexpr int kSlots = 7;
 constexpr uint32_t kBarOff = kSlots * kTileB;
 constexpr uint32_t kChainSmem = kBarOff + 64 + kT * 4 + kT * 4 + 1024;
@@ -62,9 +56,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     constexpr int KD = HD / 16, K8 = 8;
     constexpr uint32_t cDW = 0, cA = 128, cB = 256, cG = 384;   // tensor-memory columns: dw, two work accumulators, W W^T
     bool ok = true;
-#ifdef CHAIN_STAMPS
-    long long* stamps = g_chain_stamps;
-#endif
     uint32_t ph_load = 0, ph_mma = 0;
     float v[32];
 
@@ -136,20 +127,25 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     // slots: 0 U->W   1 dQl->dT->tmp->dGm   2 Y^T->-Xq->Xk->T->Ah->K   3 dSd->T lo->dT lo->tmp lo->dSd   4 dXq   5 dKr->dY->dXk
     //        6 dP->dU->Al->Q
     // first tiles of a chunk: U, Y, (s dSd)^T (every use below takes the transposed view), dQl, dKr, dP
-    auto first_loads = [&](int ch) {
+    // They are requested in two parts: four of the six slots are free as soon as phase 5's products have retired, the
+    // other two (0, 1) feed the chunk's very last products.  All bytes are announced with the first part.
+    auto first_loads_a = [&](int ch) {
         mbar_expect_tx(&bars[0], 4 * kT * HD * 2 + 2 * kTileB);
         tma_tile(slot(6), &tm.dp, &bars[0], HD, ch * HD);
-        tma_tile(slot(0), &tm.u, &bars[0], HD, ch * kT);
         tma_tile(slot(2), &tm.yt, &bars[0], kT, ch * kT);
         tma_tile(slot(3), &tm.dsdt, &bars[0], kT, ch * kT);
-        tma_tile(slot(1), &tm.dql, &bars[0], HD, ch * kT);
         tma_tile(slot(5), &tm.dkr, &bars[0], HD, ch * kT);
     };
-    if (tid == 0 && (int)blockIdx.x < nchunks) first_loads(blockIdx.x);
-
+    auto first_loads_b = [&](int ch) {
+        tma_tile(slot(0), &tm.u, &bars[0], HD, ch * kT);
+        tma_tile(slot(1), &tm.dql, &bars[0], HD, ch * kT);
+    };
+    if (tid == 0 && (int)blockIdx.x < nchunks) {
+        first_loads_a(blockIdx.x);
+        first_loads_b(blockIdx.x);
+    }
 #pragma unroll 1
     for (int chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
-    STAMP(30);
     const int s_idx = chunk / p.N, pos = (chunk % p.N) * kT + row;   // slice and position of this thread's row
     const bool row_valid = pos < p.L;
     const size_t urow = (size_t)s_idx * p.L + pos;                   // row in the caller's [S][L][.] tensors
@@ -159,9 +155,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     if (tid < kT) bt[tid] = p.beta[(size_t)chunk * kT + tid];   // first read after several barriers (phase 4)
     // ---- phase 0a: dXq = lower(-(dQl U^T + s dSd Y^T))
     loads_wait();
-    STAMP(0);
     publish();
-    STAMP(1);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(1), OP_K, sa(0), OP_K, KD, 128, false);
@@ -172,7 +166,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    STAMP(2);
     if (!ok) break;
     // ---- phase 1: dY = -(W dKr^T + Xq^T s dSd),  dU = -(Xq^T dQl + W dP),  Gm = W W^T
     // (every group's tiles are requested as soon as the products that read the slots have retired, before the
@@ -184,9 +177,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     acc_to_tile(cA, kT, slot(4), -1.f, M_LOWER);                    // dXq
     loads_wait();
-    STAMP(3);
     publish();
-    STAMP(4);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(0), OP_K, sa(5), OP_K, KD, 128, false);
@@ -197,7 +188,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    STAMP(5);
     if (!ok) break;
     // ---- phase 2: dT = lower(dY Xk^T + dU W^T)
     if (tid == 0) {
@@ -207,9 +197,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     acc_to_tile(cA, kT, slot(5), -1.f, M_NONE);                     // dY (over dKr)
     acc_to_tile(cB, HD, slot(6), -1.f, M_NONE);                     // dU (over dP)
     loads_wait();
-    STAMP(6);
     publish();
-    STAMP(7);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(5), OP_K, sa(2), OP_K, K8, 128, false);
@@ -217,7 +205,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    STAMP(8);
     if (!ok) break;
     // ---- phase 3: dXk = strictLower(T~^T dY) -> cB,  dw += T~^T dU.  (s dSd)^T is not needed again before phase 5, where
     // it is loaded once more: until then its slot (3) takes the lo parts of the bf16 pairs, so that the hi and lo products
@@ -230,9 +217,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     // dT stays in tensor memory (cA); its bf16 hi part goes to slot 1 now, the lo part follows in phase 4
     split_to_tile(cA, slot(1), false, f_dT);
     loads_wait();
-    STAMP(9);
     publish();
-    STAMP(10);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cB, sa(2), OP_MN, sa(5), OP_MN, K8, 128, false);
@@ -242,7 +227,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    STAMP(11);
     if (!ok) break;
     // ---- phase 4: M = Ainv^T dT -> cB;  dbeta_c = M_cc;  tmp = M D;  dA = strictLower(-tmp Ainv^T) -> cA
     if (tid == 0) {
@@ -253,9 +237,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     acc_to_tile(cB, kT, slot(5), 1.f, M_STRICT);                    // dXk (over dY)
     split_to_tile(cA, slot(3), true, f_dT);                         // dT lo (over T~ lo)
     loads_wait();
-    STAMP(12);
     publish();
-    STAMP(13);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, 128, false);
@@ -264,7 +246,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    STAMP(14);
     if (!ok) break;
     {   // diagonal of M -> t1
         const int c0 = (row >> 5) << 5;
@@ -277,7 +258,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     }
     split_both(cB, slot(1), slot(3), f_tmp);                        // tmp = M D, hi (over dT hi) and lo (over dT lo)
     publish();
-    STAMP(15);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cA, sa(1), OP_K, sa(2), OP_K, K8, 128, false);
@@ -286,7 +266,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    STAMP(16);
     if (!ok) break;
     if (tid == 0) {   // phase 5's K and Q replace Ainv hi / lo, whose last products have just retired; (s dSd)^T returns
         mbar_expect_tx(&bars[0], 2 * kT * HD * 2 + kTileB);
@@ -314,9 +293,7 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
     split_to_tile(cA, slot(1), false, f_dGm);                       // dGm = D dA, hi
     // ---- phase 5: dq -> cB, dk -> cG and the rest of dw
     loads_wait();
-    STAMP(17);
     publish();
-    STAMP(18);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cB, sa(3), OP_MN, sa(2), OP_MN, K8, HD, false);   // s dSd K
@@ -330,11 +307,10 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     mma_wait();
-    STAMP(19);
     if (!ok) break;
+    if (tid == 0 && chunk + (int)gridDim.x < nchunks) first_loads_a(chunk + gridDim.x);   // slots 2, 3, 5, 6 are free
     split_to_tile(cA, slot(1), true, f_dGm);                        // dGm lo
     publish();
-    STAMP(20);
     if (tid == 0) {
         tc_fence_after_sync();
         mma_call(tmem + cDW, sa(1), OP_K, sa(0), OP_MN, K8, HD, true);
@@ -342,9 +318,10 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         umma_commit(&bars[1]);
     }
     // the dQl / dKr rows of the final sums are fetched while the last products run
-    uint4 pre_q[HD / 64][4], pre_k[HD / 64][4];
+    constexpr int NI = HD / 64;
+    uint4 pre_q[NI][4], pre_k[NI][4];
 #pragma unroll
-    for (int c = 0; c < HD / 64; ++c) {
+    for (int c = 0; c < NI; ++c) {
         const int c0 = half * (HD / 2) + c * 32;
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
@@ -353,12 +330,11 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         }
     }
     mma_wait();
-    STAMP(21);
     if (!ok) break;
-    // every product of this chunk has retired: all tile slots are free for the next chunk's first tiles
-    if (tid == 0 && chunk + (int)gridDim.x < nchunks) first_loads(chunk + gridDim.x);
+    // every product of this chunk has retired: the last two slots are free for the next chunk's first tiles
+    if (tid == 0 && chunk + (int)gridDim.x < nchunks) first_loads_b(chunk + gridDim.x);
 #pragma unroll
-    for (int c = 0; c < HD / 64; ++c) {
+    for (int c = 0; c < NI; ++c) {
         const int c0 = half * (HD / 2) + c * 32;
         float in[32];
         tmem_row32(tl + cB + c0, v);
@@ -374,7 +350,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
         tmem_row32(tl + cDW + c0, v);
         gstore_bf16x32(p.dw + urow * HD + c0, v, row_valid);
     }
-    STAMP(31);
     // the next chunk's first products overwrite the accumulators read above
     tc_fence_before_sync();
     __syncthreads();
@@ -391,12 +366,6 @@ __global__ void __launch_bounds__(256, 1) chunk_chain_kernel(const __grid_consta
 }
 
 }  // namespace
-
-#ifdef CHAIN_STAMPS
-extern "C" int path_attn_debug_chain_stamps(long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, g_chain_stamps, sizeof(long long) * 32);
-}
-#endif
 
 cudaError_t launch_chunk_chain(const ChainTensorMaps& tm, const ChainParams& p, int hd, int nchunks, cudaStream_t st) {
     int dev = 0, sms = 0;
