@@ -57,6 +57,51 @@ __host__ __device__ inline int lowest_set(unsigned x) {
 __host__ __device__ inline int qslot(int level, int I) { return level == lowest_set((unsigned)I) ? 0 : level; }
 __host__ __device__ inline int kslot(int level, int J) { return level == lowest_set(~(unsigned)J) ? 0 : level; }
 
+// Where the versions live.  Plane 0 is [S][Lp][d]: every chunk's boundary-adjusted tile (= its version at its first usable
+// level).  The other versions follow, packed: slice after slice, chunk after chunk, level after level.  Query chunk I
+// has one per set bit of I above the lowest, key chunk J one per clear bit of J (below nlev) above the lowest, so a
+// slice holds about N log2(N) / 2 extra tiles instead of N (log2(N) - 1).  All positions are closed forms of the chunk
+// index (prefix sums of bit counts), so no table is stored.
+__host__ __device__ inline int popcount32(unsigned x) {
+#ifdef __CUDA_ARCH__
+    return __popc(x);
+#else
+    return __builtin_popcount(x);
+#endif
+}
+__host__ __device__ inline int popcount_prefix(unsigned n) {   // sum of popcount(c) over c = 0 .. n-1
+    int total = 0;
+    for (int j = 0; j < 31 && (1u << j) < n; ++j) {
+        const int rem = (int)(n & ((2u << j) - 1u)) - (int)(1u << j);
+        total += (int)((n >> (j + 1)) << j) + (rem > 0 ? rem : 0);
+    }
+    return total;
+}
+struct VerLayout {
+    int S, N, Lp, nlev;
+    int eq, ek;   // extra tiles per slice on the query / key side
+};
+__host__ __device__ inline int q_extra_before(int I) { return I > 0 ? popcount_prefix((unsigned)I) - (I - 1) : 0; }
+__host__ __device__ inline int k_extra_before(int J, int nlev) { return nlev > 0 ? J * (nlev - 1) - popcount_prefix((unsigned)J) : 0; }
+__host__ __device__ inline VerLayout make_ver_layout(int S, int N, int Lp, int nlev) {
+    VerLayout v{S, N, Lp, nlev, 0, 0};
+    v.eq = q_extra_before(N);
+    const int last = nlev - popcount32((unsigned)(N - 1)) - 1;
+    v.ek = k_extra_before(N - 1, nlev) + (last > 0 ? last : 0);
+    return v;
+}
+// First row (in units of rows of d elements) of the level-`level` version of query chunk I / key chunk J of slice s.
+__host__ __device__ inline long qver_row(const VerLayout& v, int s, int level, int I) {
+    if (level == lowest_set((unsigned)I)) return (long)s * v.Lp + (long)I * CHUNK;
+    const int rank = popcount32((unsigned)I & ((1u << level) - 1u)) - 1;
+    return ((long)v.S * v.N + (long)s * v.eq + q_extra_before(I) + rank) * CHUNK;
+}
+__host__ __device__ inline long kver_row(const VerLayout& v, int s, int level, int J) {
+    if (level == lowest_set(~(unsigned)J)) return (long)s * v.Lp + (long)J * CHUNK;
+    const int rank = level - popcount32((unsigned)J & ((1u << level) - 1u)) - 1;
+    return ((long)v.S * v.N + (long)s * v.ek + k_extra_before(J, v.nlev) + rank) * CHUNK;
+}
+
 struct FwdTensorMaps {
     CUtensorMap q_raw, k_raw, v, qv, kv, xqn, yt;  // qv/kv also serve as the low parts' maps in split mode
 };
@@ -68,6 +113,7 @@ struct FwdParams {
     const int* nkeep;   // [S, N] key chunks each query chunk has to visit (gated problems), or nullptr = all
     uint32_t* status;   // device status word
     int S, L, Lp, N;
+    VerLayout vl;       // placement of the query / key versions behind tm.qv / tm.kv
     float scale;
     int out_fp32;
     // segment-against-segment sweep of the context-parallel path only (launch_fa_fwd_cross): the key segment's padded
@@ -85,19 +131,20 @@ struct LevelTable {
 
 struct LevelTensorMaps {
     CUtensorMap dyh, dyl;   // [matrices * d][d] bf16 hi / lo planes of the run products
-    CUtensorMap qv, kv;     // [slots * S * Lp][d] bf16 versions
+    CUtensorMap qv, kv;     // bf16 versions, rows of d elements placed by VerLayout
     CUtensorMap dqv, dkv;   // same shape: bf16 gradients of the versions (backward only)
     CUtensorMap ddy;        // [matrices * d][d] bf16 gradients of the run products (backward only)
 };
 
 struct LevelParams {
     LevelTable lv;
+    VerLayout vl;
     int l;                  // dyadic forward: level consumed (l -> l + 1); version forward: number of levels; level backward: the
                             // level of the run products whose gradients the launch finishes
     int nlev;               // number of levels (level backward)
     int S, N, Lp;
     __nv_bfloat16 *dyh, *dyl, *qv, *kv;
-    __nv_bfloat16 *dqv, *dkv;     // [slots][S][Lp][d] gradients of the versions; slot 0 ends up holding the final sums
+    __nv_bfloat16 *dqv, *dkv;     // gradients of the versions (placed like them); plane 0 ends up holding the final sums
     __nv_bfloat16* ddy16;         // gradients of the run products, same placement as the run products themselves
     float* kc;                    // edge kernels: [S][cap][d] float32 out (rows < L of every slice), or nullptr
     int cap, L;
@@ -162,7 +209,8 @@ struct BwdTensorMaps {
 };
 
 struct BwdParams {
-    __nv_bfloat16* dqv;  // [slots][S][Lp][d] gradients of the query versions (slot convention as the versions), bf16
+    VerLayout vl;        // placement of the versions and of their gradients
+    __nv_bfloat16* dqv;  // gradients of the query versions (placed like the versions), bf16
     __nv_bfloat16* dkv;  // same for the key versions
     void* dv;            // [S, L, d] bf16, final
     float* dsd;          // [S*N][128 q][128 k] lower(dS) of the diagonal chunks, unscaled; written for gated problems only

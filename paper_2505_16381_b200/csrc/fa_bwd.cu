@@ -181,7 +181,9 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
         return true;
     };
     int J = 0, s = 0;   // current item of this thread's role
-    auto ver_row = [&](int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
+    auto qrow = [&](int lvl, int chunk) { return qver_row(p.vl, s, lvl, chunk); };   // first row of a version tile
+    auto krow = [&](int lvl, int chunk) { return kver_row(p.vl, s, lvl, chunk); };
+    auto row0 = [&](int chunk) { return (long)s * p.Lp + (long)chunk * kTile; };      // plane 0
     auto level = [&](int t) { return t == 0 ? -1 : msb32((unsigned)((J + t) ^ J)); };
     // query chunks this key chunk meets (I = J .. J + T - 1): all later ones, or fewer when the gate has made the far
     // pairs negligible (every warp role reads the same precomputed number)
@@ -222,7 +224,7 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
                         if (!ok) break;
                         mbar_expect_tx(&bars[K_KFULL], kTile * HD * 2);
                         if (t == 0) tma_tile(sK, &tm.k_raw, &bars[K_KFULL], HD, rowJ);
-                        else tma_tile(sK, &tm.kv, &bars[K_KFULL], HD, ver_row(kslot(l, J), J));
+                        else tma_tile(sK, &tm.kv, &bars[K_KFULL], HD, (int)krow(l, J));
                         ++nk;
                     }
                     if (t == 0) {
@@ -236,7 +238,7 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
                         ++nv;
                         load_do(&tm.d_o, HD, rowJ);
                     } else {
-                        load_q(&tm.qv, HD, ver_row(qslot(l, I), I));
+                        load_q(&tm.qv, HD, (int)qrow(l, I));
                         load_do(&tm.d_o, HD, s * p.Lp + I * kTile);
                     }
                     // per-query statistics of the step
@@ -360,7 +362,7 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
         int g = 0;                               // steps before the current item
         constexpr int CW = HD / 2;               // accumulator columns per thread when flushing
         auto flush_dk = [&](int lvl) {   // the version's gradient leaves as bf16, the form the version chain rule multiplies
-            store_acc_bf16<CW>(p.dkv + ((size_t)ver_row(kslot(lvl, J), J) + row) * HD + h * CW, tlane + colDK + h * CW, p.scale);
+            store_acc_bf16<CW>(p.dkv + ((size_t)krow(lvl, J) + row) * HD + h * CW, tlane + colDK + h * CW, p.scale);
         };
         auto step = [&](auto first_tag, const int t) {
             constexpr bool FIRST = decltype(first_tag)::value;   // the diagonal chunk: causal mask, dSd written out
@@ -484,7 +486,7 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
                 break;
             }
             auto zero_dk = [&](int slot) {
-                uint4* dst = reinterpret_cast<uint4*>(p.dkv + ((size_t)ver_row(slot, J) + row) * HD + h * CW);
+                uint4* dst = reinterpret_cast<uint4*>(p.dkv + ((size_t)row0(J) + row) * HD + h * CW);
                 for (int x = 0; x < CW / 8; ++x) dst[x] = make_uint4(0u, 0u, 0u, 0u);
             };
             if (T > 1) flush_dk(level(T - 1));
@@ -585,7 +587,9 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
         return true;
     };
     int I = 0, s = 0;
-    auto ver_row = [&](int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
+    auto qrow = [&](int lvl, int chunk) { return qver_row(p.vl, s, lvl, chunk); };   // first row of a version tile
+    auto krow = [&](int lvl, int chunk) { return kver_row(p.vl, s, lvl, chunk); };
+    auto row0 = [&](int chunk) { return (long)s * p.Lp + (long)chunk * kTile; };      // plane 0
     auto level = [&](int t) { return msb32((unsigned)(I ^ (I - 1 - t))); };
     // earlier key chunks this query chunk visits (J = I-1 .. I-T): all of them, or fewer when the gate has made the far
     // ones negligible (every warp role reads the same precomputed number; the diagonal chunk is not part of this sweep)
@@ -615,13 +619,13 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
                         wait_empty(Q_QEMPTY, nq);
                         if (!ok) break;
                         mbar_expect_tx(&bars[Q_QFULL], kTile * HD * 2);
-                        tma_tile(sQ, &tm.qv, &bars[Q_QFULL], HD, ver_row(qslot(l, I), I));
+                        tma_tile(sQ, &tm.qv, &bars[Q_QFULL], HD, (int)qrow(l, I));
                         ++nq;
                     }
                     wait_empty(Q_KEMPTY + kn % 3, kn / 3);
                     if (!ok) break;
                     mbar_expect_tx(&bars[Q_KFULL + kn % 3], kTile * HD * 2);
-                    tma_tile(sK + (kn % 3) * kSlotBytes, &tm.kv, &bars[Q_KFULL + kn % 3], HD, ver_row(kslot(l, J), J));
+                    tma_tile(sK + (kn % 3) * kSlotBytes, &tm.kv, &bars[Q_KFULL + kn % 3], HD, (int)krow(l, J));
                     ++kn;
                     wait_empty(Q_VEMPTY + (vn & 1), vn >> 1);
                     if (!ok) break;
@@ -704,13 +708,13 @@ __global__ void __launch_bounds__(384, 1) dq_kernel(const __grid_constant__ BwdT
         int g = 0, na = 0;
         constexpr int CW = HD / 2;
         auto flush_dq = [&](int lvl) {
-            store_acc_bf16<CW>(p.dqv + ((size_t)ver_row(qslot(lvl, I), I) + row) * HD + h * CW, tlane + colDQ + h * CW, p.scale);
+            store_acc_bf16<CW>(p.dqv + ((size_t)qrow(lvl, I) + row) * HD + h * CW, tlane + colDQ + h * CW, p.scale);
         };
 #pragma unroll 1
         for (int it = 0; item_of(it, I, s); ++it) {
             const int T = steps_of(I, s);
             auto zero_dq = [&](int slot) {   // a whole [128 x HD] version gradient tile, by the 256 math threads
-                uint4* dst = reinterpret_cast<uint4*>(p.dqv + (size_t)ver_row(slot, I) * HD);
+                uint4* dst = reinterpret_cast<uint4*>(p.dqv + (size_t)row0(I) * HD);
                 for (int i = threadIdx.x - 128; i < kTile * HD / 8; i += 256) dst[i] = make_uint4(0u, 0u, 0u, 0u);
             };
             // no key chunk visited (chunk 0, or block skipping left only the diagonal): the boundary-adjusted queries get a

@@ -145,7 +145,7 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
         if (CROSS) return p.Nk;
         return p.nkeep ? min(I + 1, p.nkeep[s * p.N + I]) : I + 1;
     };
-    auto ver_row = [&](int s, int slot, int chunk) { return (slot * p.S + s) * p.Lp + chunk * kTile; };
+
 
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
@@ -198,10 +198,10 @@ fa_fwd_kernel(const __grid_constant__ FwdTensorMaps tm, const FwdParams p) {
                 for (int n = 1; n < NS && ok; ++n) {
                     const int J = I - n, x = n & 1, l = msb32((unsigned)(I ^ J));   // l is non-decreasing in n
                     if (l != cur) {
-                        load_q(&tm.qv, HD, ver_row(s, qslot(l, I), I));
+                        load_q(&tm.qv, HD, (int)qver_row(p.vl, s, l, I));
                         cur = l;
                     }
-                    load_kv(sK, B_KFULL, B_KEMPTY, x, kf, &tm.kv, HD, ver_row(s, kslot(l, J), J));
+                    load_kv(sK, B_KFULL, B_KEMPTY, x, kf, &tm.kv, HD, (int)kver_row(p.vl, s, l, J));
                     load_kv(sV, B_VFULL, B_VEMPTY, x, vf, &tm.v, HD, s * p.Lp + J * kTile);
                 }
             }

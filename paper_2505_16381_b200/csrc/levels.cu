@@ -178,11 +178,11 @@ __global__ void __launch_bounds__(256, 2) version_fwd_kernel(const __grid_consta
     for (; l2 < lim && c.ok; ++l2) {
         if (!version_step(is_key, ch, l2, p.N, l1, b, src)) continue;
         const long mat = p.lv.dy_off[l1] / (HD * HD) + (long)s * p.lv.dy_cnt[l1] + b;
-        const long row_dst = ((long)l2 * p.S + s) * p.Lp + (long)ch * kT;
+        const long row_dst = is_key ? kver_row(p.vl, s, l2, ch) : qver_row(p.vl, s, l2, ch);
         if (c.tid == 0) {
             mbar_expect_tx(&c.bars[0], (first ? 3 : 2) * kT * HD * 2);
             if (first) {
-                const long row_src = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
+                const long row_src = is_key ? kver_row(p.vl, s, l1, ch) : qver_row(p.vl, s, l1, ch);
                 tma_tile(sm, is_key ? &tm.kv : &tm.qv, &c.bars[0], HD, (int)row_src);
             }
             tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(256, 2) version_fwd_kernel(const __grid_consta
 //         queries (b even, b >= 2, ch = (b << l1) + 2^l1 + x):   dDy += Qv[l1][ch]^T g,   dQv[l1][ch] += g Dy^T
 //         keys    (b odd,          ch = ((b-1) << l1) + x):      dDy += g^T Kv[l1][ch],   dKv[l1][ch] += g Dy
 //       (the second product is the chain's carry: added in place to the gradient the sweep left at level l1, which the
-//       launch of level l1's own source level, or the chunk chain rule for slot 0, reads next).
+//       launch of level l1's own source level, or the chunk chain rule for plane 0, reads next).
 // The run products enter as single bf16 operands (their hi plane), like every other operand of a gradient product.
 // dDy is written once, as bf16: it is only ever read as an MMA operand (by the next launch and, at level 0, by the
 // chunk chain rule as dP).  Runs with b = 0 multiply nothing (no boundary lies before chunk 0): only level 0 writes them.
@@ -270,19 +270,19 @@ __global__ void __launch_bounds__(256, 1) level_bwd_kernel(const __grid_constant
     setup<256>(c, smem_raw, 7 * kTileB);
     uint8_t* sm = c.smem;   // slots: 0 Dy, 1 dC, 2 the other factor of the level above, (3, 4) and (5, 6): g and Xv[l1] of a chunk
     constexpr uint32_t colCarry = 0, colAcc = 128;
-    auto chunk_loads = [&](int chx, int buf) {   // (valid(chx) has left the chunk's source slot in `src`)
+    auto ver_row = [&](int lvl, int chx) { return is_key ? kver_row(p.vl, s, lvl, chx) : qver_row(p.vl, s, lvl, chx); };
+    auto chunk_loads = [&](int chx, int buf) {
         uint8_t* base = sm + (3 + 2 * buf) * kTileB;
         const CUtensorMap* gm = is_key ? &tm.dkv : &tm.dqv;
         const CUtensorMap* xm = is_key ? &tm.kv : &tm.qv;
-        tma_tile(base, gm, &c.bars[0], HD, (int)(((long)l2 * p.S + s) * p.Lp + (long)chx * kT));
-        tma_tile(base + kTileB, xm, &c.bars[0], HD, (int)(((long)src * p.S + s) * p.Lp + (long)chx * kT));
+        tma_tile(base, gm, &c.bars[0], HD, (int)ver_row(l2, chx));
+        tma_tile(base + kTileB, xm, &c.bars[0], HD, (int)ver_row(l1, chx));
     };
     if (c.tid == 0) {   // first group: the run product itself, the operands of the level above, the first chunk
         const uint32_t tile = kT * HD * 2;
         mbar_expect_tx(&c.bars[0], (ch >= 0 ? 3 : 0) * tile + (parent ? 2 : 0) * tile);
         if (ch >= 0) {
             tma_tile(sm, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
-            valid(ch);
             chunk_loads(ch, 0);
         }
         if (parent) {
@@ -309,8 +309,7 @@ __global__ void __launch_bounds__(256, 1) level_bwd_kernel(const __grid_constant
     bool first = true;
 #pragma unroll 1
     while (ch >= 0 && c.ok) {
-        valid(ch);   // refreshes `src` for this chunk
-        const long row_lo = ((long)src * p.S + s) * p.Lp + (long)ch * kT;
+        const long row_lo = ver_row(l1, ch);
         request(row_lo);
         const int nxt = next_chunk(ch + 1);
         loads_wait(c);
@@ -320,7 +319,6 @@ __global__ void __launch_bounds__(256, 1) level_bwd_kernel(const __grid_constant
         if (c.tid == 0 && c.ok) {
             if (nxt >= 0) {   // the other buffer's products retired before the previous mma_wait returned
                 mbar_expect_tx(&c.bars[0], 2 * kT * HD * 2);
-                valid(nxt);
                 chunk_loads(nxt, buf ^ 1);
             }
             tc_fence_after_sync();

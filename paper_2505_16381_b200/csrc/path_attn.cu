@@ -101,8 +101,10 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t c
 
 // ------------------------------------------------------------------------------------------- workspace plan
 struct Plan {
-    int S, L, Lp, N, d, nlev, nslot, gate, bwd, ragged;
+    int S, L, Lp, N, d, nlev, gate, bwd, ragged;
     LevelTable lv;
+    VerLayout vl;
+    uint64_t rows_q, rows_k;   // rows (of d elements) of the query / key version buffers
     size_t total;
     // offsets (bytes)
     size_t status, qp, kp, vp, wp, betap, G, tstats, nkeep, nvisit, Dyh, Dyl, Xqn, Yt, Qv16, Kv16;
@@ -127,7 +129,9 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
     memset(&p, 0, sizeof(p));
     p.S = (int)S; p.L = L; p.Lp = (int)Lp; p.N = (int)(Lp / CHUNK); p.d = d; p.gate = gate; p.bwd = bwd;
     p.nlev = p.N > 1 ? msb32((unsigned)(p.N - 1)) + 1 : 0;
-    p.nslot = p.nlev > 0 ? p.nlev : 1;
+    p.vl = make_ver_layout(p.S, p.N, p.Lp, p.nlev);
+    p.rows_q = (uint64_t)S * Lp + (uint64_t)S * p.vl.eq * CHUNK;
+    p.rows_k = (uint64_t)S * Lp + (uint64_t)S * p.vl.ek * CHUNK;
     p.ragged = (L != p.Lp);
     size_t cur = 0;
     const size_t SLd = (size_t)S * Lp * d, SL = (size_t)S * Lp, SNBB = (size_t)S * p.N * CHUNK * CHUNK;
@@ -164,16 +168,18 @@ static bool make_plan(int B, int H, int L, int d, int dt, int gate, int bwd, Pla
     p.dy_mats = dy_elems / ((size_t)d * d);
     p.Xqn = bump(cur, SL * CHUNK * 2);
     p.Yt = bump(cur, SL * CHUNK * 2);
-    p.Qv16 = bump(cur, SLd * 2 * p.nslot);
-    p.Kv16 = bump(cur, SLd * 2 * p.nslot);
+    p.Qv16 = bump(cur, p.rows_q * d * 2);
+    p.Kv16 = bump(cur, p.rows_k * d * 2);
     p.dy_bytes = dy_elems * 2;
     if (bwd) {
         if (p.ragged) p.dop = bump(cur, SLd * 2);
         p.delta = bump(cur, SL * 4); p.lse2 = bump(cur, SL * 4);
-        p.dQv = bump(cur, SLd * 2 * p.nslot); p.dKv = bump(cur, SLd * 2 * p.nslot);   // bf16
+        p.dQv = bump(cur, p.rows_q * d * 2); p.dKv = bump(cur, p.rows_k * d * 2);   // bf16
         p.dSd = bump(cur, gate ? SNBB * 4 : 0); p.dSdT = bump(cur, SNBB * 2); p.dG = bump(cur, SL * 4);
         p.dGrow = bump(cur, gate ? SL * 4 : 0); p.dGdiag = bump(cur, gate ? SL * 4 : 0);
-        p.dDy = bump(cur, dy_elems * 2);   // bf16, each matrix written once by the CTA that owns it
+        // bf16, each matrix written once by the CTA that owns it.  The backward never reads the run products' low planes
+        // (gradient products take single bf16 operands), so their gradients take that place.
+        p.dDy = p.Dyl;
     }
     p.total = cur;
     return true;
@@ -184,17 +190,16 @@ static T* at(void* ws, size_t off) { return reinterpret_cast<T*>((char*)ws + off
 
 static bool make_level_maps(const Plan& p, void* ws, LevelTensorMaps& tm) {
     memset(&tm, 0, sizeof(tm));
-    const uint64_t rows = (uint64_t)p.S * p.Lp * p.nslot;
     return make_map(&tm.dyh, at<void>(ws, p.Dyh), (uint64_t)p.dy_mats * p.d, p.d) &&
            make_map(&tm.dyl, at<void>(ws, p.Dyl), (uint64_t)p.dy_mats * p.d, p.d) &&
-           make_map(&tm.qv, at<void>(ws, p.Qv16), rows, p.d) && make_map(&tm.kv, at<void>(ws, p.Kv16), rows, p.d) &&
-           (!p.bwd || (make_map(&tm.dqv, at<void>(ws, p.dQv), rows, p.d) && make_map(&tm.dkv, at<void>(ws, p.dKv), rows, p.d) &&
+           make_map(&tm.qv, at<void>(ws, p.Qv16), p.rows_q, p.d) && make_map(&tm.kv, at<void>(ws, p.Kv16), p.rows_k, p.d) &&
+           (!p.bwd || (make_map(&tm.dqv, at<void>(ws, p.dQv), p.rows_q, p.d) && make_map(&tm.dkv, at<void>(ws, p.dKv), p.rows_k, p.d) &&
                        make_map(&tm.ddy, at<void>(ws, p.dDy), (uint64_t)p.dy_mats * p.d, p.d)));
 }
 
 static LevelParams level_params(const Plan& p, void* ws) {
     LevelParams lp{};
-    lp.lv = p.lv; lp.S = p.S; lp.N = p.N; lp.Lp = p.Lp; lp.nlev = p.nlev;
+    lp.lv = p.lv; lp.vl = p.vl; lp.S = p.S; lp.N = p.N; lp.Lp = p.Lp; lp.nlev = p.nlev;
     lp.dyh = at<__nv_bfloat16>(ws, p.Dyh); lp.dyl = at<__nv_bfloat16>(ws, p.Dyl);
     lp.qv = at<__nv_bfloat16>(ws, p.Qv16); lp.kv = at<__nv_bfloat16>(ws, p.Kv16);
     if (p.bwd) {
@@ -342,8 +347,8 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     BwdTensorMaps tm;
     const uint64_t rows = (uint64_t)p.S * p.Lp;
     bool ok = make_map(&tm.q_raw, q, rows, d) && make_map(&tm.k_raw, k, rows, d) && make_map(&tm.v, v, rows, d) &&
-              make_map(&tm.qv, at<void>(ws, p.Qv16), rows * p.nslot, d) &&
-              make_map(&tm.kv, at<void>(ws, p.Kv16), rows * p.nslot, d) &&
+              make_map(&tm.qv, at<void>(ws, p.Qv16), p.rows_q, d) &&
+              make_map(&tm.kv, at<void>(ws, p.Kv16), p.rows_k, d) &&
               make_map(&tm.xqn, at<void>(ws, p.Xqn), rows, CHUNK) && make_map(&tm.yt, at<void>(ws, p.Yt), rows, CHUNK) &&
               make_map(&tm.d_o, dop, rows, d);
     if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
@@ -353,7 +358,7 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     bp.G = p.gate ? at<float>(ws, p.G) : nullptr;
     bp.status = at<uint32_t>(ws, p.status);
     bp.zero_ptr = nullptr; bp.zero_bytes = 0;
-    bp.S = p.S; bp.L = p.L; bp.Lp = p.Lp; bp.N = p.N; bp.scale = scale;
+    bp.S = p.S; bp.L = p.L; bp.Lp = p.Lp; bp.N = p.N; bp.scale = scale; bp.vl = p.vl;
     if (p.gate) { bp.nkeep = at<int>(ws, p.nkeep); bp.nvisit = at<int>(ws, p.nvisit); }   // block skipping: see run_gate_skip
     prof_mark(STG_ROWSTATS, 1, st);
     prof_mark(STG_FA_DKV, 0, st);
@@ -459,15 +464,15 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
     FwdTensorMaps tm;
     const uint64_t rows = (uint64_t)p.S * p.Lp;
     bool ok = make_map(&tm.q_raw, q, rows, d) && make_map(&tm.k_raw, k, rows, d) && make_map(&tm.v, v, rows, d) &&
-              make_map(&tm.qv, at<void>(workspace, p.Qv16), rows * p.nslot, d) &&
-              make_map(&tm.kv, at<void>(workspace, p.Kv16), rows * p.nslot, d) &&
+              make_map(&tm.qv, at<void>(workspace, p.Qv16), p.rows_q, d) &&
+              make_map(&tm.kv, at<void>(workspace, p.Kv16), p.rows_k, d) &&
               make_map(&tm.xqn, at<void>(workspace, p.Xqn), rows, CHUNK) &&
               make_map(&tm.yt, at<void>(workspace, p.Yt), rows, CHUNK);
     if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
     FwdParams fp{};
     fp.o = o; fp.lse = lse; fp.G = log_f ? at<float>(workspace, p.G) : nullptr;
     fp.status = at<uint32_t>(workspace, p.status);
-    fp.S = p.S; fp.L = L; fp.Lp = p.Lp; fp.N = p.N; fp.scale = scale; fp.out_fp32 = 0;
+    fp.S = p.S; fp.L = L; fp.Lp = p.Lp; fp.N = p.N; fp.scale = scale; fp.out_fp32 = 0; fp.vl = p.vl;
     prof_mark(STG_FA_FWD, 0, st);
     if (log_f) fp.nkeep = at<int>(workspace, p.nkeep);   // block skipping: see run_gate_skip
     LAUNCH(launch_fa_fwd(tm, fp, d, st));
@@ -671,14 +676,14 @@ int path_attn_cp_prepare(const void* q, const void* k, const void* v, const void
         FwdTensorMaps tm;
         const uint64_t rows = (uint64_t)p.S * p.Lp;
         bool ok = make_map(&tm.q_raw, q, rows, d) && make_map(&tm.k_raw, k, rows, d) && make_map(&tm.v, v, rows, d) &&
-                  make_map(&tm.qv, at<void>(workspace, p.Qv16), rows * p.nslot, d) &&
-                  make_map(&tm.kv, at<void>(workspace, p.Kv16), rows * p.nslot, d) &&
+                  make_map(&tm.qv, at<void>(workspace, p.Qv16), p.rows_q, d) &&
+                  make_map(&tm.kv, at<void>(workspace, p.Kv16), p.rows_k, d) &&
                   make_map(&tm.xqn, at<void>(workspace, p.Xqn), rows, CHUNK) && make_map(&tm.yt, at<void>(workspace, p.Yt), rows, CHUNK);
         if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
         FwdParams fp{};
         fp.o = at<float>(state, c.o_acc); fp.lse = at<float>(state, c.lse_acc); fp.G = log_f ? at<float>(workspace, p.G) : nullptr;
         fp.status = at<uint32_t>(workspace, p.status);
-        fp.S = p.S; fp.L = L; fp.Lp = p.Lp; fp.N = p.N; fp.scale = scale; fp.out_fp32 = 1;
+        fp.S = p.S; fp.L = L; fp.Lp = p.Lp; fp.N = p.N; fp.scale = scale; fp.out_fp32 = 1; fp.vl = p.vl;
         if (log_f) fp.nkeep = at<int>(workspace, p.nkeep);
         LAUNCH(launch_fa_fwd(tm, fp, d, st));
     }
