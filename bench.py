@@ -630,6 +630,33 @@ def run_frontend(args):
                          "frac": gbs / peaks["hbm"], "traffic": NCU_FRONTEND_BWD_TRAFFIC_PER_BATCH_ROW * B,
                          "peak_source": f"{peaks['source']} copy bandwidth", "bytes_per_launch": byt_b},
             "detail": {"fwd_ms": ms_f, "bwd_ms": ms_b, "fwd_GBps": byt_f / (ms_f * 1e-3) / 1e9, "fwd_bytes_per_launch": byt_f}}
+    # the low-rank linear layer in front (hidden size D = H*d, rank 64): z = (x W1^T) W2^T and its backward
+    Dm, rk, C = H * d, 64, H * d
+    gl = torch.Generator(device=dev); gl.manual_seed(synth.BASE_SEED + 1)
+    xl = torch.randn(B, L, Dm, device=dev, generator=gl).bfloat16()
+    w1 = (torch.randn(rk, Dm, device=dev, generator=gl) / Dm ** 0.5).bfloat16()
+    w2 = (torch.randn(C, rk, device=dev, generator=gl) / rk ** 0.5).bfloat16()
+    zl, tl = binding.path_attn_lowrank_fwd(xl, w1, w2)
+    lws = torch.empty(int(binding.load().path_attn_lowrank_workspace_bytes(B * L, Dm, rk, C)), dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        binding.path_attn_lowrank_fwd(xl, w1, w2); binding.path_attn_lowrank_bwd(xl, w1, w2, tl, x["z"], workspace=lws)
+    la, lb, lc = ev(), ev(), ev()
+    torch.cuda.synchronize()
+    la.record()
+    for _ in range(args.steps):
+        binding.path_attn_lowrank_fwd(xl, w1, w2)
+    lb.record()
+    for _ in range(args.steps):
+        binding.path_attn_lowrank_bwd(xl, w1, w2, tl, x["z"], workspace=lws)
+    lc.record()
+    torch.cuda.synchronize()
+    lr_f, lr_b = la.elapsed_time(lb) / args.steps, lb.elapsed_time(lc) / args.steps
+    Mr = B * L
+    lr_bytes_f = Mr * (Dm + 2 * rk + C) * 2                       # x in; t out and in again; z out
+    lr_bytes_b = Mr * (2 * C + 2 * rk + rk + 2 * Dm) * 2          # dz twice, dt out and in twice, t, x, dx
+    line["detail"].update({"lowrank_fwd_ms": lr_f, "lowrank_bwd_ms": lr_b, "lowrank_fwd_GBps": lr_bytes_f / (lr_f * 1e-3) / 1e9,
+                           "lowrank_bwd_GBps": lr_bytes_b / (lr_b * 1e-3) / 1e9,
+                           "lowrank_shape": f"M={Mr} D={Dm} r={rk} C={C}"})
     if not args.no_cpu_baseline:
         from oracle import frontend_oracle as fo
         import time

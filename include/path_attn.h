@@ -229,8 +229,8 @@ int path_attn_cp_finish(const void* state, void* o, float* lse, int B, int H, in
 
 /*
  * Layer front-end: how a PaTH layer obtains the operator's w, beta and log_f (paper Sec. 2.2, footnote to the
- * definition of H_t; gate of Sec. 2.4).  The linear maps in front (the low-rank layer giving z, and u^T x + b for the
- * two logits) are plain matrix products and stay with the caller's GEMM library; these two calls are the rest:
+ * definition of H_t; gate of Sec. 2.4).  The low-rank layer giving z is path_attn_lowrank_fwd / _bwd below; the two
+ * logits u^T x + b are one matrix-vector product per head and stay with the caller; these two calls are the rest:
  *   y_t[c]  = conv_w[c][0] z_{t-2}[c] + conv_w[c][1] z_{t-1}[c] + conv_w[c][2] z_t[c]   (causal, depthwise, z = 0 before t = 0)
  *   w_t     = y_t / sqrt(sum over the head's d channels of y_t^2 + eps)               (per head)
  *   beta_t  = 2 sigmoid(beta_logit_t),      log_f_t = log sigmoid(gate_logit_t)
@@ -243,6 +243,24 @@ int path_attn_cp_finish(const void* state, void* o, float* lse, int B, int H, in
  * tensors (memory-bound), no workspace.  Same conventions as above: device pointers, outputs fully overwritten,
  * asynchronous on cuda_stream, argument errors detected on the host.
  */
+/*
+ * The low-rank linear layer in front of them (paper Sec. 2.2, same footnote: "a low-rank linear layer followed by a
+ * short convolution and L2 normalisation"), forward and backward, as tcgen05 products inside this library:
+ *     t = x W1^T  [M, r],    z = t W2^T  [M, C]              x : [M, D] bf16 (M = B*L rows of the layer's input)
+ *     dt = dz W2,  dW2 = dz^T t,  dx = dt W1,  dW1 = dt^T x    W1 : [r, D], W2 : [C, r] bf16 (nn.Linear layouts), C = H*d
+ * t, z, dx are bf16 (t is the forward's by-product the backward takes back); dW1 [r, D] and dW2 [C, r] are float32,
+ * fully overwritten, summed over the M rows with float32 atomics (reproducible to rounding).  D and C multiples of 64,
+ * r = 64 or 128.  z is what path_attn_frontend_fwd takes (viewed as [B, L, H*d]) and dz what path_attn_frontend_bwd
+ * returns.  workspace: path_attn_lowrank_workspace_bytes(M, D, r, C) bytes, 256-byte aligned (status word + dt).
+ * Same conventions as above: device pointers, asynchronous on cuda_stream, no allocation, error codes.
+ */
+size_t path_attn_lowrank_workspace_bytes(long long M, int D, int r, int C);
+int path_attn_lowrank_fwd(const void* x, const void* w1, const void* w2, void* t, void* z, long long M, int D, int r, int C,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+int path_attn_lowrank_bwd(const void* x, const void* w1, const void* w2, const void* t, const void* dz, void* dx,
+                          float* dw1, float* dw2, long long M, int D, int r, int C, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream);
+
 int path_attn_frontend_fwd(const void* z, const float* conv_w, const float* beta_logit, const float* gate_logit,
                            void* w, float* beta, float* log_f, int B, int H, int L, int d, float eps,
                            void* cuda_stream);

@@ -7,8 +7,9 @@ What it computes (paper Sec. 2.2, the footnote to the definition of H_t, and the
 gate of Sec. 2.4):
 
 * ``w_t``: the output ``z`` of a low-rank linear layer goes through a short
-  convolution of filter size 3 and an L2 normalisation.  The linear layer is a
-  plain matrix product and is not part of this module: ``z`` is its input.
+  convolution of filter size 3 and an L2 normalisation.  The linear layer is two
+  plain matrix products, ``z = (x W1^T) W2^T`` (``lowrank_fwd`` / ``lowrank_bwd``
+  at the end of this module); the front-end proper starts from ``z``.
 * ``beta_t = 2 * sigmoid(beta_logit_t)`` with ``beta_logit_t = u^T x_t + b``.
 * ``log f_t = log sigmoid(gate_logit_t)`` with ``gate_logit_t = u_f^T x_t + b_f``.
 
@@ -92,3 +93,19 @@ def frontend_bwd(z, cw, beta_logit, gate_logit, dw, dbeta, dlog_f, H: int, eps: 
         gl = np.asarray(gate_logit, np.float64)
         dgl = np.asarray(dlog_f, np.float64).transpose(0, 2, 1) * (1.0 / (1.0 + np.exp(gl)))   # d log sigmoid = sigmoid(-x)
     return dz, dcw, dbl.copy(), None if dgl is None else dgl.copy()
+
+
+def lowrank_fwd(x: np.ndarray, w1: np.ndarray, w2: np.ndarray):
+    """The low-rank linear layer in front of the convolution (paper Sec. 2.2 footnote): x [M, D], W1 [r, D], W2 [C, r]
+    (the layouts of a linear layer's weight) -> ``t = x W1^T`` [M, r] and ``z = t W2^T`` [M, C]."""
+    x, w1, w2 = (np.asarray(a, np.float64) for a in (x, w1, w2))
+    t = x @ w1.T
+    return t @ w2.T, t
+
+
+def lowrank_bwd(x: np.ndarray, w1: np.ndarray, w2: np.ndarray, dz: np.ndarray):
+    """Gradients of ``sum(z * dz)``: ``dt = dz W2``, ``dW2 = dz^T t``, ``dx = dt W1``, ``dW1 = dt^T x``."""
+    x, w1, w2, dz = (np.asarray(a, np.float64) for a in (x, w1, w2, dz))
+    t = x @ w1.T
+    dt = dz @ w2
+    return dt @ w1, dt.T @ x, dz.T @ t

@@ -21,6 +21,7 @@ EXPORTS = ["path_attn_workspace_bytes", "path_attn_fwd", "path_attn_bwd", "path_
            "path_attn_device_status", "path_attn_selftest_timeout",
            "path_attn_prefill_cache", "path_attn_decode_workspace_bytes", "path_attn_decode_step",
            "path_attn_frontend_fwd", "path_attn_frontend_bwd", "path_attn_skipped_chunk_pairs",
+           "path_attn_lowrank_workspace_bytes", "path_attn_lowrank_fwd", "path_attn_lowrank_bwd",
            "path_attn_cp_state_bytes", "path_attn_cp_message_bytes", "path_attn_cp_workspace_bytes",
            "path_attn_cp_prepare", "path_attn_cp_step", "path_attn_cp_finish",
            "path_attn_strerror", "path_attn_last_cuda_error", "path_attn_last_launch_count",
@@ -77,6 +78,13 @@ def load():
         lib.path_attn_cp_step.argtypes = [P, P, I, I, I, I, I, F, P, Z, P]
         lib.path_attn_cp_finish.restype = I
         lib.path_attn_cp_finish.argtypes = [P, P, P, I, I, I, I, P]
+        LL = ctypes.c_longlong
+        lib.path_attn_lowrank_workspace_bytes.restype = Z
+        lib.path_attn_lowrank_workspace_bytes.argtypes = [LL, I, I, I]
+        lib.path_attn_lowrank_fwd.restype = I
+        lib.path_attn_lowrank_fwd.argtypes = [P] * 5 + [LL, I, I, I, P, Z, P]
+        lib.path_attn_lowrank_bwd.restype = I
+        lib.path_attn_lowrank_bwd.argtypes = [P] * 8 + [LL, I, I, I, P, Z, P]
         lib.path_attn_skipped_chunk_pairs.restype = I
         lib.path_attn_skipped_chunk_pairs.argtypes = [P, P, ctypes.POINTER(ctypes.c_ulonglong), ctypes.POINTER(ctypes.c_ulonglong)]
         lib.path_attn_device_status.restype = I
@@ -373,6 +381,51 @@ def path_attn_frontend_bwd(z, conv_w, beta_logit, dw, dbeta, gate_logit=None, dl
     if rc != PATH_OK:
         raise PathAttnError(rc, "path_attn_frontend_bwd")
     return dz, dcw, dbl, dgl
+
+
+def _lowrank_check(x, w1, w2):
+    for t in (x, w1, w2):
+        if not (t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16):
+            raise ValueError("low-rank layer operands must be contiguous bf16 CUDA tensors")
+    M, D = x.reshape(-1, x.shape[-1]).shape
+    r, C = w1.shape[0], w2.shape[0]
+    if w1.shape != (r, D) or w2.shape != (C, r):
+        raise ValueError("w1 must be [r, D] and w2 [C, r]")
+    return M, D, r, C
+
+
+def path_attn_lowrank_fwd(x, w1, w2):
+    """``x [..., D]``, ``w1 [r, D]``, ``w2 [C, r]`` bf16 -> ``(z [..., C], t [..., r])``: ``t = x w1^T``, ``z = t w2^T``."""
+    M, D, r, C = _lowrank_check(x, w1, w2)
+    lib = load()
+    t = torch.empty(*x.shape[:-1], r, dtype=torch.bfloat16, device=x.device)
+    z = torch.empty(*x.shape[:-1], C, dtype=torch.bfloat16, device=x.device)
+    ws = torch.empty(256, dtype=torch.uint8, device=x.device)
+    st = torch.cuda.current_stream(x.device).cuda_stream
+    with torch.cuda.device(x.device):
+        rc = lib.path_attn_lowrank_fwd(_ptr(x), _ptr(w1), _ptr(w2), _ptr(t), _ptr(z), M, D, r, C, _ptr(ws), ws.numel(),
+                                       ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_lowrank_fwd")
+    return z, t
+
+
+def path_attn_lowrank_bwd(x, w1, w2, t, dz, workspace=None):
+    """Backward of :func:`path_attn_lowrank_fwd`: ``(dx bf16, dw1 float32 [r, D], dw2 float32 [C, r])``."""
+    M, D, r, C = _lowrank_check(x, w1, w2)
+    lib = load()
+    if workspace is None:
+        workspace = torch.empty(int(lib.path_attn_lowrank_workspace_bytes(M, D, r, C)), dtype=torch.uint8, device=x.device)
+    dx = torch.empty_like(x)
+    dw1 = torch.empty(r, D, dtype=torch.float32, device=x.device)
+    dw2 = torch.empty(C, r, dtype=torch.float32, device=x.device)
+    st = torch.cuda.current_stream(x.device).cuda_stream
+    with torch.cuda.device(x.device):
+        rc = lib.path_attn_lowrank_bwd(_ptr(x), _ptr(w1), _ptr(w2), _ptr(t), _ptr(dz.contiguous()), _ptr(dx), _ptr(dw1), _ptr(dw2),
+                                       M, D, r, C, _ptr(workspace), workspace.numel(), ctypes.c_void_p(st))
+    if rc != PATH_OK:
+        raise PathAttnError(rc, "path_attn_lowrank_bwd")
+    return dx, dw1, dw2
 
 
 # ----------------------------------------------------------------------------------------- context-parallel path

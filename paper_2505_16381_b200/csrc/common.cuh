@@ -16,6 +16,7 @@ enum : uint32_t {
     ST_DKV_PRODUCER = 0x201, ST_DKV_MMA = 0x202, ST_DKV_COMPUTE = 0x203,
     ST_DQ_PRODUCER = 0x301, ST_DQ_MMA = 0x302, ST_DQ_COMPUTE = 0x303,
     ST_PREP = 0x401, ST_CHAIN = 0x501, ST_LEVELS = 0x601,
+    ST_GEMM = 0x801,
     ST_STATE = 0x701,      // path_attn_bwd_reuse: the workspace does not hold the forward state of this problem
     ST_SELFTEST = 0x7f1,   // path_attn_selftest_timeout: the wait it makes run out
 };
@@ -250,5 +251,17 @@ cudaError_t launch_frontend_fwd(const void* z, const float* cw, const float* bl,
 cudaError_t launch_frontend_bwd(const void* z, const float* cw, const float* bl, const float* gl, const void* dw,
                                 const float* dbeta, const float* dlogf, void* dz, float* dcw, float* dbl, float* dgl, int B,
                                 int H, int L, int hd, float eps, cudaStream_t st);
+
+// One product C[M, N] (+)= op(A) op(B) of the low-rank layer (lowrank.cu).  a_mn / b_mn: the operand is stored as
+// [K][rows] (tensor map box 64 x 64) instead of [rows][K] (box 128 rows x 64).  c: bf16 [M][ldc] overwritten, or, with
+// c_atomic, float32 [M][ldc] added to.
+struct GemmParams {
+    int M, N, K;
+    int a_mn, b_mn;
+    void* c;
+    int ldc, c_atomic;
+    uint32_t* status;
+};
+cudaError_t launch_gemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmParams& p, int split_k, cudaStream_t st);
 
 }  // namespace path

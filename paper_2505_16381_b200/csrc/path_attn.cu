@@ -99,6 +99,19 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t c
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bf16 matrix [rows][cols], box = [box_rows][64 cols], 128-byte swizzle (the low-rank layer's operands).
+static bool make_map_box(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // ------------------------------------------------------------------------------------------- workspace plan
 struct Plan {
     int S, L, Lp, N, d, nlev, gate, bwd, ragged;
@@ -827,6 +840,83 @@ int path_attn_decode_step(const void* q_t, const void* k_t, const void* v_t, con
     LAUNCH(launch_decode_step(q_t, k_t, v_t, w_t, beta_t, log_f_t, kc, vc, gc, t, cap, o_t, lse_t, B * H, d, scale,
                               (float*)((uint8_t*)workspace + 256), st));
     return PATH_OK;
+}
+
+// ------------------------------------------------------------------------------------------- low-rank linear layer
+// C[Mo, No] (+)= op(A) op(B) with a contraction of K; an operand given as [K][rows] enters transposed (MN-major).
+static int run_gemm(const void* a, int a_mn, const void* b, int b_mn, void* c, int c_atomic, int Mo, int No, int K,
+                    uint32_t* status, cudaStream_t st) {
+    CUtensorMap ma, mb;
+    const bool ok = (a_mn ? make_map_box(&ma, a, (uint64_t)K, (uint64_t)Mo, 64) : make_map_box(&ma, a, (uint64_t)Mo, (uint64_t)K, 128)) &&
+                    (b_mn ? make_map_box(&mb, b, (uint64_t)K, (uint64_t)No, 64) : make_map_box(&mb, b, (uint64_t)No, (uint64_t)K, 128));
+    if (!ok) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+    GemmParams gp{};
+    gp.M = Mo; gp.N = No; gp.K = K; gp.a_mn = a_mn; gp.b_mn = b_mn; gp.c = c; gp.ldc = No; gp.c_atomic = c_atomic; gp.status = status;
+    int split = 1;
+    if (c_atomic) {   // weight gradients: few output tiles, a contraction over all tokens: spread it over about two waves of CTAs
+        const int tiles = ((Mo + 127) / 128) * ((No + 127) / 128), stages = (K + 63) / 64;
+        split = 296 / tiles;
+        split = split < 1 ? 1 : (split > stages ? stages : split);
+    }
+    LAUNCH(launch_gemm(ma, mb, gp, split, st));
+    return PATH_OK;
+}
+
+static bool lowrank_shape_ok(long long M, int D, int r, int C) {
+    return M >= 1 && M <= (1LL << 30) && D >= 64 && D % 64 == 0 && D <= (1 << 20) && (r == 64 || r == 128) && C >= 64 &&
+           C % 64 == 0 && C <= (1 << 20);
+}
+
+size_t path_attn_lowrank_workspace_bytes(long long M, int D, int r, int C) {
+    if (!lowrank_shape_ok(M, D, r, C)) return 0;
+    return 256 + (((size_t)M * r * 2 + 255) & ~(size_t)255);
+}
+
+int path_attn_lowrank_fwd(const void* x, const void* w1, const void* w2, void* t, void* z, long long M, int D, int r, int C,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    g_launches = 0;
+    if (!x || !w1 || !w2 || !t || !z || !workspace) return PATH_ERR_NULL;
+    if (!lowrank_shape_ok(M, D, r, C)) return PATH_ERR_SHAPE;
+    const void* ptrs[] = {x, w1, w2, t, z};
+    for (const void* q_ : ptrs)
+        if (!aligned16(q_)) return PATH_ERR_ALIGN;
+    if ((uintptr_t)workspace & 255) return PATH_ERR_ALIGN;
+    if (workspace_bytes < 256) return PATH_ERR_WORKSPACE;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    CK(cudaMemsetAsync(workspace, 0, 256, st));
+    rc = run_gemm(x, 0, w1, 0, t, 0, (int)M, r, D, (uint32_t*)workspace, st);         // t = x W1^T
+    if (rc != PATH_OK) return rc;
+    return run_gemm(t, 0, w2, 0, z, 0, (int)M, C, r, (uint32_t*)workspace, st);       // z = t W2^T
+}
+
+int path_attn_lowrank_bwd(const void* x, const void* w1, const void* w2, const void* t, const void* dz, void* dx, float* dw1,
+                          float* dw2, long long M, int D, int r, int C, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream) {
+    g_launches = 0;
+    if (!x || !w1 || !w2 || !t || !dz || !dx || !dw1 || !dw2 || !workspace) return PATH_ERR_NULL;
+    if (!lowrank_shape_ok(M, D, r, C)) return PATH_ERR_SHAPE;
+    const void* ptrs[] = {x, w1, w2, t, dz, dx, dw1, dw2};
+    for (const void* q_ : ptrs)
+        if (!aligned16(q_)) return PATH_ERR_ALIGN;
+    if ((uintptr_t)workspace & 255) return PATH_ERR_ALIGN;
+    if (workspace_bytes < path_attn_lowrank_workspace_bytes(M, D, r, C)) return PATH_ERR_WORKSPACE;
+    int rc = check_arch();
+    if (rc != PATH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    uint32_t* status = (uint32_t*)workspace;
+    void* dt = (uint8_t*)workspace + 256;
+    CK(cudaMemsetAsync(workspace, 0, 256, st));
+    CK(cudaMemsetAsync(dw1, 0, (size_t)r * D * sizeof(float), st));
+    CK(cudaMemsetAsync(dw2, 0, (size_t)C * r * sizeof(float), st));
+    rc = run_gemm(dz, 0, w2, 1, dt, 0, (int)M, r, C, status, st);                     // dt = dz W2
+    if (rc != PATH_OK) return rc;
+    rc = run_gemm(dz, 1, t, 1, dw2, 1, C, r, (int)M, status, st);                     // dW2 = dz^T t
+    if (rc != PATH_OK) return rc;
+    rc = run_gemm(dt, 0, w1, 1, dx, 0, (int)M, D, r, status, st);                     // dx = dt W1
+    if (rc != PATH_OK) return rc;
+    return run_gemm(dt, 1, x, 1, dw1, 1, r, D, (int)M, status, st);                   // dW1 = dt^T x
 }
 
 // ------------------------------------------------------------------------------------------- layer front-end

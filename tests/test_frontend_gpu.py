@@ -144,3 +144,38 @@ def test_frontend_feeds_the_operator(binding, oracle):
                                         H, eps)
     assert rel_fro(f64(dz), rz) <= 1e-2 and rel_fro(f64(dcw), rcw) <= 1e-2
     assert rel_fro(f64(dbl), rbl) <= 1e-2 and rel_fro(f64(dgl), rgl) <= 1e-2
+
+
+@pytest.mark.parametrize("B,L,D,r,C", [
+    (2, 300, 256, 64, 128),        # ragged row count, one output tile per product
+    (1, 1, 64, 64, 64),            # a single row, the smallest sizes
+    (3, 517, 1024, 128, 512),      # several tiles and stages in every direction
+    (2, 1024, 2048, 64, 2048),     # the headline layer: H = 16 heads of d = 128, hidden size 2048
+])
+def test_lowrank_layer_matches_oracle(binding, B, L, D, r, C):
+    """Forward and backward of the low-rank linear layer (paper Sec. 2.2 footnote) against float64 matrix products."""
+    g = torch.Generator().manual_seed(77 + L + D)
+    x = torch.randn(B, L, D, generator=g).bfloat16()
+    w1 = (torch.randn(r, D, generator=g) / D ** 0.5).bfloat16()
+    w2 = (torch.randn(C, r, generator=g) / r ** 0.5).bfloat16()
+    dz = torch.randn(B, L, C, generator=g).bfloat16()
+    z, t = binding.path_attn_lowrank_fwd(x.cuda(), w1.cuda(), w2.cuda())
+    z_ref, t_ref = fo.lowrank_fwd(f64(x).reshape(-1, D), f64(w1), f64(w2))
+    assert rel_fro(f64(t).reshape(-1, r), t_ref) <= 3e-3 and rel_fro(f64(z).reshape(-1, C), z_ref) <= 5e-3
+    assert close_bf16(f64(z).reshape(-1, C), z_ref)
+    dx, dw1, dw2 = binding.path_attn_lowrank_bwd(x.cuda(), w1.cuda(), w2.cuda(), t, dz.cuda())
+    rx, r1, r2 = fo.lowrank_bwd(f64(x).reshape(-1, D), f64(w1), f64(w2), f64(dz).reshape(-1, C))
+    assert rel_fro(f64(dx).reshape(-1, D), rx) <= 5e-3
+    assert rel_fro(f64(dw1), r1) <= 5e-3 and rel_fro(f64(dw2), r2) <= 5e-3      # (t and dt enter rounded to bf16)
+    dx2, dw1b, dw2b = binding.path_attn_lowrank_bwd(x.cuda(), w1.cuda(), w2.cuda(), t, dz.cuda())
+    assert torch.equal(dx, dx2)
+    for a, b_ in ((dw1, dw1b), (dw2, dw2b)):                      # float32 atomics: equal to rounding, not bitwise
+        assert (a - b_).abs().max().item() <= 1e-5 * a.abs().max().item()
+
+
+def test_lowrank_layer_argument_errors(binding):
+    x = torch.zeros(4, 96, dtype=torch.bfloat16, device="cuda")                   # D not a multiple of 64
+    with pytest.raises(binding.PathAttnError) as e:
+        binding.path_attn_lowrank_fwd(x, torch.zeros(64, 96, dtype=torch.bfloat16, device="cuda"),
+                                      torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda"))
+    assert e.value.status == -2

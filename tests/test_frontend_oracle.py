@@ -149,3 +149,22 @@ def test_backward_invariants_of_the_normalisation():
     w, _, _ = fo.frontend_fwd(z, cw, bl, None, H, 0.0)
     dz2, dcw2, _, _ = fo.frontend_bwd(z, cw, bl, None, w, np.zeros((B, H, L)), None, H, 0.0)
     assert np.abs(dz2).max() < 1e-13 and np.abs(dcw2).max() < 1e-13
+
+
+def test_lowrank_layer_is_two_library_linear_layers_and_its_backward_is_their_autograd():
+    """z = Linear_2(Linear_1(x)) without biases, against torch's own linear layers and their autograd in float64."""
+    import torch
+    rng = np.random.default_rng(21)
+    M, D, r, C = 7, 10, 3, 8
+    x, w1, w2, dz = rng.standard_normal((M, D)), rng.standard_normal((r, D)), rng.standard_normal((C, r)), rng.standard_normal((M, C))
+    z, t = fo.lowrank_fwd(x, w1, w2)
+    tx, t1, t2 = (torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in (x, w1, w2))
+    tz = torch.nn.functional.linear(torch.nn.functional.linear(tx, t1), t2)
+    assert np.abs(z - tz.detach().numpy()).max() < 1e-12
+    assert np.abs(t - (x @ w1.T)).max() < 1e-12
+    (tz * torch.tensor(dz)).sum().backward()
+    dx, dw1, dw2 = fo.lowrank_bwd(x, w1, w2, dz)
+    for got, ref in ((dx, tx.grad), (dw1, t1.grad), (dw2, t2.grad)):
+        assert np.abs(got - ref.numpy()).max() < 1e-12
+    # rank: z has at most r independent columns
+    assert np.linalg.matrix_rank(z) <= r
