@@ -47,11 +47,13 @@ UNIT = "TFLOP/s"
 # DRAM bytes per launch PER (batch, head) SLICE at the C3 shape (L=4096, d=128), from the ncu captures at batch 1
 # (16 slices) summarised under profiles/; slices are independent, so a launch over S slices moves S times this.
 NCU_TRAFFIC_BYTES_PER_SLICE = {
-    "chunk_prep": (54.62e6 + 146.33e6) / 16,        # backward instance (the step's forward runs on the shared workspace)
-    "fa_fwd": (169.10e6 + 10.06e6) / 16,
-    "fa_bwd_dkv": (187.31e6 + 122.91e6) / 16,       # includes clearing the run-product gradient buffer on the side
-    "fa_bwd_dq": (117.25e6 + 20.75e6) / 16,
-    "bwd_chunk_chain": (282.82e6 + 33.00e6) / 16,
+    "chunk_prep": 12.62e6,         # backward instance (the step's forward runs on the shared workspace)
+    "levels_fwd": 3.67e6 + 6.37e6,   # dyadic_fwd (3 launches) + version_fwd
+    "fa_fwd": 11.18e6,
+    "fa_bwd_dkv": 15.24e6,
+    "fa_bwd_dq": 8.62e6,
+    "bwd_levels": 12.62e6,         # level_bwd (4 launches)
+    "bwd_chunk_chain": 18.87e6,
 }
 
 # DRAM bytes per launch of frontend_bwd_kernel PER BATCH ROW at H=32, L=4096, d=64 with the gate, from the ncu capture at
@@ -319,7 +321,7 @@ def run_ours(args, cfg):
     if rank == 0:
         sampler.start()
     passes = [timed_pass()]
-    n_pass = int(min(40, max(3, -(-1200.0 // (passes[0][0] * args.steps)))))
+    n_pass = args.passes if args.passes > 0 else int(min(40, max(3, -(-1200.0 // (passes[0][0] * args.steps)))))
     n_pass += 1 - n_pass % 2
     while len(passes) < n_pass:
         passes.append(timed_pass())
@@ -356,9 +358,12 @@ def run_ours(args, cfg):
             res.append(e0.elapsed_time(e1) / args.steps)
         return max_over_ranks(sorted(res)[len(res) // 2], world, dev)
 
-    fwd_ms = time_fn(fwd_only)
-    fwd_stage_ms = {k_: v_ for k_, v_ in binding.profile_read().items() if k_ in ("chunk_prep", "levels_fwd", "fa_fwd")}
-    no_reuse_ms = time_fn(step_no_reuse)
+    fwd_ms = no_reuse_ms = float("nan")
+    fwd_stage_ms = {}
+    if not args.only_step:
+        fwd_ms = time_fn(fwd_only)
+        fwd_stage_ms = {k_: v_ for k_, v_ in binding.profile_read().items() if k_ in ("chunk_prep", "levels_fwd", "fa_fwd")}
+        no_reuse_ms = time_fn(step_no_reuse)
     binding.profile_enable(False)
     binding.device_status(ws_fwd)
     del ws_fwd
@@ -410,13 +415,15 @@ def run_ours(args, cfg):
         for st in (s_in, s_cmp, s_out):
             cur.wait_stream(st)
 
-    e2e_run(min(args.warmup, 3))
-    barrier()
-    e0.record()
-    e2e_run(args.steps)
-    e1.record()
-    barrier()
-    ms_e2e = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, dev)
+    ms_e2e = float("nan")
+    if not args.only_step:
+        e2e_run(min(args.warmup, 3))
+        barrier()
+        e0.record()
+        e2e_run(args.steps)
+        e1.record()
+        barrier()
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, dev)
 
     # ---- report
     f1, b1 = flops_m1(B, H, L, d)
@@ -433,6 +440,11 @@ def run_ours(args, cfg):
     prep_fl, chain_fl = chunk_kernel_flops(d)
     stage_flops = {"fa_fwd": f1 + diag, "fa_bwd_dkv": 2.0 * f1 + diag, "fa_bwd_dq": 1.5 * f1,
                    "chunk_prep": nch * prep_fl, "bwd_chunk_prep": nch * prep_fl, "bwd_chunk_chain": nch * chain_fl}
+    if cfg["gate"]:   # the sweeps execute the kept chunk pairs only: their rooflines count those
+        kept_, total_ = binding.skipped_chunk_pairs(ws)
+        pair_fl = 4.0 * CHUNK * CHUNK * d          # one S product + one P V product of a full 128 x 128 pair
+        stage_flops.update({"fa_fwd": kept_ * pair_fl, "fa_bwd_dkv": 2.0 * kept_ * pair_fl,
+                            "fa_bwd_dq": 1.5 * max(kept_ - nch, 0) * pair_fl})
     t_d, t_b = CHUNK * d * 2, CHUNK * CHUNK * 2                 # bytes of a [128 x d] / [128 x 128] bf16 tile
     prep_bytes = nch * (3 * t_d + 2 * t_d + 2 * t_b + 2 * d * d * 2)
     lev_f, lev_b = level_bytes(S, N, d)
@@ -442,6 +454,9 @@ def run_ours(args, cfg):
     stage_bytes = {"chunk_prep": prep_bytes + nch * (5 * t_b + t_d), "bwd_chunk_prep": prep_bytes + nch * (5 * t_b + t_d),
                    "bwd_chunk_chain": nch * (4 * t_d + 7 * t_b + t_b + 2 * t_d + d * d * 2 + 3 * t_d),
                    "levels_fwd": lev_f, "bwd_levels": lev_b, "bwd_levels_fwd": lev_f}
+    if cfg["gate"]:   # version chains are built only up to the levels the kept pairs use: no closed-form byte count
+        for k_ in ("levels_fwd", "bwd_levels", "bwd_levels_fwd"):
+            stage_bytes.pop(k_)
 
     def ncu_traffic(kernel):
         per_slice = NCU_TRAFFIC_BYTES_PER_SLICE.get(kernel)
@@ -681,6 +696,10 @@ def main():
     ap.add_argument("--workload", default="C3", choices=[n for n, c in synth.CONFIGS.items() if c["backward"]])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling captures)")
+    ap.add_argument("--only-step", action="store_true",
+                    help="time the fwd+bwd step only: no forward-only / no-reuse / end-to-end arms (profiling captures)")
+    ap.add_argument("--passes", type=int, default=0,
+                    help="number of timed passes of --steps steps (default: as many as keep the GPU busy for > 1 s; profiling captures pass 1)")
     ap.add_argument("--path", choices=["train", "decode", "frontend"], default="train",
                     help="train: the fwd+bwd step (the headline); decode: the inference arm; frontend: the layer front-end "
                          "kernels (both 1 GPU, not part of the headline)")

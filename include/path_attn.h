@@ -91,8 +91,8 @@ int path_attn_fwd(const void* q, const void* k, const void* v, const void* w, co
  *   d_o     : [B,H,L,d] in dt
  *   dq,dk,dv,dw : [B,H,L,d] in dt (out)   dbeta : [B,H,L] float32 (out)
  *   dlog_f  : [B,H,L] float32 (out); must be NULL exactly when log_f is NULL
- * dt must be PATH_BF16.  Uses float32 atomics: results are reproducible to
- * rounding, not bitwise.
+ * dt must be PATH_BF16.  Bitwise reproducible from run to run, like the forward
+ * (nothing on this path is accumulated atomically).
  *
  * path_attn_bwd always recomputes the chunk preparation (Sec. 3.1 / 3.3
  * quantities) from q, k, w, beta, log_f: it depends on nothing a previous call

@@ -223,8 +223,6 @@ struct BwdParams {
     const float* G;      // [S][Lp] gate prefix or nullptr
     const int* nkeep;    // [S][N] key chunks a query chunk has to visit / nvisit: query chunks a key chunk has to meet
     const int* nvisit;   //        (block skipping in gated problems), or nullptr = all
-    void* zero_ptr;      // dK/dV sweep: buffer it clears on the side (32-byte aligned, zero_bytes % 32 == 0), or zero_bytes = 0
-    size_t zero_bytes;
     uint32_t* status;
     int S, L, Lp, N;
     float scale;

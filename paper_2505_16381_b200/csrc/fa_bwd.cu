@@ -331,24 +331,6 @@ __global__ void __launch_bounds__(384, 1) dkv_kernel(const __grid_constant__ Bwd
                 }
                 g += T; qb += T + 1; db += T + 1;
             }
-        } else if (warp >= 2) {
-            // The two spare warps clear this CTA's share of the run-product gradient buffer, which later kernels
-            // accumulate into: the sweep leaves most of the memory bandwidth unused.
-            const uint32_t n32 = (uint32_t)(p.zero_bytes / 32), per = (n32 + gridDim.x - 1) / gridDim.x;   // < 2^32 pieces of 32 bytes
-            const uint32_t lo = blockIdx.x * per, hi = lo + per < n32 ? lo + per : n32;
-            // Paced, so that the sweep's own stores are not delayed, but never so slowly that the CTA would outlast its
-            // sweep: the clearing is spread over about half of the sweep's expected duration (a chunk pair takes about
-            // 2 us here; the items of a slice average (N + 1) / 2 pairs).  A sweep shortened by block skipping has no
-            // such estimate: there the clearing runs at full speed.
-            const uint32_t iters = (hi > lo ? hi - lo : 0u) / 64u + 1u;
-            const float sweep_ns = (float)items / (float)gridDim.x * 0.5f * (float)(p.N + 1) * 2000.f;
-            const float gap_ns = 0.5f * sweep_ns / (float)iters - 100.f;   // 100 ns: what a store costs anyway
-            const unsigned sleep_ns = p.nvisit != nullptr || gap_ns < 20.f ? 0u : (unsigned)fminf(gap_ns, 1000.f);
-            for (uint32_t i = lo + (threadIdx.x - 64); i < hi; i += 64) {
-                asm volatile("st.global.v8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"l"((uint8_t*)p.zero_ptr + (size_t)i * 32), "r"(0u)
-                             : "memory");
-                if (sleep_ns) __nanosleep(sleep_ns);
-            }
         }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");

@@ -370,7 +370,6 @@ static int run_backward(const Plan& p, void* ws, const void* q, const void* k, c
     bp.lse2 = at<float>(ws, p.lse2); bp.delta = at<float>(ws, p.delta);
     bp.G = p.gate ? at<float>(ws, p.G) : nullptr;
     bp.status = at<uint32_t>(ws, p.status);
-    bp.zero_ptr = nullptr; bp.zero_bytes = 0;
     bp.S = p.S; bp.L = p.L; bp.Lp = p.Lp; bp.N = p.N; bp.scale = scale; bp.vl = p.vl;
     if (p.gate) { bp.nkeep = at<int>(ws, p.nkeep); bp.nvisit = at<int>(ws, p.nvisit); }   // block skipping: see run_gate_skip
     prof_mark(STG_ROWSTATS, 1, st);
