@@ -28,19 +28,58 @@ def to_dev(inp):
     return {k: (v.cuda() if torch.is_tensor(v) else v) for k, v in inp.items()}
 
 
+GUARD = 4096    # bytes of guard band on either side of every buffer a call may write
+
+
+class Guarded:
+    """A device buffer with a guard band on either side, filled with a pattern: with compute-sanitizer closed on the test
+    machines, a store that leaves its buffer is caught here (`check()` after the call) instead of by luck."""
+
+    def __init__(self, shape, dtype, device, fill=0xFF):
+        n = int(np.prod(shape)) * torch.empty(0, dtype=dtype).element_size()
+        pad = (-n) % 256
+        self.raw = torch.empty(GUARD + n + pad + GUARD, dtype=torch.uint8, device=device)
+        self.raw.fill_(0x5A)
+        body = self.raw[GUARD:GUARD + n]
+        body.fill_(fill)             # NaN patterns: whatever a call leaves unwritten shows
+        self.t = body.view(dtype).view(*shape)
+        assert self.t.data_ptr() % 256 == 0
+
+    def check(self, what):
+        lo, hi = self.raw[:GUARD], self.raw[self.raw.numel() - GUARD:]
+        assert bool((lo == 0x5A).all()) and bool((hi == 0x5A).all()), f"{what}: a store left its buffer"
+
+
 def gpu_forward(b, dev, scale):
-    ws = b.alloc_workspace(dev["q"], dev["log_f"] is not None, False)
-    o, lse = b.path_attn_fwd(dev["q"], dev["k"], dev["v"], dev["w"], dev["beta"], dev["log_f"], scale=scale, workspace=ws)
-    assert b.device_status(ws) == 0
-    return o, lse
+    q = dev["q"]
+    B, H, L, d = q.shape
+    ws = Guarded((b.workspace_bytes(B, H, L, d, b.PATH_BF16 if q.dtype == torch.bfloat16 else b.PATH_FP32,
+                                    dev["log_f"] is not None, False),), torch.uint8, q.device)
+    o, lse = Guarded(q.shape, q.dtype, q.device), Guarded((B, H, L), torch.float32, q.device)
+    b.path_attn_fwd(q, dev["k"], dev["v"], dev["w"], dev["beta"], dev["log_f"], scale=scale, workspace=ws.t, out=(o.t, lse.t))
+    assert b.device_status(ws.t) == 0
+    for g_, name in ((ws, "workspace"), (o, "o"), (lse, "lse")):
+        g_.check("path_attn_fwd " + name)
+    return o.t, lse.t
 
 
 def gpu_backward(b, dev, o, lse, scale):
-    ws = b.alloc_workspace(dev["q"], dev["log_f"] is not None, True)
-    ws.fill_(0xFF)      # (NaN patterns) whatever an earlier problem left at these addresses must not matter: the backward recomputes
-    g = b.path_attn_bwd(dev["q"], dev["k"], dev["v"], dev["w"], dev["beta"], o, lse, dev["d_o"], dev["log_f"],
-                        scale=scale, workspace=ws)
-    assert b.device_status(ws) == 0
+    """Plain backward on a workspace full of NaN patterns (whatever an earlier problem left at these addresses must not
+    matter: the backward recomputes), every output in a guarded buffer."""
+    q = dev["q"]
+    B, H, L, d = q.shape
+    gate = dev["log_f"] is not None
+    ws = Guarded((b.workspace_bytes(B, H, L, d, b.PATH_BF16, gate, True),), torch.uint8, q.device)
+    out = {n: Guarded(q.shape, q.dtype, q.device) for n in ("dq", "dk", "dv", "dw")}
+    out["dbeta"] = Guarded((B, H, L), torch.float32, q.device)
+    if gate:
+        out["dlog_f"] = Guarded((B, H, L), torch.float32, q.device)
+    g = b.path_attn_bwd(q, dev["k"], dev["v"], dev["w"], dev["beta"], o, lse, dev["d_o"], dev["log_f"],
+                        scale=scale, workspace=ws.t, out={n: x.t for n, x in out.items()})
+    assert b.device_status(ws.t) == 0
+    ws.check("path_attn_bwd workspace")
+    for n, x in out.items():
+        x.check("path_attn_bwd " + n)
     return g
 
 
