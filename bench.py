@@ -561,13 +561,18 @@ def run_decode(args):
     cache = binding.alloc_cache(B, H, L + n_tok, d, False, dev)
     ws = binding.alloc_workspace(k, False, False)
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    binding.path_attn_prefill_cache(k, v, w, beta, cache, workspace=ws)
+    for _ in range(3):
+        binding.path_attn_prefill_cache(k, v, w, beta, cache, workspace=ws)
     torch.cuda.synchronize()
-    p0, p1 = ev(), ev()
-    p0.record()
-    binding.path_attn_prefill_cache(k, v, w, beta, cache, workspace=ws)
-    p1.record()
-    torch.cuda.synchronize()
+    prefill_ms = []
+    for _ in range(5):       # (one call moves 1.4 GB: more than L2, no flush needed)
+        p0, p1 = ev(), ev()
+        p0.record()
+        binding.path_attn_prefill_cache(k, v, w, beta, cache, workspace=ws)
+        p1.record()
+        torch.cuda.synchronize()
+        prefill_ms.append(p0.elapsed_time(p1))
+    prefill_ms = sorted(prefill_ms)[2]
     assert binding.device_status(ws) == 0
     tok = [(rn(B, H, d) / d ** 0.5).bfloat16() for _ in range(2)] + [rn(B, H, d).bfloat16()]
     wt = rn(B, H, d); wt = (wt / wt.norm(dim=-1, keepdim=True)).bfloat16(); bt = 2 * torch.sigmoid(rn(B, H))
@@ -599,7 +604,7 @@ def run_decode(args):
             "roofline": {"kernel": "decode_update_kernel", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
                          "frac": gbs / peaks["hbm"], "traffic": None, "peak_source": f"{peaks['source']} copy bandwidth",
                          "bytes_per_launch": byt},
-            "detail": {"prefill_cache_ms": p0.elapsed_time(p1), "prefill_tokens": B * L}}
+            "detail": {"prefill_cache_ms": prefill_ms, "prefill_tokens": B * L}}
     print(json.dumps(line), flush=True)
 
 

@@ -68,9 +68,13 @@ __device__ __forceinline__ bool wsync_and(bool ok) {   // barrier over the worke
     return r != 0;
 }
 
-template <int HD, bool SAVE>
+// MODE: PREP_FWD = everything the forward needs; PREP_SAVE = also keeps the tiles of the chain rule (the backward's instance);
+// PREP_KEYS = the key side only (prompt key cache: Kright and the chunk products; no query is involved, so Xq, Xq U,
+// Qleft and the diagonal-correction operands are left out and q is not even loaded).
+template <int HD, int MODE>
 __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_constant__ PrepTensorMaps tm, const PrepParams p,
                                                                       const int nchunks) {
+    constexpr bool SAVE = MODE == PREP_SAVE, KEYS = MODE == PREP_KEYS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sW = smem + PrepSmem::offW;
@@ -113,10 +117,10 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
         if (tid == kWorkers) {
             auto wait = [&](int b, uint32_t par) { return mbar_wait(&bars[b], par, abort_flag, ST_PREP); };
             auto load = [&](int chunk) {
-                mbar_expect_tx(&bars[B_LOAD], 3 * kT * HD * 2);
+                mbar_expect_tx(&bars[B_LOAD], (KEYS ? 2 : 3) * kT * HD * 2);
                 for (int h = 0; h < HD / 64; ++h) {
                     tma_load_2d(sW + h * kPanelB, &tm.w, &bars[B_LOAD], h * 64, chunk * kT);
-                    tma_load_2d(sQK + h * kPanelB, &tm.q, &bars[B_LOAD], h * 64, chunk * kT);
+                    if (!KEYS) tma_load_2d(sQK + h * kPanelB, &tm.q, &bars[B_LOAD], h * 64, chunk * kT);
                     tma_load_2d(sQK + kTileB + h * kPanelB, &tm.k, &bars[B_LOAD], h * 64, chunk * kT);
                 }
             };
@@ -143,7 +147,7 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 // Xq, Xk: their columns held the previous chunk's W^T U and Xq U
                 if (it > 0 && !wait(R_E3, par ^ 1)) break;
                 tc_fence_after_sync();
-                mma_small(tmem + 128, aQ, OP_K, aW, OP_K, KS, 128, false);
+                if (!KEYS) mma_small(tmem + 128, aQ, OP_K, aW, OP_K, KS, 128, false);
                 mma_small(tmem + 256, aW, OP_K, aK, OP_K, KS, 128, false);
                 umma_commit(&bars[B_XQK]);
                 // U = T~ W  (lo x lo terms are dropped everywhere)
@@ -171,9 +175,11 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 // Xq U and W^T U
                 if (!wait(R_U, par)) break;
                 tc_fence_after_sync();
-                mma_small(tmem + 256, aBig, OP_K, aQ, OP_MN, 8, HD, false);
-                mma_small(tmem + 256, aBig + kTileB, OP_K, aQ, OP_MN, 8, HD, true);
-                mma_small(tmem + 256, aBig, OP_K, aK, OP_MN, 8, HD, true);
+                if (!KEYS) {
+                    mma_small(tmem + 256, aBig, OP_K, aQ, OP_MN, 8, HD, false);
+                    mma_small(tmem + 256, aBig + kTileB, OP_K, aQ, OP_MN, 8, HD, true);
+                    mma_small(tmem + 256, aBig, OP_K, aK, OP_MN, 8, HD, true);
+                }
                 mma_small(tmem + 128, aW, OP_MN, aQ, OP_MN, 8, HD, false);
                 mma_small(tmem + 128, aW, OP_MN, aK, OP_MN, 8, HD, true);
                 umma_commit(&bars[B_G3A]);
@@ -355,7 +361,7 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars[R_XK]);
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < (KEYS ? 0 : 2); ++c) {
                 const int c0 = half * 64 + c * 32;
                 tmem_ld32(tl + 128 + c0, r);
                 tmem_ld_wait();
@@ -401,11 +407,13 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 split32(v, hi, lo);
                 tile_store_w16(sBig + 2 * kTileB, row, c0, hi);
                 tile_store_w16(sBig + 3 * kTileB, row, c0, lo);
-                unsigned short* yt = reinterpret_cast<unsigned short*>(p.Yt) + ((size_t)chunk * kT + c0) * kT + row;
+                if (!KEYS) {
+                    unsigned short* yt = reinterpret_cast<unsigned short*>(p.Yt) + ((size_t)chunk * kT + c0) * kT + row;
 #pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    yt[(size_t)(2 * x) * kT] = (unsigned short)(hi[x] & 0xffffu);
-                    yt[(size_t)(2 * x + 1) * kT] = (unsigned short)(hi[x] >> 16);
+                    for (int x = 0; x < 16; ++x) {
+                        yt[(size_t)(2 * x) * kT] = (unsigned short)(hi[x] & 0xffffu);
+                        yt[(size_t)(2 * x + 1) * kT] = (unsigned short)(hi[x] >> 16);
+                    }
                 }
             }
             fence_proxy_async_smem();
@@ -420,7 +428,7 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 const int c0 = half * (HD / 2) + c * 32;
 #pragma unroll
                 for (int x = 0; x < 4; ++x) {
-                    pre_q[c][x] = reinterpret_cast<const uint4*>(p.q + grow * HD + c0)[x];
+                    if (!KEYS) pre_q[c][x] = reinterpret_cast<const uint4*>(p.q + grow * HD + c0)[x];
                     pre_k[c][x] = reinterpret_cast<const uint4*>(p.k + grow * HD + c0)[x];
                 }
             }
@@ -431,13 +439,15 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
 #pragma unroll
             for (int c = 0; c < HD / 64; ++c) {
                 const int c0 = half * (HD / 2) + c * 32;
-                float in[32];
-                tmem_ld32(tl + 256 + c0, r);
-                tmem_ld_wait();
-                unpack_bf16x32(pre_q[c], in);
+                if (!KEYS) {
+                    float in[32];
+                    tmem_ld32(tl + 256 + c0, r);
+                    tmem_ld_wait();
+                    unpack_bf16x32(pre_q[c], in);
 #pragma unroll
-                for (int x = 0; x < 32; ++x) v[x] = in[x] - __uint_as_float(r[x]);
-                gstore_bf16x32(p.ql + grow * HD + c0, v);
+                    for (int x = 0; x < 32; ++x) v[x] = in[x] - __uint_as_float(r[x]);
+                    gstore_bf16x32(p.ql + grow * HD + c0, v);
+                }
                 tmem_ld32(tl + 128 + c0, r);
                 tmem_ld_wait();
 #pragma unroll
@@ -489,8 +499,9 @@ cudaError_t launch_chunk_prep(const PrepTensorMaps& tm, const PrepParams& p, int
         kern<<<grid, kThreads, PrepSmem::alloc, st>>>(tm, p, nchunks);
         return cudaGetLastError();
     };
-    if (hd == 64) return save ? go(chunk_prep_kernel<64, true>) : go(chunk_prep_kernel<64, false>);
-    return save ? go(chunk_prep_kernel<128, true>) : go(chunk_prep_kernel<128, false>);
+    if (save == PREP_KEYS) return hd == 64 ? go(chunk_prep_kernel<64, PREP_KEYS>) : go(chunk_prep_kernel<128, PREP_KEYS>);
+    if (hd == 64) return save ? go(chunk_prep_kernel<64, PREP_SAVE>) : go(chunk_prep_kernel<64, PREP_FWD>);
+    return save ? go(chunk_prep_kernel<128, PREP_SAVE>) : go(chunk_prep_kernel<128, PREP_FWD>);
 }
 
 }  // namespace path

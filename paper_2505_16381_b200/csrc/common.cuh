@@ -150,14 +150,16 @@ struct LevelParams {
     float* kc;                    // edge kernels: [S][cap][d] float32 out (rows < L of every slice), or nullptr
     int cap, L;
     __nv_bfloat16* edge16;        // edge kernels: [S][L][d] bf16 out, or nullptr
-    __nv_bfloat16* pseg;          // query-edge kernel: [S][2][d][d] product of the whole segment as bf16 hi, lo; or nullptr
+    __nv_bfloat16* pseg;          // edge kernels: [S][nseg][2][d][d] product of the walked range as bf16 hi, lo; or nullptr
+    __nv_bfloat16* sfx;           // suffix kernel: [S][nseg][2][d][d] out
+    int nseg, seg_chunks;         // key-side edge / suffix / apply-product kernels: ranges per slice (<= 1: none), chunks per range
     float* gq;                    // apply-product kernel: [S][Lp] gate terms of the rows (+= gtot[slice]), or nullptr
     const float* gtot;            // [S]
     const int *nkeep, *nvisit;    // version backward: chunk counts of a sweep shortened by block skipping ([S][N]), or nullptr
     uint32_t* status;
 };
 
-enum { LEVEL_DYADIC_FWD = 0, LEVEL_VERSION_FWD, LEVEL_BWD, LEVEL_KEY_CACHE, LEVEL_QUERY_EDGE, LEVEL_APPLY_PRODUCT };
+enum { LEVEL_DYADIC_FWD = 0, LEVEL_VERSION_FWD, LEVEL_BWD, LEVEL_KEY_CACHE, LEVEL_QUERY_EDGE, LEVEL_SUFFIX, LEVEL_APPLY_PRODUCT };
 cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const LevelParams& p, int hd, cudaStream_t st);
 
 struct PrepTensorMaps {
@@ -181,7 +183,9 @@ struct PrepParams {
     uint32_t* status;
 };
 
-cudaError_t launch_chunk_prep(const PrepTensorMaps& tm, const PrepParams& p, int hd, int save, int nchunks,
+// `mode`: what the kernel produces (see chunk_prep.cu).
+enum { PREP_FWD = 0, PREP_SAVE = 1, PREP_KEYS = 2 };
+cudaError_t launch_chunk_prep(const PrepTensorMaps& tm, const PrepParams& p, int hd, int mode, int nchunks,
                               cudaStream_t st);
 
 struct ChainTensorMaps {

@@ -412,12 +412,20 @@ __global__ void __launch_bounds__(256, 1) key_cache_kernel(const __grid_constant
         tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)(mat * HD));
         tma_tile(sm + 2 * kTileB, &tm.dyl, &c.bars[0], HD, (int)(mat * HD));
     };
-    const int first = QUERY ? 0 : p.N - 1, step = QUERY ? 1 : -1;
+    // Segments (key side, p.nseg > 1): blockIdx.z walks only the chunks [z * seg_chunks, (z+1) * seg_chunks) and leaves its keys
+    // advanced to the end of THAT range (bf16, p.edge16) together with the range's product (p.pseg); a second pass
+    // (suffix_kernel, apply_product_kernel) carries them on to the end of the sequence.  The walk itself is a serial
+    // chain of dependent products, so this is what lets a long prompt use all SMs.
+    const int c_lo = p.nseg > 1 ? (int)blockIdx.z * p.seg_chunks : 0;
+    const int c_hi = p.nseg > 1 ? min(p.N, c_lo + p.seg_chunks) : p.N, cnt = c_hi - c_lo;
+    const int first = QUERY ? c_lo : c_hi - 1, step = QUERY ? 1 : -1;
+    if (cnt <= 0) { teardown<256>(c, p.status); return; }
     if (c.tid == 0) issue(first);
 #pragma unroll 1
-    for (int n = 0, J = first; n < p.N && c.ok; ++n, J += step) {
-        const bool more = n + 1 < p.N;
-        const bool update = QUERY || more;         // the query side also wants the product of the whole segment
+    for (int n = 0, J = first; n < cnt && c.ok; ++n, J += step) {
+        const bool more = n + 1 < cnt;
+        // the query side also wants the product of the whole segment; so does every key range but the first
+        const bool update = QUERY || more || (p.nseg > 1 && blockIdx.z > 0);
         loads_wait(c);
         publish();
         if (c.tid == 0 && c.ok) {
@@ -449,19 +457,90 @@ __global__ void __launch_bounds__(256, 1) key_cache_kernel(const __grid_constant
                 tile_store_w16(sm + 3 * kTileB, c.row, c0, hi);
                 tile_store_w16(sm + 4 * kTileB, c.row, c0, lo);
             }
-            if (QUERY && !more && p.pseg) {   // the segment's product, [S][2 (hi, lo)][d][d]
-                gstore_bf16_w16(p.pseg + (((size_t)s * 2 + 0) * HD + c.row) * HD + col0 + c0, hi, c.row < HD);
-                gstore_bf16_w16(p.pseg + (((size_t)s * 2 + 1) * HD + c.row) * HD + col0 + c0, lo, c.row < HD);
+            if (!more && p.pseg) {   // the range's product, [S][nseg][2 (hi, lo)][d][d]
+                const size_t mi = (size_t)s * (p.nseg > 1 ? p.nseg : 1) + (p.nseg > 1 ? blockIdx.z : 0);
+                gstore_bf16_w16(p.pseg + ((mi * 2 + 0) * HD + c.row) * HD + col0 + c0, hi, c.row < HD);
+                gstore_bf16_w16(p.pseg + ((mi * 2 + 1) * HD + c.row) * HD + col0 + c0, lo, c.row < HD);
             }
         }
     }
     teardown<256>(c, p.status);
 }
 
-// ---------------------------------------------------------------------------------------------- segment product applied to a tile
-// grid = S * N.  x <- x M  for every 128-row tile of x ([S][Lp][d] bf16, in place), with one matrix M = hi + lo per slice
-// ([S][2][d][d] bf16): the update of the query state after a key segment has been attended (paper Sec. 3.5).  The
-// gate term of the rows moves on as well: gq[row] += gtot[slice].
+// ---------------------------------------------------------------------------------------------- products of key ranges towards the end
+// grid = (S, d / 64).  With M_g = the product of key range g (p.pseg, [S][nseg][2][d][d]):  Sfx_{nseg-1} = I,
+// Sfx_g = M_{g+1} Sfx_{g+1}  (p.sfx, same layout): what a key advanced to the end of range g still has to be multiplied
+// by to reach the end of the sequence.  nseg - 1 dependent products of 64 columns each.
+template <int HD>
+__global__ void __launch_bounds__(256, 1) suffix_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    Ctx c;
+    setup<128>(c, smem_raw, kBar4);
+    constexpr int NC = 64;
+    const int s = blockIdx.x, col0 = blockIdx.y * NC, c0 = c.half * 32;
+    uint8_t* sm = c.smem;   // slots: 0 M hi, 1 M lo, 2 R hi, 3 R lo
+    for (int i = c.tid; i < (int)(4 * kTileB / 16); i += 256) reinterpret_cast<uint4*>(sm)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    if (c.tid < NC) {
+        const uint32_t r = (uint32_t)(col0 + c.tid), j = (uint32_t)c.tid;
+        *reinterpret_cast<__nv_bfloat16*>(sm + 2 * kTileB + sw128_off(r, j >> 3) + (j & 7) * 2) = __float2bfloat16_rn(1.f);
+    }
+    auto store = [&](int g, const uint32_t (&hi)[16], const uint32_t (&lo)[16]) {
+        const size_t mi = (size_t)s * p.nseg + g;
+        gstore_bf16_w16(p.sfx + ((mi * 2 + 0) * HD + c.row) * HD + col0 + c0, hi, c.row < HD);
+        gstore_bf16_w16(p.sfx + ((mi * 2 + 1) * HD + c.row) * HD + col0 + c0, lo, c.row < HD);
+    };
+    {   // Sfx of the last range: the identity
+        uint32_t hi[16], lo[16];
+#pragma unroll
+        for (int x = 0; x < 16; ++x) {
+            const int col = col0 + c0 + 2 * x;
+            hi[x] = (col == c.row ? 0x3f80u : 0u) | (col + 1 == c.row ? 0x3f800000u : 0u);
+            lo[x] = 0u;
+        }
+        store(p.nseg - 1, hi, lo);
+    }
+    fence_proxy_async_smem();
+    __syncthreads();
+#pragma unroll 1
+    for (int g = p.nseg - 1; g >= 1 && c.ok; --g) {
+        if (c.tid == 0) {
+            const long mrow = ((long)s * p.nseg + g) * 2 * HD;
+            mbar_expect_tx(&c.bars[0], 2 * kT * HD * 2);
+            tma_tile(sm, &tm.dyh, &c.bars[0], HD, (int)mrow);
+            tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)(mrow + HD));
+        }
+        loads_wait(c);
+        publish();
+        if (c.tid == 0 && c.ok) {
+            tc_fence_after_sync();
+            const uint32_t a = smem_u32(sm);
+            mma(c.tmem, a, OP_K, a + 2 * kTileB, OP_MN, HD / 16, NC, false);       // M R
+            mma(c.tmem, a + kTileB, OP_K, a + 2 * kTileB, OP_MN, HD / 16, NC, true);
+            mma(c.tmem, a, OP_K, a + 3 * kTileB, OP_MN, HD / 16, NC, true);
+            umma_commit(&c.bars[1]);
+        }
+        mma_wait(c);
+        if (!c.ok) break;
+        float v[32];
+        uint32_t hi[16], lo[16];
+        tmem_row32(c.tl + c0, v);
+        split32(v, hi, lo);
+        if (c.row < HD) {
+            tile_store_w16(sm + 2 * kTileB, c.row, c0, hi);
+            tile_store_w16(sm + 3 * kTileB, c.row, c0, lo);
+        }
+        store(g - 1, hi, lo);
+    }
+    teardown<128>(c, p.status);
+}
+
+// ---------------------------------------------------------------------------------------------- a product applied to row tiles
+// grid = S * N.  x M  for every 128-row tile of x ([S][Lp][d] bf16), with M = hi + lo from [S][nseg][2][d][d] bf16 (tm.dyh):
+// the matrix of the tile's slice and, with nseg > 1, of the range of seg_chunks chunks the tile lies in.  The result
+// replaces x (bf16, p.qv: the query state of the context-parallel path after a key segment has been attended, paper
+// Sec. 3.5; the gate terms of the rows move on as well: gq[row] += gtot[slice]) or goes to a float32 matrix
+// (p.kc, [S][cap][d]: the prompt's key cache, second pass).
 template <int HD>
 __global__ void __launch_bounds__(256, 2) apply_product_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -470,11 +549,12 @@ __global__ void __launch_bounds__(256, 2) apply_product_kernel(const __grid_cons
     const int s = blockIdx.x / p.N, ch = blockIdx.x % p.N;
     uint8_t* sm = c.smem;   // slots: 0 x tile, 1 M hi, 2 M lo
     const long row0 = (long)s * p.Lp + (long)ch * kT;
+    const long mi = p.nseg > 1 ? (long)s * p.nseg + ch / p.seg_chunks : (long)s;
     if (c.tid == 0) {
         mbar_expect_tx(&c.bars[0], 3 * kT * HD * 2);
         tma_tile(sm, &tm.qv, &c.bars[0], HD, (int)row0);
-        tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)((long)(2 * s) * HD));
-        tma_tile(sm + 2 * kTileB, &tm.dyh, &c.bars[0], HD, (int)((long)(2 * s + 1) * HD));
+        tma_tile(sm + kTileB, &tm.dyh, &c.bars[0], HD, (int)(2 * mi * HD));
+        tma_tile(sm + 2 * kTileB, &tm.dyh, &c.bars[0], HD, (int)((2 * mi + 1) * HD));
     }
     if (p.gq && c.tid < kT) p.gq[row0 + c.tid] += p.gtot[s];
     loads_wait(c);
@@ -488,10 +568,12 @@ __global__ void __launch_bounds__(256, 2) apply_product_kernel(const __grid_cons
     mma_wait(c);
     if (c.ok) {
         float v[32];
+        const int pos = ch * kT + c.row;
         for (int i = 0; i < HD / 64; ++i) {
             const int c0 = c.half * (HD / 2) + i * 32;
             tmem_row32(c.tl + c0, v);
-            gstore_bf16x32(p.qv + ((size_t)row0 + c.row) * HD + c0, v);
+            if (p.kc) gstore_f32x32(p.kc + ((size_t)s * p.cap + pos) * HD + c0, v, pos < p.L);
+            else gstore_bf16x32(p.qv + ((size_t)row0 + c.row) * HD + c0, v);
         }
     }
     teardown<128>(c, p.status);
@@ -523,12 +605,16 @@ cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const Leve
             return hd == 64 ? launch(level_bwd_kernel<64>, g, 7, tm, p, st) : launch(level_bwd_kernel<128>, g, 7, tm, p, st);
         }
         case LEVEL_KEY_CACHE: {
-            dim3 g(p.S, hd / 64);
+            dim3 g(p.S, hd / 64, p.nseg > 1 ? p.nseg : 1);
             return hd == 64 ? launch(key_cache_kernel<64, false>, g, 5, tm, p, st) : launch(key_cache_kernel<128, false>, g, 5, tm, p, st);
         }
         case LEVEL_QUERY_EDGE: {
             dim3 g(p.S, hd / 64);
             return hd == 64 ? launch(key_cache_kernel<64, true>, g, 5, tm, p, st) : launch(key_cache_kernel<128, true>, g, 5, tm, p, st);
+        }
+        case LEVEL_SUFFIX: {
+            dim3 g(p.S, hd / 64);
+            return hd == 64 ? launch(suffix_kernel<64>, g, 4, tm, p, st) : launch(suffix_kernel<128>, g, 4, tm, p, st);
         }
         case LEVEL_APPLY_PRODUCT: {
             dim3 g(p.S * p.N);

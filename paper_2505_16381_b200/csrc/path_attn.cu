@@ -236,7 +236,7 @@ static int run_gate_skip(const Plan& p, void* ws, const void* q, const void* k, 
 
 // Chunk preparation + dyadic run products + version chains (paper Sec. 3.1, 3.3).  Shared by forward and backward.
 static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const void* w, bool in_backward,
-                    cudaStream_t st, bool with_levels = true) {
+                    cudaStream_t st, bool with_levels = true, bool keys_only = false) {
     const int d = p.d, nch = p.S * p.N;
     const int stg_prep = in_backward ? STG_PREP_BWD : STG_PREP, stg_lev = in_backward ? STG_LEVELS_BWDPREP : STG_LEVELS;
     // fused per-chunk kernel: UT transform, boundary-adjusted tiles (version slot 0), chunk products (level 0)
@@ -264,7 +264,7 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
         }
         pp.status = at<uint32_t>(ws, p.status);
         prof_mark(stg_prep, 0, st);
-        LAUNCH(launch_chunk_prep(tm, pp, d, p.bwd, nch, st));
+        LAUNCH(launch_chunk_prep(tm, pp, d, keys_only ? PREP_KEYS : (p.bwd ? PREP_SAVE : PREP_FWD), nch, st));
         prof_mark(stg_prep, 1, st);
     }
     if (p.nlev < 2 || !with_levels) return PATH_OK;
@@ -799,13 +799,39 @@ int path_attn_prefill_cache(const void* k, const void* v, const void* w, const f
     const void* qd = k; const void* kd = k; const void* vd = v; const void* wd = w;
     rc = stage_inputs(p, workspace, qd, kd, vd, wd, beta, log_f, true, st);
     if (rc != PATH_OK) return rc;
-    rc = run_prep(p, workspace, qd, kd, wd, false, st, false);
+    rc = run_prep(p, workspace, qd, kd, wd, false, st, false, true);
     if (rc != PATH_OK) return rc;
     LevelTensorMaps tm;
     if (!make_level_maps(p, workspace, tm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
     LevelParams lp = level_params(p, workspace);
-    lp.kc = kc; lp.cap = cap; lp.L = L;
-    LAUNCH(launch_level_kernel(LEVEL_KEY_CACHE, tm, lp, d, st));
+    lp.cap = cap; lp.L = L;
+    // A long prompt is cut into up to eight ranges of at least eight chunks per head: the serial walk over the chunks runs
+    // per range (keys advanced to the range's end, bf16, in the unused plane of query tiles), then the ranges' products
+    // are multiplied up towards the end of the sequence and applied, tile by tile, into the float32 cache.  The scratch
+    // for the products is the (here unused) buffer of diagonal-correction operands.
+    const int nseg = p.N >= 32 ? (p.N / 8 < 8 ? p.N / 8 : 8) : 1;
+    if (nseg <= 1) {
+        lp.kc = kc;
+        LAUNCH(launch_level_kernel(LEVEL_KEY_CACHE, tm, lp, d, st));
+    } else {
+        typedef __nv_bfloat16 bf;
+        const size_t mats = (size_t)p.S * nseg * 2 * d * d;          // elements of one [S][nseg][2][d][d] buffer
+        bf* edge = at<bf>(workspace, p.Qv16);
+        bf* pseg = at<bf>(workspace, p.Xqn);
+        bf* sfx = pseg + mats;
+        lp.nseg = nseg; lp.seg_chunks = (p.N + nseg - 1) / nseg;
+        lp.edge16 = edge; lp.pseg = pseg; lp.sfx = sfx; lp.L = p.Lp;   // (whole padded chunks: padded rows are zero)
+        LAUNCH(launch_level_kernel(LEVEL_KEY_CACHE, tm, lp, d, st));
+        LevelTensorMaps tm2 = tm;
+        if (!make_map(&tm2.dyh, pseg, (uint64_t)p.S * nseg * 2 * d, d)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
+        LAUNCH(launch_level_kernel(LEVEL_SUFFIX, tm2, lp, d, st));
+        if (!(make_map(&tm2.dyh, sfx, (uint64_t)p.S * nseg * 2 * d, d) && make_map(&tm2.qv, edge, (uint64_t)p.S * p.Lp, d))) {
+            g_last_cuda_error = (int)cudaErrorUnknown;
+            return PATH_ERR_LAUNCH;
+        }
+        lp.kc = kc; lp.L = L; lp.edge16 = nullptr; lp.qv = edge; lp.gq = nullptr;
+        LAUNCH(launch_level_kernel(LEVEL_APPLY_PRODUCT, tm2, lp, d, st));
+    }
     CK(cudaMemcpy2DAsync(vc, (size_t)cap * d * 2, v, (size_t)L * d * 2, (size_t)L * d * 2, (size_t)p.S, cudaMemcpyDeviceToDevice, st));
     if (gc)
         CK(cudaMemcpy2DAsync(gc, (size_t)cap * 4, at<float>(workspace, p.G), (size_t)p.Lp * 4, (size_t)L * 4, (size_t)p.S,

@@ -39,6 +39,8 @@ def rel_fro(a, b):
     (2, 1, 700, 128, True),      # ragged length
     (1, 3, 100, 128, False),     # a single chunk
     (1, 1, 2304, 64, True),      # 18 chunks
+    (1, 2, 4224, 128, True),     # 33 chunks: the walk is cut into 4 ranges (9, 9, 9, 6 chunks) + suffix products
+    (2, 1, 8300, 64, False),     # 65 chunks, ragged: 8 ranges of 9 chunks, the last one of 2
 ])
 def test_prefill_cache_matches_oracle(binding, oracle, B, H, L, d, gate):
     inp = synth.make_inputs(B, H, L, d, "bf16", gate=gate, seed=50 + L)
