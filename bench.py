@@ -692,6 +692,65 @@ def run_frontend(args):
     print(json.dumps(line), flush=True)
 
 
+def run_ring(args):
+    """Context-parallel arm (paper Sec. 3.5), 1 GPU: the headline sequence cut into `--segments` equal segments, all ranks of
+    the ring played one after the other on this device (prepare for every segment, then every step of every rank:
+    D (D - 1) / 2 segment-against-segment sweeps).  One JSON line: forward TFLOP/s (attention-equivalent FLOPs of the
+    whole causal problem) of the virtual ring next to the monolithic forward.  Nothing is sent anywhere: this times the
+    per-device arithmetic, not a ring."""
+    from paper_2505_16381_b200 import binding, ring
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    c = synth.CONFIGS[args.workload]
+    B, H, L, d, D = (args.batch or c["B"]), c["H"], c["L"], c["d"], args.segments
+    inp = synth.make_inputs(B, H, L, d, dtype="bf16", qk_scaled=c["qk_scaled"], gate=c["gate"], seed=synth.BASE_SEED + c["index"])
+    names = ["q", "k", "v", "w", "beta"] + (["log_f"] if c["gate"] else [])
+    full = {n: inp[n].to(dev) for n in names}
+    cuts = [L * (i + 1) // D for i in range(D)]
+    segs, lo = [], 0
+    for hi in cuts:
+        segs.append({n: full[n][:, :, lo:hi].contiguous() for n in names})
+        lo = hi
+    ops = ring.GpuOps(B, H, d, scale=inp["scale"], has_gate=c["gate"], device=dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(fn):
+        for _ in range(args.warmup):
+            fn()
+        res = []
+        for _ in range(args.steps):
+            a, b_ = ev(), ev()
+            torch.cuda.synchronize()
+            a.record(); fn(); b_.record()
+            torch.cuda.synchronize()
+            res.append(a.elapsed_time(b_))
+        return sorted(res)[len(res) // 2]
+
+    sampler = ClockSampler(physical_gpu_index(0))
+    sampler.start()
+    ms_ring = timed(lambda: ring.virtual_ring_forward(ops, segs))
+    ws = binding.alloc_workspace(full["q"], c["gate"], False)
+    ms_mono = timed(lambda: binding.path_attn_fwd(full["q"], full["k"], full["v"], full["w"], full["beta"], full.get("log_f"),
+                                                  scale=inp["scale"], workspace=ws))
+    clocks = sampler.stop()
+    f1, _ = flops_m1(B, H, L, d)
+    peaks = load_peaks()
+    line = {"metric": f"PaTH attn forward TFLOP/s (attention-equivalent FLOPs), {D} virtual context-parallel ranks on one GPU, L={L}, d={d}",
+            "value": f1 / (ms_ring * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_ring, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"{args.workload} forward: B={B} H={H} L={L} d={d}, {D} segments of {L // D} positions, "
+                                   f"prepare x{D} + {D * (D - 1) // 2} steps + finish x{D}, no communication",
+                       "l2_policy": "inputs + workspaces exceed L2 (no flush needed)"},
+            "clocks": clocks, "gpu_launches": None,
+            "roofline": {"kernel": "whole virtual ring (sweeps + preparations)", "bound": "tensor", "achieved": f1 / (ms_ring * 1e-3) / 1e12,
+                         "peak": peaks["burst"], "unit": "TFLOP/s", "frac": f1 / (ms_ring * 1e-3) / 1e12 / peaks["burst"], "traffic": None,
+                         "peak_source": f"{peaks['source']} cuBLAS bf16, burst"},
+            "detail": {"monolithic_forward_ms": ms_mono, "monolithic_forward_tflops": f1 / (ms_mono * 1e-3) / 1e12,
+                       "ring_over_monolithic": ms_ring / ms_mono}}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -705,9 +764,10 @@ def main():
                     help="time the fwd+bwd step only: no forward-only / no-reuse / end-to-end arms (profiling captures)")
     ap.add_argument("--passes", type=int, default=0,
                     help="number of timed passes of --steps steps (default: as many as keep the GPU busy for > 1 s; profiling captures pass 1)")
-    ap.add_argument("--path", choices=["train", "decode", "frontend"], default="train",
+    ap.add_argument("--path", choices=["train", "decode", "frontend", "ring"], default="train",
                     help="train: the fwd+bwd step (the headline); decode: the inference arm; frontend: the layer front-end "
-                         "kernels (both 1 GPU, not part of the headline)")
+                         "kernels; ring: the context-parallel calls as virtual ranks (all 1 GPU, not part of the headline)")
+    ap.add_argument("--segments", type=int, default=4, help="--path ring: number of virtual ranks")
     args = ap.parse_args()
     if args.path == "decode":
         args.warmup = max(args.warmup, 3)
@@ -715,6 +775,9 @@ def main():
     if args.path == "frontend":
         args.warmup = max(args.warmup, 3)
         return run_frontend(args)
+    if args.path == "ring":
+        args.warmup = max(args.warmup, 3)
+        return run_ring(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = dict(synth.CONFIGS[args.workload])
     if args.batch > 0:
