@@ -31,8 +31,8 @@ __global__ void __launch_bounds__(kChainThreads, 1) chunk_chain_kernel(const __g
                                                              const ChainParams p, const int nchunks) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint64_t* bars = (uint64_t*)(smem + kBarOff);  // loads, two for product groups, two for the workers' hand-overs
-    uint32_t* tmem_slot = (uint32_t*)(bars + 5);
+    uint64_t* bars = (uint64_t*)(smem + kBarOff);  // two for loads, two for product groups, two for the workers' hand-overs
+    uint32_t* tmem_slot = (uint32_t*)(bars + 6);
     volatile uint32_t* abort_flag = (volatile uint32_t*)(tmem_slot + 1);
     float* bt = (float*)(smem + kBarOff + 64);
     float* t1 = bt + kT;
@@ -41,8 +41,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) chunk_chain_kernel(const __g
     const int row = (warp & 3) * 32 + lane, half = (warp >> 2) & 1;
 
     if (tid == 0) {
-        for (int i = 0; i < 3; ++i) mbar_init(&bars[i], 1);
-        for (int i = 3; i < 5; ++i) mbar_init(&bars[i], 256);
+        for (int i = 0; i < 6; ++i) mbar_init(&bars[i], i < 4 ? 1u : 256u);   // B_R0, B_R1: every worker arrives
         *abort_flag = 0;
         mbar_fence_init();
     }
@@ -56,30 +55,37 @@ __global__ void __launch_bounds__(kChainThreads, 1) chunk_chain_kernel(const __g
     auto sa = [&](int i) { return smem_u32(smem + i * kTileB); };
     constexpr int KD = HD / 16, K8 = 8;
     constexpr uint32_t cDW = 0, cA = 128, cB = 256, cG = 384;   // tensor-memory columns: dw, two work accumulators, W W^T
-    enum { B_LOAD = 0, B_MMA, B_MMA2, B_R0, B_R1 };
+    enum { B_LOAD = 0, B_LOAD2, B_MMA, B_MMA2, B_R0, B_R1, B_COUNT };
     const int grid = (int)gridDim.x;
 
     if (warp == 8) {
     if (lane == 0) {
     // ------------------------------------------------------------------ leader: TMA loads and every product
     bool ok = true;
-    uint32_t ph[5] = {0, 0, 0, 0, 0};
+    uint32_t ph[7] = {0, 0, 0, 0, 0, 0, 0};
     auto wait = [&](int b) {   // false (and nothing more is issued) once a wait has run out
         if (ok && !mbar_wait(&bars[b], ph[b], abort_flag, ST_CHAIN)) ok = false;
         ph[b] ^= 1;
         tc_fence_after_sync();
         return ok;
     };
+    // slots: 0 U->dXq   1 dQl->T~ hi->Ainv hi->K   2 Y^T->-Xq->Xk->dT hi->tmp hi->dGm hi   3 dSd->T~ lo->dT lo->tmp lo->dSd
+    //        4 W   5 dKr->dY->dXk->dGm lo   6 dP->dU->Ainv lo->Q
+    // First tiles of a chunk, in two parts: five of the seven slots are free as soon as the products that finish dq and dk
+    // have retired, and these five tiles are all that the chunk's first two products read; the other two slots feed the
+    // previous chunk's very last products.
     auto first_loads_a = [&](int ch) {
-        mbar_expect_tx(&bars[B_LOAD], 4 * kT * HD * 2 + 2 * kTileB);
-        tma_tile(slot(6), &tm.dp, &bars[B_LOAD], HD, ch * HD);
+        mbar_expect_tx(&bars[B_LOAD], 3 * kT * HD * 2 + 2 * kTileB);
         tma_tile(slot(1), &tm.dql, &bars[B_LOAD], HD, ch * kT);
-        tma_tile(slot(3), &tm.dsdt, &bars[B_LOAD], kT, ch * kT);
-        tma_tile(slot(5), &tm.dkr, &bars[B_LOAD], HD, ch * kT);
+        tma_tile(slot(0), &tm.u, &bars[B_LOAD], HD, ch * kT);
+        tma_tile(slot(3), &tm.dsdt, &bars[B_LOAD], kT, ch * kT);   // (s dSd)^T: every use takes the transposed view
+        tma_tile(slot(2), &tm.yt, &bars[B_LOAD], kT, ch * kT);
+        tma_tile(slot(6), &tm.dp, &bars[B_LOAD], HD, ch * HD);
     };
     auto first_loads_b = [&](int ch) {
-        tma_tile(slot(0), &tm.u, &bars[B_LOAD], HD, ch * kT);
-        tma_tile(slot(2), &tm.yt, &bars[B_LOAD], kT, ch * kT);
+        mbar_expect_tx(&bars[B_LOAD2], 2 * kT * HD * 2);
+        tma_tile(slot(5), &tm.dkr, &bars[B_LOAD2], HD, ch * kT);
+        tma_tile(slot(4), &tm.w, &bars[B_LOAD2], HD, ch * kT);
     };
     if ((int)blockIdx.x < nchunks) {
         first_loads_a(blockIdx.x);
@@ -88,25 +94,26 @@ __global__ void __launch_bounds__(kChainThreads, 1) chunk_chain_kernel(const __g
 #pragma unroll 1
     for (int chunk = blockIdx.x; chunk < nchunks && ok; chunk += grid) {
         const int r0 = chunk * kT;
-        // ---- phase 0: dXq = lower(-(dQl U^T + s dSd Y^T)) -> cA,  dw = -Y dKr - U dP^T
-        if (chunk != (int)blockIdx.x && !wait(B_R1)) break;   // the previous chunk's accumulators have been read
+        // ---- phase 0: dXq = lower(-(dQl U^T + s dSd Y^T)) -> cA, while the previous chunk's results are still leaving
+        // the other columns; then dw = -Y dKr - U dP^T
         if (!wait(B_LOAD)) break;
         mma_call(tmem + cA, sa(1), OP_K, sa(0), OP_K, KD, 128, false);
         mma_call(tmem + cA, sa(3), OP_MN, sa(2), OP_MN, K8, 128, true);          // slot 2 holds Y^T
+        if (chunk != (int)blockIdx.x && !wait(B_R1)) break;                      // the previous chunk's dw has left cDW
+        if (!wait(B_LOAD2)) break;
         mma_call(tmem + cDW, sa(2), OP_MN, sa(5), OP_MN, K8, HD, false, true);
         mma_call(tmem + cDW, sa(0), OP_K, sa(6), OP_K, KD, HD, true, true);
         umma_commit(&bars[B_MMA]);
         // ---- phase 1: dY = -(W dKr^T + Xq^T s dSd) -> cA,  dU = -(Xq^T dQl + W dP) -> cB.  dU's products read no tile
         // that the workers are writing and go to their own columns: they run underneath the read-out of dXq.
         if (!wait(B_MMA)) break;
-        mbar_expect_tx(&bars[B_LOAD], kT * HD * 2 + kTileB);
-        tma_tile(slot(0), &tm.w, &bars[B_LOAD], HD, r0);
+        mbar_expect_tx(&bars[B_LOAD], kTileB);
         tma_tile(slot(2), &tm.xqn, &bars[B_LOAD], kT, r0);
+        mma_call(tmem + cB, sa(4), OP_K, sa(6), OP_MN, KD, HD, false);           // W dP needs no new tile
         if (!wait(B_LOAD)) break;
-        mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, HD, false, true);    // slot 2 holds -Xq: negated back
-        mma_call(tmem + cB, sa(0), OP_K, sa(6), OP_MN, KD, HD, true);
+        mma_call(tmem + cB, sa(2), OP_MN, sa(1), OP_MN, K8, HD, true, true);     // slot 2 holds -Xq: negated back
         if (!wait(B_R0)) break;                                                  // dXq has left cA
-        mma_call(tmem + cA, sa(0), OP_K, sa(5), OP_K, KD, 128, false);
+        mma_call(tmem + cA, sa(4), OP_K, sa(5), OP_K, KD, 128, false);
         mma_call(tmem + cA, sa(2), OP_MN, sa(3), OP_K, K8, 128, true, true);
         umma_commit(&bars[B_MMA]);
         // ---- phase 2: dT = lower(dY Xk^T + dU W^T) -> cA, and phase 3 right behind it (the same dY and dU tiles and T~):
@@ -117,10 +124,10 @@ __global__ void __launch_bounds__(kChainThreads, 1) chunk_chain_kernel(const __g
         tma_tile(slot(2), &tm.xk, &bars[B_LOAD], kT, r0);
         tma_tile(slot(1), &tm.th, &bars[B_LOAD], kT, r0);
         tma_tile(slot(3), &tm.tl, &bars[B_LOAD], kT, r0);
-        if (!wait(B_LOAD)) break;
         if (!wait(B_R1)) break;                                                  // dY, dU tiles
-        mma_call(tmem + cA, sa(5), OP_K, sa(2), OP_K, K8, 128, false);
-        mma_call(tmem + cA, sa(6), OP_K, sa(0), OP_K, KD, 128, true);
+        mma_call(tmem + cA, sa(6), OP_K, sa(4), OP_K, KD, 128, false);           // dU W^T needs no new tile
+        if (!wait(B_LOAD)) break;
+        mma_call(tmem + cA, sa(5), OP_K, sa(2), OP_K, K8, 128, true);
         umma_commit(&bars[B_MMA]);
         mma_call(tmem + cB, sa(1), OP_MN, sa(5), OP_MN, K8, 128, false);
         mma_call(tmem + cB, sa(3), OP_MN, sa(5), OP_MN, K8, 128, true);
@@ -139,40 +146,43 @@ __global__ void __launch_bounds__(kChainThreads, 1) chunk_chain_kernel(const __g
         mma_call(tmem + cG, sa(1), OP_MN, sa(3), OP_MN, K8, 128, true);
         umma_commit(&bars[B_MMA]);
         if (!wait(B_R1)) break;                                                  // dXk has left cB
-        mma_call(tmem + cB, sa(0), OP_K, sa(0), OP_K, KD, 128, false);          // retires with the next group
+        mma_call(tmem + cB, sa(4), OP_K, sa(4), OP_K, KD, 128, false);          // retires with the next group
         if (!wait(B_MMA)) break;
         if (!wait(B_R0)) break;                                                  // tmp hi, lo tiles
         mma_call(tmem + cA, sa(2), OP_K, sa(1), OP_K, K8, 128, false);
         mma_call(tmem + cA, sa(2), OP_K, sa(6), OP_K, K8, 128, true);
         mma_call(tmem + cA, sa(3), OP_K, sa(1), OP_K, K8, 128, true);
         umma_commit(&bars[B_MMA]);
-        // ---- phase 5: dq -> cB, dk -> cG and the rest of dw.  K and Q replace Ainv hi / lo, (s dSd)^T returns.  The
-        // products that need neither dGm nor the columns that dbeta still reads go out first, underneath that read-out.
+        // ---- phase 5: dq -> cB, dk -> cG and the rest of dw, in three groups.  K and Q replace Ainv hi / lo, (s dSd)^T
+        // returns.  First the products that need neither dGm nor the columns that dbeta still reads; when they have
+        // retired, dXk's slot is free for dGm lo.  The second group finishes dq and dk, the third (dGm lo) only dw.
         if (!wait(B_MMA)) break;
         mbar_expect_tx(&bars[B_LOAD], 2 * kT * HD * 2 + kTileB);
-        tma_tile(slot(1), &tm.k, &bars[B_LOAD], HD, r0);
-        tma_tile(slot(6), &tm.q, &bars[B_LOAD], HD, r0);
         tma_tile(slot(3), &tm.dsdt, &bars[B_LOAD], kT, r0);
+        tma_tile(slot(6), &tm.q, &bars[B_LOAD], HD, r0);
+        tma_tile(slot(1), &tm.k, &bars[B_LOAD], HD, r0);
+        mma_call(tmem + cG, sa(5), OP_MN, sa(4), OP_MN, K8, HD, false);          // dXk^T W needs no new tile
         if (!wait(B_LOAD)) break;
-        mma_call(tmem + cG, sa(3), OP_K, sa(6), OP_MN, K8, HD, false);           // s dSd^T Q
-        mma_call(tmem + cG, sa(5), OP_MN, sa(0), OP_MN, K8, HD, true);           // dXk^T W
-        mma_call(tmem + cDW, sa(4), OP_MN, sa(6), OP_MN, K8, HD, true);          // dXq^T Q
+        mma_call(tmem + cG, sa(3), OP_K, sa(6), OP_MN, K8, HD, true);            // s dSd^T Q
+        mma_call(tmem + cDW, sa(0), OP_MN, sa(6), OP_MN, K8, HD, true);          // dXq^T Q
         mma_call(tmem + cDW, sa(5), OP_K, sa(1), OP_MN, K8, HD, true);           // dXk K
+        umma_commit(&bars[B_MMA2]);
         if (!wait(B_R1)) break;                                                  // dGm hi tile; W W^T has left cB
         mma_call(tmem + cB, sa(3), OP_MN, sa(1), OP_MN, K8, HD, false);          // s dSd K
-        mma_call(tmem + cB, sa(4), OP_K, sa(0), OP_MN, K8, HD, true);            // dXq W
-        mma_call(tmem + cDW, sa(2), OP_K, sa(0), OP_MN, K8, HD, true);           // dGm W
-        mma_call(tmem + cDW, sa(2), OP_MN, sa(0), OP_MN, K8, HD, true);          // dGm^T W
+        mma_call(tmem + cB, sa(0), OP_K, sa(4), OP_MN, K8, HD, true);            // dXq W
+        mma_call(tmem + cDW, sa(2), OP_K, sa(4), OP_MN, K8, HD, true);           // dGm W
+        mma_call(tmem + cDW, sa(2), OP_MN, sa(4), OP_MN, K8, HD, true);          // dGm^T W
         umma_commit(&bars[B_MMA]);
-        if (!wait(B_MMA)) break;
+        if (!wait(B_MMA2)) break;
+        if (!wait(B_R0)) break;                                                  // dGm lo tile (over dXk)
+        mma_call(tmem + cDW, sa(5), OP_K, sa(4), OP_MN, K8, HD, true);
+        mma_call(tmem + cDW, sa(5), OP_MN, sa(4), OP_MN, K8, HD, true);
+        umma_commit(&bars[B_MMA2]);
         const int next = chunk + grid;
-        if (next < nchunks) first_loads_a(next);                                 // slots 1, 3, 5, 6 are free
-        if (!wait(B_R0)) break;                                                  // dGm lo tile
-        mma_call(tmem + cDW, sa(2), OP_K, sa(0), OP_MN, K8, HD, true);
-        mma_call(tmem + cDW, sa(2), OP_MN, sa(0), OP_MN, K8, HD, true);
-        umma_commit(&bars[B_MMA]);
         if (!wait(B_MMA)) break;
-        if (next < nchunks) first_loads_b(next);                                 // and the last two
+        if (next < nchunks) first_loads_a(next);                                 // slots 0 - 3 and 6 are free
+        if (!wait(B_MMA2)) break;
+        if (next < nchunks) first_loads_b(next);                                 // and the other two
     }
     }
     __syncwarp();
@@ -264,12 +274,10 @@ __global__ void __launch_bounds__(kChainThreads, 1) chunk_chain_kernel(const __g
         const int s_idx = chunk / p.N, pos = (chunk % p.N) * kT + row;   // slice and position of this thread's row
         const bool row_valid = pos < p.L;
         const size_t urow = (size_t)s_idx * p.L + pos;                   // row in the caller's [S][L][.] tensors
-        const __nv_bfloat16* g_dql = p.dql + ((size_t)chunk * kT + row) * HD;
-        const __nv_bfloat16* g_dkr = p.dkr + ((size_t)chunk * kT + row) * HD;
         if (tid < kT) bt[tid] = p.beta[(size_t)chunk * kT + tid];   // first read after several barriers (phase 4)
         mma_wait();                                                 // phase 0
         if (!ok) break;
-        acc_to_tile(cA, kT, slot(4), -1.f, M_LOWER);                // dXq
+        acc_to_tile(cA, kT, slot(0), -1.f, M_LOWER);                // dXq (over U)
         publish(B_R0);
         mma_wait();                                                 // phase 1
         if (!ok) break;
@@ -302,6 +310,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) chunk_chain_kernel(const __g
         publish(B_R0);
         mma_wait();                                                 // dA and W W^T
         if (!ok) break;
+        float dbeta_row;
         {   // dA = strictLower(-cA);  dbeta_r = t1_r + sum_c dA_rc (W W^T)_rc
             float part = 0.f;
             for (int c = 0; c < 2; ++c) {
@@ -317,43 +326,72 @@ __global__ void __launch_bounds__(kChainThreads, 1) chunk_chain_kernel(const __g
             wsync();
             if (half == 1) t1[row] += part;
             wsync();
-            if (half == 0 && row_valid) p.dbeta[urow] = t1[row] + part;
+            dbeta_row = t1[row] + part;
         }
         split_to_tile(cA, slot(2), false, f_dGm);                   // dGm = D dA, hi
         publish(B_R1);
-        // the dQl / dKr rows of the final sums are fetched while the products run
+        // (global stores and loads come after a hand-over, never just before it: the hand-over waits for them)
+        if (half == 0 && row_valid) p.dbeta[urow] = dbeta_row;
+        // The dQl / dKr rows of the final sums are fetched while the products run.  At d = 128 a thread's half row is one
+        // 128-byte line: four lanes fetch four lines together, a quarter of each per instruction (whole lines per request
+        // instead of 32 scattered pieces, which held up the products' operand reads as well).
         constexpr int NI = HD / 64;
-        uint4 pre_q[NI][4], pre_k[NI][4];
+        uint32_t rq[4][8], rk[4][8];
+        uint4 pre_q[4], pre_k[4];
+        {
+            const __nv_bfloat16* g_dql = p.dql + ((size_t)chunk * kT + row) * HD + half * (HD / 2);
+            const __nv_bfloat16* g_dkr = p.dkr + ((size_t)chunk * kT + row) * HD + half * (HD / 2);
+            if (HD == 128) {
+                gload_f32x32_issue(reinterpret_cast<const float*>(g_dql), rq);
+                gload_f32x32_issue(reinterpret_cast<const float*>(g_dkr), rk);
+            } else {
 #pragma unroll
-        for (int c = 0; c < NI; ++c) {
-            const int c0 = half * (HD / 2) + c * 32;
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                pre_q[c][x] = reinterpret_cast<const uint4*>(g_dql + c0)[x];
-                pre_k[c][x] = reinterpret_cast<const uint4*>(g_dkr + c0)[x];
+                for (int x = 0; x < 4; ++x) {
+                    pre_q[x] = reinterpret_cast<const uint4*>(g_dql)[x];
+                    pre_k[x] = reinterpret_cast<const uint4*>(g_dkr)[x];
+                }
             }
         }
-        mma_wait();                                                 // phase 5
+        mma_wait(B_MMA2);                                           // phase 5, first group: dXk's slot is free
         if (!ok) break;
-        split_to_tile(cA, slot(2), true, f_dGm);                    // dGm lo
+        split_to_tile(cA, slot(5), true, f_dGm);                    // dGm lo (over dXk)
         publish(B_R0);
+        mma_wait();                                                 // phase 5, second group
+        if (!ok) break;
         // dq and dk are complete: they leave while the last two products run
+        {
+            float wq[32], wk[32];   // HD == 128: the fetched half rows, two bf16 per word
+            if (HD == 128) {
+                gload_f32x32_finish(rq, wq);
+                gload_f32x32_finish(rk, wk);
+            }
+            auto add_row = [&](const float (&words)[32], const uint4 (&pre)[4], int c, float (&acc)[32]) {
+                if (HD == 128) {
 #pragma unroll
-        for (int c = 0; c < NI; ++c) {
-            const int c0 = half * (HD / 2) + c * 32;
-            float in[32];
-            tmem_row32(tl + cB + c0, v);
-            unpack_bf16x32(pre_q[c], in);
+                    for (int x = 0; x < 16; ++x) {
+                        const uint32_t u = __float_as_uint(words[16 * c + x]);
+                        acc[2 * x] += __uint_as_float(u << 16);
+                        acc[2 * x + 1] += __uint_as_float(u & 0xffff0000u);
+                    }
+                } else {
+                    float in[32];
+                    unpack_bf16x32(pre, in);
 #pragma unroll
-            for (int x = 0; x < 32; ++x) v[x] += in[x];
-            gstore_bf16x32(p.dq + urow * HD + c0, v, row_valid);
-            tmem_row32(tl + cG + c0, v);
-            unpack_bf16x32(pre_k[c], in);
+                    for (int x = 0; x < 32; ++x) acc[x] += in[x];
+                }
+            };
 #pragma unroll
-            for (int x = 0; x < 32; ++x) v[x] += in[x];
-            gstore_bf16x32(p.dk + urow * HD + c0, v, row_valid);
+            for (int c = 0; c < NI; ++c) {
+                const int c0 = half * (HD / 2) + c * 32;
+                tmem_row32(tl + cB + c0, v);
+                add_row(wq, pre_q, c, v);
+                gstore_bf16x32(p.dq + urow * HD + c0, v, row_valid);
+                tmem_row32(tl + cG + c0, v);
+                add_row(wk, pre_k, c, v);
+                gstore_bf16x32(p.dk + urow * HD + c0, v, row_valid);
+            }
         }
-        mma_wait();                                                 // the last of dw
+        mma_wait(B_MMA2);                                           // the last of dw
         if (!ok) break;
 #pragma unroll
         for (int c = 0; c < NI; ++c) {

@@ -398,44 +398,72 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
             fence_proxy_async_smem();   // also covers the Xq tiles written above
             tc_fence_before_sync();
             mbar_arrive(&bars[R_U]);
+            uint32_t yh[2][16];
+#pragma unroll
             for (int c = 0; c < 2; ++c) {
                 const int c0 = half * 64 + c * 32;
                 tmem_ld32(tl + 384 + c0, r);
                 tmem_ld_wait();
 #pragma unroll
                 for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
-                split32(v, hi, lo);
-                tile_store_w16(sBig + 2 * kTileB, row, c0, hi);
+                split32(v, yh[c], lo);
+                tile_store_w16(sBig + 2 * kTileB, row, c0, yh[c]);
                 tile_store_w16(sBig + 3 * kTileB, row, c0, lo);
-                if (!KEYS) {
-                    unsigned short* yt = reinterpret_cast<unsigned short*>(p.Yt) + ((size_t)chunk * kT + c0) * kT + row;
-#pragma unroll
-                    for (int x = 0; x < 16; ++x) {
-                        yt[(size_t)(2 * x) * kT] = (unsigned short)(hi[x] & 0xffffu);
-                        yt[(size_t)(2 * x + 1) * kT] = (unsigned short)(hi[x] >> 16);
-                    }
-                }
             }
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars[R_Y]);
+            if (!KEYS) {
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    unsigned short* yt = reinterpret_cast<unsigned short*>(p.Yt) + ((size_t)chunk * kT + half * 64 + c * 32) * kT + row;
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) {
+                        yt[(size_t)(2 * x) * kT] = (unsigned short)(yh[c][x] & 0xffffu);
+                        yt[(size_t)(2 * x + 1) * kT] = (unsigned short)(yh[c][x] >> 16);
+                    }
+                }
+            }
 
             // ---- E3: Qleft = Q - Xq U, P = I - W^T U, then Kright = K - Y^T W; the q / k rows are fetched while the
             // products run
-            uint4 pre_q[HD / 64][4], pre_k[HD / 64][4];
+            // At d = 128 a thread's half row is one 128-byte line: four lanes fetch four lines together, a quarter of each per
+            // instruction (whole lines per request instead of 32 scattered pieces, which also hold up the products' operand reads)
+            uint32_t rq[4][8], rk[4][8];
+            uint4 pre_q[4], pre_k[4];
+            {
+                const __nv_bfloat16* gq = p.q + grow * HD + half * (HD / 2);
+                const __nv_bfloat16* gk = p.k + grow * HD + half * (HD / 2);
+                if (HD == 128) {
+                    if (!KEYS) gload_f32x32_issue(reinterpret_cast<const float*>(gq), rq);
+                    gload_f32x32_issue(reinterpret_cast<const float*>(gk), rk);
+                } else {
 #pragma unroll
-            for (int c = 0; c < HD / 64; ++c) {
-                const int c0 = half * (HD / 2) + c * 32;
-#pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    if (!KEYS) pre_q[c][x] = reinterpret_cast<const uint4*>(p.q + grow * HD + c0)[x];
-                    pre_k[c][x] = reinterpret_cast<const uint4*>(p.k + grow * HD + c0)[x];
+                    for (int x = 0; x < 4; ++x) {
+                        if (!KEYS) pre_q[x] = reinterpret_cast<const uint4*>(gq)[x];
+                        pre_k[x] = reinterpret_cast<const uint4*>(gk)[x];
+                    }
                 }
             }
+            // in[] <- columns c * 32 .. + 31 of a fetched half row (`words`: the whole half row at d = 128, two bf16 per word)
+            auto row_part = [&](const float (&words)[32], const uint4 (&pre)[4], int c, float (&in)[32]) {
+                if (HD == 128) {
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) {
+                        const uint32_t u = __float_as_uint(words[16 * c + x]);
+                        in[2 * x] = __uint_as_float(u << 16);
+                        in[2 * x + 1] = __uint_as_float(u & 0xffff0000u);
+                    }
+                } else {
+                    unpack_bf16x32(pre, in);
+                }
+            };
             const int next = chunk + (int)gridDim.x;
             float next_beta = 0.f;
             if (tid < kT && next < nchunks) next_beta = p.beta[(size_t)next * kT + tid];
             if (!(ok = wwait(B_G3A, par))) break;
+            float words[32];
+            if (HD == 128 && !KEYS) gload_f32x32_finish(rq, words);
 #pragma unroll
             for (int c = 0; c < HD / 64; ++c) {
                 const int c0 = half * (HD / 2) + c * 32;
@@ -443,7 +471,7 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                     float in[32];
                     tmem_ld32(tl + 256 + c0, r);
                     tmem_ld_wait();
-                    unpack_bf16x32(pre_q[c], in);
+                    row_part(words, pre_q, c, in);
 #pragma unroll
                     for (int x = 0; x < 32; ++x) v[x] = in[x] - __uint_as_float(r[x]);
                     gstore_bf16x32(p.ql + grow * HD + c0, v);
@@ -457,13 +485,14 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 gstore_bf16_w16(p.Pl + ((size_t)chunk * HD + row) * HD + c0, lo, row < HD);
             }
             if (!(ok = wwait(B_G3B, par))) break;
+            if (HD == 128) gload_f32x32_finish(rk, words);
 #pragma unroll
             for (int c = 0; c < HD / 64; ++c) {
                 const int c0 = half * (HD / 2) + c * 32;
                 float in[32];
                 tmem_ld32(tl + 384 + c0, r);
                 tmem_ld_wait();
-                unpack_bf16x32(pre_k[c], in);
+                row_part(words, pre_k, c, in);
 #pragma unroll
                 for (int x = 0; x < 32; ++x) v[x] = in[x] - __uint_as_float(r[x]);
                 gstore_bf16x32(p.kr + grow * HD + c0, v);
