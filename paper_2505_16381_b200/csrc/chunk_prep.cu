@@ -3,7 +3,8 @@
 //
 // With W, Q, K the rows of one 128-token chunk and D = diag(beta):
 //   Gm = W W^T,  Xq = lower(Q W^T),  Xk = strictLower(W K^T)
-//   T~ = (I + strictLower(D Gm))^-1 D                                             (float32, blocked substitution)
+//   T~ = (I + strictLower(D Gm))^-1 D        (float32 blocked substitution up to 64-row blocks; the last merge level is two
+//                                             64 x 64 x 64 products of bf16 pairs on the tensor cores)
 //   U = T~ W,  Y = T~ Xk
 //   Qleft = Q - Xq U,  Kright = K - Y^T W,  P = I - W^T U
 // and the bf16 operands of the diagonal-chunk correction of the attention sweep, Xqn = -Xq and Yt = Y^T.
@@ -28,8 +29,9 @@ namespace {
 
 using namespace tile;
 constexpr int kLd = kT + 4;  // row stride of the float32 triangular buffer (rows stay 16-byte aligned)
+constexpr uint32_t kInvTileB = 8192;   // a [64 x 64] bf16 operand tile of the inverse's last merge level
 
-// Seven 32 KB tile slots.  0: W.  1, 2: Q, K -> T~ hi, lo -> U hi, lo.  3..6: float32 triangular buffer and its
+// Seven 32 KB tile slots.  0: W.  1, 2: Q, K -> operands of the inverse's last merge level -> T~ hi, lo -> U hi, lo.  3..6: float32 triangular buffer and its
 // scratch -> Xq hi, lo, Xk hi, lo -> (5, 6) Y hi, lo.
 struct PrepSmem {
     static constexpr uint32_t offW = 0;
@@ -45,7 +47,7 @@ struct PrepSmem {
 
 // mbarriers.  Issuer -> workers: one per group of products (and the TMA load, which only the issuer waits for).
 // Workers -> issuer (256 arrivals): operands published / accumulators drained.  Each completes once per chunk.
-enum { B_LOAD = 0, B_GM, B_XQK, B_U, B_Y, B_G3A, B_G3B, R_TT, R_XK, R_U, R_Y, R_E3, B_COUNT };
+enum { B_LOAD = 0, B_GM, B_XQK, B_M1, B_M2, B_U, B_Y, B_G3A, B_G3B, R_TT, R_M1, R_M2, R_XK, R_U, R_Y, R_E3, B_COUNT };
 constexpr int kWorkers = 256, kThreads = 384;   // warps 8..11: the issuer's warpgroup (one active lane)
 
 // Barriers over the eight worker warps.  bar.sync / bar.red are warp-aligned instructions: a warp whose lanes left a
@@ -109,7 +111,8 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
     const uint32_t tl = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t aW_ = smem_u32(sW), aQ_ = smem_u32(sQK), aK_ = smem_u32(sQK + kTileB), aBig_ = smem_u32(sBig);
     constexpr int KS = HD / 16;  // k-steps over the head dimension
-    // tensor-memory columns:  0: Gm -> U   128: Xq -> W^T U   256: Xk -> Xq U   384: Y -> Y^T W
+    // tensor-memory columns:  0: Gm -> the inverse's last merge level (0: C A^-1, 64: B^-1 C A^-1) -> U   128: Xq -> W^T U
+    //                         256: Xk -> Xq U   384: Y -> Y^T W
 
     if (warp >= kWorkers / 32) {
         // ------------------------------------------------------------------ issuer
@@ -150,6 +153,20 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 if (!KEYS) mma_small(tmem + 128, aQ, OP_K, aW, OP_K, KS, 128, false);
                 mma_small(tmem + 256, aW, OP_K, aK, OP_K, KS, 128, false);
                 umma_commit(&bars[B_XQK]);
+                // last merge level of the triangular inverse: T = C A^-1, then B^-1 T, as bf16 pairs (64 x 64 x 64 each; the
+                // eight 8 KB operand tiles sit in the Q / K slots, whose products have retired by then)
+                if (!wait(R_M1, par)) break;
+                tc_fence_after_sync();
+                mma_small(tmem + 0, aQ, OP_K, aQ + 2 * kInvTileB, OP_MN, 4, 64, false);
+                mma_small(tmem + 0, aQ, OP_K, aQ + 3 * kInvTileB, OP_MN, 4, 64, true);
+                mma_small(tmem + 0, aQ + kInvTileB, OP_K, aQ + 2 * kInvTileB, OP_MN, 4, 64, true);
+                umma_commit(&bars[B_M1]);
+                if (!wait(R_M2, par)) break;
+                tc_fence_after_sync();
+                mma_small(tmem + 64, aQ + 4 * kInvTileB, OP_K, aQ + 6 * kInvTileB, OP_MN, 4, 64, false);
+                mma_small(tmem + 64, aQ + 4 * kInvTileB, OP_K, aQ + 7 * kInvTileB, OP_MN, 4, 64, true);
+                mma_small(tmem + 64, aQ + 5 * kInvTileB, OP_K, aQ + 6 * kInvTileB, OP_MN, 4, 64, true);
+                umma_commit(&bars[B_M2]);
                 // U = T~ W  (lo x lo terms are dropped everywhere)
                 if (!wait(R_TT, par)) break;
                 tc_fence_after_sync();
@@ -319,11 +336,66 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 };
                 merge(std::integral_constant<int, 16>{});
                 merge(std::integral_constant<int, 32>{});
-                merge(std::integral_constant<int, 64>{});
+            }
+            // Last level (64-row blocks) on the tensor cores: both products are 64 x 64 x 64, which the CUDA cores take
+            // ten thousand cycles for (the triangular second product keeps only the warps with the long rows busy).  The
+            // operands go as bf16 pairs (hi hi + hi lo + lo hi), the precision T~ itself is kept in afterwards.
+            if (!(ok = wwait(B_XQK, par))) break;   // the products that read the Q and K tiles have retired
+            {
+                const int r_ = tid >> 2, seg = tid & 3;   // this thread: 16 columns of one row of C, A^-1 and B^-1
+                const float* src[3] = {Xb + (64 + r_) * kLd + seg * 16, Xb + r_ * kLd + seg * 16, Xb + (64 + r_) * kLd + 64 + seg * 16};
+#pragma unroll
+                for (int m = 0; m < 3; ++m) {
+                    uint32_t h8[8], l8[8];
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const float4 f = *reinterpret_cast<const float4*>(src[m] + 4 * x);
+                        const uint32_t a = pack_bf16(f.x, f.y), b = pack_bf16(f.z, f.w);
+                        h8[2 * x] = a;
+                        h8[2 * x + 1] = b;
+                        l8[2 * x] = pack_bf16(f.x - __uint_as_float(a << 16), f.y - __uint_as_float(a & 0xffff0000u));
+                        l8[2 * x + 1] = pack_bf16(f.z - __uint_as_float(b << 16), f.w - __uint_as_float(b & 0xffff0000u));
+                    }
+                    uint8_t* th_ = sQK + (2 * m) * kInvTileB;
+                    uint8_t* tl_ = th_ + kInvTileB;
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        const uint32_t off = sw128_off((uint32_t)r_, (uint32_t)(seg * 2 + c));
+                        *reinterpret_cast<uint4*>(th_ + off) = make_uint4(h8[4 * c], h8[4 * c + 1], h8[4 * c + 2], h8[4 * c + 3]);
+                        *reinterpret_cast<uint4*>(tl_ + off) = make_uint4(l8[4 * c], l8[4 * c + 1], l8[4 * c + 2], l8[4 * c + 3]);
+                    }
+                }
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                mbar_arrive(&bars[R_M1]);
+                if (!(ok = wwait(B_M1, par))) break;
+                if (row < 64) {   // T: rows 0..63 of the accumulator -> bf16 pair, the right-hand operand of the second product
+                    tmem_ld32(tl + 0 + half * 32, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]);
+                    split32(v, hi, lo);
+                    tile_store_w16(sQK + 6 * kInvTileB, row, half * 32, hi);
+                    tile_store_w16(sQK + 7 * kInvTileB, row, half * 32, lo);
+                }
+                fence_proxy_async_smem();
+                tc_fence_before_sync();
+                mbar_arrive(&bars[R_M2]);
+                if (!(ok = wwait(B_M2, par))) break;
+                if (row < 64) {   // -B^-1 T replaces C
+                    tmem_ld32(tl + 64 + half * 32, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int x = 0; x < 8; ++x)
+                        *reinterpret_cast<float4*>(Xb + (64 + row) * kLd + half * 32 + 4 * x) =
+                            make_float4(-__uint_as_float(r[4 * x]), -__uint_as_float(r[4 * x + 1]), -__uint_as_float(r[4 * x + 2]),
+                                        -__uint_as_float(r[4 * x + 3]));
+                }
+                tc_fence_before_sync();
+                wsync();
             }
 
-            // ---- T~ = X D as a bf16 pair into the Q / K tiles' space, once the products that read Q and K have retired
-            if (!(ok = wwait(B_XQK, par))) break;
+            // ---- T~ = X D as a bf16 pair into the Q / K tiles' space
             for (int c = 0; c < 2; ++c) {
                 const int c0 = half * 64 + c * 32;
                 float t[32];
