@@ -174,13 +174,15 @@ __global__ void __launch_bounds__(kChainThreads, 1) chunk_chain_kernel(const __g
         mma_call(tmem + cDW, sa(2), OP_MN, sa(4), OP_MN, K8, HD, true);          // dGm^T W
         umma_commit(&bars[B_MMA]);
         if (!wait(B_MMA2)) break;
+        // (the last two products cannot start before the second group has left the pipe anyway: the next chunk's tiles are
+        // requested first, the moment their slots are free)
+        const int next = chunk + grid;
+        if (!wait(B_MMA)) break;
+        if (next < nchunks) first_loads_a(next);                                 // slots 0 - 3 and 6 are free
         if (!wait(B_R0)) break;                                                  // dGm lo tile (over dXk)
         mma_call(tmem + cDW, sa(5), OP_K, sa(4), OP_MN, K8, HD, true);
         mma_call(tmem + cDW, sa(5), OP_MN, sa(4), OP_MN, K8, HD, true);
         umma_commit(&bars[B_MMA2]);
-        const int next = chunk + grid;
-        if (!wait(B_MMA)) break;
-        if (next < nchunks) first_loads_a(next);                                 // slots 0 - 3 and 6 are free
         if (!wait(B_MMA2)) break;
         if (next < nchunks) first_loads_b(next);                                 // and the other two
     }
