@@ -8,12 +8,14 @@
 //   dbeta_r += sum_c dA_rc (W W^T)_rc,           dGm = D dA
 //   dq = dQl + s dSd K + dXq W                   dk = dKr + s dSd^T Q + dXk^T W
 //   dw = -Y dKr - U dP^T + T~^T dU + dXq^T Q + dXk K + (dGm + dGm^T) W
-// A persistent CTA (one per SM) walks over chunks and runs these ~25 products per chunk as tcgen05 MMAs on swizzled
-// shared-memory tiles, in lockstep: thread 0 loads tiles (TMA) and issues MMAs, all 256 threads turn accumulators
-// (tensor memory, one row per thread) into the next operand tiles.  dQl and dKr arrive as bf16 tiles; the next
-// chunk's first tiles are requested before the current chunk's results are written out.  T~ and Ainv enter as bf16
-// hi + lo pairs, and so do the in-kernel intermediates dT, M D and dGm (the lo tile follows the hi tile through
-// the same slot); everything else is rounded to bf16 once.  dw accumulates in tensor memory across all phases.
+// A persistent CTA (one per SM) walks over chunks and runs these ~31 products per chunk as tcgen05 MMAs on swizzled
+// shared-memory tiles.  Eight worker warps turn accumulators (tensor memory, one row per thread) into the next operand
+// tiles; the first lane of a ninth warp requests every tile (TMA) and issues every product.  The two sides meet only
+// through mbarriers: the workers hand tiles over and go on (they wait for products, never for the issuer), the issuer
+// sends out first whatever does not depend on the read-out in progress, starts the next chunk's first products while
+// the current chunk's results are still leaving, and requests tiles the moment their slots are free.  dQl and dKr
+// arrive as bf16 tiles.  T~ and Ainv enter as bf16 hi + lo pairs, and so do the in-kernel intermediates dT, M D and dGm;
+// everything else is rounded to bf16 once.  dw accumulates in tensor memory across all phases.
 #include "tileops.cuh"
 
 namespace path {

@@ -1,7 +1,7 @@
-// Building blocks of the "lockstep" chunk kernels: every matrix of the chunk-level algebra is a 128-row
+// Building blocks of the per-chunk kernels: every matrix of the chunk-level algebra is a 128-row
 // bf16 tile in shared memory (row-major, 64-column panels, 128-byte swizzle), every product a tcgen05 MMA into
-// tensor memory issued by thread 0, every result read back one row per thread (256 threads: two per row, each
-// taking half of the columns).
+// tensor memory issued by one thread, every result read back one row per thread (256 worker threads: two per row,
+// each taking half of the columns).
 #pragma once
 #include "common.cuh"
 #include "tc5.cuh"
