@@ -180,14 +180,15 @@ __global__ void __launch_bounds__(kThreads, 1) chunk_prep_kernel(const __grid_co
                 // Y = T~ Xk
                 if (!wait(R_XK, par)) break;
                 tc_fence_after_sync();
+                if (SAVE) {   // (requested before the products are issued: the issue takes as long as the store's reads)
+                    store(&tm.xk, sBig + 2 * kTileB, kT, chunk);
+                    tma_store_commit();
+                }
                 mma_small(tmem + 384, aQ, OP_K, aBig + 2 * kTileB, OP_MN, 8, 128, false);
                 mma_small(tmem + 384, aK, OP_K, aBig + 2 * kTileB, OP_MN, 8, 128, true);
                 mma_small(tmem + 384, aQ, OP_K, aBig + 3 * kTileB, OP_MN, 8, 128, true);
-                if (SAVE) {   // B_Y lets the workers overwrite T~ (with U) and Xk (with Y): the stores must have read them
-                    store(&tm.xk, sBig + 2 * kTileB, kT, chunk);
-                    tma_store_commit();
-                    tma_store_wait_read();
-                }
+                // B_Y lets the workers overwrite T~ (with U) and Xk (with Y): the stores must have read them
+                if (SAVE) tma_store_wait_read();
                 umma_commit(&bars[B_Y]);
                 // Xq U and W^T U
                 if (!wait(R_U, par)) break;
