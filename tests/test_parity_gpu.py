@@ -206,7 +206,7 @@ def test_short_gated_problems_down_to_one_token(binding, oracle):
         for  sum(O dO) - sum(eps lse),  i.e. the gradient the definition gives for the o the call was handed.
     (2) dbeta / dw of such a problem can be carried by one or two entries of magnitude 1e-3; each comes out of four to five
         products of bf16-rounded operands (2^-9 relative each), which average out over a workload's thousands of
-        entries but not here.  A tensor whose largest reference entry is below 0.05 is therefore judged by
+        entries but not here.  A tensor whose largest reference entry is below 0.05 is therefore compared by
         max-abs <= 1e-3 (the absolute bound 2e-2 scaled to that floor) where it misses the relative bound.
     Against the plain oracle every tensor still meets the absolute bound."""
     import random
