@@ -143,6 +143,7 @@ struct LevelParams {
     int l;                  // dyadic forward: level consumed (l -> l + 1); version forward: number of levels; level backward: the
                             // level of the run products whose gradients the launch finishes
     int nlev;               // number of levels (level backward)
+    int fuse;               // fused dyadic forward: levels l + 1 .. l + fuse are produced by one launch (2 or 3)
     int S, N, Lp;
     __nv_bfloat16 *dyh, *dyl, *qv, *kv;
     __nv_bfloat16 *dqv, *dkv;     // gradients of the versions (placed like them); plane 0 ends up holding the final sums
@@ -159,7 +160,7 @@ struct LevelParams {
     uint32_t* status;
 };
 
-enum { LEVEL_DYADIC_FWD = 0, LEVEL_VERSION_FWD, LEVEL_BWD, LEVEL_KEY_CACHE, LEVEL_QUERY_EDGE, LEVEL_SUFFIX, LEVEL_APPLY_PRODUCT };
+enum { LEVEL_DYADIC_FWD = 0, LEVEL_DYADIC_FUSED, LEVEL_VERSION_FWD, LEVEL_BWD, LEVEL_KEY_CACHE, LEVEL_QUERY_EDGE, LEVEL_SUFFIX, LEVEL_APPLY_PRODUCT };
 cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const LevelParams& p, int hd, cudaStream_t st);
 
 struct PrepTensorMaps {

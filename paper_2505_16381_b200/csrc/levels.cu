@@ -144,6 +144,135 @@ __global__ void __launch_bounds__(256, 1) dyadic_fwd_kernel(const __grid_constan
     teardown<128>(c, p.status);
 }
 
+// ---------------------------------------------------------------------------------------------- dyadic forward, fused
+// Two or three consecutive levels in one launch (p.fuse): a CTA takes 2^fuse neighbouring products of level p.l and
+// builds the whole tree above them,
+//     A_k = Dy[l][2k+1] Dy[l][2k]  (k < 2^(fuse-1)),    B_k = A_{2k+1} A_{2k},    C = B_1 B_0,
+// writing every product to global memory as it appears and keeping it in shared memory as the next product's operand,
+// so the intermediate levels are read back by nobody and the launches (and their tails) between the levels are gone.
+// Six tile slots: a product's result replaces the tiles of its own left factor; B_0 waits in tensor memory (columns
+// 128..255) while A_2, A_3 and B_1 are made.  grid.x = S * groups, groups = ceil(cnt(l + 1) / 2^(fuse-1)).
+template <int HD>
+__global__ void __launch_bounds__(256, 1) dyadic_fused_kernel(const __grid_constant__ LevelTensorMaps tm, const LevelParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    Ctx c;
+    setup<256>(c, smem_raw, 6 * kTileB);
+    const int half_w = 1 << (p.fuse - 1);                        // A products per group
+    const int groups = (p.lv.dy_cnt[p.l + 1] + half_w - 1) / half_w;
+    const int s = blockIdx.x / groups, g = blockIdx.x % groups;
+    uint8_t* sm = c.smem;
+    auto mat = [&](int lvl, int idx) { return p.lv.dy_off[lvl] / (HD * HD) + (long)s * p.lv.dy_cnt[lvl] + idx; };
+    // acc(col) = left (slots a, a + 1) x right (slots b, b + 1), the lo x lo term left out
+    auto product = [&](uint32_t col, int a, int b) {
+        publish();   // operands written by this CTA's threads are visible, and nobody still reads the accumulator
+        if (c.tid == 0 && c.ok) {
+            tc_fence_after_sync();
+            const uint32_t base = smem_u32(sm);
+            mma(c.tmem + col, base + a * kTileB, OP_K, base + b * kTileB, OP_MN, HD / 16, HD, false);
+            mma(c.tmem + col, base + a * kTileB, OP_K, base + (b + 1) * kTileB, OP_MN, HD / 16, HD, true);
+            mma(c.tmem + col, base + (a + 1) * kTileB, OP_K, base + b * kTileB, OP_MN, HD / 16, HD, true);
+            umma_commit(&c.bars[1]);
+        }
+        mma_wait(c);
+    };
+    // accumulator -> bf16 pair: to global memory as Dy[lvl][idx] (if to_global) and / or into slots a, a + 1 (a >= 0)
+    auto readout = [&](uint32_t col, int lvl, int idx, bool to_global, int a) {
+        if (!c.ok) return;
+        float v[32], hi[32];
+        for (int i = 0; i < HD / 64; ++i) {
+            const int c0 = c.half * (HD / 2) + i * 32;
+            tmem_row32(c.tl + col + c0, v);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+                hi[x] = __bfloat162float(__float2bfloat16_rn(v[x]));
+                v[x] -= hi[x];
+            }
+            if (a >= 0) {
+                tile_store32(sm + a * kTileB, c.row, c0, hi);
+                tile_store32(sm + (a + 1) * kTileB, c.row, c0, v);
+            }
+            if (to_global) {
+                const size_t o = ((size_t)mat(lvl, idx) * HD + c.row) * HD + c0;
+                gstore_bf16x32(p.dyh + o, hi, c.row < HD);
+                gstore_bf16x32(p.dyl + o, v, c.row < HD);
+            }
+        }
+    };
+    const int l = p.l;
+    const int a0 = g * half_w;                                   // first A product of this group (index at level l + 1)
+    const int cntA = p.lv.dy_cnt[l + 1], cntB = p.lv.dy_cnt[l + 2], cntC = p.fuse >= 3 ? p.lv.dy_cnt[l + 3] : 0;
+    const bool hasA1 = a0 + 1 < cntA, hasB0 = (a0 >> 1) < cntB;
+    const bool more = p.fuse >= 3 && hasB0 && a0 + 2 < cntA;     // is there a second half of the tree?
+    const bool hasA3 = more && a0 + 3 < cntA, hasB1 = more && (a0 >> 1) + 1 < cntB, hasC = hasB1 && (a0 >> 2) < cntC;
+    // The operands of A_k (level-l pair 2k+1, 2k) are requested as soon as their slots are free, on a barrier of their
+    // own per parity of k: left factor into slots a, a + 1, right factor into b, b + 1.
+    uint64_t* lbar[2] = {&c.bars[0], c.bars + 4};
+    uint32_t lph[2] = {0, 0};
+    if (c.tid == 0) {
+        mbar_init(lbar[1], 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    // part 1 announces all four tiles and fetches the right factor, part 2 the left one (its slots free up later)
+    auto request_a1 = [&](int k, int b_) {
+        if (c.tid != 0) return;
+        mbar_expect_tx(lbar[k & 1], 4 * kT * HD * 2);
+        tma_tile(sm + b_ * kTileB, &tm.dyh, lbar[k & 1], HD, (int)(mat(l, 2 * (a0 + k)) * HD));
+        tma_tile(sm + (b_ + 1) * kTileB, &tm.dyl, lbar[k & 1], HD, (int)(mat(l, 2 * (a0 + k)) * HD));
+    };
+    auto request_a2 = [&](int k, int a) {
+        if (c.tid != 0) return;
+        tma_tile(sm + a * kTileB, &tm.dyh, lbar[k & 1], HD, (int)(mat(l, 2 * (a0 + k) + 1) * HD));
+        tma_tile(sm + (a + 1) * kTileB, &tm.dyl, lbar[k & 1], HD, (int)(mat(l, 2 * (a0 + k) + 1) * HD));
+    };
+    auto wait_a = [&](int k) {
+        if (!mbar_wait(lbar[k & 1], lph[k & 1], c.abort_flag, ST_LEVELS)) c.ok = false;
+        lph[k & 1] ^= 1;
+    };
+    request_a1(0, 2);
+    request_a2(0, 0);
+    if (hasA1) request_a1(1, 4);                                 // slots 4, 5 are free from the start
+    wait_a(0);
+    product(0, 0, 2);                                            // A_0
+    if (hasA1) request_a2(1, 2);                                 // slots 2, 3 are free again
+    readout(0, l + 1, a0, true, 0);                              // A_0 -> slots 0, 1
+    if (hasA1) {
+        wait_a(1);
+        product(0, 2, 4);                                        // A_1
+        readout(0, l + 1, a0 + 1, true, 2);                      // -> slots 2, 3
+    }
+    if (hasB0) {
+        product(more ? 128 : 0, 2, 0);                           // B_0 = A_1 A_0; it waits in columns 128.. if there is more
+        if (more) {                                              // every slot is free now
+            request_a1(2, 2);
+            request_a2(2, 0);
+        }
+        if (hasA3) request_a1(3, 4);
+        readout(more ? 128 : 0, l + 2, a0 >> 1, true, -1);
+        if (more) {
+            wait_a(2);
+            product(0, 0, 2);                                    // A_2
+            if (hasA3) request_a2(3, 2);
+            readout(0, l + 1, a0 + 2, true, 0);                  // -> slots 0, 1
+            if (hasA3) {
+                wait_a(3);
+                product(0, 2, 4);                                // A_3
+                readout(0, l + 1, a0 + 3, true, 2);              // -> slots 2, 3
+            }
+            if (hasB1) {
+                product(0, 2, 0);                                // B_1 = A_3 A_2
+                readout(0, l + 2, (a0 >> 1) + 1, true, 0);       // -> slots 0, 1 (A_2 has been read)
+                if (hasC) {
+                    readout(128, 0, 0, false, 4);                // B_0 from its columns -> slots 4, 5
+                    product(0, 0, 4);                            // C = B_1 B_0
+                    readout(0, l + 3, a0 >> 2, true, -1);
+                }
+            }
+        }
+    }
+    teardown<256>(c, p.status);
+}
+
 // ---------------------------------------------------------------------------------------------- version forward
 // grid = (S * N, 2): y = 0 queries, y = 1 keys; p.l = number of levels.  One CTA walks the whole chain of its chunk,
 // bottom level first:  Xv[l2] = Xv[l1] * Dy (queries) or Dy^T (keys).  The version just produced stays in shared
@@ -592,6 +721,11 @@ cudaError_t launch(K kern, dim3 grid, uint32_t slots, const LevelTensorMaps& tm,
 
 cudaError_t launch_level_kernel(int which, const LevelTensorMaps& tm, const LevelParams& p, int hd, cudaStream_t st) {
     switch (which) {
+        case LEVEL_DYADIC_FUSED: {
+            const int half_w = 1 << (p.fuse - 1);
+            dim3 g(p.S * ((p.lv.dy_cnt[p.l + 1] + half_w - 1) / half_w));
+            return hd == 64 ? launch(dyadic_fused_kernel<64>, g, 6, tm, p, st) : launch(dyadic_fused_kernel<128>, g, 6, tm, p, st);
+        }
         case LEVEL_DYADIC_FWD: {
             dim3 g(p.S * p.lv.dy_cnt[p.l + 1]);
             return hd == 64 ? launch(dyadic_fwd_kernel<64>, g, 4, tm, p, st) : launch(dyadic_fwd_kernel<128>, g, 4, tm, p, st);

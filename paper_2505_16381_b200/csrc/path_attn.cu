@@ -272,9 +272,12 @@ static int run_prep(const Plan& p, void* ws, const void* q, const void* k, const
     if (!make_level_maps(p, ws, tm)) { g_last_cuda_error = (int)cudaErrorUnknown; return PATH_ERR_LAUNCH; }
     LevelParams lp = level_params(p, ws);
     prof_mark(stg_lev, 0, st);
-    for (int l = 0; l + 1 <= p.nlev - 2; ++l) {   // run products of 2, 4, ... chunks
+    for (int l = 0; l + 1 <= p.nlev - 2;) {       // run products of 2, 4, ... chunks, up to three levels per launch
+        const int left = p.nlev - 2 - l;
         lp.l = l;
-        LAUNCH(launch_level_kernel(LEVEL_DYADIC_FWD, tm, lp, d, st));
+        lp.fuse = left >= 3 ? 3 : left;
+        LAUNCH(launch_level_kernel(lp.fuse >= 2 ? LEVEL_DYADIC_FUSED : LEVEL_DYADIC_FWD, tm, lp, d, st));
+        l += lp.fuse;
     }
     lp.l = p.nlev;                                // query and key versions: one CTA per chunk walks its chain
     LAUNCH(launch_level_kernel(LEVEL_VERSION_FWD, tm, lp, d, st));
