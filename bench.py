@@ -48,7 +48,7 @@ UNIT = "TFLOP/s"
 # (16 slices) summarised under profiles/; slices are independent, so a launch over S slices moves S times this.
 NCU_TRAFFIC_BYTES_PER_SLICE = {
     "chunk_prep": 12.64e6,         # backward instance (the step's forward runs on the shared workspace)
-    "levels_fwd": 3.68e6 + 6.37e6,   # dyadic_fwd (3 launches) + version_fwd
+    "levels_fwd": 3.68e6 + 6.37e6,   # dyadic_fwd (3 launches, before they became one) + version_fwd
     "fa_fwd": 11.19e6,
     "fa_bwd_dkv": 15.22e6,
     "fa_bwd_dq": 8.58e6,
@@ -127,8 +127,15 @@ def level_bytes(S, N, d):
     chains_k = nk and sum(1 for c in range(N) if any(
         not (c >> l2) & 1 and (~c & ((1 << l2) - 1)) and (((c >> l2) + 1) << l2) <= N - 1 for l2 in range(1, nlev)))
     runs = lambda l: N >> l
-    dy_out = sum(runs(l) for l in range(1, max(nlev - 1, 1)))
-    fwd = S * (dy_out * 6 * m + (nq + nk) * (2 * m + t) + (chains_q + chains_k) * t)
+    # run products: a launch builds up to three levels; it reads the hi + lo pairs of its input level once and writes
+    # every product's pair (the levels in between stay in shared memory)
+    dy = 0
+    l = 0
+    while l + 1 <= nlev - 2:
+        fuse = min(3, nlev - 2 - l)
+        dy += 2 * runs(l + 1) * 2 * m + sum(runs(l + j) for j in range(1, fuse + 1)) * 2 * m
+        l += fuse
+    fwd = S * (dy + (nq + nk) * (2 * m + t) + (chains_q + chains_k) * t)
     top = max(nlev - 2, 0)
     run_cnt = sum(runs(l) for l in range(0, top + 1))
     parents = sum(runs(l) for l in range(0, top))
