@@ -47,13 +47,13 @@ UNIT = "TFLOP/s"
 # DRAM bytes per launch PER (batch, head) SLICE at the C3 shape (L=4096, d=128), from the ncu captures at batch 1
 # (16 slices) summarised under profiles/; slices are independent, so a launch over S slices moves S times this.
 NCU_TRAFFIC_BYTES_PER_SLICE = {
-    "chunk_prep": 12.64e6,         # backward instance (the step's forward runs on the shared workspace)
-    "levels_fwd": 3.68e6 + 6.37e6,   # dyadic_fwd (3 launches, before they became one) + version_fwd
-    "fa_fwd": 11.19e6,
-    "fa_bwd_dkv": 15.22e6,
-    "fa_bwd_dq": 8.58e6,
-    "bwd_levels": 12.65e6,         # level_bwd (4 launches)
-    "bwd_chunk_chain": 18.30e6,
+    "chunk_prep": 12.71e6,         # backward instance (the step's forward runs on the shared workspace)
+    "levels_fwd": 2.13e6 + 6.35e6,   # dyadic_fused (one launch for three levels) + version_fwd
+    "fa_fwd": 11.18e6,
+    "fa_bwd_dkv": 15.24e6,
+    "fa_bwd_dq": 8.62e6,
+    "bwd_levels": 12.64e6,         # level_bwd (4 launches)
+    "bwd_chunk_chain": 18.29e6,
 }
 
 # DRAM bytes per launch of frontend_bwd_kernel PER BATCH ROW at H=32, L=4096, d=64 with the gate, from the ncu capture at
